@@ -1,0 +1,192 @@
+/*
+ * sparsepr.h -- C ABI of the SparsePR attention library for NVIDIA B200 (sm_100a).
+ *
+ * One call replaces dense self-attention O = softmax(s Q K^T) V (Eq. 1 of the
+ * SparsePR paper) for every (batch, head) of a long token sequence by
+ *   plan   : Response-Coupled Partitioning (Section 4.1, Appendix B), group-major
+ *            permutations, probe selection (Algorithm A.1) and routing under a
+ *            query-key pair budget (Section 4.3);
+ *   attend : block-sparse attention with renormalised hard drop (Eq. 3), exact
+ *            probe rows, the weighted ridge fit restricted to the probe-residual
+ *            subspace (Eq. 8-9, Appendix A.3) and the corrected output (Eq. 10),
+ *            written back in the original token order.
+ *
+ * Conventions
+ *   - Every pointer argument is marked HOST or DEVICE.  Device pointers must be
+ *     valid on the CUDA device that is current when the call is made.
+ *   - Q, K, V, O are [B, H, N, d] tensors addressed through element strides for
+ *     B, H and N; the last dimension is contiguous.  Rows must start on a
+ *     16-byte boundary.  N_q = N_k = N and d_v = d.
+ *   - The library never allocates or frees device memory and keeps no global
+ *     state.  The caller owns all tensors and both workspaces.  A plan handle is a small
+ *     host object that points into the plan workspace; it is valid until the
+ *     workspace is released or sparsepr_plan_destroy is called.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*)
+ *     and is asynchronous, except the calls documented as synchronising.
+ *   - Errors are return codes.  Argument errors are detected before anything
+ *     is launched.  Conditions found on the device (non-finite input, a
+ *     breakdown of the Cholesky factorisation, a bounded wait that ran out)
+ *     are recorded in a device error word that sparsepr_plan_stats reports.
+ *     No call aborts, throws or traps.
+ */
+#ifndef SPARSEPR_H_
+#define SPARSEPR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPARSEPR_OK = 0,
+  SPARSEPR_ERR_INVALID_ARG = 1,
+  SPARSEPR_ERR_UNSUPPORTED = 2,
+  SPARSEPR_ERR_WORKSPACE = 3,   /* workspace too small or misaligned (256 B) */
+  SPARSEPR_ERR_CUDA = 4,
+  SPARSEPR_ERR_NUMERIC = 5,
+  SPARSEPR_ERR_TIMEOUT = 6
+} sparsepr_status_t;
+
+typedef enum { SPARSEPR_F32 = 0, SPARSEPR_BF16 = 1 } sparsepr_dtype_t;
+
+/* Problem shape: Q, K in R^{N x d}, V in R^{N x d_v} per (batch, head) -- the
+ * paper's problem statement (Section 3).  Strides are in elements. */
+typedef struct {
+  int32_t B, H, N, d, dv;
+  int32_t dtype;                       /* sparsepr_dtype_t of Q, K, V and O */
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* B, H, N */
+} sparsepr_shape_t;
+
+/* Method parameters (Appendix C, Table C.1, plus the knobs the paper leaves
+ * open).  A zero in a field with a stated default selects the default. */
+typedef struct {
+  float density;         /* target rho_exec, probes included (Section 4.3); >= 1 selects every cell */
+  int32_t block;         /* nominal group size: C_k = C_q = ceil(N / block) unless given below */
+  int32_t Ck, Cq;        /* number of K/V groups and of query groups; 0 = derive from block */
+  int32_t n_sample;      /* M_s sampled query rows for the key-response metric (Appendix B.1) */
+  int32_t n_probe;       /* M exact probe rows per head (Appendix A.2) */
+  int32_t rK, rQ;        /* feature ranks, defaults 48 and 64, clamped to d */
+  int32_t r_out;         /* probe-residual output rank r, default 16, clamped to min(M, d_v) */
+  float lambda;          /* ridge coefficient (Eq. 8); negative selects the default 0.1, 0 is honoured */
+  float eps_rms;         /* stabiliser of the RMS normalisation (Eq. 7), default 1e-6 */
+  float eps_std;         /* epsilon inside the feature scale s_x (Appendix A.3), default 1e-6 */
+  int32_t kmeans_iters;  /* Lloyd iterations T (assignments), default 8 */
+  float softmax_scale;   /* s; 0 selects 1/sqrt(d) */
+  uint64_t seed;         /* offsets the deterministic row samples */
+  int32_t mode;          /* 0 = probe-fitted reconstruction, 1 = renormalised hard drop only */
+} sparsepr_params_t;
+
+typedef struct sparsepr_plan_s sparsepr_plan_t;
+
+/* Densities and group statistics of a plan, aggregated over all heads
+ * (Eq. 2 and Section 4.3).  `device_error` is 0 or the sparsepr_status_t that
+ * a kernel recorded. */
+typedef struct {
+  int64_t routed_pairs;        /* sum over heads of sum_ab z_ab |G_a||G_b| */
+  int64_t routed_cells;        /* number of selected cells */
+  int64_t padded_tile_pairs;   /* pairs the block-sparse kernel issues, padding included */
+  double rho_route, rho_exec;  /* mean over heads */
+  double rho_route_min, rho_route_max;
+  int32_t nonempty_kv_groups_min, nonempty_q_groups_min;
+  int32_t max_kv_group, max_q_group;
+  int32_t assign_rechecked_rows;   /* rows of the last k-means assignments decided by the exact recheck */
+  int32_t device_error;
+} sparsepr_stats_t;
+
+/* Host-side view of a plan, one entry per (batch, head) in b-major order, used
+ * to export a plan for inspection and to import one made elsewhere.  Every
+ * pointer is HOST memory owned by the caller; NULL skips the field on export.
+ *   kv_assign, q_assign : [BH, N]   group id of every token (Section 3)
+ *   kv_perm, q_perm     : [BH, N]   original index of the token at each group-major position
+ *   kv_off, q_off       : [BH, C+1] ragged group offsets
+ *   route_ptr           : [BH, Cq+1]; route_idx : [BH, Cq*Ck] slab per head, rows ascending in b
+ *   probe_idx, probe_w  : [BH, M]   probe rows in selection order and coverage weights w_p
+ *   routed_pairs        : [BH]
+ */
+typedef struct {
+  int32_t *kv_assign, *q_assign;
+  int32_t *kv_perm, *q_perm;
+  int32_t *kv_off, *q_off;
+  int32_t *route_ptr, *route_idx;
+  int32_t *probe_idx;
+  float *probe_w;
+  int64_t *routed_pairs;
+} sparsepr_plan_host_t;
+
+const char* sparsepr_status_string(sparsepr_status_t s);
+
+/* Bytes of DEVICE workspace that sparsepr_plan / sparsepr_plan_import and
+ * sparsepr_attend need for this shape and these parameters.  0 on invalid input. */
+size_t sparsepr_plan_workspace_bytes(const sparsepr_shape_t* shape, const sparsepr_params_t* params);
+size_t sparsepr_attend_workspace_bytes(const sparsepr_shape_t* shape, const sparsepr_params_t* params);
+
+/* Stages 1-2 (Sections 4.1 and 4.3, Algorithm A.1): builds partition, permutations,
+ * probe set and routes of every head from Q and K (DEVICE, read only; V is not
+ * read -- values never enter the partition features -- and may be NULL).
+ * `workspace` is DEVICE memory of at least sparsepr_plan_workspace_bytes, 256-byte
+ * aligned; the plan lives in it.  *out receives a HOST handle. */
+sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                const void* Q, const void* K, const void* V,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                sparsepr_plan_t** out);
+
+/* Stages 3-4 (Eq. 3, Eq. 8-10): O (DEVICE, written in original token order) from
+ * Q, K, V (DEVICE) and a plan.  `workspace`: DEVICE, sparsepr_attend_workspace_bytes,
+ * 256-byte aligned; its contents are scratch.  `O_sparse` (DEVICE, float32
+ * [B,H,N,dv] contiguous, may be NULL) additionally receives the uncorrected
+ * hard-drop output O^sp in original order, for error reporting. */
+sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* plan, const void* Q, const void* K, const void* V,
+                                  void* O, float* O_sparse, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+
+/* Dense attention, Eq. 1, with the same kernels run over the full key range.
+ * Needs no workspace.  softmax_scale 0 selects 1/sqrt(d). */
+sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_scale,
+                                 const void* Q, const void* K, const void* V, void* O, void* cuda_stream);
+
+/* Synchronises the stream the plan was built on, then fills *host_out. */
+sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* plan, sparsepr_stats_t* host_out);
+sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* plan, sparsepr_plan_host_t* host_out);
+
+/* Builds a plan from host-side assignments, routes (CSR slabs as in
+ * sparsepr_plan_host_t) and probes; permutations and offsets are recomputed on
+ * the device.  Used to run stages 3-4 on a partition produced elsewhere. */
+sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                       const sparsepr_plan_host_t* host_in,
+                                       void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                       sparsepr_plan_t** out);
+
+/* Frees the HOST handle only. */
+void sparsepr_plan_destroy(sparsepr_plan_t* plan);
+
+/* ---- single stages, exposed so that the integer work can be checked bit for bit ---- */
+
+/* a[j] = argmin_c sum_k (X[j,k]-mu[c,k])^2 with ties to the lowest c: the
+ * assignment step of k-means (Section 4.1).  X [n,r], mu [C,r] float32 DEVICE,
+ * a [n] int32 DEVICE.  The decision equals the one taken in float64 with the
+ * terms accumulated in order of k.  `ws`: DEVICE scratch of at least
+ * sparsepr_stage_assign_workspace_bytes(n, C, r). */
+size_t sparsepr_stage_assign_workspace_bytes(int32_t n, int32_t C, int32_t r);
+sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const float* X, const float* mu,
+                                        int32_t* a, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Stable counting sort by group id (Section 4.3, group-major layout):
+ * perm [n], inv [n], off [C+1], all int32 DEVICE. */
+sparsepr_status_t sparsepr_stage_permute(int32_t n, int32_t C, const int32_t* a,
+                                         int32_t* perm, int32_t* inv, int32_t* off, void* cuda_stream);
+
+/* Cell selection under a pair budget (Section 4.3) for one head from given
+ * float32 cell scores [Cq,Ck], group sizes nq [Cq], nk [Ck] (int32) -- all DEVICE.
+ * Writes route_ptr [Cq+1], route_idx [Cq*Ck] (ascending inside a row) and
+ * *pairs_out (int64), all DEVICE.  select_all != 0 takes every non-empty cell. */
+sparsepr_status_t sparsepr_stage_route(int32_t Cq, int32_t Ck, const float* score,
+                                       const int32_t* nq, const int32_t* nk, int64_t pair_budget,
+                                       int32_t select_all, int32_t* route_ptr, int32_t* route_idx,
+                                       int64_t* pairs_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SPARSEPR_H_ */

@@ -1,0 +1,321 @@
+"""Thin ctypes binding of libsparsepr.so (the C ABI declared in include/sparsepr.h).
+
+Only argument marshalling happens here: PyTorch supplies device memory and the
+current CUDA stream, every step of the computation runs inside the library.
+There is no fallback: if the library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparsepr.so")
+_lib = None
+
+OK = 0
+F32, BF16 = 0, 1
+STATUS = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_UNSUPPORTED", 3: "ERR_WORKSPACE", 4: "ERR_CUDA",
+          5: "ERR_NUMERIC", 6: "ERR_TIMEOUT"}
+
+
+class SparsePRError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s failed: %s (%s)" % (where, STATUS.get(code, code), status_string(code)))
+
+
+class Shape(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("N", C.c_int32), ("d", C.c_int32), ("dv", C.c_int32),
+                ("dtype", C.c_int32), ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+                ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3)]
+
+
+class Params(C.Structure):
+    _fields_ = [("density", C.c_float), ("block", C.c_int32), ("Ck", C.c_int32), ("Cq", C.c_int32),
+                ("n_sample", C.c_int32), ("n_probe", C.c_int32), ("rK", C.c_int32), ("rQ", C.c_int32),
+                ("r_out", C.c_int32), ("lam", C.c_float), ("eps_rms", C.c_float), ("eps_std", C.c_float),
+                ("kmeans_iters", C.c_int32), ("softmax_scale", C.c_float), ("seed", C.c_uint64), ("mode", C.c_int32)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("routed_pairs", C.c_int64), ("routed_cells", C.c_int64), ("padded_tile_pairs", C.c_int64),
+                ("rho_route", C.c_double), ("rho_exec", C.c_double), ("rho_route_min", C.c_double),
+                ("rho_route_max", C.c_double), ("nonempty_kv_groups_min", C.c_int32),
+                ("nonempty_q_groups_min", C.c_int32), ("max_kv_group", C.c_int32), ("max_q_group", C.c_int32),
+                ("assign_rechecked_rows", C.c_int32), ("device_error", C.c_int32)]
+
+
+class PlanHost(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("kv_assign", "q_assign", "kv_perm", "q_perm", "kv_off", "q_off",
+                                            "route_ptr", "route_idx", "probe_idx", "probe_w", "routed_pairs")]
+
+
+EXPORTS = ["sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
+           "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
+           "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
+           "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
+
+
+def lib():
+    """Loads the CUDA library on first use; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libsparsepr.so is missing: run `python -m paper_2608_18484_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, sz, i32, i64 = C.c_void_p, C.c_size_t, C.c_int32, C.c_int64
+        L.sparsepr_status_string.restype = C.c_char_p
+        L.sparsepr_status_string.argtypes = [C.c_int]
+        for f in (L.sparsepr_plan_workspace_bytes, L.sparsepr_attend_workspace_bytes):
+            f.restype = sz
+            f.argtypes = [C.POINTER(Shape), C.POINTER(Params)]
+        L.sparsepr_plan.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, sz, vp, C.POINTER(vp)]
+        L.sparsepr_attend.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.sparsepr_dense.argtypes = [C.POINTER(Shape), C.c_float, vp, vp, vp, vp, vp]
+        L.sparsepr_plan_stats.argtypes = [vp, C.POINTER(Stats)]
+        L.sparsepr_plan_export.argtypes = [vp, C.POINTER(PlanHost)]
+        L.sparsepr_plan_import.argtypes = [C.POINTER(Shape), C.POINTER(Params), C.POINTER(PlanHost), vp, sz, vp,
+                                           C.POINTER(vp)]
+        L.sparsepr_plan_destroy.argtypes = [vp]
+        L.sparsepr_plan_destroy.restype = None
+        L.sparsepr_stage_assign_workspace_bytes.restype = sz
+        L.sparsepr_stage_assign_workspace_bytes.argtypes = [i32, i32, i32]
+        L.sparsepr_stage_assign.argtypes = [i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.sparsepr_stage_permute.argtypes = [i32, i32, vp, vp, vp, vp, vp]
+        L.sparsepr_stage_route.argtypes = [i32, i32, vp, vp, vp, i64, i32, vp, vp, vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().sparsepr_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != OK:
+        raise SparsePRError(code, where)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("Q, K, V must be float32 or bfloat16")
+
+
+def make_shape(Q, K, V, O) -> Shape:
+    for t in (Q, K, V, O):
+        if t.dim() != 4 or not t.is_cuda or t.stride(3) != 1:
+            raise ValueError("expected CUDA tensors [B, H, N, d] with a contiguous last dimension")
+    B, H, N, d = Q.shape
+    s = Shape(B=B, H=H, N=N, d=d, dv=V.shape[3], dtype=_dtype_code(Q))
+    for name, t in (("q_stride", Q), ("k_stride", K), ("v_stride", V), ("o_stride", O)):
+        getattr(s, name)[:] = [t.stride(0), t.stride(1), t.stride(2)]
+    return s
+
+
+def make_params(density=0.25, block=128, Ck=0, Cq=0, n_sample=256, n_probe=128, rK=48, rQ=64, r_out=16, lam=0.1,
+                eps_rms=1e-6, eps_std=1e-6, kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0) -> Params:
+    return Params(density=density, block=block, Ck=Ck, Cq=Cq, n_sample=n_sample, n_probe=n_probe, rK=rK, rQ=rQ,
+                  r_out=r_out, lam=lam, eps_rms=eps_rms, eps_std=eps_std, kmeans_iters=kmeans_iters,
+                  softmax_scale=softmax_scale, seed=seed, mode=mode)
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+class Plan:
+    """Owns the host handle and the device workspace a plan lives in."""
+
+    def __init__(self, handle, workspace, shape: Shape, params: Params, attend_bytes: int):
+        self.handle, self.workspace, self.shape, self.params = handle, workspace, shape, params
+        self.attend_bytes = attend_bytes
+        self.attend_workspace = None
+
+    @property
+    def BH(self):
+        return self.shape.B * self.shape.H
+
+    @property
+    def groups(self):
+        blk = self.params.block or 128
+        n = -(-self.shape.N // blk)
+        return (self.params.Ck or n, self.params.Cq or n)
+
+    @property
+    def M(self):
+        return 0 if self.params.mode == 1 else min(self.params.n_probe, self.shape.N)
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.sparsepr_plan_destroy(self.handle)
+            self.handle = None
+
+
+def sparsepr_plan(Q, K, V=None, params: Params | None = None, **kw) -> Plan:
+    """Stages 1-2: partition, permutations, probe set and routes for every head."""
+    params = params or make_params(**kw)
+    shape = make_shape(Q, K, K if V is None else V, Q)
+    L = lib()
+    nbytes = L.sparsepr_plan_workspace_bytes(C.byref(shape), C.byref(params))
+    if nbytes == 0:
+        raise SparsePRError(1, "sparsepr_plan_workspace_bytes")
+    ws = _workspace(nbytes, Q.device)
+    handle = C.c_void_p()
+    _check(L.sparsepr_plan(C.byref(shape), C.byref(params), Q.data_ptr(), K.data_ptr(),
+                           None if V is None else V.data_ptr(), ws.data_ptr(), ws.numel(), _stream(),
+                           C.byref(handle)), "sparsepr_plan")
+    return Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+def sparsepr_attend(plan: Plan, Q, K, V, out=None, return_sparse=False):
+    """Stages 3-4: block-sparse attention, probe rows, fit and corrected output."""
+    O = torch.empty_like(Q) if out is None else out
+    shape = make_shape(Q, K, V, O)
+    for f in ("q_stride", "k_stride", "v_stride", "o_stride"):
+        if list(getattr(shape, f)) != list(getattr(plan.shape, f)):
+            raise ValueError("tensor strides differ from the ones the plan was built for")
+    if plan.attend_workspace is None:
+        plan.attend_workspace = _workspace(plan.attend_bytes, Q.device)
+    ws = plan.attend_workspace
+    Osp = torch.empty(Q.shape, dtype=torch.float32, device=Q.device) if return_sparse else None
+    _check(lib().sparsepr_attend(plan.handle, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
+                                 None if Osp is None else Osp.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "sparsepr_attend")
+    return (O, Osp) if return_sparse else O
+
+
+def sparsepr_dense(Q, K, V, softmax_scale=0.0, out=None):
+    """Dense attention, Eq. 1, by the same build's kernels."""
+    O = torch.empty_like(Q) if out is None else out
+    shape = make_shape(Q, K, V, O)
+    _check(lib().sparsepr_dense(C.byref(shape), float(softmax_scale), Q.data_ptr(), K.data_ptr(), V.data_ptr(),
+                                O.data_ptr(), _stream()), "sparsepr_dense")
+    return O
+
+
+def sparsepr_plan_stats(plan: Plan) -> dict:
+    st = Stats()
+    _check(lib().sparsepr_plan_stats(plan.handle, C.byref(st)), "sparsepr_plan_stats")
+    return {n: getattr(st, n) for n, _ in Stats._fields_}
+
+
+def _host_arrays(plan: Plan) -> dict:
+    BH, N = plan.BH, plan.shape.N
+    Ck, Cq = plan.groups
+    M = max(plan.M, 1)
+    return dict(kv_assign=np.empty((BH, N), np.int32), q_assign=np.empty((BH, N), np.int32),
+                kv_perm=np.empty((BH, N), np.int32), q_perm=np.empty((BH, N), np.int32),
+                kv_off=np.empty((BH, Ck + 1), np.int32), q_off=np.empty((BH, Cq + 1), np.int32),
+                route_ptr=np.empty((BH, Cq + 1), np.int32), route_idx=np.empty((BH, Cq * Ck), np.int32),
+                probe_idx=np.empty((BH, M), np.int32), probe_w=np.empty((BH, M), np.float32),
+                routed_pairs=np.empty((BH,), np.int64))
+
+
+def sparsepr_plan_export(plan: Plan) -> dict:
+    """Copies the plan to host numpy arrays (synchronises)."""
+    arrs = _host_arrays(plan)
+    ph = PlanHost(**{k: v.ctypes.data for k, v in arrs.items()})
+    _check(lib().sparsepr_plan_export(plan.handle, C.byref(ph)), "sparsepr_plan_export")
+    if plan.M == 0:
+        arrs["probe_idx"] = arrs["probe_idx"][:, :0]
+        arrs["probe_w"] = arrs["probe_w"][:, :0]
+    return arrs
+
+
+def sparsepr_plan_import(Q, K, V, host: dict, params: Params | None = None, **kw) -> Plan:
+    """Builds a device plan from host assignments, routes and probes.
+
+    host: kv_assign/q_assign [BH,N]; route_ptr [BH,Cq+1]; route_idx [BH,Cq*Ck] slab
+    (or a list of per-head index arrays); probe_idx/probe_w [BH,M]."""
+    params = params or make_params(**kw)
+    shape = make_shape(Q, K, V, Q)
+    L = lib()
+    BH, N = shape.B * shape.H, shape.N
+    blk = params.block or 128
+    Ck, Cq = params.Ck or -(-N // blk), params.Cq or -(-N // blk)
+    a = {k: np.ascontiguousarray(host[k], dtype=np.int32) for k in ("kv_assign", "q_assign", "route_ptr")}
+    ridx = host["route_idx"]
+    if isinstance(ridx, (list, tuple)):
+        slab = np.zeros((BH, Cq * Ck), np.int32)
+        for i, r in enumerate(ridx):
+            slab[i, :len(r)] = r
+        ridx = slab
+    a["route_idx"] = np.ascontiguousarray(ridx, dtype=np.int32)
+    assert a["route_idx"].shape == (BH, Cq * Ck) and a["kv_assign"].shape == (BH, N)
+    M = 0 if params.mode == 1 else min(params.n_probe, N)
+    if M:
+        a["probe_idx"] = np.ascontiguousarray(host["probe_idx"], dtype=np.int32)
+        a["probe_w"] = np.ascontiguousarray(host["probe_w"], dtype=np.float32)
+        assert a["probe_idx"].shape == (BH, M)
+    ph = PlanHost(**{k: v.ctypes.data for k, v in a.items()})
+    ws = _workspace(L.sparsepr_plan_workspace_bytes(C.byref(shape), C.byref(params)), Q.device)
+    handle = C.c_void_p()
+    _check(L.sparsepr_plan_import(C.byref(shape), C.byref(params), C.byref(ph), ws.data_ptr(), ws.numel(),
+                                  _stream(), C.byref(handle)), "sparsepr_plan_import")
+    return Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+# ---- single stages -------------------------------------------------------------------
+def sparsepr_stage_assign(X: torch.Tensor, mu: torch.Tensor) -> torch.Tensor:
+    X, mu = X.contiguous().float(), mu.contiguous().float()
+    n, r = X.shape
+    Cn = mu.shape[0]
+    L = lib()
+    ws = _workspace(L.sparsepr_stage_assign_workspace_bytes(n, Cn, r), X.device)
+    a = torch.empty(n, dtype=torch.int32, device=X.device)
+    _check(L.sparsepr_stage_assign(n, Cn, r, X.data_ptr(), mu.data_ptr(), a.data_ptr(), ws.data_ptr(), ws.numel(),
+                                   _stream()), "sparsepr_stage_assign")
+    return a
+
+
+def sparsepr_stage_permute(a: torch.Tensor, Cn: int):
+    a = a.contiguous().to(torch.int32)
+    n = a.numel()
+    perm, inv = torch.empty_like(a), torch.empty_like(a)
+    off = torch.empty(Cn + 1, dtype=torch.int32, device=a.device)
+    _check(lib().sparsepr_stage_permute(n, Cn, a.data_ptr(), perm.data_ptr(), inv.data_ptr(), off.data_ptr(),
+                                        _stream()), "sparsepr_stage_permute")
+    return perm, inv, off
+
+
+def sparsepr_stage_route(score: torch.Tensor, nq: torch.Tensor, nk: torch.Tensor, budget: int, select_all=False):
+    score = score.contiguous().float()
+    Cq, Ck = score.shape
+    nq, nk = nq.contiguous().to(torch.int32), nk.contiguous().to(torch.int32)
+    ptr = torch.empty(Cq + 1, dtype=torch.int32, device=score.device)
+    idx = torch.zeros(Cq * Ck, dtype=torch.int32, device=score.device)
+    pairs = torch.zeros(1, dtype=torch.int64, device=score.device)
+    _check(lib().sparsepr_stage_route(Cq, Ck, score.data_ptr(), nq.data_ptr(), nk.data_ptr(), int(budget),
+                                      int(bool(select_all)), ptr.data_ptr(), idx.data_ptr(), pairs.data_ptr(),
+                                      _stream()), "sparsepr_stage_route")
+    return ptr, idx, pairs
+
+
+# ---- whole call on host buffers ----------------------------------------------------------
+def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, dev_buffers=None):
+    """One full call for a user whose tensors live in (pinned) host memory:
+    host->device copies, plan, attend, device->host copy of O.  Returns O on host."""
+    dev = torch.device("cuda")
+    if dev_buffers is None:
+        dev_buffers = [torch.empty(t.shape, dtype=t.dtype, device=dev) for t in (Qh, Kh, Vh)]
+    Qd, Kd, Vd = dev_buffers
+    Qd.copy_(Qh, non_blocking=True)
+    Kd.copy_(Kh, non_blocking=True)
+    Vd.copy_(Vh, non_blocking=True)
+    plan = sparsepr_plan(Qd, Kd, Vd, params=params)
+    O = sparsepr_attend(plan, Qd, Kd, Vd)
+    Oh.copy_(O, non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    return Oh

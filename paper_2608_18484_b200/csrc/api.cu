@@ -1,0 +1,526 @@
+// C-ABI layer: argument validation, workspace carving, launch order.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+#include "kernels.cuh"
+
+using namespace spr;
+
+namespace {
+
+struct Carver {                       // bump allocator over a caller-owned workspace (or a dry run)
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+  template <typename T> T* take(size_t n) {
+    off = (off + 255) & ~size_t(255);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+  size_t bytes() const { return (off + 255) & ~size_t(255); }
+};
+
+struct Resolved {
+  int B, H, BH, N, d, dtype, es;
+  int Ck, Cq, Cmax, Ms, M, rK, rQ, RK, RQ, Rmax, r_out, T, mode;
+  float density, lambda, eps_rms, eps_std, scale;
+  u64 seed;
+  i64 qs[3], ks[3], vs[3], os[3];
+};
+
+int round16(int r) { return r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64; }
+
+sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p, Resolved* r) {
+  if (!s || !r) return SPARSEPR_ERR_INVALID_ARG;
+  if (s->B < 1 || s->H < 1 || s->N < 1) return SPARSEPR_ERR_INVALID_ARG;
+  if (s->dtype != SPARSEPR_F32 && s->dtype != SPARSEPR_BF16) return SPARSEPR_ERR_INVALID_ARG;
+  if ((s->d != 64 && s->d != 128) || s->dv != s->d) return SPARSEPR_ERR_UNSUPPORTED;
+  r->B = s->B; r->H = s->H; r->BH = s->B * s->H; r->N = s->N; r->d = s->d; r->dtype = s->dtype;
+  r->es = s->dtype == SPARSEPR_BF16 ? 2 : 4;
+  const int vec = 16 / r->es;
+  for (int i = 0; i < 3; ++i) {
+    r->qs[i] = s->q_stride[i]; r->ks[i] = s->k_stride[i]; r->vs[i] = s->v_stride[i]; r->os[i] = s->o_stride[i];
+    if (r->qs[i] < 0 || r->ks[i] < 0 || r->vs[i] < 0 || r->os[i] < 0) return SPARSEPR_ERR_INVALID_ARG;
+    if (r->qs[i] % vec || r->ks[i] % vec || r->vs[i] % vec || r->os[i] % vec) return SPARSEPR_ERR_UNSUPPORTED;
+  }
+  if (r->qs[2] < s->d || r->ks[2] < s->d || r->vs[2] < s->d || r->os[2] < s->d) return SPARSEPR_ERR_INVALID_ARG;
+  if (!p) return SPARSEPR_OK;
+  if (!(p->density > 0.f) || p->block < 0 || p->Ck < 0 || p->Cq < 0 || p->n_sample < 0 || p->n_probe < 0 ||
+      p->rK < 0 || p->rQ < 0 || p->r_out < 0 || p->kmeans_iters < 0 || p->mode < 0 || p->mode > 1 ||
+      !(p->softmax_scale >= 0.f) || !(p->eps_rms >= 0.f) || !(p->eps_std >= 0.f) || std::isnan(p->lambda))
+    return SPARSEPR_ERR_INVALID_ARG;
+  const int block = p->block ? p->block : 128;
+  r->Ck = p->Ck ? p->Ck : (s->N + block - 1) / block;
+  r->Cq = p->Cq ? p->Cq : (s->N + block - 1) / block;
+  if (r->Ck > s->N || r->Cq > s->N) return SPARSEPR_ERR_INVALID_ARG;
+  if (r->Ck > kMaxGroups || r->Cq > kMaxGroups) return SPARSEPR_ERR_UNSUPPORTED;
+  r->Cmax = r->Ck > r->Cq ? r->Ck : r->Cq;
+  r->Ms = std::min(p->n_sample ? p->n_sample : 256, s->N);
+  r->mode = p->mode;
+  r->M = r->mode == 1 ? 0 : std::min(p->n_probe, s->N);
+  if (r->M > kMaxProbes) return SPARSEPR_ERR_UNSUPPORTED;
+  r->rK = std::min(p->rK ? p->rK : 48, s->d);
+  r->rQ = std::min(p->rQ ? p->rQ : 64, s->d);
+  if (r->rK > kMaxRank || r->rQ > kMaxRank) return SPARSEPR_ERR_UNSUPPORTED;
+  r->RK = round16(r->rK); r->RQ = round16(r->rQ); r->Rmax = std::max(r->RK, r->RQ);
+  r->r_out = std::max(1, std::min(p->r_out ? p->r_out : 16, std::min(std::max(r->M, 1), s->d)));
+  r->T = p->kmeans_iters ? p->kmeans_iters : 8;
+  r->density = p->density;
+  r->lambda = p->lambda < 0.f ? 0.1f : p->lambda;
+  r->eps_rms = p->eps_rms > 0.f ? p->eps_rms : 1e-6f;
+  r->eps_std = p->eps_std > 0.f ? p->eps_std : 1e-6f;
+  r->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / std::sqrt((float)s->d);
+  r->seed = p->seed;
+  return SPARSEPR_OK;
+}
+
+std::once_flag g_init_once;
+cudaError_t g_init_err = cudaSuccess;
+cudaError_t ensure_init() {
+  std::call_once(g_init_once, [] {
+    cudaError_t e;
+    if ((e = init_jacobi()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_group_sort()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_routing()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
+  });
+  return g_init_err;
+}
+
+bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
+
+}  // namespace
+
+struct sparsepr_plan_s {
+  Resolved r;
+  cudaStream_t stream;
+  // device state (all inside the caller's plan workspace)
+  int* err; int* recheck;
+  double* Mmat; double* lam;
+  float *FK, *FQ, *phi;
+  unsigned* maxabs; int* fx_shift;
+  float *mu, *mu2, *mumax; i64* sums; int* counts;
+  int *a_K, *a_Q, *kv_perm, *kv_inv, *q_perm, *q_inv, *kv_off, *q_off, *nk, *nq;
+  float *kappa, *theta, *score;
+  int *route_ptr, *route_idx, *tile_off;
+  RouteState* rstate;
+  double* probe_dist; int* probe_idx; float* probe_w;
+};
+
+namespace {
+
+void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
+  const size_t BH = r.BH, N = r.N, d = r.d;
+  int* err = c.take<int>(64);
+  int* recheck = err ? err + 1 : nullptr;
+  double* Mmat = c.take<double>(BH * d * d);
+  double* lam = c.take<double>(BH * d);
+  float* FK = c.take<float>(BH * d * r.rK);
+  float* FQ = c.take<float>(BH * d * r.rQ);
+  float* phi = c.take<float>(BH * N * r.Rmax);
+  unsigned* maxabs = c.take<unsigned>(BH);
+  int* fx = c.take<int>(BH);
+  float* mu = c.take<float>(BH * r.Cmax * r.Rmax);
+  float* mu2 = c.take<float>(BH * r.Cmax);
+  float* mumax = c.take<float>(BH);
+  i64* sums = c.take<i64>(BH * r.Cmax * r.Rmax);
+  int* counts = c.take<int>(BH * r.Cmax);
+  int* aK = c.take<int>(BH * N); int* aQ = c.take<int>(BH * N);
+  int* kvp = c.take<int>(BH * N); int* kvi = c.take<int>(BH * N);
+  int* qp = c.take<int>(BH * N); int* qi = c.take<int>(BH * N);
+  int* kvo = c.take<int>(BH * (r.Ck + 1)); int* qo = c.take<int>(BH * (r.Cq + 1));
+  int* nk = c.take<int>(BH * r.Ck); int* nq = c.take<int>(BH * r.Cq);
+  float* kappa = c.take<float>(BH * r.Ck * d); float* theta = c.take<float>(BH * r.Cq * d);
+  float* score = c.take<float>(BH * (size_t)r.Cq * r.Ck);
+  int* rptr = c.take<int>(BH * (r.Cq + 1)); int* ridx = c.take<int>(BH * (size_t)r.Cq * r.Ck);
+  int* toff = c.take<int>(BH * (r.Cq + 1));
+  RouteState* rs = c.take<RouteState>(BH);
+  double* pd = c.take<double>(BH * N);
+  int* pidx = c.take<int>(BH * std::max(r.M, 1)); float* pw = c.take<float>(BH * std::max(r.M, 1));
+  if (p) {
+    p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
+    p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
+    p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
+    p->nk = nk; p->nq = nq; p->kappa = kappa; p->theta = theta; p->score = score; p->route_ptr = rptr; p->route_idx = ridx;
+    p->tile_off = toff; p->rstate = rs; p->probe_dist = pd; p->probe_idx = pidx; p->probe_w = pw;
+  }
+}
+
+struct AttendWs {
+  void *Qg, *Kg, *Vg;
+  float *partial, *X, *Dn, *A, *c, *Psi;
+  double* fit;
+  int n_split;
+};
+
+int probe_splits(const Resolved& r) {
+  if (r.M == 0) return 1;
+  const int row_tiles = (r.M + 63) / 64;
+  int s = (2 * 148 + r.BH * row_tiles - 1) / (r.BH * row_tiles);
+  const int key_tiles = (r.N + 63) / 64;
+  s = std::max(1, std::min(s, std::max(1, key_tiles / 4)));
+  return s;
+}
+
+void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
+  const size_t BH = r.BH, N = r.N, d = r.d;
+  const int ns = probe_splits(r);
+  void* Qg = c.take<char>(BH * N * d * r.es);
+  void* Kg = c.take<char>(BH * N * d * r.es);
+  void* Vg = c.take<char>(BH * N * d * r.es);
+  const size_t M1 = std::max(r.M, 1);
+  float* partial = c.take<float>(probe_partial_floats(r.BH, ns, (int)M1, r.d));
+  float* X = c.take<float>(BH * M1 * d); float* Dn = c.take<float>(BH * M1 * d);
+  float* A = c.take<float>(BH * d * d); float* cc = c.take<float>(BH * d);
+  float* Psi = c.take<float>(BH * d * d);
+  double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
+  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->fit = fit; w->n_split = ns; }
+}
+
+i64 pair_budget(const Resolved& r) {
+  const i64 total = (i64)std::floor((double)r.density * (double)r.N * (double)r.N);
+  return std::max<i64>(total - (i64)r.M * r.N, 0);
+}
+
+void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cudaStream_t st) {
+  const Resolved& R = p->r;
+  const int ld = round16(r);
+  launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
+  launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st);
+  for (int t = 1; t <= R.T; ++t) {
+    const bool upd = t < R.T;
+    if (!upd) cudaMemsetAsync(p->recheck, 0, sizeof(int), st);
+    launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
+                         upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
+    if (upd) launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st);
+  }
+}
+
+// pads [n][r] rows to [n][R] with zeros
+__global__ void k_pad_rows(const float* __restrict__ in, int n, int r, int R, float* __restrict__ out) {
+  for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < (i64)n * R; e += (i64)gridDim.x * blockDim.x) {
+    const int k = (int)(e % R);
+    out[e] = k < r ? in[(e / R) * r + k] : 0.f;
+  }
+}
+__global__ void k_sizes_from_off(const int* __restrict__ off, int C, int* __restrict__ sizes) {
+  const int bh = blockIdx.y;
+  for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < C; g += gridDim.x * blockDim.x)
+    sizes[(i64)bh * C + g] = off[(i64)bh * (C + 1) + g + 1] - off[(i64)bh * (C + 1) + g];
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sparsepr_status_string(sparsepr_status_t s) {
+  switch (s) {
+    case SPARSEPR_OK: return "ok";
+    case SPARSEPR_ERR_INVALID_ARG: return "invalid argument";
+    case SPARSEPR_ERR_UNSUPPORTED: return "unsupported shape or parameter";
+    case SPARSEPR_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case SPARSEPR_ERR_CUDA: return "CUDA error";
+    case SPARSEPR_ERR_NUMERIC: return "numerical breakdown or non-finite input";
+    case SPARSEPR_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+size_t sparsepr_plan_workspace_bytes(const sparsepr_shape_t* shape, const sparsepr_params_t* params) {
+  Resolved r;
+  if (!params || resolve(shape, params, &r) != SPARSEPR_OK) return 0;
+  Carver c(nullptr);
+  carve_plan(c, r, nullptr);
+  return c.bytes();
+}
+
+size_t sparsepr_attend_workspace_bytes(const sparsepr_shape_t* shape, const sparsepr_params_t* params) {
+  Resolved r;
+  if (!params || resolve(shape, params, &r) != SPARSEPR_OK) return 0;
+  Carver c(nullptr);
+  carve_attend(c, r, nullptr);
+  return c.bytes();
+}
+
+static sparsepr_status_t make_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream, sparsepr_plan_s** out) {
+  if (!params || !out) return SPARSEPR_ERR_INVALID_ARG;
+  Resolved r;
+  sparsepr_status_t s = resolve(shape, params, &r);
+  if (s != SPARSEPR_OK) return s;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SPARSEPR_ERR_WORKSPACE;
+  Carver dry(nullptr);
+  carve_plan(dry, r, nullptr);
+  if (workspace_bytes < dry.bytes()) return SPARSEPR_ERR_WORKSPACE;
+  if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  sparsepr_plan_s* p = new (std::nothrow) sparsepr_plan_s();
+  if (!p) return SPARSEPR_ERR_INVALID_ARG;
+  p->r = r;
+  p->stream = static_cast<cudaStream_t>(cuda_stream);
+  Carver c(workspace);
+  carve_plan(c, r, p);
+  *out = p;
+  return SPARSEPR_OK;
+}
+
+sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
+                                const void* K, const void* V, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream, sparsepr_plan_t** out) {
+  (void)V;
+  if (!Q || !K) return SPARSEPR_ERR_INVALID_ARG;
+  sparsepr_plan_s* p = nullptr;
+  sparsepr_status_t s = make_plan(shape, params, workspace, workspace_bytes, cuda_stream, &p);
+  if (s != SPARSEPR_OK) return s;
+  const Resolved& r = p->r;
+  cudaStream_t st = p->stream;
+  cudaGetLastError();
+  cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
+  cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
+  // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means
+  launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
+  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, p->FK, p->lam, st);
+  launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+  run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, st);
+  launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
+  launch_group_means(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
+  // query partition: centroid metric -> F_Q -> phi_Q -> k-means
+  launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
+  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, p->FQ, p->lam, st);
+  cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
+  launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+  run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, st);
+  launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
+  launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
+  // probes and routes
+  if (r.M > 0)
+    launch_probe_select(p->phi, r.RQ, r.rQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, st);
+  launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
+  launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
+                      p->route_idx, p->rstate, nullptr, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
+  if (!launch_ok()) { delete p; return SPARSEPR_ERR_CUDA; }
+  *out = p;
+  return SPARSEPR_OK;
+}
+
+sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                       const sparsepr_plan_host_t* in, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream, sparsepr_plan_t** out) {
+  if (!in || !in->kv_assign || !in->q_assign || !in->route_ptr || !in->route_idx) return SPARSEPR_ERR_INVALID_ARG;
+  sparsepr_plan_s* p = nullptr;
+  sparsepr_status_t s = make_plan(shape, params, workspace, workspace_bytes, cuda_stream, &p);
+  if (s != SPARSEPR_OK) return s;
+  const Resolved& r = p->r;
+  if (r.M > 0 && (!in->probe_idx || !in->probe_w)) { delete p; return SPARSEPR_ERR_INVALID_ARG; }
+  cudaStream_t st = p->stream;
+  cudaGetLastError();
+  const size_t BH = r.BH, N = r.N;
+  cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
+  cudaMemcpyAsync(p->a_K, in->kv_assign, BH * N * sizeof(int), cudaMemcpyHostToDevice, st);
+  cudaMemcpyAsync(p->a_Q, in->q_assign, BH * N * sizeof(int), cudaMemcpyHostToDevice, st);
+  cudaMemcpyAsync(p->route_ptr, in->route_ptr, BH * (r.Cq + 1) * sizeof(int), cudaMemcpyHostToDevice, st);
+  cudaMemcpyAsync(p->route_idx, in->route_idx, BH * (size_t)r.Cq * r.Ck * sizeof(int), cudaMemcpyHostToDevice, st);
+  if (r.M > 0) {
+    cudaMemcpyAsync(p->probe_idx, in->probe_idx, BH * r.M * sizeof(int), cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(p->probe_w, in->probe_w, BH * r.M * sizeof(float), cudaMemcpyHostToDevice, st);
+  }
+  launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
+  launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
+  k_sizes_from_off<<<dim3((r.Ck + 255) / 256, r.BH), 256, 0, st>>>(p->kv_off, r.Ck, p->nk);
+  k_sizes_from_off<<<dim3((r.Cq + 255) / 256, r.BH), 256, 0, st>>>(p->q_off, r.Cq, p->nq);
+  launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
+  if (!launch_ok() || cudaStreamSynchronize(st) != cudaSuccess) { delete p; return SPARSEPR_ERR_CUDA; }
+  *out = p;
+  return SPARSEPR_OK;
+}
+
+void sparsepr_plan_destroy(sparsepr_plan_t* plan) { delete plan; }
+
+sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                  float* O_sparse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!p || !Q || !K || !V || !O) return SPARSEPR_ERR_INVALID_ARG;
+  const Resolved& r = p->r;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SPARSEPR_ERR_WORKSPACE;
+  Carver dry(nullptr);
+  carve_attend(dry, r, nullptr);
+  if (workspace_bytes < dry.bytes()) return SPARSEPR_ERR_WORKSPACE;
+  AttendWs w;
+  Carver c(workspace);
+  carve_attend(c, r, &w);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaGetLastError();
+  launch_gather_rows(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, r.N, r.d, w.Qg, st);
+  launch_gather_rows(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, r.N, r.d, w.Kg, st);
+  launch_gather_rows(r.dtype, V, r.vs, r.BH, r.H, p->kv_perm, r.N, r.d, w.Vg, st);
+  const bool fitted = r.mode == 0 && r.M > 0;
+  if (fitted) {
+    ProbeArgs pa{};
+    pa.dtype = r.dtype; pa.BH = r.BH; pa.H = r.H; pa.N = r.N; pa.d = r.d; pa.M = r.M; pa.Ck = r.Ck; pa.Cq = r.Cq;
+    pa.n_split = w.n_split; pa.scale = r.scale; pa.Q = Q;
+    for (int i = 0; i < 3; ++i) pa.qs[i] = r.qs[i];
+    pa.Kg = w.Kg; pa.Vg = w.Vg; pa.probe_idx = p->probe_idx; pa.q_assign = p->a_Q; pa.kv_off = p->kv_off;
+    pa.route_ptr = p->route_ptr; pa.route_idx = p->route_idx; pa.partial = w.partial; pa.X = w.X; pa.Dn = w.Dn;
+    launch_probe_rows(pa, st);
+    FitArgs fa{};
+    fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std;
+    fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
+    launch_fit(fa, st);
+  }
+  AttnArgs aa{};
+  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.scale = r.scale;
+  aa.Q = w.Qg; aa.K = w.Kg; aa.V = w.Vg;
+  aa.q_off = p->q_off; aa.kv_off = p->kv_off; aa.route_ptr = p->route_ptr; aa.route_idx = p->route_idx;
+  aa.q_perm = p->q_perm; aa.tile_off = p->tile_off; aa.Cq = r.Cq; aa.Ck = r.Ck;
+  aa.A = fitted ? w.A : nullptr; aa.c = fitted ? w.c : nullptr;
+  aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
+  aa.O_sparse = O_sparse;
+  launch_attention_simt(aa, st);
+  if (fitted) launch_write_probe_rows(r.dtype, w.Dn, p->probe_idx, r.BH, r.H, r.M, r.d, O, r.os, st);
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_scale, const void* Q, const void* K,
+                                 const void* V, void* O, void* cuda_stream) {
+  if (!Q || !K || !V || !O) return SPARSEPR_ERR_INVALID_ARG;
+  Resolved r;
+  sparsepr_status_t s = resolve(shape, nullptr, &r);
+  if (s != SPARSEPR_OK) return s;
+  if (!(softmax_scale >= 0.f)) return SPARSEPR_ERR_INVALID_ARG;
+  if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  cudaGetLastError();
+  AttnArgs aa{};
+  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d;
+  aa.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)r.d);
+  aa.Q = Q; aa.K = K; aa.V = V; aa.O = O;
+  for (int i = 0; i < 3; ++i) { aa.qs[i] = r.qs[i]; aa.ks[i] = r.ks[i]; aa.vs[i] = r.vs[i]; aa.os[i] = r.os[i]; }
+  launch_attention_simt(aa, static_cast<cudaStream_t>(cuda_stream));
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t* out) {
+  if (!p || !out) return SPARSEPR_ERR_INVALID_ARG;
+  const Resolved& r = p->r;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  std::memset(out, 0, sizeof(*out));
+  std::vector<RouteState> rs(r.BH);
+  std::vector<int> qo((size_t)r.BH * (r.Cq + 1)), ko((size_t)r.BH * (r.Ck + 1)), rp((size_t)r.BH * (r.Cq + 1));
+  std::vector<int> ri((size_t)r.BH * r.Cq * r.Ck);
+  int errw[2] = {0, 0};
+  if (cudaMemcpy(rs.data(), p->rstate, rs.size() * sizeof(RouteState), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(qo.data(), p->q_off, qo.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(ko.data(), p->kv_off, ko.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(rp.data(), p->route_ptr, rp.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(ri.data(), p->route_idx, ri.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(errw, p->err, sizeof(errw), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SPARSEPR_ERR_CUDA;
+  out->rho_route_min = 1e300; out->rho_route_max = -1.0;
+  out->nonempty_kv_groups_min = r.Ck; out->nonempty_q_groups_min = r.Cq;
+  const double nn = (double)r.N * (double)r.N;
+  for (int bh = 0; bh < r.BH; ++bh) {
+    out->routed_pairs += rs[bh].pairs;
+    out->routed_cells += rs[bh].cells;
+    const double rho = (double)rs[bh].pairs / nn;
+    out->rho_route += rho / r.BH;
+    out->rho_route_min = std::min(out->rho_route_min, rho);
+    out->rho_route_max = std::max(out->rho_route_max, rho);
+    int neK = 0, neQ = 0;
+    const int* k = &ko[(size_t)bh * (r.Ck + 1)];
+    const int* q = &qo[(size_t)bh * (r.Cq + 1)];
+    for (int g = 0; g < r.Ck; ++g) { neK += k[g + 1] > k[g]; out->max_kv_group = std::max(out->max_kv_group, k[g + 1] - k[g]); }
+    for (int g = 0; g < r.Cq; ++g) { neQ += q[g + 1] > q[g]; out->max_q_group = std::max(out->max_q_group, q[g + 1] - q[g]); }
+    out->nonempty_kv_groups_min = std::min(out->nonempty_kv_groups_min, neK);
+    out->nonempty_q_groups_min = std::min(out->nonempty_q_groups_min, neQ);
+    // pairs issued by the tiled kernel: query tiles of 64 rows x key tiles of 64 over the concatenated routed keys
+    const int* rpp = &rp[(size_t)bh * (r.Cq + 1)];
+    const int* rii = &ri[(size_t)bh * r.Cq * r.Ck];
+    for (int a = 0; a < r.Cq; ++a) {
+      i64 keys = 0;
+      for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += k[rii[t] + 1] - k[rii[t]];
+      const i64 qt = (q[a + 1] - q[a] + 63) / 64, kt = (keys + 63) / 64;
+      out->padded_tile_pairs += qt * 64 * kt * 64;
+    }
+  }
+  out->rho_exec = out->rho_route + (double)r.M / (double)r.N;
+  out->assign_rechecked_rows = errw[1];
+  out->device_error = errw[0];
+  return SPARSEPR_OK;
+}
+
+sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* p, sparsepr_plan_host_t* o) {
+  if (!p || !o) return SPARSEPR_ERR_INVALID_ARG;
+  const Resolved& r = p->r;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  const size_t BH = r.BH, N = r.N;
+  bool ok = true;
+  auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };
+  cp(o->kv_assign, p->a_K, BH * N * 4); cp(o->q_assign, p->a_Q, BH * N * 4);
+  cp(o->kv_perm, p->kv_perm, BH * N * 4); cp(o->q_perm, p->q_perm, BH * N * 4);
+  cp(o->kv_off, p->kv_off, BH * (r.Ck + 1) * 4); cp(o->q_off, p->q_off, BH * (r.Cq + 1) * 4);
+  cp(o->route_ptr, p->route_ptr, BH * (r.Cq + 1) * 4); cp(o->route_idx, p->route_idx, BH * (size_t)r.Cq * r.Ck * 4);
+  cp(o->probe_idx, p->probe_idx, BH * r.M * 4); cp(o->probe_w, p->probe_w, BH * r.M * 4);
+  if (o->routed_pairs) {
+    std::vector<RouteState> rs(BH);
+    cp(rs.data(), p->rstate, BH * sizeof(RouteState));
+    for (size_t i = 0; i < BH; ++i) o->routed_pairs[i] = rs[i].pairs;
+  }
+  return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+// ---- single stages ---------------------------------------------------------------------
+size_t sparsepr_stage_assign_workspace_bytes(int32_t n, int32_t C, int32_t r) {
+  if (n < 1 || C < 1 || r < 1 || r > kMaxRank) return 0;
+  const size_t R = round16(r);
+  Carver c(nullptr);
+  c.take<float>((size_t)n * R); c.take<float>((size_t)C * R); c.take<float>(C); c.take<float>(1); c.take<int>(2);
+  return c.bytes();
+}
+
+sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const float* X, const float* mu, int32_t* a,
+                                        void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (n < 1 || C < 1 || r < 1 || !X || !mu || !a) return SPARSEPR_ERR_INVALID_ARG;
+  if (r > kMaxRank) return SPARSEPR_ERR_UNSUPPORTED;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) || ws_bytes < sparsepr_stage_assign_workspace_bytes(n, C, r))
+    return SPARSEPR_ERR_WORKSPACE;
+  if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int R = round16(r);
+  Carver c(ws);
+  float* Xp = c.take<float>((size_t)n * R); float* mup = c.take<float>((size_t)C * R);
+  float* mu2 = c.take<float>(C); float* mumax = c.take<float>(1); int* fx = c.take<int>(2);
+  cudaGetLastError();
+  k_pad_rows<<<(unsigned)std::min<i64>(((i64)n * R + 255) / 256, 65535), 256, 0, st>>>(X, n, r, R, Xp);
+  k_pad_rows<<<(unsigned)std::min<i64>(((i64)C * R + 255) / 256, 65535), 256, 0, st>>>(mu, C, r, R, mup);
+  launch_kmeans_finalize(mup, mu2, mumax, nullptr, nullptr, fx, 1, C, r, 0, st);
+  launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, st);
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_stage_permute(int32_t n, int32_t C, const int32_t* a, int32_t* perm, int32_t* inv,
+                                         int32_t* off, void* cuda_stream) {
+  if (n < 1 || C < 1 || !a || !perm || !inv || !off) return SPARSEPR_ERR_INVALID_ARG;
+  if (C > kMaxGroups) return SPARSEPR_ERR_UNSUPPORTED;
+  if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  cudaGetLastError();
+  launch_group_sort(a, 1, n, C, perm, inv, off, nullptr, static_cast<cudaStream_t>(cuda_stream));
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_stage_route(int32_t Cq, int32_t Ck, const float* score, const int32_t* nq, const int32_t* nk,
+                                       int64_t pair_budget, int32_t select_all, int32_t* route_ptr, int32_t* route_idx,
+                                       int64_t* pairs_out, void* cuda_stream) {
+  if (Cq < 1 || Ck < 1 || !score || !nq || !nk || !route_ptr || !route_idx || !pairs_out) return SPARSEPR_ERR_INVALID_ARG;
+  if (Cq > kMaxGroups || Ck > kMaxGroups) return SPARSEPR_ERR_UNSUPPORTED;
+  if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  cudaGetLastError();
+  launch_route_select(score, nq, nk, 1, Cq, Ck, pair_budget, select_all, route_ptr, route_idx, nullptr, reinterpret_cast<i64*>(pairs_out),
+                      static_cast<cudaStream_t>(cuda_stream));
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+}  // extern "C"

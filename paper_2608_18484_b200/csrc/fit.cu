@@ -1,0 +1,209 @@
+// Probe-Fitted Residual Reconstruction, the per-head fit (Appendix A.3): weighted
+// standardisation, weighted ridge normal equations solved by Cholesky, the
+// probe-residual output subspace, and the composed affine map
+//   R_hat_i = c + x_i A,  A = diag(1/s_x) B_lambda Psi_r Psi_r^T,  c = mu_R - mu_x A,
+// which is algebraically Eq. 9.  All arithmetic is float64; one CTA per head.
+#include "kernels.cuh"
+
+namespace spr {
+
+// scratch per head (doubles): Xb[M*d] Rb[M*d] G[d*d] B[d*d] S[d*d] T[d*d] mu_x[d] mu_R[d] s_x[d] wt[M] flag[1]
+struct FitLayout {
+  size_t Xb, Rb, G, B, S, T, mu_x, mu_R, s_x, wt, flag, total;
+  __host__ __device__ FitLayout(int M, int d) {
+    size_t o = 0;
+    Xb = o; o += (size_t)M * d;
+    Rb = o; o += (size_t)M * d;
+    G = o; o += (size_t)d * d;
+    B = o; o += (size_t)d * d;
+    S = o; o += (size_t)d * d;
+    T = o; o += (size_t)d * d;
+    mu_x = o; o += d; mu_R = o; o += d; s_x = o; o += d;
+    wt = o; o += M;
+    flag = o; o += 1;
+    total = (o + 31) / 32 * 32;
+  }
+};
+size_t fit_scratch_doubles(int BH, int M, int d) { return FitLayout(M, d).total * BH; }
+
+// alpha, weighted means, feature scale, standardised probes, unit-mean weights
+__global__ void __launch_bounds__(256) k_fit_prepare(FitArgs a) {
+  __shared__ double red[34];
+  const int bh = blockIdx.x, M = a.M, d = a.d;
+  const FitLayout L(M, d);
+  double* sc = a.scratch + (size_t)bh * L.total;
+  const float* X = a.X + (i64)bh * M * d;
+  const float* Dn = a.Dn + (i64)bh * M * d;
+  const float* w = a.w + (i64)bh * M;
+  double sw = 0.0, cnt = 0.0;
+  for (int p = threadIdx.x; p < M; p += 256) { sw += (double)w[p]; cnt += w[p] > 0.f ? 1.0 : 0.0; }
+  sw = block_sum(sw, red);
+  cnt = block_sum(cnt, red);
+  if (threadIdx.x == 0) sc[L.flag] = (sw > 0.0 && cnt > 0.0) ? 0.0 : 1.0;
+  if (!(sw > 0.0)) sw = 1.0;
+  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = cnt * (double)w[p] / sw;
+  for (int j = threadIdx.x; j < d; j += 256) {
+    double mx = 0.0, mr = 0.0;
+    for (int p = 0; p < M; ++p) {
+      const double al = (double)w[p] / sw, x = (double)X[p * d + j];
+      mx += al * x;
+      mr += al * ((double)Dn[p * d + j] - x);
+    }
+    double var = 0.0;
+    for (int p = 0; p < M; ++p) { const double t = (double)X[p * d + j] - mx; var += (double)w[p] / sw * t * t; }
+    const double s = sqrt(var + (double)a.eps_std);
+    sc[L.mu_x + j] = mx; sc[L.mu_R + j] = mr; sc[L.s_x + j] = s;
+    for (int p = 0; p < M; ++p) {
+      const double x = (double)X[p * d + j];
+      sc[L.Xb + (size_t)p * d + j] = (x - mx) / s;
+      sc[L.Rb + (size_t)p * d + j] = ((double)Dn[p * d + j] - x) - mr;
+    }
+  }
+}
+
+// blockIdx.x selects G = Xb^T W Xb + lam I, B(rhs) = Xb^T W Rb, S = Rb^T W Rb
+__global__ void __launch_bounds__(256) k_fit_gram(FitArgs a) {
+  extern __shared__ double sm_gram[];      // [2][32][d] row chunks of the left and right factor
+  const int bh = blockIdx.y, which = blockIdx.x, M = a.M, d = a.d;
+  const FitLayout L(M, d);
+  double* sc = a.scratch + (size_t)bh * L.total;
+  const double* Lm = sc + (which == 2 ? L.Rb : L.Xb);
+  const double* Rm = sc + (which == 0 ? L.Xb : L.Rb);
+  double* out = sc + (which == 0 ? L.G : which == 1 ? L.B : L.S);
+  double* ls = sm_gram;
+  double* rs = sm_gram + 32 * d;
+  const int per = d * d / 256;             // entries per thread (d = 64 or 128)
+  double acc[64];
+#pragma unroll
+  for (int e = 0; e < 64; ++e) acc[e] = 0.0;
+  for (int p0 = 0; p0 < M; p0 += 32) {
+    const int nr = min(32, M - p0);
+    __syncthreads();
+    for (int t = threadIdx.x; t < nr * d; t += 256) {
+      const int p = t / d;
+      ls[t] = Lm[(size_t)(p0 + p) * d + t % d] * sc[L.wt + p0 + p];
+      rs[t] = Rm[(size_t)(p0 + p) * d + t % d];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 64; ++e) {
+      if (e < per) {
+        const int idx = threadIdx.x + e * 256, i = idx / d, j = idx % d;
+        double s = acc[e];
+        for (int p = 0; p < nr; ++p) s += ls[p * d + i] * rs[p * d + j];
+        acc[e] = s;
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 64; ++e) {
+    if (e < per) {
+      const int idx = threadIdx.x + e * 256, i = idx / d, j = idx % d;
+      out[idx] = acc[e] + ((which == 0 && i == j) ? (double)a.lambda : 0.0);
+    }
+  }
+}
+
+// Cholesky G = L L^T in shared memory, then L Y = RHS and L^T B = Y column by column.
+__global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
+  extern __shared__ double Gs[];           // [d][d+1]
+  const int bh = blockIdx.x, d = a.d, ld = d + 1;
+  const FitLayout L(a.M, d);
+  double* sc = a.scratch + (size_t)bh * L.total;
+  __shared__ int bad;
+  if (threadIdx.x == 0) bad = sc[L.flag] != 0.0;
+  for (int e = threadIdx.x; e < d * d; e += blockDim.x) Gs[(e / d) * ld + e % d] = sc[L.G + e];
+  __syncthreads();
+  for (int k = 0; k < d; ++k) {
+    const double piv = Gs[k * ld + k];
+    if (!(piv > 0.0)) { if (threadIdx.x == 0) bad = 1; break; }     // uniform: every thread reads the same value
+    const double inv = 1.0 / sqrt(piv);
+    __syncthreads();
+    for (int i = k + threadIdx.x; i < d; i += blockDim.x) Gs[i * ld + k] *= inv;   // includes the diagonal: L_kk = sqrt(piv)
+    __syncthreads();
+    const int n = d - k - 1;
+    for (int e = threadIdx.x; e < n * n; e += blockDim.x) {
+      const int i = k + 1 + e / n, j = k + 1 + e % n;
+      if (j <= i) Gs[i * ld + j] -= Gs[i * ld + k] * Gs[j * ld + k];
+    }
+    __syncthreads();
+  }
+  __syncthreads();
+  if (bad) {
+    if (threadIdx.x == 0) { sc[L.flag] = 1.0; set_error(a.err, SPARSEPR_ERR_NUMERIC); }
+    return;
+  }
+  double* Bm = sc + L.B;
+  if (threadIdx.x < d) {
+    const int c = threadIdx.x;
+    for (int i = 0; i < d; ++i) {
+      double s = Bm[(size_t)i * d + c];
+      for (int j = 0; j < i; ++j) s -= Gs[i * ld + j] * Bm[(size_t)j * d + c];
+      Bm[(size_t)i * d + c] = s / Gs[i * ld + i];
+    }
+    for (int i = d - 1; i >= 0; --i) {
+      double s = Bm[(size_t)i * d + c];
+      for (int j = i + 1; j < d; ++j) s -= Gs[j * ld + i] * Bm[(size_t)j * d + c];
+      Bm[(size_t)i * d + c] = s / Gs[i * ld + i];
+    }
+  }
+}
+
+// T = B Psi (d x r); A = diag(1/s_x) T Psi^T; c = mu_R - mu_x A
+__global__ void __launch_bounds__(256) k_fit_compose(FitArgs a, int r) {
+  const int bh = blockIdx.x, d = a.d;
+  const FitLayout L(a.M, d);
+  double* sc = a.scratch + (size_t)bh * L.total;
+  float* A = a.A + (i64)bh * d * d;
+  float* c = a.c + (i64)bh * d;
+  if (sc[L.flag] != 0.0) {                 // no usable fit: the head falls back to hard drop
+    for (int e = threadIdx.x; e < d * d; e += 256) A[e] = 0.f;
+    for (int j = threadIdx.x; j < d; j += 256) c[j] = 0.f;
+    return;
+  }
+  const float* Psi = a.Psi + (i64)bh * d * r;
+  const double* Bm = sc + L.B;
+  double* T = sc + L.T;
+  for (int e = threadIdx.x; e < d * r; e += 256) {
+    const int i = e / r, t = e % r;
+    double s = 0.0;
+    for (int k = 0; k < d; ++k) s += Bm[(size_t)i * d + k] * (double)Psi[k * r + t];
+    T[e] = s;
+  }
+  __syncthreads();
+  double* Ad = sc + L.G;                   // G is no longer needed
+  for (int e = threadIdx.x; e < d * d; e += 256) {
+    const int i = e / d, j = e % d;
+    double s = 0.0;
+    for (int t = 0; t < r; ++t) s += T[i * r + t] * (double)Psi[j * r + t];
+    s /= sc[L.s_x + i];
+    Ad[e] = s;
+    A[e] = (float)s;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < d; j += 256) {
+    double s = sc[L.mu_R + j];
+    for (int i = 0; i < d; ++i) s -= sc[L.mu_x + i] * Ad[(size_t)i * d + j];
+    c[j] = (float)s;
+  }
+}
+
+cudaError_t init_fit() {
+  cudaError_t e = cudaFuncSetAttribute(k_fit_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 8);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_fit_gram, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 32 * 128 * 8);
+}
+
+void launch_fit(const FitArgs& a, cudaStream_t st) {
+  const int d = a.d;
+  const int r = min(a.r_out, min(a.M, d));
+  const FitLayout L(a.M, d);
+  k_fit_prepare<<<a.BH, 256, 0, st>>>(a);
+  k_fit_gram<<<dim3(3, a.BH), 256, (size_t)2 * 32 * d * 8, st>>>(a);
+  k_fit_solve<<<a.BH, 1024, (size_t)d * (d + 1) * 8, st>>>(a);
+  // Psi_r: leading eigenvectors of S = Rb^T W Rb, i.e. right singular vectors of W^(1/2) Rb.
+  launch_jacobi_eig(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.Psi, nullptr, st);
+  k_fit_compose<<<a.BH, 256, 0, st>>>(a, r);
+}
+
+}  // namespace spr

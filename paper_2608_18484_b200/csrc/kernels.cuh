@@ -1,0 +1,93 @@
+// Internal launch interface between the C-ABI layer and the kernels.
+#pragma once
+#include "common.cuh"
+
+namespace spr {
+
+// ---- partition.cu -------------------------------------------------------------
+cudaError_t init_jacobi();
+cudaError_t init_group_sort();
+void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
+                        double* Mout, cudaStream_t st);
+void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
+// Min: `batch` symmetric n x n matrices, `stride` doubles apart
+void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout,
+                       double* lam_out, cudaStream_t st);
+void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
+                    bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
+void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
+                        i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
+void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
+                            int C, int r, int update, cudaStream_t st);
+void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
+                          const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
+                          int* recheck_count, cudaStream_t st);
+void launch_group_sort(const int* assign, int BH, int N, int C, int* perm, int* inv, int* off, int* err, cudaStream_t st);
+void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, const int* off, int N,
+                        int C, int d, float* out, int* sizes, cudaStream_t st);
+void launch_gather_rows(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, int N, int d, void* out,
+                        cudaStream_t st);
+
+// ---- routing.cu ---------------------------------------------------------------
+struct RouteState {      // per head, device
+  i64 pairs;             // routed pairs
+  i64 cells;             // selected cells
+};
+void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
+                        int d, float scale, float* score, cudaStream_t st);
+void launch_route_select(const float* score, const int* nq, const int* nk, int BH, int Cq, int Ck, i64 budget,
+                         int select_all, int* route_ptr, int* route_idx, RouteState* state, i64* pairs_out,
+                         cudaStream_t st);
+void launch_count_pairs(const int* q_off, const int* kv_off, const int* route_ptr, const int* route_idx, int BH, int Cq,
+                        int Ck, RouteState* state, cudaStream_t st);
+cudaError_t init_routing();
+void launch_probe_select(const float* phiQ, int ldphi, int r, const int* q_perm, const int* q_off, const int* nq, int BH,
+                         int N, int Cq, int M, double* dist_scratch, int* probe_idx, float* probe_w, cudaStream_t st);
+
+// ---- attention_simt.cu ----------------------------------------------------------
+struct AttnArgs {
+  int dtype, BH, H, N, d;
+  float scale;
+  // group-major inputs [BH][N][d] (sparse) or strided originals (dense)
+  const void *Q, *K, *V;
+  i64 qs[3], ks[3], vs[3];
+  // sparse metadata (null for dense)
+  const int *q_off, *kv_off, *route_ptr, *route_idx, *q_perm, *tile_off;
+  int Cq, Ck;
+  // epilogue
+  const float *A, *c;         // [BH][d][d], [BH][d]; null = no correction
+  void* O; i64 os[3];
+  float* O_sparse;            // optional [BH][N][d] in original order
+};
+cudaError_t init_attention_simt();
+void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int* tile_off, cudaStream_t st);
+void launch_attention_simt(const AttnArgs& a, cudaStream_t st);
+struct ProbeArgs {
+  int dtype, BH, H, N, d, M, Ck, Cq, n_split;
+  float scale;
+  const void *Q; i64 qs[3];            // original layout (probe rows are gathered by index)
+  const void *Kg, *Vg;                 // group-major [BH][N][d]
+  const int *probe_idx, *q_assign, *kv_off, *route_ptr, *route_idx;
+  float* partial;                      // [BH][n_split][M][2][d+2]
+  float *X, *Dn;                       // outputs [BH][M][d]: sparse and dense rows
+};
+size_t probe_partial_floats(int BH, int n_split, int M, int d);
+void launch_probe_rows(const ProbeArgs& a, cudaStream_t st);
+void launch_write_probe_rows(int dtype, const float* Dn, const int* probe_idx, int BH, int H, int M, int d, void* O,
+                             const i64* os, cudaStream_t st);
+
+// ---- fit.cu -----------------------------------------------------------------------
+struct FitArgs {
+  int BH, M, d, r_out;
+  float lambda, eps_std;
+  const float *X, *Dn, *w;             // [BH][M][d], [BH][M][d], [BH][M]
+  double* scratch;                     // see fit_scratch_doubles
+  float *A, *c;                        // outputs [BH][d][d], [BH][d]
+  float* Psi;                          // [BH][d][r] scratch
+  int* err;
+};
+size_t fit_scratch_doubles(int BH, int M, int d);
+cudaError_t init_fit();
+void launch_fit(const FitArgs& a, cudaStream_t st);
+
+}  // namespace spr

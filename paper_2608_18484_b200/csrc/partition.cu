@@ -1,0 +1,654 @@
+// Response-Coupled Partitioning kernels (Section 4.1, Appendix B): sampled-query
+// Gram matrix, batched Jacobi eigen-decomposition -> feature maps, response
+// projections, k-means assignment/update, stable counting sort, group means.
+#include "kernels.cuh"
+
+namespace spr {
+
+// =============================================================================
+// Gram matrices: M_K = Q_s^T Q_s / M_s (Appendix B.1) and
+// M_Q = Ktilde^T Ktilde / (C_k^+ d) (Appendix B.2).  One CTA per head, every
+// thread owns d*d/256 entries accumulated in float64.
+// =============================================================================
+constexpr int kGramChunk = 32;
+
+template <int D>
+__device__ __forceinline__ void gram_accumulate(const float* rows, int nrows, double (&acc)[D * D / 256]) {
+  // rows: [kGramChunk][D] in shared memory
+#pragma unroll
+  for (int e = 0; e < D * D / 256; ++e) {
+    const int idx = threadIdx.x + e * 256;
+    const int i = idx / D, j = idx % D;
+    double a = acc[e];
+    for (int s = 0; s < nrows; ++s) a += (double)rows[s * D + i] * (double)rows[s * D + j];
+    acc[e] = a;
+  }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i64 sb, i64 sh, i64 sn, int H, int N,
+                                                     int Ms, u64 seed, double* __restrict__ Mout) {
+  __shared__ float rows[kGramChunk * D];
+  const int bh = blockIdx.x, b = bh / H, h = bh % H;
+  const T* base = Q + b * sb + h * sh;
+  const u64 U = sample_offset(seed, kTagQuerySample, bh);
+  double acc[D * D / 256];
+#pragma unroll
+  for (int e = 0; e < D * D / 256; ++e) acc[e] = 0.0;
+  for (int s0 = 0; s0 < Ms; s0 += kGramChunk) {
+    const int nr = min(kGramChunk, Ms - s0);
+    for (int t = threadIdx.x; t < nr * (D / 8); t += 256) {
+      const int s = t / (D / 8), c = t % (D / 8);
+      float v[8];
+      load8(base + (i64)strided_row(s0 + s, Ms, N, U) * sn + c * 8, v);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) rows[s * D + c * 8 + k] = v[k];
+    }
+    __syncthreads();
+    gram_accumulate<D>(rows, nr, acc);
+    __syncthreads();
+  }
+#pragma unroll
+  for (int e = 0; e < D * D / 256; ++e) Mout[(i64)bh * D * D + threadIdx.x + e * 256] = acc[e] / (double)Ms;
+}
+
+// kappa [BH][C][D] float32, n [BH][C] group sizes.  Empty groups are skipped and the
+// remaining centroids are centred by their uniform mean.
+template <int D>
+__global__ void __launch_bounds__(256) k_centroid_gram(const float* __restrict__ kappa, const int* __restrict__ n, int C,
+                                                       double* __restrict__ Mout) {
+  __shared__ float rows[kGramChunk * D];
+  __shared__ float mean[D];
+  __shared__ int s_cnt;
+  const int bh = blockIdx.x;
+  const float* kp = kappa + (i64)bh * C * D;
+  const int* nn = n + (i64)bh * C;
+  if (threadIdx.x == 0) s_cnt = 0;
+  __syncthreads();
+  {
+    int c = 0;
+    for (int g = threadIdx.x; g < C; g += 256) c += nn[g] > 0;
+    c = warp_sum(c);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_cnt, c);
+  }
+  __syncthreads();
+  const int cplus = s_cnt;
+  if (threadIdx.x < D) {
+    double m = 0.0;
+    for (int g = 0; g < C; ++g)
+      if (nn[g] > 0) m += (double)kp[(i64)g * D + threadIdx.x];
+    mean[threadIdx.x] = cplus > 0 ? (float)(m / cplus) : 0.f;
+  }
+  __syncthreads();
+  double acc[D * D / 256];
+#pragma unroll
+  for (int e = 0; e < D * D / 256; ++e) acc[e] = 0.0;
+  for (int g0 = 0; g0 < C; g0 += kGramChunk) {
+    const int nr = min(kGramChunk, C - g0);
+    for (int t = threadIdx.x; t < nr * D; t += 256) {
+      const int s = t / D, j = t % D;
+      rows[t] = nn[g0 + s] > 0 ? kp[(i64)(g0 + s) * D + j] - mean[j] : 0.f;
+    }
+    __syncthreads();
+    gram_accumulate<D>(rows, nr, acc);
+    __syncthreads();
+  }
+  const double denom = cplus > 0 ? (double)cplus * (double)D : 1.0;
+#pragma unroll
+  for (int e = 0; e < D * D / 256; ++e) Mout[(i64)bh * D * D + threadIdx.x + e * 256] = acc[e] / denom;
+}
+
+void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
+                        double* Mout, cudaStream_t st) {
+  if (dtype == SPARSEPR_BF16) {
+    if (d == 128) k_sample_gram<__nv_bfloat16, 128><<<BH, 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    else k_sample_gram<__nv_bfloat16, 64><<<BH, 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+  } else {
+    if (d == 128) k_sample_gram<float, 128><<<BH, 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    else k_sample_gram<float, 64><<<BH, 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+  }
+}
+void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st) {
+  if (d == 128) k_centroid_gram<128><<<BH, 256, 0, st>>>(kappa, n, C, Mout);
+  else k_centroid_gram<64><<<BH, 256, 0, st>>>(kappa, n, C, Mout);
+}
+
+// =============================================================================
+// Batched symmetric eigen-decomposition by parallel cyclic Jacobi, one CTA per
+// matrix (n = 64 or 128).  A lives in shared memory in float64, the accumulated
+// rotations V in float32.  Every round rotates n/2 disjoint (p,q) pairs; because
+// the rotation matrix is block diagonal in that pairing, each 2x2 block of A is
+// updated in place from its own four entries: A'_ij = J_i^T A_ij J_j.
+// Output: the leading r eigenvectors, scaled by sqrt(lambda_i / mean retained lambda)
+// (the feature map F of Section 4.1) or unscaled (orthonormal basis Psi_r, Eq. 9).
+// =============================================================================
+template <int NN>
+__global__ void __launch_bounds__(1024) k_jacobi_eig(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+                                                    float* __restrict__ Fout, double* __restrict__ lam_out) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* A = reinterpret_cast<double*>(smem_raw);                 // [NN][NN+1]
+  float* V = reinterpret_cast<float*>(A + NN * (NN + 1));          // [NN][NN+1]
+  double* cs = reinterpret_cast<double*>(V + NN * (NN + 1) + (NN & 1));   // [NN/2][2]
+  int* pq = reinterpret_cast<int*>(cs + NN);                        // [NN/2][2]
+  double* red = reinterpret_cast<double*>(pq + NN);                 // [34]
+  __shared__ int s_rank[NN];
+  constexpr int LD = NN + 1;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const double* Mi = Min + (i64)blockIdx.x * stride;
+  for (int e = tid; e < NN * NN; e += nt) {
+    const int i = e / NN, j = e % NN;
+    A[i * LD + j] = 0.5 * (Mi[e] + Mi[j * NN + i]);
+    V[i * LD + j] = i == j ? 1.f : 0.f;
+  }
+  __syncthreads();
+  double fro = 0.0;
+  for (int e = tid; e < NN * NN; e += nt) { const double a = A[(e / NN) * LD + e % NN]; fro += a * a; }
+  fro = block_sum(fro, red);
+  const double tol = fro * 1e-26;
+  for (int sweep = 0; sweep < 20; ++sweep) {
+    double off = 0.0;
+    for (int e = tid; e < NN * NN; e += nt) {
+      const int i = e / NN, j = e % NN;
+      if (i != j) { const double a = A[i * LD + j]; off += a * a; }
+    }
+    off = block_sum(off, red);
+    if (off <= tol) break;
+    for (int round = 0; round < NN - 1; ++round) {
+      if (tid < NN / 2) {
+        int p, q;
+        if (tid == 0) { p = NN - 1; q = round; }
+        else { p = (round + tid) % (NN - 1); q = (round - tid + (NN - 1)) % (NN - 1); }
+        if (p > q) { const int t = p; p = q; q = t; }
+        const double app = A[p * LD + p], aqq = A[q * LD + q], apq = A[p * LD + q];
+        double c = 1.0, s = 0.0;
+        if (fabs(apq) > 1e-300 && apq * apq > 1e-34 * fabs(app * aqq) ) {
+          const double tau = (aqq - app) / (2.0 * apq);
+          const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+          c = 1.0 / sqrt(1.0 + t * t);
+          s = t * c;
+        }
+        pq[2 * tid] = p; pq[2 * tid + 1] = q;
+        cs[2 * tid] = c; cs[2 * tid + 1] = s;
+      }
+      __syncthreads();
+      for (int e = tid; e < (NN / 2) * (NN / 2); e += nt) {
+        const int ki = e / (NN / 2), kj = e % (NN / 2);
+        const int pi = pq[2 * ki], qi = pq[2 * ki + 1], pj = pq[2 * kj], qj = pq[2 * kj + 1];
+        const double ci = cs[2 * ki], si = cs[2 * ki + 1], cj = cs[2 * kj], sj = cs[2 * kj + 1];
+        const double a00 = A[pi * LD + pj], a01 = A[pi * LD + qj], a10 = A[qi * LD + pj], a11 = A[qi * LD + qj];
+        // rows: J_i^T from the left
+        const double b00 = ci * a00 - si * a10, b01 = ci * a01 - si * a11;
+        const double b10 = si * a00 + ci * a10, b11 = si * a01 + ci * a11;
+        // columns: J_j from the right
+        A[pi * LD + pj] = cj * b00 - sj * b01; A[pi * LD + qj] = sj * b00 + cj * b01;
+        A[qi * LD + pj] = cj * b10 - sj * b11; A[qi * LD + qj] = sj * b10 + cj * b11;
+      }
+      for (int e = tid; e < NN * (NN / 2); e += nt) {
+        const int i = e / (NN / 2), kj = e % (NN / 2);
+        const int pj = pq[2 * kj], qj = pq[2 * kj + 1];
+        const float cj = (float)cs[2 * kj], sj = (float)cs[2 * kj + 1];
+        const float vp = V[i * LD + pj], vq = V[i * LD + qj];
+        V[i * LD + pj] = cj * vp - sj * vq;
+        V[i * LD + qj] = sj * vp + cj * vq;
+      }
+      __syncthreads();
+    }
+  }
+  // rank eigenvalues descending (ties by index), scale and emit the leading r
+  if (tid < NN) {
+    const double li = A[tid * LD + tid];
+    int rank = 0;
+    for (int j = 0; j < NN; ++j) {
+      const double lj = A[j * LD + j];
+      rank += (lj > li) || (lj == li && j < tid);
+    }
+    s_rank[tid] = rank;
+    if (lam_out) lam_out[(i64)blockIdx.x * NN + rank] = li;
+  }
+  __syncthreads();
+  double part = 0.0;
+  if (tid < NN && s_rank[tid] < r) part = fmax(A[tid * LD + tid], 0.0);
+  const double mean = block_sum(part, red) / (double)r;
+  for (int e = tid; e < NN * NN; e += nt) {
+    const int i = e / NN, col = e % NN;     // column `col` of V is the eigenvector of A[col][col]
+    const int rank = s_rank[col];
+    if (rank < r) {
+      float sc = 1.f;
+      if (scale_mode == 0) sc = mean > 0.0 ? (float)sqrt(fmax(A[col * LD + col], 0.0) / mean) : 0.f;
+      Fout[(i64)blockIdx.x * NN * r + (i64)i * r + rank] = V[i * LD + col] * sc;
+    }
+  }
+}
+
+static size_t jacobi_smem(int n) {
+  return (size_t)n * (n + 1) * 8 + (size_t)(n * (n + 1) + (n & 1)) * 4 + n * 8 + n * 4 + 34 * 8 + 16;
+}
+cudaError_t init_jacobi() {
+  cudaError_t e = cudaFuncSetAttribute(k_jacobi_eig<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(128));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_jacobi_eig<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(64));
+}
+void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout,
+                       double* lam_out, cudaStream_t st) {
+  if (n == 128) k_jacobi_eig<128><<<batch, 1024, jacobi_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  else k_jacobi_eig<64><<<batch, 1024, jacobi_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+}
+
+// =============================================================================
+// Response projections: phi_K = K F_K (Eq. 6) and phi_Q = RMS-normalised Q F_Q
+// (Eq. 7).  Each thread produces two rows of R outputs; F is staged in shared
+// memory and read by broadcast.  Also tracks max |phi| per head (for the
+// fixed-point centroid sums) and flags non-finite values.
+// =============================================================================
+template <typename T, int D, int R, bool RMS>
+__global__ void __launch_bounds__(128) k_project(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H, int N, int r,
+                                                 const float* __restrict__ F, float eps, float* __restrict__ phi,
+                                                 int ldphi, unsigned* __restrict__ maxabs_bits, int* err) {
+  __shared__ __align__(16) float Fs[D * R];
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const float* Fh = F + (i64)bh * D * r;
+  for (int e = threadIdx.x; e < D * R; e += 128) {
+    const int k = e / R, c = e % R;
+    Fs[e] = c < r ? Fh[k * r + c] : 0.f;
+  }
+  __syncthreads();
+  const T* base = X + b * sb + h * sh;
+  const int row0 = blockIdx.x * 256 + threadIdx.x, row1 = row0 + 128;
+  const bool v0 = row0 < N, v1 = row1 < N;
+  const T* p0 = base + (i64)(v0 ? row0 : 0) * sn;
+  const T* p1 = base + (i64)(v1 ? row1 : 0) * sn;
+  float acc0[R], acc1[R];
+#pragma unroll
+  for (int c = 0; c < R; ++c) { acc0[c] = 0.f; acc1[c] = 0.f; }
+  for (int k0 = 0; k0 < D; k0 += 8) {
+    float x0[8], x1[8];
+    load8(p0 + k0, x0);
+    load8(p1 + k0, x1);
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      const float4* f4 = reinterpret_cast<const float4*>(Fs + (k0 + kk) * R);
+#pragma unroll
+      for (int c = 0; c < R / 4; ++c) {
+        const float4 f = f4[c];
+        acc0[4 * c] = fmaf(x0[kk], f.x, acc0[4 * c]); acc0[4 * c + 1] = fmaf(x0[kk], f.y, acc0[4 * c + 1]);
+        acc0[4 * c + 2] = fmaf(x0[kk], f.z, acc0[4 * c + 2]); acc0[4 * c + 3] = fmaf(x0[kk], f.w, acc0[4 * c + 3]);
+        acc1[4 * c] = fmaf(x1[kk], f.x, acc1[4 * c]); acc1[4 * c + 1] = fmaf(x1[kk], f.y, acc1[4 * c + 1]);
+        acc1[4 * c + 2] = fmaf(x1[kk], f.z, acc1[4 * c + 2]); acc1[4 * c + 3] = fmaf(x1[kk], f.w, acc1[4 * c + 3]);
+      }
+    }
+  }
+  float m = 0.f;
+  bool bad = false;
+  auto finish = [&](float (&acc)[R], int row, bool valid) {
+    if (!valid) return;
+    if (RMS) {
+      float ss = 0.f;
+#pragma unroll
+      for (int c = 0; c < R; ++c) ss = fmaf(acc[c], acc[c], ss);
+      const float inv = 1.f / fmaxf(sqrtf(ss / (float)r), eps);
+#pragma unroll
+      for (int c = 0; c < R; ++c) acc[c] *= inv;
+    }
+    float* out = phi + ((i64)bh * N + row) * ldphi;
+#pragma unroll
+    for (int c = 0; c < R; c += 4)      // columns r..R-1 are written as zeros (ldphi >= R)
+      *reinterpret_cast<float4*>(out + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+      m = fmaxf(m, fabsf(acc[c]));
+      bad |= !(fabsf(acc[c]) <= 3.0e38f);
+    }
+  };
+  finish(acc0, row0, v0);
+  finish(acc1, row1, v1);
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0) atomicMax(maxabs_bits + bh, __float_as_uint(m));
+  if (bad) set_error(err, SPARSEPR_ERR_NUMERIC);
+}
+
+template <typename T, int D, bool RMS>
+static void project_dispatch_r(const T* X, const i64* xs, int BH, int H, int N, int r, const float* F, float eps,
+                               float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st) {
+  dim3 grid((N + 255) / 256, BH);
+  if (r <= 16) k_project<T, D, 16, RMS><<<grid, 128, 0, st>>>(X, xs[0], xs[1], xs[2], H, N, r, F, eps, phi, ldphi, maxabs, err);
+  else if (r <= 32) k_project<T, D, 32, RMS><<<grid, 128, 0, st>>>(X, xs[0], xs[1], xs[2], H, N, r, F, eps, phi, ldphi, maxabs, err);
+  else if (r <= 48) k_project<T, D, 48, RMS><<<grid, 128, 0, st>>>(X, xs[0], xs[1], xs[2], H, N, r, F, eps, phi, ldphi, maxabs, err);
+  else k_project<T, D, 64, RMS><<<grid, 128, 0, st>>>(X, xs[0], xs[1], xs[2], H, N, r, F, eps, phi, ldphi, maxabs, err);
+}
+void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
+                    bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st) {
+#define SPR_PROJ(TT, DD)                                                                                        \
+  do {                                                                                                          \
+    if (rms) project_dispatch_r<TT, DD, true>((const TT*)X, xs, BH, H, N, r, F, eps, phi, ldphi, maxabs, err, st); \
+    else project_dispatch_r<TT, DD, false>((const TT*)X, xs, BH, H, N, r, F, eps, phi, ldphi, maxabs, err, st);    \
+  } while (0)
+  if (dtype == SPARSEPR_BF16) { if (d == 128) SPR_PROJ(__nv_bfloat16, 128); else SPR_PROJ(__nv_bfloat16, 64); }
+  else { if (d == 128) SPR_PROJ(float, 128); else SPR_PROJ(float, 64); }
+#undef SPR_PROJ
+}
+
+// =============================================================================
+// k-means (Section 4.1).  Assignment: a[j] = argmin_c ||x_j - mu_c||^2, ties to the
+// lowest c.  Fast path in float32 via s_c = ||mu_c||^2 - 2 x.mu_c; whenever the
+// gap between the best and the second-best score is inside a proven rounding
+// bound the row is decided by the exact float64 evaluation (terms added in order
+// of k, one multiply and one add each), so the decision always equals that
+// evaluation.  Optionally accumulates order-independent fixed-point centroid sums.
+// =============================================================================
+__device__ __noinline__ int exact_assign(const float* __restrict__ x, const float* __restrict__ mu, int C, int r, int ldmu) {
+  double best = 0.0;
+  int bi = 0;
+  for (int c = 0; c < C; ++c) {
+    const float* m = mu + (i64)c * ldmu;
+    double dsum = 0.0;
+    for (int k = 0; k < r; ++k) {
+      const double diff = __dsub_rn((double)x[k], (double)m[k]);
+      dsum = __dadd_rn(dsum, __dmul_rn(diff, diff));
+    }
+    if (c == 0 || dsum < best) { best = dsum; bi = c; }
+  }
+  return bi;
+}
+
+constexpr int kAssignChunk = 64;   // centroids staged per shared-memory chunk
+
+template <int R>
+__global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__ phi, int ldphi, int N, int r,
+                                                       const float* __restrict__ mu, const float* __restrict__ mu2,
+                                                       const float* __restrict__ mumax, int C, int* __restrict__ assign,
+                                                       i64* __restrict__ sums, int* __restrict__ counts,
+                                                       const int* __restrict__ fx_shift, int* __restrict__ recheck_count) {
+  __shared__ __align__(16) float mus[kAssignChunk * R];
+  __shared__ float mu2s[kAssignChunk];
+  const int bh = blockIdx.y;
+  const float* ph = phi + (i64)bh * N * ldphi;
+  const float* muh = mu + (i64)bh * C * R;
+  const int rows[2] = {(int)(blockIdx.x * 256 + threadIdx.x), (int)(blockIdx.x * 256 + threadIdx.x + 128)};
+  float x[2][R];
+  float xn2[2] = {0.f, 0.f};
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const float* p = ph + (i64)min(rows[t], N - 1) * ldphi;
+#pragma unroll
+    for (int k = 0; k < R; k += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(p + k);      // columns r..R-1 hold zeros
+      x[t][k] = v.x; x[t][k + 1] = v.y; x[t][k + 2] = v.z; x[t][k + 3] = v.w;
+    }
+#pragma unroll
+    for (int k = 0; k < R; ++k) xn2[t] = fmaf(x[t][k], x[t][k], xn2[t]);
+  }
+  float best[2] = {3.0e38f, 3.0e38f}, second[2] = {3.0e38f, 3.0e38f};
+  int bi[2] = {0, 0};
+  for (int c0 = 0; c0 < C; c0 += kAssignChunk) {
+    const int nc = min(kAssignChunk, C - c0);
+    __syncthreads();
+    for (int e = threadIdx.x; e < nc * R; e += 128) mus[e] = muh[(i64)c0 * R + e];
+    if (threadIdx.x < nc) mu2s[threadIdx.x] = mu2[(i64)bh * C + c0 + threadIdx.x];
+    __syncthreads();
+    for (int c = 0; c < nc; ++c) {
+      const float4* m4 = reinterpret_cast<const float4*>(mus + c * R);
+      float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < R / 4; ++k) {
+        const float4 m = m4[k];
+        d0 = fmaf(x[0][4 * k], m.x, d0); d0 = fmaf(x[0][4 * k + 1], m.y, d0);
+        d0 = fmaf(x[0][4 * k + 2], m.z, d0); d0 = fmaf(x[0][4 * k + 3], m.w, d0);
+        d1 = fmaf(x[1][4 * k], m.x, d1); d1 = fmaf(x[1][4 * k + 1], m.y, d1);
+        d1 = fmaf(x[1][4 * k + 2], m.z, d1); d1 = fmaf(x[1][4 * k + 3], m.w, d1);
+      }
+      const float s0 = fmaf(-2.f, d0, mu2s[c]), s1 = fmaf(-2.f, d1, mu2s[c]);
+      if (s0 < best[0]) { second[0] = best[0]; best[0] = s0; bi[0] = c0 + c; } else if (s0 < second[0]) second[0] = s0;
+      if (s1 < best[1]) { second[1] = best[1]; best[1] = s1; bi[1] = c0 + c; } else if (s1 < second[1]) second[1] = s1;
+    }
+  }
+  const float mm = mumax[bh];
+  const int shift = fx_shift ? fx_shift[bh] : 0;
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    if (rows[t] >= N) continue;
+    // |computed score - true score| <= E for every centroid (float32 rounding of the
+    // dot product, of ||mu||^2 and of the final combination)
+    const float E = 1.5f * 5.9604645e-8f * (2.f * mm * mm + (2.f * r + 2.f) * sqrtf(xn2[t]) * mm);
+    int a = bi[t];
+    if (!(second[t] - best[t] > 2.f * E)) {
+      a = exact_assign(ph + (i64)rows[t] * ldphi, muh, C, r, R);
+      if (recheck_count) atomicAdd(recheck_count, 1);
+    }
+    assign[(i64)bh * N + rows[t]] = a;
+    if (sums) {
+      i64* s = sums + ((i64)bh * C + a) * R;
+      const double sc = ldexp(1.0, shift);
+#pragma unroll
+      for (int k = 0; k < R; ++k)
+        if (k < r) atomicAdd(reinterpret_cast<u64*>(s + k), (u64)__double2ll_rn((double)x[t][k] * sc));
+      atomicAdd(counts + (i64)bh * C + a, 1);
+    }
+  }
+}
+
+void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
+                          const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
+                          int* recheck_count, cudaStream_t st) {
+  dim3 grid((N + 255) / 256, BH);
+  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+#define SPR_ASSIGN(RR) k_kmeans_assign<RR><<<grid, 128, 0, st>>>(phi, ldphi, N, r, mu, mu2, mumax, C, assign, sums, counts, fx_shift, recheck_count)
+  if (R == 16) SPR_ASSIGN(16); else if (R == 32) SPR_ASSIGN(32); else if (R == 48) SPR_ASSIGN(48); else SPR_ASSIGN(64);
+#undef SPR_ASSIGN
+}
+
+// Initial centroids = feature rows of the strided init sample; also clears the sums
+// and derives the fixed-point shift of the head from max |phi|.
+__global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, int r, int R, int C, u64 seed, int tag,
+                              float* __restrict__ mu, i64* __restrict__ sums, int* __restrict__ counts,
+                              const unsigned* __restrict__ maxabs_bits, int* __restrict__ fx_shift) {
+  const int bh = blockIdx.y;
+  const u64 U = sample_offset(seed, tag, bh);
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < C * R; e += gridDim.x * blockDim.x) {
+    const int c = e / R, k = e % R;
+    const int row = strided_row(c, C, N, U);
+    mu[(i64)bh * C * R + e] = k < r ? phi[((i64)bh * N + row) * ldphi + k] : 0.f;
+    sums[(i64)bh * C * R + e] = 0;
+    if (k == 0) counts[(i64)bh * C + c] = 0;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    // sums of up to N values of magnitude <= maxabs must stay below 2^62
+    const float m = fmaxf(__uint_as_float(maxabs_bits[bh]), 1e-30f);
+    int e2;
+    frexpf(m, &e2);                                  // m < 2^e2
+    int nb = 0;
+    while ((1ll << nb) < (i64)N) ++nb;
+    int sh = 61 - nb - e2;
+    fx_shift[bh] = max(-60, min(sh, 60));
+  }
+}
+
+// mu <- sums / counts for non-empty clusters (empty ones keep their centroid), then
+// ||mu_c||^2 (float64 -> float32) and the largest centroid norm of the head.
+// One CTA per head.
+__global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu, float* __restrict__ mu2,
+                                                          float* __restrict__ mumax, i64* __restrict__ sums,
+                                                          int* __restrict__ counts, const int* __restrict__ fx_shift,
+                                                          int C, int r, int R, int update) {
+  __shared__ float red[34];
+  const int bh = blockIdx.x;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const double inv_sc = update ? ldexp(1.0, -fx_shift[bh]) : 0.0;
+  float mx = 0.f;
+  for (int c = w; c < C; c += nw) {
+    float* m = mu + ((i64)bh * C + c) * R;
+    i64* s = sums + ((i64)bh * C + c) * R;
+    const int cnt = update ? counts[(i64)bh * C + c] : 0;
+    double n2 = 0.0;
+    for (int k = lane; k < R; k += 32) {
+      float v = m[k];
+      if (update) {
+        if (cnt > 0 && k < r) { v = (float)((double)s[k] * inv_sc / (double)cnt); m[k] = v; }
+        s[k] = 0;
+      }
+      n2 += (double)v * (double)v;
+    }
+    n2 = warp_sum(n2);
+    __syncwarp();
+    if (lane == 0) {
+      mu2[(i64)bh * C + c] = (float)n2;
+      if (update) counts[(i64)bh * C + c] = 0;
+      mx = fmaxf(mx, (float)sqrt(n2) * 1.0000002f);
+    }
+  }
+  mx = block_max(mx, red);
+  if (threadIdx.x == 0) mumax[bh] = mx;
+}
+
+void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
+                        i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st) {
+  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  dim3 grid((C * R + 255) / 256, BH);
+  k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, mu, sums, counts, maxabs_bits, fx_shift);
+}
+void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
+                            int C, int r, int update, cudaStream_t st) {
+  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update);
+}
+
+// =============================================================================
+// Stable counting sort by group id (Section 4.3, group-major layout).  One CTA of
+// 16 warps per head; warp w owns a contiguous segment of tokens, so that ranks
+// inside a group follow the original token order.
+// =============================================================================
+constexpr int kSortWarps = 16;
+
+__global__ void __launch_bounds__(kSortWarps * 32) k_group_sort(const int* __restrict__ assign, int N, int C,
+                                                                 int* __restrict__ perm, int* __restrict__ inv,
+                                                                 int* __restrict__ off, int* err) {
+  extern __shared__ int sm_sort[];
+  int* hist = sm_sort;                    // [kSortWarps][C]
+  int* tot = hist + kSortWarps * C;       // [C]
+  __shared__ int scratch[34];
+  const int bh = blockIdx.x;
+  const int* a = assign + (i64)bh * N;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  for (int e = threadIdx.x; e < kSortWarps * C; e += blockDim.x) hist[e] = 0;
+  __syncthreads();
+  const int L = (((N + kSortWarps - 1) / kSortWarps) + 31) / 32 * 32;
+  const int s0 = w * L, s1 = min(N, s0 + L);
+  for (int i = s0 + lane; i < s1; i += 32) {
+    const int key = a[i];
+    if (key < 0 || key >= C) { set_error(err, SPARSEPR_ERR_INVALID_ARG); continue; }
+    atomicAdd(&hist[w * C + key], 1);
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    int t = 0;
+    for (int ww = 0; ww < kSortWarps; ++ww) t += hist[ww * C + c];
+    tot[c] = t;
+  }
+  __syncthreads();
+  const int total = block_exclusive_scan(tot, C, scratch);
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    int run = tot[c];
+    off[(i64)bh * (C + 1) + c] = run;
+    for (int ww = 0; ww < kSortWarps; ++ww) { const int t = hist[ww * C + c]; hist[ww * C + c] = run; run += t; }
+  }
+  if (threadIdx.x == 0) off[(i64)bh * (C + 1) + C] = total;
+  __syncthreads();
+  for (int i0 = s0; i0 < s1; i0 += 32) {
+    const int i = i0 + lane;
+    int key = i < s1 ? a[i] : -1;
+    if (key >= C) key = -1;
+    const unsigned same = __match_any_sync(0xffffffffu, key);
+    const int rank = __popc(same & ((1u << lane) - 1));
+    int pos = -1;
+    if (key >= 0) pos = hist[w * C + key] + rank;
+    __syncwarp();
+    if (key >= 0 && rank == 0) hist[w * C + key] += __popc(same);
+    __syncwarp();
+    if (key >= 0) { perm[(i64)bh * N + pos] = i; inv[(i64)bh * N + i] = pos; }
+  }
+}
+
+void launch_group_sort(const int* assign, int BH, int N, int C, int* perm, int* inv, int* off, int* err, cudaStream_t st) {
+  k_group_sort<<<BH, kSortWarps * 32, (size_t)(kSortWarps + 1) * C * sizeof(int), st>>>(assign, N, C, perm, inv, off, err);
+}
+cudaError_t init_group_sort() {
+  return cudaFuncSetAttribute(k_group_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)((kSortWarps + 1) * kMaxGroups * sizeof(int)));
+}
+
+// =============================================================================
+// Group means in the original activation space: kappa_b (Appendix B.2) and
+// theta_a (router).  One warp per group walks its members in group-major order,
+// so the float32 sums have a fixed order.
+// =============================================================================
+template <typename T, int D>
+__global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H,
+                                                     const int* __restrict__ perm, const int* __restrict__ off, int N,
+                                                     int C, float* __restrict__ out, int* __restrict__ sizes) {
+  constexpr int LPR = D / 8;                 // lanes per row (8 elements each)
+  constexpr int RPW = 32 / LPR;              // rows per warp step
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (g >= C) return;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, col = (lane % LPR) * 8;
+  const T* base = X + b * sb + h * sh;
+  const int* pm = perm + (i64)bh * N;
+  const int p0 = off[(i64)bh * (C + 1) + g], p1 = off[(i64)bh * (C + 1) + g + 1];
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int p = p0 + sub; p < p1; p += RPW) {
+    float v[8];
+    load8(base + (i64)pm[p] * sn + col, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] += v[k];
+  }
+  // combine the RPW interleaved partial sums in a fixed order
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    for (int o = LPR; o < 32; o <<= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], o);
+  const int n = p1 - p0;
+  if (sub == 0) {
+    const float invn = n > 0 ? 1.f / (float)n : 0.f;
+    float* o = out + ((i64)bh * C + g) * D + col;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o[k] = acc[k] * invn;
+  }
+  if (lane == 0 && sizes) sizes[(i64)bh * C + g] = n;
+}
+
+void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, const int* off, int N,
+                        int C, int d, float* out, int* sizes, cudaStream_t st) {
+  dim3 grid((C + 7) / 8, BH);
+#define SPR_GM(TT, DD) k_group_means<TT, DD><<<grid, 256, 0, st>>>((const TT*)X, xs[0], xs[1], xs[2], H, perm, off, N, C, out, sizes)
+  if (dtype == SPARSEPR_BF16) { if (d == 128) SPR_GM(__nv_bfloat16, 128); else SPR_GM(__nv_bfloat16, 64); }
+  else { if (d == 128) SPR_GM(float, 128); else SPR_GM(float, 64); }
+#undef SPR_GM
+}
+
+// =============================================================================
+// Row gather into the group-major layout: out[bh][p][:] = in[b,h,perm[p],:].
+// =============================================================================
+template <typename T, int D>
+__global__ void __launch_bounds__(256) k_gather_rows(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H,
+                                                     const int* __restrict__ perm, int N, T* __restrict__ out) {
+  constexpr int VEC = 16 / sizeof(T);
+  constexpr int TPR = D / VEC;               // threads per row
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const T* base = X + b * sb + h * sh;
+  const i64 t = (i64)blockIdx.x * 256 + threadIdx.x;
+  const int p = (int)(t / TPR), c = (int)(t % TPR) * VEC;
+  if (p >= N) return;
+  const int src = perm[(i64)bh * N + p];
+  *reinterpret_cast<uint4*>(out + ((i64)bh * N + p) * D + c) = *reinterpret_cast<const uint4*>(base + (i64)src * sn + c);
+}
+
+void launch_gather_rows(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, int N, int d, void* out,
+                        cudaStream_t st) {
+  const int es = dtype == SPARSEPR_BF16 ? 2 : 4;
+  const int tpr = d * es / 16;
+  dim3 grid((unsigned)(((i64)N * tpr + 255) / 256), BH);
+#define SPR_GA(TT, DD) k_gather_rows<TT, DD><<<grid, 256, 0, st>>>((const TT*)X, xs[0], xs[1], xs[2], H, perm, N, (TT*)out)
+  if (dtype == SPARSEPR_BF16) { if (d == 128) SPR_GA(__nv_bfloat16, 128); else SPR_GA(__nv_bfloat16, 64); }
+  else { if (d == 128) SPR_GA(float, 128); else SPR_GA(float, 64); }
+#undef SPR_GA
+}
+
+}  // namespace spr

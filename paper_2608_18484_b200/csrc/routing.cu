@@ -1,0 +1,383 @@
+// Shared routing (Section 4.3) and query-group-stratified probe selection
+// (Algorithm A.1, Appendix A.2).
+#include "kernels.cuh"
+
+namespace spr {
+
+// =============================================================================
+// Cell scores.  The paper fixes the pair budget and the cost model but no score;
+// this library scores cell (a,b) by the attention weight a query at the centroid
+// theta_a would give ONE key at the centroid kappa_b:
+//   p_ab = exp(l_ab - LSE_a),  l_ab = s theta_a.kappa_b,
+//   LSE_a = log sum_{b non-empty} n_b exp(l_ab).
+// One CTA per query group; logits in float64, scores stored as float32.
+// =============================================================================
+__global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ theta, const float* __restrict__ kappa,
+                                                     const int* __restrict__ nq, const int* __restrict__ nk, int Cq,
+                                                     int Ck, int d, float scale, float* __restrict__ score) {
+  __shared__ float th[128];
+  __shared__ double lg[kMaxGroups];
+  __shared__ double red[34];
+  const int bh = blockIdx.y, a = blockIdx.x;
+  float* out = score + ((i64)bh * Cq + a) * Ck;
+  if (nq[(i64)bh * Cq + a] == 0) {
+    for (int b = threadIdx.x; b < Ck; b += 256) out[b] = 0.f;
+    return;
+  }
+  if (threadIdx.x < d) th[threadIdx.x] = theta[((i64)bh * Cq + a) * d + threadIdx.x];
+  __syncthreads();
+  const int* nkh = nk + (i64)bh * Ck;
+  double mx = -1.0e300;
+  for (int b = threadIdx.x; b < Ck; b += 256) {
+    const float* kp = kappa + ((i64)bh * Ck + b) * d;
+    double l = 0.0;
+    for (int k = 0; k < d; k += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(kp + k);
+      l += (double)th[k] * (double)v.x + (double)th[k + 1] * (double)v.y + (double)th[k + 2] * (double)v.z +
+           (double)th[k + 3] * (double)v.w;
+    }
+    l *= (double)scale;
+    lg[b] = l;
+    if (nkh[b] > 0) mx = fmax(mx, l);
+  }
+  mx = block_max(mx, red);
+  double z = 0.0;
+  for (int b = threadIdx.x; b < Ck; b += 256)
+    if (nkh[b] > 0) z += (double)nkh[b] * exp(lg[b] - mx);
+  z = block_sum(z, red);
+  const double lse = mx + log(z);
+  for (int b = threadIdx.x; b < Ck; b += 256) out[b] = nkh[b] > 0 ? (float)exp(lg[b] - lse) : 0.f;
+}
+
+void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
+                        int d, float scale, float* score, cudaStream_t st) {
+  dim3 grid(Cq, BH);
+  k_cell_scores<<<grid, 256, 0, st>>>(theta, kappa, nq, nk, Cq, Ck, d, scale, score);
+}
+
+// =============================================================================
+// Cell selection under the pair budget, one CTA per head.
+//   1. forced cell per non-empty query group: its best non-empty cell (ties -> lowest b);
+//   2. the remaining cells are taken in the order (score desc, a asc, b asc) while the
+//      cumulative cost n_a n_b stays within the budget; the first cell that does not
+//      fit ends the selection.  Instead of sorting, the cut is located by a binary
+//      search over the 32-bit pattern of the (non-negative) float32 scores: the
+//      smallest threshold t with cost{cells with bits >= t} <= remaining budget, and
+//      the cells whose bits equal t-1 are then walked in (a,b) order.
+//   3. CSR emission with ascending b inside a row.
+// Everything is integer arithmetic on the given score bits.
+// =============================================================================
+__device__ __forceinline__ i64 block_sum_i64(i64 v, i64* scratch) { return block_sum<i64>(v, scratch); }
+
+__global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__ score, const int* __restrict__ nq,
+                                                       const int* __restrict__ nk, int Cq, int Ck, i64 budget,
+                                                       int select_all, int* __restrict__ route_ptr,
+                                                       int* __restrict__ route_idx, RouteState* __restrict__ state,
+                                                       i64* __restrict__ pairs_out) {
+  extern __shared__ int sm_route[];
+  int* forced = sm_route;            // [Cq]
+  int* cnt = forced + Cq;            // [Cq]
+  int* nks = cnt + Cq;               // [Ck]
+  int* nqs = nks + Ck;               // [Cq]
+  __shared__ i64 red[34];
+  __shared__ int scratch[34];
+  __shared__ i64 s_last_tie;
+  const int bh = blockIdx.x;
+  const unsigned* u = reinterpret_cast<const unsigned*>(score) + (i64)bh * Cq * Ck;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int b = threadIdx.x; b < Ck; b += blockDim.x) nks[b] = nk[(i64)bh * Ck + b];
+  for (int a = threadIdx.x; a < Cq; a += blockDim.x) nqs[a] = nq[(i64)bh * Cq + a];
+  __syncthreads();
+
+  // 1. forced cells
+  i64 fcost = 0;
+  for (int a = w; a < Cq; a += nw) {
+    u64 best = 0;      // (bits+1) << 32 | (0xFFFFFFFF - b): larger = better score, then lower b
+    if (nqs[a] > 0)
+      for (int b = lane; b < Ck; b += 32)
+        if (nks[b] > 0) {
+          const u64 key = (((u64)u[(i64)a * Ck + b] + 1ull) << 32) | (u64)(0xFFFFFFFFu - (unsigned)b);
+          best = key > best ? key : best;
+        }
+    best = warp_max(best);
+    const int fb = best ? (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull)) : -1;
+    if (lane == 0) {
+      forced[a] = fb;
+      if (fb >= 0) fcost += (i64)nqs[a] * nks[fb];
+    }
+  }
+  fcost = block_sum_i64(fcost, red);     // contains a __syncthreads: forced[] visible below
+  const i64 rem = budget - fcost;
+
+  // 2. threshold search: S(t) = cost of live, non-forced cells with bits >= t
+  u64 tstar;
+  if (select_all) tstar = 0;
+  else if (rem < 0) tstar = 1ull << 32;
+  else {
+    u64 lo = 0, hi = 1ull << 32;
+    while (lo < hi) {
+      const u64 mid = (lo + hi) >> 1;
+      i64 s = 0;
+      for (int a = w; a < Cq; a += nw) {
+        if (nqs[a] == 0) continue;
+        const int fb = forced[a];
+        i64 rs = 0;
+        for (int b = lane; b < Ck; b += 32)
+          if ((u64)u[(i64)a * Ck + b] >= mid && b != fb) rs += nks[b];     // empty groups cost 0
+        s += rs * nqs[a];
+      }
+      s = block_sum_i64(s, red);
+      if (s <= rem) hi = mid; else lo = mid + 1;
+    }
+    tstar = lo;
+  }
+  // cost already taken by the threshold tier
+  i64 taken = 0;
+  if (!select_all && rem >= 0) {
+    for (int a = w; a < Cq; a += nw) {
+      if (nqs[a] == 0) continue;
+      const int fb = forced[a];
+      i64 rs = 0;
+      for (int b = lane; b < Ck; b += 32)
+        if ((u64)u[(i64)a * Ck + b] >= tstar && b != fb) rs += nks[b];
+      taken += rs * nqs[a];
+    }
+    taken = block_sum_i64(taken, red);
+  }
+  // tie tier: cells with bits == tstar-1, in (a,b) order, longest prefix that fits
+  if (threadIdx.x == 0) s_last_tie = -1;
+  __syncthreads();
+  const bool tie_tier = !select_all && rem >= 0 && tstar > 0 && tstar <= 0xFFFFFFFFull + 1ull;
+  if (tie_tier && w == 0) {
+    const unsigned tv = (unsigned)(tstar - 1);
+    i64 cum = taken, last = -1;
+    bool stop = false;
+    for (int a = 0; a < Cq && !stop; ++a) {
+      if (nqs[a] == 0) continue;
+      const int fb = forced[a];
+      for (int b0 = 0; b0 < Ck && !stop; b0 += 32) {
+        const int b = b0 + lane;
+        const bool is = b < Ck && nks[b] > 0 && b != fb && u[(i64)a * Ck + b] == tv;
+        i64 c = is ? (i64)nqs[a] * nks[b] : 0;
+        i64 inc = c;                                        // inclusive scan over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const i64 t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        const bool over = is && (cum + inc > rem);
+        const unsigned om = __ballot_sync(0xffffffffu, over);
+        const unsigned im = __ballot_sync(0xffffffffu, is);
+        if (om) {
+          const unsigned before = im & ((1u << (__ffs(om) - 1)) - 1u);
+          if (before) last = (i64)a * Ck + b0 + (31 - __clz(before));
+          stop = true;
+        } else {
+          if (im) last = (i64)a * Ck + b0 + (31 - __clz(im));
+          cum += __shfl_sync(0xffffffffu, inc, 31);
+        }
+      }
+    }
+    if (lane == 0) s_last_tie = last;
+  }
+  __syncthreads();
+  const i64 last_tie = s_last_tie;
+  const unsigned tvv = tie_tier ? (unsigned)(tstar - 1) : 0u;
+
+  auto selected = [&](int a, int b) -> bool {
+    if (nqs[a] == 0 || nks[b] == 0) return false;
+    if (forced[a] == b) return true;
+    const unsigned bits = u[(i64)a * Ck + b];
+    if ((u64)bits >= tstar) return true;
+    return tie_tier && bits == tvv && (i64)a * Ck + b <= last_tie;
+  };
+
+  // 3. counts, offsets, lists
+  i64 pairs = 0;
+  for (int a = w; a < Cq; a += nw) {
+    int c = 0;
+    i64 rs = 0;
+    for (int b0 = 0; b0 < Ck; b0 += 32) {
+      const int b = b0 + lane;
+      const bool s = b < Ck && selected(a, b);
+      c += __popc(__ballot_sync(0xffffffffu, s));
+      if (s) rs += nks[b];
+    }
+    pairs += rs * nqs[a];
+    if (lane == 0) cnt[a] = c;
+  }
+  pairs = block_sum_i64(pairs, red);
+  const int total = block_exclusive_scan(cnt, Cq, scratch);
+  int* rp = route_ptr + (i64)bh * (Cq + 1);
+  int* ri = route_idx + (i64)bh * Cq * Ck;
+  for (int a = threadIdx.x; a < Cq; a += blockDim.x) rp[a] = cnt[a];
+  if (threadIdx.x == 0) {
+    rp[Cq] = total;
+    if (state) { state[bh].pairs = pairs; state[bh].cells = total; }
+    if (pairs_out) pairs_out[bh] = pairs;
+  }
+  for (int a = w; a < Cq; a += nw) {
+    int pos = cnt[a];
+    for (int b0 = 0; b0 < Ck; b0 += 32) {
+      const int b = b0 + lane;
+      const bool s = b < Ck && selected(a, b);
+      const unsigned m = __ballot_sync(0xffffffffu, s);
+      if (s) ri[pos + __popc(m & ((1u << lane) - 1u))] = b;
+      pos += __popc(m);
+    }
+  }
+}
+
+static size_t route_smem(int Cq, int Ck) { return (size_t)(3 * Cq + Ck) * sizeof(int); }
+// routed pairs and cells of given routes (used when a plan is imported)
+__global__ void __launch_bounds__(256) k_count_pairs(const int* __restrict__ q_off, const int* __restrict__ kv_off,
+                                                     const int* __restrict__ route_ptr, const int* __restrict__ route_idx,
+                                                     int Cq, int Ck, RouteState* __restrict__ state) {
+  __shared__ i64 red[34];
+  const int bh = blockIdx.x;
+  const int* qo = q_off + (i64)bh * (Cq + 1);
+  const int* ko = kv_off + (i64)bh * (Ck + 1);
+  const int* rp = route_ptr + (i64)bh * (Cq + 1);
+  const int* ri = route_idx + (i64)bh * Cq * Ck;
+  i64 pairs = 0;
+  for (int a = threadIdx.x; a < Cq; a += 256) {
+    i64 keys = 0;
+    for (int t = rp[a]; t < rp[a + 1]; ++t) keys += ko[ri[t] + 1] - ko[ri[t]];
+    pairs += keys * (qo[a + 1] - qo[a]);
+  }
+  pairs = block_sum<i64>(pairs, red);
+  if (threadIdx.x == 0) { state[bh].pairs = pairs; state[bh].cells = rp[Cq]; }
+}
+void launch_count_pairs(const int* q_off, const int* kv_off, const int* route_ptr, const int* route_idx, int BH, int Cq,
+                        int Ck, RouteState* state, cudaStream_t st) {
+  k_count_pairs<<<BH, 256, 0, st>>>(q_off, kv_off, route_ptr, route_idx, Cq, Ck, state);
+}
+void launch_route_select(const float* score, const int* nq, const int* nk, int BH, int Cq, int Ck, i64 budget,
+                         int select_all, int* route_ptr, int* route_idx, RouteState* state, i64* pairs_out,
+                         cudaStream_t st) {
+  k_route_select<<<BH, 1024, route_smem(Cq, Ck), st>>>(score, nq, nk, Cq, Ck, budget, select_all, route_ptr, route_idx,
+                                                        state, pairs_out);
+}
+
+// =============================================================================
+// Probe selection, Algorithm A.1.  Kernel 1 (one warp per query group): centroid
+// c_a of the group in phi_Q space and the distance d_i of every member, stored at
+// the member's group-major position.  Kernel 2 (one CTA per head): round t takes,
+// from every group that still has rows, the unpicked row with the smallest
+// (d_i, i); groups are visited in ascending id; stops at M rows.  Then the
+// coverage weights w_p = |G_a| / m_a (Appendix A.2).
+// =============================================================================
+__global__ void __launch_bounds__(256) k_probe_dist(const float* __restrict__ phi, int ldphi, int r,
+                                                    const int* __restrict__ perm, const int* __restrict__ off, int N,
+                                                    int C, double* __restrict__ dist) {
+  const int bh = blockIdx.y;
+  const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (g >= C) return;
+  const int lane = threadIdx.x & 31;
+  const int p0 = off[(i64)bh * (C + 1) + g], p1 = off[(i64)bh * (C + 1) + g + 1];
+  if (p1 <= p0) return;
+  const float* ph = phi + (i64)bh * N * ldphi;
+  const int* pm = perm + (i64)bh * N;
+  // lane owns columns lane and lane+32
+  double c0 = 0.0, c1 = 0.0;
+  for (int p = p0; p < p1; ++p) {
+    const float* row = ph + (i64)pm[p] * ldphi;
+    if (lane < r) c0 += (double)row[lane];
+    if (lane + 32 < r) c1 += (double)row[lane + 32];
+  }
+  c0 /= (double)(p1 - p0);
+  c1 /= (double)(p1 - p0);
+  for (int p = p0; p < p1; ++p) {
+    const float* row = ph + (i64)pm[p] * ldphi;
+    double s = 0.0;
+    if (lane < r) { const double t = (double)row[lane] - c0; s += t * t; }
+    if (lane + 32 < r) { const double t = (double)row[lane + 32] - c1; s += t * t; }
+    s = warp_sum(s);
+    if (lane == 0) dist[(i64)bh * N + p] = sqrt(s);
+  }
+}
+
+__global__ void __launch_bounds__(1024) k_probe_pick(const double* __restrict__ dist, const int* __restrict__ perm,
+                                                     const int* __restrict__ off, int N, int C, int M,
+                                                     int* __restrict__ probe_idx, float* __restrict__ probe_w) {
+  extern __shared__ unsigned char sm_probe[];
+  double* prev_d = reinterpret_cast<double*>(sm_probe);       // [C] last picked distance per group
+  int* prev_i = reinterpret_cast<int*>(prev_d + C);           // [C] last picked row
+  int* pick = prev_i + C;                                     // [C] row picked this round or -1
+  int* flag = pick + C;                                       // [C] scan buffer
+  int* m_a = flag + C;                                        // [C] probes per group
+  int* pgrp = m_a + C;                                        // [M] group of every probe
+  __shared__ int scratch[34];
+  const int bh = blockIdx.x;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int* of = off + (i64)bh * (C + 1);
+  const int* pm = perm + (i64)bh * N;
+  const double* ds = dist + (i64)bh * N;
+  for (int a = threadIdx.x; a < C; a += blockDim.x) { prev_d[a] = -1.0; prev_i[a] = -1; m_a[a] = 0; }
+  __syncthreads();
+  int count = 0;
+  for (int t = 0; count < M; ++t) {
+    for (int a = w; a < C; a += nw) {
+      const int p0 = of[a], p1 = of[a + 1];
+      int bi = -1;
+      double bd = 0.0;
+      if (p1 - p0 > t) {
+        const double pd = prev_d[a];
+        const int pi = prev_i[a];
+        for (int p = p0 + lane; p < p1; p += 32) {
+          const double dd = ds[p];
+          const int i = pm[p];
+          const bool after = dd > pd || (dd == pd && i > pi);            // not yet picked
+          if (after && (bi < 0 || dd < bd || (dd == bd && i < bi))) { bd = dd; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const double od = __shfl_xor_sync(0xffffffffu, bd, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (oi >= 0 && (bi < 0 || od < bd || (od == bd && oi < bi))) { bd = od; bi = oi; }
+        }
+      }
+      if (lane == 0) {
+        pick[a] = bi;
+        flag[a] = bi >= 0;
+        if (bi >= 0) { prev_d[a] = bd; prev_i[a] = bi; }
+      }
+    }
+    __syncthreads();
+    const int got = block_exclusive_scan(flag, C, scratch);
+    for (int a = threadIdx.x; a < C; a += blockDim.x) {
+      const int pos = count + flag[a];
+      if (pick[a] >= 0 && pos < M) {
+        probe_idx[(i64)bh * M + pos] = pick[a];
+        pgrp[pos] = a;
+        atomicAdd(&m_a[a], 1);
+      }
+    }
+    __syncthreads();
+    count += got;
+    if (got == 0) break;                       // fewer than M rows exist
+  }
+  __syncthreads();
+  for (int p = threadIdx.x; p < M; p += blockDim.x) {
+    if (p < count) {
+      const int a = pgrp[p];
+      probe_w[(i64)bh * M + p] = (float)(of[a + 1] - of[a]) / (float)m_a[a];
+    } else {
+      probe_idx[(i64)bh * M + p] = -1;
+      probe_w[(i64)bh * M + p] = 0.f;
+    }
+  }
+}
+
+static size_t probe_smem(int C, int M) { return (size_t)C * (8 + 5 * 4) + (size_t)M * 4 + 16; }
+cudaError_t init_routing() {
+  cudaError_t e = cudaFuncSetAttribute(k_route_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)route_smem(kMaxGroups, kMaxGroups));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_probe_pick, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)probe_smem(kMaxGroups, kMaxProbes));
+}
+void launch_probe_select(const float* phiQ, int ldphi, int r, const int* q_perm, const int* q_off, const int* nq, int BH,
+                         int N, int Cq, int M, double* dist_scratch, int* probe_idx, float* probe_w, cudaStream_t st) {
+  (void)nq;
+  dim3 grid((Cq + 7) / 8, BH);
+  k_probe_dist<<<grid, 256, 0, st>>>(phiQ, ldphi, r, q_perm, q_off, N, Cq, dist_scratch);
+  k_probe_pick<<<BH, 1024, probe_smem(Cq, M), st>>>(dist_scratch, q_perm, q_off, N, Cq, M, probe_idx, probe_w);
+}
+
+}  // namespace spr
