@@ -116,6 +116,11 @@ def test_strided_layout_bnhd():
     p1 = B.sparsepr_plan(Qs, Ks, Vs, **kw)
     p2 = B.sparsepr_plan(Qd, Kd, Vd, **kw)
     e1, e2 = B.sparsepr_plan_export(p1), B.sparsepr_plan_export(p2)
-    for k in e1:
-        assert np.array_equal(e1[k], e2[k]), k                  # the plan does not depend on the memory layout
+    for k in e1:                                                # the plan does not depend on the memory layout
+        if k == "route_idx":                                    # only the first route_ptr[-1] entries of a slab are defined
+            for i in range(2):
+                n = e1["route_ptr"][i][-1]
+                assert np.array_equal(e1[k][i][:n], e2[k][i][:n])
+        else:
+            assert np.array_equal(e1[k], e2[k]), k
     assert torch.equal(B.sparsepr_attend(p1, Qs, Ks, Vs), B.sparsepr_attend(p2, Qd, Kd, Vd))

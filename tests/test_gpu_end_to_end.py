@@ -77,7 +77,12 @@ def test_plan_is_deterministic():
     e1 = B.sparsepr_plan_export(B.sparsepr_plan(Qd, Kd, Vd, **kw))
     e2 = B.sparsepr_plan_export(B.sparsepr_plan(Qd, Kd, Vd, **kw))
     for k in e1:
-        assert np.array_equal(e1[k], e2[k]), k
+        if k == "route_idx":
+            for i in range(2):
+                n = e1["route_ptr"][i][-1]
+                assert np.array_equal(e1[k][i][:n], e2[k][i][:n])
+        else:
+            assert np.array_equal(e1[k], e2[k]), k
 
 
 def test_degenerate_inputs():
