@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of one SparsePR attention call (plan + attend) on synthetic video-DiT-like inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the whole hot path over all heads of the workload.  At
+--gpus 1 the workload is the 480p-like configuration (B=1, H=24, N=32760, d=128,
+bf16, density 25 %, 256 sampled queries, 128 probes).  With N > 1 every rank runs
+an independent replica of the same call on its own GPU (heads are independent;
+there is no collective on the data path).  Rank 0 prints ONE JSON line.
+
+--impl reference times the fp64 CPU oracle on a bounded sample of the same
+workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparsepr_attn_ms_per_call"
+UNIT = "ms/call"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------
+def launches_per_call(T, fitted):
+    """Kernels of this library launched by one plan + attend call (memsets excluded)."""
+    kmeans = 2 + T + (T - 1)                       # init, first norms, T assignments, T-1 updates
+    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 1   # per side: Gram+eig, projection, k-means, sort+means; probes; route; tiles
+    if not fitted:
+        plan -= 2
+    attend = 3 + 1 + ((2 + 5 + 1) if fitted else 0)   # gathers, attention, (probe rows+merge, fit, probe write)
+    return plan + attend
+
+
+def reference_arm(args, wl):
+    """The oracle, as it stands, on a bounded sample: every step is one full call for one
+    head of the workload cut to its first 3 frames."""
+    import multiprocessing
+    from oracle import sparsepr_oracle as orc
+    from paper_2608_18484_b200 import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    frames = 3
+    small = wl.scaled(grid=(frames,) + tuple(wl.grid[1:]))
+    prm = orc.default_params(density=wl.density, block=wl.block, n_sample=wl.n_sample,
+                             n_probe=min(wl.n_probe, 64), softmax_scale=wl.softmax_scale)
+    times = []
+    for step in range(args.warmup + args.steps):
+        Q, K, V = W.make_head(small, step % wl.H)
+        t0 = time.perf_counter()
+        orc.sparsepr_head(Q, K, V, prm, step % wl.H)
+        if step >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    per_head = float(np.mean(times))
+    # attention work grows with N^2: extrapolate the sample to one call over all heads at full length
+    value = per_head * wl.H * (wl.N / small.N) ** 2 * 1e3
+    sample = "1 head of %d per step, first %d of %d frames (N=%d of %d); value extrapolated by H*(N/N_s)^2" % (
+        wl.H, frames, wl.grid[0], small.N, wl.N)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_head * 1e3, "higher_is_better": False,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": wl.name, "N": wl.N, "H": wl.H, "d": wl.d, "density": wl.density,
+                      "n_sample": wl.n_sample, "n_probe": wl.n_probe},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
+                            "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def cpu_baseline(wl):
+    """Oracle timed on the host cores on about 10-20 s of work: one head, first 11 frames."""
+    import multiprocessing
+    from oracle import sparsepr_oracle as orc
+    from paper_2608_18484_b200 import workloads as W
+    frames = min(11, wl.grid[0])
+    small = wl.scaled(grid=(frames,) + tuple(wl.grid[1:]))
+    prm = orc.default_params(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+                             softmax_scale=wl.softmax_scale)
+    Q, K, V = W.make_head(small, 0)
+    t0 = time.perf_counter()
+    orc.sparsepr_head(Q, K, V, prm, 0)
+    dt = time.perf_counter() - t0
+    value = dt * wl.H * (wl.N / small.N) ** 2 * 1e3
+    return {"value": value, "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
+            "sample": "head 0, first %d of %d frames (N=%d): %.1f s measured; value = that x H x (N/N_s)^2" % (
+                frames, wl.grid[0], small.N, dt)}
+
+
+# --------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="video-dit-480p-like")
+    ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2608_18484_b200 import workloads as W
+    wl = W.CONFIGS[args.workload]
+    if args.heads:
+        wl = wl.scaled(H=args.heads)
+    if args.impl == "reference":
+        reference_arm(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_18484_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+
+    # ---- inputs: generated per head on the host, rounded to the storage type, made resident ----
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    Qd, Kd, Vd = [torch.empty(1, wl.H, wl.N, wl.d, dtype=dt, device=dev) for _ in range(3)]
+    pinned = [torch.empty(1, wl.H, wl.N, wl.d, dtype=dt).pin_memory() for _ in range(3)]
+    for h in range(wl.H):
+        for t, x in enumerate(W.make_head(wl, h, seed=rank)):
+            pinned[t][0, h].copy_(torch.from_numpy(x).to(dt))
+    for d_, p_ in zip((Qd, Kd, Vd), pinned):
+        d_.copy_(p_)
+    Oh = torch.empty(1, wl.H, wl.N, wl.d, dtype=dt).pin_memory()
+    params = B.make_params(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+                           softmax_scale=wl.softmax_scale)
+    O = torch.empty_like(Qd)
+
+    def step():
+        plan = B.sparsepr_plan(Qd, Kd, Vd, params=params)
+        B.sparsepr_attend(plan, Qd, Kd, Vd, out=O)
+        return plan
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        plan = step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    # ---- timed region: exactly K steps, CUDA events on the launching stream ----
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for k in range(args.steps):
+        plan = step()
+        ev[k + 1].record()
+    barrier()
+    step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[-1])
+    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    # ---- per-stage decomposition and the dense kernel of the same build (same K steps) ----
+    prof, dprof = B.Profile(), B.Profile()
+    Odense = torch.empty_like(Qd)
+    for _ in range(args.steps):
+        plan = B.sparsepr_plan(Qd, Kd, Vd, params=params, profile=prof)
+        B.sparsepr_attend(plan, Qd, Kd, Vd, out=O, profile=prof)
+    dense_steps = max(1, min(args.steps, 3))
+    B.sparsepr_dense(Qd, Kd, Vd, wl.softmax_scale, out=Odense)
+    for _ in range(dense_steps):
+        B.sparsepr_dense(Qd, Kd, Vd, wl.softmax_scale, out=Odense, profile=dprof)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    stages = {k: v / args.steps for k, v in prof.as_dict().items() if k != "dense"}
+    dense_ms = dprof.as_dict()["dense"] / dense_steps
+    st = B.sparsepr_plan_stats(plan)
+
+    # ---- accuracy against the same build's dense kernel, with and without the repair ----
+    _, Osp = B.sparsepr_attend(plan, Qd, Kd, Vd, out=O, return_sparse=True)
+    ref = Odense.float()
+    den = ref.norm()
+    rel_fit = float((O.float() - ref).norm() / den)
+    rel_hard = float((Osp - ref).norm() / den)
+    del Osp, ref
+
+    # ---- end to end through the host-buffer call ----
+    e2e = None
+    if not args.no_e2e:
+        bufs = [Qd, Kd, Vd]
+        for _ in range(2):
+            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs)
+        barrier()
+        n_e2e = max(1, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs)
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        nbytes = Qd.numel() * Qd.element_size()
+        e2e = {"value": float(t.item()), "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (block-sparse attention) ----
+    attn_ms = stages["attention"]
+    flops = 4.0 * wl.d * st["routed_pairs"]                       # QK^T and PV on executed pairs, all heads
+    issued = 4.0 * wl.d * st["padded_tile_pairs"]
+    achieved = flops / (attn_ms * 1e-3) / 1e12
+    # this build's attention kernel runs on the FP32 CUDA cores: 148 SMs x 128 lanes x 2 flop x max SM clock
+    sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak_alu = 148 * 128 * 2 * sm_max * 1e6 / 1e12
+    roofline = {"kernel": "k_attention_simt (block-sparse)", "bound": "alu", "achieved": achieved, "peak": peak_alu,
+                "unit": "TFLOP/s", "frac": achieved / peak_alu, "traffic": None,
+                "peak_source": "derived: 148 SM x 128 FP32 lanes x 2 x %.0f MHz" % sm_max,
+                "issued_tflops": issued / (attn_ms * 1e-3) / 1e12,
+                "frac_of_bf16_tensor_peak": achieved / peaks["bf16_sustained"],
+                "tensor_peak": peaks["bf16_sustained"], "tensor_peak_source": peaks["source"] + " (sustained)"}
+
+    out = {"metric": METRIC, "value": ms_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+           "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+           "config": {"workload": wl.name, "B": 1, "H": wl.H, "N": wl.N, "d": wl.d, "block": wl.block,
+                      "density_target": wl.density, "n_sample": wl.n_sample, "n_probe": wl.n_probe,
+                      "softmax_scale": wl.softmax_scale, "parallelism": "replicas x%d" % world,
+                      "l2": "inputs (3 x %.0f MB) larger than L2" % (Qd.numel() * Qd.element_size() / 1e6)},
+           "calls_per_s": world * 1e3 / ms_per_step,
+           "step_ms_min_median": [float(np.min(step_ms)), float(np.median(step_ms))],
+           "dense_ms": dense_ms, "speedup_vs_dense": dense_ms / ms_per_step,
+           "rho_route": st["rho_route"], "rho_exec": st["rho_exec"],
+           "tile_padding_factor": st["padded_tile_pairs"] / max(st["routed_pairs"], 1),
+           "rel_l2_vs_dense_kernel": {"probe_fitted": rel_fit, "hard_drop": rel_hard},
+           "stage_ms": stages, "plan_ms": sum(v for k, v in stages.items() if k in B.STAGES[:10]),
+           "attend_ms": sum(v for k, v in stages.items() if k in B.STAGES[10:15]),
+           "device_error": st["device_error"], "assign_rechecked_rows": st["assign_rechecked_rows"],
+           "gpu_launches": launches_per_call(params.kmeans_iters or 8, True) * args.steps,
+           "roofline": roofline, "clocks": clocks, "e2e": e2e}
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(wl)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -115,6 +115,26 @@ typedef struct {
   int64_t *routed_pairs;
 } sparsepr_plan_host_t;
 
+/* Stages of one call, in launch order, as indices into sparsepr_profile_t.ms.  Plan
+ * (Section 4.1, 4.3, Algorithm A.1): KEY_METRIC = sampled-query Gram and its
+ * eigen-decomposition; *_PROJECT = response coordinates (Eq. 6, Eq. 7); *_KMEANS;
+ * *_PERMUTE = counting sort and group means; QUERY_METRIC = centroid Gram and its
+ * eigen-decomposition; PROBE_SELECT; ROUTE = cell scores and selection.  Attend:
+ * GATHER = group-major copies of Q, K, V; PROBE_ROWS = exact and hard-drop rows of
+ * the probes; FIT = ridge fit and subspace; ATTENTION = block-sparse kernel with the
+ * correction epilogue; PROBE_WRITE.  DENSE = the dense entry point. */
+enum {
+  SPARSEPR_STAGE_KEY_METRIC = 0, SPARSEPR_STAGE_KEY_PROJECT, SPARSEPR_STAGE_KEY_KMEANS, SPARSEPR_STAGE_KEY_PERMUTE,
+  SPARSEPR_STAGE_QUERY_METRIC, SPARSEPR_STAGE_QUERY_PROJECT, SPARSEPR_STAGE_QUERY_KMEANS, SPARSEPR_STAGE_QUERY_PERMUTE,
+  SPARSEPR_STAGE_PROBE_SELECT, SPARSEPR_STAGE_ROUTE,
+  SPARSEPR_STAGE_GATHER, SPARSEPR_STAGE_PROBE_ROWS, SPARSEPR_STAGE_FIT, SPARSEPR_STAGE_ATTENTION,
+  SPARSEPR_STAGE_PROBE_WRITE, SPARSEPR_STAGE_DENSE, SPARSEPR_STAGE_COUNT
+};
+/* Milliseconds per stage, measured with CUDA events on the call's stream.  The
+ * *_timed calls ADD to the entries, so one zero-initialised struct can accumulate
+ * several calls. */
+typedef struct { float ms[SPARSEPR_STAGE_COUNT]; } sparsepr_profile_t;
+
 const char* sparsepr_status_string(sparsepr_status_t s);
 
 /* Bytes of DEVICE workspace that sparsepr_plan / sparsepr_plan_import and
@@ -145,6 +165,21 @@ sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* plan, const void* Q, co
  * Needs no workspace.  softmax_scale 0 selects 1/sqrt(d). */
 sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_scale,
                                  const void* Q, const void* K, const void* V, void* O, void* cuda_stream);
+
+/* The same calls with per-stage timing (the latency decomposition of the paper's
+ * Section 5.3): identical work and results; they record CUDA events between the
+ * stages, synchronise the stream before returning and add the elapsed
+ * milliseconds to *profile (HOST). */
+sparsepr_status_t sparsepr_plan_timed(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                      const void* Q, const void* K, const void* V,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                      sparsepr_plan_t** out, sparsepr_profile_t* profile);
+sparsepr_status_t sparsepr_attend_timed(const sparsepr_plan_t* plan, const void* Q, const void* K, const void* V,
+                                        void* O, float* O_sparse, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream, sparsepr_profile_t* profile);
+sparsepr_status_t sparsepr_dense_timed(const sparsepr_shape_t* shape, float softmax_scale,
+                                       const void* Q, const void* K, const void* V, void* O, void* cuda_stream,
+                                       sparsepr_profile_t* profile);
 
 /* Synchronises the stream the plan was built on, then fills *host_out. */
 sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* plan, sparsepr_stats_t* host_out);

@@ -54,7 +54,18 @@ class PlanHost(C.Structure):
                                             "route_ptr", "route_idx", "probe_idx", "probe_w", "routed_pairs")]
 
 
-EXPORTS = ["sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
+STAGES = ["key_metric", "key_project", "key_kmeans", "key_permute", "query_metric", "query_project", "query_kmeans",
+          "query_permute", "probe_select", "route", "gather", "probe_rows", "fit", "attention", "probe_write", "dense"]
+
+
+class Profile(C.Structure):
+    _fields_ = [("ms", C.c_float * len(STAGES))]
+
+    def as_dict(self):
+        return {n: float(self.ms[i]) for i, n in enumerate(STAGES)}
+
+
+EXPORTS = ["sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
@@ -77,6 +88,9 @@ def lib():
         L.sparsepr_plan.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, sz, vp, C.POINTER(vp)]
         L.sparsepr_attend.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.sparsepr_dense.argtypes = [C.POINTER(Shape), C.c_float, vp, vp, vp, vp, vp]
+        L.sparsepr_plan_timed.argtypes = L.sparsepr_plan.argtypes + [C.POINTER(Profile)]
+        L.sparsepr_attend_timed.argtypes = L.sparsepr_attend.argtypes + [C.POINTER(Profile)]
+        L.sparsepr_dense_timed.argtypes = L.sparsepr_dense.argtypes + [C.POINTER(Profile)]
         L.sparsepr_plan_stats.argtypes = [vp, C.POINTER(Stats)]
         L.sparsepr_plan_export.argtypes = [vp, C.POINTER(PlanHost)]
         L.sparsepr_plan_import.argtypes = [C.POINTER(Shape), C.POINTER(Params), C.POINTER(PlanHost), vp, sz, vp,
@@ -163,8 +177,9 @@ class Plan:
             self.handle = None
 
 
-def sparsepr_plan(Q, K, V=None, params: Params | None = None, **kw) -> Plan:
-    """Stages 1-2: partition, permutations, probe set and routes for every head."""
+def sparsepr_plan(Q, K, V=None, params: Params | None = None, profile: Profile | None = None, **kw) -> Plan:
+    """Stages 1-2: partition, permutations, probe set and routes for every head.
+    With `profile` the timed entry point is used and per-stage milliseconds are added to it."""
     params = params or make_params(**kw)
     shape = make_shape(Q, K, K if V is None else V, Q)
     L = lib()
@@ -173,13 +188,16 @@ def sparsepr_plan(Q, K, V=None, params: Params | None = None, **kw) -> Plan:
         raise SparsePRError(1, "sparsepr_plan_workspace_bytes")
     ws = _workspace(nbytes, Q.device)
     handle = C.c_void_p()
-    _check(L.sparsepr_plan(C.byref(shape), C.byref(params), Q.data_ptr(), K.data_ptr(),
-                           None if V is None else V.data_ptr(), ws.data_ptr(), ws.numel(), _stream(),
-                           C.byref(handle)), "sparsepr_plan")
+    args = (C.byref(shape), C.byref(params), Q.data_ptr(), K.data_ptr(), None if V is None else V.data_ptr(),
+            ws.data_ptr(), ws.numel(), _stream(), C.byref(handle))
+    if profile is None:
+        _check(L.sparsepr_plan(*args), "sparsepr_plan")
+    else:
+        _check(L.sparsepr_plan_timed(*args, C.byref(profile)), "sparsepr_plan_timed")
     return Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
 
 
-def sparsepr_attend(plan: Plan, Q, K, V, out=None, return_sparse=False):
+def sparsepr_attend(plan: Plan, Q, K, V, out=None, return_sparse=False, profile: Profile | None = None):
     """Stages 3-4: block-sparse attention, probe rows, fit and corrected output."""
     O = torch.empty_like(Q) if out is None else out
     shape = make_shape(Q, K, V, O)
@@ -190,18 +208,24 @@ def sparsepr_attend(plan: Plan, Q, K, V, out=None, return_sparse=False):
         plan.attend_workspace = _workspace(plan.attend_bytes, Q.device)
     ws = plan.attend_workspace
     Osp = torch.empty(Q.shape, dtype=torch.float32, device=Q.device) if return_sparse else None
-    _check(lib().sparsepr_attend(plan.handle, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
-                                 None if Osp is None else Osp.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
-           "sparsepr_attend")
+    args = (plan.handle, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
+            None if Osp is None else Osp.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    if profile is None:
+        _check(lib().sparsepr_attend(*args), "sparsepr_attend")
+    else:
+        _check(lib().sparsepr_attend_timed(*args, C.byref(profile)), "sparsepr_attend_timed")
     return (O, Osp) if return_sparse else O
 
 
-def sparsepr_dense(Q, K, V, softmax_scale=0.0, out=None):
+def sparsepr_dense(Q, K, V, softmax_scale=0.0, out=None, profile: Profile | None = None):
     """Dense attention, Eq. 1, by the same build's kernels."""
     O = torch.empty_like(Q) if out is None else out
     shape = make_shape(Q, K, V, O)
-    _check(lib().sparsepr_dense(C.byref(shape), float(softmax_scale), Q.data_ptr(), K.data_ptr(), V.data_ptr(),
-                                O.data_ptr(), _stream()), "sparsepr_dense")
+    args = (C.byref(shape), float(softmax_scale), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), _stream())
+    if profile is None:
+        _check(lib().sparsepr_dense(*args), "sparsepr_dense")
+    else:
+        _check(lib().sparsepr_dense_timed(*args, C.byref(profile)), "sparsepr_dense_timed")
     return O
 
 

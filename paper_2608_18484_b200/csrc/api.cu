@@ -94,6 +94,35 @@ cudaError_t ensure_init() {
 
 bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
 
+// Optional per-stage CUDA-event timing of one call.  Events are recorded on the call's
+// stream between stages; finish() synchronises once and accumulates the elapsed times.
+struct StageTimer {
+  sparsepr_profile_t* out;
+  cudaStream_t st;
+  std::vector<cudaEvent_t> ev;
+  std::vector<int> stage;
+  StageTimer(sparsepr_profile_t* o, cudaStream_t s) : out(o), st(s) { mark(-1); }
+  void mark(int stage_done) {
+    if (!out) return;
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) { out = nullptr; return; }
+    cudaEventRecord(e, st);
+    ev.push_back(e);
+    stage.push_back(stage_done);
+  }
+  void finish() {
+    if (out && !ev.empty() && cudaEventSynchronize(ev.back()) == cudaSuccess) {
+      for (size_t i = 1; i < ev.size(); ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ev[i - 1], ev[i]) == cudaSuccess && stage[i] >= 0 && stage[i] < SPARSEPR_STAGE_COUNT)
+          out->ms[stage[i]] += ms;
+      }
+    }
+    for (cudaEvent_t e : ev) cudaEventDestroy(e);
+    ev.clear();
+  }
+};
+
 }  // namespace
 
 struct sparsepr_plan_s {
@@ -268,10 +297,9 @@ static sparsepr_status_t make_plan(const sparsepr_shape_t* shape, const sparsepr
   return SPARSEPR_OK;
 }
 
-sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
-                                const void* K, const void* V, void* workspace, size_t workspace_bytes,
-                                void* cuda_stream, sparsepr_plan_t** out) {
-  (void)V;
+static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
+                                   const void* K, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                   sparsepr_plan_t** out, sparsepr_profile_t* prof) {
   if (!Q || !K) return SPARSEPR_ERR_INVALID_ARG;
   sparsepr_plan_s* p = nullptr;
   sparsepr_status_t s = make_plan(shape, params, workspace, workspace_bytes, cuda_stream, &p);
@@ -281,31 +309,58 @@ sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_pa
   cudaGetLastError();
   cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
+  StageTimer tm(prof, st);
   // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means
   launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
   launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, p->FK, p->lam, st);
+  tm.mark(SPARSEPR_STAGE_KEY_METRIC);
   launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+  tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
   run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, st);
+  tm.mark(SPARSEPR_STAGE_KEY_KMEANS);
   launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
   launch_group_means(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
+  tm.mark(SPARSEPR_STAGE_KEY_PERMUTE);
   // query partition: centroid metric -> F_Q -> phi_Q -> k-means
   launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
   launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, p->FQ, p->lam, st);
+  tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
   launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+  tm.mark(SPARSEPR_STAGE_QUERY_PROJECT);
   run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, st);
+  tm.mark(SPARSEPR_STAGE_QUERY_KMEANS);
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
   launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
+  tm.mark(SPARSEPR_STAGE_QUERY_PERMUTE);
   // probes and routes
   if (r.M > 0)
     launch_probe_select(p->phi, r.RQ, r.rQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, st);
+  tm.mark(SPARSEPR_STAGE_PROBE_SELECT);
   launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
                       p->route_idx, p->rstate, nullptr, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
+  tm.mark(SPARSEPR_STAGE_ROUTE);
+  tm.finish();
   if (!launch_ok()) { delete p; return SPARSEPR_ERR_CUDA; }
   *out = p;
   return SPARSEPR_OK;
+}
+
+sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
+                                const void* K, const void* V, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream, sparsepr_plan_t** out) {
+  (void)V;
+  return plan_impl(shape, params, Q, K, workspace, workspace_bytes, cuda_stream, out, nullptr);
+}
+
+sparsepr_status_t sparsepr_plan_timed(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
+                                      const void* K, const void* V, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream, sparsepr_plan_t** out, sparsepr_profile_t* profile) {
+  (void)V;
+  if (!profile) return SPARSEPR_ERR_INVALID_ARG;
+  return plan_impl(shape, params, Q, K, workspace, workspace_bytes, cuda_stream, out, profile);
 }
 
 sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
@@ -342,8 +397,9 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
 
 void sparsepr_plan_destroy(sparsepr_plan_t* plan) { delete plan; }
 
-sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const void* K, const void* V, void* O,
-                                  float* O_sparse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                     float* O_sparse, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                     sparsepr_profile_t* prof) {
   if (!p || !Q || !K || !V || !O) return SPARSEPR_ERR_INVALID_ARG;
   const Resolved& r = p->r;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return SPARSEPR_ERR_WORKSPACE;
@@ -355,9 +411,11 @@ sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const
   carve_attend(c, r, &w);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaGetLastError();
+  StageTimer tm(prof, st);
   launch_gather_rows(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, r.N, r.d, w.Qg, st);
   launch_gather_rows(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, r.N, r.d, w.Kg, st);
   launch_gather_rows(r.dtype, V, r.vs, r.BH, r.H, p->kv_perm, r.N, r.d, w.Vg, st);
+  tm.mark(SPARSEPR_STAGE_GATHER);
   const bool fitted = r.mode == 0 && r.M > 0;
   if (fitted) {
     ProbeArgs pa{};
@@ -367,10 +425,12 @@ sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const
     pa.Kg = w.Kg; pa.Vg = w.Vg; pa.probe_idx = p->probe_idx; pa.q_assign = p->a_Q; pa.kv_off = p->kv_off;
     pa.route_ptr = p->route_ptr; pa.route_idx = p->route_idx; pa.partial = w.partial; pa.X = w.X; pa.Dn = w.Dn;
     launch_probe_rows(pa, st);
+    tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
     fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std;
     fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
     launch_fit(fa, st);
+    tm.mark(SPARSEPR_STAGE_FIT);
   }
   AttnArgs aa{};
   aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.scale = r.scale;
@@ -381,8 +441,33 @@ sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const
   aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
   aa.O_sparse = O_sparse;
   launch_attention_simt(aa, st);
+  tm.mark(SPARSEPR_STAGE_ATTENTION);
   if (fitted) launch_write_probe_rows(r.dtype, w.Dn, p->probe_idx, r.BH, r.H, r.M, r.d, O, r.os, st);
+  tm.mark(SPARSEPR_STAGE_PROBE_WRITE);
+  tm.finish();
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                  float* O_sparse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return attend_impl(p, Q, K, V, O, O_sparse, workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+sparsepr_status_t sparsepr_attend_timed(const sparsepr_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                        float* O_sparse, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                        sparsepr_profile_t* profile) {
+  if (!profile) return SPARSEPR_ERR_INVALID_ARG;
+  return attend_impl(p, Q, K, V, O, O_sparse, workspace, workspace_bytes, cuda_stream, profile);
+}
+
+sparsepr_status_t sparsepr_dense_timed(const sparsepr_shape_t* shape, float softmax_scale, const void* Q, const void* K,
+                                       const void* V, void* O, void* cuda_stream, sparsepr_profile_t* profile) {
+  if (!profile) return SPARSEPR_ERR_INVALID_ARG;
+  StageTimer tm(profile, static_cast<cudaStream_t>(cuda_stream));
+  sparsepr_status_t s = sparsepr_dense(shape, softmax_scale, Q, K, V, O, cuda_stream);
+  tm.mark(SPARSEPR_STAGE_DENSE);
+  tm.finish();
+  return s;
 }
 
 sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_scale, const void* Q, const void* K,
