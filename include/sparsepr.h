@@ -207,6 +207,28 @@ size_t sparsepr_stage_assign_workspace_bytes(int32_t n, int32_t C, int32_t r);
 sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const float* X, const float* mu,
                                         int32_t* a, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* The assignment stage for callers that cannot allocate.  The paper has no
+ * counterpart of this call; it exists for users of the library such as a plug-in
+ * that runs inside an inference server which has already handed every byte of
+ * device memory to its own pool, or a control loop that may not call cudaMalloc
+ * because of the device-wide synchronisation an allocation implies.  Such a caller
+ * has nowhere to get the workspace of sparsepr_stage_assign from.  Here the scratch
+ * is a fixed array inside the library image (about 4.3 MB on every GPU that loads
+ * the library, held until the process exits), so only the inputs X [n,r], mu [C,r]
+ * (float32, DEVICE) and the output a [n] (int32, DEVICE) are passed.  The result is
+ * identical to sparsepr_stage_assign.
+ *   - Limits: n <= 16384, C <= 1024, r <= 64.  Anything larger is refused with
+ *     SPARSEPR_ERR_UNSUPPORTED ("unsupported shape or parameter") before any launch.
+ *   - The call allocates and frees nothing, on the device or through any library.
+ *   - The first call on each device looks up the device address of the array (with
+ *     that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous
+ *     call's data; every element that is read is rewritten first, so nothing has
+ *     to be cleared by the caller.  Two calls that may run on the GPU at the same
+ *     time (different streams, different threads) race on it: serialise them. */
+sparsepr_status_t sparsepr_stage_assign_static(int32_t n, int32_t C, int32_t r, const float* X, const float* mu,
+                                               int32_t* a, void* cuda_stream);
+
 /* Stable counting sort by group id (Section 4.3, group-major layout):
  * perm [n], inv [n], off [C+1], all int32 DEVICE. */
 sparsepr_status_t sparsepr_stage_permute(int32_t n, int32_t C, const int32_t* a,

@@ -65,7 +65,7 @@ class Profile(C.Structure):
         return {n: float(self.ms[i]) for i, n in enumerate(STAGES)}
 
 
-EXPORTS = ["sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
+EXPORTS = ["sparsepr_stage_assign_static", "sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
@@ -100,6 +100,7 @@ def lib():
         L.sparsepr_stage_assign_workspace_bytes.restype = sz
         L.sparsepr_stage_assign_workspace_bytes.argtypes = [i32, i32, i32]
         L.sparsepr_stage_assign.argtypes = [i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.sparsepr_stage_assign_static.argtypes = [i32, i32, i32, vp, vp, vp, vp]
         L.sparsepr_stage_permute.argtypes = [i32, i32, vp, vp, vp, vp, vp]
         L.sparsepr_stage_route.argtypes = [i32, i32, vp, vp, vp, i64, i32, vp, vp, vp, vp]
         _lib = L
@@ -302,6 +303,23 @@ def sparsepr_stage_assign(X: torch.Tensor, mu: torch.Tensor) -> torch.Tensor:
     _check(L.sparsepr_stage_assign(n, Cn, r, X.data_ptr(), mu.data_ptr(), a.data_ptr(), ws.data_ptr(), ws.numel(),
                                    _stream()), "sparsepr_stage_assign")
     return a
+
+
+def sparsepr_stage_assign_static(X: torch.Tensor, mu: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """The assignment stage without any workspace: for callers that cannot allocate device
+    memory (all of it already belongs to their own pool, or an allocation's device-wide
+    synchronisation is not acceptable where they run).  X [n,r] and mu [C,r] must be
+    contiguous float32 CUDA tensors and `out` a contiguous int32 CUDA tensor [n]; nothing
+    is allocated here or in the library.  Limits n <= 16384, C <= 1024, r <= 64; calls that
+    may overlap on the GPU must be serialised by the caller (they share one scratch array)."""
+    for t in (X, mu):
+        if t.dtype != torch.float32 or not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("X and mu must be contiguous float32 CUDA tensors")
+    if out.dtype != torch.int32 or not out.is_contiguous() or out.numel() != X.shape[0]:
+        raise ValueError("out must be a contiguous int32 tensor with one entry per row of X")
+    _check(lib().sparsepr_stage_assign_static(X.shape[0], mu.shape[0], X.shape[1], X.data_ptr(), mu.data_ptr(),
+                                              out.data_ptr(), _stream()), "sparsepr_stage_assign_static")
+    return out
 
 
 def sparsepr_stage_permute(a: torch.Tensor, Cn: int):
