@@ -87,6 +87,7 @@ cudaError_t ensure_init() {
     if ((e = init_group_sort()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_routing()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
   });
   return g_init_err;
@@ -136,7 +137,7 @@ struct sparsepr_plan_s {
   float *mu, *mu2, *mumax; i64* sums; int* counts;
   int *a_K, *a_Q, *kv_perm, *kv_inv, *q_perm, *q_inv, *kv_off, *q_off, *nk, *nq;
   float *kappa, *theta, *score;
-  int *route_ptr, *route_idx, *tile_off;
+  int *route_ptr, *route_idx, *tile_off, *tile_off128;
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
 };
@@ -168,6 +169,7 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   float* score = c.take<float>(BH * (size_t)r.Cq * r.Ck);
   int* rptr = c.take<int>(BH * (r.Cq + 1)); int* ridx = c.take<int>(BH * (size_t)r.Cq * r.Ck);
   int* toff = c.take<int>(BH * (r.Cq + 1));
+  int* toff128 = c.take<int>(BH * (r.Cq + 1));
   RouteState* rs = c.take<RouteState>(BH);
   double* pd = c.take<double>(BH * N);
   int* pidx = c.take<int>(BH * std::max(r.M, 1)); float* pw = c.take<float>(BH * std::max(r.M, 1));
@@ -176,13 +178,14 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
     p->nk = nk; p->nq = nq; p->kappa = kappa; p->theta = theta; p->score = score; p->route_ptr = rptr; p->route_idx = ridx;
-    p->tile_off = toff; p->rstate = rs; p->probe_dist = pd; p->probe_idx = pidx; p->probe_w = pw;
+    p->tile_off = toff; p->tile_off128 = toff128; p->rstate = rs; p->probe_dist = pd; p->probe_idx = pidx; p->probe_w = pw;
   }
 }
 
 struct AttendWs {
   void *Qg, *Kg, *Vg;
   float *partial, *X, *Dn, *A, *c, *Psi;
+  __nv_bfloat16* At;
   double* fit;
   int n_split;
 };
@@ -207,8 +210,9 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   float* X = c.take<float>(BH * M1 * d); float* Dn = c.take<float>(BH * M1 * d);
   float* A = c.take<float>(BH * d * d); float* cc = c.take<float>(BH * d);
   float* Psi = c.take<float>(BH * d * d);
+  __nv_bfloat16* At = c.take<__nv_bfloat16>(BH * d * d);
   double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
-  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->fit = fit; w->n_split = ns; }
+  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->fit = fit; w->n_split = ns; }
 }
 
 i64 pair_budget(const Resolved& r) {
@@ -341,6 +345,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
                       p->route_idx, p->rstate, nullptr, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, p->tile_off128, st);
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
   if (!launch_ok()) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -390,6 +395,7 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   k_sizes_from_off<<<dim3((r.Cq + 255) / 256, r.BH), 256, 0, st>>>(p->q_off, r.Cq, p->nq);
   launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, p->tile_off128, st);
   if (!launch_ok() || cudaStreamSynchronize(st) != cudaSuccess) { delete p; return SPARSEPR_ERR_CUDA; }
   *out = p;
   return SPARSEPR_OK;
@@ -440,7 +446,13 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   aa.A = fitted ? w.A : nullptr; aa.c = fitted ? w.c : nullptr;
   aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
   aa.O_sparse = O_sparse;
-  launch_attention_simt(aa, st);
+  aa.err = p->err;
+  if (attention_tc_supported(aa)) {
+    aa.tile_off = p->tile_off128;
+    if (!launch_attention_tc(aa, w.At, st)) return SPARSEPR_ERR_CUDA;
+  } else {
+    launch_attention_simt(aa, st);
+  }
   tm.mark(SPARSEPR_STAGE_ATTENTION);
   if (fitted) launch_write_probe_rows(r.dtype, w.Dn, p->probe_idx, r.BH, r.H, r.M, r.d, O, r.os, st);
   tm.mark(SPARSEPR_STAGE_PROBE_WRITE);
@@ -484,7 +496,11 @@ sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_sc
   aa.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)r.d);
   aa.Q = Q; aa.K = K; aa.V = V; aa.O = O;
   for (int i = 0; i < 3; ++i) { aa.qs[i] = r.qs[i]; aa.ks[i] = r.ks[i]; aa.vs[i] = r.vs[i]; aa.os[i] = r.os[i]; }
-  launch_attention_simt(aa, static_cast<cudaStream_t>(cuda_stream));
+  if (attention_tc_supported(aa)) {
+    if (!launch_attention_tc(aa, nullptr, static_cast<cudaStream_t>(cuda_stream))) return SPARSEPR_ERR_CUDA;
+  } else {
+    launch_attention_simt(aa, static_cast<cudaStream_t>(cuda_stream));
+  }
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 

@@ -58,10 +58,17 @@ struct AttnArgs {
   const float *A, *c;         // [BH][d][d], [BH][d]; null = no correction
   void* O; i64 os[3];
   float* O_sparse;            // optional [BH][N][d] in original order
+  int* err;                   // device error word (may be null)
 };
 cudaError_t init_attention_simt();
 void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int* tile_off, cudaStream_t st);
 void launch_attention_simt(const AttnArgs& a, cudaStream_t st);
+// ---- attention_tc.cu (tcgen05 / TMEM / TMA; bf16, d = 128) -------------------------------------
+cudaError_t init_attention_tc();
+bool attention_tc_supported(const AttnArgs& a);
+// tile_off in `a` must have been built for 128-row tiles; At: bf16 scratch [BH][128][128] when a.A != null
+bool launch_attention_tc(const AttnArgs& a, __nv_bfloat16* At, cudaStream_t st);
+
 struct ProbeArgs {
   int dtype, BH, H, N, d, M, Ck, Cq, n_split;
   float scale;
