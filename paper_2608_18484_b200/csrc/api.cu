@@ -88,6 +88,7 @@ cudaError_t ensure_init() {
     if ((e = init_routing()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
   });
   return g_init_err;
@@ -140,6 +141,7 @@ struct sparsepr_plan_s {
   int *route_ptr, *route_idx, *tile_off, *tile_off128;
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
+  __nv_bfloat16 *xh, *xl, *mh, *ml; float* xnorm; int* flagged;
 };
 
 namespace {
@@ -173,11 +175,15 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   RouteState* rs = c.take<RouteState>(BH);
   double* pd = c.take<double>(BH * N);
   int* pidx = c.take<int>(BH * std::max(r.M, 1)); float* pw = c.take<float>(BH * std::max(r.M, 1));
+  __nv_bfloat16* xh = c.take<__nv_bfloat16>(BH * N * 64); __nv_bfloat16* xl = c.take<__nv_bfloat16>(BH * N * 64);
+  __nv_bfloat16* mh = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64); __nv_bfloat16* ml = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64);
+  float* xnorm = c.take<float>(BH * N); int* flagged = c.take<int>(BH * N);
   if (p) {
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
     p->nk = nk; p->nq = nq; p->kappa = kappa; p->theta = theta; p->score = score; p->route_ptr = rptr; p->route_idx = ridx;
+    p->xh = xh; p->xl = xl; p->mh = mh; p->ml = ml; p->xnorm = xnorm; p->flagged = flagged;
     p->tile_off = toff; p->tile_off128 = toff128; p->rstate = rs; p->probe_dist = pd; p->probe_idx = pidx; p->probe_w = pw;
   }
 }
@@ -225,11 +231,23 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
   const int ld = round16(r);
   launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
   launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st);
+  const bool tcp = kmeans_tc_supported();
+  if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
-    if (!upd) cudaMemsetAsync(p->recheck, 0, sizeof(int), st);
-    launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
-                         upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
+    if (tcp) {
+      launch_split_bf16(p->mu, ld, (i64)R.BH * C, r, p->mh, p->ml, nullptr, st);
+      KmeansTcArgs ka{};
+      ka.BH = R.BH; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
+      ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2; ka.mumax = p->mumax;
+      ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
+      ka.flagged = p->flagged; ka.flag_count = p->recheck + 1; ka.recheck_total = p->recheck; ka.err = p->err;
+      launch_kmeans_assign_tc(ka, st);
+    } else {
+      if (!upd) cudaMemsetAsync(p->recheck, 0, sizeof(int), st);
+      launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
+                           upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
+    }
     if (upd) launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st);
   }
 }
@@ -316,7 +334,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   StageTimer tm(prof, st);
   // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means
   launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
-  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, p->FK, p->lam, st);
+  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
   tm.mark(SPARSEPR_STAGE_KEY_METRIC);
   launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
   tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
@@ -327,7 +345,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   tm.mark(SPARSEPR_STAGE_KEY_PERMUTE);
   // query partition: centroid metric -> F_Q -> phi_Q -> k-means
   launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
-  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, p->FQ, p->lam, st);
+  launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
   tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
   launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
@@ -433,7 +451,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     launch_probe_rows(pa, st);
     tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
-    fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std;
+    fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;
     fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
     launch_fit(fa, st);
     tm.mark(SPARSEPR_STAGE_FIT);
@@ -578,7 +596,9 @@ size_t sparsepr_stage_assign_workspace_bytes(int32_t n, int32_t C, int32_t r) {
   if (n < 1 || C < 1 || r < 1 || r > kMaxRank) return 0;
   const size_t R = round16(r);
   Carver c(nullptr);
-  c.take<float>((size_t)n * R); c.take<float>((size_t)C * R); c.take<float>(C); c.take<float>(1); c.take<int>(2);
+  c.take<float>((size_t)n * R); c.take<float>((size_t)C * R); c.take<float>(C); c.take<float>(1); c.take<int>(4);
+  c.take<__nv_bfloat16>((size_t)n * 64); c.take<__nv_bfloat16>((size_t)n * 64);
+  c.take<__nv_bfloat16>((size_t)C * 64); c.take<__nv_bfloat16>((size_t)C * 64); c.take<float>(n); c.take<int>(n);
   return c.bytes();
 }
 
@@ -593,12 +613,25 @@ sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const f
   const int R = round16(r);
   Carver c(ws);
   float* Xp = c.take<float>((size_t)n * R); float* mup = c.take<float>((size_t)C * R);
-  float* mu2 = c.take<float>(C); float* mumax = c.take<float>(1); int* fx = c.take<int>(2);
+  float* mu2 = c.take<float>(C); float* mumax = c.take<float>(1); int* fx = c.take<int>(4);
+  __nv_bfloat16* xh = c.take<__nv_bfloat16>((size_t)n * 64); __nv_bfloat16* xl = c.take<__nv_bfloat16>((size_t)n * 64);
+  __nv_bfloat16* mh = c.take<__nv_bfloat16>((size_t)C * 64); __nv_bfloat16* ml = c.take<__nv_bfloat16>((size_t)C * 64);
+  float* xnorm = c.take<float>(n); int* flagged = c.take<int>(n);
   cudaGetLastError();
   k_pad_rows<<<(unsigned)std::min<i64>(((i64)n * R + 255) / 256, 65535), 256, 0, st>>>(X, n, r, R, Xp);
   k_pad_rows<<<(unsigned)std::min<i64>(((i64)C * R + 255) / 256, 65535), 256, 0, st>>>(mu, C, r, R, mup);
   launch_kmeans_finalize(mup, mu2, mumax, nullptr, nullptr, fx, 1, C, r, 0, st);
-  launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, st);
+  if (kmeans_tc_supported() && C <= kMaxGroups) {
+    launch_split_bf16(Xp, R, n, r, xh, xl, xnorm, st);
+    launch_split_bf16(mup, R, C, r, mh, ml, nullptr, st);
+    KmeansTcArgs ka{};
+    ka.BH = 1; ka.N = n; ka.C = C; ka.r = r; ka.R = R; ka.xh = xh; ka.xl = xl; ka.mh = mh; ka.ml = ml;
+    ka.phi = Xp; ka.ldphi = R; ka.xnorm = xnorm; ka.mu = mup; ka.mu2 = mu2; ka.mumax = mumax; ka.assign = a;
+    ka.flagged = flagged; ka.flag_count = fx + 1; ka.recheck_total = fx + 2;
+    if (!launch_kmeans_assign_tc(ka, st)) return SPARSEPR_ERR_CUDA;
+  } else {
+    launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, st);
+  }
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 

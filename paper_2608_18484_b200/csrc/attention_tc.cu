@@ -16,6 +16,7 @@
 #include <cuda.h>
 #include <mutex>
 #include "kernels.cuh"
+#include "tc_common.cuh"
 
 namespace spr {
 
@@ -48,89 +49,6 @@ constexpr size_t kSmemBytes = Smem::total + 1024;                 // slack for m
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, P_FULL = 11, T_FULL = 12,
            T_EMPTY = 13, C_FULL = 14, META_FULL = 15 };
 
-// ---- PTX wrappers -------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// bounded wait: gives up after 2^28 clock cycles (more than 0.1 s; a healthy wait lasts microseconds)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  if (*abort_flag) return false;
-  const long long t0 = clock64();
-  int spins = 0;
-  while (!mbar_try(bar, parity)) {
-    if (++spins > 64) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-      if (clock64() - t0 > (1ll << 28)) { *abort_flag = 1; return false; }
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-                 "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-                 "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-               : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// shared-memory matrix descriptor, 128-byte swizzle, 8-row atoms 1024 bytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; b_mn = 1 when B is stored N-contiguous
-__device__ __forceinline__ constexpr uint32_t idesc_bf16(int b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-}
 
 struct Params {
   int BH, H, N, Cq, Ck, sparse;
@@ -298,7 +216,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   } else if (warp == 9) {
     // =========================== MMA issuer ==============================================
     if (lane == 0 && n_tiles > 0) {
-      const uint32_t idesc_qk = idesc_bf16(0), idesc_pv = idesc_bf16(1);
+      const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
       auto issue_qk = [&](int i) -> bool {
         const int s = i % kStages;
@@ -544,13 +462,15 @@ EncodeTiledFn encode_fn() {
   return g_encode;
 }
 
-// bf16 tensor viewed as (d=128, N, H, B) with element strides sb, sh, sn; box = 64 columns x box_rows rows
-bool make_map(CUtensorMap* m, const void* ptr, int N, int H, int B, i64 sb, i64 sh, i64 sn, int box_rows) {
+bool tma_available() { return encode_fn() != nullptr; }
+
+bool make_map(CUtensorMap* m, const void* ptr, int cols, int rows, int H, int B, i64 sb, i64 sh, i64 sn, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
-  const cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)(H > 1 ? sh : (i64)N * sn) * 2,
-                                 (cuuint64_t)(B > 1 ? sb : (i64)H * (H > 1 ? sh : (i64)N * sn)) * 2};
+  const i64 hstride = H > 1 ? sh : (i64)rows * sn;
+  const i64 bstride = B > 1 ? sb : (i64)H * hstride;
+  const cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)H, (cuuint64_t)B};
+  const cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)hstride * 2, (cuuint64_t)bstride * 2};
   const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -565,7 +485,7 @@ cudaError_t init_attention_tc() {
 }
 
 bool attention_tc_supported(const AttnArgs& a) {
-  return a.dtype == SPARSEPR_BF16 && a.d == 128 && tc::encode_fn() != nullptr;
+  return a.dtype == SPARSEPR_BF16 && a.d == 128 && tc::tma_available();
 }
 
 // `At` is scratch for the transposed bf16 correction matrix [BH][128][128] (only with a.A != null)
@@ -576,16 +496,16 @@ bool launch_attention_tc(const AttnArgs& a, __nv_bfloat16* At, cudaStream_t st) 
   const int B = a.BH / a.H;
   bool ok;
   if (sparse) {
-    ok = make_map(&mq, a.Q, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) && make_map(&mk, a.K, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) &&
-         make_map(&mv, a.V, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub);
+    ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) && make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) &&
+         make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub);
   } else {
-    ok = make_map(&mq, a.Q, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile) && make_map(&mk, a.K, a.N, a.H, B, a.ks[0], a.ks[1], a.ks[2], kSub) &&
-         make_map(&mv, a.V, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub);
+    ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile) && make_map(&mk, a.K, kD, a.N, a.H, B, a.ks[0], a.ks[1], a.ks[2], kSub) &&
+         make_map(&mv, a.V, kD, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub);
   }
   if (!ok) return false;
   if (a.A) {
     k_transpose_correction<<<dim3(kD / 32, kD / 32, a.BH), dim3(32, 8), 0, st>>>(a.A, At);
-    if (!make_map(&ma, At, kD, a.BH, 1, 0, (i64)kD * kD, kD, kTile)) return false;
+    if (!make_map(&ma, At, kD, kD, a.BH, 1, 0, (i64)kD * kD, kD, kTile)) return false;
   } else ma = mq;
   Params p{};
   p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.sparse = sparse;

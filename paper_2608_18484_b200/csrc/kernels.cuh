@@ -11,7 +11,8 @@ void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, 
                         double* Mout, cudaStream_t st);
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
 // Min: `batch` symmetric n x n matrices, `stride` doubles apart
-void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout,
+// precise: float64 shared-memory variant (float32 tensors); otherwise float32 in registers
+void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
                        double* lam_out, cudaStream_t st);
 void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
@@ -27,6 +28,22 @@ void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, 
                         int C, int d, float* out, int* sizes, cudaStream_t st);
 void launch_gather_rows(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, int N, int d, void* out,
                         cudaStream_t st);
+
+// ---- kmeans_tc.cu (tcgen05 score contraction + exact recheck) --------------------------------------
+struct KmeansTcArgs {
+  int BH, N, C, r, R;
+  const __nv_bfloat16 *xh, *xl, *mh, *ml;      // [BH][N][64], [BH][C][64] split operands
+  const float* phi; int ldphi;                 // fp32 features [BH][N][ldphi]
+  const float *xnorm, *mu, *mu2, *mumax;       // [BH][N], [BH][C][R], [BH][C], [BH]
+  int* assign;
+  i64* sums; int* counts; const int* fx_shift; // null sums = assignment only
+  int *flagged, *flag_count, *recheck_total, *err;
+};
+cudaError_t init_kmeans_tc();
+bool kmeans_tc_supported();
+void launch_split_bf16(const float* x, int ld, i64 rows, int r, __nv_bfloat16* hi, __nv_bfloat16* lo, float* norm,
+                       cudaStream_t st);
+bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st);
 
 // ---- routing.cu ---------------------------------------------------------------
 struct RouteState {      // per head, device
@@ -87,6 +104,7 @@ void launch_write_probe_rows(int dtype, const float* Dn, const int* probe_idx, i
 struct FitArgs {
   int BH, M, d, r_out;
   float lambda, eps_std;
+  bool precise;                        // float64 eigen-solver for the subspace
   const float *X, *Dn, *w;             // [BH][M][d], [BH][M][d], [BH][M]
   double* scratch;                     // see fit_scratch_doubles
   float *A, *c;                        // outputs [BH][d][d], [BH][d]

@@ -1,0 +1,353 @@
+// k-means assignment (Section 4.1) with the score contraction on the tensor cores.
+//
+// score(x, c) = ||mu_c||^2 - 2 x.mu_c.  The dot products run on tcgen05.mma with both
+// operands split into two bf16 words (x = xh + xl, mu = mh + ml; the products xh.mh,
+// xh.ml, xl.mh are accumulated in fp32 in TMEM; the dropped term is ~2^-18 relative).
+// Each row keeps its best and second-best score; a row whose gap is not larger than a
+// conservative bound on the score error is NOT decided here but handed to the exact
+// float64 recheck (one warp per row, same operation order as the definition), so the
+// final assignment always equals the exact float64 decision with ties to the lowest id.
+//
+// Persistent CTAs: each owns row tiles (128 rows) of one head; centroid chunks of 256
+// stream through shared memory (resident when C <= 256).  Roles: warps 0-3 epilogue
+// (one row per thread: tcgen05.ld, best/second, fixed-point centroid sums with
+// warp-level pre-aggregation), warp 4 TMA producer, warp 5 MMA issuer.
+#include "kernels.cuh"
+#include "tc_common.cuh"
+
+namespace spr {
+namespace tc {
+
+constexpr int kKmThreads = 192;
+constexpr int kKmChunk = 256;                         // centroids per MMA (N)
+constexpr uint32_t kXBytes = 128 * 128;               // one [128 rows x 64 bf16] block
+constexpr uint32_t kMuBytes = kKmChunk * 128;         // one [256 x 64 bf16] block
+
+struct KmSmem {
+  static constexpr uint32_t x = 0;                              // 2 stages x (hi, lo)
+  static constexpr uint32_t mu = x + 2 * 2 * kXBytes;           // 2 stages x (hi, lo)
+  static constexpr uint32_t bars = mu + 2 * 2 * kMuBytes;       // 12 mbarriers
+  static constexpr uint32_t misc = bars + 12 * 8;
+  static constexpr uint32_t total = misc + 32;
+};
+constexpr size_t kKmSmemBytes = KmSmem::total + 1024;
+enum KmBar { X_FULL = 0, X_EMPTY = 2, MU_FULL = 4, MU_EMPTY = 6, ACC_FULL = 8, ACC_EMPTY = 10 };
+
+struct KmParams {
+  int N, C, r, R, n_chunks, ctas_per_head;
+  const float* phi; int ldphi;          // fp32 features (for the centroid sums)
+  const float* xnorm;                   // [BH][N]
+  const float* mu2;                     // [BH][C]
+  const float* mumax;                   // [BH]
+  int* assign;
+  i64* sums; int* counts; const int* fx_shift;
+  int* flagged; int* flag_count;        // rows left to the exact recheck
+  int* err;
+};
+
+__global__ void __launch_bounds__(kKmThreads, 1)
+k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_constant__ CUtensorMap mapXl,
+                   const __grid_constant__ CUtensorMap mapMh, const __grid_constant__ CUtensorMap mapMl, KmParams prm) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw);
+  volatile int* misc = reinterpret_cast<volatile int*>(sm + KmSmem::misc);   // [0] tmem base, [1] abort
+  const uint32_t bars = base + KmSmem::bars;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y, cta = blockIdx.x;
+
+  __shared__ __align__(16) float mu2s[kMaxGroups];          // ||mu_c||^2, +inf beyond C
+  __shared__ int s_skip;
+  for (int c = tid; c < kMaxGroups; c += kKmThreads) mu2s[c] = c < prm.C ? prm.mu2[(i64)bh * prm.C + c] : INFINITY;
+  if (tid == 0) s_skip = prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT;
+  __syncthreads();
+  if (s_skip) return;
+
+  const int row_tiles = (prm.N + 127) / 128;
+  const int my_tiles = cta < row_tiles ? (row_tiles - cta + prm.ctas_per_head - 1) / prm.ctas_per_head : 0;
+  const int n_chunks = prm.n_chunks;
+  const int steps = my_tiles * n_chunks;
+  if (tid == 0) {
+    for (int i = 0; i < 12; ++i) mbar_init(bar(i), (i == ACC_EMPTY || i == ACC_EMPTY + 1) ? 128 : 1);
+    misc[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(base + KmSmem::misc, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = (uint32_t)misc[0];
+  volatile int* abort_flag = &misc[1];
+
+  if (warp == 4) {
+    // =========================== TMA producer ============================================
+    if (lane == 0) {
+      for (int q = 0; q < steps; ++q) {
+        const int tl = q / n_chunks, ch = q % n_chunks;
+        if (n_chunks > 1 || q == 0) {
+          const int ms = n_chunks > 1 ? (q & 1) : 0;
+          if (n_chunks > 1 && !mbar_wait(bar(MU_EMPTY + ms), ((q >> 1) & 1) ^ 1, abort_flag)) break;
+          mbar_expect_tx(bar(MU_FULL + ms), 2 * kMuBytes);
+          tma_load_4d(base + KmSmem::mu + ms * 2 * kMuBytes, &mapMh, bar(MU_FULL + ms), 0, ch * kKmChunk, bh, 0);
+          tma_load_4d(base + KmSmem::mu + ms * 2 * kMuBytes + kMuBytes, &mapMl, bar(MU_FULL + ms), 0, ch * kKmChunk, bh, 0);
+        }
+        if (ch == 0) {
+          const int xs = tl & 1;
+          if (!mbar_wait(bar(X_EMPTY + xs), ((tl >> 1) & 1) ^ 1, abort_flag)) break;
+          const int row0 = (cta + tl * prm.ctas_per_head) * 128;
+          mbar_expect_tx(bar(X_FULL + xs), 2 * kXBytes);
+          tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes, &mapXh, bar(X_FULL + xs), 0, row0, bh, 0);
+          tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes + kXBytes, &mapXl, bar(X_FULL + xs), 0, row0, bh, 0);
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // =========================== MMA issuer ================================================
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16(0, kKmChunk);
+      const int ksteps = prm.R / 16;
+      for (int q = 0; q < steps; ++q) {
+        const int tl = q / n_chunks, ch = q % n_chunks;
+        const int xs = tl & 1, ms = n_chunks > 1 ? (q & 1) : 0;
+        if (ch == 0 && !mbar_wait(bar(X_FULL + xs), (tl >> 1) & 1, abort_flag)) break;
+        if ((n_chunks > 1 || q == 0) && !mbar_wait(bar(MU_FULL + ms), n_chunks > 1 ? ((q >> 1) & 1) : 0, abort_flag)) break;
+        if (!mbar_wait(bar(ACC_EMPTY + (q & 1)), ((q >> 1) & 1) ^ 1, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d = tmem + (uint32_t)(q & 1) * 256u;
+        const uint32_t xh = base + KmSmem::x + xs * 2 * kXBytes, xl = xh + kXBytes;
+        const uint32_t mh = base + KmSmem::mu + ms * 2 * kMuBytes, ml = mh + kMuBytes;
+        uint32_t acc = 0;
+        for (int kk = 0; kk < ksteps; ++kk) { umma_bf16(d, smem_desc(xh + kk * 32, 16), smem_desc(mh + kk * 32, 16), idesc, acc); acc = 1; }
+        for (int kk = 0; kk < ksteps; ++kk) umma_bf16(d, smem_desc(xh + kk * 32, 16), smem_desc(ml + kk * 32, 16), idesc, 1);
+        for (int kk = 0; kk < ksteps; ++kk) umma_bf16(d, smem_desc(xl + kk * 32, 16), smem_desc(mh + kk * 32, 16), idesc, 1);
+        if (ch == n_chunks - 1) umma_commit(bar(X_EMPTY + xs));
+        if (n_chunks > 1) umma_commit(bar(MU_EMPTY + ms));
+        umma_commit(bar(ACC_FULL + (q & 1)));
+      }
+    }
+  } else {
+    // =========================== epilogue: argmin, sums =====================================
+    const uint32_t FULL = 0xffffffffu;
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const float mm = prm.mumax[bh];
+    bool ok = true;
+    for (int tl = 0; tl < my_tiles; ++tl) {
+      const int row = (cta + tl * prm.ctas_per_head) * 128 + warp * 32 + lane;
+      float best = 3.0e38f, second = 3.0e38f;
+      int bi = 0;
+      // features of the warp's 32 rows for this lane's two columns (used by the centroid sums);
+      // issued before the score wait so that the loads overlap it
+      float pv0[32], pv1[32];
+      if (prm.sums) {
+        const int rowbase = (cta + tl * prm.ctas_per_head) * 128 + warp * 32;
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) {
+          const int rw = min(rowbase + rr, prm.N - 1);
+          const float* xr = prm.phi + ((i64)bh * prm.N + rw) * prm.ldphi;
+          pv0[rr] = lane < prm.r ? xr[lane] : 0.f;
+          pv1[rr] = lane + 32 < prm.r ? xr[lane + 32] : 0.f;
+        }
+      }
+      for (int ch = 0; ch < n_chunks; ++ch) {
+        const int q = tl * n_chunks + ch;
+        ok = __all_sync(FULL, ok && mbar_wait(bar(ACC_FULL + (q & 1)), (q >> 1) & 1, abort_flag));
+        if (!ok) continue;
+        tc_fence_after();
+        const int c0 = ch * kKmChunk;
+        const int nvalid = min(kKmChunk, prm.C - c0);
+#pragma unroll 1
+        for (int g = 0; g < kKmChunk / 32; ++g) {
+          if (g * 32 >= nvalid) break;                       // uniform: whole column groups beyond C
+          float t[32];
+          tmem_ld32(tmem + lane_addr + (uint32_t)(q & 1) * 256u + g * 32, t);
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const int c = c0 + g * 32 + j;
+            const float4 m4 = *reinterpret_cast<const float4*>(mu2s + c);
+            const float mv[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const float s = fmaf(-2.f, t[j + u], mv[u]);
+              second = fminf(second, fmaxf(s, best));
+              bi = s < best ? c + u : bi;
+              best = fminf(best, s);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar(ACC_EMPTY + (q & 1)));
+      }
+      // decide, or hand the row to the exact recheck
+      const bool valid = ok && row < prm.N;
+      bool decided = false;
+      if (valid) {
+        const float xn = prm.xnorm[(i64)bh * prm.N + row];
+        // bound on |computed score - true score|: split-operand products (2^-13 relative with
+        // margin), fp32 accumulation and the final combination
+        const float E = 2.5e-4f * xn * mm + 1.0e-6f * (mm * mm + xn * mm);
+        decided = second - best > 2.f * E;
+        prm.assign[(i64)bh * prm.N + row] = bi;
+        if (!decided) {
+          const int pos = atomicAdd(prm.flag_count, 1);
+          prm.flagged[pos] = bh * prm.N + row;
+        }
+      }
+      if (prm.sums) {
+        // warp-level pre-aggregation: lanes = feature columns (lane, lane+32); the 32 rows of the
+        // warp were prefetched above; rows of one cluster are summed in row order, then one
+        // fixed-point atomic per (cluster, column)
+        unsigned todo = __ballot_sync(FULL, decided);
+        const double scl = ldexp(1.0, prm.fx_shift[bh]);
+        i64 f0[32], f1[32];
+#pragma unroll
+        for (int rr = 0; rr < 32; ++rr) {
+          f0[rr] = __double2ll_rn((double)pv0[rr] * scl);
+          f1[rr] = __double2ll_rn((double)pv1[rr] * scl);
+        }
+        while (todo) {
+          const int leader = __ffs(todo) - 1;
+          const int cl = __shfl_sync(FULL, bi, leader);
+          const unsigned members = __ballot_sync(FULL, decided && bi == cl) & todo;
+          todo &= ~members;
+          i64 acc0 = 0, acc1 = 0;
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr) {
+            const bool in = (members >> rr) & 1u;
+            acc0 += in ? f0[rr] : 0;
+            acc1 += in ? f1[rr] : 0;
+          }
+          i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
+          if (lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane), (u64)acc0);
+          if (lane + 32 < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane + 32), (u64)acc1);
+          if (lane == 0) atomicAdd(prm.counts + (i64)bh * prm.C + cl, __popc(members));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int k = 0; k < 64; ++k) __nanosleep(1000);
+    if (tid == 0) set_error(prm.err, SPARSEPR_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// Exact decision for the rows the fast path could not prove: one warp per row, lanes over
+// centroids, squared distance in float64 with the terms added in order of k.
+__global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ flagged, const int* __restrict__ flag_count,
+                                                        const float* __restrict__ phi, int ldphi, int N, int r, int R,
+                                                        const float* __restrict__ mu, int C, int* __restrict__ assign,
+                                                        i64* __restrict__ sums, int* __restrict__ counts,
+                                                        const int* __restrict__ fx_shift, int* __restrict__ recheck_total) {
+  const int lane = threadIdx.x & 31;
+  const int warps = gridDim.x * (blockDim.x >> 5);
+  const int n = *flag_count;
+  for (int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n; i += warps) {
+    const int gr = flagged[i];
+    const int bh = gr / N;
+    const float* x = phi + (i64)gr * ldphi;
+    const float* muh = mu + (i64)bh * C * R;
+    double best = 0.0;
+    int bi = -1;
+    for (int c = lane; c < C; c += 32) {
+      const float4* m4 = reinterpret_cast<const float4*>(muh + (i64)c * R);
+      const float4* x4 = reinterpret_cast<const float4*>(x);
+      double dsum = 0.0;
+      for (int k4 = 0; k4 < (r + 3) / 4; ++k4) {            // columns r..R-1 hold zeros on both sides
+        const float4 xv = x4[k4], mv = m4[k4];
+        const float xs[4] = {xv.x, xv.y, xv.z, xv.w}, ms[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (k4 * 4 + u < r) {
+            const double diff = __dsub_rn((double)xs[u], (double)ms[u]);
+            dsum = __dadd_rn(dsum, __dmul_rn(diff, diff));
+          }
+        }
+      }
+      if (bi < 0 || dsum < best) { best = dsum; bi = c; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (oi >= 0 && (bi < 0 || ob < best || (ob == best && oi < bi))) { best = ob; bi = oi; }
+    }
+    if (lane == 0) assign[gr] = bi;
+    if (sums) {
+      const double scl = ldexp(1.0, fx_shift[bh]);
+      i64* s = sums + ((i64)bh * C + bi) * R;
+      for (int k = lane; k < r; k += 32) atomicAdd(reinterpret_cast<u64*>(s + k), (u64)__double2ll_rn((double)x[k] * scl));
+      if (lane == 0) atomicAdd(counts + (i64)bh * C + bi, 1);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && recheck_total) *recheck_total = n;
+}
+
+// phi fp32 [rows][ld] -> hi/lo bf16 [rows][64] (zero padded) and the row norms
+__global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ x, int ld, i64 rows, int r,
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                    float* __restrict__ norm) {
+  const i64 t = (i64)blockIdx.x * 256 + threadIdx.x;
+  const i64 row = t >> 3;
+  const int c0 = (int)(t & 7) * 8;
+  if (row >= rows) return;
+  float v[8], h[8], l[8];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    v[k] = c0 + k < r ? x[row * ld + c0 + k] : 0.f;
+    const __nv_bfloat16 hb = __float2bfloat16_rn(v[k]);
+    h[k] = __bfloat162float(hb);
+    l[k] = v[k] - h[k];
+    ss = fmaf(v[k], v[k], ss);
+  }
+  store8(hi + row * 64 + c0, h);
+  store8(lo + row * 64 + c0, l);
+  if (norm) {
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+    if ((t & 7) == 0) norm[row] = sqrtf(ss) * 1.000001f;
+  }
+}
+
+}  // namespace tc
+
+cudaError_t init_kmeans_tc() {
+  return cudaFuncSetAttribute(tc::k_kmeans_assign_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kKmSmemBytes);
+}
+bool kmeans_tc_supported() { return tc::tma_available(); }
+
+void launch_split_bf16(const float* x, int ld, i64 rows, int r, __nv_bfloat16* hi, __nv_bfloat16* lo, float* norm,
+                       cudaStream_t st) {
+  tc::k_split_bf16<<<(unsigned)((rows * 8 + 255) / 256), 256, 0, st>>>(x, ld, rows, r, hi, lo, norm);
+}
+
+// One assignment pass.  xh/xl: bf16 [BH][N][64]; mh/ml: bf16 [BH][C][64]; sums may be null (no update wanted).
+bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
+  using namespace tc;
+  CUtensorMap mxh, mxl, mmh, mml;
+  if (!make_map(&mxh, a.xh, 64, a.N, a.BH, 1, 0, (i64)a.N * 64, 64, 128) || !make_map(&mxl, a.xl, 64, a.N, a.BH, 1, 0, (i64)a.N * 64, 64, 128) ||
+      !make_map(&mmh, a.mh, 64, a.C, a.BH, 1, 0, (i64)a.C * 64, 64, kKmChunk) || !make_map(&mml, a.ml, 64, a.C, a.BH, 1, 0, (i64)a.C * 64, 64, kKmChunk))
+    return false;
+  KmParams p{};
+  p.N = a.N; p.C = a.C; p.r = a.r; p.R = a.R; p.n_chunks = (a.C + kKmChunk - 1) / kKmChunk;
+  const int row_tiles = (a.N + 127) / 128;
+  p.ctas_per_head = std::max(1, std::min(row_tiles, 148 / a.BH));
+  p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.mumax = a.mumax; p.assign = a.assign;
+  p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
+  cudaMemsetAsync(a.flag_count, 0, sizeof(int), st);
+  k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
+  k_assign_recheck<<<148 * 2, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
+                                            a.counts, a.fx_shift, a.recheck_total);
+  return true;
+}
+
+}  // namespace spr

@@ -115,15 +115,152 @@ void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d
 
 // =============================================================================
 // Batched symmetric eigen-decomposition by parallel cyclic Jacobi, one CTA per
-// matrix (n = 64 or 128).  A lives in shared memory in float64, the accumulated
-// rotations V in float32.  Every round rotates n/2 disjoint (p,q) pairs; because
-// the rotation matrix is block diagonal in that pairing, each 2x2 block of A is
-// updated in place from its own four entries: A'_ij = J_i^T A_ij J_j.
-// Output: the leading r eigenvectors, scaled by sqrt(lambda_i / mean retained lambda)
-// (the feature map F of Section 4.1) or unscaled (orthonormal basis Psi_r, Eq. 9).
+// matrix (n = 64 or 128), float32, register resident.
+//   threads [0,n)  : thread i holds row i of A in registers
+//   threads [n,2n) : thread n+i holds row i of V (accumulated rotations)
+// The round-robin tournament is realised by MOVING rows and columns so that the
+// pairs of a round are always the adjacent positions (2k, 2k+1): a row rotation
+// is then a shuffle between neighbouring lanes, a column rotation touches two
+// adjacent registers, and the permutation between rounds is a compile-time
+// renaming of registers for the columns and one trip through shared memory for
+// the rows of A.  Output: the leading r eigenvectors, scaled by
+// sqrt(lambda_i / mean retained lambda) (the feature map F of Section 4.1) or
+// unscaled (the orthonormal basis Psi_r of Eq. 9).
 // =============================================================================
+__host__ __device__ constexpr int rr_next(int pos, int n) {
+  // where the content of position `pos` goes for the next round (position 0 is fixed; the even
+  // positions shift up, the last one turns around, the odd positions shift down)
+  return pos == 0 ? 0 : pos == 1 ? 2 : (pos % 2 == 0) ? (pos / 2 < n / 2 - 1 ? pos + 2 : n - 1) : pos - 2;
+}
+
 template <int NN>
-__global__ void __launch_bounds__(1024) k_jacobi_eig(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+__global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+                                                      float* __restrict__ Fout, double* __restrict__ lam_out) {
+  constexpr int LD = NN + 4;
+  extern __shared__ __align__(16) float sm_j[];
+  float* rows = sm_j;                                   // [NN][LD] rows of A in the current position order
+  float2* cs = reinterpret_cast<float2*>(rows + NN * LD);   // [NN/2] rotation of every pair
+  __shared__ float red[34];
+  __shared__ int s_rank[NN];
+  const int tid = threadIdx.x;
+  const bool is_a = tid < NN;
+  const int i = is_a ? tid : tid - NN;
+  const double* Mi = Min + (i64)blockIdx.x * stride;
+  float a[NN];                                          // row i of A (A threads) or of V (V threads)
+  if (is_a) {
+#pragma unroll
+    for (int c = 0; c < NN; ++c) a[c] = (float)(0.5 * (Mi[(i64)i * NN + c] + Mi[(i64)c * NN + i]));
+#pragma unroll
+    for (int c = 0; c < NN; c += 4) *reinterpret_cast<float4*>(rows + i * LD + c) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
+  } else {
+#pragma unroll
+    for (int c = 0; c < NN; ++c) a[c] = c == i ? 1.f : 0.f;
+  }
+  float fro = 0.f;
+  if (is_a) {
+#pragma unroll
+    for (int c = 0; c < NN; ++c) fro = fmaf(a[c], a[c], fro);
+  }
+  fro = block_sum(fro, red);                            // contains __syncthreads: rows[] is complete
+  // float32 rounding leaves an off-diagonal floor near 5e-13 of the squared norm: stop there,
+  // or as soon as a sweep no longer halves the off-diagonal mass
+  const float tol = fro * 4e-12f;
+  float prev_off = 3.0e38f;
+  for (int sweep = 0; sweep < 16; ++sweep) {
+    float off = 0.f;
+    if (is_a) {
+#pragma unroll
+      for (int c = 0; c < NN; ++c) off = fmaf(a[c], a[c], off);
+      const float dg = rows[i * LD + i];
+      off -= dg * dg;
+    }
+    off = block_sum(off, red);
+    if (!(off > tol) || (sweep >= 4 && off > 0.5f * prev_off)) break;
+    prev_off = off;
+    for (int round = 0; round < NN - 1; ++round) {
+      const int p = i & ~1;                             // pair (p, p+1)
+      const float app = rows[p * LD + p], apq = rows[p * LD + p + 1], aqq = rows[(p + 1) * LD + p + 1];
+      float c = 1.f, s = 0.f;
+      if (apq != 0.f) {
+        const float tau = (aqq - app) / (2.f * apq);
+        const float t = copysignf(1.f, tau) / (fabsf(tau) + sqrtf(fmaf(tau, tau, 1.f)));   // -> 0 when tau overflows
+        c = rsqrtf(fmaf(t, t, 1.f));
+        s = t * c;
+      }
+      if (is_a && !(i & 1)) cs[i >> 1] = make_float2(c, s);
+      __syncthreads();                                  // all reads of rows[] done, cs[] visible
+      if (is_a) {
+        // rows: (a_p, a_q) <- (c a_p - s a_q, s a_p + c a_q); the partner row lives in the neighbouring lane
+        const float ss = (i & 1) ? s : -s;
+#pragma unroll
+        for (int col = 0; col < NN; ++col) {
+          const float b = __shfl_xor_sync(0xffffffffu, a[col], 1);
+          a[col] = fmaf(ss, b, c * a[col]);
+        }
+      }
+      // columns (A and V alike): (x_p, x_q) <- (c x_p - s x_q, s x_p + c x_q), then move to the next round's positions
+      float nx[NN];
+#pragma unroll
+      for (int k = 0; k < NN / 2; ++k) {
+        const float2 r2 = cs[k];
+        const float x = a[2 * k], y = a[2 * k + 1];
+        nx[rr_next(2 * k, NN)] = r2.x * x - r2.y * y;
+        nx[rr_next(2 * k + 1, NN)] = fmaf(r2.y, x, r2.x * y);
+      }
+#pragma unroll
+      for (int col = 0; col < NN; ++col) a[col] = nx[col];
+      if (is_a) {
+        const int dst = rr_next(i, NN);                 // the row moves as well
+#pragma unroll
+        for (int col = 0; col < NN; col += 4)
+          *reinterpret_cast<float4*>(rows + dst * LD + col) = make_float4(a[col], a[col + 1], a[col + 2], a[col + 3]);
+      }
+      __syncthreads();
+      if (is_a) {
+#pragma unroll
+        for (int col = 0; col < NN; col += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(rows + i * LD + col);
+          a[col] = v.x; a[col + 1] = v.y; a[col + 2] = v.z; a[col + 3] = v.w;
+        }
+      }
+    }
+  }
+  // eigenvalue of position c = A[c][c]; eigenvector = column c of V.  Rank descending (ties by position).
+  __syncthreads();
+  float lam_i = 0.f;
+  if (is_a) lam_i = rows[i * LD + i];
+  __syncthreads();
+  float* lam_s = reinterpret_cast<float*>(cs);          // NN floats fit in the NN/2 float2 slots
+  if (is_a) lam_s[i] = lam_i;
+  __syncthreads();
+  if (is_a) {
+    int rank = 0;
+    for (int j = 0; j < NN; ++j) { const float lj = lam_s[j]; rank += (lj > lam_i) || (lj == lam_i && j < i); }
+    s_rank[i] = rank;
+    if (lam_out) lam_out[(i64)blockIdx.x * NN + rank] = (double)lam_i;
+  } else {
+#pragma unroll
+    for (int c = 0; c < NN; c += 4) *reinterpret_cast<float4*>(rows + i * LD + c) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
+  }
+  __syncthreads();
+  float part = (is_a && s_rank[i] < r) ? fmaxf(lam_i, 0.f) : 0.f;
+  const float mean = block_sum(part, red) / (float)r;
+  for (int e = tid; e < NN * NN; e += 2 * NN) {
+    const int row = e / NN, col = e % NN;
+    const int rank = s_rank[col];
+    if (rank < r) {
+      float sc = 1.f;
+      if (scale_mode == 0) sc = mean > 0.f ? sqrtf(fmaxf(lam_s[col], 0.f) / mean) : 0.f;
+      Fout[(i64)blockIdx.x * NN * r + (i64)row * r + rank] = rows[row * LD + col] * sc;
+    }
+  }
+}
+
+// Float64 variant (A in shared memory, one CTA per matrix, in-place 2x2 block updates):
+// slower, used when the caller's tensors are float32 and the 1e-5 output tolerance
+// leaves no room for a float32 eigen-basis.
+template <int NN>
+__global__ void __launch_bounds__(1024) k_jacobi_eig_f64(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
                                                     float* __restrict__ Fout, double* __restrict__ lam_out) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* A = reinterpret_cast<double*>(smem_raw);                 // [NN][NN+1]
@@ -220,18 +357,28 @@ __global__ void __launch_bounds__(1024) k_jacobi_eig(const double* __restrict__ 
   }
 }
 
-static size_t jacobi_smem(int n) {
+static size_t jacobi64_smem(int n) {
   return (size_t)n * (n + 1) * 8 + (size_t)(n * (n + 1) + (n & 1)) * 4 + n * 8 + n * 4 + 34 * 8 + 16;
 }
+static size_t jacobi_smem(int n) { return (size_t)n * (n + 4) * 4 + (size_t)n * 4 + 16; }
 cudaError_t init_jacobi() {
   cudaError_t e = cudaFuncSetAttribute(k_jacobi_eig<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(128));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_jacobi_eig<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(64));
+  e = cudaFuncSetAttribute(k_jacobi_eig<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(64));
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_jacobi_eig_f64<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(128));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_jacobi_eig_f64<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(64));
 }
-void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout,
+void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
                        double* lam_out, cudaStream_t st) {
-  if (n == 128) k_jacobi_eig<128><<<batch, 1024, jacobi_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
-  else k_jacobi_eig<64><<<batch, 1024, jacobi_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  if (precise) {
+    if (n == 128) k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    else k_jacobi_eig_f64<64><<<batch, 1024, jacobi64_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  } else {
+    if (n == 128) k_jacobi_eig<128><<<batch, 256, jacobi_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    else k_jacobi_eig<64><<<batch, 128, jacobi_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  }
 }
 
 // =============================================================================
