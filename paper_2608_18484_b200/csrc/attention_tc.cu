@@ -38,8 +38,8 @@ struct Smem {                          // offsets from a 1024-byte aligned base
   static constexpr uint32_t v = k + kStages * kTileBytes;
   static constexpr uint32_t p = v + kStages * kTileBytes;
   static constexpr uint32_t ranges = p + kTileBytes;              // int2[kMaxGroups]: (start row, length)
-  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;       // float[2][128]
-  static constexpr uint32_t meta = xchg + 2 * 128 * 4;            // uint2[4]
+  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;       // float[2][2][128]
+  static constexpr uint32_t meta = xchg + 4 * 128 * 4;            // uint2[4]
   static constexpr uint32_t bars = meta + 4 * 8;                  // 20 mbarriers
   static constexpr uint32_t misc = bars + 20 * 8;                 // tmem base, abort flag, counters
   static constexpr uint32_t total = misc + 64;
@@ -127,7 +127,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       mbar_init(bar(V_FULL + s), 1); mbar_init(bar(V_EMPTY + s), 1);
       mbar_init(bar(S_FULL + s), 1);
     }
-    mbar_init(bar(P_FULL), 256); mbar_init(bar(T_FULL), 1); mbar_init(bar(T_EMPTY), 256); mbar_init(bar(C_FULL), 1);
+    mbar_init(bar(P_FULL), 256); mbar_init(bar(T_FULL), 1); mbar_init(bar(T_EMPTY), 1); mbar_init(bar(C_FULL), 1);
     for (int s = 0; s < 4; ++s) mbar_init(bar(META_FULL + s), 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -239,15 +239,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int s = i % kStages;
         const uint2 mt = meta[i & 3];
         if (!mbar_wait(bar(V_FULL + s), (i / kStages) & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }
-        if (i >= 1 && !mbar_wait(bar(T_EMPTY), (i - 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }   // P(i) stored, O rescaled if needed
         tc_fence_after();
         const uint32_t d = tmem + 256u;
         const int nsub = (int)mt.y;
         for (int kk = 0; kk < nsub; ++kk) {
           const uint64_t a = smem_desc(base + Smem::p + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16);
           const uint64_t bdesc = smem_desc(base + Smem::v + s * kTileBytes + kk * kSubBytes, kHalfBytes);
-          umma_bf16(d, a, bdesc, idesc_pv, kk > 0);
+          umma_bf16(d, a, bdesc, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);          // O accumulates over all tiles
         }
         umma_commit(bar(V_EMPTY + s));
         umma_commit(bar(T_FULL));
@@ -266,17 +265,19 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
     }
   } else {
-    // =========================== softmax / accumulate (warps 0-7) =========================
+    // =========================== softmax (warps 0-7) =======================================
+    // Two threads per query row (64 score columns each).  The output accumulator O stays in
+    // TMEM for the whole key stream: P V products accumulate into it, and it is rescaled only
+    // when the running row maximum has grown by more than 2^8 since the reference maximum
+    // m_ref was fixed (the exponentials then stay below 2^8 and nothing overflows); the final
+    // normalisation by the row sum removes the stale factor exactly.
     // Control flow stays uniform inside a warp (`ok` is voted) and the pair barriers are executed
     // by both warps of a row quad whatever happened, so a timed-out wait cannot strand a partner.
     const int wq = warp & 3, half = warp >> 2;
     const int row = wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t FULL = 0xffffffffu;
-    float o[64];
-#pragma unroll
-    for (int c = 0; c < 64; ++c) o[c] = 0.f;
-    float m = -INFINITY, l = 0.f;
+    float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
     for (int i = 0; i < n_tiles; ++i) {
@@ -311,40 +312,44 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < 64; ++c) s[c] = 0.f;
       }
-      xchg[half * 128 + row] = mx;
+      float* xb = xchg + (i & 1) * 256;                                    // double buffered: one pair barrier per tile
+      xb[half * 128 + row] = mx;
       asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");           // the two warps that share these rows
-      mx = fmaxf(mx, xchg[(half ^ 1) * 128 + row]);
-      const float m_new = fmaxf(m, mx);
-      const float corr = ex2((m - m_new) * sc);                            // 0 on the first tile
+      mx = fmaxf(mx, xb[(half ^ 1) * 128 + row]);
+      // reference maximum: moved only when the tile maximum exceeds it by more than 8 (log2 units)
+      const bool move = (mx - m_ref) * sc > 8.f;                           // true on the first tile (m_ref = -inf)
+      const float m_new = move ? mx : m_ref;
+      const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f;           // 0 on the first tile
       const float mneg = -m_new * sc;
-      m = m_new;
+      m_ref = m_new;
       float psum = 0.f;
 #pragma unroll
       for (int c = 0; c < 64; ++c) { s[c] = ex2(fmaf(s[c], sc, mneg)); psum += s[c]; }
       l = l * corr + psum;
-      // the P buffer is free once the previous P V product has completed
+      // P buffer and O are free once the previous P V product has completed
       if (i >= 1) ok = __all_sync(FULL, ok && mbar_wait(bar(T_FULL), (i - 1) & 1, abort_flag));
       if (ok) {
         tc_fence_after();
+        if (i >= 1 && __any_sync(FULL, move)) {                            // rescale this warp's O rows (rare)
+#pragma unroll
+          for (int hblk = 0; hblk < 2; ++hblk) {
+            float t[32];
+            tmem_ld32(tmem + lane_addr + 256u + half * 64 + hblk * 32, t);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) t[c] *= corr;
+            tmem_st32(tmem + lane_addr + 256u + half * 64 + hblk * 32, t);
+          }
+        }
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) store_p_chunk(base + Smem::p, row, half * 8 + ch, &s[ch * 8]);
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(bar(P_FULL));
-        if (i >= 1) {
-          float t[32];
-          tmem_ld32(tmem + lane_addr + 256u + half * 64, t);
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = (o[c] + t[c]) * corr;
-          tmem_ld32(tmem + lane_addr + 256u + half * 64 + 32, t);
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[32 + c] = (o[32 + c] + t[c]) * corr;
-          tc_fence_before();
-          mbar_arrive(bar(T_EMPTY));
-        }
       }
-      asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");           // xchg may be overwritten by the next tile
     }
+    float o[64];
+#pragma unroll
+    for (int c = 0; c < 64; ++c) o[c] = 0.f;
     if (n_tiles > 0) {
       ok = __all_sync(FULL, ok && mbar_wait(bar(T_FULL), (n_tiles - 1) & 1, abort_flag));
       if (ok) {
@@ -352,16 +357,17 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         float t[32];
         tmem_ld32(tmem + lane_addr + 256u + half * 64, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[c] += t[c];
+        for (int c = 0; c < 32; ++c) o[c] = t[c];
         tmem_ld32(tmem + lane_addr + 256u + half * 64 + 32, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[32 + c] += t[c];
+        for (int c = 0; c < 32; ++c) o[32 + c] = t[c];
       }
     }
     // total row sum from both halves
-    xchg[half * 128 + row] = l;
+    float* xe = xchg + (n_tiles & 1) * 256;
+    xe[half * 128 + row] = l;
     asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
-    const float ltot = l + xchg[(half ^ 1) * 128 + row];
+    const float ltot = l + xe[(half ^ 1) * 128 + row];
     const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
 #pragma unroll
     for (int c = 0; c < 64; ++c) o[c] *= inv;
