@@ -2,16 +2,20 @@
 //
 // One CTA processes one 128-row query tile (of one query group, Eq. 3; or of the whole
 // head for dense attention, Eq. 1).  Roles:
-//   warps 0-7  softmax: two threads per query row (64 score columns each)
+//   warps 0-3  softmax group A: even key tiles, one thread per query row
+//   warps 4-7  softmax group B: odd key tiles
 //   warp  8    TMA producer: streams the routed keys/values as one concatenated
 //              sequence in 16-row boxes (tiles of 128 keys, only range ends are ragged)
 //   warp  9    tcgen05.mma issuer; owns the TMEM allocation
-// Data path per key tile i:
-//   S_i = Q K_i^T      tcgen05.mma (smem x smem -> TMEM, fp32), two S buffers
-//   P_i = exp2(.)      softmax threads: tcgen05.ld S, running max / sum, bf16 P -> smem
-//   T_i = P_i V_i      tcgen05.mma -> TMEM, accumulated into registers o = (o + T_{i-1}) * corr_i
-// Epilogue: O_sp = o / l; correction O_sp A on the tensor cores (A = composed affine map
-// of Eq. 9, bf16), + c, store at the original token index (inverse permutation).
+// Data path per key tile i (group g = i mod 2):
+//   S_g = Q K_i^T        tcgen05.mma, smem x smem -> TMEM (fp32)
+//   P   = exp2(.)        softmax thread: tcgen05.ld S_g, reference max / row sum, bf16 P written
+//                        back over the first half of S_g with tcgen05.st
+//   O_g += P V_i         tcgen05.mma with the A operand read from TMEM; O_g stays in TMEM
+// While group A works on tile i the tensor cores already produce S_B for tile i+1.
+// Epilogue: merge (O_A, O_B) like two splits of the key range, O_sp = O / l; correction
+// O_sp A on the tensor cores (A = composed affine map of Eq. 9, bf16), + c, store at the
+// original token index (inverse permutation).
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
@@ -22,7 +26,7 @@ namespace spr {
 
 namespace tc {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kTile = 128;            // query rows per CTA, keys per tile
 constexpr int kD = 128;
 constexpr int kSub = 16;              // rows per TMA box of the K/V stream
@@ -30,25 +34,32 @@ constexpr int kSubPerTile = kTile / kSub;
 constexpr uint32_t kHalfBytes = kTile * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr uint32_t kSubBytes = kSub * 128;            // 2 KB per box
-constexpr int kStages = 2;
+#ifndef SPR_K_STAGES
+#define SPR_K_STAGES 3
+#endif
+#ifndef SPR_V_STAGES
+#define SPR_V_STAGES 2
+#endif
+constexpr int kKStages = SPR_K_STAGES;  // K tiles in flight (consumed by Q K^T)
+constexpr int kVStages = SPR_V_STAGES;  // V tiles in flight (consumed by P V)
 
 struct Smem {                          // offsets from a 1024-byte aligned base
   static constexpr uint32_t q = 0;
-  static constexpr uint32_t k = q + kTileBytes;                   // kStages tiles
-  static constexpr uint32_t v = k + kStages * kTileBytes;
-  static constexpr uint32_t p = v + kStages * kTileBytes;
-  static constexpr uint32_t ranges = p + kTileBytes;              // int2[kMaxGroups]: (start row, length)
-  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;       // float[2][2][128]
-  static constexpr uint32_t meta = xchg + 4 * 128 * 4;            // uint2[4]
-  static constexpr uint32_t bars = meta + 4 * 8;                  // 20 mbarriers
-  static constexpr uint32_t misc = bars + 20 * 8;                 // tmem base, abort flag, counters
+  static constexpr uint32_t k = q + kTileBytes;
+  static constexpr uint32_t v = k + kKStages * kTileBytes;
+  static constexpr uint32_t ranges = v + kVStages * kTileBytes;
+  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;     // float2[2][128]
+  static constexpr uint32_t meta = xchg + 2 * 128 * 8;            // uint2[8]: ring of per-tile box counts
+  static constexpr uint32_t bars = meta + 8 * 8;                  // kNumBars mbarriers
+  static constexpr uint32_t misc = bars + 32 * 8;                 // tmem base, abort flag, counters
   static constexpr uint32_t total = misc + 64;
 };
-constexpr size_t kSmemBytes = Smem::total + 1024;                 // slack for manual alignment
+constexpr size_t kSmemBytes = Smem::total;                        // the dynamic segment is 1024-byte aligned and the only shared memory
 
-enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, P_FULL = 11, T_FULL = 12,
-           T_EMPTY = 13, C_FULL = 14, META_FULL = 15 };
-
+enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kKStages, V_FULL = K_EMPTY + kKStages, V_EMPTY = V_FULL + kVStages,
+           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, C_FULL, X_FULL, X_DONE, META_FULL,
+           kNumBars = META_FULL + 8 };
+static_assert(kNumBars <= 32, "barrier area");
 
 struct Params {
   int BH, H, N, Cq, Ck, sparse;
@@ -61,28 +72,19 @@ struct Params {
   int* err;
 };
 
-// write 8 consecutive bf16 (one 16-byte chunk) of row `row`, chunk index `chunk` (0..15 over 128 columns)
-__device__ __forceinline__ void store_p_chunk(uint32_t p_base, int row, int chunk, const float* v8) {
-  const uint32_t half = chunk >> 3, c = chunk & 7;
-  const uint32_t addr = p_base + half * kHalfBytes + row * 128 + ((c ^ (row & 7)) << 4);
-  uint32_t w[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(v8[2 * i], v8[2 * i + 1]);
-    w[i] = *reinterpret_cast<uint32_t*>(&h);
-  }
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapA, Params prm) {
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  unsigned char* sm = smem_raw + (base - raw);
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* sm = smem_raw;
   int2* ranges = reinterpret_cast<int2*>(sm + Smem::ranges);
-  float* xchg = reinterpret_cast<float*>(sm + Smem::xchg);
+  float2* stat = reinterpret_cast<float2*>(sm + Smem::xchg);               // [2][128] (m_ref, l) of both groups
   uint2* meta = reinterpret_cast<uint2*>(sm + Smem::meta);
   volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem base, [1] abort, [2] total boxes
   const uint32_t bars = base + Smem::bars;
@@ -91,10 +93,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y, b = bh / prm.H, h = bh % prm.H;
   // once any CTA has recorded a timeout the remaining CTAs of the launch leave at once
-  __shared__ int s_skip;
-  if (tid == 0) s_skip = prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT;
+  // (also if the shared-memory base is not aligned as the swizzled tiles require)
+  if (tid == 0) {
+    misc[3] = (prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT) || (base & 1023u) != 0;
+    if ((base & 1023u) != 0) set_error(prm.err, SPARSEPR_ERR_CUDA);
+  }
   __syncthreads();
-  if (s_skip) return;
+  if (misc[3]) return;
 
   // ---- which query tile ---------------------------------------------------------------
   int row0, nrows, nroute;
@@ -121,14 +126,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar(Q_FULL), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar(K_FULL + s), 1); mbar_init(bar(K_EMPTY + s), 1);
-      mbar_init(bar(V_FULL + s), 1); mbar_init(bar(V_EMPTY + s), 1);
-      mbar_init(bar(S_FULL + s), 1);
-    }
-    mbar_init(bar(P_FULL), 256); mbar_init(bar(T_FULL), 1); mbar_init(bar(T_EMPTY), 1); mbar_init(bar(C_FULL), 1);
-    for (int s = 0; s < 4; ++s) mbar_init(bar(META_FULL + s), 1);
+    for (int i = 0; i < kNumBars; ++i)
+      mbar_init(bar(i), (i == P_FULL || i == P_FULL + 1) ? 128 : i == X_FULL ? 256 : 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -153,59 +152,73 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int n_tiles = (total_boxes + kSubPerTile - 1) / kSubPerTile;
   volatile int* abort_flag = &misc[1];
 
-  if (warp == 8) {
-    // =========================== TMA producer ===========================================
-    if (lane == 0 && n_tiles > 0) {
-      mbar_expect_tx(bar(Q_FULL), kTileBytes);
-      tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, prm.sparse ? bh : h, prm.sparse ? 0 : b);
-      tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, prm.sparse ? bh : h, prm.sparse ? 0 : b);
+  if (warp == 8 || warp == 10) {
+    // =========================== TMA producers ==========================================
+    // warp 8 streams Q and the key tiles, warp 10 the value tiles.  All lanes of a producer walk
+    // the concatenated key ranges together (uniform); lane j issues the copies of box j.
+    if (n_tiles > 0) {
+      const bool is_k = warp == 8;
       const int c2 = prm.sparse ? bh : h, c3 = prm.sparse ? 0 : b;
-      int ri = 0, off = 0;                       // walk state shared by the K and the V stream of a tile
-      for (int i = 0; i < n_tiles; ++i) {
-        const int s = i % kStages;
-        const uint32_t ph = ((i / kStages) & 1) ^ 1;         // empty barriers: first pass completes immediately
-        // box list of this tile
-        int starts[kSubPerTile];
+      if (is_k && lane == 0) {
+        mbar_expect_tx(bar(Q_FULL), kTileBytes);
+        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, c2, c3);
+        tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, c2, c3);
+      }
+      const int nst = is_k ? kKStages : kVStages;
+      const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
+      const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
+      const CUtensorMap* map = is_k ? &mapK : &mapV;
+      // key ranges (start row, length) of 32 consecutive routes live in the lanes' registers; the next
+      // 32 are prefetched while the current ones are consumed
+      auto load_range = [&](int t) -> int2 {
+        if (t >= nroute) return make_int2(0, 0);
+        if (!prm.sparse) return make_int2(0, prm.N);
+        const int g = ridx[t];
+        const int st = kvoff[g];
+        return make_int2(st, kvoff[g + 1] - st);
+      };
+      int ri = 0, off = 0;
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int s = i % nst;
+        const uint32_t ph = ((i / nst) & 1) ^ 1;             // empty barriers: the first pass completes immediately
+        int my_start = 0;
         uint32_t cnt_bits = 0;
-        int nsub = 0, ri2 = ri, off2 = off;
+        int nsub = 0;
 #pragma unroll
         for (int j = 0; j < kSubPerTile; ++j) {
-          starts[j] = 0;
-          if (ri2 < nroute) {
-            const int2 rg = ranges[ri2];
-            starts[j] = rg.x + off2;
-            const int cnt = min(kSub, rg.y - off2);
+          if (ri < nroute) {
+            const int2 rg = ranges[ri];
+            if (j == lane) my_start = rg.x + off;
+            const int cnt = min(kSub, rg.y - off);
             cnt_bits |= (uint32_t)(cnt - 1) << (4 * j);
             nsub = j + 1;
-            off2 += kSub;
-            if (off2 >= rg.y) { ++ri2; off2 = 0; }
+            off += kSub;
+            if (off >= rg.y) {
+              ++ri; off = 0;
+            }
           }
         }
-        ri = ri2; off = off2;
-        if (!mbar_wait(bar(K_EMPTY + s), ph, abort_flag)) break;
-        meta[i & 3] = make_uint2(cnt_bits, (uint32_t)nsub);
-        mbar_arrive(bar(META_FULL + (i & 3)));
-        mbar_expect_tx(bar(K_FULL + s), nsub * 2 * kSubBytes);
-#pragma unroll
-        for (int j = 0; j < kSubPerTile; ++j)
-          if (j < nsub) {
-            const uint32_t dst = base + Smem::k + s * kTileBytes + j * kSubBytes;
-            tma_load_4d(dst, &mapK, bar(K_FULL + s), 0, starts[j], c2, c3);
-            tma_load_4d(dst + kHalfBytes, &mapK, bar(K_FULL + s), 64, starts[j], c2, c3);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(empty0 + s), ph, abort_flag));
+        if (!ok) break;
+        if (lane == 0) {
+          if (is_k) {
+            // the key producer runs at most four tiles ahead of the last reader of meta[i]: ring of 8
+            meta[i & 7] = make_uint2(cnt_bits, (uint32_t)nsub);
+            mbar_arrive(bar(META_FULL + (i & 7)));
           }
-        if (!mbar_wait(bar(V_EMPTY + s), ph, abort_flag)) break;
-        mbar_expect_tx(bar(V_FULL + s), nsub * 2 * kSubBytes);
-#pragma unroll
-        for (int j = 0; j < kSubPerTile; ++j)
-          if (j < nsub) {
-            const uint32_t dst = base + Smem::v + s * kTileBytes + j * kSubBytes;
-            tma_load_4d(dst, &mapV, bar(V_FULL + s), 0, starts[j], c2, c3);
-            tma_load_4d(dst + kHalfBytes, &mapV, bar(V_FULL + s), 64, starts[j], c2, c3);
-          }
+          mbar_expect_tx(bar(full0 + s), nsub * 2 * kSubBytes);
+        }
+        __syncwarp();
+        if (lane < nsub) {
+          const uint32_t dst = buf0 + s * kTileBytes + lane * kSubBytes;
+          tma_load_4d(dst, map, bar(full0 + s), 0, my_start, c2, c3);
+          tma_load_4d(dst + kHalfBytes, map, bar(full0 + s), 64, my_start, c2, c3);
+        }
       }
-      if (prm.has_corr && !*abort_flag) {
-        // the composed correction matrix (transposed, bf16) goes into K stage 0 once every QK^T is done
-        const int uses0 = (n_tiles + kStages - 1) / kStages;       // completed phases of K_EMPTY[0]
+      if (is_k && lane == 0 && prm.has_corr && !*abort_flag) {
+        // the composed correction matrix (transposed, bf16) goes into K stage 0 once every QK^T that used it is done
+        const int uses0 = (n_tiles + kKStages - 1) / kKStages;
         if (mbar_wait(bar(K_EMPTY + 0), (uint32_t)((uses0 - 1) & 1), abort_flag)) {
           mbar_expect_tx(bar(C_FULL), kTileBytes);
           tma_load_4d(base + Smem::k, &mapA, bar(C_FULL), 0, 0, bh, 0);
@@ -215,13 +228,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
   } else if (warp == 9) {
     // =========================== MMA issuer ==============================================
+    // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,384), O_B [384,512); P_g overwrites S_g[0,64)
     if (lane == 0 && n_tiles > 0) {
       const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
       auto issue_qk = [&](int i) -> bool {
-        const int s = i % kStages;
-        if (!mbar_wait(bar(K_FULL + s), (i / kStages) & 1, abort_flag)) return false;
-        // S buffer i&1 was last read by softmax(i-2); the P_FULL wait of P V (i-2) below already covers that
+        const int s = i % kKStages;
+        if (!mbar_wait(bar(K_FULL + s), (i / kKStages) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
 #pragma unroll
@@ -234,176 +247,178 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         return true;
       };
       if (ok) ok = issue_qk(0);
+      if (ok && n_tiles > 1) ok = issue_qk(1);
       for (int i = 0; i < n_tiles && ok; ++i) {
-        if (i + 1 < n_tiles) { ok = issue_qk(i + 1); if (!ok) break; }
-        const int s = i % kStages;
-        const uint2 mt = meta[i & 3];
-        if (!mbar_wait(bar(V_FULL + s), (i / kStages) & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }   // P(i) stored, O rescaled if needed
+        const int g = i & 1, j = i >> 1, s = i % kVStages;
+        const uint2 mt = meta[i & 7];
+        if (!mbar_wait(bar(V_FULL + s), (i / kVStages) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar(P_FULL + g), j & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, O_g rescaled if needed
         tc_fence_after();
-        const uint32_t d = tmem + 256u;
+        const uint32_t d = tmem + 256u + (uint32_t)g * 128u;
+        const uint32_t pa = tmem + (uint32_t)g * 128u;
         const int nsub = (int)mt.y;
         for (int kk = 0; kk < nsub; ++kk) {
-          const uint64_t a = smem_desc(base + Smem::p + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16);
           const uint64_t bdesc = smem_desc(base + Smem::v + s * kTileBytes + kk * kSubBytes, kHalfBytes);
-          umma_bf16(d, a, bdesc, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);          // O accumulates over all tiles
+          umma_bf16_ts(d, pa + kk * 8, bdesc, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);   // O_g accumulates over its tiles
         }
         umma_commit(bar(V_EMPTY + s));
-        umma_commit(bar(T_FULL));
+        if (i + 2 < n_tiles) ok = issue_qk(i + 2);          // S_g (and the P_g inside it) is rewritten after P V (i)
       }
+      if (ok) umma_commit(bar(O_DONE));
       if (ok && prm.has_corr) {
-        // correction product: bf16(O_sp) (in the P buffer) times A (in K stage 0) -> S buffer 0
-        if (mbar_wait(bar(C_FULL), 0, abort_flag) && mbar_wait(bar(P_FULL), n_tiles & 1, abort_flag)) {
+        // correction product: bf16(O_sp) in TMEM [0,64) times A (in K stage 0) -> TMEM [128,256)
+        if (mbar_wait(bar(C_FULL), 0, abort_flag) && mbar_wait(bar(X_FULL), 0, abort_flag)) {
           tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < kD / 16; ++kk) {
             const uint32_t koff = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            umma_bf16(tmem, smem_desc(base + Smem::p + koff, 16), smem_desc(base + Smem::k + koff, 16), idesc_qk, kk > 0);
+            umma_bf16_ts(tmem + 128u, tmem + kk * 8, smem_desc(base + Smem::k + koff, 16), idesc_qk, kk > 0);
           }
-          umma_commit(bar(S_FULL + 0));
+          umma_commit(bar(X_DONE));
         }
       }
     }
   } else {
     // =========================== softmax (warps 0-7) =======================================
-    // Two threads per query row (64 score columns each).  The output accumulator O stays in
-    // TMEM for the whole key stream: P V products accumulate into it, and it is rescaled only
-    // when the running row maximum has grown by more than 2^8 since the reference maximum
-    // m_ref was fixed (the exponentials then stay below 2^8 and nothing overflows); the final
-    // normalisation by the row sum removes the stale factor exactly.
-    // Control flow stays uniform inside a warp (`ok` is voted) and the pair barriers are executed
-    // by both warps of a row quad whatever happened, so a timed-out wait cannot strand a partner.
-    const int wq = warp & 3, half = warp >> 2;
+    // Group A (warps 0-3) takes the even key tiles, group B (warps 4-7) the odd ones; one thread
+    // per query row and tile (128 scores).  Each group has its own score buffer, its own output
+    // accumulator O_g in TMEM and its own running (m_ref, l); the two partial results are merged
+    // at the end like two splits of the key range.  O_g is rescaled only when the row maximum has
+    // grown by more than 2^8 over the reference maximum, so exponentials stay below 2^8.
+    const int g = warp >> 2, wq = warp & 3;
     const int row = wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t FULL = 0xffffffffu;
+    const uint32_t s_addr = tmem + lane_addr + (uint32_t)g * 128u;
+    const uint32_t o_addr = tmem + lane_addr + 256u + (uint32_t)g * 128u;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
-    for (int i = 0; i < n_tiles; ++i) {
-      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
-                                mbar_wait(bar(META_FULL + (i & 3)), (i >> 2) & 1, abort_flag));
-      float s[64];
-      float mx = -INFINITY;
-      if (ok) {
-        tc_fence_after();
-        const uint2 mt = meta[i & 3];
-        {
-          float t[32];
-          tmem_ld32(tmem + lane_addr + (uint32_t)(i & 1) * 128u + half * 64, t);
+    for (int i = g, j = 0; i < n_tiles; i += 2, ++j) {
+      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + g), j & 1, abort_flag) &&
+                                mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
+      if (!ok) continue;                                         // warp-uniform
+      tc_fence_after();
+      const uint2 mt = meta[i & 7];
+      float s[128];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) s[c] = t[c];
-          tmem_ld32(tmem + lane_addr + (uint32_t)(i & 1) * 128u + half * 64 + 32, t);
+      for (int q = 0; q < 4; ++q) {
+        float t[32];
+        tmem_ld32(s_addr + q * 32, t);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) s[32 + c] = t[c];
-        }
-        if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int box = half * 4 + g;
-            const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;    // last valid column of the box
-#pragma unroll
-            for (int c = 0; c < 16; ++c) s[g * 16 + c] = (c <= lim) ? s[g * 16 + c] : -INFINITY;
-          }
-        }
-#pragma unroll
-        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, s[c]);
-      } else {
-#pragma unroll
-        for (int c = 0; c < 64; ++c) s[c] = 0.f;
+        for (int c = 0; c < 32; ++c) s[q * 32 + c] = t[c];
       }
-      float* xb = xchg + (i & 1) * 256;                                    // double buffered: one pair barrier per tile
-      xb[half * 128 + row] = mx;
-      asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");           // the two warps that share these rows
-      mx = fmaxf(mx, xb[(half ^ 1) * 128 + row]);
-      // reference maximum: moved only when the tile maximum exceeds it by more than 8 (log2 units)
-      const bool move = (mx - m_ref) * sc > 8.f;                           // true on the first tile (m_ref = -inf)
+      if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
+#pragma unroll
+        for (int box = 0; box < 8; ++box) {
+          const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;      // last valid column of the box
+#pragma unroll
+          for (int c = 0; c < 16; ++c) s[box * 16 + c] = (c <= lim) ? s[box * 16 + c] : -INFINITY;
+        }
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+        mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+        mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      const bool move = (mx - m_ref) * sc > 8.f;                 // true on the group's first tile (m_ref = -inf)
       const float m_new = move ? mx : m_ref;
-      const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f;           // 0 on the first tile
+      const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f; // 0 on the first tile
       const float mneg = -m_new * sc;
       m_ref = m_new;
-      float psum = 0.f;
+      if (j > 0 && __any_sync(FULL, move)) {                     // rescale this warp's rows of O_g (rare)
 #pragma unroll
-      for (int c = 0; c < 64; ++c) { s[c] = ex2(fmaf(s[c], sc, mneg)); psum += s[c]; }
-      l = l * corr + psum;
-      // P buffer and O are free once the previous P V product has completed
-      if (i >= 1) ok = __all_sync(FULL, ok && mbar_wait(bar(T_FULL), (i - 1) & 1, abort_flag));
-      if (ok) {
-        tc_fence_after();
-        if (i >= 1 && __any_sync(FULL, move)) {                            // rescale this warp's O rows (rare)
+        for (int q = 0; q < 4; ++q) {
+          float t[32];
+          tmem_ld32(o_addr + q * 32, t);
 #pragma unroll
-          for (int hblk = 0; hblk < 2; ++hblk) {
-            float t[32];
-            tmem_ld32(tmem + lane_addr + 256u + half * 64 + hblk * 32, t);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) t[c] *= corr;
-            tmem_st32(tmem + lane_addr + 256u + half * 64 + hblk * 32, t);
-          }
+          for (int c = 0; c < 32; ++c) t[c] *= corr;
+          tmem_st32(o_addr + q * 32, t);
         }
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) store_p_chunk(base + Smem::p, row, half * 8 + ch, &s[ch * 8]);
-        fence_async_smem();
-        tc_fence_before();
-        mbar_arrive(bar(P_FULL));
       }
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+        s[c] = ex2(fmaf(s[c], sc, mneg)); s[c + 1] = ex2(fmaf(s[c + 1], sc, mneg));
+        s[c + 2] = ex2(fmaf(s[c + 2], sc, mneg)); s[c + 3] = ex2(fmaf(s[c + 3], sc, mneg));
+        ps4[0] += s[c]; ps4[1] += s[c + 1]; ps4[2] += s[c + 2]; ps4[3] += s[c + 3];
+      }
+      l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+      // P (bf16, two per 32-bit column) over the first 64 columns of the score buffer
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        uint32_t w[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[q * 64 + 2 * c], s[q * 64 + 2 * c + 1]);
+        tmem_st32u(s_addr + q * 32, w);
+      }
+      tc_fence_before();
+      mbar_arrive(bar(P_FULL + g));
     }
+    // ---- merge the two groups, normalise ------------------------------------------------------
+    if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
+    stat[g * 128 + row] = make_float2(m_ref, l);
+    asm volatile("bar.sync 1, 256;" ::: "memory");               // all softmax threads, whatever happened
+    const float2 sa = stat[row], sb = stat[128 + row];
+    const float mm = fmaxf(sa.x, sb.x);
+    const float wa = sa.y > 0.f ? ex2((sa.x - mm) * sc) : 0.f;
+    const float wb = sb.y > 0.f ? ex2((sb.x - mm) * sc) : 0.f;
+    const float ltot = sa.y * wa + sb.y * wb;
+    const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
+    // this thread finishes output columns [64 g, 64 g + 64) of its row
     float o[64];
 #pragma unroll
     for (int c = 0; c < 64; ++c) o[c] = 0.f;
-    if (n_tiles > 0) {
-      ok = __all_sync(FULL, ok && mbar_wait(bar(T_FULL), (n_tiles - 1) & 1, abort_flag));
-      if (ok) {
-        tc_fence_after();
+    if (ok && n_tiles > 0) {
+      tc_fence_after();
+      const float fa = wa * inv, fb = wb * inv;
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
         float t[32];
-        tmem_ld32(tmem + lane_addr + 256u + half * 64, t);
+        tmem_ld32(tmem + lane_addr + 256u + g * 64 + q * 32, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[c] = t[c];
-        tmem_ld32(tmem + lane_addr + 256u + half * 64 + 32, t);
+        for (int c = 0; c < 32; ++c) o[q * 32 + c] = fa != 0.f ? t[c] * fa : 0.f;
+        if (n_tiles > 1) {                                        // group B exists only then (uniform)
+          tmem_ld32(tmem + lane_addr + 384u + g * 64 + q * 32, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[32 + c] = t[c];
+          for (int c = 0; c < 32; ++c) o[q * 32 + c] += fb != 0.f ? t[c] * fb : 0.f;
+        }
       }
     }
-    // total row sum from both halves
-    float* xe = xchg + (n_tiles & 1) * 256;
-    xe[half * 128 + row] = l;
-    asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
-    const float ltot = l + xe[(half ^ 1) * 128 + row];
-    const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
-#pragma unroll
-    for (int c = 0; c < 64; ++c) o[c] *= inv;
     float res[64];
 #pragma unroll
     for (int c = 0; c < 64; ++c) res[c] = o[c];
     if (prm.has_corr && n_tiles > 0) {
       if (ok) {
+        uint32_t w[32];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) store_p_chunk(base + Smem::p, row, half * 8 + ch, &o[ch * 8]);
-        fence_async_smem();
+        for (int c = 0; c < 32; ++c) w[c] = pack_bf16(o[2 * c], o[2 * c + 1]);
+        tmem_st32u(tmem + lane_addr + g * 32, w);                // bf16(O_sp): columns [0,64) = 128 values
         tc_fence_before();
-        mbar_arrive(bar(P_FULL));
+        mbar_arrive(bar(X_FULL));
       }
-      // S buffer 0 completes once more: its phase index = number of earlier completions
-      const int prev = (n_tiles + 1) / 2;
-      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + 0), prev & 1, abort_flag));
+      ok = __all_sync(FULL, ok && mbar_wait(bar(X_DONE), 0, abort_flag));
       if (ok) {
         tc_fence_after();
-        const float* cv = prm.c + (i64)bh * kD + half * 64;
-        float t[32];
-        tmem_ld32(tmem + lane_addr + half * 64, t);
+        const float* cv = prm.c + (i64)bh * kD + g * 64;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) res[c] = o[c] + t[c] + cv[c];
-        tmem_ld32(tmem + lane_addr + half * 64 + 32, t);
+        for (int q = 0; q < 2; ++q) {
+          float t[32];
+          tmem_ld32(tmem + lane_addr + 128u + g * 64 + q * 32, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) res[32 + c] = o[32 + c] + t[c] + cv[32 + c];
+          for (int c = 0; c < 32; ++c) res[q * 32 + c] = o[q * 32 + c] + t[c] + cv[q * 32 + c];
+        }
       }
     } else if (prm.has_corr) {
-      const float* cv = prm.c + (i64)bh * kD + half * 64;
+      const float* cv = prm.c + (i64)bh * kD + g * 64;
 #pragma unroll
       for (int c = 0; c < 64; ++c) res[c] = cv[c];
     }
     if (ok && row < nrows) {
       const int dst = prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + row] : row0 + row;
-      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + half * 64;
+      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + g * 64;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
         float v8[8];
@@ -412,7 +427,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         store8(op + ch * 8, v8);
       }
       if (prm.O_sparse) {
-        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + half * 64;
+        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + g * 64;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
           float v8[8];
