@@ -89,6 +89,7 @@ cudaError_t ensure_init() {
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_probe_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
   });
   return g_init_err;
@@ -191,7 +192,8 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
 struct AttendWs {
   void *Qg, *Kg, *Vg;
   float *partial, *X, *Dn, *A, *c, *Psi;
-  __nv_bfloat16* At;
+  __nv_bfloat16 *At, *Qp;
+  int n_split_tc;
   double* fit;
   int n_split;
 };
@@ -212,13 +214,16 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   void* Kg = c.take<char>(BH * N * d * r.es);
   void* Vg = c.take<char>(BH * N * d * r.es);
   const size_t M1 = std::max(r.M, 1);
-  float* partial = c.take<float>(probe_partial_floats(r.BH, ns, (int)M1, r.d));
+  // tensor-core probe kernel: one CTA per (128 probe rows, key slice), about one wave
+  const int ns_tc = std::max(1, std::min(148 / std::max(1, r.BH * (int)((M1 + 127) / 128)), std::max(1, r.N / 128 / 4)));
+  float* partial = c.take<float>(probe_partial_floats(r.BH, std::max(ns, ns_tc), (int)M1, r.d));
+  __nv_bfloat16* Qp = c.take<__nv_bfloat16>(BH * M1 * d);
   float* X = c.take<float>(BH * M1 * d); float* Dn = c.take<float>(BH * M1 * d);
   float* A = c.take<float>(BH * d * d); float* cc = c.take<float>(BH * d);
   float* Psi = c.take<float>(BH * d * d);
   __nv_bfloat16* At = c.take<__nv_bfloat16>(BH * d * d);
   double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
-  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->fit = fit; w->n_split = ns; }
+  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->n_split = ns; }
 }
 
 i64 pair_budget(const Resolved& r) {
@@ -448,7 +453,13 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     for (int i = 0; i < 3; ++i) pa.qs[i] = r.qs[i];
     pa.Kg = w.Kg; pa.Vg = w.Vg; pa.probe_idx = p->probe_idx; pa.q_assign = p->a_Q; pa.kv_off = p->kv_off;
     pa.route_ptr = p->route_ptr; pa.route_idx = p->route_idx; pa.partial = w.partial; pa.X = w.X; pa.Dn = w.Dn;
-    launch_probe_rows(pa, st);
+    if (probe_tc_supported(pa)) {
+      pa.n_split = w.n_split_tc;
+      if (!launch_probe_rows_tc(pa, w.Qp, p->err, st)) return SPARSEPR_ERR_CUDA;
+      launch_probe_merge(pa, st);
+    } else {
+      launch_probe_rows(pa, st);
+    }
     tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
     fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;

@@ -474,6 +474,11 @@ static void probe_dispatch(const ProbeArgs& a, cudaStream_t st) {
   dim3 g2((a.M + 7) / 8, a.BH);
   k_probe_merge<D><<<g2, 256, 0, st>>>(a.partial, a.n_split, a.M, a.X, a.Dn);
 }
+void launch_probe_merge(const ProbeArgs& a, cudaStream_t st) {
+  dim3 g2((a.M + 7) / 8, a.BH);
+  if (a.d == 128) k_probe_merge<128><<<g2, 256, 0, st>>>(a.partial, a.n_split, a.M, a.X, a.Dn);
+  else k_probe_merge<64><<<g2, 256, 0, st>>>(a.partial, a.n_split, a.M, a.X, a.Dn);
+}
 void launch_probe_rows(const ProbeArgs& a, cudaStream_t st) {
   if (a.dtype == SPARSEPR_BF16) { if (a.d == 128) probe_dispatch<__nv_bfloat16, 128>(a, st); else probe_dispatch<__nv_bfloat16, 64>(a, st); }
   else { if (a.d == 128) probe_dispatch<float, 128>(a, st); else probe_dispatch<float, 64>(a, st); }

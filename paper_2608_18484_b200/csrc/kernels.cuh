@@ -97,6 +97,11 @@ struct ProbeArgs {
 };
 size_t probe_partial_floats(int BH, int n_split, int M, int d);
 void launch_probe_rows(const ProbeArgs& a, cudaStream_t st);
+void launch_probe_merge(const ProbeArgs& a, cudaStream_t st);
+// probe_tc.cu: the same partial states from the tensor-core kernel (bf16, d = 128); Qp: scratch [BH][M][128] bf16
+cudaError_t init_probe_tc();
+bool probe_tc_supported(const ProbeArgs& a);
+bool launch_probe_rows_tc(const ProbeArgs& a, __nv_bfloat16* Qp, int* err, cudaStream_t st);
 void launch_write_probe_rows(int dtype, const float* Dn, const int* probe_idx, int BH, int H, int M, int d, void* O,
                              const i64* os, cudaStream_t st);
 

@@ -66,7 +66,11 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   if (s_skip) return;
 
   const int row_tiles = (prm.N + 127) / 128;
-  const int my_tiles = cta < row_tiles ? (row_tiles - cta + prm.ctas_per_head - 1) / prm.ctas_per_head : 0;
+  // contiguous chunk of row tiles per CTA: CTAs that run at the same time then work on distant
+  // tokens, i.e. on different clusters, and do not contend for the same centroid sums
+  const int per_cta = (row_tiles + prm.ctas_per_head - 1) / prm.ctas_per_head;
+  const int tile0 = cta * per_cta;
+  const int my_tiles = max(0, min(per_cta, row_tiles - tile0));
   const int n_chunks = prm.n_chunks;
   const int steps = my_tiles * n_chunks;
   if (tid == 0) {
@@ -96,7 +100,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         if (ch == 0) {
           const int xs = tl & 1;
           if (!mbar_wait(bar(X_EMPTY + xs), ((tl >> 1) & 1) ^ 1, abort_flag)) break;
-          const int row0 = (cta + tl * prm.ctas_per_head) * 128;
+          const int row0 = (tile0 + tl) * 128;
           mbar_expect_tx(bar(X_FULL + xs), 2 * kXBytes);
           tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes, &mapXh, bar(X_FULL + xs), 0, row0, bh, 0);
           tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes + kXBytes, &mapXl, bar(X_FULL + xs), 0, row0, bh, 0);
@@ -134,14 +138,14 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     const float mm = prm.mumax[bh];
     bool ok = true;
     for (int tl = 0; tl < my_tiles; ++tl) {
-      const int row = (cta + tl * prm.ctas_per_head) * 128 + warp * 32 + lane;
+      const int row = (tile0 + tl) * 128 + warp * 32 + lane;
       float best = 3.0e38f, second = 3.0e38f;
       int bi = 0;
       // features of the warp's 32 rows for this lane's two columns (used by the centroid sums);
       // issued before the score wait so that the loads overlap it
       float pv0[32], pv1[32];
       if (prm.sums) {
-        const int rowbase = (cta + tl * prm.ctas_per_head) * 128 + warp * 32;
+        const int rowbase = (tile0 + tl) * 128 + warp * 32;
 #pragma unroll
         for (int rr = 0; rr < 32; ++rr) {
           const int rw = min(rowbase + rr, prm.N - 1);
@@ -196,28 +200,24 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       }
       if (prm.sums) {
         // warp-level pre-aggregation: lanes = feature columns (lane, lane+32); the 32 rows of the
-        // warp were prefetched above; rows of one cluster are summed in row order, then one
-        // fixed-point atomic per (cluster, column)
+        // warp were prefetched above; one fixed-point atomic per (cluster, column)
         unsigned todo = __ballot_sync(FULL, decided);
         const double scl = ldexp(1.0, prm.fx_shift[bh]);
-        i64 f0[32], f1[32];
-#pragma unroll
-        for (int rr = 0; rr < 32; ++rr) {
-          f0[rr] = __double2ll_rn((double)pv0[rr] * scl);
-          f1[rr] = __double2ll_rn((double)pv1[rr] * scl);
-        }
         while (todo) {
           const int leader = __ffs(todo) - 1;
           const int cl = __shfl_sync(FULL, bi, leader);
           const unsigned members = __ballot_sync(FULL, decided && bi == cl) & todo;
           todo &= ~members;
-          i64 acc0 = 0, acc1 = 0;
+          // float32 partial sums in ascending row order (a fixed order, hence reproducible), one
+          // conversion to fixed point per (cluster, column)
+          float a0 = 0.f, a1 = 0.f;
 #pragma unroll
           for (int rr = 0; rr < 32; ++rr) {
             const bool in = (members >> rr) & 1u;
-            acc0 += in ? f0[rr] : 0;
-            acc1 += in ? f1[rr] : 0;
+            a0 += in ? pv0[rr] : 0.f;
+            a1 += in ? pv1[rr] : 0.f;
           }
+          const i64 acc0 = __double2ll_rn((double)a0 * scl), acc1 = __double2ll_rn((double)a1 * scl);
           i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
           if (lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane), (u64)acc0);
           if (lane + 32 < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane + 32), (u64)acc1);
