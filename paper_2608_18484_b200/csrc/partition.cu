@@ -7,49 +7,50 @@ namespace spr {
 
 // =============================================================================
 // Gram matrices: M_K = Q_s^T Q_s / M_s (Appendix B.1) and
-// M_Q = Ktilde^T Ktilde / (C_k^+ d) (Appendix B.2).  One CTA per head, every
-// thread owns d*d/256 entries accumulated in float64.
+// M_Q = Ktilde^T Ktilde / (C_k^+ d) (Appendix B.2), float64 accumulation.
+// Grid (D/16, heads): a CTA owns 16 rows of the D x D result; thread t owns column
+// t % D and 8 consecutive rows.  Input rows are staged in shared memory as doubles.
 // =============================================================================
 constexpr int kGramChunk = 32;
+constexpr int kGramSlab = 16;
 
 template <int D>
-__device__ __forceinline__ void gram_accumulate(const float* rows, int nrows, double (&acc)[D * D / 256]) {
-  // rows: [kGramChunk][D] in shared memory
+__device__ __forceinline__ void gram_accumulate(const double* rows, int nrows, int i0, int j, double (&acc)[8]) {
+  for (int s = 0; s < nrows; ++s) {
+    const double xj = rows[s * D + j];
+    const double* xi = rows + s * D + i0;                 // the same 8 values for the whole half-block: broadcast
 #pragma unroll
-  for (int e = 0; e < D * D / 256; ++e) {
-    const int idx = threadIdx.x + e * 256;
-    const int i = idx / D, j = idx % D;
-    double a = acc[e];
-    for (int s = 0; s < nrows; ++s) a += (double)rows[s * D + i] * (double)rows[s * D + j];
-    acc[e] = a;
+    for (int k = 0; k < 8; ++k) acc[k] = fma(xi[k], xj, acc[k]);
   }
 }
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i64 sb, i64 sh, i64 sn, int H, int N,
                                                      int Ms, u64 seed, double* __restrict__ Mout) {
-  __shared__ float rows[kGramChunk * D];
-  const int bh = blockIdx.x, b = bh / H, h = bh % H;
+  __shared__ __align__(16) double rows[kGramChunk * D];
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
   const T* base = Q + b * sb + h * sh;
   const u64 U = sample_offset(seed, kTagQuerySample, bh);
-  double acc[D * D / 256];
-#pragma unroll
-  for (int e = 0; e < D * D / 256; ++e) acc[e] = 0.0;
+  const int j = threadIdx.x % D, i0 = blockIdx.x * kGramSlab + (threadIdx.x / D) * 8;
+  const bool active = threadIdx.x < 2 * D;
+  double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   for (int s0 = 0; s0 < Ms; s0 += kGramChunk) {
     const int nr = min(kGramChunk, Ms - s0);
+    __syncthreads();
     for (int t = threadIdx.x; t < nr * (D / 8); t += 256) {
       const int s = t / (D / 8), c = t % (D / 8);
       float v[8];
       load8(base + (i64)strided_row(s0 + s, Ms, N, U) * sn + c * 8, v);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) rows[s * D + c * 8 + k] = v[k];
+      for (int k = 0; k < 8; ++k) rows[s * D + c * 8 + k] = (double)v[k];
     }
     __syncthreads();
-    gram_accumulate<D>(rows, nr, acc);
-    __syncthreads();
+    if (active) gram_accumulate<D>(rows, nr, i0, j, acc);
   }
+  if (active) {
 #pragma unroll
-  for (int e = 0; e < D * D / 256; ++e) Mout[(i64)bh * D * D + threadIdx.x + e * 256] = acc[e] / (double)Ms;
+    for (int k = 0; k < 8; ++k) Mout[(i64)bh * D * D + (i64)(i0 + k) * D + j] = acc[k] / (double)Ms;
+  }
 }
 
 // kappa [BH][C][D] float32, n [BH][C] group sizes.  Empty groups are skipped and the
@@ -57,10 +58,10 @@ __global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i6
 template <int D>
 __global__ void __launch_bounds__(256) k_centroid_gram(const float* __restrict__ kappa, const int* __restrict__ n, int C,
                                                        double* __restrict__ Mout) {
-  __shared__ float rows[kGramChunk * D];
-  __shared__ float mean[D];
+  __shared__ __align__(16) double rows[kGramChunk * D];
+  __shared__ double mean[D];
   __shared__ int s_cnt;
-  const int bh = blockIdx.x;
+  const int bh = blockIdx.y;
   const float* kp = kappa + (i64)bh * C * D;
   const int* nn = n + (i64)bh * C;
   if (threadIdx.x == 0) s_cnt = 0;
@@ -77,40 +78,41 @@ __global__ void __launch_bounds__(256) k_centroid_gram(const float* __restrict__
     double m = 0.0;
     for (int g = 0; g < C; ++g)
       if (nn[g] > 0) m += (double)kp[(i64)g * D + threadIdx.x];
-    mean[threadIdx.x] = cplus > 0 ? (float)(m / cplus) : 0.f;
+    mean[threadIdx.x] = cplus > 0 ? m / cplus : 0.0;
   }
-  __syncthreads();
-  double acc[D * D / 256];
-#pragma unroll
-  for (int e = 0; e < D * D / 256; ++e) acc[e] = 0.0;
+  const int j = threadIdx.x % D, i0 = blockIdx.x * kGramSlab + (threadIdx.x / D) * 8;
+  const bool active = threadIdx.x < 2 * D;
+  double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   for (int g0 = 0; g0 < C; g0 += kGramChunk) {
     const int nr = min(kGramChunk, C - g0);
+    __syncthreads();
     for (int t = threadIdx.x; t < nr * D; t += 256) {
-      const int s = t / D, j = t % D;
-      rows[t] = nn[g0 + s] > 0 ? kp[(i64)(g0 + s) * D + j] - mean[j] : 0.f;
+      const int s = t / D, jj = t % D;
+      rows[t] = nn[g0 + s] > 0 ? (double)kp[(i64)(g0 + s) * D + jj] - mean[jj] : 0.0;
     }
     __syncthreads();
-    gram_accumulate<D>(rows, nr, acc);
-    __syncthreads();
+    if (active) gram_accumulate<D>(rows, nr, i0, j, acc);
   }
   const double denom = cplus > 0 ? (double)cplus * (double)D : 1.0;
+  if (active) {
 #pragma unroll
-  for (int e = 0; e < D * D / 256; ++e) Mout[(i64)bh * D * D + threadIdx.x + e * 256] = acc[e] / denom;
+    for (int k = 0; k < 8; ++k) Mout[(i64)bh * D * D + (i64)(i0 + k) * D + j] = acc[k] / denom;
+  }
 }
 
 void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
                         double* Mout, cudaStream_t st) {
   if (dtype == SPARSEPR_BF16) {
-    if (d == 128) k_sample_gram<__nv_bfloat16, 128><<<BH, 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
-    else k_sample_gram<__nv_bfloat16, 64><<<BH, 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    if (d == 128) k_sample_gram<__nv_bfloat16, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    else k_sample_gram<__nv_bfloat16, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
   } else {
-    if (d == 128) k_sample_gram<float, 128><<<BH, 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
-    else k_sample_gram<float, 64><<<BH, 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    if (d == 128) k_sample_gram<float, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    else k_sample_gram<float, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
   }
 }
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st) {
-  if (d == 128) k_centroid_gram<128><<<BH, 256, 0, st>>>(kappa, n, C, Mout);
-  else k_centroid_gram<64><<<BH, 256, 0, st>>>(kappa, n, C, Mout);
+  if (d == 128) k_centroid_gram<128><<<dim3(128 / kGramSlab, BH), 256, 0, st>>>(kappa, n, C, Mout);
+  else k_centroid_gram<64><<<dim3(64 / kGramSlab, BH), 256, 0, st>>>(kappa, n, C, Mout);
 }
 
 // =============================================================================

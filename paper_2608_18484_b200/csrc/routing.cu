@@ -109,46 +109,125 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   fcost = block_sum_i64(fcost, red);     // contains a __syncthreads: forced[] visible below
   const i64 rem = budget - fcost;
 
-  // 2. threshold search: S(t) = cost of live, non-forced cells with bits >= t
+  // 2. threshold search: S(t) = cost of live, non-forced cells with bits >= t; find the smallest t with
+  //    S(t) <= rem.  Radix descent, one byte of the bit pattern per pass: per-warp cost histograms over
+  //    the next byte of the cells that share the prefix found so far, then the bucket that contains the
+  //    threshold is the first one whose suffix cost fits.
   u64 tstar;
+  i64 taken = 0;                        // cost of the cells with bits >= tstar
   if (select_all) tstar = 0;
   else if (rem < 0) tstar = 1ull << 32;
   else {
-    u64 lo = 0, hi = 1ull << 32;
-    while (lo < hi) {
-      const u64 mid = (lo + hi) >> 1;
-      i64 s = 0;
+    i64* whist = reinterpret_cast<i64*>(nqs + Cq + ((Cq + Ck) & 1));   // [nw][256], 8-byte aligned (see route_smem)
+    __shared__ i64 s_above;
+    __shared__ int s_dstar;
+    unsigned prefix = 0;
+    i64 above = 0;                      // cost of the cells above the current bucket
+    bool all_fit = false;
+    for (int level = 0; level < 4; ++level) {
+      const int shift = 24 - 8 * level;
+      for (int e = threadIdx.x; e < nw * 256; e += blockDim.x) whist[e] = 0;
+      __syncthreads();
+      i64* myh = whist + w * 256;
       for (int a = w; a < Cq; a += nw) {
         if (nqs[a] == 0) continue;
         const int fb = forced[a];
-        i64 rs = 0;
-        for (int b = lane; b < Ck; b += 32)
-          if ((u64)u[(i64)a * Ck + b] >= mid && b != fb) rs += nks[b];     // empty groups cost 0
-        s += rs * nqs[a];
+        const i64 na = nqs[a];
+        for (int b0 = 0; b0 < Ck; b0 += 32) {
+          const int b = b0 + lane;
+          unsigned bits = 0;
+          bool in = b < Ck && b != fb && nks[b] > 0;
+          if (in) {
+            bits = u[(i64)a * Ck + b];
+            in = level == 0 || (bits >> (shift + 8)) == (prefix >> (shift + 8));
+          }
+          unsigned todo = __ballot_sync(0xffffffffu, in);
+          const int digit = (bits >> shift) & 255;
+          while (todo) {                                         // lanes of one digit add their key counts together
+            const int leader = __ffs(todo) - 1;
+            const int dl = __shfl_sync(0xffffffffu, digit, leader);
+            const unsigned grp = __ballot_sync(0xffffffffu, in && digit == dl) & todo;
+            const int keys = __reduce_add_sync(0xffffffffu, (in && digit == dl) ? nks[b] : 0);
+            if (lane == leader) myh[dl] += na * keys;
+            todo &= ~grp;
+          }
+        }
       }
-      s = block_sum_i64(s, red);
-      if (s <= rem) hi = mid; else lo = mid + 1;
+      __syncthreads();
+      if (w == 0) {
+        // lane l owns digits 8l .. 8l+7
+        i64 loc[8], lsum = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          i64 t = 0;
+          for (int ww = 0; ww < nw; ++ww) t += whist[ww * 256 + lane * 8 + k];
+          loc[k] = t; lsum += t;
+        }
+        i64 suf = lsum;                                          // sum over lanes >= this lane
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const i64 t = __shfl_down_sync(0xffffffffu, suf, o); if (lane + o < 32) suf += t; }
+        i64 run = suf;                                           // suffix cost from digit 8l
+        int first = -1;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          if (first < 0 && above + run <= rem) first = lane * 8 + k;
+          run -= loc[k];
+        }
+        const unsigned have = __ballot_sync(0xffffffffu, first >= 0);
+        int dstar = 256;
+        if (have) dstar = __shfl_sync(0xffffffffu, first, __ffs(have) - 1);
+        // cost of the digits >= dstar
+        i64 sfx = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) if (lane * 8 + k >= dstar) sfx += loc[k];
+        sfx = warp_sum(sfx);
+        if (lane == 0) { s_dstar = dstar; s_above = above + sfx; }
+      }
+      __syncthreads();
+      const int dstar = s_dstar;
+      above = s_above;
+      if (dstar == 0) { all_fit = true; break; }                 // the whole bucket fits (only possible at the top level)
+      prefix |= (unsigned)(dstar - 1) << shift;
     }
-    tstar = lo;
+    tstar = all_fit ? (u64)prefix : (u64)prefix + 1ull;
+    taken = above;
   }
-  // cost already taken by the threshold tier
-  i64 taken = 0;
-  if (!select_all && rem >= 0) {
+  // tie tier: cells with bits == tstar-1, in (a,b) order, longest prefix that fits
+  __shared__ int s_tie_cnt, s_tie_idx[32];
+  if (threadIdx.x == 0) { s_last_tie = -1; s_tie_cnt = 0; }
+  __syncthreads();
+  const bool tie_tier = !select_all && rem >= 0 && tstar > 0 && tstar <= 0xFFFFFFFFull + 1ull;
+  // The tier usually holds a single cell: collect its cells in parallel; up to 32 are ordered and
+  // cut by one warp, larger tiers (many equal scores) take the sequential walk below.
+  if (tie_tier) {
+    const unsigned tv = (unsigned)(tstar - 1);
     for (int a = w; a < Cq; a += nw) {
       if (nqs[a] == 0) continue;
       const int fb = forced[a];
-      i64 rs = 0;
       for (int b = lane; b < Ck; b += 32)
-        if ((u64)u[(i64)a * Ck + b] >= tstar && b != fb) rs += nks[b];
-      taken += rs * nqs[a];
+        if (nks[b] > 0 && b != fb && u[(i64)a * Ck + b] == tv) {
+          const int pos = atomicAdd(&s_tie_cnt, 1);
+          if (pos < 32) s_tie_idx[pos] = a * Ck + b;
+        }
     }
-    taken = block_sum_i64(taken, red);
   }
-  // tie tier: cells with bits == tstar-1, in (a,b) order, longest prefix that fits
-  if (threadIdx.x == 0) s_last_tie = -1;
   __syncthreads();
-  const bool tie_tier = !select_all && rem >= 0 && tstar > 0 && tstar <= 0xFFFFFFFFull + 1ull;
-  if (tie_tier && w == 0) {
+  const int tie_cnt = s_tie_cnt;
+  if (tie_tier && tie_cnt <= 32 && w == 0) {
+    const int idx = lane < tie_cnt ? s_tie_idx[lane] : 0x7fffffff;
+    const i64 cost = lane < tie_cnt ? (i64)nqs[idx / Ck] * nks[idx % Ck] : 0;
+    i64 cum = taken;                                     // cost of the tier cells up to and including this one, in (a,b) order
+    for (int j = 0; j < tie_cnt; ++j) {
+      const int oj = __shfl_sync(0xffffffffu, idx, j);
+      const i64 cj = __shfl_sync(0xffffffffu, cost, j);
+      if (oj <= idx) cum += cj;
+    }
+    const bool fits = lane < tie_cnt && cum <= rem;      // monotone along the order: costs are positive
+    int best = fits ? idx : -1;
+    best = warp_max(best);
+    if (lane == 0) s_last_tie = best;
+  }
+  if (tie_tier && tie_cnt > 32 && w == 0) {
     const unsigned tv = (unsigned)(tstar - 1);
     i64 cum = taken, last = -1;
     bool stop = false;
@@ -225,7 +304,9 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   }
 }
 
-static size_t route_smem(int Cq, int Ck) { return (size_t)(3 * Cq + Ck) * sizeof(int); }
+static size_t route_smem(int Cq, int Ck) {      // forced, cnt, nqs [Cq], nks [Ck] ints, then 32 x 256 int64 histograms
+  return (size_t)(3 * Cq + Ck + ((Cq + Ck) & 1)) * sizeof(int) + (size_t)32 * 256 * sizeof(long long);
+}
 // routed pairs and cells of given routes (used when a plan is imported)
 __global__ void __launch_bounds__(256) k_count_pairs(const int* __restrict__ q_off, const int* __restrict__ kv_off,
                                                      const int* __restrict__ route_ptr, const int* __restrict__ route_idx,
