@@ -164,17 +164,15 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
     for (int c = 0; c < NN; ++c) fro = fmaf(a[c], a[c], fro);
   }
   fro = block_sum(fro, red);                            // contains __syncthreads: rows[] is complete
-  // float32 rounding leaves an off-diagonal floor near 5e-13 of the squared norm: stop there,
-  // or as soon as a sweep no longer halves the off-diagonal mass
-  const float tol = fro * 4e-12f;
+  // stop once the off-diagonal mass is below 1e-8 of the squared norm (off/||A|| < 1e-4; the sweep
+  // that got there has already squared the previous level), or when a sweep no longer halves it
+  const float tol = fro * 1e-8f;
   float prev_off = 3.0e38f;
   for (int sweep = 0; sweep < 16; ++sweep) {
     float off = 0.f;
     if (is_a) {
 #pragma unroll
-      for (int c = 0; c < NN; ++c) off = fmaf(a[c], a[c], off);
-      const float dg = rows[i * LD + i];
-      off -= dg * dg;
+      for (int c = 0; c < NN; ++c) off += c == i ? 0.f : a[c] * a[c];
     }
     off = block_sum(off, red);
     if (!(off > tol) || (sweep >= 4 && off > 0.5f * prev_off)) break;
@@ -193,11 +191,14 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
       __syncthreads();                                  // all reads of rows[] done, cs[] visible
       if (is_a) {
         // rows: (a_p, a_q) <- (c a_p - s a_q, s a_p + c a_q); the partner row lives in the neighbouring lane
+        // the partner row is still in shared memory (written at the end of the previous round)
         const float ss = (i & 1) ? s : -s;
+        const float* prow = rows + (i ^ 1) * LD;
 #pragma unroll
-        for (int col = 0; col < NN; ++col) {
-          const float b = __shfl_xor_sync(0xffffffffu, a[col], 1);
-          a[col] = fmaf(ss, b, c * a[col]);
+        for (int col = 0; col < NN; col += 4) {
+          const float4 b = *reinterpret_cast<const float4*>(prow + col);
+          a[col] = fmaf(ss, b.x, c * a[col]); a[col + 1] = fmaf(ss, b.y, c * a[col + 1]);
+          a[col + 2] = fmaf(ss, b.z, c * a[col + 2]); a[col + 3] = fmaf(ss, b.w, c * a[col + 3]);
         }
       }
       // columns (A and V alike): (x_p, x_q) <- (c x_p - s x_q, s x_p + c x_q), then move to the next round's positions
@@ -211,6 +212,7 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
       }
 #pragma unroll
       for (int col = 0; col < NN; ++col) a[col] = nx[col];
+      __syncthreads();                                  // every partner row has been read
       if (is_a) {
         const int dst = rr_next(i, NN);                 // the row moves as well
 #pragma unroll
