@@ -9,16 +9,17 @@
 // final assignment always equals the exact float64 decision with ties to the lowest id.
 //
 // Persistent CTAs: each owns row tiles (128 rows) of one head; centroid chunks of 256
-// stream through shared memory (resident when C <= 256).  Roles: warps 0-3 epilogue
-// (one row per thread: tcgen05.ld, best/second, fixed-point centroid sums with
-// warp-level pre-aggregation), warp 4 TMA producer, warp 5 MMA issuer.
+// stream through shared memory (resident when C <= 256).  Roles: warps 0-3 and 6-9 are two
+// epilogue groups on alternate row tiles (one row per thread: tcgen05.ld, best/second,
+// fixed-point centroid sums with warp-level pre-aggregation), warp 4 TMA producer, warp 5
+// MMA issuer.
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
 namespace spr {
 namespace tc {
 
-constexpr int kKmThreads = 192;
+constexpr int kKmThreads = 320;
 constexpr int kKmChunk = 256;                         // centroids per MMA (N)
 constexpr uint32_t kXBytes = 128 * 128;               // one [128 rows x 64 bf16] block
 constexpr uint32_t kMuBytes = kKmChunk * 128;         // one [256 x 64 bf16] block
@@ -133,19 +134,21 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     }
   } else {
     // =========================== epilogue: argmin, sums =====================================
+    // two groups of four warps (warps 0-3 and 6-9) take alternate row tiles
     const uint32_t FULL = 0xffffffffu;
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const int grp = warp < 4 ? 0 : 1, wq = warp & 3;
+    const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const float mm = prm.mumax[bh];
     bool ok = true;
-    for (int tl = 0; tl < my_tiles; ++tl) {
-      const int row = (tile0 + tl) * 128 + warp * 32 + lane;
+    for (int tl = grp; tl < my_tiles; tl += 2) {
+      const int row = (tile0 + tl) * 128 + wq * 32 + lane;
       float best = 3.0e38f, second = 3.0e38f;
       int bi = 0;
       // features of the warp's 32 rows for this lane's two columns (used by the centroid sums);
       // issued before the score wait so that the loads overlap it
       float pv0[32], pv1[32];
       if (prm.sums) {
-        const int rowbase = (tile0 + tl) * 128 + warp * 32;
+        const int rowbase = (tile0 + tl) * 128 + wq * 32;
 #pragma unroll
         for (int rr = 0; rr < 32; ++rr) {
           const int rw = min(rowbase + rr, prm.N - 1);
