@@ -1,5 +1,6 @@
 // C-ABI layer: argument validation, workspace carving, launch order.
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -95,7 +96,11 @@ cudaError_t ensure_init() {
   return g_init_err;
 }
 
-bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
+bool launch_ok() {
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess && std::getenv("SPARSEPR_DEBUG")) std::fprintf(stderr, "sparsepr: CUDA error: %s\n", cudaGetErrorString(e));
+  return e == cudaSuccess;
+}
 
 // Optional per-stage CUDA-event timing of one call.  Events are recorded on the call's
 // stream between stages; finish() synchronises once and accumulates the elapsed times.

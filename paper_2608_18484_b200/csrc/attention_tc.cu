@@ -19,6 +19,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
+#include <cstdio>
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -228,16 +229,22 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,384), O_B [384,512); P_g overwrites S_g[0,64)
     if (lane == 0 && n_tiles > 0) {
       const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
+      // descriptors are built once; inside the loops only their address field moves (in 16-byte units),
+      // so that issuing an MMA costs a couple of integer adds in this single thread
+      const uint64_t q_desc = smem_desc(base + Smem::q, 16);
+      const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
+      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
       auto issue_qk = [&](int i) -> bool {
         const int s = i % kKStages;
         if (!mbar_wait(bar(K_FULL + s), (i / kKStages) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
+        const uint64_t kd = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint32_t koff = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          umma_bf16(d, smem_desc(base + Smem::q + koff, 16), smem_desc(base + Smem::k + s * kTileBytes + koff, 16), idesc_qk, kk > 0);
+          const uint64_t koff = (uint64_t)((kk >> 2) * (kHalfBytes >> 4) + (kk & 3) * 2);     // compile-time constant
+          umma_bf16(d, q_desc + koff, kd + koff, idesc_qk, kk > 0);
         }
         umma_commit(bar(K_EMPTY + s));
         umma_commit(bar(S_FULL + (i & 1)));
@@ -245,22 +252,41 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       };
       if (ok) ok = issue_qk(0);
       if (ok && n_tiles > 1) ok = issue_qk(1);
+#ifdef SPR_ATTN_TIMING
+      long long mv = 0, mp = 0, mi = 0, mq = 0, m0;
+#define SPR_M0() m0 = clock64()
+#define SPR_MACC(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
+#else
+#define SPR_M0()
+#define SPR_MACC(v)
+#endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int g = i & 1, j = i >> 1, s = i % kVStages;
         const uint2 mt = meta[i & 7];
+        SPR_M0();
         if (!mbar_wait(bar(V_FULL + s), (i / kVStages) & 1, abort_flag)) { ok = false; break; }
+        SPR_MACC(mv);
         if (!mbar_wait(bar(P_FULL + g), j & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, O_g rescaled if needed
+        SPR_MACC(mp);
         tc_fence_after();
         const uint32_t d = tmem + 256u + (uint32_t)g * 128u;
         const uint32_t pa = tmem + (uint32_t)g * 128u;
         const int nsub = (int)mt.y;
-        for (int kk = 0; kk < nsub; ++kk) {
-          const uint64_t bdesc = smem_desc(base + Smem::v + s * kTileBytes + kk * kSubBytes, kHalfBytes);
-          umma_bf16_ts(d, pa + kk * 8, bdesc, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);   // O_g accumulates over its tiles
-        }
+        const uint64_t vd = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < kSubPerTile; ++kk)
+          if (kk < nsub)
+            umma_bf16_ts(d, pa + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);   // O_g accumulates over its tiles
         umma_commit(bar(V_EMPTY + s));
+        SPR_MACC(mi);
         if (i + 2 < n_tiles) ok = issue_qk(i + 2);          // S_g (and the P_g inside it) is rewritten after P V (i)
+        SPR_MACC(mq);
       }
+#ifdef SPR_ATTN_TIMING
+      if (blockIdx.x == 7 && blockIdx.y == 0)
+        printf("mma thread tiles %d: wait V %lld  wait P %lld  issue PV %lld  wait K + issue QK %lld (cycles per tile)\n", n_tiles,
+               mv / n_tiles, mp / n_tiles, mi / n_tiles, mq / n_tiles);
+#endif
       if (ok) umma_commit(bar(O_DONE));
       if (ok && prm.has_corr) {
         // correction product: bf16(O_sp) in TMEM [0,64) times A (in K stage 0) -> TMEM [128,256)
@@ -291,7 +317,16 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
+#ifdef SPR_ATTN_TIMING
+    long long tw = 0, tl = 0, tm = 0, ts = 0, t0;
+#define SPR_T0() t0 = clock64()
+#define SPR_ACC(v) do { const long long t1 = clock64(); v += t1 - t0; t0 = t1; } while (0)
+#else
+#define SPR_T0()
+#define SPR_ACC(v)
+#endif
     for (int i = g, j = 0; i < n_tiles; i += 2, ++j) {
+      SPR_T0();
       ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + g), j & 1, abort_flag) &&
                                 mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
       if (!ok) continue;                                         // warp-uniform
@@ -299,12 +334,10 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint2 mt = meta[i & 7];
       float s[128];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float t[32];
-        tmem_ld32(s_addr + q * 32, t);
-#pragma unroll
-        for (int c = 0; c < 32; ++c) s[q * 32 + c] = t[c];
-      }
+      for (int q = 0; q < 4; ++q) tmem_ld32_nowait(s_addr + q * 32, *reinterpret_cast<float(*)[32]>(&s[q * 32]));   // four loads in flight, one wait
+      SPR_ACC(tw);
+      tmem_ld_wait();
+      SPR_ACC(tl);
       if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
 #pragma unroll
         for (int box = 0; box < 8; ++box) {
@@ -349,11 +382,18 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         uint32_t w[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[q * 64 + 2 * c], s[q * 64 + 2 * c + 1]);
+        if (q == 0) SPR_ACC(tm);
         tmem_st32u(s_addr + q * 32, w);
       }
       tc_fence_before();
       mbar_arrive(bar(P_FULL + g));
+      SPR_ACC(ts);
     }
+#ifdef SPR_ATTN_TIMING
+    if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 4))
+      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  math %lld  pack+st %lld (cycles per tile)\n", warp, (n_tiles + 1 - g) / 2,
+             tw / max(1, (n_tiles + 1 - g) / 2), tl / max(1, (n_tiles + 1 - g) / 2), tm / max(1, (n_tiles + 1 - g) / 2), ts / max(1, (n_tiles + 1 - g) / 2));
+#endif
     // ---- merge the two groups, normalise ------------------------------------------------------
     if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
     stat[g * 128 + row] = make_float2(m_ref, l);
