@@ -88,13 +88,19 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------
-def launches_per_call(T, fitted):
+def launches_per_call(T, fitted, tensor_path):
     """Kernels of this library launched by one plan + attend call (memsets excluded)."""
-    kmeans = 2 + T + (T - 1)                       # init, first norms, T assignments, T-1 updates
-    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 1   # per side: Gram+eig, projection, k-means, sort+means; probes; route; tiles
+    if tensor_path:      # per side: split features; per iteration: split centroids, assign, recheck; T-1 updates
+        kmeans = 2 + 1 + 3 * T + (T - 1)
+    else:                # init, first norms, T assignments, T-1 updates
+        kmeans = 2 + T + (T - 1)
+    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 2      # per side: Gram+eig, projection, k-means, sort+means; probes; route; tile offsets
     if not fitted:
         plan -= 2
-    attend = 3 + 1 + ((2 + 5 + 1) if fitted else 0)   # gathers, attention, (probe rows+merge, fit, probe write)
+    attend = 3 + 1                                   # gathers, attention
+    if fitted:
+        attend += (3 if tensor_path else 2) + 5 + 1  # probe rows (+gather) + merge, fit, probe write
+        attend += 1 if tensor_path else 0            # transposed correction matrix
     return plan + attend
 
 
@@ -322,7 +328,7 @@ def main():
            "stage_ms": stages, "plan_ms": sum(v for k, v in stages.items() if k in B.STAGES[:10]),
            "attend_ms": sum(v for k, v in stages.items() if k in B.STAGES[10:15]),
            "device_error": st["device_error"], "assign_rechecked_rows": st["assign_rechecked_rows"],
-           "gpu_launches": launches_per_call(params.kmeans_iters or 8, True) * args.steps,
+           "gpu_launches": launches_per_call(params.kmeans_iters or 8, True, wl.dtype == "bf16" and wl.d == 128) * args.steps,
            "roofline": roofline, "clocks": clocks, "e2e": e2e}
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(wl)

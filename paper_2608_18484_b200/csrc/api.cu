@@ -571,14 +571,17 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     for (int g = 0; g < r.Cq; ++g) { neQ += q[g + 1] > q[g]; out->max_q_group = std::max(out->max_q_group, q[g + 1] - q[g]); }
     out->nonempty_kv_groups_min = std::min(out->nonempty_kv_groups_min, neK);
     out->nonempty_q_groups_min = std::min(out->nonempty_q_groups_min, neQ);
-    // pairs issued by the tiled kernel: query tiles of 64 rows x key tiles of 64 over the concatenated routed keys
+    // pairs issued by the tiled kernel over the concatenated routed keys: the tensor-core kernel uses
+    // 128-row query tiles and 128-key tiles built from 16-row boxes, the float32 kernel 64 x 64 tiles
+    const bool tcpath = r.dtype == SPARSEPR_BF16 && r.d == 128;
+    const int qtile = tcpath ? 128 : 64, ktile = tcpath ? 128 : 64, box = tcpath ? 16 : 1;
     const int* rpp = &rp[(size_t)bh * (r.Cq + 1)];
     const int* rii = &ri[(size_t)bh * r.Cq * r.Ck];
     for (int a = 0; a < r.Cq; ++a) {
       i64 keys = 0;
-      for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += k[rii[t] + 1] - k[rii[t]];
-      const i64 qt = (q[a + 1] - q[a] + 63) / 64, kt = (keys + 63) / 64;
-      out->padded_tile_pairs += qt * 64 * kt * 64;
+      for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += (k[rii[t] + 1] - k[rii[t]] + box - 1) / box * box;
+      const i64 qt = (q[a + 1] - q[a] + qtile - 1) / qtile, kt = (keys + ktile - 1) / ktile;
+      out->padded_tile_pairs += qt * qtile * kt * ktile;
     }
   }
   out->rho_exec = out->rho_route + (double)r.M / (double)r.N;
