@@ -100,7 +100,7 @@ def launches_per_call(T, fitted, tensor_path):
     attend = 3 + 1                                   # gathers, attention
     if fitted:
         attend += (3 if tensor_path else 2) + 5 + 1  # probe rows (+gather) + merge, fit, probe write
-        attend += 1 if tensor_path else 0            # transposed correction matrix
+        attend += 2 if tensor_path else 0            # transposed correction matrix, correction pass
     return plan + attend
 
 
@@ -326,7 +326,7 @@ def main():
            "tile_padding_factor": st["padded_tile_pairs"] / max(st["routed_pairs"], 1),
            "rel_l2_vs_dense_kernel": {"probe_fitted": rel_fit, "hard_drop": rel_hard},
            "stage_ms": stages, "plan_ms": sum(v for k, v in stages.items() if k in B.STAGES[:10]),
-           "attend_ms": sum(v for k, v in stages.items() if k in B.STAGES[10:15]),
+           "attend_ms": sum(v for k, v in stages.items() if k in B.STAGES[10:16]),
            "device_error": st["device_error"], "assign_rechecked_rows": st["assign_rechecked_rows"],
            "gpu_launches": launches_per_call(params.kmeans_iters or 8, True, wl.dtype == "bf16" and wl.d == 128) * args.steps,
            "roofline": roofline, "clocks": clocks, "e2e": e2e}

@@ -121,14 +121,17 @@ typedef struct {
  * *_PERMUTE = counting sort and group means; QUERY_METRIC = centroid Gram and its
  * eigen-decomposition; PROBE_SELECT; ROUTE = cell scores and selection.  Attend:
  * GATHER = group-major copies of Q, K, V; PROBE_ROWS = exact and hard-drop rows of
- * the probes; FIT = ridge fit and subspace; ATTENTION = block-sparse kernel with the
- * correction epilogue; PROBE_WRITE.  DENSE = the dense entry point. */
+ * the probes; FIT = ridge fit and subspace; ATTENTION = block-sparse kernel;
+ * CORRECTION = residual correction of Eq. 9 (zero where the block-sparse kernel applies
+ * it in its epilogue); PROBE_WRITE.  DENSE = the dense entry point.  A call without a
+ * profile runs PROBE_SELECT beside ROUTE and PROBE_ROWS + FIT beside ATTENTION on a second
+ * stream, so its duration is less than the sum of the stages. */
 enum {
   SPARSEPR_STAGE_KEY_METRIC = 0, SPARSEPR_STAGE_KEY_PROJECT, SPARSEPR_STAGE_KEY_KMEANS, SPARSEPR_STAGE_KEY_PERMUTE,
   SPARSEPR_STAGE_QUERY_METRIC, SPARSEPR_STAGE_QUERY_PROJECT, SPARSEPR_STAGE_QUERY_KMEANS, SPARSEPR_STAGE_QUERY_PERMUTE,
   SPARSEPR_STAGE_PROBE_SELECT, SPARSEPR_STAGE_ROUTE,
   SPARSEPR_STAGE_GATHER, SPARSEPR_STAGE_PROBE_ROWS, SPARSEPR_STAGE_FIT, SPARSEPR_STAGE_ATTENTION,
-  SPARSEPR_STAGE_PROBE_WRITE, SPARSEPR_STAGE_DENSE, SPARSEPR_STAGE_COUNT
+  SPARSEPR_STAGE_CORRECTION, SPARSEPR_STAGE_PROBE_WRITE, SPARSEPR_STAGE_DENSE, SPARSEPR_STAGE_COUNT
 };
 /* Milliseconds per stage, measured with CUDA events on the call's stream.  The
  * *_timed calls ADD to the entries, so one zero-initialised struct can accumulate

@@ -55,7 +55,7 @@ class PlanHost(C.Structure):
 
 
 STAGES = ["key_metric", "key_project", "key_kmeans", "key_permute", "query_metric", "query_project", "query_kmeans",
-          "query_permute", "probe_select", "route", "gather", "probe_rows", "fit", "attention", "probe_write", "dense"]
+          "query_permute", "probe_select", "route", "gather", "probe_rows", "fit", "attention", "correction", "probe_write", "dense"]
 
 
 class Profile(C.Structure):

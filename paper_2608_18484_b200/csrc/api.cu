@@ -89,6 +89,7 @@ cudaError_t ensure_init() {
     if ((e = init_routing()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_correction_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_probe_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
@@ -136,6 +137,15 @@ struct StageTimer {
 struct sparsepr_plan_s {
   Resolved r;
   cudaStream_t stream;
+  // second stream for work that is independent of the main chain (probe selection next to routing;
+  // probe rows and fit next to the block-sparse kernel), forked and joined with the two events
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  ~sparsepr_plan_s() {
+    if (ev_fork) cudaEventDestroy(ev_fork);
+    if (ev_join) cudaEventDestroy(ev_join);
+    if (side) cudaStreamDestroy(side);
+  }
   // device state (all inside the caller's plan workspace)
   int* err; int* recheck;
   double* Mmat; double* lam;
@@ -323,10 +333,29 @@ static sparsepr_status_t make_plan(const sparsepr_shape_t* shape, const sparsepr
   if (!p) return SPARSEPR_ERR_INVALID_ARG;
   p->r = r;
   p->stream = static_cast<cudaStream_t>(cuda_stream);
+  int prio_lo = 0, prio_hi = 0;
+  cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+  if (cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+      cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    delete p;
+    return SPARSEPR_ERR_CUDA;
+  }
   Carver c(workspace);
   carve_plan(c, r, p);
   *out = p;
   return SPARSEPR_OK;
+}
+
+// the side stream starts after everything queued on `st` so far ...
+void fork_side(const sparsepr_plan_s* p, cudaStream_t st) {
+  cudaEventRecord(p->ev_fork, st);
+  cudaStreamWaitEvent(p->side, p->ev_fork, 0);
+}
+// ... and `st` continues once the side stream's work is done
+void join_side(const sparsepr_plan_s* p, cudaStream_t st) {
+  cudaEventRecord(p->ev_join, p->side);
+  cudaStreamWaitEvent(st, p->ev_join, 0);
 }
 
 static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
@@ -365,15 +394,19 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
   launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
   tm.mark(SPARSEPR_STAGE_QUERY_PERMUTE);
-  // probes and routes
+  // probes and routes; without a profile the probe selection runs beside the routing
+  const bool overlap = prof == nullptr && r.M > 0;
+  cudaStream_t ps = st;
+  if (overlap) { fork_side(p, st); ps = p->side; }
   if (r.M > 0)
-    launch_probe_select(p->phi, r.RQ, r.rQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, st);
+    launch_probe_select(p->phi, r.RQ, r.rQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, ps);
   tm.mark(SPARSEPR_STAGE_PROBE_SELECT);
   launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
                       p->route_idx, p->rstate, nullptr, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, p->tile_off128, st);
+  if (overlap) join_side(p, st);
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
   if (!launch_ok()) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -451,7 +484,22 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   launch_gather_rows(r.dtype, V, r.vs, r.BH, r.H, p->kv_perm, r.N, r.d, w.Vg, st);
   tm.mark(SPARSEPR_STAGE_GATHER);
   const bool fitted = r.mode == 0 && r.M > 0;
+  AttnArgs aa{};
+  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.scale = r.scale;
+  aa.Q = w.Qg; aa.K = w.Kg; aa.V = w.Vg;
+  aa.q_off = p->q_off; aa.kv_off = p->kv_off; aa.route_ptr = p->route_ptr; aa.route_idx = p->route_idx;
+  aa.q_perm = p->q_perm; aa.tile_off = p->tile_off; aa.Cq = r.Cq; aa.Ck = r.Ck;
+  aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
+  aa.O_sparse = O_sparse;
+  aa.err = p->err;
+  const bool tensor = attention_tc_supported(aa);
+  // The probe rows and the fit depend only on the gathered K, V and the plan.  With the tensor-core
+  // kernel (whose correction is a separate pass) they run on the plan's second stream beside the
+  // block-sparse kernel; a profiled call keeps everything on one stream so that stage times add up.
+  const bool overlap = fitted && tensor && prof == nullptr;
   if (fitted) {
+    cudaStream_t fs = st;
+    if (overlap) { fork_side(p, st); fs = p->side; }
     ProbeArgs pa{};
     pa.dtype = r.dtype; pa.BH = r.BH; pa.H = r.H; pa.N = r.N; pa.d = r.d; pa.M = r.M; pa.Ck = r.Ck; pa.Cq = r.Cq;
     pa.n_split = w.n_split; pa.scale = r.scale; pa.Q = Q;
@@ -460,34 +508,30 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     pa.route_ptr = p->route_ptr; pa.route_idx = p->route_idx; pa.partial = w.partial; pa.X = w.X; pa.Dn = w.Dn;
     if (probe_tc_supported(pa)) {
       pa.n_split = w.n_split_tc;
-      if (!launch_probe_rows_tc(pa, w.Qp, p->err, st)) return SPARSEPR_ERR_CUDA;
-      launch_probe_merge(pa, st);
+      if (!launch_probe_rows_tc(pa, w.Qp, p->err, fs)) return SPARSEPR_ERR_CUDA;
+      launch_probe_merge(pa, fs);
     } else {
-      launch_probe_rows(pa, st);
+      launch_probe_rows(pa, fs);
     }
     tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
     fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;
     fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
-    launch_fit(fa, st);
+    launch_fit(fa, fs);
     tm.mark(SPARSEPR_STAGE_FIT);
   }
-  AttnArgs aa{};
-  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.scale = r.scale;
-  aa.Q = w.Qg; aa.K = w.Kg; aa.V = w.Vg;
-  aa.q_off = p->q_off; aa.kv_off = p->kv_off; aa.route_ptr = p->route_ptr; aa.route_idx = p->route_idx;
-  aa.q_perm = p->q_perm; aa.tile_off = p->tile_off; aa.Cq = r.Cq; aa.Ck = r.Ck;
-  aa.A = fitted ? w.A : nullptr; aa.c = fitted ? w.c : nullptr;
-  aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
-  aa.O_sparse = O_sparse;
-  aa.err = p->err;
-  if (attention_tc_supported(aa)) {
+  if (tensor) {
     aa.tile_off = p->tile_off128;
-    if (!launch_attention_tc(aa, w.At, st)) return SPARSEPR_ERR_CUDA;
+    if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
+    tm.mark(SPARSEPR_STAGE_ATTENTION);
+    if (overlap) join_side(p, st);
+    if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
+    tm.mark(SPARSEPR_STAGE_CORRECTION);
   } else {
+    aa.A = fitted ? w.A : nullptr; aa.c = fitted ? w.c : nullptr;      // correction fused into this kernel's epilogue
     launch_attention_simt(aa, st);
+    tm.mark(SPARSEPR_STAGE_ATTENTION);
   }
-  tm.mark(SPARSEPR_STAGE_ATTENTION);
   if (fitted) launch_write_probe_rows(r.dtype, w.Dn, p->probe_idx, r.BH, r.H, r.M, r.d, O, r.os, st);
   tm.mark(SPARSEPR_STAGE_PROBE_WRITE);
   tm.finish();
@@ -531,7 +575,7 @@ sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_sc
   aa.Q = Q; aa.K = K; aa.V = V; aa.O = O;
   for (int i = 0; i < 3; ++i) { aa.qs[i] = r.qs[i]; aa.ks[i] = r.ks[i]; aa.vs[i] = r.vs[i]; aa.os[i] = r.os[i]; }
   if (attention_tc_supported(aa)) {
-    if (!launch_attention_tc(aa, nullptr, static_cast<cudaStream_t>(cuda_stream))) return SPARSEPR_ERR_CUDA;
+    if (!launch_attention_tc(aa, static_cast<cudaStream_t>(cuda_stream))) return SPARSEPR_ERR_CUDA;
   } else {
     launch_attention_simt(aa, static_cast<cudaStream_t>(cuda_stream));
   }

@@ -13,9 +13,9 @@
 //                        back over the first half of S_g with tcgen05.st
 //   O_g += P V_i         tcgen05.mma with the A operand read from TMEM; O_g stays in TMEM
 // While group A works on tile i the tensor cores already produce S_B for tile i+1.
-// Epilogue: merge (O_A, O_B) like two splits of the key range, O_sp = O / l; correction
-// O_sp A on the tensor cores (A = composed affine map of Eq. 9, bf16), + c, store at the
-// original token index (inverse permutation).
+// Epilogue: merge (O_A, O_B) like two splits of the key range, O_sp = O / l, store at the
+// original token index (inverse permutation).  The residual correction of Eq. 9 is a pass
+// of its own (correction_tc.cu) so that the fit can overlap this kernel.
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
@@ -58,7 +58,7 @@ struct Smem {                          // offsets from a 1024-byte aligned base
 constexpr size_t kSmemBytes = Smem::total;                        // the dynamic segment is 1024-byte aligned and the only shared memory
 
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kKStages, V_FULL = K_EMPTY + kKStages, V_EMPTY = V_FULL + kVStages,
-           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, C_FULL, X_FULL, X_DONE, META_FULL,
+           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, META_FULL,
            kNumBars = META_FULL + 8 };
 static_assert(kNumBars <= 32, "barrier area");
 
@@ -66,8 +66,6 @@ struct Params {
   int BH, H, N, Cq, Ck, sparse;
   float scale_log2;
   const int *q_off, *kv_off, *route_ptr, *route_idx, *q_perm, *tile_off;
-  const float* c;                 // [BH][128] or null
-  int has_corr;
   __nv_bfloat16* O; i64 os[3];
   float* O_sparse;
   int* err;
@@ -77,7 +75,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) { return pack_bf
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapA, Params prm) {
+               const __grid_constant__ CUtensorMap mapV, Params prm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
@@ -125,7 +123,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i)
-      mbar_init(bar(i), (i == P_FULL || i == P_FULL + 1) ? 128 : i == X_FULL ? 256 : 1);
+      mbar_init(bar(i), (i == P_FULL || i == P_FULL + 1) ? 128 : 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -214,15 +212,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           tma_load_4d(dst + kHalfBytes, map, bar(full0 + s), 64, my_start, c2, c3);
         }
       }
-      if (is_k && lane == 0 && prm.has_corr && !*abort_flag) {
-        // the composed correction matrix (transposed, bf16) goes into K stage 0 once every QK^T that used it is done
-        const int uses0 = (n_tiles + kKStages - 1) / kKStages;
-        if (mbar_wait(bar(K_EMPTY + 0), (uint32_t)((uses0 - 1) & 1), abort_flag)) {
-          mbar_expect_tx(bar(C_FULL), kTileBytes);
-          tma_load_4d(base + Smem::k, &mapA, bar(C_FULL), 0, 0, bh, 0);
-          tma_load_4d(base + Smem::k + kHalfBytes, &mapA, bar(C_FULL), 64, 0, bh, 0);
-        }
-      }
     }
   } else if (warp == 9) {
     // =========================== MMA issuer ==============================================
@@ -288,18 +277,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                mv / n_tiles, mp / n_tiles, mi / n_tiles, mq / n_tiles);
 #endif
       if (ok) umma_commit(bar(O_DONE));
-      if (ok && prm.has_corr) {
-        // correction product: bf16(O_sp) in TMEM [0,64) times A (in K stage 0) -> TMEM [128,256)
-        if (mbar_wait(bar(C_FULL), 0, abort_flag) && mbar_wait(bar(X_FULL), 0, abort_flag)) {
-          tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint32_t koff = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            umma_bf16_ts(tmem + 128u, tmem + kk * 8, smem_desc(base + Smem::k + koff, 16), idesc_qk, kk > 0);
-          }
-          umma_commit(bar(X_DONE));
-        }
-      }
     }
   } else {
     // =========================== softmax (warps 0-7) =======================================
@@ -424,35 +401,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
       }
     }
-    float res[64];
-#pragma unroll
-    for (int c = 0; c < 64; ++c) res[c] = o[c];
-    if (prm.has_corr && n_tiles > 0) {
-      if (ok) {
-        uint32_t w[32];
-#pragma unroll
-        for (int c = 0; c < 32; ++c) w[c] = pack_bf16(o[2 * c], o[2 * c + 1]);
-        tmem_st32u(tmem + lane_addr + g * 32, w);                // bf16(O_sp): columns [0,64) = 128 values
-        tc_fence_before();
-        mbar_arrive(bar(X_FULL));
-      }
-      ok = __all_sync(FULL, ok && mbar_wait(bar(X_DONE), 0, abort_flag));
-      if (ok) {
-        tc_fence_after();
-        const float* cv = prm.c + (i64)bh * kD + g * 64;
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          float t[32];
-          tmem_ld32(tmem + lane_addr + 128u + g * 64 + q * 32, t);
-#pragma unroll
-          for (int c = 0; c < 32; ++c) res[q * 32 + c] = o[q * 32 + c] + t[c] + cv[q * 32 + c];
-        }
-      }
-    } else if (prm.has_corr) {
-      const float* cv = prm.c + (i64)bh * kD + g * 64;
-#pragma unroll
-      for (int c = 0; c < 64; ++c) res[c] = cv[c];
-    }
     if (ok && row < nrows) {
       const int dst = prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + row] : row0 + row;
       __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + g * 64;
@@ -460,7 +408,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int ch = 0; ch < 8; ++ch) {
         float v8[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) v8[k] = res[ch * 8 + k];
+        for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
         store8(op + ch * 8, v8);
       }
       if (prm.O_sparse) {
@@ -488,18 +436,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
-}
-
-// A [BH][128][128] float32 (row k, column n) -> At [BH][n][k] bf16
-__global__ void k_transpose_correction(const float* __restrict__ A, __nv_bfloat16* __restrict__ At) {
-  __shared__ float tile[32][33];
-  const int bh = blockIdx.z;
-  const float* a = A + (i64)bh * kD * kD;
-  __nv_bfloat16* t = At + (i64)bh * kD * kD;
-  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-  for (int r = threadIdx.y; r < 32; r += 8) tile[r][threadIdx.x] = a[(k0 + r) * kD + n0 + threadIdx.x];
-  __syncthreads();
-  for (int r = threadIdx.y; r < 32; r += 8) t[(n0 + r) * kD + k0 + threadIdx.x] = __float2bfloat16_rn(tile[threadIdx.x][r]);
 }
 
 // ---- tensor maps (driver entry point fetched through the runtime; libcuda is not linked) -------
@@ -546,10 +482,9 @@ bool attention_tc_supported(const AttnArgs& a) {
   return a.dtype == SPARSEPR_BF16 && a.d == 128 && tc::tma_available();
 }
 
-// `At` is scratch for the transposed bf16 correction matrix [BH][128][128] (only with a.A != null)
-bool launch_attention_tc(const AttnArgs& a, __nv_bfloat16* At, cudaStream_t st) {
+bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   using namespace tc;
-  CUtensorMap mq, mk, mv, ma;
+  CUtensorMap mq, mk, mv;
   const bool sparse = a.route_ptr != nullptr;
   const int B = a.BH / a.H;
   bool ok;
@@ -561,19 +496,15 @@ bool launch_attention_tc(const AttnArgs& a, __nv_bfloat16* At, cudaStream_t st) 
          make_map(&mv, a.V, kD, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub);
   }
   if (!ok) return false;
-  if (a.A) {
-    k_transpose_correction<<<dim3(kD / 32, kD / 32, a.BH), dim3(32, 8), 0, st>>>(a.A, At);
-    if (!make_map(&ma, At, kD, kD, a.BH, 1, 0, (i64)kD * kD, kD, kTile)) return false;
-  } else ma = mq;
   Params p{};
   p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.sparse = sparse;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.q_off = a.q_off; p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;
-  p.tile_off = a.tile_off; p.c = a.c; p.has_corr = a.A != nullptr;
+  p.tile_off = a.tile_off;
   p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
   p.O_sparse = a.O_sparse; p.err = a.err;
   const int tiles = (a.N + kTile - 1) / kTile + (sparse ? a.Cq : 0);
-  k_attention_tc<<<dim3(tiles, a.BH), kThreads, kSmemBytes, st>>>(mq, mk, mv, ma, p);
+  k_attention_tc<<<dim3(tiles, a.BH), kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
   return true;
 }
 

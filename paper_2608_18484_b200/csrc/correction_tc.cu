@@ -1,0 +1,156 @@
+// Residual correction of Eq. 9 as a pass of its own on the sm_100a tensor cores:
+//   O <- O + O A + c     (in place, bf16, d_v = 128; A, c = composed affine map of one head)
+// It runs after the block-sparse kernel, so that the probe rows and the fit (which produce A and c)
+// can execute on a second stream while the block-sparse kernel is busy.  The pass is bandwidth
+// bound: each 128-row tile of O is read once by TMA and written once.
+//   warps 0-3  one thread per row: O A from TMEM, O from the swizzled tile, + c, store
+//   warp  4    TMA loads (O tile, A^T), eight tcgen05.mma, TMEM owner
+// Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
+#include <cuda.h>
+#include "kernels.cuh"
+#include "tc_common.cuh"
+
+namespace spr {
+namespace tc {
+
+constexpr int kCorrThreads = 160;
+constexpr int kCorrTile = 128;
+constexpr uint32_t kCorrHalf = kCorrTile * 128;      // one [128 rows x 64 bf16] swizzled block
+constexpr uint32_t kCorrTileBytes = 2 * kCorrHalf;
+struct CorrSmem {
+  static constexpr uint32_t o = 0;
+  static constexpr uint32_t a = o + kCorrTileBytes;
+  static constexpr uint32_t bars = a + kCorrTileBytes;
+  static constexpr uint32_t misc = bars + 16;
+  static constexpr uint32_t total = misc + 16;
+};
+
+struct CorrParams {
+  int H, N;
+  const float* c;                  // [BH][128]
+  __nv_bfloat16* O; i64 os[3];
+  int* err;
+};
+
+__global__ void __launch_bounds__(kCorrThreads)
+k_correction_tc(const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapA, CorrParams prm) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  volatile int* misc = reinterpret_cast<volatile int*>(smem_raw + CorrSmem::misc);   // [0] tmem base, [1] abort, [2] skip
+  const uint32_t bar_full = base + CorrSmem::bars, bar_done = bar_full + 8;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y, b = bh / prm.H, h = bh % prm.H;
+  const int row0 = blockIdx.x * kCorrTile;
+  if (tid == 0) {
+    misc[2] = (prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT) || (base & 1023u) != 0;
+    if ((base & 1023u) != 0) set_error(prm.err, SPARSEPR_ERR_CUDA);
+    mbar_init(bar_full, 1);
+    mbar_init(bar_done, 1);
+    misc[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (misc[2]) return;
+  if (warp == 4) tmem_alloc(base + CorrSmem::misc, 128);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = (uint32_t)misc[0];
+  volatile int* abort_flag = &misc[1];
+
+  if (warp == 4) {
+    if (lane == 0) {
+      mbar_expect_tx(bar_full, 2 * kCorrTileBytes);
+      tma_load_4d(base + CorrSmem::o, &mapO, bar_full, 0, row0, h, b);
+      tma_load_4d(base + CorrSmem::o + kCorrHalf, &mapO, bar_full, 64, row0, h, b);
+      tma_load_4d(base + CorrSmem::a, &mapA, bar_full, 0, 0, bh, 0);
+      tma_load_4d(base + CorrSmem::a + kCorrHalf, &mapA, bar_full, 64, 0, bh, 0);
+      if (mbar_wait(bar_full, 0, abort_flag)) {
+        tc_fence_after();
+        const uint64_t od = smem_desc(base + CorrSmem::o, 16), ad = smem_desc(base + CorrSmem::a, 16);
+        const uint32_t idesc = idesc_bf16(0, 128);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t koff = (uint64_t)((kk >> 2) * (kCorrHalf >> 4) + (kk & 3) * 2);
+          umma_bf16(tmem, od + koff, ad + koff, idesc, kk > 0);          // (O A)[m][n] = sum_k O[m][k] At[n][k]
+        }
+        umma_commit(bar_done);
+      }
+    }
+  } else {
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag));
+    const int row = warp * 32 + lane;
+    if (ok) {
+      tc_fence_after();
+      const float* cv = prm.c + (i64)bh * 128;
+      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)(row0 + row) * prm.os[2];
+      const unsigned char* orow = smem_raw + CorrSmem::o + row * 128;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float t[32];
+        tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + q * 32, t);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int j = (q & 1) * 4 + ch;                                // 16-byte chunk of the 128-byte row
+          const uint4 raw = *reinterpret_cast<const uint4*>(orow + (q >> 1) * kCorrHalf + ((j ^ (row & 7)) << 4));
+          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&raw);
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float2 f = __bfloat1622float2(hp[k]);
+            const int col = q * 32 + ch * 8 + 2 * k;
+            v8[2 * k] = f.x + t[ch * 8 + 2 * k] + cv[col];
+            v8[2 * k + 1] = f.y + t[ch * 8 + 2 * k + 1] + cv[col + 1];
+          }
+          if (row0 + row < prm.N) store8(op + q * 32 + ch * 8, v8);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int k = 0; k < 64; ++k) __nanosleep(1000);      // let copies that may still be in flight land
+    if (tid == 0) set_error(prm.err, SPARSEPR_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+// A [BH][128][128] float32 (row k, column n) -> At [BH][n][k] bf16
+__global__ void k_transpose_correction(const float* __restrict__ A, __nv_bfloat16* __restrict__ At) {
+  __shared__ float tile[32][33];
+  const int bh = blockIdx.z;
+  const float* a = A + (i64)bh * 128 * 128;
+  __nv_bfloat16* t = At + (i64)bh * 128 * 128;
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int r = threadIdx.y; r < 32; r += 8) tile[r][threadIdx.x] = a[(k0 + r) * 128 + n0 + threadIdx.x];
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += 8) t[(n0 + r) * 128 + k0 + threadIdx.x] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+}
+
+}  // namespace tc
+
+cudaError_t init_correction_tc() {
+  return cudaFuncSetAttribute(tc::k_correction_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::CorrSmem::total);
+}
+
+bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
+                          int* err, cudaStream_t st) {
+  using namespace tc;
+  CUtensorMap mo, ma;
+  k_transpose_correction<<<dim3(4, 4, BH), dim3(32, 8), 0, st>>>(A, At);
+  if (!make_map(&mo, O, 128, N, H, BH / H, os[0], os[1], os[2], kCorrTile) ||
+      !make_map(&ma, At, 128, 128, BH, 1, 0, (i64)128 * 128, 128, kCorrTile))
+    return false;
+  CorrParams p{};
+  p.H = H; p.N = N; p.c = c; p.O = (__nv_bfloat16*)O; p.err = err;
+  for (int i = 0; i < 3; ++i) p.os[i] = os[i];
+  k_correction_tc<<<dim3((N + kCorrTile - 1) / kCorrTile, BH), kCorrThreads, CorrSmem::total, st>>>(mo, ma, p);
+  return true;
+}
+
+}  // namespace spr

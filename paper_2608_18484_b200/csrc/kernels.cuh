@@ -83,8 +83,12 @@ void launch_attention_simt(const AttnArgs& a, cudaStream_t st);
 // ---- attention_tc.cu (tcgen05 / TMEM / TMA; bf16, d = 128) -------------------------------------
 cudaError_t init_attention_tc();
 bool attention_tc_supported(const AttnArgs& a);
-// tile_off in `a` must have been built for 128-row tiles; At: bf16 scratch [BH][128][128] when a.A != null
-bool launch_attention_tc(const AttnArgs& a, __nv_bfloat16* At, cudaStream_t st);
+// tile_off in `a` must have been built for 128-row tiles; a.A and a.c are ignored (no correction epilogue)
+bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
+// correction_tc.cu: O <- O + O A + c in place (bf16, d_v = 128); At: bf16 scratch [BH][128][128]
+cudaError_t init_correction_tc();
+bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
+                          int* err, cudaStream_t st);
 
 struct ProbeArgs {
   int dtype, BH, H, N, d, M, Ck, Cq, n_split;
