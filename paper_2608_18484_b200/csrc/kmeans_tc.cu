@@ -5,7 +5,7 @@
 // xh.ml, xl.mh are accumulated in fp32 in TMEM; the dropped term is ~2^-18 relative).
 // Each row keeps its best and second-best score; a row whose gap is not larger than a
 // conservative bound on the score error is NOT decided here but handed to the exact
-// float64 recheck (one warp per row, same operation order as the definition), so the
+// float64 recheck (one CTA per row, same operation order as the definition), so the
 // final assignment always equals the exact float64 decision with ties to the lowest id.
 //
 // Persistent CTAs: each owns row tiles (128 rows) of one head; centroid chunks of 256
@@ -242,34 +242,39 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   }
 }
 
-// Exact decision for the rows the fast path could not prove: one warp per row, lanes over
-// centroids, squared distance in float64 with the terms added in order of k.
+// Exact decision for the rows the fast path could not prove: one CTA per row, one thread per
+// centroid, squared distance in float64 with the terms added in order of k (the definition;
+// the zero padding of columns r..R-1 adds exact zeros), ties to the lowest id.
 __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ flagged, const int* __restrict__ flag_count,
                                                         const float* __restrict__ phi, int ldphi, int N, int r, int R,
                                                         const float* __restrict__ mu, int C, int* __restrict__ assign,
                                                         i64* __restrict__ sums, int* __restrict__ counts,
                                                         const int* __restrict__ fx_shift, int* __restrict__ recheck_total) {
-  const int lane = threadIdx.x & 31;
-  const int warps = gridDim.x * (blockDim.x >> 5);
+  __shared__ double s_best[8];
+  __shared__ int s_bi[8];
+  const unsigned FULL = 0xffffffffu;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = *flag_count;
-  for (int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n; i += warps) {
+  for (int i = blockIdx.x; i < n; i += gridDim.x) {
     const int gr = flagged[i];
     const int bh = gr / N;
-    const float* x = phi + (i64)gr * ldphi;
+    const float4* x4 = reinterpret_cast<const float4*>(phi + (i64)gr * ldphi);
     const float* muh = mu + (i64)bh * C * R;
     double best = 0.0;
     int bi = -1;
-    for (int c = lane; c < C; c += 32) {
+    for (int c = tid; c < C; c += 256) {
       const float4* m4 = reinterpret_cast<const float4*>(muh + (i64)c * R);
-      const float4* x4 = reinterpret_cast<const float4*>(x);
       double dsum = 0.0;
-      for (int k4 = 0; k4 < (r + 3) / 4; ++k4) {            // columns r..R-1 hold zeros on both sides
-        const float4 xv = x4[k4], mv = m4[k4];
-        const float xs[4] = {xv.x, xv.y, xv.z, xv.w}, ms[4] = {mv.x, mv.y, mv.z, mv.w};
+      for (int k4 = 0; k4 < R / 4; k4 += 4) {               // R is a multiple of 16: four vector loads in flight
+        float4 xv[4], mv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { xv[u] = x4[k4 + u]; mv[u] = m4[k4 + u]; }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          if (k4 * 4 + u < r) {
-            const double diff = __dsub_rn((double)xs[u], (double)ms[u]);
+          const float xs[4] = {xv[u].x, xv[u].y, xv[u].z, xv[u].w}, ms[4] = {mv[u].x, mv[u].y, mv[u].z, mv[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const double diff = __dsub_rn((double)xs[e], (double)ms[e]);
             dsum = __dadd_rn(dsum, __dmul_rn(diff, diff));
           }
         }
@@ -278,19 +283,30 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      const double ob = __shfl_xor_sync(FULL, best, o);
+      const int oi = __shfl_xor_sync(FULL, bi, o);
       if (oi >= 0 && (bi < 0 || ob < best || (ob == best && oi < bi))) { best = ob; bi = oi; }
     }
-    if (lane == 0) assign[gr] = bi;
-    if (sums) {
-      const double scl = ldexp(1.0, fx_shift[bh]);
-      i64* s = sums + ((i64)bh * C + bi) * R;
-      for (int k = lane; k < r; k += 32) atomicAdd(reinterpret_cast<u64*>(s + k), (u64)__double2ll_rn((double)x[k] * scl));
-      if (lane == 0) atomicAdd(counts + (i64)bh * C + bi, 1);
+    if (lane == 0) { s_best[warp] = best; s_bi[warp] = bi; }
+    __syncthreads();
+    best = s_best[0]; bi = s_bi[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) {
+      const double ob = s_best[w];
+      const int oi = s_bi[w];
+      if (oi >= 0 && (bi < 0 || ob < best || (ob == best && oi < bi))) { best = ob; bi = oi; }
     }
+    if (tid == 0) assign[gr] = bi;
+    if (sums) {
+      const float* x = phi + (i64)gr * ldphi;
+      const double scl = ldexp(1.0, fx_shift[bh]);
+      i64* sp = sums + ((i64)bh * C + bi) * R;
+      if (tid < r) atomicAdd(reinterpret_cast<u64*>(sp + tid), (u64)__double2ll_rn((double)x[tid] * scl));
+      if (tid == 0) atomicAdd(counts + (i64)bh * C + bi, 1);
+    }
+    __syncthreads();
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0 && recheck_total) *recheck_total = n;
+  if (blockIdx.x == 0 && tid == 0 && recheck_total) *recheck_total = n;
 }
 
 // phi fp32 [rows][ld] -> hi/lo bf16 [rows][64] (zero padded) and the row norms
@@ -348,7 +364,7 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
   cudaMemsetAsync(a.flag_count, 0, sizeof(int), st);
   k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
-  k_assign_recheck<<<148 * 2, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
+  k_assign_recheck<<<148 * 4, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
                                             a.counts, a.fx_shift, a.recheck_total);
   return true;
 }
