@@ -140,8 +140,8 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
                                                       float* __restrict__ Fout, double* __restrict__ lam_out) {
   constexpr int LD = NN + 4;
   extern __shared__ __align__(16) float sm_j[];
-  float* rows = sm_j;                                   // [NN][LD] rows of A in the current position order
-  float2* cs = reinterpret_cast<float2*>(rows + NN * LD);   // [NN/2] rotation of every pair
+  float* rows = sm_j;                                   // [2][NN][LD] rows of A by position, double buffered over rounds
+  float2* cs = reinterpret_cast<float2*>(rows + 2 * NN * LD);   // [NN/2] rotation of every pair
   __shared__ float red[34];
   __shared__ int s_rank[NN];
   const int tid = threadIdx.x;
@@ -168,32 +168,40 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
   // that got there has already squared the previous level), or when a sweep no longer halves it
   const float tol = fro * 1e-8f;
   float prev_off = 3.0e38f;
+  // An A thread keeps its matrix row for the whole run; `pos` is the position of that row (and of
+  // the matching column) in the round-robin order.  Columns move physically inside the register
+  // arrays, so that every register index is a compile-time constant.
+  int pos = i;
   for (int sweep = 0; sweep < 16; ++sweep) {
     float off = 0.f;
     if (is_a) {
 #pragma unroll
-      for (int c = 0; c < NN; ++c) off += c == i ? 0.f : a[c] * a[c];
+      for (int c = 0; c < NN; ++c) off = fmaf(a[c], a[c], off);
+      const float dg = rows[pos * LD + pos];
+      off -= dg * dg;
     }
     off = block_sum(off, red);
     if (!(off > tol) || (sweep >= 4 && off > 0.5f * prev_off)) break;
     prev_off = off;
     for (int round = 0; round < NN - 1; ++round) {
-      const int p = i & ~1;                             // pair (p, p+1)
-      const float app = rows[p * LD + p], apq = rows[p * LD + p + 1], aqq = rows[(p + 1) * LD + p + 1];
       float c = 1.f, s = 0.f;
-      if (apq != 0.f) {
-        const float tau = (aqq - app) / (2.f * apq);
-        const float t = copysignf(1.f, tau) / (fabsf(tau) + sqrtf(fmaf(tau, tau, 1.f)));   // -> 0 when tau overflows
-        c = rsqrtf(fmaf(t, t, 1.f));
-        s = t * c;
-      }
-      if (is_a && !(i & 1)) cs[i >> 1] = make_float2(c, s);
-      __syncthreads();                                  // all reads of rows[] done, cs[] visible
       if (is_a) {
-        // rows: (a_p, a_q) <- (c a_p - s a_q, s a_p + c a_q); the partner row lives in the neighbouring lane
-        // the partner row is still in shared memory (written at the end of the previous round)
-        const float ss = (i & 1) ? s : -s;
-        const float* prow = rows + (i ^ 1) * LD;
+        const int p = pos & ~1;                           // pair (p, p+1)
+        const float app = rows[p * LD + p], apq = rows[p * LD + p + 1], aqq = rows[(p + 1) * LD + p + 1];
+        if (apq != 0.f) {
+          const float tau = (aqq - app) / (2.f * apq);
+          const float t = copysignf(1.f, tau) / (fabsf(tau) + sqrtf(fmaf(tau, tau, 1.f)));   // -> 0 when tau overflows
+          c = rsqrtf(fmaf(t, t, 1.f));
+          s = t * c;
+        }
+        if (!(pos & 1)) cs[pos >> 1] = make_float2(c, s);
+      }
+      __syncthreads();                                  // cs[] visible
+      if (is_a) {
+        // rows: (a_p, a_q) <- (c a_p - s a_q, s a_p + c a_q); the partner row was stored by its owner at the
+        // end of the previous round
+        const float ss = (pos & 1) ? s : -s;
+        const float* prow = rows + (pos ^ 1) * LD;
 #pragma unroll
         for (int col = 0; col < NN; col += 4) {
           const float4 b = *reinterpret_cast<const float4*>(prow + col);
@@ -212,27 +220,20 @@ __global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict_
       }
 #pragma unroll
       for (int col = 0; col < NN; ++col) a[col] = nx[col];
-      __syncthreads();                                  // every partner row has been read
+      rows = (rows == sm_j) ? sm_j + NN * LD : sm_j;     // the other buffer: nobody reads it during this round
       if (is_a) {
-        const int dst = rr_next(i, NN);                 // the row moves as well
+        pos = rr_next(pos, NN);                         // the row moves as well
 #pragma unroll
         for (int col = 0; col < NN; col += 4)
-          *reinterpret_cast<float4*>(rows + dst * LD + col) = make_float4(a[col], a[col + 1], a[col + 2], a[col + 3]);
+          *reinterpret_cast<float4*>(rows + pos * LD + col) = make_float4(a[col], a[col + 1], a[col + 2], a[col + 3]);
       }
-      __syncthreads();
-      if (is_a) {
-#pragma unroll
-        for (int col = 0; col < NN; col += 4) {
-          const float4 v = *reinterpret_cast<const float4*>(rows + i * LD + col);
-          a[col] = v.x; a[col + 1] = v.y; a[col + 2] = v.z; a[col + 3] = v.w;
-        }
-      }
+      __syncthreads();                                  // rows of the new round complete; every cs[] read done
     }
   }
   // eigenvalue of position c = A[c][c]; eigenvector = column c of V.  Rank descending (ties by position).
   __syncthreads();
   float lam_i = 0.f;
-  if (is_a) lam_i = rows[i * LD + i];
+  if (is_a) lam_i = rows[i * LD + i];                   // by position: thread i reports position i
   __syncthreads();
   float* lam_s = reinterpret_cast<float*>(cs);          // NN floats fit in the NN/2 float2 slots
   if (is_a) lam_s[i] = lam_i;
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(1024) k_jacobi_eig_f64(const double* __restric
 static size_t jacobi64_smem(int n) {
   return (size_t)n * (n + 1) * 8 + (size_t)(n * (n + 1) + (n & 1)) * 4 + n * 8 + n * 4 + 34 * 8 + 16;
 }
-static size_t jacobi_smem(int n) { return (size_t)n * (n + 4) * 4 + (size_t)n * 4 + 16; }
+static size_t jacobi_smem(int n) { return (size_t)2 * n * (n + 4) * 4 + (size_t)n * 4 + 16; }
 cudaError_t init_jacobi() {
   cudaError_t e = cudaFuncSetAttribute(k_jacobi_eig<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(128));
   if (e != cudaSuccess) return e;
