@@ -90,6 +90,7 @@ cudaError_t ensure_init() {
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_correction_tc()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_project_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_probe_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_fit()) != cudaSuccess) { g_init_err = e; return; }
@@ -157,7 +158,7 @@ struct sparsepr_plan_s {
   int *route_ptr, *route_idx, *tile_off, *tile_off128;
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
-  __nv_bfloat16 *xh, *xl, *mh, *ml; float* xnorm; int* flagged;
+  __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged;
 };
 
 namespace {
@@ -194,7 +195,9 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   __nv_bfloat16* xh = c.take<__nv_bfloat16>(BH * N * 64); __nv_bfloat16* xl = c.take<__nv_bfloat16>(BH * N * 64);
   __nv_bfloat16* mh = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64); __nv_bfloat16* ml = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64);
   float* xnorm = c.take<float>(BH * N); int* flagged = c.take<int>(BH * N);
+  __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
   if (p) {
+    p->Ft = Ft;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -375,7 +378,11 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
   launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
   tm.mark(SPARSEPR_STAGE_KEY_METRIC);
-  launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+  if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
+    if (!launch_project_tc(K, r.ks, r.BH, r.H, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+  } else {
+    launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+  }
   tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
   run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, st);
   tm.mark(SPARSEPR_STAGE_KEY_KMEANS);
@@ -387,7 +394,11 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_jacobi_eig(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
   tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
-  launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+  if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {
+    if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+  } else {
+    launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+  }
   tm.mark(SPARSEPR_STAGE_QUERY_PROJECT);
   run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, st);
   tm.mark(SPARSEPR_STAGE_QUERY_KMEANS);

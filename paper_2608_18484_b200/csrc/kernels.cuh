@@ -29,6 +29,12 @@ void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, 
 void launch_gather_rows(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, int N, int d, void* out,
                         cudaStream_t st);
 
+// project_tc.cu: the same projection on the tensor cores (bf16, d = 128, r <= 64); Ft: bf16 scratch [BH][3][64][128]
+cudaError_t init_project_tc();
+bool project_tc_supported(int dtype, int d, int r, const i64* xs);
+bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r, const float* F, bool rms, float eps,
+                       float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st);
+
 // ---- kmeans_tc.cu (tcgen05 score contraction + exact recheck) --------------------------------------
 struct KmeansTcArgs {
   int BH, N, C, r, R;
