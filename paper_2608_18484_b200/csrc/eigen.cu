@@ -1,0 +1,543 @@
+// Leading eigenpairs of batched symmetric matrices (n = 64 or 128), one CTA per matrix:
+// the feature maps F_K, F_Q of Section 4.1 and the probe-residual basis Psi_r of Eq. 9.
+//
+// Float64 throughout, matrix resident in shared memory:
+//   1. Householder reduction to tridiagonal form T (reflectors kept in the lower triangle)
+//   2. the r largest eigenvalues of T by Sturm-count bisection, one thread per eigenvalue
+//   3. their eigenvectors by inverse iteration on T - lambda I (Gaussian elimination with
+//      partial pivoting, factored once per eigenvalue), one thread per eigenvector
+//   4. modified Gram-Schmidt inside groups of close eigenvalues, one warp per group
+//   5. Rayleigh quotients, residuals ||T z - lambda z|| and all pairwise inner products are
+//      checked; a matrix that fails the check is marked (NaN in its first output element)
+//      and left to the cyclic Jacobi kernel, which is launched behind this one and returns
+//      at once for unmarked matrices
+//   6. back-transformation with the reflectors, scaling, output
+// The work per matrix is O(n^3) for step 1 and O(r n^2) for step 6, each spread over the CTA;
+// steps 2-3 are O(n) recurrences per thread.
+#include <cstdio>
+#include "kernels.cuh"
+
+namespace spr {
+
+namespace {
+
+constexpr int kEigThreads = 1024;
+constexpr int kEigMaxR = 64;
+constexpr int kZld = kEigMaxR + 1;
+constexpr int kTpr = 8;                                            // threads per matrix row in the Householder steps
+
+__device__ __forceinline__ double hash_unit(int i, int j) {        // deterministic start vector entries in [0.5, 1.5)
+  u64 x = (u64)(i + 1) * 0x9E3779B97F4A7C15ull + (u64)(j + 1) * 0xBF58476D1CE4E5B9ull;
+  x ^= x >> 31; x *= 0x94D049BB133111EBull; x ^= x >> 29;
+  return 0.5 + (double)(x >> 11) * (1.0 / 9007199254740992.0);
+}
+
+// sum over the 32 warps of the CTA with one barrier: partial sums go to one of two buffers in turn,
+// every warp then adds the 32 partials itself (same order everywhere, so all threads agree bit for bit)
+__device__ __forceinline__ double cta_sum(double v, double* red, int& turn) {
+  v = warp_sum(v);
+  double* buf = red + (turn & 1) * 32;
+  ++turn;
+  if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return warp_sum(buf[threadIdx.x & 31]);
+}
+__device__ __forceinline__ double cta_max(double v, double* red, int& turn) {
+  v = warp_max(v);
+  double* buf = red + (turn & 1) * 32;
+  ++turn;
+  if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return warp_max(buf[threadIdx.x & 31]);
+}
+
+template <int NN> struct EigSmem {
+  static constexpr int LD = NN + 1;
+  static constexpr size_t a = 0;                                           // double [NN][LD]
+  static constexpr size_t z = a + sizeof(double) * NN * LD;                // double [NN][kZld]
+  static constexpr size_t vec = z + sizeof(double) * NN * kZld;            // v, w, d, e, e2, beta: 6 x double[NN]
+  static constexpr size_t lam = vec + sizeof(double) * 6 * NN;             // double [kEigMaxR]
+  static constexpr size_t red = lam + sizeof(double) * kEigMaxR;           // double [2][32]
+  static constexpr size_t cst = red + sizeof(double) * 64;                 // int [kEigMaxR] group start; int flags[4]
+  static constexpr size_t total = cst + sizeof(int) * (kEigMaxR + 4);
+};
+
+// eigenvalues of T below x (Sturm count) by the three-term recurrence of the leading principal
+// minors, p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}: one dependent multiply-add per step.  A zero
+// minor takes the sign opposite to its predecessor; both running minors are rescaled by a power of
+// two every eight steps, which changes no sign.
+template <int NN>
+__device__ __forceinline__ int sturm_count(const double* __restrict__ dd, const double* __restrict__ e2, double x) {
+  double p2 = 1.0, p1 = dd[0] - x;
+  bool neg1 = p1 < 0.0 || p1 == 0.0;                            // sign of p_1 (zero counts as a change from p_0 = 1)
+  int cnt = neg1;
+#pragma unroll 8
+  for (int i = 1; i < NN; ++i) {
+    const double p = fma(dd[i] - x, p1, -(e2[i - 1] * p2));
+    const bool neg = p == 0.0 ? !neg1 : p < 0.0;
+    cnt += neg != neg1;
+    neg1 = neg;
+    p2 = p1; p1 = p;
+    if ((i & 7) == 7) {
+      const double mx = fmax(fabs(p1), fabs(p2));
+      if (mx > 1.0e90) { p1 *= 1.0e-90; p2 *= 1.0e-90; }
+      else if (mx < 1.0e-90) { p1 *= 1.0e90; p2 *= 1.0e90; }
+    }
+  }
+  return cnt;
+}
+
+template <int NN>
+__global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+                                                             float* __restrict__ Fout, double* __restrict__ lam_out) {
+  using S = EigSmem<NN>;
+  constexpr int LD = S::LD;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* A = reinterpret_cast<double*>(smem_raw + S::a);
+  double* Z = reinterpret_cast<double*>(smem_raw + S::z);
+  double* v = reinterpret_cast<double*>(smem_raw + S::vec);
+  double* w = v + NN;
+  double* dd = w + NN;
+  double* ee = dd + NN;
+  double* e2 = ee + NN;
+  double* beta = e2 + NN;
+  double* lam = reinterpret_cast<double*>(smem_raw + S::lam);
+  double* red = reinterpret_cast<double*>(smem_raw + S::red);
+  int* cstart = reinterpret_cast<int*>(smem_raw + S::cst);
+  int* flags = cstart + kEigMaxR;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const double* Mi = Min + (i64)blockIdx.x * stride;
+  float* Fo = Fout + (i64)blockIdx.x * NN * r;
+  int turn = 0;
+
+  // ---- load, symmetrise, scale to max |a_ij| = 1 ---------------------------------------------------
+  double amax = 0.0;
+  for (int e = tid; e < NN * NN; e += kEigThreads) {
+    const int i = e / NN, j = e % NN;
+    const double a = 0.5 * (Mi[e] + Mi[j * NN + i]);
+    A[i * LD + j] = a;
+    amax = fmax(amax, fabs(a));
+  }
+  const double scale = cta_max(amax, red, turn);
+  if (!(scale > 0.0) || !(scale < 1.0e300)) {
+    // zero matrix: eigenvalues 0, unit vectors; anything non-finite is left to the error checks downstream
+    for (int e = tid; e < NN * r; e += kEigThreads) Fo[e] = (scale_mode == 1 && e / r == e % r) ? 1.f : 0.f;
+    if (lam_out) for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = 0.0;
+    return;
+  }
+  const double inv_scale = 1.0 / scale;
+  for (int e = tid; e < NN * NN; e += kEigThreads) A[(e / NN) * LD + e % NN] *= inv_scale;
+  __syncthreads();
+
+#ifdef SPR_EIG_TIMING
+  const long long T0 = clock64();
+#endif
+  // ---- 1. Householder tridiagonalisation ----------------------------------------------------------------
+  // kTpr threads per row of the trailing block, interleaved columns
+  const int row = tid / kTpr, h = tid % kTpr;
+  for (int k = 0; k < NN - 2; ++k) {
+    const int m = NN - k - 1;                                   // order of the trailing block
+    double part = 0.0;
+    if (tid >= 1 && tid < m) { const double x = A[(k + 1 + tid) * LD + k]; part = x * x; }
+    const double below2 = cta_sum(part, red, turn);             // squares below the subdiagonal
+    const double x0 = A[(k + 1) * LD + k];
+    if (!(below2 > 0.0)) {                                      // column already reduced (uniform branch)
+      if (tid == 0) { ee[k] = x0; beta[k] = 0.0; }
+      continue;
+    }
+    const double alpha = sqrt(below2 + x0 * x0);
+    const double sgn = x0 >= 0.0 ? 1.0 : -1.0;
+    const double b = 1.0 / (alpha * (alpha + fabs(x0)));        // 2 / ||v||^2 with v = x + sgn alpha e_1
+    if (tid < m) v[tid] = tid == 0 ? x0 + sgn * alpha : A[(k + 1 + tid) * LD + k];
+    __syncthreads();
+    // p = b * A22 v
+    double acc = 0.0;
+    if (row < m) {
+      const double* ar = A + (k + 1 + row) * LD + k + 1;
+      double acc1 = 0.0;
+      int c = h;
+      for (; c + kTpr < m; c += 2 * kTpr) { acc = fma(ar[c], v[c], acc); acc1 = fma(ar[c + kTpr], v[c + kTpr], acc1); }
+      if (c < m) acc = fma(ar[c], v[c], acc);
+      acc += acc1;
+    }
+#pragma unroll
+    for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    const double p_row = b * acc;
+    const double pv = cta_sum((h == 0 && row < m) ? p_row * v[row] : 0.0, red, turn);
+    if (h == 0 && row < m) w[row] = p_row - 0.5 * b * pv * v[row];
+    __syncthreads();
+    // A22 <- A22 - v w^T - w v^T
+    if (row < m) {
+      double* ar = A + (k + 1 + row) * LD + k + 1;
+      const double vi = v[row], wi = w[row];
+      for (int c = h; c < m; c += kTpr) ar[c] -= vi * w[c] + wi * v[c];
+    }
+    if (tid < m) A[(k + 1 + tid) * LD + k] = v[tid];            // reflector k lives in column k below the diagonal
+    if (tid == 0) { ee[k] = -sgn * alpha; beta[k] = b; }
+    __syncthreads();
+  }
+#ifdef SPR_EIG_TIMING
+  const long long T1 = clock64();
+#endif
+  if (tid == 0) { ee[NN - 2] = A[(NN - 1) * LD + NN - 2]; ee[NN - 1] = 0.0; beta[NN - 2] = 0.0; beta[NN - 1] = 0.0; }
+  if (tid < NN) dd[tid] = A[tid * LD + tid];
+  __syncthreads();
+  if (tid < NN) e2[tid] = ee[tid] * ee[tid];
+  double g = 0.0;
+  if (tid < NN) g = fabs(dd[tid]) + fabs(ee[tid]) + (tid > 0 ? fabs(ee[tid - 1]) : 0.0);
+  const double tnorm = cta_max(g, red, turn);                   // Gershgorin bound on |lambda|; also makes e2[] visible
+
+  // ---- 2. multi-section: 16 threads per eigenvalue, 17-fold interval reduction per pass ----------------
+  {
+    const int j = tid >> 4, t = tid & 15;                       // eigenvalue (j+1)-th largest, probe point t
+    const bool active = j < r;
+    const int kth = NN - 1 - j;                                 // ascending index
+    double lo = -tnorm, hi = tnorm;
+    for (int it = 0; it < 11; ++it) {
+      const double wdt = (hi - lo) * (1.0 / 17.0);
+      const double x = lo + wdt * (double)(t + 1);
+      const bool below = active && sturm_count<NN>(dd, e2, x) <= kth;   // eigenvalue kth is >= x
+      const unsigned bal = __ballot_sync(0xffffffffu, below);
+      const int s = __popc((bal >> (lane & 16)) & 0xFFFFu);     // probes (of this group of 16 lanes) still below the eigenvalue
+      const double nlo = lo + wdt * (double)s;
+      hi = s < 16 ? lo + wdt * (double)(s + 1) : hi;
+      lo = nlo;
+    }
+    if (active && t == 0) lam[j] = 0.5 * (lo + hi);
+  }
+  __syncthreads();
+#ifdef SPR_EIG_TIMING
+  const long long T2 = clock64();
+#endif
+
+  // ---- 3. inverse iteration: thread j computes eigenvector j of T ------------------------------------
+  if (tid < r) {
+    const double shift = lam[tid];
+    const double tiny = tnorm * 1.0e-15;
+    double pinv[NN], u1[NN], u2[NN], mul[NN];                  // pivots^-1, two superdiagonals of U, multipliers
+    unsigned long long swp[(NN + 63) / 64];
+#pragma unroll
+    for (int q = 0; q < (NN + 63) / 64; ++q) swp[q] = 0ull;
+    double acur = dd[0] - shift, ucur = ee[0];                 // current row i: diagonal and superdiagonal entries
+    for (int i = 0; i < NN - 1; ++i) {
+      const double sub = ee[i];
+      const double anext = dd[i + 1] - shift, unext = ee[i + 1];   // ee[NN-1] = 0
+      if (fabs(acur) >= fabs(sub)) {
+        double piv = acur;
+        if (fabs(piv) <= tiny) piv = piv >= 0.0 ? tiny : -tiny;
+        const double ip = 1.0 / piv;
+        const double m = sub * ip;
+        pinv[i] = ip; u1[i] = ucur; u2[i] = 0.0; mul[i] = m;
+        acur = anext - m * ucur;
+        ucur = unext;
+      } else {
+        const double ip = 1.0 / sub;
+        const double m = acur * ip;                             // rows i and i+1 swapped
+        swp[i >> 6] |= 1ull << (i & 63);
+        pinv[i] = ip; u1[i] = anext; u2[i] = unext; mul[i] = m;
+        acur = ucur - m * anext;
+        ucur = -m * unext;
+      }
+    }
+    {
+      double piv = acur;
+      if (fabs(piv) <= tiny) piv = piv >= 0.0 ? tiny : -tiny;
+      pinv[NN - 1] = 1.0 / piv; u1[NN - 1] = 0.0; u2[NN - 1] = 0.0; mul[NN - 1] = 0.0;
+    }
+    double* z = Z + tid;                                        // z_i = z[i * kZld]
+    for (int i = 0; i < NN; ++i) z[i * kZld] = hash_unit(i, tid);
+    for (int it = 0; it < 3; ++it) {
+      double zi = z[0];
+#pragma unroll 4
+      for (int i = 0; i < NN - 1; ++i) {                        // forward elimination
+        const double zn = z[(i + 1) * kZld];
+        const bool sw = (swp[i >> 6] >> (i & 63)) & 1ull;
+        const double keep = sw ? zn : zi, other = sw ? zi : zn;
+        z[i * kZld] = keep;
+        zi = fma(-mul[i], keep, other);
+      }
+      double z1 = zi * pinv[NN - 1], z2 = 0.0;                  // back substitution
+      z[(NN - 1) * kZld] = z1;
+      double big = fabs(z1);
+#pragma unroll 4
+      for (int i = NN - 2; i >= 0; --i) {
+        const double zz = (z[i * kZld] - u1[i] * z1 - u2[i] * z2) * pinv[i];
+        z[i * kZld] = zz;
+        big = fmax(big, fabs(zz));
+        z2 = z1; z1 = zz;
+      }
+      const double sc = big > 0.0 ? 1.0 / big : 1.0;
+      for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
+    }
+    double nn = 0.0;
+    for (int i = 0; i < NN; ++i) nn = fma(z[i * kZld], z[i * kZld], nn);
+    const double sc = nn > 0.0 ? rsqrt(nn) : 0.0;
+    for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
+  }
+  __syncthreads();
+#ifdef SPR_EIG_TIMING
+  const long long T3 = clock64();
+#endif
+
+  // ---- 4. groups of close eigenvalues: modified Gram-Schmidt, one warp per group ----------------------
+  if (tid == 0) {
+    const double gap = 1.0e-3 * tnorm;
+    int start = 0;
+    for (int j = 0; j < r; ++j) {
+      if (j > 0 && fabs(lam[j - 1] - lam[j]) >= gap) start = j;
+      cstart[j] = start;
+    }
+    flags[0] = 0;
+  }
+  __syncthreads();
+  {
+    int group = 0;
+    for (int j0 = 0; j0 < r; ++group) {
+      int j1 = j0;
+      while (j1 + 1 < r && cstart[j1 + 1] == j0) ++j1;
+      if (j1 > j0 && (group & 31) == warp) {
+        for (int a = j0 + 1; a <= j1; ++a) {
+          for (int bq = j0; bq < a; ++bq) {
+            double dot = 0.0;
+            for (int i = lane; i < NN; i += 32) dot = fma(Z[i * kZld + bq], Z[i * kZld + a], dot);
+            dot = warp_sum(dot);
+            for (int i = lane; i < NN; i += 32) Z[i * kZld + a] -= dot * Z[i * kZld + bq];
+            __syncwarp();
+          }
+          double nn = 0.0;
+          for (int i = lane; i < NN; i += 32) nn = fma(Z[i * kZld + a], Z[i * kZld + a], nn);
+          nn = warp_sum(nn);
+          const double sc = nn > 0.0 ? rsqrt(nn) : 0.0;
+          for (int i = lane; i < NN; i += 32) Z[i * kZld + a] *= sc;
+          __syncwarp();
+        }
+      }
+      j0 = j1 + 1;
+    }
+  }
+  __syncthreads();
+#ifdef SPR_EIG_TIMING
+  const long long T4 = clock64();
+#endif
+
+  // ---- 5. Rayleigh quotients, residuals, orthogonality -------------------------------------------------
+  bool bad = false;
+  if (tid < r) {
+    const double* z = Z + tid;
+    double num = 0.0, den = 0.0;
+    for (int i = 0; i < NN; ++i) {
+      const double zi = z[i * kZld];
+      double t = dd[i] * zi;
+      if (i > 0) t = fma(ee[i - 1], z[(i - 1) * kZld], t);
+      if (i + 1 < NN) t = fma(ee[i], z[(i + 1) * kZld], t);
+      num = fma(zi, t, num);
+      den = fma(zi, zi, den);
+    }
+    const double rq = den > 0.0 ? num / den : 0.0;
+    double res = 0.0;
+    for (int i = 0; i < NN; ++i) {
+      const double zi = z[i * kZld];
+      double t = (dd[i] - rq) * zi;
+      if (i > 0) t = fma(ee[i - 1], z[(i - 1) * kZld], t);
+      if (i + 1 < NN) t = fma(ee[i], z[(i + 1) * kZld], t);
+      res = fmax(res, fabs(t));
+    }
+    lam[tid] = rq;
+    bad = !(res <= 1.0e-7 * tnorm) || !(fabs(den - 1.0) <= 1.0e-7);
+  }
+  for (int pr = tid; pr < r * r; pr += kEigThreads) {
+    const int a = pr / r, bq = pr % r;
+    if (a < bq) {
+      double d0 = 0.0, d1 = 0.0;
+      for (int i = 0; i < NN; i += 2) {
+        d0 = fma(Z[i * kZld + a], Z[i * kZld + bq], d0);
+        d1 = fma(Z[(i + 1) * kZld + a], Z[(i + 1) * kZld + bq], d1);
+      }
+      bad |= !(fabs(d0 + d1) <= 1.0e-7);
+    }
+  }
+  if (bad) flags[0] = 1;
+  __syncthreads();
+  if (flags[0]) {
+    if (tid == 0) Fo[0] = __int_as_float(0x7fc00000);           // marked for the Jacobi kernel
+#ifdef SPR_EIG_TIMING
+    if (tid == 0) printf("eig matrix %d marked for Jacobi\n", (int)blockIdx.x);
+#endif
+    return;
+  }
+#ifdef SPR_EIG_TIMING
+  const long long T5 = clock64();
+#endif
+
+  // ---- 6. back-transformation z <- H_0 ... H_{n-3} z, scaling, output -------------------------------------
+  {
+    constexpr int tpv = 16;                                      // threads per vector (1024 threads cover 64 vectors)
+    const int j = tid / tpv, q = tid % tpv;
+    const bool active = j < r;
+    for (int k = NN - 3; k >= 0; --k) {
+      const double bk = beta[k];
+      if (bk == 0.0) continue;                                   // uniform
+      double dot = 0.0;
+      if (active)
+        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[i * LD + k], Z[i * kZld + j], dot);
+#pragma unroll
+      for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      const double f = bk * dot;
+      if (active)
+        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[i * LD + k];
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+  double part = tid < r ? fmax(lam[tid], 0.0) : 0.0;
+  const double mean = cta_sum(part, red, turn) / (double)r;
+#ifdef SPR_EIG_TIMING
+  if (tid == 0 && blockIdx.x == 0)
+    printf("eig n=%d r=%d cycles: householder %lld bisection %lld inverse-it %lld mgs %lld check %lld backtransform %lld\n", NN, r,
+           T1 - T0, T2 - T1, T3 - T2, T4 - T3, T5 - T4, clock64() - T5);
+#endif
+  if (lam_out)
+    for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = j < r ? lam[j] * scale : 0.0;
+  for (int e = tid; e < NN * r; e += kEigThreads) {
+    const int rw = e / r, j = e % r;
+    double sc = 1.0;
+    if (scale_mode == 0) sc = mean > 0.0 ? sqrt(fmax(lam[j], 0.0) / mean) : 0.0;
+    Fo[e] = (float)(Z[rw * kZld + j] * sc);
+  }
+}
+
+// Cyclic Jacobi in float64 (A in shared memory, one CTA per matrix, in-place 2x2 block updates):
+// slow and unconditionally robust; processes only the matrices that the kernel above marked.
+template <int NN>
+__global__ void __launch_bounds__(1024) k_jacobi_eig_f64(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+                                                         float* __restrict__ Fout, double* __restrict__ lam_out) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* A = reinterpret_cast<double*>(smem_raw);                 // [NN][NN+1]
+  float* V = reinterpret_cast<float*>(A + NN * (NN + 1));          // [NN][NN+1]
+  double* cs = reinterpret_cast<double*>(V + NN * (NN + 1) + (NN & 1));   // [NN/2][2]
+  int* pq = reinterpret_cast<int*>(cs + NN);                        // [NN/2][2]
+  double* red = reinterpret_cast<double*>(pq + NN);                 // [34]
+  __shared__ int s_rank[NN];
+  __shared__ int s_marked;
+  constexpr int LD = NN + 1;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  if (tid == 0) s_marked = isnan(Fout[(i64)blockIdx.x * NN * r]);
+  __syncthreads();
+  if (!s_marked) return;
+  const double* Mi = Min + (i64)blockIdx.x * stride;
+  for (int e = tid; e < NN * NN; e += nt) {
+    const int i = e / NN, j = e % NN;
+    A[i * LD + j] = 0.5 * (Mi[e] + Mi[j * NN + i]);
+    V[i * LD + j] = i == j ? 1.f : 0.f;
+  }
+  __syncthreads();
+  double fro = 0.0;
+  for (int e = tid; e < NN * NN; e += nt) { const double a = A[(e / NN) * LD + e % NN]; fro += a * a; }
+  fro = block_sum(fro, red);
+  const double tol = fro * 1e-26;
+  for (int sweep = 0; sweep < 20; ++sweep) {
+    double off = 0.0;
+    for (int e = tid; e < NN * NN; e += nt) {
+      const int i = e / NN, j = e % NN;
+      if (i != j) { const double a = A[i * LD + j]; off += a * a; }
+    }
+    off = block_sum(off, red);
+    if (!(off > tol)) break;
+    for (int round = 0; round < NN - 1; ++round) {
+      if (tid < NN / 2) {
+        int p, q;
+        if (tid == 0) { p = NN - 1; q = round; }
+        else { p = (round + tid) % (NN - 1); q = (round - tid + (NN - 1)) % (NN - 1); }
+        if (p > q) { const int t = p; p = q; q = t; }
+        const double app = A[p * LD + p], aqq = A[q * LD + q], apq = A[p * LD + q];
+        double c = 1.0, s = 0.0;
+        if (fabs(apq) > 1e-300 && apq * apq > 1e-34 * fabs(app * aqq) ) {
+          const double tau = (aqq - app) / (2.0 * apq);
+          const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+          c = 1.0 / sqrt(1.0 + t * t);
+          s = t * c;
+        }
+        pq[2 * tid] = p; pq[2 * tid + 1] = q;
+        cs[2 * tid] = c; cs[2 * tid + 1] = s;
+      }
+      __syncthreads();
+      for (int e = tid; e < (NN / 2) * (NN / 2); e += nt) {
+        const int ki = e / (NN / 2), kj = e % (NN / 2);
+        const int pi = pq[2 * ki], qi = pq[2 * ki + 1], pj = pq[2 * kj], qj = pq[2 * kj + 1];
+        const double ci = cs[2 * ki], si = cs[2 * ki + 1], cj = cs[2 * kj], sj = cs[2 * kj + 1];
+        const double a00 = A[pi * LD + pj], a01 = A[pi * LD + qj], a10 = A[qi * LD + pj], a11 = A[qi * LD + qj];
+        // rows: J_i^T from the left
+        const double b00 = ci * a00 - si * a10, b01 = ci * a01 - si * a11;
+        const double b10 = si * a00 + ci * a10, b11 = si * a01 + ci * a11;
+        // columns: J_j from the right
+        A[pi * LD + pj] = cj * b00 - sj * b01; A[pi * LD + qj] = sj * b00 + cj * b01;
+        A[qi * LD + pj] = cj * b10 - sj * b11; A[qi * LD + qj] = sj * b10 + cj * b11;
+      }
+      for (int e = tid; e < NN * (NN / 2); e += nt) {
+        const int i = e / (NN / 2), kj = e % (NN / 2);
+        const int pj = pq[2 * kj], qj = pq[2 * kj + 1];
+        const float cj = (float)cs[2 * kj], sj = (float)cs[2 * kj + 1];
+        const float vp = V[i * LD + pj], vq = V[i * LD + qj];
+        V[i * LD + pj] = cj * vp - sj * vq;
+        V[i * LD + qj] = sj * vp + cj * vq;
+      }
+      __syncthreads();
+    }
+  }
+  // rank eigenvalues descending (ties by index), scale and emit the leading r
+  if (tid < NN) {
+    const double li = A[tid * LD + tid];
+    int rank = 0;
+    for (int j = 0; j < NN; ++j) {
+      const double lj = A[j * LD + j];
+      rank += (lj > li) || (lj == li && j < tid);
+    }
+    s_rank[tid] = rank;
+    if (lam_out) lam_out[(i64)blockIdx.x * NN + rank] = li;
+  }
+  __syncthreads();
+  double part = 0.0;
+  if (tid < NN && s_rank[tid] < r) part = fmax(A[tid * LD + tid], 0.0);
+  const double mean = block_sum(part, red) / (double)r;
+  for (int e = tid; e < NN * NN; e += nt) {
+    const int i = e / NN, col = e % NN;     // column `col` of V is the eigenvector of A[col][col]
+    const int rank = s_rank[col];
+    if (rank < r) {
+      float sc = 1.f;
+      if (scale_mode == 0) sc = mean > 0.0 ? (float)sqrt(fmax(A[col * LD + col], 0.0) / mean) : 0.f;
+      Fout[(i64)blockIdx.x * NN * r + (i64)i * r + rank] = V[i * LD + col] * sc;
+    }
+  }
+}
+
+size_t jacobi64_smem(int n) {
+  return (size_t)n * (n + 1) * 8 + (size_t)(n * (n + 1) + (n & 1)) * 4 + n * 8 + n * 4 + 34 * 8 + 16;
+}
+
+}  // namespace
+
+cudaError_t init_eigen() {
+  cudaError_t e = cudaFuncSetAttribute(k_eig_tridiag<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<128>::total);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_eig_tridiag<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<64>::total);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_jacobi_eig_f64<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(128));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_jacobi_eig_f64<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(64));
+}
+
+// Min: `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart; r <= 64 leading pairs.
+// scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda) (feature map of Section 4.1);
+// 1: orthonormal columns (basis of Eq. 9).  Fout [batch][n][r]; lam_out [batch][n] or null (entries >= r are 0).
+void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout, double* lam_out,
+                    cudaStream_t st) {
+  if (n == 128) {
+    k_eig_tridiag<128><<<batch, kEigThreads, EigSmem<128>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  } else {
+    k_eig_tridiag<64><<<batch, kEigThreads, EigSmem<64>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    k_jacobi_eig_f64<64><<<batch, 1024, jacobi64_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+  }
+}
+
+}  // namespace spr

@@ -5,15 +5,16 @@
 namespace spr {
 
 // ---- partition.cu -------------------------------------------------------------
-cudaError_t init_jacobi();
 cudaError_t init_group_sort();
 void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
                         double* Mout, cudaStream_t st);
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
-// Min: `batch` symmetric n x n matrices, `stride` doubles apart
-// precise: float64 shared-memory variant (float32 tensors); otherwise float32 in registers
-void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
-                       double* lam_out, cudaStream_t st);
+// eigen.cu: leading r <= 64 eigenpairs of `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart.
+// scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda); 1: orthonormal columns.
+// Fout [batch][n][r]; lam_out [batch][n] or null.
+cudaError_t init_eigen();
+void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout, double* lam_out,
+                    cudaStream_t st);
 void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,

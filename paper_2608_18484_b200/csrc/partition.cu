@@ -116,277 +116,6 @@ void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d
 }
 
 // =============================================================================
-// Batched symmetric eigen-decomposition by parallel cyclic Jacobi, one CTA per
-// matrix (n = 64 or 128), float32, register resident.
-//   threads [0,n)  : thread i holds row i of A in registers
-//   threads [n,2n) : thread n+i holds row i of V (accumulated rotations)
-// The round-robin tournament is realised by MOVING rows and columns so that the
-// pairs of a round are always the adjacent positions (2k, 2k+1): a row rotation
-// is then a shuffle between neighbouring lanes, a column rotation touches two
-// adjacent registers, and the permutation between rounds is a compile-time
-// renaming of registers for the columns and one trip through shared memory for
-// the rows of A.  Output: the leading r eigenvectors, scaled by
-// sqrt(lambda_i / mean retained lambda) (the feature map F of Section 4.1) or
-// unscaled (the orthonormal basis Psi_r of Eq. 9).
-// =============================================================================
-__host__ __device__ constexpr int rr_next(int pos, int n) {
-  // where the content of position `pos` goes for the next round (position 0 is fixed; the even
-  // positions shift up, the last one turns around, the odd positions shift down)
-  return pos == 0 ? 0 : pos == 1 ? 2 : (pos % 2 == 0) ? (pos / 2 < n / 2 - 1 ? pos + 2 : n - 1) : pos - 2;
-}
-
-template <int NN>
-__global__ void __launch_bounds__(2 * NN) k_jacobi_eig(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
-                                                      float* __restrict__ Fout, double* __restrict__ lam_out) {
-  constexpr int LD = NN + 4;
-  extern __shared__ __align__(16) float sm_j[];
-  float* rows = sm_j;                                   // [2][NN][LD] rows of A by position, double buffered over rounds
-  float2* cs = reinterpret_cast<float2*>(rows + 2 * NN * LD);   // [NN/2] rotation of every pair
-  __shared__ float red[34];
-  __shared__ int s_rank[NN];
-  const int tid = threadIdx.x;
-  const bool is_a = tid < NN;
-  const int i = is_a ? tid : tid - NN;
-  const double* Mi = Min + (i64)blockIdx.x * stride;
-  float a[NN];                                          // row i of A (A threads) or of V (V threads)
-  if (is_a) {
-#pragma unroll
-    for (int c = 0; c < NN; ++c) a[c] = (float)(0.5 * (Mi[(i64)i * NN + c] + Mi[(i64)c * NN + i]));
-#pragma unroll
-    for (int c = 0; c < NN; c += 4) *reinterpret_cast<float4*>(rows + i * LD + c) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
-  } else {
-#pragma unroll
-    for (int c = 0; c < NN; ++c) a[c] = c == i ? 1.f : 0.f;
-  }
-  float fro = 0.f;
-  if (is_a) {
-#pragma unroll
-    for (int c = 0; c < NN; ++c) fro = fmaf(a[c], a[c], fro);
-  }
-  fro = block_sum(fro, red);                            // contains __syncthreads: rows[] is complete
-  // stop once the off-diagonal mass is below 1e-8 of the squared norm (off/||A|| < 1e-4; the sweep
-  // that got there has already squared the previous level), or when a sweep no longer halves it
-  const float tol = fro * 1e-8f;
-  float prev_off = 3.0e38f;
-  // An A thread keeps its matrix row for the whole run; `pos` is the position of that row (and of
-  // the matching column) in the round-robin order.  Columns move physically inside the register
-  // arrays, so that every register index is a compile-time constant.
-  int pos = i;
-  for (int sweep = 0; sweep < 16; ++sweep) {
-    float off = 0.f;
-    if (is_a) {
-#pragma unroll
-      for (int c = 0; c < NN; ++c) off = fmaf(a[c], a[c], off);
-      const float dg = rows[pos * LD + pos];
-      off -= dg * dg;
-    }
-    off = block_sum(off, red);
-    if (!(off > tol) || (sweep >= 4 && off > 0.5f * prev_off)) break;
-    prev_off = off;
-    for (int round = 0; round < NN - 1; ++round) {
-      float c = 1.f, s = 0.f;
-      if (is_a) {
-        const int p = pos & ~1;                           // pair (p, p+1)
-        const float app = rows[p * LD + p], apq = rows[p * LD + p + 1], aqq = rows[(p + 1) * LD + p + 1];
-        if (apq != 0.f) {
-          const float tau = (aqq - app) / (2.f * apq);
-          const float t = copysignf(1.f, tau) / (fabsf(tau) + sqrtf(fmaf(tau, tau, 1.f)));   // -> 0 when tau overflows
-          c = rsqrtf(fmaf(t, t, 1.f));
-          s = t * c;
-        }
-        if (!(pos & 1)) cs[pos >> 1] = make_float2(c, s);
-      }
-      __syncthreads();                                  // cs[] visible
-      if (is_a) {
-        // rows: (a_p, a_q) <- (c a_p - s a_q, s a_p + c a_q); the partner row was stored by its owner at the
-        // end of the previous round
-        const float ss = (pos & 1) ? s : -s;
-        const float* prow = rows + (pos ^ 1) * LD;
-#pragma unroll
-        for (int col = 0; col < NN; col += 4) {
-          const float4 b = *reinterpret_cast<const float4*>(prow + col);
-          a[col] = fmaf(ss, b.x, c * a[col]); a[col + 1] = fmaf(ss, b.y, c * a[col + 1]);
-          a[col + 2] = fmaf(ss, b.z, c * a[col + 2]); a[col + 3] = fmaf(ss, b.w, c * a[col + 3]);
-        }
-      }
-      // columns (A and V alike): (x_p, x_q) <- (c x_p - s x_q, s x_p + c x_q), then move to the next round's positions
-      float nx[NN];
-#pragma unroll
-      for (int k = 0; k < NN / 2; ++k) {
-        const float2 r2 = cs[k];
-        const float x = a[2 * k], y = a[2 * k + 1];
-        nx[rr_next(2 * k, NN)] = r2.x * x - r2.y * y;
-        nx[rr_next(2 * k + 1, NN)] = fmaf(r2.y, x, r2.x * y);
-      }
-#pragma unroll
-      for (int col = 0; col < NN; ++col) a[col] = nx[col];
-      rows = (rows == sm_j) ? sm_j + NN * LD : sm_j;     // the other buffer: nobody reads it during this round
-      if (is_a) {
-        pos = rr_next(pos, NN);                         // the row moves as well
-#pragma unroll
-        for (int col = 0; col < NN; col += 4)
-          *reinterpret_cast<float4*>(rows + pos * LD + col) = make_float4(a[col], a[col + 1], a[col + 2], a[col + 3]);
-      }
-      __syncthreads();                                  // rows of the new round complete; every cs[] read done
-    }
-  }
-  // eigenvalue of position c = A[c][c]; eigenvector = column c of V.  Rank descending (ties by position).
-  __syncthreads();
-  float lam_i = 0.f;
-  if (is_a) lam_i = rows[i * LD + i];                   // by position: thread i reports position i
-  __syncthreads();
-  float* lam_s = reinterpret_cast<float*>(cs);          // NN floats fit in the NN/2 float2 slots
-  if (is_a) lam_s[i] = lam_i;
-  __syncthreads();
-  if (is_a) {
-    int rank = 0;
-    for (int j = 0; j < NN; ++j) { const float lj = lam_s[j]; rank += (lj > lam_i) || (lj == lam_i && j < i); }
-    s_rank[i] = rank;
-    if (lam_out) lam_out[(i64)blockIdx.x * NN + rank] = (double)lam_i;
-  } else {
-#pragma unroll
-    for (int c = 0; c < NN; c += 4) *reinterpret_cast<float4*>(rows + i * LD + c) = make_float4(a[c], a[c + 1], a[c + 2], a[c + 3]);
-  }
-  __syncthreads();
-  float part = (is_a && s_rank[i] < r) ? fmaxf(lam_i, 0.f) : 0.f;
-  const float mean = block_sum(part, red) / (float)r;
-  for (int e = tid; e < NN * NN; e += 2 * NN) {
-    const int row = e / NN, col = e % NN;
-    const int rank = s_rank[col];
-    if (rank < r) {
-      float sc = 1.f;
-      if (scale_mode == 0) sc = mean > 0.f ? sqrtf(fmaxf(lam_s[col], 0.f) / mean) : 0.f;
-      Fout[(i64)blockIdx.x * NN * r + (i64)row * r + rank] = rows[row * LD + col] * sc;
-    }
-  }
-}
-
-// Float64 variant (A in shared memory, one CTA per matrix, in-place 2x2 block updates):
-// slower, used when the caller's tensors are float32 and the 1e-5 output tolerance
-// leaves no room for a float32 eigen-basis.
-template <int NN>
-__global__ void __launch_bounds__(1024) k_jacobi_eig_f64(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
-                                                    float* __restrict__ Fout, double* __restrict__ lam_out) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* A = reinterpret_cast<double*>(smem_raw);                 // [NN][NN+1]
-  float* V = reinterpret_cast<float*>(A + NN * (NN + 1));          // [NN][NN+1]
-  double* cs = reinterpret_cast<double*>(V + NN * (NN + 1) + (NN & 1));   // [NN/2][2]
-  int* pq = reinterpret_cast<int*>(cs + NN);                        // [NN/2][2]
-  double* red = reinterpret_cast<double*>(pq + NN);                 // [34]
-  __shared__ int s_rank[NN];
-  constexpr int LD = NN + 1;
-  const int tid = threadIdx.x, nt = blockDim.x;
-  const double* Mi = Min + (i64)blockIdx.x * stride;
-  for (int e = tid; e < NN * NN; e += nt) {
-    const int i = e / NN, j = e % NN;
-    A[i * LD + j] = 0.5 * (Mi[e] + Mi[j * NN + i]);
-    V[i * LD + j] = i == j ? 1.f : 0.f;
-  }
-  __syncthreads();
-  double fro = 0.0;
-  for (int e = tid; e < NN * NN; e += nt) { const double a = A[(e / NN) * LD + e % NN]; fro += a * a; }
-  fro = block_sum(fro, red);
-  const double tol = fro * 1e-26;
-  for (int sweep = 0; sweep < 20; ++sweep) {
-    double off = 0.0;
-    for (int e = tid; e < NN * NN; e += nt) {
-      const int i = e / NN, j = e % NN;
-      if (i != j) { const double a = A[i * LD + j]; off += a * a; }
-    }
-    off = block_sum(off, red);
-    if (off <= tol) break;
-    for (int round = 0; round < NN - 1; ++round) {
-      if (tid < NN / 2) {
-        int p, q;
-        if (tid == 0) { p = NN - 1; q = round; }
-        else { p = (round + tid) % (NN - 1); q = (round - tid + (NN - 1)) % (NN - 1); }
-        if (p > q) { const int t = p; p = q; q = t; }
-        const double app = A[p * LD + p], aqq = A[q * LD + q], apq = A[p * LD + q];
-        double c = 1.0, s = 0.0;
-        if (fabs(apq) > 1e-300 && apq * apq > 1e-34 * fabs(app * aqq) ) {
-          const double tau = (aqq - app) / (2.0 * apq);
-          const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-          c = 1.0 / sqrt(1.0 + t * t);
-          s = t * c;
-        }
-        pq[2 * tid] = p; pq[2 * tid + 1] = q;
-        cs[2 * tid] = c; cs[2 * tid + 1] = s;
-      }
-      __syncthreads();
-      for (int e = tid; e < (NN / 2) * (NN / 2); e += nt) {
-        const int ki = e / (NN / 2), kj = e % (NN / 2);
-        const int pi = pq[2 * ki], qi = pq[2 * ki + 1], pj = pq[2 * kj], qj = pq[2 * kj + 1];
-        const double ci = cs[2 * ki], si = cs[2 * ki + 1], cj = cs[2 * kj], sj = cs[2 * kj + 1];
-        const double a00 = A[pi * LD + pj], a01 = A[pi * LD + qj], a10 = A[qi * LD + pj], a11 = A[qi * LD + qj];
-        // rows: J_i^T from the left
-        const double b00 = ci * a00 - si * a10, b01 = ci * a01 - si * a11;
-        const double b10 = si * a00 + ci * a10, b11 = si * a01 + ci * a11;
-        // columns: J_j from the right
-        A[pi * LD + pj] = cj * b00 - sj * b01; A[pi * LD + qj] = sj * b00 + cj * b01;
-        A[qi * LD + pj] = cj * b10 - sj * b11; A[qi * LD + qj] = sj * b10 + cj * b11;
-      }
-      for (int e = tid; e < NN * (NN / 2); e += nt) {
-        const int i = e / (NN / 2), kj = e % (NN / 2);
-        const int pj = pq[2 * kj], qj = pq[2 * kj + 1];
-        const float cj = (float)cs[2 * kj], sj = (float)cs[2 * kj + 1];
-        const float vp = V[i * LD + pj], vq = V[i * LD + qj];
-        V[i * LD + pj] = cj * vp - sj * vq;
-        V[i * LD + qj] = sj * vp + cj * vq;
-      }
-      __syncthreads();
-    }
-  }
-  // rank eigenvalues descending (ties by index), scale and emit the leading r
-  if (tid < NN) {
-    const double li = A[tid * LD + tid];
-    int rank = 0;
-    for (int j = 0; j < NN; ++j) {
-      const double lj = A[j * LD + j];
-      rank += (lj > li) || (lj == li && j < tid);
-    }
-    s_rank[tid] = rank;
-    if (lam_out) lam_out[(i64)blockIdx.x * NN + rank] = li;
-  }
-  __syncthreads();
-  double part = 0.0;
-  if (tid < NN && s_rank[tid] < r) part = fmax(A[tid * LD + tid], 0.0);
-  const double mean = block_sum(part, red) / (double)r;
-  for (int e = tid; e < NN * NN; e += nt) {
-    const int i = e / NN, col = e % NN;     // column `col` of V is the eigenvector of A[col][col]
-    const int rank = s_rank[col];
-    if (rank < r) {
-      float sc = 1.f;
-      if (scale_mode == 0) sc = mean > 0.0 ? (float)sqrt(fmax(A[col * LD + col], 0.0) / mean) : 0.f;
-      Fout[(i64)blockIdx.x * NN * r + (i64)i * r + rank] = V[i * LD + col] * sc;
-    }
-  }
-}
-
-static size_t jacobi64_smem(int n) {
-  return (size_t)n * (n + 1) * 8 + (size_t)(n * (n + 1) + (n & 1)) * 4 + n * 8 + n * 4 + 34 * 8 + 16;
-}
-static size_t jacobi_smem(int n) { return (size_t)2 * n * (n + 4) * 4 + (size_t)n * 4 + 16; }
-cudaError_t init_jacobi() {
-  cudaError_t e = cudaFuncSetAttribute(k_jacobi_eig<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(128));
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_jacobi_eig<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi_smem(64));
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_jacobi_eig_f64<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(128));
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_jacobi_eig_f64<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(64));
-}
-void launch_jacobi_eig(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
-                       double* lam_out, cudaStream_t st) {
-  if (precise) {
-    if (n == 128) k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
-    else k_jacobi_eig_f64<64><<<batch, 1024, jacobi64_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
-  } else {
-    if (n == 128) k_jacobi_eig<128><<<batch, 256, jacobi_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
-    else k_jacobi_eig<64><<<batch, 128, jacobi_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
-  }
-}
-
-// =============================================================================
 // Response projections: phi_K = K F_K (Eq. 6) and phi_Q = RMS-normalised Q F_Q
 // (Eq. 7).  Each thread produces two rows of R outputs; F is staged in shared
 // memory and read by broadcast.  Also tracks max |phi| per head (for the
