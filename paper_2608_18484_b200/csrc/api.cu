@@ -376,7 +376,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   StageTimer tm(prof, st);
   // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means
   launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
-  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, p->FK, p->lam, st);
+  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
   tm.mark(SPARSEPR_STAGE_KEY_METRIC);
   if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
     if (!launch_project_tc(K, r.ks, r.BH, r.H, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -391,7 +391,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   tm.mark(SPARSEPR_STAGE_KEY_PERMUTE);
   // query partition: centroid metric -> F_Q -> phi_Q -> k-means
   launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
-  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, p->FQ, p->lam, st);
+  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
   tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
   if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {

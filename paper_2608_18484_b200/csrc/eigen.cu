@@ -1,12 +1,12 @@
 // Leading eigenpairs of batched symmetric matrices (n = 64 or 128), one CTA per matrix:
 // the feature maps F_K, F_Q of Section 4.1 and the probe-residual basis Psi_r of Eq. 9.
 //
-// Float64 throughout, matrix resident in shared memory:
+// Float64 for float32 tensors, float32 for bf16 tensors; matrix in registers, reflectors and vectors in shared memory:
 //   1. Householder reduction to tridiagonal form T (reflectors kept in the lower triangle)
 //   2. the r largest eigenvalues of T by Sturm-count bisection, one thread per eigenvalue
 //   3. their eigenvectors by inverse iteration on T - lambda I (Gaussian elimination with
 //      partial pivoting, factored once per eigenvalue), one thread per eigenvector
-//   4. modified Gram-Schmidt inside groups of close eigenvalues, one warp per group
+//   4. Gram-Schmidt with re-orthogonalisation inside groups of close eigenvalues
 //   5. Rayleigh quotients, residuals ||T z - lambda z|| and all pairwise inner products are
 //      checked; a matrix that fails the check is marked (NaN in its first output element)
 //      and left to the cyclic Jacobi kernel, which is launched behind this one and returns
@@ -26,83 +26,98 @@ constexpr int kEigMaxR = 64;
 constexpr int kZld = kEigMaxR + 1;
 constexpr int kTpr = 8;                                            // threads per matrix row in the Householder steps
 
-__device__ __forceinline__ double hash_unit(int i, int j) {        // deterministic start vector entries in [0.5, 1.5)
+__device__ __forceinline__ float hash_unit(int i, int j) {         // deterministic start vector entries in [0.5, 1.5)
   u64 x = (u64)(i + 1) * 0x9E3779B97F4A7C15ull + (u64)(j + 1) * 0xBF58476D1CE4E5B9ull;
   x ^= x >> 31; x *= 0x94D049BB133111EBull; x ^= x >> 29;
-  return 0.5 + (double)(x >> 11) * (1.0 / 9007199254740992.0);
+  return 0.5f + (float)(unsigned)(x >> 40) * (1.0f / 16777216.0f);
 }
+
+// Precision-dependent constants.  Float64 serves float32 tensors (whose output tolerance leaves no
+// room for a float32 eigen-basis); float32 serves bf16 tensors, where float64 arithmetic would
+// dominate the run time of the whole plan.
+template <typename T> struct EigNum;
+template <> struct EigNum<double> {
+  static constexpr double pivot = 1.0e-15, res_tol = 1.0e-7, orth_tol = 1.0e-7, group_gap = 1.0e-3;
+  static constexpr double big = 1.0e90, small = 1.0e-90;
+  static constexpr int rescale_mask = 7, passes = 20;
+};
+template <> struct EigNum<float> {
+  static constexpr float pivot = 1.0e-7f, res_tol = 1.0e-4f, orth_tol = 1.0e-3f, group_gap = 1.0e-2f;
+  static constexpr float big = 1.0e15f, small = 1.0e-15f;
+  static constexpr int rescale_mask = 0, passes = 12;
+};
 
 // sum over the 32 warps of the CTA with one barrier: partial sums go to one of two buffers in turn,
 // every warp then adds the 32 partials itself (same order everywhere, so all threads agree bit for bit)
-__device__ __forceinline__ double cta_sum(double v, double* red, int& turn) {
+template <typename T> __device__ __forceinline__ T cta_sum(T v, T* red, int& turn) {
   v = warp_sum(v);
-  double* buf = red + (turn & 1) * 32;
+  T* buf = red + (turn & 1) * 32;
   ++turn;
   if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
   __syncthreads();
   return warp_sum(buf[threadIdx.x & 31]);
 }
-__device__ __forceinline__ double cta_max(double v, double* red, int& turn) {
+template <typename T> __device__ __forceinline__ T cta_max(T v, T* red, int& turn) {
   v = warp_max(v);
-  double* buf = red + (turn & 1) * 32;
+  T* buf = red + (turn & 1) * 32;
   ++turn;
   if ((threadIdx.x & 31) == 0) buf[threadIdx.x >> 5] = v;
   __syncthreads();
   return warp_max(buf[threadIdx.x & 31]);
 }
 
-template <int NN> struct EigSmem {
+template <int NN, typename T> struct EigSmem {
   static constexpr int LD = NN + 1;
-  static constexpr size_t a = 0;                                           // double [NN][LD]
-  static constexpr size_t z = a + sizeof(double) * NN * LD;                // double [NN][kZld]
-  static constexpr size_t vec = z + sizeof(double) * NN * kZld;            // v, w, d, e, e2, beta: 6 x double[NN]
-  static constexpr size_t lam = vec + sizeof(double) * 6 * NN;             // double [kEigMaxR]
-  static constexpr size_t red = lam + sizeof(double) * kEigMaxR;           // double [2][32]
-  static constexpr size_t cst = red + sizeof(double) * 64;                 // int [kEigMaxR] group start; int flags[4]
+  static constexpr size_t a = 0;                                           // T [NN][LD]: reflector k in row k
+  static constexpr size_t z = a + sizeof(T) * NN * LD;                // T [NN][kZld]
+  static constexpr size_t vec = z + sizeof(T) * NN * kZld;            // p[2], d, e, e2, beta: 6 x T[NN]
+  static constexpr size_t lam = vec + sizeof(T) * 6 * NN;             // T [kEigMaxR]
+  static constexpr size_t red = lam + sizeof(T) * kEigMaxR;           // T [2][32]
+  static constexpr size_t cst = red + sizeof(T) * 64;                 // int [kEigMaxR] group start; int flags[4]
   static constexpr size_t total = cst + sizeof(int) * (kEigMaxR + 4);
 };
 
 // eigenvalues of T below x (Sturm count) by the three-term recurrence of the leading principal
 // minors, p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}: one dependent multiply-add per step.  A zero
-// minor takes the sign opposite to its predecessor; both running minors are rescaled by a power of
-// two every eight steps, which changes no sign.
-template <int NN>
-__device__ __forceinline__ int sturm_count(const double* __restrict__ dd, const double* __restrict__ e2, double x) {
-  double p2 = 1.0, p1 = dd[0] - x;
-  bool neg1 = p1 < 0.0 || p1 == 0.0;                            // sign of p_1 (zero counts as a change from p_0 = 1)
+// minor takes the sign opposite to its predecessor; both running minors are rescaled by a positive
+// factor when they leave a safe range, which changes no sign.
+template <int NN, typename T>
+__device__ __forceinline__ int sturm_count(const T* __restrict__ dd, const T* __restrict__ e2, T x) {
+  T p2 = T(1.0), p1 = dd[0] - x;
+  bool neg1 = p1 < T(0.0) || p1 == T(0.0);                            // sign of p_1 (zero counts as a change from p_0 = 1)
   int cnt = neg1;
 #pragma unroll 8
   for (int i = 1; i < NN; ++i) {
-    const double p = fma(dd[i] - x, p1, -(e2[i - 1] * p2));
-    const bool neg = p == 0.0 ? !neg1 : p < 0.0;
+    const T p = fma(dd[i] - x, p1, -(e2[i - 1] * p2));
+    const bool neg = p == T(0.0) ? !neg1 : p < T(0.0);
     cnt += neg != neg1;
     neg1 = neg;
     p2 = p1; p1 = p;
-    if ((i & 7) == 7) {
-      const double mx = fmax(fabs(p1), fabs(p2));
-      if (mx > 1.0e90) { p1 *= 1.0e-90; p2 *= 1.0e-90; }
-      else if (mx < 1.0e-90) { p1 *= 1.0e90; p2 *= 1.0e90; }
+    if ((i & EigNum<T>::rescale_mask) == EigNum<T>::rescale_mask) {
+      const T mx = fmax(fabs(p1), fabs(p2));
+      if (mx > EigNum<T>::big) { p1 *= EigNum<T>::small; p2 *= EigNum<T>::small; }
+      else if (mx < EigNum<T>::small) { p1 *= EigNum<T>::big; p2 *= EigNum<T>::big; }
     }
   }
   return cnt;
 }
 
-template <int NN>
+template <int NN, typename T>
 __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
                                                              float* __restrict__ Fout, double* __restrict__ lam_out) {
-  using S = EigSmem<NN>;
+  using S = EigSmem<NN, T>;
   constexpr int LD = S::LD;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* A = reinterpret_cast<double*>(smem_raw + S::a);
-  double* Z = reinterpret_cast<double*>(smem_raw + S::z);
-  double* v = reinterpret_cast<double*>(smem_raw + S::vec);
-  double* w = v + NN;
-  double* dd = w + NN;
-  double* ee = dd + NN;
-  double* e2 = ee + NN;
-  double* beta = e2 + NN;
-  double* lam = reinterpret_cast<double*>(smem_raw + S::lam);
-  double* red = reinterpret_cast<double*>(smem_raw + S::red);
+  T* A = reinterpret_cast<T*>(smem_raw + S::a);
+  T* Z = reinterpret_cast<T*>(smem_raw + S::z);
+  T* v = reinterpret_cast<T*>(smem_raw + S::vec);
+  T* w = v + NN;
+  T* dd = w + NN;
+  T* ee = dd + NN;
+  T* e2 = ee + NN;
+  T* beta = e2 + NN;
+  T* lam = reinterpret_cast<T*>(smem_raw + S::lam);
+  T* red = reinterpret_cast<T*>(smem_raw + S::red);
   int* cstart = reinterpret_cast<int*>(smem_raw + S::cst);
   int* flags = cstart + kEigMaxR;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -111,99 +126,130 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   int turn = 0;
 
   // ---- load, symmetrise, scale to max |a_ij| = 1 ---------------------------------------------------
-  double amax = 0.0;
-  for (int e = tid; e < NN * NN; e += kEigThreads) {
-    const int i = e / NN, j = e % NN;
-    const double a = 0.5 * (Mi[e] + Mi[j * NN + i]);
-    A[i * LD + j] = a;
-    amax = fmax(amax, fabs(a));
+  // The matrix lives in registers during the reduction: thread (row, h) owns A[row][h + kTpr t].
+  constexpr int kPer = NN / kTpr;
+  const int row = tid / kTpr, h = tid % kTpr;
+  const bool owner = row < NN;
+  T a[kPer];
+  T amax = T(0.0);
+#pragma unroll
+  for (int t = 0; t < kPer; ++t) {
+    const int c = h + kTpr * t;
+    a[t] = owner ? T(0.5 * (Mi[row * NN + c] + Mi[c * NN + row])) : T(0.0);
+    amax = fmax(amax, fabs(a[t]));
   }
-  const double scale = cta_max(amax, red, turn);
-  if (!(scale > 0.0) || !(scale < 1.0e300)) {
+  const T scale = cta_max(amax, red, turn);
+  if (!(scale > T(0.0)) || !(scale * T(0.0) == T(0.0))) {
     // zero matrix: eigenvalues 0, unit vectors; anything non-finite is left to the error checks downstream
     for (int e = tid; e < NN * r; e += kEigThreads) Fo[e] = (scale_mode == 1 && e / r == e % r) ? 1.f : 0.f;
     if (lam_out) for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = 0.0;
     return;
   }
-  const double inv_scale = 1.0 / scale;
-  for (int e = tid; e < NN * NN; e += kEigThreads) A[(e / NN) * LD + e % NN] *= inv_scale;
-  __syncthreads();
+  const T inv_scale = T(1.0) / scale;
+#pragma unroll
+  for (int t = 0; t < kPer; ++t) a[t] *= inv_scale;
 
 #ifdef SPR_EIG_TIMING
   const long long T0 = clock64();
 #endif
   // ---- 1. Householder tridiagonalisation ----------------------------------------------------------------
-  // kTpr threads per row of the trailing block, interleaved columns
-  const int row = tid / kTpr, h = tid % kTpr;
+  // Step k: x = A[k][k+1..] (row k = column k by symmetry) goes to shared memory; v = x + sgn alpha e_1;
+  // p = b A22 v; w = p - (b/2)(p.v) v; A22 <- A22 - v w^T - w v^T.  Two barriers per step: the sums over
+  // x and over p are formed redundantly by every warp from shared memory.
+  T* pbuf = v;                                             // [2][NN] (the v and w slots), alternating between steps
   for (int k = 0; k < NN - 2; ++k) {
-    const int m = NN - k - 1;                                   // order of the trailing block
-    double part = 0.0;
-    if (tid >= 1 && tid < m) { const double x = A[(k + 1 + tid) * LD + k]; part = x * x; }
-    const double below2 = cta_sum(part, red, turn);             // squares below the subdiagonal
-    const double x0 = A[(k + 1) * LD + k];
-    if (!(below2 > 0.0)) {                                      // column already reduced (uniform branch)
-      if (tid == 0) { ee[k] = x0; beta[k] = 0.0; }
+    T* xk = A + k * LD;                                    // raw x in row k of the reflector store
+    if (row == k) {
+#pragma unroll
+      for (int t = 0; t < kPer; ++t) { const int c = h + kTpr * t; if (c > k) xk[c] = a[t]; }
+    }
+    __syncthreads();
+    T part = T(0.0);
+    for (int c = k + 2 + lane; c < NN; c += 32) { const T x = xk[c]; part = fma(x, x, part); }
+    const T below2 = warp_sum(part);                       // squares beyond the subdiagonal entry
+    const T x0 = xk[k + 1];
+    if (!(below2 > T(0.0))) {                                      // already reduced (uniform)
+      if (tid == 0) { ee[k] = x0; beta[k] = T(0.0); e2[k] = T(0.0); }
       continue;
     }
-    const double alpha = sqrt(below2 + x0 * x0);
-    const double sgn = x0 >= 0.0 ? 1.0 : -1.0;
-    const double b = 1.0 / (alpha * (alpha + fabs(x0)));        // 2 / ||v||^2 with v = x + sgn alpha e_1
-    if (tid < m) v[tid] = tid == 0 ? x0 + sgn * alpha : A[(k + 1 + tid) * LD + k];
-    __syncthreads();
-    // p = b * A22 v
-    double acc = 0.0;
-    if (row < m) {
-      const double* ar = A + (k + 1 + row) * LD + k + 1;
-      double acc1 = 0.0;
-      int c = h;
-      for (; c + kTpr < m; c += 2 * kTpr) { acc = fma(ar[c], v[c], acc); acc1 = fma(ar[c + kTpr], v[c + kTpr], acc1); }
-      if (c < m) acc = fma(ar[c], v[c], acc);
-      acc += acc1;
-    }
+    const T alpha = sqrt(below2 + x0 * x0);
+    const T sgn = x0 >= T(0.0) ? T(1.0) : -T(1.0);
+    const T v0 = x0 + sgn * alpha;
+    const T b = T(1.0) / (alpha * (alpha + fabs(x0)));        // 2 / ||v||^2
+    if (tid == 0) { ee[k] = -sgn * alpha; beta[k] = b; e2[k] = sgn * alpha; }   // e2[] is free until the bisection
+    T* pk = pbuf + (k & 1) * NN;
+    const bool live = owner && row > k;
+    const bool warp_live = (warp * 32 + 31) / kTpr > k && warp * 32 / kTpr < NN;   // some row of this warp is live
+    T acc = T(0.0);
+    if (live) {
 #pragma unroll
-    for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    const double p_row = b * acc;
-    const double pv = cta_sum((h == 0 && row < m) ? p_row * v[row] : 0.0, red, turn);
-    if (h == 0 && row < m) w[row] = p_row - 0.5 * b * pv * v[row];
-    __syncthreads();
-    // A22 <- A22 - v w^T - w v^T
-    if (row < m) {
-      double* ar = A + (k + 1 + row) * LD + k + 1;
-      const double vi = v[row], wi = w[row];
-      for (int c = h; c < m; c += kTpr) ar[c] -= vi * w[c] + wi * v[c];
+      for (int t = 0; t < kPer; ++t) {
+        const int c = h + kTpr * t;
+        const T vc = c == k + 1 ? v0 : xk[c];
+        acc = c > k ? fma(a[t], vc, acc) : acc;
+      }
     }
-    if (tid < m) A[(k + 1 + tid) * LD + k] = v[tid];            // reflector k lives in column k below the diagonal
-    if (tid == 0) { ee[k] = -sgn * alpha; beta[k] = b; }
+    if (warp_live) {
+#pragma unroll
+      for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    }
+    const T p_row = b * acc;
+    if (live && h == 0) pk[row] = p_row;
     __syncthreads();
+    if (!warp_live) continue;                                   // nothing left to update in this warp's rows
+    T pvp = T(0.0);
+    for (int c = k + 1 + lane; c < NN; c += 32) pvp = fma(pk[c], c == k + 1 ? v0 : xk[c], pvp);
+    const T hb = T(0.5) * b * warp_sum(pvp);
+    if (live) {
+      const T v_row = row == k + 1 ? v0 : xk[row];
+      const T w_row = p_row - hb * v_row;
+#pragma unroll
+      for (int t = 0; t < kPer; ++t) {
+        const int c = h + kTpr * t;
+        const T vc = c == k + 1 ? v0 : xk[c];
+        const T wc = pk[c] - hb * vc;
+        a[t] = c > k ? a[t] - (v_row * wc + w_row * vc) : a[t];
+      }
+    }
   }
+  __syncthreads();
+  // diagonal and last off-diagonal from the registers; first entries of the reflectors
+  if (owner) {
+#pragma unroll
+    for (int t = 0; t < kPer; ++t) {
+      const int c = h + kTpr * t;
+      if (c == row) dd[row] = a[t];
+      if (row == NN - 1 && c == NN - 2) ee[NN - 2] = a[t];
+    }
+  }
+  if (tid < NN - 2) A[tid * LD + tid + 1] += e2[tid];           // v_0 = x_0 + sgn alpha
+  if (tid == 0) { ee[NN - 1] = T(0.0); beta[NN - 2] = T(0.0); beta[NN - 1] = T(0.0); }
+  __syncthreads();
 #ifdef SPR_EIG_TIMING
   const long long T1 = clock64();
 #endif
-  if (tid == 0) { ee[NN - 2] = A[(NN - 1) * LD + NN - 2]; ee[NN - 1] = 0.0; beta[NN - 2] = 0.0; beta[NN - 1] = 0.0; }
-  if (tid < NN) dd[tid] = A[tid * LD + tid];
-  __syncthreads();
   if (tid < NN) e2[tid] = ee[tid] * ee[tid];
-  double g = 0.0;
-  if (tid < NN) g = fabs(dd[tid]) + fabs(ee[tid]) + (tid > 0 ? fabs(ee[tid - 1]) : 0.0);
-  const double tnorm = cta_max(g, red, turn);                   // Gershgorin bound on |lambda|; also makes e2[] visible
+  T g = T(0.0);
+  if (tid < NN) g = fabs(dd[tid]) + fabs(ee[tid]) + (tid > 0 ? fabs(ee[tid - 1]) : T(0.0));
+  const T tnorm = cta_max(g, red, turn);                   // Gershgorin bound on |lambda|; also makes e2[] visible
 
-  // ---- 2. multi-section: 16 threads per eigenvalue, 17-fold interval reduction per pass ----------------
-  {
-    const int j = tid >> 4, t = tid & 15;                       // eigenvalue (j+1)-th largest, probe point t
+  // ---- 2. multi-section: 4 threads per eigenvalue, 5-fold interval reduction per pass -----------------
+  if (tid < 4 * kEigMaxR) {                                     // whole warps: 8 eigenvalues per warp
+    const int j = tid >> 2, t = tid & 3;                        // eigenvalue (j+1)-th largest, probe point t
     const bool active = j < r;
     const int kth = NN - 1 - j;                                 // ascending index
-    double lo = -tnorm, hi = tnorm;
-    for (int it = 0; it < 11; ++it) {
-      const double wdt = (hi - lo) * (1.0 / 17.0);
-      const double x = lo + wdt * (double)(t + 1);
-      const bool below = active && sturm_count<NN>(dd, e2, x) <= kth;   // eigenvalue kth is >= x
+    T lo = -tnorm, hi = tnorm;
+    for (int it = 0; it < EigNum<T>::passes; ++it) {
+      const T wdt = (hi - lo) * T(0.2);
+      const T x = lo + wdt * (T)(t + 1);
+      const bool below = active && sturm_count<NN, T>(dd, e2, x) <= kth;   // eigenvalue kth is >= x
       const unsigned bal = __ballot_sync(0xffffffffu, below);
-      const int s = __popc((bal >> (lane & 16)) & 0xFFFFu);     // probes (of this group of 16 lanes) still below the eigenvalue
-      const double nlo = lo + wdt * (double)s;
-      hi = s < 16 ? lo + wdt * (double)(s + 1) : hi;
+      const int s = __popc((bal >> (lane & 28)) & 0xFu);        // probes of this group of 4 lanes still below the eigenvalue
+      const T nlo = lo + wdt * (T)s;
+      hi = s < 4 ? lo + wdt * (T)(s + 1) : hi;
       lo = nlo;
     }
-    if (active && t == 0) lam[j] = 0.5 * (lo + hi);
+    if (active && t == 0) lam[j] = T(0.5) * (lo + hi);
   }
   __syncthreads();
 #ifdef SPR_EIG_TIMING
@@ -212,27 +258,27 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
 
   // ---- 3. inverse iteration: thread j computes eigenvector j of T ------------------------------------
   if (tid < r) {
-    const double shift = lam[tid];
-    const double tiny = tnorm * 1.0e-15;
-    double pinv[NN], u1[NN], u2[NN], mul[NN];                  // pivots^-1, two superdiagonals of U, multipliers
+    const T shift = lam[tid];
+    const T tiny = tnorm * EigNum<T>::pivot;
+    T pinv[NN], u1[NN], u2[NN], mul[NN];                  // pivots^-1, two superdiagonals of U, multipliers
     unsigned long long swp[(NN + 63) / 64];
 #pragma unroll
     for (int q = 0; q < (NN + 63) / 64; ++q) swp[q] = 0ull;
-    double acur = dd[0] - shift, ucur = ee[0];                 // current row i: diagonal and superdiagonal entries
+    T acur = dd[0] - shift, ucur = ee[0];                 // current row i: diagonal and superdiagonal entries
     for (int i = 0; i < NN - 1; ++i) {
-      const double sub = ee[i];
-      const double anext = dd[i + 1] - shift, unext = ee[i + 1];   // ee[NN-1] = 0
+      const T sub = ee[i];
+      const T anext = dd[i + 1] - shift, unext = ee[i + 1];   // ee[NN-1] = 0
       if (fabs(acur) >= fabs(sub)) {
-        double piv = acur;
-        if (fabs(piv) <= tiny) piv = piv >= 0.0 ? tiny : -tiny;
-        const double ip = 1.0 / piv;
-        const double m = sub * ip;
-        pinv[i] = ip; u1[i] = ucur; u2[i] = 0.0; mul[i] = m;
+        T piv = acur;
+        if (fabs(piv) <= tiny) piv = piv >= T(0.0) ? tiny : -tiny;
+        const T ip = T(1.0) / piv;
+        const T m = sub * ip;
+        pinv[i] = ip; u1[i] = ucur; u2[i] = T(0.0); mul[i] = m;
         acur = anext - m * ucur;
         ucur = unext;
       } else {
-        const double ip = 1.0 / sub;
-        const double m = acur * ip;                             // rows i and i+1 swapped
+        const T ip = T(1.0) / sub;
+        const T m = acur * ip;                             // rows i and i+1 swapped
         swp[i >> 6] |= 1ull << (i & 63);
         pinv[i] = ip; u1[i] = anext; u2[i] = unext; mul[i] = m;
         acur = ucur - m * anext;
@@ -240,38 +286,38 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
       }
     }
     {
-      double piv = acur;
-      if (fabs(piv) <= tiny) piv = piv >= 0.0 ? tiny : -tiny;
-      pinv[NN - 1] = 1.0 / piv; u1[NN - 1] = 0.0; u2[NN - 1] = 0.0; mul[NN - 1] = 0.0;
+      T piv = acur;
+      if (fabs(piv) <= tiny) piv = piv >= T(0.0) ? tiny : -tiny;
+      pinv[NN - 1] = T(1.0) / piv; u1[NN - 1] = T(0.0); u2[NN - 1] = T(0.0); mul[NN - 1] = T(0.0);
     }
-    double* z = Z + tid;                                        // z_i = z[i * kZld]
+    T* z = Z + tid;                                        // z_i = z[i * kZld]
     for (int i = 0; i < NN; ++i) z[i * kZld] = hash_unit(i, tid);
     for (int it = 0; it < 3; ++it) {
-      double zi = z[0];
+      T zi = z[0];
 #pragma unroll 4
       for (int i = 0; i < NN - 1; ++i) {                        // forward elimination
-        const double zn = z[(i + 1) * kZld];
+        const T zn = z[(i + 1) * kZld];
         const bool sw = (swp[i >> 6] >> (i & 63)) & 1ull;
-        const double keep = sw ? zn : zi, other = sw ? zi : zn;
+        const T keep = sw ? zn : zi, other = sw ? zi : zn;
         z[i * kZld] = keep;
         zi = fma(-mul[i], keep, other);
       }
-      double z1 = zi * pinv[NN - 1], z2 = 0.0;                  // back substitution
+      T z1 = zi * pinv[NN - 1], z2 = T(0.0);                  // back substitution
       z[(NN - 1) * kZld] = z1;
-      double big = fabs(z1);
+      T big = fabs(z1);
 #pragma unroll 4
       for (int i = NN - 2; i >= 0; --i) {
-        const double zz = (z[i * kZld] - u1[i] * z1 - u2[i] * z2) * pinv[i];
+        const T zz = (z[i * kZld] - u1[i] * z1 - u2[i] * z2) * pinv[i];
         z[i * kZld] = zz;
         big = fmax(big, fabs(zz));
         z2 = z1; z1 = zz;
       }
-      const double sc = big > 0.0 ? 1.0 / big : 1.0;
+      const T sc = big > T(0.0) ? T(1.0) / big : T(1.0);
       for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
     }
-    double nn = 0.0;
+    T nn = T(0.0);
     for (int i = 0; i < NN; ++i) nn = fma(z[i * kZld], z[i * kZld], nn);
-    const double sc = nn > 0.0 ? rsqrt(nn) : 0.0;
+    const T sc = nn > T(0.0) ? rsqrt(nn) : T(0.0);
     for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
   }
   __syncthreads();
@@ -279,9 +325,9 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   const long long T3 = clock64();
 #endif
 
-  // ---- 4. groups of close eigenvalues: modified Gram-Schmidt, one warp per group ----------------------
+  // ---- 4. groups of close eigenvalues: Gram-Schmidt inside each group ---------------------------------
   if (tid == 0) {
-    const double gap = 1.0e-3 * tnorm;
+    const T gap = EigNum<T>::group_gap * tnorm;
     int start = 0;
     for (int j = 0; j < r; ++j) {
       if (j > 0 && fabs(lam[j - 1] - lam[j]) >= gap) start = j;
@@ -290,30 +336,36 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     flags[0] = 0;
   }
   __syncthreads();
-  {
-    int group = 0;
-    for (int j0 = 0; j0 < r; ++group) {
-      int j1 = j0;
-      while (j1 + 1 < r && cstart[j1 + 1] == j0) ++j1;
-      if (j1 > j0 && (group & 31) == warp) {
-        for (int a = j0 + 1; a <= j1; ++a) {
-          for (int bq = j0; bq < a; ++bq) {
-            double dot = 0.0;
-            for (int i = lane; i < NN; i += 32) dot = fma(Z[i * kZld + bq], Z[i * kZld + a], dot);
-            dot = warp_sum(dot);
-            for (int i = lane; i < NN; i += 32) Z[i * kZld + a] -= dot * Z[i * kZld + bq];
-            __syncwarp();
-          }
-          double nn = 0.0;
-          for (int i = lane; i < NN; i += 32) nn = fma(Z[i * kZld + a], Z[i * kZld + a], nn);
-          nn = warp_sum(nn);
-          const double sc = nn > 0.0 ? rsqrt(nn) : 0.0;
-          for (int i = lane; i < NN; i += 32) Z[i * kZld + a] *= sc;
-          __syncwarp();
+  // vector a of a group is orthogonalised against all earlier vectors of the group at once: every warp
+  // forms some of the inner products, then every thread subtracts its share; two passes per vector
+  // (classical Gram-Schmidt with re-orthogonalisation)
+  for (int j0 = 0; j0 < r;) {
+    int j1 = j0;
+    while (j1 + 1 < r && cstart[j1 + 1] == j0) ++j1;
+    for (int a = j0 + 1; a <= j1; ++a) {
+      for (int pass = 0; pass < 2; ++pass) {
+        for (int bq = j0 + warp; bq < a; bq += 32) {
+          T dot = T(0.0);
+          for (int i = lane; i < NN; i += 32) dot = fma(Z[i * kZld + bq], Z[i * kZld + a], dot);
+          dot = warp_sum(dot);
+          if (lane == 0) pbuf[bq] = dot;
         }
+        __syncthreads();
+        if (tid < NN) {
+          T acc = Z[tid * kZld + a];
+          for (int bq = j0; bq < a; ++bq) acc = fma(-pbuf[bq], Z[tid * kZld + bq], acc);
+          Z[tid * kZld + a] = acc;
+        }
+        __syncthreads();
       }
-      j0 = j1 + 1;
+      T nn = T(0.0);
+      if (tid < NN) nn = Z[tid * kZld + a] * Z[tid * kZld + a];
+      nn = cta_sum(nn, red, turn);
+      const T sc = nn > T(0.0) ? rsqrt(nn) : T(0.0);
+      if (tid < NN) Z[tid * kZld + a] *= sc;
+      __syncthreads();
     }
+    j0 = j1 + 1;
   }
   __syncthreads();
 #ifdef SPR_EIG_TIMING
@@ -323,37 +375,37 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   // ---- 5. Rayleigh quotients, residuals, orthogonality -------------------------------------------------
   bool bad = false;
   if (tid < r) {
-    const double* z = Z + tid;
-    double num = 0.0, den = 0.0;
+    const T* z = Z + tid;
+    T num = T(0.0), den = T(0.0);
     for (int i = 0; i < NN; ++i) {
-      const double zi = z[i * kZld];
-      double t = dd[i] * zi;
+      const T zi = z[i * kZld];
+      T t = dd[i] * zi;
       if (i > 0) t = fma(ee[i - 1], z[(i - 1) * kZld], t);
       if (i + 1 < NN) t = fma(ee[i], z[(i + 1) * kZld], t);
       num = fma(zi, t, num);
       den = fma(zi, zi, den);
     }
-    const double rq = den > 0.0 ? num / den : 0.0;
-    double res = 0.0;
+    const T rq = den > T(0.0) ? num / den : T(0.0);
+    T res = T(0.0);
     for (int i = 0; i < NN; ++i) {
-      const double zi = z[i * kZld];
-      double t = (dd[i] - rq) * zi;
+      const T zi = z[i * kZld];
+      T t = (dd[i] - rq) * zi;
       if (i > 0) t = fma(ee[i - 1], z[(i - 1) * kZld], t);
       if (i + 1 < NN) t = fma(ee[i], z[(i + 1) * kZld], t);
       res = fmax(res, fabs(t));
     }
     lam[tid] = rq;
-    bad = !(res <= 1.0e-7 * tnorm) || !(fabs(den - 1.0) <= 1.0e-7);
+    bad = !(res <= EigNum<T>::res_tol * tnorm) || !(fabs(den - T(1.0)) <= EigNum<T>::orth_tol);
   }
   for (int pr = tid; pr < r * r; pr += kEigThreads) {
     const int a = pr / r, bq = pr % r;
     if (a < bq) {
-      double d0 = 0.0, d1 = 0.0;
+      T d0 = T(0.0), d1 = T(0.0);
       for (int i = 0; i < NN; i += 2) {
         d0 = fma(Z[i * kZld + a], Z[i * kZld + bq], d0);
         d1 = fma(Z[(i + 1) * kZld + a], Z[(i + 1) * kZld + bq], d1);
       }
-      bad |= !(fabs(d0 + d1) <= 1.0e-7);
+      bad |= !(fabs(d0 + d1) <= EigNum<T>::orth_tol);
     }
   }
   if (bad) flags[0] = 1;
@@ -375,33 +427,33 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     const int j = tid / tpv, q = tid % tpv;
     const bool active = j < r;
     for (int k = NN - 3; k >= 0; --k) {
-      const double bk = beta[k];
-      if (bk == 0.0) continue;                                   // uniform
-      double dot = 0.0;
+      const T bk = beta[k];
+      if (bk == T(0.0)) continue;                                   // uniform
+      T dot = T(0.0);
       if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[i * LD + k], Z[i * kZld + j], dot);
+        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[k * LD + i], Z[i * kZld + j], dot);
 #pragma unroll
       for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      const double f = bk * dot;
+      const T f = bk * dot;
       if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[i * LD + k];
+        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[k * LD + i];
       __syncwarp();
     }
   }
   __syncthreads();
-  double part = tid < r ? fmax(lam[tid], 0.0) : 0.0;
-  const double mean = cta_sum(part, red, turn) / (double)r;
+  T part = tid < r ? fmax(lam[tid], T(0.0)) : T(0.0);
+  const T mean = cta_sum(part, red, turn) / (T)r;
 #ifdef SPR_EIG_TIMING
   if (tid == 0 && blockIdx.x == 0)
     printf("eig n=%d r=%d cycles: householder %lld bisection %lld inverse-it %lld mgs %lld check %lld backtransform %lld\n", NN, r,
            T1 - T0, T2 - T1, T3 - T2, T4 - T3, T5 - T4, clock64() - T5);
 #endif
   if (lam_out)
-    for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = j < r ? lam[j] * scale : 0.0;
+    for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = j < r ? (double)(lam[j] * scale) : 0.0;
   for (int e = tid; e < NN * r; e += kEigThreads) {
     const int rw = e / r, j = e % r;
-    double sc = 1.0;
-    if (scale_mode == 0) sc = mean > 0.0 ? sqrt(fmax(lam[j], 0.0) / mean) : 0.0;
+    T sc = T(1.0);
+    if (scale_mode == 0) sc = mean > T(0.0) ? sqrt(fmax(lam[j], T(0.0)) / mean) : T(0.0);
     Fo[e] = (float)(Z[rw * kZld + j] * sc);
   }
 }
@@ -517,9 +569,13 @@ size_t jacobi64_smem(int n) {
 }  // namespace
 
 cudaError_t init_eigen() {
-  cudaError_t e = cudaFuncSetAttribute(k_eig_tridiag<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<128>::total);
+  cudaError_t e = cudaFuncSetAttribute(k_eig_tridiag<128, double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<128, double>::total);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_eig_tridiag<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<64>::total);
+  e = cudaFuncSetAttribute(k_eig_tridiag<64, double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<64, double>::total);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_eig_tridiag<128, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<128, float>::total);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(k_eig_tridiag<64, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EigSmem<64, float>::total);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(k_jacobi_eig_f64<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(128));
   if (e != cudaSuccess) return e;
@@ -528,16 +584,19 @@ cudaError_t init_eigen() {
 
 // Min: `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart; r <= 64 leading pairs.
 // scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda) (feature map of Section 4.1);
-// 1: orthonormal columns (basis of Eq. 9).  Fout [batch][n][r]; lam_out [batch][n] or null (entries >= r are 0).
-void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout, double* lam_out,
-                    cudaStream_t st) {
+// 1: orthonormal columns (basis of Eq. 9).  precise: float64 arithmetic.  Fout [batch][n][r];
+// lam_out [batch][n] or null (entries >= r are 0).
+void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
+                    double* lam_out, cudaStream_t st) {
+#define SPR_EIG(NN, TT) k_eig_tridiag<NN, TT><<<batch, kEigThreads, EigSmem<NN, TT>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out)
   if (n == 128) {
-    k_eig_tridiag<128><<<batch, kEigThreads, EigSmem<128>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    if (precise) SPR_EIG(128, double); else SPR_EIG(128, float);
     k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
   } else {
-    k_eig_tridiag<64><<<batch, kEigThreads, EigSmem<64>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    if (precise) SPR_EIG(64, double); else SPR_EIG(64, float);
     k_jacobi_eig_f64<64><<<batch, 1024, jacobi64_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
   }
+#undef SPR_EIG
 }
 
 }  // namespace spr

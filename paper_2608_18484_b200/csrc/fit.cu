@@ -202,7 +202,7 @@ void launch_fit(const FitArgs& a, cudaStream_t st) {
   k_fit_gram<<<dim3(3, a.BH), 256, (size_t)2 * 32 * d * 8, st>>>(a);
   k_fit_solve<<<a.BH, 1024, (size_t)d * (d + 1) * 8, st>>>(a);
   // Psi_r: leading eigenvectors of S = Rb^T W Rb, i.e. right singular vectors of W^(1/2) Rb.
-  launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.Psi, nullptr, st);
+  launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, st);
   k_fit_compose<<<a.BH, 256, 0, st>>>(a, r);
 }
 

@@ -10,11 +10,11 @@ void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, 
                         double* Mout, cudaStream_t st);
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
 // eigen.cu: leading r <= 64 eigenpairs of `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart.
-// scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda); 1: orthonormal columns.
+// scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda); 1: orthonormal columns; precise: float64.
 // Fout [batch][n][r]; lam_out [batch][n] or null.
 cudaError_t init_eigen();
-void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, float* Fout, double* lam_out,
-                    cudaStream_t st);
+void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
+                    double* lam_out, cudaStream_t st);
 void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
