@@ -47,6 +47,29 @@ template <> struct EigNum<float> {
   static constexpr int rescale_mask = 0, passes = 12;
 };
 
+// kN consecutive elements (a multiple of 16 bytes, 16-byte aligned) between shared memory and registers
+template <typename T, int kN> __device__ __forceinline__ void ld_vec(const T* p, T (&o)[kN]) {
+  constexpr int kV = 16 / sizeof(T);
+#pragma unroll
+  for (int i = 0; i < kN / kV; ++i) {
+    const uint4 raw = reinterpret_cast<const uint4*>(p)[i];
+    T tmp[kV];
+    *reinterpret_cast<uint4*>(tmp) = raw;
+#pragma unroll
+    for (int e = 0; e < kV; ++e) o[i * kV + e] = tmp[e];
+  }
+}
+template <typename T, int kN> __device__ __forceinline__ void st_vec(T* p, const T (&o)[kN]) {
+  constexpr int kV = 16 / sizeof(T);
+#pragma unroll
+  for (int i = 0; i < kN / kV; ++i) {
+    T tmp[kV];
+#pragma unroll
+    for (int e = 0; e < kV; ++e) tmp[e] = o[i * kV + e];
+    reinterpret_cast<uint4*>(p)[i] = *reinterpret_cast<const uint4*>(tmp);
+  }
+}
+
 // sum over the 32 warps of the CTA with one barrier: partial sums go to one of two buffers in turn,
 // every warp then adds the 32 partials itself (same order everywhere, so all threads agree bit for bit)
 template <typename T> __device__ __forceinline__ T cta_sum(T v, T* red, int& turn) {
@@ -67,10 +90,14 @@ template <typename T> __device__ __forceinline__ T cta_max(T v, T* red, int& tur
 }
 
 template <int NN, typename T> struct EigSmem {
-  static constexpr int LD = NN + 1;
+  // a vector of NN entries is stored as kTpr segments of NN / kTpr entries, each followed by 16 bytes of
+  // padding: the eight threads of a row then read their segments with conflict-free 16-byte accesses
+  static constexpr int kPad = 16 / (int)sizeof(T);
+  static constexpr int LD = NN + kTpr * kPad;
   static constexpr size_t a = 0;                                           // T [NN][LD]: reflector k in row k
-  static constexpr size_t z = a + sizeof(T) * NN * LD;                // T [NN][kZld]
-  static constexpr size_t vec = z + sizeof(T) * NN * kZld;            // p[2], d, e, e2, beta: 6 x T[NN]
+  static constexpr size_t z = a + sizeof(T) * NN * LD;                     // T [NN][kZld]
+  static constexpr size_t pb = z + sizeof(T) * NN * kZld;                  // T [2][LD]: p of two consecutive steps
+  static constexpr size_t vec = pb + sizeof(T) * 2 * LD;                   // (2 spare), d, e, e2, beta: 6 x T[NN]
   static constexpr size_t lam = vec + sizeof(T) * 6 * NN;             // T [kEigMaxR]
   static constexpr size_t red = lam + sizeof(T) * kEigMaxR;           // T [2][32]
   static constexpr size_t cst = red + sizeof(T) * 64;                 // int [kEigMaxR] group start; int flags[4]
@@ -107,8 +134,11 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
                                                              float* __restrict__ Fout, double* __restrict__ lam_out) {
   using S = EigSmem<NN, T>;
   constexpr int LD = S::LD;
+  constexpr int kPer = NN / kTpr, kSeg = kPer + S::kPad;       // padded position of entry c: c + (c / kPer) * kPad
+  auto pos = [](int c) { return c + (c / (NN / kTpr)) * (16 / (int)sizeof(T)); };
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* A = reinterpret_cast<T*>(smem_raw + S::a);
+  T* pbuf = reinterpret_cast<T*>(smem_raw + S::pb);
   T* Z = reinterpret_cast<T*>(smem_raw + S::z);
   T* v = reinterpret_cast<T*>(smem_raw + S::vec);
   T* w = v + NN;
@@ -126,15 +156,14 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   int turn = 0;
 
   // ---- load, symmetrise, scale to max |a_ij| = 1 ---------------------------------------------------
-  // The matrix lives in registers during the reduction: thread (row, h) owns A[row][h + kTpr t].
-  constexpr int kPer = NN / kTpr;
+  // The matrix lives in registers during the reduction: thread (row, h) owns A[row][kPer h .. kPer h + kPer).
   const int row = tid / kTpr, h = tid % kTpr;
   const bool owner = row < NN;
   T a[kPer];
   T amax = T(0.0);
 #pragma unroll
   for (int t = 0; t < kPer; ++t) {
-    const int c = h + kTpr * t;
+    const int c = kPer * h + t;
     a[t] = owner ? T(0.5 * (Mi[row * NN + c] + Mi[c * NN + row])) : T(0.0);
     amax = fmax(amax, fabs(a[t]));
   }
@@ -156,58 +185,85 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   // Step k: x = A[k][k+1..] (row k = column k by symmetry) goes to shared memory; v = x + sgn alpha e_1;
   // p = b A22 v; w = p - (b/2)(p.v) v; A22 <- A22 - v w^T - w v^T.  Two barriers per step: the sums over
   // x and over p are formed redundantly by every warp from shared memory.
-  T* pbuf = v;                                             // [2][NN] (the v and w slots), alternating between steps
+  T* scal = lam;                                                // step scalars {reduce?, v_0, b, sgn alpha}; lam[] is free until step 2
+  T* pvpart = red;                                              // [32] per-warp parts of p.v (red[] is idle inside the loop)
   for (int k = 0; k < NN - 2; ++k) {
-    T* xk = A + k * LD;                                    // raw x in row k of the reflector store
-    if (row == k) {
+    T* xk = A + k * LD;                                         // raw x in row k of the reflector store
+    T* pk = pbuf + (k & 1) * LD;
+    if (warp == (k * kTpr) / 32) {
+      // the eight threads that own row k publish it together with the scalars of the reflector
+      T part = T(0.0), x0p = T(0.0);
+      if (row == k) {
+        st_vec<T, kPer>(xk + kSeg * h, a);                     // entries at columns <= k are never read
 #pragma unroll
-      for (int t = 0; t < kPer; ++t) { const int c = h + kTpr * t; if (c > k) xk[c] = a[t]; }
-    }
-    __syncthreads();
-    T part = T(0.0);
-    for (int c = k + 2 + lane; c < NN; c += 32) { const T x = xk[c]; part = fma(x, x, part); }
-    const T below2 = warp_sum(part);                       // squares beyond the subdiagonal entry
-    const T x0 = xk[k + 1];
-    if (!(below2 > T(0.0))) {                                      // already reduced (uniform)
-      if (tid == 0) { ee[k] = x0; beta[k] = T(0.0); e2[k] = T(0.0); }
-      continue;
-    }
-    const T alpha = sqrt(below2 + x0 * x0);
-    const T sgn = x0 >= T(0.0) ? T(1.0) : -T(1.0);
-    const T v0 = x0 + sgn * alpha;
-    const T b = T(1.0) / (alpha * (alpha + fabs(x0)));        // 2 / ||v||^2
-    if (tid == 0) { ee[k] = -sgn * alpha; beta[k] = b; e2[k] = sgn * alpha; }   // e2[] is free until the bisection
-    T* pk = pbuf + (k & 1) * NN;
-    const bool live = owner && row > k;
-    const bool warp_live = (warp * 32 + 31) / kTpr > k && warp * 32 / kTpr < NN;   // some row of this warp is live
-    T acc = T(0.0);
-    if (live) {
+        for (int t = 0; t < kPer; ++t) {
+          const int c = kPer * h + t;
+          part = c > k + 1 ? fma(a[t], a[t], part) : part;
+          x0p = c == k + 1 ? a[t] : x0p;
+        }
+      }
 #pragma unroll
-      for (int t = 0; t < kPer; ++t) {
-        const int c = h + kTpr * t;
-        const T vc = c == k + 1 ? v0 : xk[c];
-        acc = c > k ? fma(a[t], vc, acc) : acc;
+      for (int o = 1; o < kTpr; o <<= 1) {
+        part += __shfl_xor_sync(0xffffffffu, part, o);
+        x0p += __shfl_xor_sync(0xffffffffu, x0p, o);
+      }
+      if (row == k && h == 0) {
+        const T below2 = part, x0 = x0p;                        // squares beyond the subdiagonal entry
+        if (below2 > T(0.0)) {
+          const T alpha = sqrt(below2 + x0 * x0);
+          const T sa = x0 >= T(0.0) ? alpha : -alpha;
+          scal[0] = T(1.0); scal[1] = x0 + sa; scal[2] = T(1.0) / (alpha * (alpha + fabs(x0))); scal[3] = sa;
+          ee[k] = -sa; beta[k] = scal[2]; e2[k] = sa;           // e2[] is free until the bisection
+        } else {
+          scal[0] = T(0.0);
+          ee[k] = x0; beta[k] = T(0.0); e2[k] = T(0.0);         // already reduced
+        }
       }
     }
+    __syncthreads();
+    if (scal[0] == T(0.0)) continue;                            // uniform
+    const T v0 = scal[1], b = scal[2];
+    const bool live = owner && row > k;
+    const bool warp_live = (warp * 32 + 31) / kTpr > k && warp * 32 / kTpr < NN;   // some row of this warp is live
+    T p_row = T(0.0);
     if (warp_live) {
+      T acc = T(0.0);
+      if (live && kPer * h + kPer - 1 > k) {                   // some column of this thread is in the trailing block
+        T xv[kPer];
+        ld_vec<T, kPer>(xk + kSeg * h, xv);
+#pragma unroll
+        for (int t = 0; t < kPer; ++t) {
+          const int c = kPer * h + t;
+          const T vc = c == k + 1 ? v0 : xv[t];
+          acc = c > k ? fma(a[t], vc, acc) : acc;
+        }
+      }
 #pragma unroll
       for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      p_row = b * acc;
+      if (live && h == 0) pk[pos(row)] = p_row;
+      // this warp's part of p.v (rows of the warp, one lane per row)
+      T pvw = (live && h == 0) ? p_row * (row == k + 1 ? v0 : xk[pos(row)]) : T(0.0);
+#pragma unroll
+      for (int o = kTpr; o < 32; o <<= 1) pvw += __shfl_xor_sync(0xffffffffu, pvw, o);
+      if (lane == 0) pvpart[warp] = pvw;
+    } else if (lane == 0) {
+      pvpart[warp] = T(0.0);
     }
-    const T p_row = b * acc;
-    if (live && h == 0) pk[row] = p_row;
     __syncthreads();
     if (!warp_live) continue;                                   // nothing left to update in this warp's rows
-    T pvp = T(0.0);
-    for (int c = k + 1 + lane; c < NN; c += 32) pvp = fma(pk[c], c == k + 1 ? v0 : xk[c], pvp);
-    const T hb = T(0.5) * b * warp_sum(pvp);
-    if (live) {
-      const T v_row = row == k + 1 ? v0 : xk[row];
+    const T hb = T(0.5) * b * warp_sum(pvpart[lane]);
+    if (live && kPer * h + kPer - 1 > k) {
+      const T v_row = row == k + 1 ? v0 : xk[pos(row)];
       const T w_row = p_row - hb * v_row;
+      T xv[kPer], pv[kPer];
+      ld_vec<T, kPer>(xk + kSeg * h, xv);
+      ld_vec<T, kPer>(pk + kSeg * h, pv);
 #pragma unroll
       for (int t = 0; t < kPer; ++t) {
-        const int c = h + kTpr * t;
-        const T vc = c == k + 1 ? v0 : xk[c];
-        const T wc = pk[c] - hb * vc;
+        const int c = kPer * h + t;
+        const T vc = c == k + 1 ? v0 : xv[t];
+        const T wc = pv[t] - hb * vc;
         a[t] = c > k ? a[t] - (v_row * wc + w_row * vc) : a[t];
       }
     }
@@ -217,12 +273,12 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   if (owner) {
 #pragma unroll
     for (int t = 0; t < kPer; ++t) {
-      const int c = h + kTpr * t;
+      const int c = kPer * h + t;
       if (c == row) dd[row] = a[t];
       if (row == NN - 1 && c == NN - 2) ee[NN - 2] = a[t];
     }
   }
-  if (tid < NN - 2) A[tid * LD + tid + 1] += e2[tid];           // v_0 = x_0 + sgn alpha
+  if (tid < NN - 2) A[tid * LD + pos(tid + 1)] += e2[tid];           // v_0 = x_0 + sgn alpha
   if (tid == 0) { ee[NN - 1] = T(0.0); beta[NN - 2] = T(0.0); beta[NN - 1] = T(0.0); }
   __syncthreads();
 #ifdef SPR_EIG_TIMING
@@ -431,12 +487,12 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
       if (bk == T(0.0)) continue;                                   // uniform
       T dot = T(0.0);
       if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[k * LD + i], Z[i * kZld + j], dot);
+        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[k * LD + pos(i)], Z[i * kZld + j], dot);
 #pragma unroll
       for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
       const T f = bk * dot;
       if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[k * LD + i];
+        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[k * LD + pos(i)];
       __syncwarp();
     }
   }
