@@ -90,6 +90,7 @@ cudaError_t ensure_init() {
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_correction_tc()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_attention_rem()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_project_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_probe_tc()) != cudaSuccess) { g_init_err = e; return; }
@@ -415,8 +416,8 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
                       p->route_idx, p->rstate, nullptr, st);
-  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
-  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, p->tile_off128, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
   if (overlap) join_side(p, st);
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
@@ -466,8 +467,8 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   k_sizes_from_off<<<dim3((r.Ck + 255) / 256, r.BH), 256, 0, st>>>(p->kv_off, r.Ck, p->nk);
   k_sizes_from_off<<<dim3((r.Cq + 255) / 256, r.BH), 256, 0, st>>>(p->q_off, r.Cq, p->nq);
   launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, st);
-  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, p->tile_off, st);
-  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, p->tile_off128, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
+  launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
   if (!launch_ok() || cudaStreamSynchronize(st) != cudaSuccess) { delete p; return SPARSEPR_ERR_CUDA; }
   *out = p;
   return SPARSEPR_OK;
@@ -533,7 +534,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   }
   if (tensor) {
     aa.tile_off = p->tile_off128;
-    if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
+    if (!launch_attention_tc(aa, st) || !launch_attention_rem(aa, st)) return SPARSEPR_ERR_CUDA;
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) join_side(p, st);
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
@@ -635,8 +636,14 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     for (int a = 0; a < r.Cq; ++a) {
       i64 keys = 0;
       for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += (k[rii[t] + 1] - k[rii[t]] + box - 1) / box * box;
-      const i64 qt = (q[a + 1] - q[a] + qtile - 1) / qtile, kt = (keys + ktile - 1) / ktile;
-      out->padded_tile_pairs += qt * qtile * kt * ktile;
+      const i64 kt = (keys + ktile - 1) / ktile;
+      const int nrow = q[a + 1] - q[a], rem = nrow % qtile;
+      if (tcpath && rem > 0 && rem <= kRemRows) {
+        // full tiles by the 128-row kernel, the short remainder (rounded to 16 rows) by the remainder kernel
+        out->padded_tile_pairs += ((i64)(nrow / qtile) * qtile + (rem + 15) / 16 * 16) * kt * ktile;
+      } else {
+        out->padded_tile_pairs += (i64)((nrow + qtile - 1) / qtile) * qtile * kt * ktile;
+      }
     }
   }
   out->rho_exec = out->rho_route + (double)r.M / (double)r.N;

@@ -275,20 +275,25 @@ __global__ void __launch_bounds__(256) k_attention_simt(AttnArgs a) {
   }
 }
 
-__global__ void __launch_bounds__(1024) k_tile_offsets(const int* __restrict__ q_off, int Cq, int tile_rows,
+// tiles per query group: ceil(n / tile_rows), or, with small_rem > 0, without the last tile when it
+// would hold at most small_rem rows (those rows belong to the remainder kernel)
+__global__ void __launch_bounds__(1024) k_tile_offsets(const int* __restrict__ q_off, int Cq, int tile_rows, int small_rem,
                                                        int* __restrict__ tile_off) {
   __shared__ int cnt[kMaxGroups];
   __shared__ int scratch[34];
   const int bh = blockIdx.x;
   const int* qo = q_off + (i64)bh * (Cq + 1);
-  for (int a = threadIdx.x; a < Cq; a += blockDim.x) cnt[a] = (qo[a + 1] - qo[a] + tile_rows - 1) / tile_rows;
+  for (int a = threadIdx.x; a < Cq; a += blockDim.x) {
+    const int n = qo[a + 1] - qo[a], rem = n % tile_rows;
+    cnt[a] = n / tile_rows + (rem > small_rem ? 1 : 0);
+  }
   __syncthreads();
   const int total = block_exclusive_scan(cnt, Cq, scratch);
   for (int a = threadIdx.x; a < Cq; a += blockDim.x) tile_off[(i64)bh * (Cq + 1) + a] = cnt[a];
   if (threadIdx.x == 0) tile_off[(i64)bh * (Cq + 1) + Cq] = total;
 }
-void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int* tile_off, cudaStream_t st) {
-  k_tile_offsets<<<BH, 1024, 0, st>>>(q_off, Cq, tile_rows, tile_off);
+void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int small_rem, int* tile_off, cudaStream_t st) {
+  k_tile_offsets<<<BH, 1024, 0, st>>>(q_off, Cq, tile_rows, small_rem, tile_off);
 }
 
 template <typename T, int D>

@@ -85,13 +85,19 @@ struct AttnArgs {
   int* err;                   // device error word (may be null)
 };
 cudaError_t init_attention_simt();
-void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int* tile_off, cudaStream_t st);
+// tile_off [BH][Cq+1]: prefix of the tiles per query group; small_rem > 0 leaves out a last tile of at most small_rem rows
+void launch_tile_offsets(const int* q_off, int BH, int Cq, int tile_rows, int small_rem, int* tile_off, cudaStream_t st);
 void launch_attention_simt(const AttnArgs& a, cudaStream_t st);
 // ---- attention_tc.cu (tcgen05 / TMEM / TMA; bf16, d = 128) -------------------------------------
 cudaError_t init_attention_tc();
 bool attention_tc_supported(const AttnArgs& a);
 // tile_off in `a` must have been built for 128-row tiles; a.A and a.c are ignored (no correction epilogue)
 bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
+// attention_rem.cu: the remainders of 1..64 rows per query group that the 128-row kernel leaves out when its tile
+// offsets were built with small_rem = kRemRows
+constexpr int kRemRows = 64;
+cudaError_t init_attention_rem();
+bool launch_attention_rem(const AttnArgs& a, cudaStream_t st);
 // correction_tc.cu: O <- O + O A + c in place (bf16, d_v = 128); At: bf16 scratch [BH][128][128]
 cudaError_t init_correction_tc();
 bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
