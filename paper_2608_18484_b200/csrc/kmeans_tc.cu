@@ -13,6 +13,7 @@
 // epilogue groups on alternate row tiles (one row per thread: tcgen05.ld, best/second,
 // fixed-point centroid sums with warp-level pre-aggregation), warp 4 TMA producer, warp 5
 // MMA issuer.
+#include <cstdio>
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -113,12 +114,20 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(0, kKmChunk);
       const int ksteps = prm.R / 16;
+#ifdef SPR_KM_TIMING
+      long long mX = 0, mA = 0, mI = 0, m0 = clock64();
+#define SPR_KM(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
+#else
+#define SPR_KM(v)
+#endif
       for (int q = 0; q < steps; ++q) {
         const int tl = q / n_chunks, ch = q % n_chunks;
         const int xs = tl & 1, ms = n_chunks > 1 ? (q & 1) : 0;
         if (ch == 0 && !mbar_wait(bar(X_FULL + xs), (tl >> 1) & 1, abort_flag)) break;
+        SPR_KM(mX);
         if ((n_chunks > 1 || q == 0) && !mbar_wait(bar(MU_FULL + ms), n_chunks > 1 ? ((q >> 1) & 1) : 0, abort_flag)) break;
         if (!mbar_wait(bar(ACC_EMPTY + (q & 1)), ((q >> 1) & 1) ^ 1, abort_flag)) break;
+        SPR_KM(mA);
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(q & 1) * 256u;
         const uint32_t xh = base + KmSmem::x + xs * 2 * kXBytes, xl = xh + kXBytes;
@@ -130,7 +139,12 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         if (ch == n_chunks - 1) umma_commit(bar(X_EMPTY + xs));
         if (n_chunks > 1) umma_commit(bar(MU_EMPTY + ms));
         umma_commit(bar(ACC_FULL + (q & 1)));
+        SPR_KM(mI);
       }
+#ifdef SPR_KM_TIMING
+      if (blockIdx.x == 1 && blockIdx.y == 0 && steps > 0)
+        printf("km mma steps %d sums %d: wait X %lld  wait ACC_EMPTY %lld  issue %lld (cycles per tile)\n", steps, prm.sums != nullptr, mX / steps, mA / steps, mI / steps);
+#endif
     }
   } else {
     // =========================== epilogue: argmin, sums =====================================
@@ -140,6 +154,12 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const float mm = prm.mumax[bh];
     bool ok = true;
+#ifdef SPR_KM_TIMING
+    long long eP = 0, eW = 0, eA = 0, eD = 0, eS = 0, e0 = clock64();
+#define SPR_KE(v) do { const long long t1 = clock64(); v += t1 - e0; e0 = t1; } while (0)
+#else
+#define SPR_KE(v)
+#endif
     for (int tl = grp; tl < my_tiles; tl += 2) {
       const int row = (tile0 + tl) * 128 + wq * 32 + lane;
       float best = 3.0e38f, second = 3.0e38f;
@@ -147,19 +167,32 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       // features of the warp's 32 rows for this lane's two columns (used by the centroid sums);
       // issued before the score wait so that the loads overlap it
       float pv0[32], pv1[32];
+      const float xn = row < prm.N ? prm.xnorm[(i64)bh * prm.N + row] : 0.f;   // needed after the scores: fetched now
       if (prm.sums) {
         const int rowbase = (tile0 + tl) * 128 + wq * 32;
+        const bool c0ok = lane < prm.r, c1ok = lane + 32 < prm.r;
+        if (rowbase + 31 < prm.N) {                            // every tile but the last of a head (uniform)
+          const float* xb = prm.phi + ((i64)bh * prm.N + rowbase) * prm.ldphi + lane;
 #pragma unroll
-        for (int rr = 0; rr < 32; ++rr) {
-          const int rw = min(rowbase + rr, prm.N - 1);
-          const float* xr = prm.phi + ((i64)bh * prm.N + rw) * prm.ldphi;
-          pv0[rr] = lane < prm.r ? xr[lane] : 0.f;
-          pv1[rr] = lane + 32 < prm.r ? xr[lane + 32] : 0.f;
+          for (int rr = 0; rr < 32; ++rr) {
+            pv0[rr] = c0ok ? xb[rr * prm.ldphi] : 0.f;
+            pv1[rr] = c1ok ? xb[rr * prm.ldphi + 32] : 0.f;
+          }
+        } else {
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr) {
+            const int rw = min(rowbase + rr, prm.N - 1);
+            const float* xr = prm.phi + ((i64)bh * prm.N + rw) * prm.ldphi;
+            pv0[rr] = c0ok ? xr[lane] : 0.f;
+            pv1[rr] = c1ok ? xr[lane + 32] : 0.f;
+          }
         }
       }
+      SPR_KE(eP);
       for (int ch = 0; ch < n_chunks; ++ch) {
         const int q = tl * n_chunks + ch;
         ok = __all_sync(FULL, ok && mbar_wait(bar(ACC_FULL + (q & 1)), (q >> 1) & 1, abort_flag));
+        SPR_KE(eW);
         if (!ok) continue;
         tc_fence_after();
         const int c0 = ch * kKmChunk;
@@ -185,12 +218,12 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         }
         tc_fence_before();
         mbar_arrive(bar(ACC_EMPTY + (q & 1)));
+        SPR_KE(eA);
       }
       // decide, or hand the row to the exact recheck
       const bool valid = ok && row < prm.N;
       bool decided = false;
       if (valid) {
-        const float xn = prm.xnorm[(i64)bh * prm.N + row];
         // bound on |computed score - true score|: split-operand products (2^-13 relative with
         // margin), fp32 accumulation and the final combination
         const float E = 2.5e-4f * xn * mm + 1.0e-6f * (mm * mm + xn * mm);
@@ -201,11 +234,14 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           prm.flagged[pos] = bh * prm.N + row;
         }
       }
+      SPR_KE(eD);
       if (prm.sums) {
         // warp-level pre-aggregation: lanes = feature columns (lane, lane+32); the 32 rows of the
         // warp were prefetched above; one fixed-point atomic per (cluster, column)
         unsigned todo = __ballot_sync(FULL, decided);
-        const double scl = ldexp(1.0, prm.fx_shift[bh]);
+        // 2^shift as a float: scaling a float32 partial sum by a power of two is exact, so the conversion below
+        // gives the same integer as a float64 product would
+        const float scl = __int_as_float((127 + prm.fx_shift[bh]) << 23);
         while (todo) {
           const int leader = __ffs(todo) - 1;
           const int cl = __shfl_sync(FULL, bi, leader);
@@ -220,14 +256,22 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
             a0 += in ? pv0[rr] : 0.f;
             a1 += in ? pv1[rr] : 0.f;
           }
-          const i64 acc0 = __double2ll_rn((double)a0 * scl), acc1 = __double2ll_rn((double)a1 * scl);
+          const i64 acc0 = __float2ll_rn(a0 * scl), acc1 = __float2ll_rn(a1 * scl);
           i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
           if (lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane), (u64)acc0);
           if (lane + 32 < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane + 32), (u64)acc1);
           if (lane == 0) atomicAdd(prm.counts + (i64)bh * prm.C + cl, __popc(members));
         }
       }
+      SPR_KE(eS);
     }
+#ifdef SPR_KM_TIMING
+    if (blockIdx.x == 1 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 6)) {
+      const int nt = max(1, (my_tiles + 1 - grp) / 2);
+      printf("km epilogue warp %d tiles %d sums %d: prefetch %lld  wait ACC %lld  argmin %lld  decide %lld  sums %lld (cycles per tile)\n", warp, nt,
+             prm.sums != nullptr, eP / nt, eW / nt, eA / nt, eD / nt, eS / nt);
+    }
+#endif
   }
   tc_fence_before();
   __syncthreads();

@@ -10,7 +10,8 @@ namespace spr {
 // theta_a would give ONE key at the centroid kappa_b:
 //   p_ab = exp(l_ab - LSE_a),  l_ab = s theta_a.kappa_b,
 //   LSE_a = log sum_{b non-empty} n_b exp(l_ab).
-// One CTA per query group; logits in float64, scores stored as float32.
+// One CTA per query group; inner products and exponentials in float32 (differences and sums in float64),
+// scores stored as float32.
 // =============================================================================
 __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ theta, const float* __restrict__ kappa,
                                                      const int* __restrict__ nq, const int* __restrict__ nk, int Cq,
@@ -30,12 +31,13 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
   double mx = -1.0e300;
   for (int b = threadIdx.x; b < Ck; b += 256) {
     const float* kp = kappa + ((i64)bh * Ck + b) * d;
-    double l = 0.0;
+    // float32 products in four independent chains (this GPU's float64 pipe is narrow)
+    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
     for (int k = 0; k < d; k += 4) {
       const float4 v = *reinterpret_cast<const float4*>(kp + k);
-      l += (double)th[k] * (double)v.x + (double)th[k + 1] * (double)v.y + (double)th[k + 2] * (double)v.z +
-           (double)th[k + 3] * (double)v.w;
+      l0 = fmaf(th[k], v.x, l0); l1 = fmaf(th[k + 1], v.y, l1); l2 = fmaf(th[k + 2], v.z, l2); l3 = fmaf(th[k + 3], v.w, l3);
     }
+    double l = ((double)l0 + (double)l1) + ((double)l2 + (double)l3);
     l *= (double)scale;
     lg[b] = l;
     if (nkh[b] > 0) mx = fmax(mx, l);
@@ -43,10 +45,10 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
   mx = block_max(mx, red);
   double z = 0.0;
   for (int b = threadIdx.x; b < Ck; b += 256)
-    if (nkh[b] > 0) z += (double)nkh[b] * exp(lg[b] - mx);
+    if (nkh[b] > 0) z += (double)nkh[b] * (double)expf((float)(lg[b] - mx));
   z = block_sum(z, red);
   const double lse = mx + log(z);
-  for (int b = threadIdx.x; b < Ck; b += 256) out[b] = nkh[b] > 0 ? (float)exp(lg[b] - lse) : 0.f;
+  for (int b = threadIdx.x; b < Ck; b += 256) out[b] = nkh[b] > 0 ? expf((float)(lg[b] - lse)) : 0.f;
 }
 
 void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
