@@ -348,16 +348,32 @@ def sparsepr_stage_route(score: torch.Tensor, nq: torch.Tensor, nk: torch.Tensor
 # ---- whole call on host buffers ----------------------------------------------------------
 def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, dev_buffers=None):
     """One full call for a user whose tensors live in (pinned) host memory:
-    host->device copies, plan, attend, device->host copy of O.  Returns O on host."""
+    host->device copies, plan, attend, device->host copy of O.  Returns O on host.
+    The plan needs only Q and K, so V travels on a second stream while the plan runs."""
     dev = torch.device("cuda")
     if dev_buffers is None:
         dev_buffers = [torch.empty(t.shape, dtype=t.dtype, device=dev) for t in (Qh, Kh, Vh)]
     Qd, Kd, Vd = dev_buffers
+    main = torch.cuda.current_stream()
+    side = _copy_stream()
     Qd.copy_(Qh, non_blocking=True)
     Kd.copy_(Kh, non_blocking=True)
-    Vd.copy_(Vh, non_blocking=True)
+    side.wait_stream(main)                      # V follows Q and K on the link; earlier work on Vd is finished too
+    with torch.cuda.stream(side):
+        Vd.copy_(Vh, non_blocking=True)
     plan = sparsepr_plan(Qd, Kd, Vd, params=params)
+    main.wait_stream(side)
     O = sparsepr_attend(plan, Qd, Kd, Vd)
     Oh.copy_(O, non_blocking=True)
-    torch.cuda.current_stream().synchronize()
+    main.synchronize()
     return Oh
+
+
+_COPY_STREAM = {}
+
+
+def _copy_stream():
+    d = torch.cuda.current_device()
+    if d not in _COPY_STREAM:
+        _COPY_STREAM[d] = torch.cuda.Stream(device=d)
+    return _COPY_STREAM[d]
