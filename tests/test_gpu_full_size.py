@@ -1,0 +1,67 @@
+"""Parity at the full size of the bench workload, on sampled output rows.
+
+The whole call runs on the GPU exactly as bench.py launches it (video-dit-480p-like:
+N = 32760, d = 128, bf16; four heads keep host memory and the oracle's time small).
+The oracle then evaluates, for the GPU's own plan, a sample of output rows one by
+one: ordinary rows, rows of short group remainders (handled by the remainder kernel),
+first rows of 128-row tiles, and probe rows.  Properties that hold at any size are
+checked on every head."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sparsepr_oracle as orc
+from paper_2608_18484_b200 import binding as B
+from paper_2608_18484_b200 import workloads as W
+from tests.gpu_util import heads_to_device, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def test_full_size_480p_sampled_rows():
+    wl = W.VIDEO_480P.scaled(H=4)
+    heads = [0, 1, 2, 3]
+    host, (Qd, Kd, Vd) = heads_to_device(wl, heads)
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale)
+    plan = B.sparsepr_plan(Qd, Kd, Vd, **kw)
+    O, Osp = B.sparsepr_attend(plan, Qd, Kd, Vd, return_sparse=True)
+    st = B.sparsepr_plan_stats(plan)
+    exp = B.sparsepr_plan_export(plan)
+    assert st["device_error"] == 0
+    assert torch.isfinite(O).all()
+    prm = orc.default_params(**kw)
+    C = -(-wl.N // wl.block)
+    budget = orc.pair_budget(wl.density, wl.N, wl.N, wl.n_probe)
+    rng = np.random.default_rng(7)
+    for i in heads:
+        aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
+        ptr, idx = exp["route_ptr"][i], exp["route_idx"][i]
+        n_q, n_k = np.bincount(aQ, minlength=C), np.bincount(aK, minlength=C)
+        # properties at any size: permutations, budget, probes
+        p0, _, o0 = orc.group_permutation(aQ, C)
+        assert np.array_equal(exp["q_perm"][i], p0) and np.array_equal(exp["q_off"][i], o0)
+        pairs = orc.routed_pairs(n_q, n_k, ptr, idx[:ptr[-1]])
+        assert pairs == exp["routed_pairs"][i] and pairs <= budget
+        assert len(set(exp["probe_idx"][i].tolist())) == wl.n_probe
+    # sampled rows against the oracle's evaluation of the GPU plan (head 0 and the last head)
+    for i in (0, 3):
+        Q, K, V = host[i]
+        aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
+        ptr, idx = exp["route_ptr"][i], exp["route_idx"][i]
+        P = exp["probe_idx"][i]
+        gplan = dict(scale=wl.softmax_scale, a_Q=aQ, a_K=aK, route_ptr=ptr, route_idx=idx[:ptr[-1]], probe_idx=P,
+                     M=len(P), probe_w=exp["probe_w"][i].astype(np.float64))
+        q_perm, q_off = exp["q_perm"][i], exp["q_off"][i]
+        sizes = np.diff(q_off)
+        rows = list(rng.choice(wl.N, 24, replace=False))
+        small = [a for a in range(C) if 0 < sizes[a] % 128 <= 64]
+        assert small, "the workload is expected to leave short remainders"
+        for a in small[:6]:                                     # last row of a short remainder, first row of the group
+            rows += [int(q_perm[q_off[a + 1] - 1]), int(q_perm[q_off[a]])]
+        rows += [int(p) for p in P[:4]]
+        rows = np.array(sorted(set(rows)), dtype=np.int64)
+        O_hat, O_sp, _ = orc.attend_head(Q, K, V, gplan, prm, rows=rows)
+        got, got_sp = to_np(O[0, i])[rows], to_np(Osp[0, i])[rows]
+        assert np.abs(got_sp - O_sp).max() <= 2e-2 and orc.rel_l2(got_sp, O_sp) <= 1e-2
+        assert np.abs(got - O_hat).max() <= 2e-2 and orc.rel_l2(got, O_hat) <= 1e-2

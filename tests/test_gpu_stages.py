@@ -9,7 +9,7 @@ from paper_2608_18484_b200 import binding as B
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("n,C,r", [(5000, 100, 48), (3001, 37, 64), (777, 300, 20), (64, 1, 7), (130, 130, 16)])
+@pytest.mark.parametrize("n,C,r", [(5000, 100, 48), (3001, 37, 64), (777, 300, 20), (64, 1, 7), (130, 130, 16), (6000, 1100, 64)])
 def test_assign_bit_exact(n, C, r):
     rng = np.random.default_rng(n + C)
     X = rng.normal(size=(n, r)).astype(np.float32)
