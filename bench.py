@@ -104,6 +104,17 @@ def launches_per_call(T, fitted, tensor_path):
     return plan + attend
 
 
+def max_over_ranks(value, device, world):
+    """The slowest replica decides: MAX of a per-rank time over the process group (identity at one rank)."""
+    import torch
+    if world <= 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def reference_arm(args, wl):
     """The oracle, as it stands, on a bounded sample: every step is one full call for one
     head of the workload cut to its first 3 frames."""
@@ -234,10 +245,7 @@ def main():
     barrier()
     step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
     total_ms = ev[0].elapsed_time(ev[-1])
-    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
 
     # ---- per-stage decomposition and the dense kernel of the same build (same K steps) ----
@@ -279,11 +287,9 @@ def main():
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1) / n_e2e
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = max_over_ranks(e2e_ms, dev, world)
         nbytes = Qd.numel() * Qd.element_size()
-        e2e = {"value": float(t.item()), "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes}
+        e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes}
 
     if rank != 0:
         if world > 1:
