@@ -164,15 +164,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
       const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
       const CUtensorMap* map = is_k ? &mapK : &mapV;
-      // key ranges (start row, length) of 32 consecutive routes live in the lanes' registers; the next
-      // 32 are prefetched while the current ones are consumed
-      auto load_range = [&](int t) -> int2 {
-        if (t >= nroute) return make_int2(0, 0);
-        if (!prm.sparse) return make_int2(0, prm.N);
-        const int g = ridx[t];
-        const int st = kvoff[g];
-        return make_int2(st, kvoff[g + 1] - st);
-      };
       int ri = 0, off = 0;
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {

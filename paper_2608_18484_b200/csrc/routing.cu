@@ -10,50 +10,74 @@ namespace spr {
 // theta_a would give ONE key at the centroid kappa_b:
 //   p_ab = exp(l_ab - LSE_a),  l_ab = s theta_a.kappa_b,
 //   LSE_a = log sum_{b non-empty} n_b exp(l_ab).
-// One CTA per query group; inner products and exponentials in float32 (differences and sums in float64),
-// scores stored as float32.
+// One CTA per eight query groups: the kappa slabs staged through shared memory are reused by all eight.
+// Inner products and exponentials in float32, the weighted sum of the exponentials in float64, scores stored as float32.
 // =============================================================================
+constexpr int kCsRows = 8;     // query groups per CTA
+
 __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ theta, const float* __restrict__ kappa,
                                                      const int* __restrict__ nq, const int* __restrict__ nk, int Cq,
                                                      int Ck, int d, float scale, float* __restrict__ score) {
-  __shared__ float th[128];
-  __shared__ double lg[kMaxGroups];
-  __shared__ double red[34];
-  const int bh = blockIdx.y, a = blockIdx.x;
+  __shared__ float th[kCsRows][128];
+  __shared__ float kt[32][257];                              // a [256 groups x 32 dims] slab of kappa, transposed
+  const int bh = blockIdx.y, a0 = blockIdx.x * kCsRows;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < kCsRows * d; e += 256) {
+    const int r = e / d, k = e % d;
+    th[r][k] = a0 + r < Cq ? theta[((i64)bh * Cq + a0 + r) * d + k] : 0.f;
+  }
+  // phase 1: logits l_ab = s theta_a . kappa_b of eight query groups against all K/V groups
+  for (int b0 = 0; b0 < Ck; b0 += 256) {
+    float acc[kCsRows];
+#pragma unroll
+    for (int r = 0; r < kCsRows; ++r) acc[r] = 0.f;
+    for (int k0 = 0; k0 < d; k0 += 32) {
+      __syncthreads();
+#pragma unroll 8
+      for (int r = 0; r < 32; ++r) {
+        const int b = b0 + warp * 32 + r;
+        kt[lane][warp * 32 + r] = (b < Ck && k0 + lane < d) ? kappa[((i64)bh * Ck + b) * d + k0 + lane] : 0.f;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < 32; ++k) {
+        const float kv = kt[k][tid];
+#pragma unroll
+        for (int r = 0; r < kCsRows; ++r) acc[r] = fmaf(th[r][k0 + k], kv, acc[r]);
+      }
+    }
+    const int b = b0 + tid;
+    if (b < Ck) {
+#pragma unroll
+      for (int r = 0; r < kCsRows; ++r)
+        if (a0 + r < Cq) score[((i64)bh * Cq + a0 + r) * Ck + b] = acc[r] * scale;
+    }
+  }
+  __syncthreads();                                           // the block's logits are visible to the block
+  // phase 2: one warp per query group: weighted log-sum-exp over the non-empty K/V groups, scores in place
+  const int a = a0 + warp;
+  if (a >= Cq) return;
   float* out = score + ((i64)bh * Cq + a) * Ck;
+  const int* nkh = nk + (i64)bh * Ck;
   if (nq[(i64)bh * Cq + a] == 0) {
-    for (int b = threadIdx.x; b < Ck; b += 256) out[b] = 0.f;
+    for (int b = lane; b < Ck; b += 32) out[b] = 0.f;
     return;
   }
-  if (threadIdx.x < d) th[threadIdx.x] = theta[((i64)bh * Cq + a) * d + threadIdx.x];
-  __syncthreads();
-  const int* nkh = nk + (i64)bh * Ck;
-  double mx = -1.0e300;
-  for (int b = threadIdx.x; b < Ck; b += 256) {
-    const float* kp = kappa + ((i64)bh * Ck + b) * d;
-    // float32 products in four independent chains (this GPU's float64 pipe is narrow)
-    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-    for (int k = 0; k < d; k += 4) {
-      const float4 v = *reinterpret_cast<const float4*>(kp + k);
-      l0 = fmaf(th[k], v.x, l0); l1 = fmaf(th[k + 1], v.y, l1); l2 = fmaf(th[k + 2], v.z, l2); l3 = fmaf(th[k + 3], v.w, l3);
-    }
-    double l = ((double)l0 + (double)l1) + ((double)l2 + (double)l3);
-    l *= (double)scale;
-    lg[b] = l;
-    if (nkh[b] > 0) mx = fmax(mx, l);
-  }
-  mx = block_max(mx, red);
+  float mx = -3.0e38f;
+  for (int b = lane; b < Ck; b += 32)
+    if (nkh[b] > 0) mx = fmaxf(mx, out[b]);
+  mx = warp_max(mx);
   double z = 0.0;
-  for (int b = threadIdx.x; b < Ck; b += 256)
-    if (nkh[b] > 0) z += (double)nkh[b] * (double)expf((float)(lg[b] - mx));
-  z = block_sum(z, red);
-  const double lse = mx + log(z);
-  for (int b = threadIdx.x; b < Ck; b += 256) out[b] = nkh[b] > 0 ? expf((float)(lg[b] - lse)) : 0.f;
+  for (int b = lane; b < Ck; b += 32)
+    if (nkh[b] > 0) z += (double)nkh[b] * (double)expf(out[b] - mx);
+  z = warp_sum(z);
+  const float lse = mx + (float)log(z);
+  for (int b = lane; b < Ck; b += 32) out[b] = nkh[b] > 0 ? expf(out[b] - lse) : 0.f;
 }
 
 void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
                         int d, float scale, float* score, cudaStream_t st) {
-  dim3 grid(Cq, BH);
+  dim3 grid((Cq + kCsRows - 1) / kCsRows, BH);
   k_cell_scores<<<grid, 256, 0, st>>>(theta, kappa, nq, nk, Cq, Ck, d, scale, score);
 }
 
