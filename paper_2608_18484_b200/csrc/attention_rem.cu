@@ -34,31 +34,35 @@ constexpr int kSubPerTile = kKeys / kSub;
 constexpr uint32_t kHalfBytes = kKeys * 128;          // [128 rows x 64 bf16]
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr uint32_t kSubBytes = kSub * 128;
-constexpr uint32_t kQHalf = kMaxQ * 128;              // [64 rows x 64 bf16]
-constexpr uint32_t kQBytes = 2 * kQHalf;              // 16 KB; the P^T buffers have the same shape
-constexpr int kStages = 2;
-
-struct Smem {
+// Shared memory and barriers of the instantiation for NQ = 16 NQC query rows.  The Q tile and the two P^T
+// buffers are [NQ rows x 128 bytes] x 2 halves; the bytes they do not need at small NQ go into deeper K and V
+// rings, because with few rows per tile the kernel is bound by the latency of the K/V stream (bytes in flight).
+template <int NQC> struct Cfg {
+  static constexpr int NQ = 16 * NQC;
+  static constexpr uint32_t kQHalf = NQ * 128;
+  static constexpr uint32_t kQBytes = 2 * kQHalf;
+  static constexpr int kStages = NQC == 1 ? 3 : 2;                  // per ring
   static constexpr uint32_t q = 0;
-  static constexpr uint32_t k = q + kQBytes;
+  static constexpr uint32_t p = q + ((kQBytes + 1023u) & ~1023u);                    // 2 groups
+  static constexpr uint32_t k = p + ((2 * kQBytes + 1023u) & ~1023u);
   static constexpr uint32_t v = k + kStages * kTileBytes;
-  static constexpr uint32_t p = v + kStages * kTileBytes;          // 2 groups
-  static constexpr uint32_t ranges = p + 2 * kQBytes;
+  static constexpr uint32_t ranges = v + kStages * kTileBytes;
   static constexpr uint32_t wmax = ranges + kMaxGroups * 8;        // float [2][4][64] per-warp tile maxima
-  static constexpr uint32_t mref = wmax + 2 * 4 * 64 * 4;          // float [2][64] reference maximum times scale (log2 domain)
+  static constexpr uint32_t mref = wmax + 2 * 4 * 64 * 4;          // float [2][64] reference maximum (log2 domain)
   static constexpr uint32_t corr = mref + 2 * 64 * 4;              // float [2][64] rescale factor of the current tile
   static constexpr uint32_t lsum = corr + 2 * 64 * 4;              // float [2][4][64] per-warp row sums (end)
-  static constexpr uint32_t fin = lsum + 2 * 4 * 64 * 4;           // float [2][64] final weights of the two groups; float [64] 1/l
+  static constexpr uint32_t fin = lsum + 2 * 4 * 64 * 4;           // float [2][64] final weights of the two groups
   static constexpr uint32_t gmask = fin + 3 * 64 * 4;              // unsigned [2][4][2] per-warp masks of queries whose maximum grew
   static constexpr uint32_t meta = gmask + 64;                     // uint2[8]
   static constexpr uint32_t bars = meta + 8 * 8;
   static constexpr uint32_t misc = bars + 32 * 8;                  // tmem base, abort, boxes, skip, moved[2]
   static constexpr uint32_t total = misc + 64;
+  enum { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kStages, V_FULL = K_EMPTY + kStages, V_EMPTY = V_FULL + kStages,
+         S_FULL = V_EMPTY + kStages, P_FULL = S_FULL + 2, P_EMPTY = P_FULL + 2, O_DONE = P_EMPTY + 2, META_FULL,
+         kNumBars = META_FULL + 8 };
+  static_assert(kNumBars <= 32, "barrier area");
+  static_assert(total <= 227 * 1024, "shared memory");
 };
-enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kStages, V_FULL = K_EMPTY + kStages, V_EMPTY = V_FULL + kStages,
-           S_FULL = V_EMPTY + kStages, P_FULL = S_FULL + 2, P_EMPTY = P_FULL + 2, O_DONE = P_EMPTY + 2, META_FULL,
-           kNumBars = META_FULL + 8 };
-static_assert(kNumBars <= 32, "barrier area");
 
 struct Params {
   int BH, N, Cq, Ck;
@@ -101,7 +105,13 @@ template <int NQC>
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_rem(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, Params prm) {
-  constexpr int NQ = 16 * NQC;
+  using Smem = Cfg<NQC>;
+  using C = Cfg<NQC>;
+  constexpr int NQ = C::NQ;
+  constexpr int kStages = C::kStages;
+  constexpr uint32_t kQHalf = C::kQHalf, kQBytes = C::kQBytes;
+  constexpr int Q_FULL = C::Q_FULL, K_FULL = C::K_FULL, K_EMPTY = C::K_EMPTY, V_FULL = C::V_FULL, V_EMPTY = C::V_EMPTY, S_FULL = C::S_FULL,
+                P_FULL = C::P_FULL, P_EMPTY = C::P_EMPTY, O_DONE = C::O_DONE, META_FULL = C::META_FULL, kNumBars = C::kNumBars;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
@@ -169,7 +179,7 @@ k_attention_rem(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const bool is_k = warp == 8;
       if (is_k && lane == 0) {
         mbar_expect_tx(bar(Q_FULL), kQBytes);
-        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, bh, 0);               // 64-row box; rows past nq are never used
+        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, bh, 0);               // NQ-row box; rows past nq are never used
         tma_load_4d(base + Smem::q + kQHalf, &mapQ, bar(Q_FULL), 64, row0, bh, 0);
       }
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
@@ -487,10 +497,10 @@ k_attention_rem(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 cudaError_t init_attention_rem() {
   using namespace tc::rem;
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(k_attention_rem<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(k_attention_rem<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(k_attention_rem<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_attention_rem<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total);
+  if ((e = cudaFuncSetAttribute(k_attention_rem<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<1>::total)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(k_attention_rem<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<2>::total)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(k_attention_rem<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<3>::total)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_attention_rem<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<4>::total);
 }
 
 // Remainders of 1..64 rows of every query group (the 128-row kernel must have been given tile offsets
@@ -498,9 +508,10 @@ cudaError_t init_attention_rem() {
 bool launch_attention_rem(const AttnArgs& a, cudaStream_t st) {
   using namespace tc;
   using namespace tc::rem;
-  CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kMaxQ) || !make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) ||
-      !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub))
+  CUtensorMap mq[4], mk, mv;
+  for (int z = 0; z < 4; ++z)
+    if (!make_map(&mq[z], a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, 16 * (z + 1))) return false;
+  if (!make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) || !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub))
     return false;
   Params p{};
   p.BH = a.BH; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.scale_log2 = a.scale * 1.4426950408889634f;
@@ -508,10 +519,10 @@ bool launch_attention_rem(const AttnArgs& a, cudaStream_t st) {
   p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
   p.H = a.H; p.O_sparse = a.O_sparse; p.err = a.err;
   const dim3 grid(a.Cq, a.BH);
-  k_attention_rem<1><<<grid, kThreads, Smem::total, st>>>(mq, mk, mv, p);
-  k_attention_rem<2><<<grid, kThreads, Smem::total, st>>>(mq, mk, mv, p);
-  k_attention_rem<3><<<grid, kThreads, Smem::total, st>>>(mq, mk, mv, p);
-  k_attention_rem<4><<<grid, kThreads, Smem::total, st>>>(mq, mk, mv, p);
+  k_attention_rem<1><<<grid, kThreads, Cfg<1>::total, st>>>(mq[0], mk, mv, p);
+  k_attention_rem<2><<<grid, kThreads, Cfg<2>::total, st>>>(mq[1], mk, mv, p);
+  k_attention_rem<3><<<grid, kThreads, Cfg<3>::total, st>>>(mq[2], mk, mv, p);
+  k_attention_rem<4><<<grid, kThreads, Cfg<4>::total, st>>>(mq[3], mk, mv, p);
   return true;
 }
 
