@@ -170,21 +170,23 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       const float xn = row < prm.N ? prm.xnorm[(i64)bh * prm.N + row] : 0.f;   // needed after the scores: fetched now
       if (prm.sums) {
         const int rowbase = (tile0 + tl) * 128 + wq * 32;
-        const bool c0ok = lane < prm.r, c1ok = lane + 32 < prm.r;
+        // this lane's columns are (2 lane, 2 lane + 1): one 8-byte load per row (ldphi is a multiple of 16, and
+        // columns r..ldphi-1 hold zeros, so a pair that straddles r reads a zero)
+        const bool cok = 2 * lane < prm.r;
         if (rowbase + 31 < prm.N) {                            // every tile but the last of a head (uniform)
-          const float* xb = prm.phi + ((i64)bh * prm.N + rowbase) * prm.ldphi + lane;
+          const float* xb = prm.phi + ((i64)bh * prm.N + rowbase) * prm.ldphi + 2 * lane;
 #pragma unroll
           for (int rr = 0; rr < 32; ++rr) {
-            pv0[rr] = c0ok ? xb[rr * prm.ldphi] : 0.f;
-            pv1[rr] = c1ok ? xb[rr * prm.ldphi + 32] : 0.f;
+            const float2 x2 = cok ? *reinterpret_cast<const float2*>(xb + rr * prm.ldphi) : make_float2(0.f, 0.f);
+            pv0[rr] = x2.x; pv1[rr] = x2.y;
           }
         } else {
 #pragma unroll
           for (int rr = 0; rr < 32; ++rr) {
             const int rw = min(rowbase + rr, prm.N - 1);
-            const float* xr = prm.phi + ((i64)bh * prm.N + rw) * prm.ldphi;
-            pv0[rr] = c0ok ? xr[lane] : 0.f;
-            pv1[rr] = c1ok ? xr[lane + 32] : 0.f;
+            const float* xr = prm.phi + ((i64)bh * prm.N + rw) * prm.ldphi + 2 * lane;
+            const float2 x2 = cok ? *reinterpret_cast<const float2*>(xr) : make_float2(0.f, 0.f);
+            pv0[rr] = x2.x; pv1[rr] = x2.y;
           }
         }
       }
@@ -236,7 +238,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       }
       SPR_KE(eD);
       if (prm.sums) {
-        // warp-level pre-aggregation: lanes = feature columns (lane, lane+32); the 32 rows of the
+        // warp-level pre-aggregation: lanes = feature columns (2 lane, 2 lane + 1); the 32 rows of the
         // warp were prefetched above; one fixed-point atomic per (cluster, column)
         unsigned todo = __ballot_sync(FULL, decided);
         // 2^shift as a float: scaling a float32 partial sum by a power of two is exact, so the conversion below
@@ -258,8 +260,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           }
           const i64 acc0 = __float2ll_rn(a0 * scl), acc1 = __float2ll_rn(a1 * scl);
           i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
-          if (lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane), (u64)acc0);
-          if (lane + 32 < prm.r) atomicAdd(reinterpret_cast<u64*>(s + lane + 32), (u64)acc1);
+          if (2 * lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + 2 * lane), (u64)acc0);
+          if (2 * lane + 1 < prm.r) atomicAdd(reinterpret_cast<u64*>(s + 2 * lane + 1), (u64)acc1);
           if (lane == 0) atomicAdd(prm.counts + (i64)bh * prm.C + cl, __popc(members));
         }
       }
