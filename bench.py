@@ -152,11 +152,11 @@ def reference_arm(args, wl):
 
 
 def cpu_baseline(wl):
-    """Oracle timed on the host cores on about 10-20 s of work: one head, first 11 frames."""
+    """Oracle timed on the host cores on about 10-20 s of work: one head, first 16 frames."""
     import multiprocessing
     from oracle import sparsepr_oracle as orc
     from paper_2608_18484_b200 import workloads as W
-    frames = min(11, wl.grid[0])
+    frames = min(16, wl.grid[0])
     small = wl.scaled(grid=(frames,) + tuple(wl.grid[1:]))
     prm = orc.default_params(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
                              softmax_scale=wl.softmax_scale)

@@ -40,6 +40,9 @@ CASES = [
     ("tiny-f32-ragged", W.TINY.scaled(grid=(3, 31, 29)), dict()),               # N = 2697: ragged tiles everywhere
     ("480p-like-bf16", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64), dict()),
     ("world-like-bf16", W.WORLD.scaled(grid=(3, 32, 64), H=2, n_probe=96), dict()),
+    ("720p-like-bf16", W.VIDEO_720P.scaled(grid=(2, 45, 80), H=2, n_probe=64), dict()),
+    ("480p-like-bf16-sparser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.12), dict()),
+    ("480p-like-bf16-denser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.35), dict(r_out=128)),
 ]
 
 
