@@ -307,11 +307,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tmem_ld_wait();
       SPR_ACC(tl);
       if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
+        // only the boxes that end a key range (or lie beyond the stream) have columns to mask; the test is uniform
 #pragma unroll
         for (int box = 0; box < 8; ++box) {
           const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;      // last valid column of the box
+          if (lim != 15) {
 #pragma unroll
-          for (int c = 0; c < 16; ++c) s[box * 16 + c] = (c <= lim) ? s[box * 16 + c] : -INFINITY;
+            for (int c = 0; c < 16; ++c) s[box * 16 + c] = (c <= lim) ? s[box * 16 + c] : -INFINITY;
+          }
         }
       }
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
