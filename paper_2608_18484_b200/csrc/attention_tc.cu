@@ -2,20 +2,21 @@
 //
 // One CTA processes one 128-row query tile (of one query group, Eq. 3; or of the whole
 // head for dense attention, Eq. 1).  Roles:
-//   warps 0-3  softmax group A: even key tiles, one thread per query row
-//   warps 4-7  softmax group B: odd key tiles
-//   warp  8    TMA producer: streams the routed keys/values as one concatenated
-//              sequence in 16-row boxes (tiles of 128 keys, only range ends are ragged)
+//   warps 0-7  softmax: warps w and w+4 share the 32 rows of TMEM quadrant w and split the
+//              128 scores of a row in two halves (keys 0-63 / 64-127 of the tile)
+//   warp  8    TMA producer of Q and the key tiles (+ tile meta ring)
 //   warp  9    tcgen05.mma issuer; owns the TMEM allocation
-// Data path per key tile i (group g = i mod 2):
-//   S_g = Q K_i^T        tcgen05.mma, smem x smem -> TMEM (fp32)
-//   P   = exp2(.)        softmax thread: tcgen05.ld S_g, reference max / row sum, bf16 P written
-//                        back over the first half of S_g with tcgen05.st
-//   O_g += P V_i         tcgen05.mma with the A operand read from TMEM; O_g stays in TMEM
-// While group A works on tile i the tensor cores already produce S_B for tile i+1.
-// Epilogue: merge (O_A, O_B) like two splits of the key range, O_sp = O / l, store at the
-// original token index (inverse permutation).  The residual correction of Eq. 9 is a pass
-// of its own (correction_tc.cu) so that the fit can overlap this kernel.
+//   warp  10   TMA producer of the value tiles
+// The routed keys/values arrive as one concatenated sequence in 16-row boxes (tiles of 128
+// keys, only range ends are ragged).  Data path per key tile i:
+//   S_b = Q K_i^T        tcgen05.mma, smem x smem -> TMEM (fp32), two score buffers b = i mod 2, so
+//                        the product of tile i+1 runs while tile i is in the softmax
+//   P   = exp2(.)        softmax threads: tcgen05.ld their half row of S_b, row maximum (the two
+//                        halves meet through shared memory), bf16 P to its own TMEM columns
+//   O  += P V_i          tcgen05.mma with the A operand read from TMEM; O stays in TMEM
+// The reference maximum of a row moves only when it grows by more than 2^8 (then O is rescaled).
+// Epilogue: O / l, store at the original token index (inverse permutation).  The residual
+// correction of Eq. 9 is a pass of its own (correction_tc.cu) so that the fit can overlap this kernel.
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
@@ -49,8 +50,8 @@ struct Smem {                          // offsets from a 1024-byte aligned base
   static constexpr uint32_t k = q + kTileBytes;
   static constexpr uint32_t v = k + kKStages * kTileBytes;
   static constexpr uint32_t ranges = v + kVStages * kTileBytes;
-  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;     // float2[2][128]
-  static constexpr uint32_t meta = xchg + 2 * 128 * 8;            // uint2[8]: ring of per-tile box counts
+  static constexpr uint32_t xchg = ranges + kMaxGroups * 8;     // float [2 tile parities][2 halves][128] row maxima; float [2][128] row sums
+  static constexpr uint32_t meta = xchg + 6 * 128 * 4;            // uint2[8]: ring of per-tile box counts
   static constexpr uint32_t bars = meta + 8 * 8;                  // kNumBars mbarriers
   static constexpr uint32_t misc = bars + 32 * 8;                 // tmem base, abort flag, counters
   static constexpr uint32_t total = misc + 64;
@@ -58,7 +59,7 @@ struct Smem {                          // offsets from a 1024-byte aligned base
 constexpr size_t kSmemBytes = Smem::total;                        // the dynamic segment is 1024-byte aligned and the only shared memory
 
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kKStages, V_FULL = K_EMPTY + kKStages, V_EMPTY = V_FULL + kVStages,
-           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, META_FULL,
+           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, P_EMPTY, O_DONE, META_FULL,
            kNumBars = META_FULL + 8 };
 static_assert(kNumBars <= 32, "barrier area");
 
@@ -80,7 +81,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
   int2* ranges = reinterpret_cast<int2*>(sm + Smem::ranges);
-  float2* stat = reinterpret_cast<float2*>(sm + Smem::xchg);               // [2][128] (m_ref, l) of both groups
+  float* xmax = reinterpret_cast<float*>(sm + Smem::xchg);                 // [2][2][128] half-row maxima of the current / next tile
+  float* xsum = xmax + 4 * 128;                                            // [2][128] half-row sums (end)
   uint2* meta = reinterpret_cast<uint2*>(sm + Smem::meta);
   volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem base, [1] abort, [2] total boxes
   const uint32_t bars = base + Smem::bars;
@@ -123,7 +125,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i)
-      mbar_init(bar(i), (i == P_FULL || i == P_FULL + 1) ? 128 : 1);
+      mbar_init(bar(i), i == P_FULL ? 256 : 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -206,7 +208,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
   } else if (warp == 9) {
     // =========================== MMA issuer ==============================================
-    // TMEM columns: S_A [0,128), S_B [128,256), O_A [256,384), O_B [384,512); P_g overwrites S_g[0,64)
+    // TMEM columns: S_0 [0,128), S_1 [128,256), P [256,320) (two bf16 per column), O [320,448)
     if (lane == 0 && n_tiles > 0) {
       const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
       // descriptors are built once; inside the loops only their address field moves (in 16-byte units),
@@ -241,25 +243,26 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #define SPR_MACC(v)
 #endif
       for (int i = 0; i < n_tiles && ok; ++i) {
-        const int g = i & 1, j = i >> 1, s = i % kVStages;
+        const int s = i % kVStages;
         const uint2 mt = meta[i & 7];
         SPR_M0();
         if (!mbar_wait(bar(V_FULL + s), (i / kVStages) & 1, abort_flag)) { ok = false; break; }
         SPR_MACC(mv);
-        if (!mbar_wait(bar(P_FULL + g), j & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, O_g rescaled if needed
+        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, S_(i mod 2) read, O rescaled if needed
         SPR_MACC(mp);
         tc_fence_after();
-        const uint32_t d = tmem + 256u + (uint32_t)g * 128u;
-        const uint32_t pa = tmem + (uint32_t)g * 128u;
+        const uint32_t d = tmem + 320u;
+        const uint32_t pa = tmem + 256u;
         const int nsub = (int)mt.y;
         const uint64_t vd = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
 #pragma unroll
         for (int kk = 0; kk < kSubPerTile; ++kk)
           if (kk < nsub)
-            umma_bf16_ts(d, pa + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);   // O_g accumulates over its tiles
+            umma_bf16_ts(d, pa + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(V_EMPTY + s));
+        umma_commit(bar(P_EMPTY));
         SPR_MACC(mi);
-        if (i + 2 < n_tiles) ok = issue_qk(i + 2);          // S_g (and the P_g inside it) is rewritten after P V (i)
+        if (i + 2 < n_tiles) ok = issue_qk(i + 2);          // score buffer i mod 2 is free again
         SPR_MACC(mq);
       }
 #ifdef SPR_ATTN_TIMING
@@ -271,17 +274,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
   } else {
     // =========================== softmax (warps 0-7) =======================================
-    // Group A (warps 0-3) takes the even key tiles, group B (warps 4-7) the odd ones; one thread
-    // per query row and tile (128 scores).  Each group has its own score buffer, its own output
-    // accumulator O_g in TMEM and its own running (m_ref, l); the two partial results are merged
-    // at the end like two splits of the key range.  O_g is rescaled only when the row maximum has
-    // grown by more than 2^8 over the reference maximum, so exponentials stay below 2^8.
-    const int g = warp >> 2, wq = warp & 3;
+    // Thread (half hh, quadrant wq, lane) owns the 64 scores of keys [64 hh, 64 hh + 64) of query row
+    // 32 wq + lane; warps wq and wq + 4 meet at the named barrier 1 + wq to agree on the row maximum.
+    const int hh = warp >> 2, wq = warp & 3;
     const int row = wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t FULL = 0xffffffffu;
-    const uint32_t s_addr = tmem + lane_addr + (uint32_t)g * 128u;
-    const uint32_t o_addr = tmem + lane_addr + 256u + (uint32_t)g * 128u;
+    const uint32_t p_addr = tmem + lane_addr + 256u + (uint32_t)hh * 32u;
+    const uint32_t o_addr = tmem + lane_addr + 320u + (uint32_t)hh * 64u;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
@@ -293,45 +293,58 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #define SPR_T0()
 #define SPR_ACC(v)
 #endif
-    for (int i = g, j = 0; i < n_tiles; i += 2, ++j) {
+    for (int i = 0; i < n_tiles; ++i) {
       SPR_T0();
-      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + g), j & 1, abort_flag) &&
+      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
                                 mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
-      if (!ok) continue;                                         // warp-uniform
-      tc_fence_after();
-      const uint2 mt = meta[i & 7];
-      float s[128];
+      float s[64];
+      float mx = -INFINITY;
+      if (ok) {
+        tc_fence_after();
+        const uint2 mt = meta[i & 7];
+        const uint32_t s_addr = tmem + lane_addr + (uint32_t)(i & 1) * 128u + (uint32_t)hh * 64u;
+        tmem_ld32_nowait(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
+        tmem_ld32_nowait(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+        SPR_ACC(tw);
+        tmem_ld_wait();
+        SPR_ACC(tl);
+        if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
+          // only the boxes that end a key range (or lie beyond the stream) have columns to mask; the test is uniform
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tmem_ld32_nowait(s_addr + q * 32, *reinterpret_cast<float(*)[32]>(&s[q * 32]));   // four loads in flight, one wait
-      SPR_ACC(tw);
-      tmem_ld_wait();
-      SPR_ACC(tl);
-      if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
-        // only the boxes that end a key range (or lie beyond the stream) have columns to mask; the test is uniform
+          for (int bx = 0; bx < 4; ++bx) {
+            const int box = hh * 4 + bx;
+            const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;      // last valid column of the box
+            if (lim != 15) {
 #pragma unroll
-        for (int box = 0; box < 8; ++box) {
-          const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;      // last valid column of the box
-          if (lim != 15) {
-#pragma unroll
-            for (int c = 0; c < 16; ++c) s[box * 16 + c] = (c <= lim) ? s[box * 16 + c] : -INFINITY;
+              for (int c = 0; c < 16; ++c) s[bx * 16 + c] = (c <= lim) ? s[bx * 16 + c] : -INFINITY;
+            }
           }
         }
-      }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 128; c += 4) {
-        mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
-        mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+        for (int c = 0; c < 64; c += 4) {
+          mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+          mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+        }
+        mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      const bool move = (mx - m_ref) * sc > 8.f;                 // true on the group's first tile (m_ref = -inf)
+      // the two halves of the row exchange their maxima (buffer of this tile's parity; executed whatever happened)
+      float* xm = xmax + (i & 1) * 256;
+      xm[hh * 128 + row] = mx;
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+      mx = fmaxf(mx, xm[(hh ^ 1) * 128 + row]);
+      const bool move = (mx - m_ref) * sc > 8.f;                 // true on the first tile (m_ref = -inf); same in both halves
       const float m_new = move ? mx : m_ref;
       const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f; // 0 on the first tile
       const float mneg = -m_new * sc;
       m_ref = m_new;
-      if (j > 0 && __any_sync(FULL, move)) {                     // rescale this warp's rows of O_g (rare)
+      // P and O of the previous tile must have been consumed before they are touched
+      if (i > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
+      if (!ok) continue;                                         // warp-uniform; the pair barrier above has been passed
+      tc_fence_after();
+      if (i > 0 && __any_sync(FULL, move)) {                     // rescale this half of the warp's O rows (rare)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < 2; ++q) {
           float t[32];
           tmem_ld32(o_addr + q * 32, t);
 #pragma unroll
@@ -341,63 +354,52 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 128; c += 4) {
+      for (int c = 0; c < 64; c += 4) {
         s[c] = ex2(fmaf(s[c], sc, mneg)); s[c + 1] = ex2(fmaf(s[c + 1], sc, mneg));
         s[c + 2] = ex2(fmaf(s[c + 2], sc, mneg)); s[c + 3] = ex2(fmaf(s[c + 3], sc, mneg));
         ps4[0] += s[c]; ps4[1] += s[c + 1]; ps4[2] += s[c + 2]; ps4[3] += s[c + 3];
       }
       l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
-      // P (bf16, two per 32-bit column) over the first 64 columns of the score buffer
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
+      // P (bf16, two per 32-bit column): this half's 64 probabilities -> 32 columns
+      {
         uint32_t w[32];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[q * 64 + 2 * c], s[q * 64 + 2 * c + 1]);
-        if (q == 0) SPR_ACC(tm);
-        tmem_st32u(s_addr + q * 32, w);
+        for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[2 * c], s[2 * c + 1]);
+        SPR_ACC(tm);
+        tmem_st32u(p_addr, w);
       }
       tc_fence_before();
-      mbar_arrive(bar(P_FULL + g));
+      mbar_arrive(bar(P_FULL));
       SPR_ACC(ts);
     }
 #ifdef SPR_ATTN_TIMING
     if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 4))
-      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  math %lld  pack+st %lld (cycles per tile)\n", warp, (n_tiles + 1 - g) / 2,
-             tw / max(1, (n_tiles + 1 - g) / 2), tl / max(1, (n_tiles + 1 - g) / 2), tm / max(1, (n_tiles + 1 - g) / 2), ts / max(1, (n_tiles + 1 - g) / 2));
+      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  math %lld  pack+st %lld (cycles per tile)\n", warp, n_tiles,
+             tw / max(1, n_tiles), tl / max(1, n_tiles), tm / max(1, n_tiles), ts / max(1, n_tiles));
 #endif
-    // ---- merge the two groups, normalise ------------------------------------------------------
+    // ---- row sums of the two halves, normalise, store ------------------------------------------
     if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
-    stat[g * 128 + row] = make_float2(m_ref, l);
-    asm volatile("bar.sync 1, 256;" ::: "memory");               // all softmax threads, whatever happened
-    const float2 sa = stat[row], sb = stat[128 + row];
-    const float mm = fmaxf(sa.x, sb.x);
-    const float wa = sa.y > 0.f ? ex2((sa.x - mm) * sc) : 0.f;
-    const float wb = sb.y > 0.f ? ex2((sb.x - mm) * sc) : 0.f;
-    const float ltot = sa.y * wa + sb.y * wb;
+    xsum[hh * 128 + row] = l;
+    asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+    const float ltot = l + xsum[(hh ^ 1) * 128 + row];
     const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
-    // this thread finishes output columns [64 g, 64 g + 64) of its row
+    // this thread finishes output columns [64 hh, 64 hh + 64) of its row
     float o[64];
 #pragma unroll
     for (int c = 0; c < 64; ++c) o[c] = 0.f;
     if (ok && n_tiles > 0) {
       tc_fence_after();
-      const float fa = wa * inv, fb = wb * inv;
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         float t[32];
-        tmem_ld32(tmem + lane_addr + 256u + g * 64 + q * 32, t);
+        tmem_ld32(o_addr + q * 32, t);
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[q * 32 + c] = fa != 0.f ? t[c] * fa : 0.f;
-        if (n_tiles > 1) {                                        // group B exists only then (uniform)
-          tmem_ld32(tmem + lane_addr + 384u + g * 64 + q * 32, t);
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[q * 32 + c] += fb != 0.f ? t[c] * fb : 0.f;
-        }
+        for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
       }
     }
     if (ok && row < nrows) {
       const int dst = prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + row] : row0 + row;
-      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + g * 64;
+      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + hh * 64;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {
         float v8[8];
@@ -406,7 +408,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         store8(op + ch * 8, v8);
       }
       if (prm.O_sparse) {
-        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + g * 64;
+        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
           float v8[8];
