@@ -91,6 +91,7 @@ cudaError_t ensure_init() {
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_correction_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_rem()) != cudaSuccess) { g_init_err = e; return; }
+    if ((e = init_attention_packed()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_project_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_probe_tc()) != cudaSuccess) { g_init_err = e; return; }
@@ -160,6 +161,7 @@ struct sparsepr_plan_s {
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
   __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged;
+  int *rem_pos, *rem_grp, *rem_cnt;      // rows of the short group remainders (packed attention tiles)
 };
 
 namespace {
@@ -197,8 +199,9 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   __nv_bfloat16* mh = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64); __nv_bfloat16* ml = c.take<__nv_bfloat16>(BH * (size_t)r.Cmax * 64);
   float* xnorm = c.take<float>(BH * N); int* flagged = c.take<int>(BH * N);
   __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
+  int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
   if (p) {
-    p->Ft = Ft;
+    p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -418,6 +421,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
                       p->route_idx, p->rstate, nullptr, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
+  launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
   if (overlap) join_side(p, st);
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
@@ -469,6 +473,7 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
+  launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
   if (!launch_ok() || cudaStreamSynchronize(st) != cudaSuccess) { delete p; return SPARSEPR_ERR_CUDA; }
   *out = p;
   return SPARSEPR_OK;
@@ -534,7 +539,10 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   }
   if (tensor) {
     aa.tile_off = p->tile_off128;
-    if (!launch_attention_tc(aa, st) || !launch_attention_rem(aa, st)) return SPARSEPR_ERR_CUDA;
+    if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
+    if (std::getenv("SPARSEPR_REM_TRANSPOSED") ? !launch_attention_rem(aa, st)
+                                               : !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, st))
+      return SPARSEPR_ERR_CUDA;
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) join_side(p, st);
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;

@@ -1,0 +1,415 @@
+// Block-sparse attention (Eq. 3) for the short remainders of the query groups (bf16, d = d_v = 128).
+//
+// A query group of n rows gives floor(n / 128) full tiles to the 128-row kernel; when the n mod 128 rows
+// that are left are at most kRemRows they come here.  An M = 128 tensor-core tile for a handful of rows
+// costs as much as a full one, and rows of different groups attend to different keys, so the
+// remainders of MANY groups are packed into common 128-row tiles instead: such a tile walks over ALL
+// keys of the head (group-major order) and every row masks the K/V groups that its own query group
+// does not route to.  At a routed density of 25 % and 16-row remainders that is about a third of the
+// tile passes that one tile per remainder needs.
+//
+//   warps 0-7  softmax: warps w and w+4 share the 32 rows of TMEM quadrant w and split the 128 scores
+//              of a row in two halves; they also bring the query rows into tensor memory (the rows of a
+//              packed tile are scattered, so there is no TMA box for them)
+//   warp  8    K producer; cuts the key sequence into tiles that span at most 8 K/V groups and publishes
+//              the group runs of every tile;  warp 10  V producer
+//   warp  9    tcgen05.mma issuer; owns the TMEM allocation
+// TMEM: S_0 [0,128), S_1 [128,256), P [256,320), O [320,448), Q [448,512); both products take their A
+// operand from tensor memory.  Reference maxima move lazily (growth beyond 2^8), as in the 128-row kernel.
+// Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
+#include <cuda.h>
+#include "kernels.cuh"
+#include "tc_common.cuh"
+
+namespace spr {
+namespace tc {
+namespace packed {
+
+constexpr int kThreads = 352;
+constexpr int kTile = 128;
+constexpr int kD = 128;
+constexpr uint32_t kHalfBytes = kTile * 128;          // [128 rows x 64 bf16]
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
+constexpr int kStages = 2;
+constexpr int kMaxRuns = 8;                            // K/V-group runs per key tile
+
+struct Meta { int ncols, nruns; unsigned short grp[kMaxRuns]; unsigned char end[kMaxRuns]; };   // 32 bytes
+
+struct Smem {
+  static constexpr uint32_t k = 0;
+  static constexpr uint32_t v = k + kStages * kTileBytes;
+  static constexpr uint32_t bitmap = v + kStages * kTileBytes;           // [kMaxGroups/32 words][128 rows]
+  static constexpr uint32_t xchg = bitmap + (kMaxGroups / 32) * 128 * 4; // float [2][2][128] half-row maxima, [2][128] half-row sums
+  static constexpr uint32_t meta = xchg + 6 * 128 * 4;                   // Meta[8]
+  static constexpr uint32_t bars = meta + 8 * 32;
+  static constexpr uint32_t misc = bars + 32 * 8;
+  static constexpr uint32_t total = misc + 64;
+};
+enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kStages, V_FULL = K_EMPTY + kStages, V_EMPTY = V_FULL + kStages,
+           S_FULL = V_EMPTY + kStages, P_FULL = S_FULL + 2, P_EMPTY, O_DONE, META_FULL, kNumBars = META_FULL + 8 };
+static_assert(kNumBars <= 32, "barrier area");
+
+struct Params {
+  int BH, H, N, Cq, Ck;
+  float scale_log2;
+  const int *rem_pos, *rem_grp, *rem_cnt;      // [BH][N] group-major position and query group of every packed row; [BH] their number
+  const int *kv_off, *route_ptr, *route_idx, *q_perm;
+  const __nv_bfloat16* Qg;                     // [BH][N][128] group-major
+  __nv_bfloat16* O; i64 os[3];
+  float* O_sparse;
+  int* err;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Params prm) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* sm = smem_raw;
+  unsigned* bitmap = reinterpret_cast<unsigned*>(sm + Smem::bitmap);
+  float* xmax = reinterpret_cast<float*>(sm + Smem::xchg);
+  float* xsum = xmax + 4 * 128;
+  Meta* meta = reinterpret_cast<Meta*>(sm + Smem::meta);
+  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem, [1] abort, [3] skip
+  const uint32_t bars = base + Smem::bars;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y, m0 = blockIdx.x * kTile;
+  const int cnt = prm.rem_cnt[bh];
+  if (m0 >= cnt) return;
+  const int nrows = min(kTile, cnt - m0);
+  if (tid == 0) {
+    misc[3] = (prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT) || (base & 1023u) != 0;
+    if ((base & 1023u) != 0) set_error(prm.err, SPARSEPR_ERR_CUDA);
+  }
+  __syncthreads();
+  if (misc[3]) return;
+  const int words = (prm.Ck + 31) / 32;
+  const int* rpos = prm.rem_pos + (i64)bh * prm.N + m0;
+  const int* rgrp = prm.rem_grp + (i64)bh * prm.N + m0;
+
+  if (tid == 0) {
+    for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == P_FULL || i == Q_FULL) ? 256 : 1);
+    misc[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 9) tmem_alloc(base + Smem::misc, 512);
+  // route bitmap of every row of the tile, transposed: bitmap[word][row]
+  for (int e = tid; e < words * 128; e += kThreads) bitmap[e] = 0u;
+  __syncthreads();
+  for (int r = tid >> 1; r < nrows; r += kThreads / 2) {
+    const int g = rgrp[r];
+    const int* rp = prm.route_ptr + (i64)bh * (prm.Cq + 1);
+    const int* ri = prm.route_idx + (i64)bh * prm.Cq * prm.Ck;
+    for (int t = rp[g] + (tid & 1); t < rp[g + 1]; t += 2) atomicOr(&bitmap[(ri[t] >> 5) * 128 + r], 1u << (ri[t] & 31));
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = (uint32_t)misc[0];
+  volatile int* abort_flag = &misc[1];
+  const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
+  const int p_end = prm.N;
+
+  // Tiles are cut so that none spans more than kMaxRuns K/V groups; every role that walks the key sequence
+  // uses this function.  `g` = group that contains `pos`.
+  auto next_tile = [&](int pos, int& g, Meta* out) -> int {
+    int runs = 0, c = 0;
+    while (c < kTile && pos + c < p_end && runs < kMaxRuns) {
+      while (kvoff[g + 1] <= pos + c) ++g;                        // skip empty groups
+      const int e = min(min(kvoff[g + 1], p_end) - pos, kTile);
+      if (out) { out->grp[runs] = (unsigned short)g; out->end[runs] = (unsigned char)(e - 1); }
+      c = e;
+      ++runs;
+    }
+    if (out) { out->ncols = c; out->nruns = runs; }
+    return c;
+  };
+
+  if (warp == 8 || warp == 10) {
+    // =========================== producers ==================================================
+    if (lane == 0) {
+      const bool is_k = warp == 8;
+      const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
+      const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
+      const CUtensorMap* map = is_k ? &mapK : &mapV;
+      int g = 0, pos = 0;
+      for (int i = 0; pos < p_end; ++i) {
+        const int s = i % kStages;
+        Meta mt;
+        const int nc = next_tile(pos, g, &mt);
+        if (!mbar_wait(bar(empty0 + s), ((i / kStages) & 1) ^ 1, abort_flag)) break;
+        if (is_k) {
+          meta[i & 7] = mt;
+          mbar_arrive(bar(META_FULL + (i & 7)));
+        }
+        mbar_expect_tx(bar(full0 + s), kTileBytes);
+        tma_load_4d(buf0 + s * kTileBytes, map, bar(full0 + s), 0, pos, bh, 0);
+        tma_load_4d(buf0 + s * kTileBytes + kHalfBytes, map, bar(full0 + s), 64, pos, bh, 0);
+        pos += nc;
+      }
+    }
+  } else if (warp == 9) {
+    // =========================== MMA issuer ==================================================
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
+      const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
+      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
+      int n_tiles = 0;
+      { int g = 0; for (int pos = 0; pos < p_end; ++n_tiles) pos += next_tile(pos, g, nullptr); }
+      bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
+      auto issue_qk = [&](int i) -> bool {
+        const int s = i % kStages;
+        if (!mbar_wait(bar(K_FULL + s), (i / kStages) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
+        const uint64_t kd = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint64_t koff = (uint64_t)((kk >> 2) * (kHalfBytes >> 4) + (kk & 3) * 2);
+          umma_bf16_ts(d, tmem + 448u + kk * 8, kd + koff, idesc_qk, kk > 0);
+        }
+        umma_commit(bar(K_EMPTY + s));
+        umma_commit(bar(S_FULL + (i & 1)));
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      if (ok && n_tiles > 1) ok = issue_qk(1);
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int s = i % kStages;
+        if (!mbar_wait(bar(V_FULL + s), (i / kStages) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint64_t vd = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)      // columns beyond the tile's end carry zero weights
+          umma_bf16_ts(tmem + 320u, tmem + 256u + kk * 8, vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bar(V_EMPTY + s));
+        umma_commit(bar(P_EMPTY));
+        if (i + 2 < n_tiles) ok = issue_qk(i + 2);
+      }
+      if (ok) umma_commit(bar(O_DONE));
+    }
+  } else {
+    // =========================== softmax (warps 0-7) =======================================
+    const int hh = warp >> 2, wq = warp & 3;
+    const int row = wq * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+    const uint32_t FULL = 0xffffffffu;
+    const uint32_t p_addr = tmem + lane_addr + 256u + (uint32_t)hh * 32u;
+    const uint32_t o_addr = tmem + lane_addr + 320u + (uint32_t)hh * 64u;
+    const float sc = prm.scale_log2;
+    const int my_pos = row < nrows ? rpos[row] : -1;
+    // this thread's half (64 of 128 dimensions) of its query row goes to tensor memory, two bf16 per column
+    {
+      uint32_t qw[32];
+      if (my_pos >= 0) {
+        const uint4* qp = reinterpret_cast<const uint4*>(prm.Qg + ((i64)bh * prm.N + my_pos) * kD + hh * 64);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 u = qp[c];
+          qw[4 * c] = u.x; qw[4 * c + 1] = u.y; qw[4 * c + 2] = u.z; qw[4 * c + 3] = u.w;
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) qw[c] = 0u;
+      }
+      tmem_st32u(tmem + lane_addr + 448u + (uint32_t)hh * 32u, qw);
+      tc_fence_before();
+      mbar_arrive(bar(Q_FULL));
+    }
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    int pos = 0, i = 0;
+    for (; pos < p_end; ++i) {
+      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
+                                mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
+      const Meta mt = meta[i & 7];
+      if (ok) {
+        pos += mt.ncols;
+      } else {                                                  // warp-uniform: walk on without work, keep the pair barrier in step
+        int g2 = 0;
+        pos += next_tile(pos, g2, nullptr);
+      }
+      float s[64];
+      float mx = -INFINITY;
+      unsigned keep[2] = {0u, 0u};                               // columns (of this half) that are inside the tile and routed for this row
+      if (ok) {
+        tc_fence_after();
+        int beg = 0;
+        for (int r = 0; r < mt.nruns; ++r) {
+          const int g = mt.grp[r], e = mt.end[r] + 1;
+          const bool on = (bitmap[(g >> 5) * 128 + row] >> (g & 31)) & 1u;
+          if (on) {
+#pragma unroll
+            for (int w = 0; w < 2; ++w) {
+              const int lo = max(beg - 32 * (2 * hh + w), 0), hi = min(e - 32 * (2 * hh + w), 32);
+              if (hi > lo) keep[w] |= (hi - lo == 32 ? 0xFFFFFFFFu : ((1u << (hi - lo)) - 1u) << lo);
+            }
+          }
+          beg = e;
+        }
+        const uint32_t s_addr = tmem + lane_addr + (uint32_t)(i & 1) * 128u + (uint32_t)hh * 64u;
+        tmem_ld32_nowait(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
+        tmem_ld32_nowait(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          s[c] = ((keep[c >> 5] >> (c & 31)) & 1u) ? s[c] : -INFINITY;
+          mx = fmaxf(mx, s[c]);
+        }
+      }
+      // the two halves of the row exchange their maxima (buffer of this tile's parity; executed whatever happened)
+      float* xm = xmax + (i & 1) * 256;
+      xm[hh * 128 + row] = mx;
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+      mx = fmaxf(mx, xm[(hh ^ 1) * 128 + row]);
+      const bool move = mx > -INFINITY && (mx - m_ref) * sc > 8.f;     // a row without any routed key so far keeps -inf
+      const float m_new = move ? mx : m_ref;
+      const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f;      // 0 when the reference was -inf
+      const float mneg = m_new > -INFINITY ? -m_new * sc : 0.f;
+      m_ref = m_new;
+      if (i > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
+      if (!ok) continue;
+      tc_fence_after();
+      if (i > 0 && __any_sync(FULL, move)) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float t[32];
+          tmem_ld32(o_addr + q * 32, t);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) t[c] *= corr;
+          tmem_st32(o_addr + q * 32, t);
+        }
+      }
+      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < 64; c += 4) {
+        s[c] = ex2(fmaf(s[c], sc, mneg)); s[c + 1] = ex2(fmaf(s[c + 1], sc, mneg));      // masked columns: exp2(-inf) = 0
+        s[c + 2] = ex2(fmaf(s[c + 2], sc, mneg)); s[c + 3] = ex2(fmaf(s[c + 3], sc, mneg));
+        ps4[0] += s[c]; ps4[1] += s[c + 1]; ps4[2] += s[c + 2]; ps4[3] += s[c + 3];
+      }
+      l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+      {
+        uint32_t w[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) w[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
+        tmem_st32u(p_addr, w);
+      }
+      tc_fence_before();
+      mbar_arrive(bar(P_FULL));
+    }
+    // ---- row sums of the two halves, normalise, store ------------------------------------------
+    ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
+    xsum[hh * 128 + row] = l;
+    asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+    const float ltot = l + xsum[(hh ^ 1) * 128 + row];
+    const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
+    if (ok) {
+      tc_fence_after();
+      float o[64];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        float t[32];
+        tmem_ld32(o_addr + q * 32, t);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
+      }
+      if (my_pos >= 0) {
+        const int dst = prm.q_perm[(i64)bh * prm.N + my_pos];
+        const int b = bh / prm.H, h = bh % prm.H;
+        __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + hh * 64;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
+          store8(op + ch * 8, v8);
+        }
+        if (prm.O_sparse) {
+          float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            float v8[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
+            store8(sp + ch * 8, v8);
+          }
+        }
+      }
+    }
+  }
+  // ---- teardown ----------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int k = 0; k < 64; ++k) __nanosleep(1000);
+    if (tid == 0) set_error(prm.err, SPARSEPR_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// The rows of the short remainders of one head, in group order: rem_pos = group-major position,
+// rem_grp = query group; rem_cnt = their number.  One CTA per head.
+__global__ void __launch_bounds__(1024) k_remainder_rows(const int* __restrict__ q_off, int Cq, int N, int rem_rows,
+                                                         int* __restrict__ rem_pos, int* __restrict__ rem_grp,
+                                                         int* __restrict__ rem_cnt) {
+  __shared__ int cnt[kMaxGroups];
+  __shared__ int scratch[34];
+  const int bh = blockIdx.x;
+  const int* qo = q_off + (i64)bh * (Cq + 1);
+  for (int a = threadIdx.x; a < Cq; a += blockDim.x) {
+    const int rem = (qo[a + 1] - qo[a]) % 128;
+    cnt[a] = (rem > 0 && rem <= rem_rows) ? rem : 0;
+  }
+  __syncthreads();
+  const int total = block_exclusive_scan(cnt, Cq, scratch);
+  __syncthreads();
+  for (int a = threadIdx.x >> 5; a < Cq; a += blockDim.x >> 5) {
+    const int rem = (qo[a + 1] - qo[a]) % 128;
+    if (rem > 0 && rem <= rem_rows)
+      for (int j = threadIdx.x & 31; j < rem; j += 32) {
+        rem_pos[(i64)bh * N + cnt[a] + j] = qo[a + 1] - rem + j;
+        rem_grp[(i64)bh * N + cnt[a] + j] = a;
+      }
+  }
+  if (threadIdx.x == 0) rem_cnt[bh] = total;
+}
+
+}  // namespace packed
+}  // namespace tc
+
+cudaError_t init_attention_packed() {
+  return cudaFuncSetAttribute(tc::packed::k_attention_packed, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::packed::Smem::total);
+}
+
+void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st) {
+  tc::packed::k_remainder_rows<<<BH, 1024, 0, st>>>(q_off, Cq, N, kRemRows, rem_pos, rem_grp, rem_cnt);
+}
+
+// Short remainders of every query group, packed (the 128-row kernel must have been given tile offsets that leave
+// them out).  Q, K, V group-major [BH][N][128] bf16; rem_* from launch_remainder_rows.
+bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st) {
+  using namespace tc;
+  using namespace tc::packed;
+  CUtensorMap mk, mv;
+  if (!make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) || !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile))
+    return false;
+  Params p{};
+  p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.scale_log2 = a.scale * 1.4426950408889634f;
+  p.rem_pos = rem_pos; p.rem_grp = rem_grp; p.rem_cnt = rem_cnt;
+  p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;
+  p.Qg = (const __nv_bfloat16*)a.Q;
+  p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
+  p.O_sparse = a.O_sparse; p.err = a.err;
+  // a group contributes at most kRemRows of every 128 rows it has beyond a multiple of 128, so the packed rows of a
+  // head never exceed N; CTAs past the head's count return at once
+  const int tiles = (a.N + kTile - 1) / kTile;
+  k_attention_packed<<<dim3(tiles, a.BH), kThreads, Smem::total, st>>>(mk, mv, p);
+  return true;
+}
+
+}  // namespace spr

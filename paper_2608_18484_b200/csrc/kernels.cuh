@@ -98,6 +98,11 @@ bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 constexpr int kRemRows = 64;
 cudaError_t init_attention_rem();
 bool launch_attention_rem(const AttnArgs& a, cudaStream_t st);
+// attention_packed.cu: the same remainders, packed across groups into 128-row tiles that walk over all keys with
+// per-row route masks.  rem_pos / rem_grp [BH][N], rem_cnt [BH] are built from the query offsets once per plan.
+cudaError_t init_attention_packed();
+void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st);
+bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st);
 // correction_tc.cu: O <- O + O A + c in place (bf16, d_v = 128); At: bf16 scratch [BH][128][128]
 cudaError_t init_correction_tc();
 bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
