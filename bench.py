@@ -94,10 +94,10 @@ def launches_per_call(T, fitted, tensor_path):
         kmeans = 2 + 1 + 3 * T + (T - 1)
     else:                # init, first norms, T assignments, T-1 updates
         kmeans = 2 + T + (T - 1)
-    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 2      # per side: Gram+eig, projection, k-means, sort+means; probes; route; tile offsets
+    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 3      # per side: Gram+eig, projection, k-means, sort+means; probes; route; tile offsets + remainder rows
     if not fitted:
         plan -= 2
-    attend = 3 + 1 + (4 if tensor_path else 0)       # gathers, attention (+ the four remainder-kernel launches)
+    attend = 3 + 1 + (1 if tensor_path else 0)       # gathers, attention (+ the packed-remainder kernel)
     if fitted:
         attend += (3 if tensor_path else 2) + 5 + 1  # probe rows (+gather) + merge, fit, probe write
         attend += 2 if tensor_path else 0            # transposed correction matrix, correction pass
@@ -304,7 +304,7 @@ def main():
     tensor_path = wl.dtype == "bf16" and wl.d == 128
     if tensor_path:
         # tcgen05 kernel timed inside a long step: the sustained bf16 GEMM peak is the denominator
-        roofline = {"kernel": "k_attention_tc + k_attention_rem (block-sparse, tcgen05)", "bound": "tensor", "achieved": achieved,
+        roofline = {"kernel": "k_attention_tc + k_attention_packed (block-sparse, tcgen05)", "bound": "tensor", "achieved": achieved,
                     "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"],
                     # DRAM read + write of one k_attention_tc launch: 29.6 MB per head from the ncu capture summarised
                     # in profiles/k_attention_tc_480p-like_6heads.md (177.8 MB at 6 heads of this N; heads are

@@ -90,7 +90,6 @@ cudaError_t ensure_init() {
     if ((e = init_attention_simt()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_correction_tc()) != cudaSuccess) { g_init_err = e; return; }
-    if ((e = init_attention_rem()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_attention_packed()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_project_tc()) != cudaSuccess) { g_init_err = e; return; }
     if ((e = init_kmeans_tc()) != cudaSuccess) { g_init_err = e; return; }
@@ -540,9 +539,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   if (tensor) {
     aa.tile_off = p->tile_off128;
     if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
-    if (std::getenv("SPARSEPR_REM_TRANSPOSED") ? !launch_attention_rem(aa, st)
-                                               : !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, st))
-      return SPARSEPR_ERR_CUDA;
+    if (!launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, st)) return SPARSEPR_ERR_CUDA;
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) join_side(p, st);
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
@@ -641,18 +638,21 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     const int qtile = tcpath ? 128 : 64, ktile = tcpath ? 128 : 64, box = tcpath ? 16 : 1;
     const int* rpp = &rp[(size_t)bh * (r.Cq + 1)];
     const int* rii = &ri[(size_t)bh * r.Cq * r.Ck];
+    i64 packed_rows = 0;
     for (int a = 0; a < r.Cq; ++a) {
       i64 keys = 0;
       for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += (k[rii[t] + 1] - k[rii[t]] + box - 1) / box * box;
       const i64 kt = (keys + ktile - 1) / ktile;
       const int nrow = q[a + 1] - q[a], rem = nrow % qtile;
       if (tcpath && rem > 0 && rem <= kRemRows) {
-        // full tiles by the 128-row kernel, the short remainder (rounded to 16 rows) by the remainder kernel
-        out->padded_tile_pairs += ((i64)(nrow / qtile) * qtile + (rem + 15) / 16 * 16) * kt * ktile;
+        // full tiles by the 128-row kernel; the short remainder joins the packed tiles that walk over all keys
+        out->padded_tile_pairs += (i64)(nrow / qtile) * qtile * kt * ktile;
+        packed_rows += rem;
       } else {
         out->padded_tile_pairs += (i64)((nrow + qtile - 1) / qtile) * qtile * kt * ktile;
       }
     }
+    out->padded_tile_pairs += (packed_rows + qtile - 1) / qtile * qtile * (i64)((r.N + ktile - 1) / ktile) * ktile;
   }
   out->rho_exec = out->rho_route + (double)r.M / (double)r.N;
   out->assign_rechecked_rows = errw[1];

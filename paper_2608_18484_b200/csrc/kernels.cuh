@@ -93,12 +93,10 @@ cudaError_t init_attention_tc();
 bool attention_tc_supported(const AttnArgs& a);
 // tile_off in `a` must have been built for 128-row tiles; a.A and a.c are ignored (no correction epilogue)
 bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
-// attention_rem.cu: the remainders of 1..64 rows per query group that the 128-row kernel leaves out when its tile
-// offsets were built with small_rem = kRemRows
+// Query-group remainders of 1..kRemRows rows are left out of the 128-row kernel's tiles (tile offsets built with
+// small_rem = kRemRows) and handled by attention_packed.cu
 constexpr int kRemRows = 64;
-cudaError_t init_attention_rem();
-bool launch_attention_rem(const AttnArgs& a, cudaStream_t st);
-// attention_packed.cu: the same remainders, packed across groups into 128-row tiles that walk over all keys with
+// attention_packed.cu: those remainders, packed across groups into 128-row tiles that walk over all keys with
 // per-row route masks.  rem_pos / rem_grp [BH][N], rem_cnt [BH] are built from the query offsets once per plan.
 cudaError_t init_attention_packed();
 void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st);
