@@ -143,10 +143,15 @@ struct sparsepr_plan_s {
   // probe rows and fit next to the block-sparse kernel), forked and joined with the two events
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // third stream: the packed-remainder kernel (few long CTAs) beside the 128-row kernel (many short ones)
+  cudaStream_t side2 = nullptr;
+  cudaEvent_t ev_join2 = nullptr;
   ~sparsepr_plan_s() {
     if (ev_fork) cudaEventDestroy(ev_fork);
     if (ev_join) cudaEventDestroy(ev_join);
+    if (ev_join2) cudaEventDestroy(ev_join2);
     if (side) cudaStreamDestroy(side);
+    if (side2) cudaStreamDestroy(side2);
   }
   // device state (all inside the caller's plan workspace)
   int* err; int* recheck;
@@ -342,6 +347,8 @@ static sparsepr_status_t make_plan(const sparsepr_shape_t* shape, const sparsepr
   int prio_lo = 0, prio_hi = 0;
   cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
   if (cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+      cudaStreamCreateWithPriority(&p->side2, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+      cudaEventCreateWithFlags(&p->ev_join2, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) != cudaSuccess) {
     delete p;
@@ -538,8 +545,21 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   }
   if (tensor) {
     aa.tile_off = p->tile_off128;
+    // the packed remainder tiles are few and long, the 128-row tiles many and short: without a profile they share
+    // the GPU instead of running one after the other
+    cudaStream_t rs = st;
+    if (prof == nullptr) {
+      if (!overlap) cudaEventRecord(p->ev_fork, st);              // (with the probes' overlap the event is recorded already)
+      cudaStreamWaitEvent(p->side2, p->ev_fork, 0);
+      rs = p->side2;
+    }
+    if (prof == nullptr && !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, rs)) return SPARSEPR_ERR_CUDA;
     if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
-    if (!launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, st)) return SPARSEPR_ERR_CUDA;
+    if (prof != nullptr && !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, rs)) return SPARSEPR_ERR_CUDA;
+    if (prof == nullptr) {
+      cudaEventRecord(p->ev_join2, p->side2);
+      cudaStreamWaitEvent(st, p->ev_join2, 0);
+    }
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) join_side(p, st);
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
