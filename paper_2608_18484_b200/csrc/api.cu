@@ -658,7 +658,15 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     const int qtile = tcpath ? 128 : 64, ktile = tcpath ? 128 : 64, box = tcpath ? 16 : 1;
     const int* rpp = &rp[(size_t)bh * (r.Cq + 1)];
     const int* rii = &ri[(size_t)bh * r.Cq * r.Ck];
-    i64 packed_rows = 0;
+    // packed tiles: 128 remainder rows in group order; each streams the union of the K/V groups its rows route to
+    std::vector<char> want(r.Ck, 0);
+    int packed_fill = 0;
+    auto flush_packed = [&]() {
+      i64 boxes = 0;
+      for (int g = 0; g < r.Ck; ++g) if (want[g]) { boxes += (k[g + 1] - k[g] + box - 1) / box; want[g] = 0; }
+      out->padded_tile_pairs += (i64)qtile * ((boxes * box + ktile - 1) / ktile) * ktile;
+      packed_fill = 0;
+    };
     for (int a = 0; a < r.Cq; ++a) {
       i64 keys = 0;
       for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += (k[rii[t] + 1] - k[rii[t]] + box - 1) / box * box;
@@ -667,12 +675,17 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
       if (tcpath && rem > 0 && rem <= kRemRows) {
         // full tiles by the 128-row kernel; the short remainder joins the packed tiles that walk over all keys
         out->padded_tile_pairs += (i64)(nrow / qtile) * qtile * kt * ktile;
-        packed_rows += rem;
+        for (int left = rem; left > 0;) {
+          const int take = std::min(left, qtile - packed_fill);
+          for (int t = rpp[a]; t < rpp[a + 1]; ++t) want[rii[t]] = 1;
+          packed_fill += take; left -= take;
+          if (packed_fill == qtile) flush_packed();
+        }
       } else {
         out->padded_tile_pairs += (i64)((nrow + qtile - 1) / qtile) * qtile * kt * ktile;
       }
     }
-    out->padded_tile_pairs += (packed_rows + qtile - 1) / qtile * qtile * (i64)((r.N + ktile - 1) / ktile) * ktile;
+    if (packed_fill > 0) flush_packed();
   }
   out->rho_exec = out->rho_route + (double)r.M / (double)r.N;
   out->assign_rechecked_rows = errw[1];

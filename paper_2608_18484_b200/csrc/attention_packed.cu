@@ -3,16 +3,17 @@
 // A query group of n rows gives floor(n / 128) full tiles to the 128-row kernel; when the n mod 128 rows
 // that are left are at most kRemRows they come here.  An M = 128 tensor-core tile for a handful of rows
 // costs as much as a full one, and rows of different groups attend to different keys, so the
-// remainders of MANY groups are packed into common 128-row tiles instead: such a tile walks over ALL
-// keys of the head (group-major order) and every row masks the K/V groups that its own query group
-// does not route to.  At a routed density of 25 % and 16-row remainders that is about a third of the
+// remainders of MANY groups are packed into common 128-row tiles instead: such a tile walks over the keys of
+// every K/V group that any of its rows routes to (group-major order) and every row masks the groups that its
+// own query group does not route to.  At a routed density of 25 % and 16-row remainders that is about a third of the
 // tile passes that one tile per remainder needs.
 //
 //   warps 0-7  softmax: warps w and w+4 share the 32 rows of TMEM quadrant w and split the 128 scores
 //              of a row in two halves; they also bring the query rows into tensor memory (the rows of a
 //              packed tile are scattered, so there is no TMA box for them)
-//   warp  8    K producer; cuts the key sequence into tiles that span at most 8 K/V groups and publishes
-//              the group runs of every tile;  warp 10  V producer
+//   warp  8    K producer: streams the K/V groups that some row of the tile routes to, as one sequence of 16-row
+//              boxes (tiles of 128 keys, every box inside one group), and publishes the group of every box;
+//   warp  10   V producer
 //   warp  9    tcgen05.mma issuer; owns the TMEM allocation
 // TMEM: S_0 [0,128), S_1 [128,256), P [256,320), O [320,448), Q [448,512); both products take their A
 // operand from tensor memory.  Reference maxima move lazily (growth beyond 2^8), as in the 128-row kernel.
@@ -28,23 +29,31 @@ namespace packed {
 constexpr int kThreads = 352;
 constexpr int kTile = 128;
 constexpr int kD = 128;
+constexpr int kSub = 16;                               // rows per TMA box of the K/V stream
+constexpr int kSubPerTile = kTile / kSub;
 constexpr uint32_t kHalfBytes = kTile * 128;          // [128 rows x 64 bf16]
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
+constexpr uint32_t kSubBytes = kSub * 128;
 constexpr int kStages = 2;
-constexpr int kMaxRuns = 8;                            // K/V-group runs per key tile
 
-struct Meta { int ncols, nruns; unsigned short grp[kMaxRuns]; unsigned char end[kMaxRuns]; };   // 32 bytes
+// per key tile: number of boxes, valid rows of every box (4 bits each, minus one), K/V group of every box
+struct Meta { uint32_t cnt_bits, nsub; unsigned short grp[kSubPerTile]; uint32_t pad[2]; };   // 32 bytes
 
 struct Smem {
   static constexpr uint32_t k = 0;
   static constexpr uint32_t v = k + kStages * kTileBytes;
   static constexpr uint32_t bitmap = v + kStages * kTileBytes;           // [kMaxGroups/32 words][128 rows]
-  static constexpr uint32_t xchg = bitmap + (kMaxGroups / 32) * 128 * 4; // float [2][2][128] half-row maxima, [2][128] half-row sums
+  static constexpr uint32_t uni = bitmap + (kMaxGroups / 32) * 128 * 4;  // [kMaxGroups/32] union of the rows' route bitmaps
+  static constexpr uint32_t ranges = uni + (kMaxGroups / 32) * 4;        // int2[kMaxGroups] (start, length) of the wanted K/V groups
+  static constexpr uint32_t gid = ranges + kMaxGroups * 8;               // unsigned short[kMaxGroups] their group ids
+  static constexpr uint32_t idx = gid + kMaxGroups * 2;                  // int[kMaxGroups] scan scratch
+  static constexpr uint32_t xchg = idx + kMaxGroups * 4;                 // float [2][2][128] half-row maxima, [2][128] half-row sums
   static constexpr uint32_t meta = xchg + 6 * 128 * 4;                   // Meta[8]
   static constexpr uint32_t bars = meta + 8 * 32;
   static constexpr uint32_t misc = bars + 32 * 8;
-  static constexpr uint32_t total = misc + 64;
+  static constexpr uint32_t total = misc + 256;
 };
+static_assert(Smem::total <= 227 * 1024, "shared memory");
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kStages, V_FULL = K_EMPTY + kStages, V_EMPTY = V_FULL + kStages,
            S_FULL = V_EMPTY + kStages, P_FULL = S_FULL + 2, P_EMPTY, O_DONE, META_FULL, kNumBars = META_FULL + 8 };
 static_assert(kNumBars <= 32, "barrier area");
@@ -66,10 +75,14 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
   unsigned* bitmap = reinterpret_cast<unsigned*>(sm + Smem::bitmap);
+  unsigned* uni = reinterpret_cast<unsigned*>(sm + Smem::uni);
+  int2* ranges = reinterpret_cast<int2*>(sm + Smem::ranges);
+  unsigned short* gid = reinterpret_cast<unsigned short*>(sm + Smem::gid);
+  int* idx = reinterpret_cast<int*>(sm + Smem::idx);
   float* xmax = reinterpret_cast<float*>(sm + Smem::xchg);
   float* xsum = xmax + 4 * 128;
   Meta* meta = reinterpret_cast<Meta*>(sm + Smem::meta);
-  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem, [1] abort, [3] skip
+  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem, [1] abort, [2] boxes, [3] skip, [8..41] scan scratch
   const uint32_t bars = base + Smem::bars;
   auto bar = [&](int i) { return bars + 8u * i; };
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -86,10 +99,11 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
   const int words = (prm.Ck + 31) / 32;
   const int* rpos = prm.rem_pos + (i64)bh * prm.N + m0;
   const int* rgrp = prm.rem_grp + (i64)bh * prm.N + m0;
+  const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
 
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == P_FULL || i == Q_FULL) ? 256 : 1);
-    misc[1] = 0;
+    misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 9) tmem_alloc(base + Smem::misc, 512);
@@ -102,50 +116,82 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const int* ri = prm.route_idx + (i64)bh * prm.Cq * prm.Ck;
     for (int t = rp[g] + (tid & 1); t < rp[g + 1]; t += 2) atomicOr(&bitmap[(ri[t] >> 5) * 128 + r], 1u << (ri[t] & 31));
   }
+  __syncthreads();
+  // the K/V groups that some row routes to, in order: they are streamed, the others are not even loaded
+  for (int w = tid; w < words; w += kThreads) {
+    unsigned u = 0u;
+    for (int r = 0; r < nrows; ++r) u |= bitmap[w * 128 + r];
+    uni[w] = u;
+  }
+  __syncthreads();
+  for (int g = tid; g < prm.Ck; g += kThreads) idx[g] = (((uni[g >> 5] >> (g & 31)) & 1u) && kvoff[g + 1] > kvoff[g]) ? 1 : 0;
+  __syncthreads();
+  const int nroute = block_exclusive_scan(idx, prm.Ck, const_cast<int*>(misc + 8));
+  __syncthreads();
+  {
+    int boxes = 0;
+    for (int g = tid; g < prm.Ck; g += kThreads) {
+      const int start = kvoff[g], len = kvoff[g + 1] - start;
+      if (((uni[g >> 5] >> (g & 31)) & 1u) && len > 0) {
+        ranges[idx[g]] = make_int2(start, len);
+        gid[idx[g]] = (unsigned short)g;
+        boxes += (len + kSub - 1) / kSub;
+      }
+    }
+    boxes = warp_sum(boxes);
+    if (lane == 0 && boxes) atomicAdd((int*)&misc[2], boxes);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = (uint32_t)misc[0];
+  const int total_boxes = misc[2];
+  const int n_tiles = (total_boxes + kSubPerTile - 1) / kSubPerTile;
   volatile int* abort_flag = &misc[1];
-  const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
-  const int p_end = prm.N;
-
-  // Tiles are cut so that none spans more than kMaxRuns K/V groups; every role that walks the key sequence
-  // uses this function.  `g` = group that contains `pos`.
-  auto next_tile = [&](int pos, int& g, Meta* out) -> int {
-    int runs = 0, c = 0;
-    while (c < kTile && pos + c < p_end && runs < kMaxRuns) {
-      while (kvoff[g + 1] <= pos + c) ++g;                        // skip empty groups
-      const int e = min(min(kvoff[g + 1], p_end) - pos, kTile);
-      if (out) { out->grp[runs] = (unsigned short)g; out->end[runs] = (unsigned char)(e - 1); }
-      c = e;
-      ++runs;
-    }
-    if (out) { out->ncols = c; out->nruns = runs; }
-    return c;
-  };
 
   if (warp == 8 || warp == 10) {
-    // =========================== producers ==================================================
-    if (lane == 0) {
+    // =========================== TMA producers ==========================================
+    // All lanes of a producer walk the wanted key ranges together (uniform); lane j issues the copies of box j.
+    if (n_tiles > 0) {
       const bool is_k = warp == 8;
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
       const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
       const CUtensorMap* map = is_k ? &mapK : &mapV;
-      int g = 0, pos = 0;
-      for (int i = 0; pos < p_end; ++i) {
+      int ri = 0, off = 0;
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kStages;
-        Meta mt;
-        const int nc = next_tile(pos, g, &mt);
-        if (!mbar_wait(bar(empty0 + s), ((i / kStages) & 1) ^ 1, abort_flag)) break;
-        if (is_k) {
-          meta[i & 7] = mt;
-          mbar_arrive(bar(META_FULL + (i & 7)));
+        const uint32_t ph = ((i / kStages) & 1) ^ 1;         // empty barriers: the first pass completes immediately
+        int my_start = 0, my_gid = 0;
+        uint32_t cnt_bits = 0;
+        int nsub = 0;
+#pragma unroll
+        for (int j = 0; j < kSubPerTile; ++j) {
+          if (ri < nroute) {
+            const int2 rg = ranges[ri];
+            if (j == lane) { my_start = rg.x + off; my_gid = gid[ri]; }
+            const int c = min(kSub, rg.y - off);
+            cnt_bits |= (uint32_t)(c - 1) << (4 * j);
+            nsub = j + 1;
+            off += kSub;
+            if (off >= rg.y) { ++ri; off = 0; }
+          }
         }
-        mbar_expect_tx(bar(full0 + s), kTileBytes);
-        tma_load_4d(buf0 + s * kTileBytes, map, bar(full0 + s), 0, pos, bh, 0);
-        tma_load_4d(buf0 + s * kTileBytes + kHalfBytes, map, bar(full0 + s), 64, pos, bh, 0);
-        pos += nc;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(empty0 + s), ph, abort_flag));
+        if (!ok) break;
+        if (is_k) {
+          if (lane < kSubPerTile) meta[i & 7].grp[lane] = (unsigned short)my_gid;
+          if (lane == 0) { meta[i & 7].cnt_bits = cnt_bits; meta[i & 7].nsub = (uint32_t)nsub; }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(META_FULL + (i & 7)));
+        }
+        if (lane == 0) mbar_expect_tx(bar(full0 + s), nsub * 2 * kSubBytes);
+        __syncwarp();
+        if (lane < nsub) {
+          const uint32_t dst = buf0 + s * kTileBytes + lane * kSubBytes;
+          tma_load_4d(dst, map, bar(full0 + s), 0, my_start, bh, 0);
+          tma_load_4d(dst + kHalfBytes, map, bar(full0 + s), 64, my_start, bh, 0);
+        }
       }
     }
   } else if (warp == 9) {
@@ -154,8 +200,6 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
       const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
       const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
       const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
-      int n_tiles = 0;
-      { int g = 0; for (int pos = 0; pos < p_end; ++n_tiles) pos += next_tile(pos, g, nullptr); }
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
       auto issue_qk = [&](int i) -> bool {
         const int s = i % kStages;
@@ -172,22 +216,25 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         umma_commit(bar(S_FULL + (i & 1)));
         return true;
       };
-      if (ok) ok = issue_qk(0);
+      if (ok && n_tiles > 0) ok = issue_qk(0);
       if (ok && n_tiles > 1) ok = issue_qk(1);
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kStages;
+        if (!mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag)) { ok = false; break; }
+        const int nsub = (int)meta[i & 7].nsub;
         if (!mbar_wait(bar(V_FULL + s), (i / kStages) & 1, abort_flag)) { ok = false; break; }
         if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint64_t vd = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)      // columns beyond the tile's end carry zero weights
-          umma_bf16_ts(tmem + 320u, tmem + 256u + kk * 8, vd + (uint64_t)(kk * (2048 >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < kSubPerTile; ++kk)
+          if (kk < nsub)
+            umma_bf16_ts(tmem + 320u, tmem + 256u + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(V_EMPTY + s));
         umma_commit(bar(P_EMPTY));
         if (i + 2 < n_tiles) ok = issue_qk(i + 2);
       }
-      if (ok) umma_commit(bar(O_DONE));
+      if (ok) umma_commit(bar(O_DONE));                        // completes at once when there was no tile
     }
   } else {
     // =========================== softmax (warps 0-7) =======================================
@@ -219,44 +266,43 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     }
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    int pos = 0, i = 0;
-    for (; pos < p_end; ++i) {
+    for (int i = 0; i < n_tiles; ++i) {
       ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
                                 mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
-      const Meta mt = meta[i & 7];
-      if (ok) {
-        pos += mt.ncols;
-      } else {                                                  // warp-uniform: walk on without work, keep the pair barrier in step
-        int g2 = 0;
-        pos += next_tile(pos, g2, nullptr);
-      }
       float s[64];
       float mx = -INFINITY;
-      unsigned keep[2] = {0u, 0u};                               // columns (of this half) that are inside the tile and routed for this row
       if (ok) {
         tc_fence_after();
-        int beg = 0;
-        for (int r = 0; r < mt.nruns; ++r) {
-          const int g = mt.grp[r], e = mt.end[r] + 1;
-          const bool on = (bitmap[(g >> 5) * 128 + row] >> (g & 31)) & 1u;
-          if (on) {
-#pragma unroll
-            for (int w = 0; w < 2; ++w) {
-              const int lo = max(beg - 32 * (2 * hh + w), 0), hi = min(e - 32 * (2 * hh + w), 32);
-              if (hi > lo) keep[w] |= (hi - lo == 32 ? 0xFFFFFFFFu : ((1u << (hi - lo)) - 1u) << lo);
-            }
-          }
-          beg = e;
-        }
+        const Meta& mt = meta[i & 7];
+        const uint32_t cnt_bits = mt.cnt_bits;
+        const int nsub = (int)mt.nsub;
         const uint32_t s_addr = tmem + lane_addr + (uint32_t)(i & 1) * 128u + (uint32_t)hh * 64u;
         tmem_ld32_nowait(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
         tmem_ld32_nowait(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+        // a box counts for this row when its K/V group is routed by the row's query group; lim = its last valid column
+        int lim[4];
+#pragma unroll
+        for (int bx = 0; bx < 4; ++bx) {
+          const int box = hh * 4 + bx;
+          lim[bx] = -1;
+          if (box < nsub) {
+            const int g = mt.grp[box];
+            if ((bitmap[(g >> 5) * 128 + row] >> (g & 31)) & 1u) lim[bx] = (int)((cnt_bits >> (4 * box)) & 15u);
+          }
+        }
         tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          s[c] = ((keep[c >> 5] >> (c & 31)) & 1u) ? s[c] : -INFINITY;
-          mx = fmaxf(mx, s[c]);
+        for (int bx = 0; bx < 4; ++bx) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) s[bx * 16 + c] = (c <= lim[bx]) ? s[bx * 16 + c] : -INFINITY;
         }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int c = 0; c < 64; c += 4) {
+          mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+          mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+        }
+        mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
       // the two halves of the row exchange their maxima (buffer of this tile's parity; executed whatever happened)
       float* xm = xmax + (i & 1) * 256;
@@ -308,11 +354,15 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
       tc_fence_after();
       float o[64];
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        float t[32];
-        tmem_ld32(o_addr + q * 32, t);
+      for (int c = 0; c < 64; ++c) o[c] = 0.f;
+      if (n_tiles > 0) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
+        for (int q = 0; q < 2; ++q) {
+          float t[32];
+          tmem_ld32(o_addr + q * 32, t);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
+        }
       }
       if (my_pos >= 0) {
         const int dst = prm.q_perm[(i64)bh * prm.N + my_pos];
@@ -396,7 +446,7 @@ bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* r
   using namespace tc;
   using namespace tc::packed;
   CUtensorMap mk, mv;
-  if (!make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) || !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile))
+  if (!make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) || !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub))
     return false;
   Params p{};
   p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.scale_log2 = a.scale * 1.4426950408889634f;
