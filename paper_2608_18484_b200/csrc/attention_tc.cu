@@ -28,7 +28,7 @@ namespace spr {
 
 namespace tc {
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kTile = 128;            // query rows per CTA, keys per tile
 constexpr int kD = 128;
 constexpr int kSub = 16;              // rows per TMA box of the K/V stream
@@ -59,7 +59,7 @@ struct Smem {                          // offsets from a 1024-byte aligned base
 constexpr size_t kSmemBytes = Smem::total;                        // the dynamic segment is 1024-byte aligned and the only shared memory
 
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kKStages, V_FULL = K_EMPTY + kKStages, V_EMPTY = V_FULL + kVStages,
-           S_FULL = V_EMPTY + kVStages, P_FULL = S_FULL + 2, P_EMPTY, O_DONE, META_FULL,
+           S_FULL = V_EMPTY + kVStages, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_EMPTY = P_FULL + 2, O_DONE = P_EMPTY + 2, META_FULL,
            kNumBars = META_FULL + 8 };
 static_assert(kNumBars <= 32, "barrier area");
 
@@ -72,11 +72,13 @@ struct Params {
   int* err;
 };
 
+struct Maps { CUtensorMap m[4]; };      // the same tensor with boxes of 16, 32, 64 and 128 rows
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) { return pack_bf16x2(a, b); }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-               const __grid_constant__ CUtensorMap mapV, Params prm) {
+k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ Maps mapsK,
+               const __grid_constant__ Maps mapsV, Params prm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
@@ -125,7 +127,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i)
-      mbar_init(bar(i), i == P_FULL ? 256 : 1);
+      mbar_init(bar(i), (i == P_FULL || i == P_FULL + 1 || i == S_FREE || i == S_FREE + 1) ? 256 : 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -165,30 +167,48 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const int nst = is_k ? kKStages : kVStages;
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
       const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
-      const CUtensorMap* map = is_k ? &mapK : &mapV;
+      const Maps* maps = is_k ? &mapsK : &mapsV;
       int ri = 0, off = 0;
       bool ok = true;
+#ifdef SPR_ATTN_TIMING
+      long long pa = 0, pb = 0, pc = 0, p0;
+#define SPR_P0() p0 = clock64()
+#define SPR_PACC(v) do { const long long t1 = clock64(); v += t1 - p0; p0 = t1; } while (0)
+#else
+#define SPR_P0()
+#define SPR_PACC(v)
+#endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % nst;
         const uint32_t ph = ((i / nst) & 1) ^ 1;             // empty barriers: the first pass completes immediately
-        int my_start = 0;
+        SPR_P0();
+        // the tile takes up to 8 boxes of 16 rows; consecutive boxes of one key range form a segment, and a segment
+        // of n boxes is fetched by one copy per set bit of n (128, 64, 32 or 16 rows), largest first
+        int my_start = 0, my_t = 0, my_n = 0, nsub = 0;
         uint32_t cnt_bits = 0;
-        int nsub = 0;
-#pragma unroll
-        for (int j = 0; j < kSubPerTile; ++j) {
-          if (ri < nroute) {
-            const int2 rg = ranges[ri];
-            if (j == lane) my_start = rg.x + off;
-            const int cnt = min(kSub, rg.y - off);
-            cnt_bits |= (uint32_t)(cnt - 1) << (4 * j);
-            nsub = j + 1;
-            off += kSub;
-            if (off >= rg.y) {
-              ++ri; off = 0;
-            }
+        while (nsub < kSubPerTile && ri < nroute) {
+          const int2 rg = ranges[ri];
+          const int left = rg.y - off, nb = (left + kSub - 1) / kSub;
+          const int n = min(kSubPerTile - nsub, nb);
+          if (lane >= nsub && lane < nsub + n) { my_t = lane - nsub; my_n = n; my_start = rg.x + off + my_t * kSub; }
+          uint32_t bits = n == 8 ? 0xFFFFFFFFu : ((1u << (4 * n)) - 1u);      // valid rows of every box, minus one
+          if (n == nb) {                                                       // the range ends here: its last box may be short
+            const int sh = 4 * (n - 1);
+            bits = (bits & ~(0xFu << sh)) | ((uint32_t)(left - (n - 1) * kSub - 1) << sh);
+            ++ri; off = 0;
+          } else {
+            off += n * kSub;
           }
+          cnt_bits |= bits << (4 * nsub);
+          nsub += n;
         }
+        int my_k = -1;                                                         // log2 of the boxes this lane's copy spans
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb)
+          if (lane < nsub && ((my_n >> kb) & 1) && my_t == ((my_n >> (kb + 1)) << (kb + 1))) my_k = kb;
+        SPR_PACC(pa);
         ok = __all_sync(0xffffffffu, mbar_wait(bar(empty0 + s), ph, abort_flag));
+        SPR_PACC(pb);
         if (!ok) break;
         if (lane == 0) {
           if (is_k) {
@@ -199,27 +219,46 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           mbar_expect_tx(bar(full0 + s), nsub * 2 * kSubBytes);
         }
         __syncwarp();
-        if (lane < nsub) {
+        if (my_k >= 0) {
           const uint32_t dst = buf0 + s * kTileBytes + lane * kSubBytes;
-          tma_load_4d(dst, map, bar(full0 + s), 0, my_start, c2, c3);
-          tma_load_4d(dst + kHalfBytes, map, bar(full0 + s), 64, my_start, c2, c3);
+          tma_load_4d(dst, &maps->m[my_k], bar(full0 + s), 0, my_start, c2, c3);
+          tma_load_4d(dst + kHalfBytes, &maps->m[my_k], bar(full0 + s), 64, my_start, c2, c3);
         }
+        SPR_PACC(pc);
       }
+#ifdef SPR_ATTN_TIMING
+      if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0)
+        printf("%s producer tiles %d: walk %lld  wait empty %lld  issue %lld (cycles per tile)\n", is_k ? "K" : "V", n_tiles, pa / n_tiles, pb / n_tiles, pc / n_tiles);
+#endif
     }
   } else if (warp == 9) {
-    // =========================== MMA issuer ==============================================
-    // TMEM columns: S_0 [0,128), S_1 [128,256), P [256,320) (two bf16 per column), O [320,448)
+    // =========================== Q K^T issuer ============================================
+    // TMEM columns: S_0 [0,128), S_1 [128,256), P_0 [256,320) and P_1 [448,512) (two bf16 per column), O [320,448).
+    // The two products are issued by two threads on different warp schedulers: an issuing thread shares its
+    // scheduler with two softmax warps that rarely leave it a slot, and the score tile two steps ahead must not
+    // queue behind the P V of the current one.
     if (lane == 0 && n_tiles > 0) {
-      const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
-      // descriptors are built once; inside the loops only their address field moves (in 16-byte units),
-      // so that issuing an MMA costs a couple of integer adds in this single thread
+      const uint32_t idesc_qk = idesc_bf16(0, 128);
+      // descriptors are built once; inside the loops only their address field moves (in 16-byte units)
       const uint64_t q_desc = smem_desc(base + Smem::q, 16);
       const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
-      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
-      auto issue_qk = [&](int i) -> bool {
+#ifdef SPR_ATTN_TIMING
+      long long qa = 0, qb = 0, qc = 0, m0;
+#define SPR_M0() m0 = clock64()
+#define SPR_MACC(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
+#else
+#define SPR_M0()
+#define SPR_MACC(v)
+#endif
+      for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kKStages;
-        if (!mbar_wait(bar(K_FULL + s), (i / kKStages) & 1, abort_flag)) return false;
+        SPR_M0();
+        // score buffer i mod 2 is free once every softmax thread holds tile i - 2 in registers
+        if (i >= 2 && !mbar_wait(bar(S_FREE + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+        SPR_MACC(qa);
+        if (!mbar_wait(bar(K_FULL + s), (i / kKStages) & 1, abort_flag)) { ok = false; break; }
+        SPR_MACC(qb);
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
         const uint64_t kd = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
@@ -230,49 +269,50 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         umma_commit(bar(K_EMPTY + s));
         umma_commit(bar(S_FULL + (i & 1)));
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
-      if (ok && n_tiles > 1) ok = issue_qk(1);
+        SPR_MACC(qc);
+      }
 #ifdef SPR_ATTN_TIMING
-      long long mv = 0, mp = 0, mi = 0, mq = 0, m0;
-#define SPR_M0() m0 = clock64()
-#define SPR_MACC(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
-#else
-#define SPR_M0()
-#define SPR_MACC(v)
+      if (blockIdx.x == 7 && blockIdx.y == 0)
+        printf("mma QK thread tiles %d: wait S free %lld  wait K %lld  issue %lld (cycles per tile)\n", n_tiles, qa / n_tiles, qb / n_tiles, qc / n_tiles);
+#endif
+    }
+  } else if (warp == 11) {
+    // =========================== P V issuer ==============================================
+    if (lane == 0 && n_tiles > 0) {
+      const uint32_t idesc_pv = idesc_bf16(1, 128);
+      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
+      bool ok = true;
+#ifdef SPR_ATTN_TIMING
+      long long mv = 0, mp = 0, mi = 0, m0;
 #endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kVStages;
-        const uint2 mt = meta[i & 7];
         SPR_M0();
+        if (!mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag)) { ok = false; break; }
+        const int nsub = (int)meta[i & 7].y;
         if (!mbar_wait(bar(V_FULL + s), (i / kVStages) & 1, abort_flag)) { ok = false; break; }
         SPR_MACC(mv);
-        if (!mbar_wait(bar(P_FULL), i & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, S_(i mod 2) read, O rescaled if needed
+        if (!mbar_wait(bar(P_FULL + (i & 1)), (i >> 1) & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, O rescaled if needed
         SPR_MACC(mp);
         tc_fence_after();
         const uint32_t d = tmem + 320u;
-        const uint32_t pa = tmem + 256u;
-        const int nsub = (int)mt.y;
+        const uint32_t pa = tmem + ((i & 1) ? 448u : 256u);
         const uint64_t vd = v_desc0 + (uint64_t)(s * (kTileBytes >> 4));
 #pragma unroll
         for (int kk = 0; kk < kSubPerTile; ++kk)
           if (kk < nsub)
             umma_bf16_ts(d, pa + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(V_EMPTY + s));
-        umma_commit(bar(P_EMPTY));
+        umma_commit(bar(P_EMPTY + (i & 1)));
         SPR_MACC(mi);
-        if (i + 2 < n_tiles) ok = issue_qk(i + 2);          // score buffer i mod 2 is free again
-        SPR_MACC(mq);
       }
 #ifdef SPR_ATTN_TIMING
       if (blockIdx.x == 7 && blockIdx.y == 0)
-        printf("mma thread tiles %d: wait V %lld  wait P %lld  issue PV %lld  wait K + issue QK %lld (cycles per tile)\n", n_tiles,
-               mv / n_tiles, mp / n_tiles, mi / n_tiles, mq / n_tiles);
+        printf("mma PV thread tiles %d: wait V %lld  wait P %lld  issue %lld (cycles per tile)\n", n_tiles, mv / n_tiles, mp / n_tiles, mi / n_tiles);
 #endif
       if (ok) umma_commit(bar(O_DONE));
     }
-  } else {
+  } else if (warp < 8) {
     // =========================== softmax (warps 0-7) =======================================
     // Thread (half hh, quadrant wq, lane) owns the 64 scores of keys [64 hh, 64 hh + 64) of query row
     // 32 wq + lane; warps wq and wq + 4 meet at the named barrier 1 + wq to agree on the row maximum.
@@ -280,13 +320,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const int row = wq * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t FULL = 0xffffffffu;
-    const uint32_t p_addr = tmem + lane_addr + 256u + (uint32_t)hh * 32u;
+    const uint32_t p_addr0 = tmem + lane_addr + 256u + (uint32_t)hh * 32u;      // P of even tiles; odd tiles 192 columns on
     const uint32_t o_addr = tmem + lane_addr + 320u + (uint32_t)hh * 64u;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
 #ifdef SPR_ATTN_TIMING
-    long long tw = 0, tl = 0, tm = 0, ts = 0, t0;
+    long long tw = 0, tl = 0, tm = 0, ts = 0, tx = 0, tp = 0, tmx = 0, t0;
 #define SPR_T0() t0 = clock64()
 #define SPR_ACC(v) do { const long long t1 = clock64(); v += t1 - t0; t0 = t1; } while (0)
 #else
@@ -295,8 +335,17 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #endif
     for (int i = 0; i < n_tiles; ++i) {
       SPR_T0();
-      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
-                                mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
+      // the three barriers of this tile are polled back to back (their shared-memory round trips overlap); the P
+      // buffer of this parity was consumed by the product two tiles back and is normally free long before
+      const bool t_meta = mbar_try(bar(META_FULL + (i & 7)), (i >> 3) & 1);
+      const bool t_s = mbar_try(bar(S_FULL + (i & 1)), (i >> 1) & 1);
+      const bool t_pe = i > 1 ? mbar_try(bar(P_EMPTY + (i & 1)), ((i - 2) >> 1) & 1) : true;
+      {
+        bool w = ok;
+        if (!t_meta) w = w && mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag);
+        if (!t_s) w = w && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag);
+        ok = __all_sync(FULL, w);
+      }
       float s[64];
       float mx = -INFINITY;
       if (ok) {
@@ -307,6 +356,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tmem_ld32_nowait(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
         SPR_ACC(tw);
         tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(bar(S_FREE + (i & 1)));                         // the scores are in registers
         SPR_ACC(tl);
         if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
           // only the boxes that end a key range (or lie beyond the stream) have columns to mask; the test is uniform
@@ -330,19 +381,28 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       // the two halves of the row exchange their maxima (buffer of this tile's parity; executed whatever happened)
       float* xm = xmax + (i & 1) * 256;
+      SPR_ACC(tmx);
       xm[hh * 128 + row] = mx;
       asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
       mx = fmaxf(mx, xm[(hh ^ 1) * 128 + row]);
+      SPR_ACC(tx);
       const bool move = (mx - m_ref) * sc > 8.f;                 // true on the first tile (m_ref = -inf); same in both halves
       const float m_new = move ? mx : m_ref;
       const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f; // 0 on the first tile
       const float mneg = -m_new * sc;
       m_ref = m_new;
-      // P and O of the previous tile must have been consumed before they are touched
-      if (i > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
+      // the P buffer of this parity must have been consumed by the product two tiles back
+      if (!__all_sync(FULL, t_pe)) {
+        ok = __all_sync(FULL, ok && (t_pe || mbar_wait(bar(P_EMPTY + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)));
+        tc_fence_after();
+      }
+      SPR_ACC(tp);
       if (!ok) continue;                                         // warp-uniform; the pair barrier above has been passed
-      tc_fence_after();
       if (i > 0 && __any_sync(FULL, move)) {                     // rescale this half of the warp's O rows (rare)
+        // O must be at rest: the product of the previous tile has to be complete as well
+        ok = __all_sync(FULL, mbar_wait(bar(P_EMPTY + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abort_flag));
+        if (!ok) continue;
+        tc_fence_after();
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
           float t[32];
@@ -366,16 +426,16 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[2 * c], s[2 * c + 1]);
         SPR_ACC(tm);
-        tmem_st32u(p_addr, w);
+        tmem_st32u(p_addr0 + (uint32_t)(i & 1) * 192u, w);
       }
       tc_fence_before();
-      mbar_arrive(bar(P_FULL));
+      mbar_arrive(bar(P_FULL + (i & 1)));
       SPR_ACC(ts);
     }
 #ifdef SPR_ATTN_TIMING
     if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 4))
-      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  math %lld  pack+st %lld (cycles per tile)\n", warp, n_tiles,
-             tw / max(1, n_tiles), tl / max(1, n_tiles), tm / max(1, n_tiles), ts / max(1, n_tiles));
+      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  mask+max %lld  exchange %lld  wait P empty %lld  exp+pack %lld  st+arrive %lld (cycles per tile)\n", warp, n_tiles,
+             tw / max(1, n_tiles), tl / max(1, n_tiles), tmx / max(1, n_tiles), tx / max(1, n_tiles), tp / max(1, n_tiles), tm / max(1, n_tiles), ts / max(1, n_tiles));
 #endif
     // ---- row sums of the two halves, normalise, store ------------------------------------------
     if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
@@ -480,16 +540,21 @@ bool attention_tc_supported(const AttnArgs& a) {
 
 bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   using namespace tc;
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq;
+  Maps mk, mv;
   const bool sparse = a.route_ptr != nullptr;
   const int B = a.BH / a.H;
   bool ok;
   if (sparse) {
-    ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) && make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) &&
-         make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub);
+    ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile);
+    for (int k = 0; k < 4 && ok; ++k)
+      ok = make_map(&mk.m[k], a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k) &&
+           make_map(&mv.m[k], a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k);
   } else {
-    ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile) && make_map(&mk, a.K, kD, a.N, a.H, B, a.ks[0], a.ks[1], a.ks[2], kSub) &&
-         make_map(&mv, a.V, kD, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub);
+    ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile);
+    for (int k = 0; k < 4 && ok; ++k)
+      ok = make_map(&mk.m[k], a.K, kD, a.N, a.H, B, a.ks[0], a.ks[1], a.ks[2], kSub << k) &&
+           make_map(&mv.m[k], a.V, kD, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub << k);
   }
   if (!ok) return false;
   Params p{};
