@@ -26,7 +26,8 @@ namespace spr {
 namespace tc {
 namespace packed {
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
+constexpr int kPolyOf8 = 3;                           // pairs of every 8 whose exponential is a polynomial on the FMA pipe
 constexpr int kTile = 128;
 constexpr int kD = 128;
 constexpr int kSub = 16;                               // rows per TMA box of the K/V stream
@@ -55,8 +56,10 @@ struct Smem {
 };
 static_assert(Smem::total <= 227 * 1024, "shared memory");
 enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = K_FULL + kStages, V_FULL = K_EMPTY + kStages, V_EMPTY = V_FULL + kStages,
-           S_FULL = V_EMPTY + kStages, P_FULL = S_FULL + 2, P_EMPTY, O_DONE, META_FULL, kNumBars = META_FULL + 8 };
+           S_FULL = V_EMPTY + kStages, S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_EMPTY, O_DONE, META_FULL, kNumBars = META_FULL + 8 };
 static_assert(kNumBars <= 32, "barrier area");
+
+struct Maps { CUtensorMap m[4]; };      // the same tensor with boxes of 16, 32, 64 and 128 rows
 
 struct Params {
   int BH, H, N, Cq, Ck;
@@ -70,7 +73,7 @@ struct Params {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, Params prm) {
+k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ Maps mapsV, Params prm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
@@ -102,7 +105,7 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
   const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
 
   if (tid == 0) {
-    for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == P_FULL || i == Q_FULL) ? 256 : 1);
+    for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == P_FULL || i == Q_FULL || i == S_FREE || i == S_FREE + 1) ? 256 : 1);
     misc[1] = 0; misc[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -156,27 +159,36 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
       const bool is_k = warp == 8;
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
       const uint32_t buf0 = base + (is_k ? Smem::k : Smem::v);
-      const CUtensorMap* map = is_k ? &mapK : &mapV;
+      const Maps* maps = is_k ? &mapsK : &mapsV;
       int ri = 0, off = 0;
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kStages;
         const uint32_t ph = ((i / kStages) & 1) ^ 1;         // empty barriers: the first pass completes immediately
-        int my_start = 0, my_gid = 0;
+        // up to 8 boxes of 16 rows; consecutive boxes of one group form a segment, fetched by one copy per set bit
+        // of its box count (128, 64, 32 or 16 rows), largest first
+        int my_start = 0, my_gid = 0, my_t = 0, my_n = 0, nsub = 0;
         uint32_t cnt_bits = 0;
-        int nsub = 0;
-#pragma unroll
-        for (int j = 0; j < kSubPerTile; ++j) {
-          if (ri < nroute) {
-            const int2 rg = ranges[ri];
-            if (j == lane) { my_start = rg.x + off; my_gid = gid[ri]; }
-            const int c = min(kSub, rg.y - off);
-            cnt_bits |= (uint32_t)(c - 1) << (4 * j);
-            nsub = j + 1;
-            off += kSub;
-            if (off >= rg.y) { ++ri; off = 0; }
+        while (nsub < kSubPerTile && ri < nroute) {
+          const int2 rg = ranges[ri];
+          const int left = rg.y - off, nb = (left + kSub - 1) / kSub;
+          const int n = min(kSubPerTile - nsub, nb);
+          if (lane >= nsub && lane < nsub + n) { my_t = lane - nsub; my_n = n; my_start = rg.x + off + my_t * kSub; my_gid = gid[ri]; }
+          uint32_t bits = n == 8 ? 0xFFFFFFFFu : ((1u << (4 * n)) - 1u);
+          if (n == nb) {
+            const int sh = 4 * (n - 1);
+            bits = (bits & ~(0xFu << sh)) | ((uint32_t)(left - (n - 1) * kSub - 1) << sh);
+            ++ri; off = 0;
+          } else {
+            off += n * kSub;
           }
+          cnt_bits |= bits << (4 * nsub);
+          nsub += n;
         }
+        int my_k = -1;
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb)
+          if (lane < nsub && ((my_n >> kb) & 1) && my_t == ((my_n >> (kb + 1)) << (kb + 1))) my_k = kb;
         ok = __all_sync(0xffffffffu, mbar_wait(bar(empty0 + s), ph, abort_flag));
         if (!ok) break;
         if (is_k) {
@@ -187,23 +199,24 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
         if (lane == 0) mbar_expect_tx(bar(full0 + s), nsub * 2 * kSubBytes);
         __syncwarp();
-        if (lane < nsub) {
+        if (my_k >= 0) {
           const uint32_t dst = buf0 + s * kTileBytes + lane * kSubBytes;
-          tma_load_4d(dst, map, bar(full0 + s), 0, my_start, bh, 0);
-          tma_load_4d(dst + kHalfBytes, map, bar(full0 + s), 64, my_start, bh, 0);
+          tma_load_4d(dst, &maps->m[my_k], bar(full0 + s), 0, my_start, bh, 0);
+          tma_load_4d(dst + kHalfBytes, &maps->m[my_k], bar(full0 + s), 64, my_start, bh, 0);
         }
       }
     }
   } else if (warp == 9) {
-    // =========================== MMA issuer ==================================================
+    // =========================== Q K^T issuer (the two products are issued by two threads) ====
     if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
+      const uint32_t idesc_qk = idesc_bf16(0, 128);
       const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
-      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
-      auto issue_qk = [&](int i) -> bool {
+      for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kStages;
-        if (!mbar_wait(bar(K_FULL + s), (i / kStages) & 1, abort_flag)) return false;
+        // score buffer i mod 2 is free once every softmax thread holds tile i - 2 in registers
+        if (i >= 2 && !mbar_wait(bar(S_FREE + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar(K_FULL + s), (i / kStages) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
         const uint64_t kd = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
@@ -214,10 +227,14 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
         umma_commit(bar(K_EMPTY + s));
         umma_commit(bar(S_FULL + (i & 1)));
-        return true;
-      };
-      if (ok && n_tiles > 0) ok = issue_qk(0);
-      if (ok && n_tiles > 1) ok = issue_qk(1);
+      }
+    }
+  } else if (warp == 11) {
+    // =========================== P V issuer ==================================================
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16(1, 128);
+      const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
+      bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kStages;
         if (!mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag)) { ok = false; break; }
@@ -232,11 +249,10 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
             umma_bf16_ts(tmem + 320u, tmem + 256u + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(V_EMPTY + s));
         umma_commit(bar(P_EMPTY));
-        if (i + 2 < n_tiles) ok = issue_qk(i + 2);
       }
       if (ok) umma_commit(bar(O_DONE));                        // completes at once when there was no tile
     }
-  } else {
+  } else if (warp < 8) {
     // =========================== softmax (warps 0-7) =======================================
     const int hh = warp >> 2, wq = warp & 3;
     const int row = wq * 32 + lane;
@@ -267,8 +283,15 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int i = 0; i < n_tiles; ++i) {
-      ok = __all_sync(FULL, ok && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
-                                mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
+      // the barriers of this tile are polled back to back (their shared-memory round trips overlap)
+      const bool t_meta = mbar_try(bar(META_FULL + (i & 7)), (i >> 3) & 1);
+      const bool t_s = mbar_try(bar(S_FULL + (i & 1)), (i >> 1) & 1);
+      {
+        bool w = ok;
+        if (!t_meta) w = w && mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag);
+        if (!t_s) w = w && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag);
+        ok = __all_sync(FULL, w);
+      }
       float s[64];
       float mx = -INFINITY;
       if (ok) {
@@ -291,6 +314,8 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
           }
         }
         tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(bar(S_FREE + (i & 1)));                         // the scores are in registers
 #pragma unroll
         for (int bx = 0; bx < 4; ++bx) {
 #pragma unroll
@@ -298,9 +323,9 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
-          mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+        for (int c = 0; c < 64; c += 8) {
+          mx4[0] = max3(mx4[0], s[c], s[c + 1]); mx4[1] = max3(mx4[1], s[c + 2], s[c + 3]);
+          mx4[2] = max3(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3(mx4[3], s[c + 6], s[c + 7]);
         }
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
@@ -327,14 +352,19 @@ k_attention_packed(const __grid_constant__ CUtensorMap mapK, const __grid_consta
           tmem_st32(o_addr + q * 32, t);
         }
       }
-      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+      // exponentials: kPolyOf8 of every 8 pairs on the FMA pipe, the others on the special-function unit;
+      // masked columns give exactly 0 on both
+      float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 sc2 = make_float2(sc, sc), mneg2 = make_float2(mneg, mneg);
 #pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-        s[c] = ex2(fmaf(s[c], sc, mneg)); s[c + 1] = ex2(fmaf(s[c + 1], sc, mneg));      // masked columns: exp2(-inf) = 0
-        s[c + 2] = ex2(fmaf(s[c + 2], sc, mneg)); s[c + 3] = ex2(fmaf(s[c + 3], sc, mneg));
-        ps4[0] += s[c]; ps4[1] += s[c + 1]; ps4[2] += s[c + 2]; ps4[3] += s[c + 3];
+      for (int q = 0; q < 32; ++q) {
+        float2 x = __ffma2_rn(make_float2(s[2 * q], s[2 * q + 1]), sc2, mneg2);
+        if ((q & 7) < kPolyOf8) x = ex2_poly2(x);
+        else { x.x = ex2(x.x); x.y = ex2(x.y); }
+        s[2 * q] = x.x; s[2 * q + 1] = x.y;
+        ps2[q & 1] = __fadd2_rn(ps2[q & 1], x);
       }
-      l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+      l = l * corr + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
       {
         uint32_t w[32];
 #pragma unroll
@@ -445,9 +475,11 @@ void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos
 bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st) {
   using namespace tc;
   using namespace tc::packed;
-  CUtensorMap mk, mv;
-  if (!make_map(&mk, a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub) || !make_map(&mv, a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub))
-    return false;
+  Maps mk, mv;
+  for (int k = 0; k < 4; ++k)
+    if (!make_map(&mk.m[k], a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k) ||
+        !make_map(&mv.m[k], a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k))
+      return false;
   Params p{};
   p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.scale_log2 = a.scale * 1.4426950408889634f;
   p.rem_pos = rem_pos; p.rem_grp = rem_grp; p.rem_cnt = rem_cnt;

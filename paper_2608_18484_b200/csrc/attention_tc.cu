@@ -42,6 +42,10 @@ constexpr uint32_t kSubBytes = kSub * 128;            // 2 KB per box
 #ifndef SPR_V_STAGES
 #define SPR_V_STAGES 2
 #endif
+#ifndef SPR_POLY_OF8
+#define SPR_POLY_OF8 3
+#endif
+constexpr int kPolyOf8 = SPR_POLY_OF8;  // pairs of every 8 whose exponential is a polynomial on the FMA pipe
 constexpr int kKStages = SPR_K_STAGES;  // K tiles in flight (consumed by Q K^T)
 constexpr int kVStages = SPR_V_STAGES;  // V tiles in flight (consumed by P V)
 
@@ -373,9 +377,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
-          mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+        for (int c = 0; c < 64; c += 8) {
+          mx4[0] = max3(mx4[0], s[c], s[c + 1]); mx4[1] = max3(mx4[1], s[c + 2], s[c + 3]);
+          mx4[2] = max3(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3(mx4[3], s[c + 6], s[c + 7]);
         }
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
@@ -412,14 +416,18 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           tmem_st32(o_addr + q * 32, t);
         }
       }
-      float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+      // exponentials: kPolyOf8 of every 8 pairs on the FMA pipe, the others on the special-function unit
+      float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 sc2 = make_float2(sc, sc), mneg2 = make_float2(mneg, mneg);
 #pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-        s[c] = ex2(fmaf(s[c], sc, mneg)); s[c + 1] = ex2(fmaf(s[c + 1], sc, mneg));
-        s[c + 2] = ex2(fmaf(s[c + 2], sc, mneg)); s[c + 3] = ex2(fmaf(s[c + 3], sc, mneg));
-        ps4[0] += s[c]; ps4[1] += s[c + 1]; ps4[2] += s[c + 2]; ps4[3] += s[c + 3];
+      for (int q = 0; q < 32; ++q) {
+        float2 x = __ffma2_rn(make_float2(s[2 * q], s[2 * q + 1]), sc2, mneg2);
+        if ((q & 7) < kPolyOf8) x = ex2_poly2(x);
+        else { x.x = ex2(x.x); x.y = ex2(x.y); }
+        s[2 * q] = x.x; s[2 * q + 1] = x.y;
+        ps2[q & 1] = __fadd2_rn(ps2[q & 1], x);
       }
-      l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+      l = l * corr + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
       // P (bf16, two per 32-bit column): this half's 64 probabilities -> 32 columns
       {
         uint32_t w[32];

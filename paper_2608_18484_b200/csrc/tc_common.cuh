@@ -137,6 +137,29 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // shared-memory matrix descriptor, 128-byte swizzle, 8-row atoms 1024 bytes apart
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+// 2^x for a pair of arguments on the FMA pipe (the special-function unit is the scarce resource of the softmax
+// loop): round to the nearest integer n with the 1.5 * 2^23 trick, cubic minimax polynomial for 2^f on
+// f = x - n in [-1/2, 1/2] (relative error 1.1e-4, below the bf16 rounding of the probabilities), n added
+// into the exponent field.  Arguments below -127 give exactly 0.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  const float kMagic = 12582912.f;
+  x.x = fmaxf(x.x, -127.f); x.y = fmaxf(x.y, -127.f);
+  const float2 xf = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(xf, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(f, make_float2(0.05550411f, 0.05550411f), make_float2(0.24022651f, 0.24022651f));
+  p = __ffma2_rn(p, f, make_float2(0.69314718f, 0.69314718f));
+  p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
+  float2 y;
+  y.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(xf.x) << 23));
+  y.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(xf.y) << 23));
+  return y;
+}
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
          (1ull << 46) | (2ull << 61);
