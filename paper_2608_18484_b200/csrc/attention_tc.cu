@@ -90,38 +90,48 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   float* xmax = reinterpret_cast<float*>(sm + Smem::xchg);                 // [2][2][128] half-row maxima of the current / next tile
   float* xsum = xmax + 4 * 128;                                            // [2][128] half-row sums (end)
   uint2* meta = reinterpret_cast<uint2*>(sm + Smem::meta);
-  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem base, [1] abort, [2] total boxes
+  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);   // [0] tmem base, [1] abort, [2] total boxes, [3] leave, [4] query group, [5] its first tile
   const uint32_t bars = base + Smem::bars;
   auto bar = [&](int i) { return bars + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y, b = bh / prm.H, h = bh % prm.H;
-  // once any CTA has recorded a timeout the remaining CTAs of the launch leave at once
-  // (also if the shared-memory base is not aligned as the swizzled tiles require)
+#ifdef SPR_ATTN_TIMING
+  const long long cta_t0 = clock64();
+#endif
+  // ---- which query tile ---------------------------------------------------------------
+  // Few dependent global reads: one round finds the query group of this tile (every thread tests one group),
+  // reads the error word and stages the key-group offsets in shared memory (the K ring is still idle); the
+  // second round reads the group's rows and routes.
+  // Once any CTA has recorded a timeout the remaining CTAs of the launch leave at once (also if the
+  // shared-memory base is not aligned as the swizzled tiles require).
+  int* kv_stage = reinterpret_cast<int*>(sm + Smem::k);
   if (tid == 0) {
     misc[3] = (prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT) || (base & 1023u) != 0;
     if ((base & 1023u) != 0) set_error(prm.err, SPARSEPR_ERR_CUDA);
+    misc[4] = -1;
   }
   __syncthreads();
-  if (misc[3]) return;
-
-  // ---- which query tile ---------------------------------------------------------------
-  int row0, nrows, nroute;
-  const int* ridx = nullptr;
-  const int* kvoff = nullptr;
   if (prm.sparse) {
     const int* toff = prm.tile_off + (i64)bh * (prm.Cq + 1);
-    if ((int)blockIdx.x >= toff[prm.Cq]) return;
-    int lo = 0, hi = prm.Cq - 1;
-    while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (toff[mid] <= (int)blockIdx.x) lo = mid; else hi = mid - 1; }
-    const int g = lo;
+    const int* kvo = prm.kv_off + (i64)bh * (prm.Ck + 1);
+    for (int g = tid; g < prm.Cq; g += kThreads)
+      if (toff[g] <= (int)blockIdx.x && (int)blockIdx.x < toff[g + 1]) { misc[4] = g; misc[5] = toff[g]; }
+    for (int g = tid; g <= prm.Ck; g += kThreads) kv_stage[g] = kvo[g];
+    __syncthreads();
+  }
+  if (misc[3] || (prm.sparse && misc[4] < 0)) return;        // error, or a tile index beyond this head's tiles
+  int row0, nrows, nroute;
+  const int* ridx = nullptr;
+  if (prm.sparse) {
+    const int g = misc[4];
     const int* qoff = prm.q_off + (i64)bh * (prm.Cq + 1);
-    row0 = qoff[g] + ((int)blockIdx.x - toff[g]) * kTile;
-    nrows = min(kTile, qoff[g + 1] - row0);
     const int* rp = prm.route_ptr + (i64)bh * (prm.Cq + 1);
-    ridx = prm.route_idx + (i64)bh * prm.Cq * prm.Ck + rp[g];
-    nroute = rp[g + 1] - rp[g];
-    kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
+    const int q0 = qoff[g], q1 = qoff[g + 1], r0 = rp[g], r1 = rp[g + 1];
+    row0 = q0 + ((int)blockIdx.x - misc[5]) * kTile;
+    nrows = min(kTile, q1 - row0);
+    ridx = prm.route_idx + (i64)bh * prm.Cq * prm.Ck + r0;
+    nroute = r1 - r0;
   } else {
     row0 = blockIdx.x * kTile;
     nrows = min(kTile, prm.N - row0);
@@ -141,13 +151,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     int boxes = 0;
     for (int t = tid; t < nroute; t += kThreads) {
       int start = 0, len = prm.N;
-      if (prm.sparse) { const int g = ridx[t]; start = kvoff[g]; len = kvoff[g + 1] - start; }
+      if (prm.sparse) { const int g = ridx[t]; start = kv_stage[g]; len = kv_stage[g + 1] - start; }
       ranges[t] = make_int2(start, len);
       boxes += (len + kSub - 1) / kSub;
     }
     boxes = warp_sum(boxes);
     if (lane == 0 && boxes) atomicAdd((int*)&misc[2], boxes);
   }
+  fence_async_smem();                        // the staged offsets were read from memory that the copies will overwrite
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -330,6 +341,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     bool ok = true;
     const float sc = prm.scale_log2;
 #ifdef SPR_ATTN_TIMING
+    const long long cta_t1 = clock64();
+#endif
+#ifdef SPR_ATTN_TIMING
     long long tw = 0, tl = 0, tm = 0, ts = 0, tx = 0, tp = 0, tmx = 0, t0;
 #define SPR_T0() t0 = clock64()
 #define SPR_ACC(v) do { const long long t1 = clock64(); v += t1 - t0; t0 = t1; } while (0)
@@ -446,7 +460,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
              tw / max(1, n_tiles), tl / max(1, n_tiles), tmx / max(1, n_tiles), tx / max(1, n_tiles), tp / max(1, n_tiles), tm / max(1, n_tiles), ts / max(1, n_tiles));
 #endif
     // ---- row sums of the two halves, normalise, store ------------------------------------------
+#ifdef SPR_ATTN_TIMING
+    const long long cta_t2 = clock64();
+#endif
     if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
+#ifdef SPR_ATTN_TIMING
+    const long long cta_t3 = clock64();
+#endif
     xsum[hh * 128 + row] = l;
     asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
     const float ltot = l + xsum[(hh ^ 1) * 128 + row];
@@ -486,7 +506,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
       }
     }
+#ifdef SPR_ATTN_TIMING
+    if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && warp == 0)
+      printf("cta tiles %d: prologue %lld  loop %lld  wait O %lld  epilogue %lld\n", n_tiles, cta_t1 - cta_t0, cta_t2 - cta_t1, cta_t3 - cta_t2, clock64() - cta_t3);
   }
+#else
+  }
+#endif
   // ---- teardown ----------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
