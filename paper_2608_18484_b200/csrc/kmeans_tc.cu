@@ -251,13 +251,11 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           todo &= ~members;
           // float32 partial sums in ascending row order (a fixed order, hence reproducible), one
           // conversion to fixed point per (cluster, column)
-          float a0 = 0.f, a1 = 0.f;
+          float2 a2 = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int rr = 0; rr < 32; ++rr) {
-            const bool in = (members >> rr) & 1u;
-            a0 += in ? pv0[rr] : 0.f;
-            a1 += in ? pv1[rr] : 0.f;
-          }
+          for (int rr = 0; rr < 32; ++rr)
+            if ((members >> rr) & 1u) a2 = __fadd2_rn(a2, make_float2(pv0[rr], pv1[rr]));   // one packed add per member row
+          const float a0 = a2.x, a1 = a2.y;
           const i64 acc0 = __float2ll_rn(a0 * scl), acc1 = __float2ll_rn(a1 * scl);
           i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
           if (2 * lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + 2 * lane), (u64)acc0);
