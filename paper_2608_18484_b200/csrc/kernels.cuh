@@ -95,7 +95,7 @@ bool attention_tc_supported(const AttnArgs& a);
 bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 // Query-group remainders of 1..kRemRows rows are left out of the 128-row kernel's tiles (tile offsets built with
 // small_rem = kRemRows) and handled by attention_packed.cu
-constexpr int kRemRows = 64;
+constexpr int kRemRows = 32;
 // attention_packed.cu: those remainders, packed across groups into 128-row tiles that walk over all keys with
 // per-row route masks.  rem_pos / rem_grp [BH][N], rem_cnt [BH] are built from the query offsets once per plan.
 cudaError_t init_attention_packed();

@@ -55,9 +55,10 @@ def test_full_size_480p_sampled_rows():
         q_perm, q_off = exp["q_perm"][i], exp["q_off"][i]
         sizes = np.diff(q_off)
         rows = list(rng.choice(wl.N, 24, replace=False))
-        small = [a for a in range(C) if 0 < sizes[a] % 128 <= 64]
-        assert small, "the workload is expected to leave short remainders"
-        for a in small[:6]:                                     # last row of a short remainder, first row of the group
+        small = [a for a in range(C) if 0 < sizes[a] % 128 <= 32]      # remainders packed across groups
+        mid = [a for a in range(C) if sizes[a] % 128 > 32]              # remainders with a (partly empty) tile of their own
+        assert small and mid, "the workload is expected to leave short and long remainders"
+        for a in small[:6] + mid[:3]:                           # last row of the remainder, first row of the group
             rows += [int(q_perm[q_off[a + 1] - 1]), int(q_perm[q_off[a]])]
         rows += [int(p) for p in P[:4]]
         rows = np.array(sorted(set(rows)), dtype=np.int64)
