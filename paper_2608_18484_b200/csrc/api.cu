@@ -261,8 +261,9 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
   const Resolved& R = p->r;
   const int ld = round16(r);
   launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
-  launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st);
   const bool tcp = kmeans_tc_supported();
+  float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
+  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st);
   if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
@@ -279,7 +280,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
       launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
                            upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
     }
-    if (upd) launch_kmeans_finalize(p->mu, p->mu2, p->mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st);
+    if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st);
   }
 }
 

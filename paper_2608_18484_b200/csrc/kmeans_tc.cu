@@ -62,8 +62,16 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
 
   __shared__ __align__(16) float mu2s[kMaxGroups];          // ||mu_c||^2, +inf beyond C
   __shared__ int s_skip;
-  for (int c = tid; c < kMaxGroups; c += kKmThreads) mu2s[c] = c < prm.C ? prm.mu2[(i64)bh * prm.C + c] : INFINITY;
+  __shared__ float s_red[34];
+  float mu2max = 0.f;
+  for (int c = tid; c < kMaxGroups; c += kKmThreads) {
+    const float v = c < prm.C ? prm.mu2[(i64)bh * prm.C + c] : INFINITY;
+    mu2s[c] = v;
+    if (c < prm.C) mu2max = fmaxf(mu2max, v);
+  }
   if (tid == 0) s_skip = prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT;
+  // largest centroid norm of the head, rounded up: it enters the bound on the score error only
+  const float mm_head = sqrtf(block_max(mu2max, s_red)) * 1.000001f;
   __syncthreads();
   if (s_skip) return;
 
@@ -152,7 +160,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     const uint32_t FULL = 0xffffffffu;
     const int grp = warp < 4 ? 0 : 1, wq = warp & 3;
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-    const float mm = prm.mumax[bh];
+    const float mm = mm_head;
     bool ok = true;
 #ifdef SPR_KM_TIMING
     long long eP = 0, eW = 0, eA = 0, eD = 0, eS = 0, e0 = clock64();

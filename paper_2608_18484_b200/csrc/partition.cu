@@ -1,6 +1,7 @@
 // Response-Coupled Partitioning kernels (Section 4.1, Appendix B): sampled-query
 // Gram matrix, batched Jacobi eigen-decomposition -> feature maps, response
 // projections, k-means assignment/update, stable counting sort, group means.
+#include <algorithm>
 #include "kernels.cuh"
 
 namespace spr {
@@ -345,7 +346,9 @@ __global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, i
 
 // mu <- sums / counts for non-empty clusters (empty ones keep their centroid), then
 // ||mu_c||^2 (float64 -> float32) and the largest centroid norm of the head.
-// One CTA per head.
+// gridDim.y CTAs per head share the centroids (warp w of part y takes c = y nw + w, + nw gridDim.y, ...); the
+// largest norm needs all of them and is written only when one CTA holds the whole head (mumax may be null otherwise:
+// the tensor-core assignment derives the bound from ||mu_c||^2 itself).
 __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu, float* __restrict__ mu2,
                                                           float* __restrict__ mumax, i64* __restrict__ sums,
                                                           int* __restrict__ counts, const int* __restrict__ fx_shift,
@@ -355,7 +358,7 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
   const double inv_sc = update ? ldexp(1.0, -fx_shift[bh]) : 0.0;
   float mx = 0.f;
-  for (int c = w; c < C; c += nw) {
+  for (int c = blockIdx.y * nw + w; c < C; c += nw * gridDim.y) {
     float* m = mu + ((i64)bh * C + c) * R;
     i64* s = sums + ((i64)bh * C + c) * R;
     const int cnt = update ? counts[(i64)bh * C + c] : 0;
@@ -376,8 +379,10 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
       mx = fmaxf(mx, (float)sqrt(n2) * 1.0000002f);
     }
   }
-  mx = block_max(mx, red);
-  if (threadIdx.x == 0) mumax[bh] = mx;
+  if (gridDim.y == 1 && mumax != nullptr) {
+    mx = block_max(mx, red);
+    if (threadIdx.x == 0) mumax[bh] = mx;
+  }
 }
 
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
@@ -389,7 +394,13 @@ void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st) {
   const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
-  k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update);
+  if (mumax != nullptr) {
+    k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update);
+  } else {
+    // one warp per centroid, spread over enough CTAs to fill the GPU
+    const int parts = std::max(1, std::min(32, (C + 7) / 8));
+    k_kmeans_finalize<<<dim3(BH, parts), 256, 0, st>>>(mu, mu2, nullptr, sums, counts, fx_shift, C, r, R, update);
+  }
 }
 
 // =============================================================================
