@@ -90,8 +90,8 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------
 def launches_per_call(T, fitted, tensor_path):
     """Kernels of this library launched by one plan + attend call (memsets excluded)."""
-    if tensor_path:      # per side: split features; per iteration: split centroids, assign, recheck; T-1 updates
-        kmeans = 2 + 1 + 3 * T + (T - 1)
+    if tensor_path:      # per side: init, first norms, split features; per iteration: assign, recheck; T-1 updates
+        kmeans = 2 + 1 + 2 * T + (T - 1)
     else:                # init, first norms, T assignments, T-1 updates
         kmeans = 2 + T + (T - 1)
     plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 3      # per side: Gram+eig, projection, k-means, sort+means; probes; route; tile offsets + remainder rows

@@ -263,12 +263,12 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
   launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
   const bool tcp = kmeans_tc_supported();
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
-  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st);
+  // (with the tensor-core assignment the finalize step also writes the two bf16 words of every centroid)
+  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
     if (tcp) {
-      launch_split_bf16(p->mu, ld, (i64)R.BH * C, r, p->mh, p->ml, nullptr, st);
       KmeansTcArgs ka{};
       ka.BH = R.BH; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
       ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2; ka.mumax = p->mumax;
@@ -280,7 +280,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
       launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
                            upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
     }
-    if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st);
+    if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   }
 }
 

@@ -20,7 +20,7 @@ void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int 
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
-                            int C, int r, int update, cudaStream_t st);
+                            int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh = nullptr, __nv_bfloat16* ml = nullptr);
 void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
                           const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
                           int* recheck_count, cudaStream_t st);

@@ -352,7 +352,8 @@ __global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, i
 __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu, float* __restrict__ mu2,
                                                           float* __restrict__ mumax, i64* __restrict__ sums,
                                                           int* __restrict__ counts, const int* __restrict__ fx_shift,
-                                                          int C, int r, int R, int update) {
+                                                          int C, int r, int R, int update,
+                                                          __nv_bfloat16* __restrict__ mh, __nv_bfloat16* __restrict__ ml) {
   __shared__ float red[34];
   const int bh = blockIdx.x;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -363,13 +364,23 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
     i64* s = sums + ((i64)bh * C + c) * R;
     const int cnt = update ? counts[(i64)bh * C + c] : 0;
     double n2 = 0.0;
-    for (int k = lane; k < R; k += 32) {
-      float v = m[k];
-      if (update) {
-        if (cnt > 0 && k < r) { v = (float)((double)s[k] * inv_sc / (double)cnt); m[k] = v; }
-        s[k] = 0;
+    for (int k = lane; k < 64; k += 32) {
+      float v = 0.f;
+      if (k < R) {
+        v = m[k];
+        if (update) {
+          if (cnt > 0 && k < r) { v = (float)((double)s[k] * inv_sc / (double)cnt); m[k] = v; }
+          s[k] = 0;
+        }
+        n2 += (double)v * (double)v;
       }
-      n2 += (double)v * (double)v;
+      if (mh != nullptr) {
+        // the two bf16 words of the centroid for the tensor-core assignment, [C][64] with zeros beyond r
+        const float x = k < r ? v : 0.f;
+        const __nv_bfloat16 hb = __float2bfloat16_rn(x);
+        mh[((i64)bh * C + c) * 64 + k] = hb;
+        ml[((i64)bh * C + c) * 64 + k] = __float2bfloat16_rn(x - __bfloat162float(hb));
+      }
     }
     n2 = warp_sum(n2);
     __syncwarp();
@@ -392,14 +403,14 @@ void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C
   k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, mu, sums, counts, maxabs_bits, fx_shift);
 }
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
-                            int C, int r, int update, cudaStream_t st) {
+                            int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh, __nv_bfloat16* ml) {
   const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
   if (mumax != nullptr) {
-    k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update);
+    k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update, mh, ml);
   } else {
     // one warp per centroid, spread over enough CTAs to fill the GPU
     const int parts = std::max(1, std::min(32, (C + 7) / 8));
-    k_kmeans_finalize<<<dim3(BH, parts), 256, 0, st>>>(mu, mu2, nullptr, sums, counts, fx_shift, C, r, R, update);
+    k_kmeans_finalize<<<dim3(BH, parts), 256, 0, st>>>(mu, mu2, nullptr, sums, counts, fx_shift, C, r, R, update, mh, ml);
   }
 }
 
