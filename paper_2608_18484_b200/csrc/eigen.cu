@@ -480,20 +480,34 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   // ---- 6. back-transformation z <- H_0 ... H_{n-3} z, scaling, output -------------------------------------
   {
     constexpr int tpv = 16;                                      // threads per vector (1024 threads cover 64 vectors)
+    constexpr int npt = NN / tpv;                                // entries of the vector per thread, kept in registers
     const int j = tid / tpv, q = tid % tpv;
     const bool active = j < r;
+    T zr[npt];
+#pragma unroll
+    for (int t = 0; t < npt; ++t) zr[t] = active ? Z[(q + tpv * t) * kZld + j] : T(0.0);
     for (int k = NN - 3; k >= 0; --k) {
       const T bk = beta[k];
       if (bk == T(0.0)) continue;                                   // uniform
+      // thread q holds entries i = q, q + 16, ...; the reflector is zero up to entry k
+      T av[npt];
+#pragma unroll
+      for (int t = 0; t < npt; ++t) {
+        const int i = q + tpv * t;
+        av[t] = i > k ? A[k * LD + pos(i)] : T(0.0);
+      }
       T dot = T(0.0);
-      if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) dot = fma(A[k * LD + pos(i)], Z[i * kZld + j], dot);
+#pragma unroll
+      for (int t = 0; t < npt; ++t) dot = fma(av[t], zr[t], dot);
 #pragma unroll
       for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
       const T f = bk * dot;
-      if (active)
-        for (int i = k + 1 + q; i < NN; i += tpv) Z[i * kZld + j] -= f * A[k * LD + pos(i)];
-      __syncwarp();
+#pragma unroll
+      for (int t = 0; t < npt; ++t) zr[t] = fma(-f, av[t], zr[t]);
+    }
+    if (active) {
+#pragma unroll
+      for (int t = 0; t < npt; ++t) Z[(q + tpv * t) * kZld + j] = zr[t];
     }
   }
   __syncthreads();
