@@ -1,5 +1,6 @@
 // Shared routing (Section 4.3) and query-group-stratified probe selection
 // (Algorithm A.1, Appendix A.2).
+#include <cstdio>
 #include "kernels.cuh"
 
 namespace spr {
@@ -95,6 +96,15 @@ void launch_cell_scores(const float* theta, const float* kappa, const int* nq, c
 // =============================================================================
 __device__ __forceinline__ i64 block_sum_i64(i64 v, i64* scratch) { return block_sum<i64>(v, scratch); }
 
+// Eight 32-cell chunks of one score row, loaded together: the scans below are bound by the latency of these reads
+__device__ __forceinline__ void load_row_chunks(const unsigned* __restrict__ row, int b00, int Ck, int lane, unsigned (&ub)[8]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int b = b00 + 32 * j + lane;
+    ub[j] = b < Ck ? row[b] : 0u;
+  }
+}
+
 __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__ score, const int* __restrict__ nq,
                                                        const int* __restrict__ nk, int Cq, int Ck, i64 budget,
                                                        int select_all, int* __restrict__ route_ptr,
@@ -115,16 +125,29 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   for (int a = threadIdx.x; a < Cq; a += blockDim.x) nqs[a] = nq[(i64)bh * Cq + a];
   __syncthreads();
 
+#ifdef SPR_RT_TIMING
+  long long rt[8]; int rti = 0; long long rt0 = clock64();
+#define SPR_RT() do { const long long t1 = clock64(); if (rti < 8) rt[rti++] = t1 - rt0; rt0 = t1; } while (0)
+#else
+#define SPR_RT()
+#endif
   // 1. forced cells
   i64 fcost = 0;
   for (int a = w; a < Cq; a += nw) {
     u64 best = 0;      // (bits+1) << 32 | (0xFFFFFFFF - b): larger = better score, then lower b
     if (nqs[a] > 0)
-      for (int b = lane; b < Ck; b += 32)
-        if (nks[b] > 0) {
-          const u64 key = (((u64)u[(i64)a * Ck + b] + 1ull) << 32) | (u64)(0xFFFFFFFFu - (unsigned)b);
-          best = key > best ? key : best;
+      for (int b00 = 0; b00 < Ck; b00 += 256) {
+        unsigned ub[8];
+        load_row_chunks(u + (i64)a * Ck, b00, Ck, lane, ub);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int b = b00 + 32 * j + lane;
+          if (b < Ck && nks[b] > 0) {
+            const u64 key = (((u64)ub[j] + 1ull) << 32) | (u64)(0xFFFFFFFFu - (unsigned)b);
+            best = key > best ? key : best;
+          }
         }
+      }
     best = warp_max(best);
     const int fb = best ? (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull)) : -1;
     if (lane == 0) {
@@ -134,6 +157,7 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   }
   fcost = block_sum_i64(fcost, red);     // contains a __syncthreads: forced[] visible below
   const i64 rem = budget - fcost;
+  SPR_RT();
 
   // 2. threshold search: S(t) = cost of live, non-forced cells with bits >= t; find the smallest t with
   //    S(t) <= rem.  Radix descent, one byte of the bit pattern per pass: per-warp cost histograms over
@@ -155,29 +179,45 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
       for (int e = threadIdx.x; e < nw * 256; e += blockDim.x) whist[e] = 0;
       __syncthreads();
       i64* myh = whist + w * 256;
+      int* hk = reinterpret_cast<int*>(whist + nw * 256) + w * 256;   // per-row key counts by digit, zero between rows
+      for (int k = lane; k < 256; k += 32) hk[k] = 0;
+      __syncwarp();
       for (int a = w; a < Cq; a += nw) {
         if (nqs[a] == 0) continue;
         const int fb = forced[a];
         const i64 na = nqs[a];
-        for (int b0 = 0; b0 < Ck; b0 += 32) {
-          const int b = b0 + lane;
-          unsigned bits = 0;
-          bool in = b < Ck && b != fb && nks[b] > 0;
-          if (in) {
-            bits = u[(i64)a * Ck + b];
-            in = level == 0 || (bits >> (shift + 8)) == (prefix >> (shift + 8));
-          }
-          unsigned todo = __ballot_sync(0xffffffffu, in);
-          const int digit = (bits >> shift) & 255;
-          while (todo) {                                         // lanes of one digit add their key counts together
-            const int leader = __ffs(todo) - 1;
-            const int dl = __shfl_sync(0xffffffffu, digit, leader);
-            const unsigned grp = __ballot_sync(0xffffffffu, in && digit == dl) & todo;
-            const int keys = __reduce_add_sync(0xffffffffu, (in && digit == dl) ? nks[b] : 0);
-            if (lane == leader) myh[dl] += na * keys;
-            todo &= ~grp;
+        for (int b00 = 0; b00 < Ck; b00 += 256) {
+          unsigned ub[8];
+          load_row_chunks(u + (i64)a * Ck, b00, Ck, lane, ub);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int b = b00 + 32 * j + lane;
+            if (b00 + 32 * j >= Ck) break;                           // uniform
+            const unsigned bits = ub[j];
+            const bool in = b < Ck && b != fb && nks[b] > 0 && (level == 0 || (bits >> (shift + 8)) == (prefix >> (shift + 8)));
+            // key counts of the row per digit, in the warp's 32-bit histogram: the lanes that share the first
+            // lane's digit add up together (the upper bytes of the scores take few values), the others add their own
+            const unsigned todo = __ballot_sync(0xffffffffu, in);
+            if (todo) {
+              const int digit = (bits >> shift) & 255;
+              const int dl = __shfl_sync(0xffffffffu, digit, __ffs(todo) - 1);
+              const bool mine = in && digit == dl;
+              const int keys = __reduce_add_sync(0xffffffffu, mine ? nks[b] : 0);
+              if (lane == 0) hk[dl] += keys;
+              __syncwarp();
+              if (in && !mine) atomicAdd(&hk[digit], nks[b]);
+            }
           }
         }
+        // the row's counts times its number of queries go to the 64-bit cost histogram
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int d = lane + 32 * k;
+          const int v = hk[d];
+          if (v) { myh[d] += na * v; hk[d] = 0; }
+        }
+        __syncwarp();
       }
       __syncthreads();
       if (w == 0) {
@@ -218,6 +258,7 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
     tstar = all_fit ? (u64)prefix : (u64)prefix + 1ull;
     taken = above;
   }
+  SPR_RT();
   // tie tier: cells with bits == tstar-1, in (a,b) order, longest prefix that fits
   __shared__ int s_tie_cnt, s_tie_idx[32];
   if (threadIdx.x == 0) { s_last_tie = -1; s_tie_cnt = 0; }
@@ -230,11 +271,18 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
     for (int a = w; a < Cq; a += nw) {
       if (nqs[a] == 0) continue;
       const int fb = forced[a];
-      for (int b = lane; b < Ck; b += 32)
-        if (nks[b] > 0 && b != fb && u[(i64)a * Ck + b] == tv) {
-          const int pos = atomicAdd(&s_tie_cnt, 1);
-          if (pos < 32) s_tie_idx[pos] = a * Ck + b;
+      for (int b00 = 0; b00 < Ck; b00 += 256) {
+        unsigned ub[8];
+        load_row_chunks(u + (i64)a * Ck, b00, Ck, lane, ub);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int b = b00 + 32 * j + lane;
+          if (b < Ck && nks[b] > 0 && b != fb && ub[j] == tv) {
+            const int pos = atomicAdd(&s_tie_cnt, 1);
+            if (pos < 32) s_tie_idx[pos] = a * Ck + b;
+          }
         }
+      }
     }
   }
   __syncthreads();
@@ -286,29 +334,35 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   const i64 last_tie = s_last_tie;
   const unsigned tvv = tie_tier ? (unsigned)(tstar - 1) : 0u;
 
-  auto selected = [&](int a, int b) -> bool {
+  auto selected = [&](int a, int b, unsigned bits) -> bool {       // bits = the cell's score word
     if (nqs[a] == 0 || nks[b] == 0) return false;
     if (forced[a] == b) return true;
-    const unsigned bits = u[(i64)a * Ck + b];
     if ((u64)bits >= tstar) return true;
     return tie_tier && bits == tvv && (i64)a * Ck + b <= last_tie;
   };
 
+  SPR_RT();
   // 3. counts, offsets, lists
   i64 pairs = 0;
   for (int a = w; a < Cq; a += nw) {
     int c = 0;
     i64 rs = 0;
-    for (int b0 = 0; b0 < Ck; b0 += 32) {
-      const int b = b0 + lane;
-      const bool s = b < Ck && selected(a, b);
-      c += __popc(__ballot_sync(0xffffffffu, s));
-      if (s) rs += nks[b];
+    for (int b00 = 0; b00 < Ck; b00 += 256) {
+      unsigned ub[8];
+      load_row_chunks(u + (i64)a * Ck, b00, Ck, lane, ub);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int b = b00 + 32 * j + lane;
+        const bool s = b < Ck && selected(a, b, ub[j]);
+        c += __popc(__ballot_sync(0xffffffffu, s));
+        if (s) rs += nks[b];
+      }
     }
     pairs += rs * nqs[a];
     if (lane == 0) cnt[a] = c;
   }
   pairs = block_sum_i64(pairs, red);
+  SPR_RT();
   const int total = block_exclusive_scan(cnt, Cq, scratch);
   int* rp = route_ptr + (i64)bh * (Cq + 1);
   int* ri = route_idx + (i64)bh * Cq * Ck;
@@ -320,18 +374,27 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   }
   for (int a = w; a < Cq; a += nw) {
     int pos = cnt[a];
-    for (int b0 = 0; b0 < Ck; b0 += 32) {
-      const int b = b0 + lane;
-      const bool s = b < Ck && selected(a, b);
-      const unsigned m = __ballot_sync(0xffffffffu, s);
-      if (s) ri[pos + __popc(m & ((1u << lane) - 1u))] = b;
-      pos += __popc(m);
+    for (int b00 = 0; b00 < Ck; b00 += 256) {
+      unsigned ub[8];
+      load_row_chunks(u + (i64)a * Ck, b00, Ck, lane, ub);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int b = b00 + 32 * j + lane;
+        const bool s = b < Ck && selected(a, b, ub[j]);
+        const unsigned m = __ballot_sync(0xffffffffu, s);
+        if (s) ri[pos + __popc(m & ((1u << lane) - 1u))] = b;
+        pos += __popc(m);
+      }
     }
   }
+  SPR_RT();
+#ifdef SPR_RT_TIMING
+  if (blockIdx.x == 0 && threadIdx.x == 0) printf("route select cycles: forced %lld  radix %lld  tie %lld  counts %lld  emit %lld\n", rt[0], rt[1], rt[2], rt[3], rt[4]);
+#endif
 }
 
-static size_t route_smem(int Cq, int Ck) {      // forced, cnt, nqs [Cq], nks [Ck] ints, then 32 x 256 int64 histograms
-  return (size_t)(3 * Cq + Ck + ((Cq + Ck) & 1)) * sizeof(int) + (size_t)32 * 256 * sizeof(long long);
+static size_t route_smem(int Cq, int Ck) {      // forced, cnt, nqs [Cq], nks [Ck] ints, then 32 x 256 int64 cost and int32 key histograms
+  return (size_t)(3 * Cq + Ck + ((Cq + Ck) & 1)) * sizeof(int) + (size_t)32 * 256 * (sizeof(long long) + sizeof(int));
 }
 // routed pairs and cells of given routes (used when a plan is imported)
 __global__ void __launch_bounds__(256) k_count_pairs(const int* __restrict__ q_off, const int* __restrict__ kv_off,
