@@ -146,7 +146,12 @@ struct sparsepr_plan_s {
   // third stream: the packed-remainder kernel (few long CTAs) beside the 128-row kernel (many short ones)
   cudaStream_t side2 = nullptr;
   cudaEvent_t ev_join2 = nullptr;
+  // the probe selection of the plan call may still run on `side` when the call returns: the first attend call
+  // orders it (its probe work follows on the same stream and is joined there); statistics, export and the
+  // destructor wait for it themselves
+  mutable bool side_pending = false;
   ~sparsepr_plan_s() {
+    if (side && side_pending) cudaStreamSynchronize(side);
     if (ev_fork) cudaEventDestroy(ev_fork);
     if (ev_join) cudaEventDestroy(ev_join);
     if (ev_join2) cudaEventDestroy(ev_join2);
@@ -429,7 +434,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
   launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
-  if (overlap) join_side(p, st);
+  if (overlap) p->side_pending = true;          // not joined here: the probes are not needed before the attend call
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
   if (!launch_ok()) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -521,6 +526,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   // kernel (whose correction is a separate pass) they run on the plan's second stream beside the
   // block-sparse kernel; a profiled call keeps everything on one stream so that stage times add up.
   const bool overlap = fitted && tensor && prof == nullptr;
+  if (p->side_pending && !overlap) { join_side(p, st); p->side_pending = false; }   // the plan call's probe selection, still on the second stream
   if (fitted) {
     cudaStream_t fs = st;
     if (overlap) { fork_side(p, st); fs = p->side; }
@@ -562,7 +568,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
       cudaStreamWaitEvent(st, p->ev_join2, 0);
     }
     tm.mark(SPARSEPR_STAGE_ATTENTION);
-    if (overlap) join_side(p, st);
+    if (overlap) { join_side(p, st); p->side_pending = false; }
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
     tm.mark(SPARSEPR_STAGE_CORRECTION);
   } else {
@@ -623,7 +629,7 @@ sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_sc
 sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t* out) {
   if (!p || !out) return SPARSEPR_ERR_INVALID_ARG;
   const Resolved& r = p->r;
-  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess || (p->side && cudaStreamSynchronize(p->side) != cudaSuccess)) return SPARSEPR_ERR_CUDA;
   std::memset(out, 0, sizeof(*out));
   std::vector<RouteState> rs(r.BH);
   std::vector<int> qo((size_t)r.BH * (r.Cq + 1)), ko((size_t)r.BH * (r.Ck + 1)), rp((size_t)r.BH * (r.Cq + 1));
@@ -697,7 +703,7 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
 sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* p, sparsepr_plan_host_t* o) {
   if (!p || !o) return SPARSEPR_ERR_INVALID_ARG;
   const Resolved& r = p->r;
-  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess || (p->side && cudaStreamSynchronize(p->side) != cudaSuccess)) return SPARSEPR_ERR_CUDA;
   const size_t BH = r.BH, N = r.N;
   bool ok = true;
   auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };

@@ -445,22 +445,48 @@ __global__ void __launch_bounds__(256) k_probe_dist(const float* __restrict__ ph
   if (p1 <= p0) return;
   const float* ph = phi + (i64)bh * N * ldphi;
   const int* pm = perm + (i64)bh * N;
-  // lane owns columns lane and lane+32
+  // lane owns columns lane and lane+32; the rows are read eight at a time (the loads are independent, the sums keep
+  // their order)
+  const bool h0 = lane < r, h1 = lane + 32 < r;
   double c0 = 0.0, c1 = 0.0;
-  for (int p = p0; p < p1; ++p) {
-    const float* row = ph + (i64)pm[p] * ldphi;
-    if (lane < r) c0 += (double)row[lane];
-    if (lane + 32 < r) c1 += (double)row[lane + 32];
+  for (int p = p0; p < p1; p += 8) {
+    float x0[8], x1[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float* row = ph + (i64)pm[min(p + j, p1 - 1)] * ldphi;
+      x0[j] = h0 ? row[lane] : 0.f;
+      x1[j] = h1 ? row[lane + 32] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (p + j < p1) { if (h0) c0 += (double)x0[j]; if (h1) c1 += (double)x1[j]; }
   }
   c0 /= (double)(p1 - p0);
   c1 /= (double)(p1 - p0);
-  for (int p = p0; p < p1; ++p) {
-    const float* row = ph + (i64)pm[p] * ldphi;
-    double s = 0.0;
-    if (lane < r) { const double t = (double)row[lane] - c0; s += t * t; }
-    if (lane + 32 < r) { const double t = (double)row[lane + 32] - c1; s += t * t; }
-    s = warp_sum(s);
-    if (lane == 0) dist[(i64)bh * N + p] = sqrt(s);
+  for (int p = p0; p < p1; p += 8) {
+    float x0[8], x1[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float* row = ph + (i64)pm[min(p + j, p1 - 1)] * ldphi;
+      x0[j] = h0 ? row[lane] : 0.f;
+      x1[j] = h1 ? row[lane + 32] : 0.f;
+    }
+    double s[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      s[j] = 0.0;
+      if (h0) { const double t = (double)x0[j] - c0; s[j] += t * t; }
+      if (h1) { const double t = (double)x1[j] - c1; s[j] += t * t; }
+    }
+    // eight independent butterflies
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s[j] += __shfl_xor_sync(0xffffffffu, s[j], o);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (lane == j && p + j < p1) dist[(i64)bh * N + p + j] = sqrt(s[j]);
   }
 }
 
