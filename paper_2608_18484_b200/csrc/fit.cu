@@ -41,24 +41,29 @@ __global__ void __launch_bounds__(256) k_fit_prepare(FitArgs a) {
   cnt = block_sum(cnt, red);
   if (threadIdx.x == 0) sc[L.flag] = (sw > 0.0 && cnt > 0.0) ? 0.0 : 1.0;
   if (!(sw > 0.0)) sw = 1.0;
-  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = cnt * (double)w[p] / sw;
+  // alpha_p = w_p / sum w once per probe (float64 divisions are expensive on this part), kept in the weight slot
+  // until the unit-mean weights replace it at the end
+  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = (double)w[p] / sw;
+  __syncthreads();
   for (int j = threadIdx.x; j < d; j += 256) {
     double mx = 0.0, mr = 0.0;
     for (int p = 0; p < M; ++p) {
-      const double al = (double)w[p] / sw, x = (double)X[p * d + j];
+      const double al = sc[L.wt + p], x = (double)X[p * d + j];
       mx += al * x;
       mr += al * ((double)Dn[p * d + j] - x);
     }
     double var = 0.0;
-    for (int p = 0; p < M; ++p) { const double t = (double)X[p * d + j] - mx; var += (double)w[p] / sw * t * t; }
-    const double s = sqrt(var + (double)a.eps_std);
+    for (int p = 0; p < M; ++p) { const double t = (double)X[p * d + j] - mx; var += sc[L.wt + p] * t * t; }
+    const double s = sqrt(var + (double)a.eps_std), inv_s = 1.0 / s;
     sc[L.mu_x + j] = mx; sc[L.mu_R + j] = mr; sc[L.s_x + j] = s;
     for (int p = 0; p < M; ++p) {
       const double x = (double)X[p * d + j];
-      sc[L.Xb + (size_t)p * d + j] = (x - mx) / s;
+      sc[L.Xb + (size_t)p * d + j] = (x - mx) * inv_s;
       sc[L.Rb + (size_t)p * d + j] = ((double)Dn[p * d + j] - x) - mr;
     }
   }
+  __syncthreads();
+  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = cnt * (double)w[p] / sw;
 }
 
 // blockIdx.x selects G = Xb^T W Xb + lam I, B(rhs) = Xb^T W Rb, S = Rb^T W Rb
@@ -114,11 +119,19 @@ __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
   if (threadIdx.x == 0) bad = sc[L.flag] != 0.0;
   for (int e = threadIdx.x; e < d * d; e += blockDim.x) Gs[(e / d) * ld + e % d] = sc[L.G + e];
   __syncthreads();
+  // (float64 square roots and divisions are expensive on this part: one thread forms 1/sqrt(pivot), and the
+  // reciprocals of the diagonal are kept for the triangular solves)
+  __shared__ double s_inv;
+  __shared__ double dinv[128];
   for (int k = 0; k < d; ++k) {
-    const double piv = Gs[k * ld + k];
-    if (!(piv > 0.0)) { if (threadIdx.x == 0) bad = 1; break; }     // uniform: every thread reads the same value
-    const double inv = 1.0 / sqrt(piv);
+    if (threadIdx.x == 0) {
+      const double piv = Gs[k * ld + k];
+      if (!(piv > 0.0)) bad = 1;
+      else { s_inv = 1.0 / sqrt(piv); dinv[k] = s_inv; }       // 1 / L_kk
+    }
     __syncthreads();
+    if (bad) break;                                               // uniform
+    const double inv = s_inv;
     for (int i = k + threadIdx.x; i < d; i += blockDim.x) Gs[i * ld + k] *= inv;   // includes the diagonal: L_kk = sqrt(piv)
     __syncthreads();
     const int n = d - k - 1;
@@ -133,19 +146,48 @@ __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
     if (threadIdx.x == 0) { sc[L.flag] = 1.0; set_error(a.err, SPARSEPR_ERR_NUMERIC); }
     return;
   }
+  // Triangular solves L Y = RHS, L^T B = Y: eight threads per right-hand-side column.  Thread (c, q) keeps the
+  // entries i = q, q + 8, ... of its column in registers; row i of the solve is a dot product over the entries
+  // already known, split over the eight threads and added up by shuffles (fixed order).
   double* Bm = sc + L.B;
-  if (threadIdx.x < d) {
-    const int c = threadIdx.x;
-    for (int i = 0; i < d; ++i) {
-      double s = Bm[(size_t)i * d + c];
-      for (int j = 0; j < i; ++j) s -= Gs[i * ld + j] * Bm[(size_t)j * d + c];
-      Bm[(size_t)i * d + c] = s / Gs[i * ld + i];
+  constexpr int kTq = 8, kMaxPer = 128 / kTq;
+  const int c = threadIdx.x / kTq, q = threadIdx.x % kTq;
+  const int per = d / kTq;                                   // d = 64 or 128
+  if (c < d) {
+    double y[kMaxPer];
+#pragma unroll
+    for (int t = 0; t < kMaxPer; ++t) y[t] = t < per ? Bm[(size_t)(q + kTq * t) * d + c] : 0.0;
+    for (int i = 0; i < d; ++i) {                            // forward: y_i = (b_i - sum_{j<i} L_ij y_j) / L_ii
+      double s = 0.0;
+#pragma unroll
+      for (int t = 0; t < kMaxPer; ++t) {
+        const int j = q + kTq * t;
+        if (t < per && j < i) s += Gs[i * ld + j] * y[t];
+      }
+#pragma unroll
+      for (int o = 1; o < kTq; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const double inv = dinv[i];
+#pragma unroll
+      for (int t = 0; t < kMaxPer; ++t)
+        if (q + kTq * t == i) y[t] = (y[t] - s) * inv;
     }
-    for (int i = d - 1; i >= 0; --i) {
-      double s = Bm[(size_t)i * d + c];
-      for (int j = i + 1; j < d; ++j) s -= Gs[j * ld + i] * Bm[(size_t)j * d + c];
-      Bm[(size_t)i * d + c] = s / Gs[i * ld + i];
+    for (int i = d - 1; i >= 0; --i) {                       // backward: b_i = (y_i - sum_{j>i} L_ji b_j) / L_ii
+      double s = 0.0;
+#pragma unroll
+      for (int t = 0; t < kMaxPer; ++t) {
+        const int j = q + kTq * t;
+        if (t < per && j > i) s += Gs[j * ld + i] * y[t];
+      }
+#pragma unroll
+      for (int o = 1; o < kTq; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const double inv = dinv[i];
+#pragma unroll
+      for (int t = 0; t < kMaxPer; ++t)
+        if (q + kTq * t == i) y[t] = (y[t] - s) * inv;
     }
+#pragma unroll
+    for (int t = 0; t < kMaxPer; ++t)
+      if (t < per) Bm[(size_t)(q + kTq * t) * d + c] = y[t];
   }
 }
 
@@ -170,13 +212,15 @@ __global__ void __launch_bounds__(256) k_fit_compose(FitArgs a, int r) {
     for (int k = 0; k < d; ++k) s += Bm[(size_t)i * d + k] * (double)Psi[k * r + t];
     T[e] = s;
   }
+  __shared__ double rs_x[128];             // 1 / s_x
+  for (int i = threadIdx.x; i < d; i += 256) rs_x[i] = 1.0 / sc[L.s_x + i];
   __syncthreads();
   double* Ad = sc + L.G;                   // G is no longer needed
   for (int e = threadIdx.x; e < d * d; e += 256) {
     const int i = e / d, j = e % d;
     double s = 0.0;
     for (int t = 0; t < r; ++t) s += T[i * r + t] * (double)Psi[j * r + t];
-    s /= sc[L.s_x + i];
+    s *= rs_x[i];
     Ad[e] = s;
     A[e] = (float)s;
   }
