@@ -2,7 +2,8 @@
 // standardisation, weighted ridge normal equations solved by Cholesky, the
 // probe-residual output subspace, and the composed affine map
 //   R_hat_i = c + x_i A,  A = diag(1/s_x) B_lambda Psi_r Psi_r^T,  c = mu_R - mu_x A,
-// which is algebraically Eq. 9.  All arithmetic is float64; one CTA per head.
+// which is algebraically Eq. 9.  Standardisation and composition are float64; the Gram matrices and the Cholesky
+// solve are float64 for float32 tensors and float32 for 16-bit tensors; one CTA per head.
 #include "kernels.cuh"
 
 namespace spr {
@@ -66,35 +67,38 @@ __global__ void __launch_bounds__(256) k_fit_prepare(FitArgs a) {
   for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = cnt * (double)w[p] / sw;
 }
 
-// blockIdx.x selects G = Xb^T W Xb + lam I, B(rhs) = Xb^T W Rb, S = Rb^T W Rb
+// blockIdx.x selects G = Xb^T W Xb + lam I, B(rhs) = Xb^T W Rb, S = Rb^T W Rb.
+// T = float for 16-bit tensors (the float64 pipe of this part is narrow: a float64 Gram is bound by it), double otherwise.
+template <typename T>
 __global__ void __launch_bounds__(256) k_fit_gram(FitArgs a) {
-  extern __shared__ double sm_gram[];      // [2][32][d] row chunks of the left and right factor
+  extern __shared__ unsigned char sm_gram_raw[];   // [2][32][d] row chunks of the left and right factor
+  T* sm_gram = reinterpret_cast<T*>(sm_gram_raw);
   const int bh = blockIdx.y, which = blockIdx.x, M = a.M, d = a.d;
   const FitLayout L(M, d);
   double* sc = a.scratch + (size_t)bh * L.total;
   const double* Lm = sc + (which == 2 ? L.Rb : L.Xb);
   const double* Rm = sc + (which == 0 ? L.Xb : L.Rb);
   double* out = sc + (which == 0 ? L.G : which == 1 ? L.B : L.S);
-  double* ls = sm_gram;
-  double* rs = sm_gram + 32 * d;
+  T* ls = sm_gram;
+  T* rs = sm_gram + 32 * d;
   const int per = d * d / 256;             // entries per thread (d = 64 or 128)
-  double acc[64];
+  T acc[64];
 #pragma unroll
-  for (int e = 0; e < 64; ++e) acc[e] = 0.0;
+  for (int e = 0; e < 64; ++e) acc[e] = T(0);
   for (int p0 = 0; p0 < M; p0 += 32) {
     const int nr = min(32, M - p0);
     __syncthreads();
     for (int t = threadIdx.x; t < nr * d; t += 256) {
       const int p = t / d;
-      ls[t] = Lm[(size_t)(p0 + p) * d + t % d] * sc[L.wt + p0 + p];
-      rs[t] = Rm[(size_t)(p0 + p) * d + t % d];
+      ls[t] = (T)(Lm[(size_t)(p0 + p) * d + t % d] * sc[L.wt + p0 + p]);
+      rs[t] = (T)Rm[(size_t)(p0 + p) * d + t % d];
     }
     __syncthreads();
 #pragma unroll
     for (int e = 0; e < 64; ++e) {
       if (e < per) {
         const int idx = threadIdx.x + e * 256, i = idx / d, j = idx % d;
-        double s = acc[e];
+        T s = acc[e];
         for (int p = 0; p < nr; ++p) s += ls[p * d + i] * rs[p * d + j];
         acc[e] = s;
       }
@@ -104,40 +108,42 @@ __global__ void __launch_bounds__(256) k_fit_gram(FitArgs a) {
   for (int e = 0; e < 64; ++e) {
     if (e < per) {
       const int idx = threadIdx.x + e * 256, i = idx / d, j = idx % d;
-      out[idx] = acc[e] + ((which == 0 && i == j) ? (double)a.lambda : 0.0);
+      out[idx] = (double)acc[e] + ((which == 0 && i == j) ? (double)a.lambda : 0.0);
     }
   }
 }
 
-// Cholesky G = L L^T in shared memory, then L Y = RHS and L^T B = Y column by column.
+// Cholesky G = L L^T in shared memory, then L Y = RHS and L^T B = Y.  T as in k_fit_gram.
+template <typename T>
 __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
-  extern __shared__ double Gs[];           // [d][d+1]
+  extern __shared__ unsigned char Gs_raw[];  // [d][d+1]
+  T* Gs = reinterpret_cast<T*>(Gs_raw);
   const int bh = blockIdx.x, d = a.d, ld = d + 1;
   const FitLayout L(a.M, d);
   double* sc = a.scratch + (size_t)bh * L.total;
   __shared__ int bad;
-  if (threadIdx.x == 0) bad = sc[L.flag] != 0.0;
-  for (int e = threadIdx.x; e < d * d; e += blockDim.x) Gs[(e / d) * ld + e % d] = sc[L.G + e];
-  __syncthreads();
-  // (float64 square roots and divisions are expensive on this part: one thread forms 1/sqrt(pivot), and the
+  // (square roots and divisions are expensive in float64 on this part: one thread forms 1/sqrt(pivot), and the
   // reciprocals of the diagonal are kept for the triangular solves)
-  __shared__ double s_inv;
-  __shared__ double dinv[128];
+  __shared__ T s_inv;
+  __shared__ T dinv[128];
+  if (threadIdx.x == 0) bad = sc[L.flag] != 0.0;
+  for (int e = threadIdx.x; e < d * d; e += blockDim.x) Gs[(e / d) * ld + e % d] = (T)sc[L.G + e];
+  __syncthreads();
   for (int k = 0; k < d; ++k) {
     if (threadIdx.x == 0) {
-      const double piv = Gs[k * ld + k];
-      if (!(piv > 0.0)) bad = 1;
-      else { s_inv = 1.0 / sqrt(piv); dinv[k] = s_inv; }       // 1 / L_kk
+      const T piv = Gs[k * ld + k];
+      if (!(piv > T(0))) bad = 1;
+      else { s_inv = T(1) / sqrt(piv); dinv[k] = s_inv; }       // 1 / L_kk
     }
     __syncthreads();
     if (bad) break;                                               // uniform
-    const double inv = s_inv;
+    const T inv = s_inv;
     for (int i = k + threadIdx.x; i < d; i += blockDim.x) Gs[i * ld + k] *= inv;   // includes the diagonal: L_kk = sqrt(piv)
     __syncthreads();
-    const int n = d - k - 1;
-    for (int e = threadIdx.x; e < n * n; e += blockDim.x) {
-      const int i = k + 1 + e / n, j = k + 1 + e % n;
-      if (j <= i) Gs[i * ld + j] -= Gs[i * ld + k] * Gs[j * ld + k];
+    // trailing update of the lower triangle: eight threads per row, columns k+1+q, k+1+q+8, ... up to the diagonal
+    for (int i = k + 1 + (int)(threadIdx.x >> 3); i < d; i += (int)(blockDim.x >> 3)) {
+      const T lik = Gs[i * ld + k];
+      for (int j = k + 1 + (int)(threadIdx.x & 7); j <= i; j += 8) Gs[i * ld + j] -= lik * Gs[j * ld + k];
     }
     __syncthreads();
   }
@@ -146,19 +152,19 @@ __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
     if (threadIdx.x == 0) { sc[L.flag] = 1.0; set_error(a.err, SPARSEPR_ERR_NUMERIC); }
     return;
   }
-  // Triangular solves L Y = RHS, L^T B = Y: eight threads per right-hand-side column.  Thread (c, q) keeps the
-  // entries i = q, q + 8, ... of its column in registers; row i of the solve is a dot product over the entries
-  // already known, split over the eight threads and added up by shuffles (fixed order).
+  // Triangular solves: eight threads per right-hand-side column.  Thread (c, q) keeps the entries i = q, q + 8, ...
+  // of its column in registers; row i of the solve is a dot product over the entries already known, split over the
+  // eight threads and added up by shuffles (fixed order).
   double* Bm = sc + L.B;
   constexpr int kTq = 8, kMaxPer = 128 / kTq;
   const int c = threadIdx.x / kTq, q = threadIdx.x % kTq;
   const int per = d / kTq;                                   // d = 64 or 128
   if (c < d) {
-    double y[kMaxPer];
+    T y[kMaxPer];
 #pragma unroll
-    for (int t = 0; t < kMaxPer; ++t) y[t] = t < per ? Bm[(size_t)(q + kTq * t) * d + c] : 0.0;
+    for (int t = 0; t < kMaxPer; ++t) y[t] = t < per ? (T)Bm[(size_t)(q + kTq * t) * d + c] : T(0);
     for (int i = 0; i < d; ++i) {                            // forward: y_i = (b_i - sum_{j<i} L_ij y_j) / L_ii
-      double s = 0.0;
+      T s = T(0);
 #pragma unroll
       for (int t = 0; t < kMaxPer; ++t) {
         const int j = q + kTq * t;
@@ -166,13 +172,13 @@ __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
       }
 #pragma unroll
       for (int o = 1; o < kTq; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      const double inv = dinv[i];
+      const T inv = dinv[i];
 #pragma unroll
       for (int t = 0; t < kMaxPer; ++t)
         if (q + kTq * t == i) y[t] = (y[t] - s) * inv;
     }
     for (int i = d - 1; i >= 0; --i) {                       // backward: b_i = (y_i - sum_{j>i} L_ji b_j) / L_ii
-      double s = 0.0;
+      T s = T(0);
 #pragma unroll
       for (int t = 0; t < kMaxPer; ++t) {
         const int j = q + kTq * t;
@@ -180,14 +186,14 @@ __global__ void __launch_bounds__(1024) k_fit_solve(FitArgs a) {
       }
 #pragma unroll
       for (int o = 1; o < kTq; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      const double inv = dinv[i];
+      const T inv = dinv[i];
 #pragma unroll
       for (int t = 0; t < kMaxPer; ++t)
         if (q + kTq * t == i) y[t] = (y[t] - s) * inv;
     }
 #pragma unroll
     for (int t = 0; t < kMaxPer; ++t)
-      if (t < per) Bm[(size_t)(q + kTq * t) * d + c] = y[t];
+      if (t < per) Bm[(size_t)(q + kTq * t) * d + c] = (double)y[t];
   }
 }
 
@@ -233,9 +239,11 @@ __global__ void __launch_bounds__(256) k_fit_compose(FitArgs a, int r) {
 }
 
 cudaError_t init_fit() {
-  cudaError_t e = cudaFuncSetAttribute(k_fit_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 8);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_fit_gram, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 32 * 128 * 8);
+  cudaError_t e = cudaFuncSetAttribute(k_fit_solve<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 8);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_fit_solve<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_fit_gram<double>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 32 * 128 * 8);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_fit_gram<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 32 * 128 * 4);
+  return e;
 }
 
 void launch_fit(const FitArgs& a, cudaStream_t st) {
@@ -243,8 +251,13 @@ void launch_fit(const FitArgs& a, cudaStream_t st) {
   const int r = min(a.r_out, min(a.M, d));
   const FitLayout L(a.M, d);
   k_fit_prepare<<<a.BH, 256, 0, st>>>(a);
-  k_fit_gram<<<dim3(3, a.BH), 256, (size_t)2 * 32 * d * 8, st>>>(a);
-  k_fit_solve<<<a.BH, 1024, (size_t)d * (d + 1) * 8, st>>>(a);
+  if (a.precise) {
+    k_fit_gram<double><<<dim3(3, a.BH), 256, (size_t)2 * 32 * d * 8, st>>>(a);
+    k_fit_solve<double><<<a.BH, 1024, (size_t)d * (d + 1) * 8, st>>>(a);
+  } else {
+    k_fit_gram<float><<<dim3(3, a.BH), 256, (size_t)2 * 32 * d * 4, st>>>(a);
+    k_fit_solve<float><<<a.BH, 1024, (size_t)d * (d + 1) * 4, st>>>(a);
+  }
   // Psi_r: leading eigenvectors of S = Rb^T W Rb, i.e. right singular vectors of W^(1/2) Rb.
   launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, st);
   k_fit_compose<<<a.BH, 256, 0, st>>>(a, r);
