@@ -83,6 +83,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   const int my_tiles = max(0, min(per_cta, row_tiles - tile0));
   const int n_chunks = prm.n_chunks;
   const int steps = my_tiles * n_chunks;
+  const int n_pairs = (my_tiles + 1) / 2;
   if (tid == 0) {
     for (int i = 0; i < 12; ++i) mbar_init(bar(i), (i == ACC_EMPTY || i == ACC_EMPTY + 1) ? 128 : 1);
     misc[1] = 0;
@@ -98,11 +99,19 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   if (warp == 4) {
     // =========================== TMA producer ============================================
     if (lane == 0) {
-      for (int q = 0; q < steps; ++q) {
-        const int tl = q / n_chunks, ch = q % n_chunks;
-        if (n_chunks > 1 || q == 0) {
-          const int ms = n_chunks > 1 ? (q & 1) : 0;
-          if (n_chunks > 1 && !mbar_wait(bar(MU_EMPTY + ms), ((q >> 1) & 1) ^ 1, abort_flag)) break;
+      // Step order: the row tiles are taken in pairs, and inside a pair the centroid chunks are interleaved
+      // (tile 0 chunk 0, tile 1 chunk 0, tile 0 chunk 1, ...): score buffer b then only ever holds tiles of parity b,
+      // i.e. belongs to one epilogue group, whose waits follow the buffer's phases in order.  (With the chunks of a
+      // tile back to back both groups would share both buffers, and a group waiting for a phase that lies two ahead
+      // of the barrier's current one takes the parity test for passed.)  v counts the steps that exist.
+      int v = 0;
+      for (int sidx = 0; sidx < n_pairs * 2 * n_chunks; ++sidx) {
+        const int r2 = sidx % (2 * n_chunks);
+        const int tl = 2 * (sidx / (2 * n_chunks)) + (r2 & 1), ch = r2 >> 1;
+        if (tl >= my_tiles) continue;
+        if (n_chunks > 1 || v == 0) {
+          const int ms = n_chunks > 1 ? (v & 1) : 0;
+          if (n_chunks > 1 && !mbar_wait(bar(MU_EMPTY + ms), ((v >> 1) & 1) ^ 1, abort_flag)) break;
           mbar_expect_tx(bar(MU_FULL + ms), 2 * kMuBytes);
           tma_load_4d(base + KmSmem::mu + ms * 2 * kMuBytes, &mapMh, bar(MU_FULL + ms), 0, ch * kKmChunk, bh, 0);
           tma_load_4d(base + KmSmem::mu + ms * 2 * kMuBytes + kMuBytes, &mapMl, bar(MU_FULL + ms), 0, ch * kKmChunk, bh, 0);
@@ -115,6 +124,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes, &mapXh, bar(X_FULL + xs), 0, row0, bh, 0);
           tma_load_4d(base + KmSmem::x + xs * 2 * kXBytes + kXBytes, &mapXl, bar(X_FULL + xs), 0, row0, bh, 0);
         }
+        ++v;
       }
     }
   } else if (warp == 5) {
@@ -128,16 +138,20 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
 #else
 #define SPR_KM(v)
 #endif
-      for (int q = 0; q < steps; ++q) {
-        const int tl = q / n_chunks, ch = q % n_chunks;
-        const int xs = tl & 1, ms = n_chunks > 1 ? (q & 1) : 0;
+      int v = 0;                                               // same step order as the producer
+      for (int sidx = 0; sidx < n_pairs * 2 * n_chunks; ++sidx) {
+        const int r2 = sidx % (2 * n_chunks);
+        const int tl = 2 * (sidx / (2 * n_chunks)) + (r2 & 1), ch = r2 >> 1;
+        if (tl >= my_tiles) continue;
+        const int xs = tl & 1, ms = n_chunks > 1 ? (v & 1) : 0;
+        const int ab = tl & 1, au = (tl >> 1) * n_chunks + ch;   // score buffer and how often it has been used before
         if (ch == 0 && !mbar_wait(bar(X_FULL + xs), (tl >> 1) & 1, abort_flag)) break;
         SPR_KM(mX);
-        if ((n_chunks > 1 || q == 0) && !mbar_wait(bar(MU_FULL + ms), n_chunks > 1 ? ((q >> 1) & 1) : 0, abort_flag)) break;
-        if (!mbar_wait(bar(ACC_EMPTY + (q & 1)), ((q >> 1) & 1) ^ 1, abort_flag)) break;
+        if ((n_chunks > 1 || v == 0) && !mbar_wait(bar(MU_FULL + ms), n_chunks > 1 ? ((v >> 1) & 1) : 0, abort_flag)) break;
+        if (!mbar_wait(bar(ACC_EMPTY + ab), (au & 1) ^ 1, abort_flag)) break;
         SPR_KM(mA);
         tc_fence_after();
-        const uint32_t d = tmem + (uint32_t)(q & 1) * 256u;
+        const uint32_t d = tmem + (uint32_t)ab * 256u;
         const uint32_t xh = base + KmSmem::x + xs * 2 * kXBytes, xl = xh + kXBytes;
         const uint32_t mh = base + KmSmem::mu + ms * 2 * kMuBytes, ml = mh + kMuBytes;
         uint32_t acc = 0;
@@ -146,8 +160,9 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         for (int kk = 0; kk < ksteps; ++kk) umma_bf16(d, smem_desc(xl + kk * 32, 16), smem_desc(mh + kk * 32, 16), idesc, 1);
         if (ch == n_chunks - 1) umma_commit(bar(X_EMPTY + xs));
         if (n_chunks > 1) umma_commit(bar(MU_EMPTY + ms));
-        umma_commit(bar(ACC_FULL + (q & 1)));
+        umma_commit(bar(ACC_FULL + ab));
         SPR_KM(mI);
+        ++v;
       }
 #ifdef SPR_KM_TIMING
       if (blockIdx.x == 1 && blockIdx.y == 0 && steps > 0)
@@ -200,8 +215,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       }
       SPR_KE(eP);
       for (int ch = 0; ch < n_chunks; ++ch) {
-        const int q = tl * n_chunks + ch;
-        ok = __all_sync(FULL, ok && mbar_wait(bar(ACC_FULL + (q & 1)), (q >> 1) & 1, abort_flag));
+        const int ab = tl & 1, au = (tl >> 1) * n_chunks + ch;   // this group's score buffer and its phase
+        ok = __all_sync(FULL, ok && mbar_wait(bar(ACC_FULL + ab), au & 1, abort_flag));
         SPR_KE(eW);
         if (!ok) continue;
         tc_fence_after();
@@ -211,7 +226,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         for (int g = 0; g < kKmChunk / 32; ++g) {
           if (g * 32 >= nvalid) break;                       // uniform: whole column groups beyond C
           float t[32];
-          tmem_ld32(tmem + lane_addr + (uint32_t)(q & 1) * 256u + g * 32, t);
+          tmem_ld32(tmem + lane_addr + (uint32_t)ab * 256u + g * 32, t);
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const int c = c0 + g * 32 + j;
@@ -227,7 +242,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           }
         }
         tc_fence_before();
-        mbar_arrive(bar(ACC_EMPTY + (q & 1)));
+        mbar_arrive(bar(ACC_EMPTY + ab));
         SPR_KE(eA);
       }
       // decide, or hand the row to the exact recheck

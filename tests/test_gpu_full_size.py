@@ -66,3 +66,48 @@ def test_full_size_480p_sampled_rows():
         got, got_sp = to_np(O[0, i])[rows], to_np(Osp[0, i])[rows]
         assert np.abs(got_sp - O_sp).max() <= 2e-2 and orc.rel_l2(got_sp, O_sp) <= 1e-2
         assert np.abs(got - O_hat).max() <= 2e-2 and orc.rel_l2(got, O_hat) <= 1e-2
+
+
+def test_more_than_256_groups_sampled_rows():
+    """world-model-like at full length (N = 49152, 384 groups per side): the k-means assignment streams the
+    centroids in two chunks of 256 per row tile and the attention kernels see more groups than one chunk holds.
+    Two heads; properties on both, sampled rows of the GPU's own plan against the oracle on the first."""
+    wl = W.WORLD.scaled(H=2)
+    heads = [0, 1]
+    host, (Qd, Kd, Vd) = heads_to_device(wl, heads)
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale)
+    plan = B.sparsepr_plan(Qd, Kd, Vd, **kw)
+    O, Osp = B.sparsepr_attend(plan, Qd, Kd, Vd, return_sparse=True)
+    st = B.sparsepr_plan_stats(plan)
+    exp = B.sparsepr_plan_export(plan)
+    assert st["device_error"] == 0
+    assert torch.isfinite(O).all()
+    prm = orc.default_params(**kw)
+    C = -(-wl.N // wl.block)
+    assert C > 256
+    budget = orc.pair_budget(wl.density, wl.N, wl.N, wl.n_probe)
+    rng = np.random.default_rng(11)
+    for i in heads:
+        aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
+        ptr, idx = exp["route_ptr"][i], exp["route_idx"][i]
+        n_q, n_k = np.bincount(aQ, minlength=C), np.bincount(aK, minlength=C)
+        assert aK.min() >= 0 and aK.max() < C and aQ.min() >= 0 and aQ.max() < C
+        assert (n_k > 0).sum() > 256 and (n_q > 0).sum() > 256        # groups of both chunks are in use
+        p0, _, o0 = orc.group_permutation(aK, C)
+        assert np.array_equal(exp["kv_perm"][i], p0) and np.array_equal(exp["kv_off"][i], o0)
+        p0, _, o0 = orc.group_permutation(aQ, C)
+        assert np.array_equal(exp["q_perm"][i], p0) and np.array_equal(exp["q_off"][i], o0)
+        pairs = orc.routed_pairs(n_q, n_k, ptr, idx[:ptr[-1]])
+        assert pairs == exp["routed_pairs"][i] and pairs <= budget
+        assert len(set(exp["probe_idx"][i].tolist())) == wl.n_probe
+    Q, K, V = host[0]
+    P = exp["probe_idx"][0]
+    gplan = dict(scale=wl.softmax_scale, a_Q=exp["q_assign"][0], a_K=exp["kv_assign"][0], route_ptr=exp["route_ptr"][0],
+                 route_idx=exp["route_idx"][0][:exp["route_ptr"][0][-1]], probe_idx=P, M=len(P),
+                 probe_w=exp["probe_w"][0].astype(np.float64))
+    rows = np.array(sorted(set(list(rng.choice(wl.N, 24, replace=False)) + [int(p) for p in P[:4]])), dtype=np.int64)
+    O_hat, O_sp, _ = orc.attend_head(Q, K, V, gplan, prm, rows=rows)
+    got, got_sp = to_np(O[0, 0])[rows], to_np(Osp[0, 0])[rows]
+    assert np.abs(got_sp - O_sp).max() <= 2e-2 and orc.rel_l2(got_sp, O_sp) <= 1e-2
+    assert np.abs(got - O_hat).max() <= 2e-2 and orc.rel_l2(got, O_hat) <= 1e-2
