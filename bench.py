@@ -309,7 +309,7 @@ def main():
                     # DRAM read + write of one k_attention_tc launch: 29.6 MB per head from the ncu capture summarised
                     # in profiles/k_attention_tc_480p-like_6heads.md (177.8 MB at 6 heads of this N; heads are
                     # independent CTAs over disjoint memory, so traffic scales with the head count)
-                    "traffic": (29.55e6 * wl.H if wl.name == "video-dit-480p-like" else None), "traffic_unit": "bytes",
+                    "traffic": (30.04e6 * wl.H if wl.name == "video-dit-480p-like" else None), "traffic_unit": "bytes",
                     "algorithmic_bytes": 4.0 * wl.H * wl.N * wl.d * 2,
                     "peak_source": peaks["source"] + " cuBLAS bf16, sustained",
                     "issued_tflops": issued / (attn_ms * 1e-3) / 1e12,
