@@ -452,9 +452,18 @@ __global__ void __launch_bounds__(256) k_probe_merge(const float* __restrict__ p
   for (int s = 0; s < n_split; ++s) {
     const float* p = partial + ((((i64)bh * n_split + s) * M + r) * 2) * (D + 2);
     const float wS = p[0] == -INFINITY ? 0.f : exp2f(p[0] - mS), wU = p[D + 2] == -INFINITY ? 0.f : exp2f(p[D + 2] - mU);
-    lS += p[1] * wS; lU += p[D + 3] * wU;
+    // a state without any key (empty key slice, or no retained / omitted key inside it) has weight 0 and its
+    // numerator may never have been written: it is skipped, not multiplied by 0
+    if (wS != 0.f) {
+      lS += p[1] * wS;
 #pragma unroll
-    for (int c = 0; c < PL; ++c) { nS[c] += p[2 + lane + 32 * c] * wS; nU[c] += p[D + 4 + lane + 32 * c] * wU; }
+      for (int c = 0; c < PL; ++c) nS[c] += p[2 + lane + 32 * c] * wS;
+    }
+    if (wU != 0.f) {
+      lU += p[D + 3] * wU;
+#pragma unroll
+      for (int c = 0; c < PL; ++c) nU[c] += p[D + 4 + lane + 32 * c] * wU;
+    }
   }
   const float mD = fmaxf(mS, mU);
   const float eS = mS == -INFINITY ? 0.f : exp2f(mS - mD), eU = mU == -INFINITY ? 0.f : exp2f(mU - mD);

@@ -43,6 +43,8 @@ CASES = [
     ("720p-like-bf16", W.VIDEO_720P.scaled(grid=(2, 45, 80), H=2, n_probe=64), dict()),
     ("480p-like-bf16-sparser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.12), dict()),
     ("480p-like-bf16-denser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.35), dict(r_out=128)),
+    # 38 key tiles over 9 probe slices of 5 tiles: the last slice is empty and must not contribute
+    ("480p-like-bf16-empty-probe-slice", W.VIDEO_480P.scaled(grid=(3, 30, 53), H=2, n_probe=64), dict()),
 ]
 
 
@@ -50,6 +52,9 @@ CASES = [
 def test_attend_on_injected_oracle_plan(name, wl, extra):
     heads = list(range(min(wl.H, 2)))
     host, (Qd, Kd, Vd) = heads_to_device(wl, heads)
+    # the workspaces come from the caching allocator: leave NaN behind so that anything read before it is written shows
+    junk = torch.full((64 << 20,), float("nan"), device="cuda")
+    del junk
     kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
               softmax_scale=wl.softmax_scale, **extra)
     prm = orc.default_params(**kw)
