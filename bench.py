@@ -94,12 +94,14 @@ def launches_per_call(T, fitted, tensor_path):
         kmeans = 2 + 1 + 2 * T + (T - 1)
     else:                # init, first norms, T assignments, T-1 updates
         kmeans = 2 + T + (T - 1)
-    plan = 2 * (2 + 1 + kmeans + 2) + 2 + 2 + 3      # per side: Gram+eig, projection, k-means, sort+means; probes; route; tile offsets + remainder rows
+    # per side: Gram, eigen-solver + its marked-matrix fallback, projection (+ split of the feature map), k-means,
+    # sort + means; then probes; route; tile offsets + remainder rows
+    plan = 2 * (3 + (2 if tensor_path else 1) + kmeans + 2) + 2 + 2 + 3
     if not fitted:
         plan -= 2
     attend = 3 + 1 + (1 if tensor_path else 0)       # gathers, attention (+ the packed-remainder kernel)
     if fitted:
-        attend += (3 if tensor_path else 2) + 5 + 1  # probe rows (+gather) + merge, fit, probe write
+        attend += (3 if tensor_path else 2) + 6 + 1  # probe rows (+gather) + merge, fit (eigen-solver: two launches), probe write
         attend += 2 if tensor_path else 0            # transposed correction matrix, correction pass
     return plan + attend
 
