@@ -14,7 +14,7 @@
 //   warp  8    K producer: streams the K/V groups that some row of the tile routes to, as one sequence of 16-row
 //              boxes (tiles of 128 keys, every box inside one group), and publishes the group of every box;
 //   warp  10   V producer
-//   warp  9    tcgen05.mma issuer; owns the TMEM allocation
+//   warp  9    issues Q K^T (one thread); owns the TMEM allocation;  warp 11 issues P V (one thread)
 // TMEM: S_0 [0,128), S_1 [128,256), P [256,320), O [320,448), Q [448,512); both products take their A
 // operand from tensor memory.  Reference maxima move lazily (growth beyond 2^8), as in the 128-row kernel.
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.

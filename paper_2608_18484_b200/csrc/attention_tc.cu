@@ -5,15 +5,22 @@
 //   warps 0-7  softmax: warps w and w+4 share the 32 rows of TMEM quadrant w and split the
 //              128 scores of a row in two halves (keys 0-63 / 64-127 of the tile)
 //   warp  8    TMA producer of Q and the key tiles (+ tile meta ring)
-//   warp  9    tcgen05.mma issuer; owns the TMEM allocation
+//   warp  9    issues Q K^T (one thread); owns the TMEM allocation
 //   warp  10   TMA producer of the value tiles
-// The routed keys/values arrive as one concatenated sequence in 16-row boxes (tiles of 128
-// keys, only range ends are ragged).  Data path per key tile i:
-//   S_b = Q K_i^T        tcgen05.mma, smem x smem -> TMEM (fp32), two score buffers b = i mod 2, so
-//                        the product of tile i+1 runs while tile i is in the softmax
-//   P   = exp2(.)        softmax threads: tcgen05.ld their half row of S_b, row maximum (the two
-//                        halves meet through shared memory), bf16 P to its own TMEM columns
+//   warp  11   issues P V (one thread)
+// The routed keys/values arrive as one concatenated sequence of 16-row boxes (tiles of 128 keys, only
+// range ends are ragged); consecutive boxes of one key range are fetched by one copy per set bit of their
+// number (tensor maps with 16-, 32-, 64- and 128-row boxes).  Data path per key tile i:
+//   S_b = Q K_i^T        tcgen05.mma, smem x smem -> TMEM (fp32), two score buffers b = i mod 2; a buffer is
+//                        released as soon as the softmax threads hold its scores in registers, so the product
+//                        runs two tiles ahead of the softmax
+//   P_b = exp2(.)        softmax threads: tcgen05.ld their half row of S_b, row maximum (the two halves meet
+//                        through shared memory), bf16 P to TMEM columns of its own (two buffers as well);
+//                        3 of every 8 exponentials are a cubic on the FMA pipe, the others use ex2.approx
 //   O  += P V_i          tcgen05.mma with the A operand read from TMEM; O stays in TMEM
+// A single issuing thread shares its warp scheduler with two softmax warps that rarely leave it an issue slot:
+// this is why the two products have a thread each on different schedulers, why the producers issue few, large
+// copies, and why the barrier polls of a tile are grouped.
 // The reference maximum of a row moves only when it grows by more than 2^8 (then O is rescaled).
 // Epilogue: O / l, store at the original token index (inverse permutation).  The residual
 // correction of Eq. 9 is a pass of its own (correction_tc.cu) so that the fit can overlap this kernel.
