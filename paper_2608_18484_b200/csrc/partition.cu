@@ -436,8 +436,10 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_group_sort(const int* __res
   const int L = (((N + kSortWarps - 1) / kSortWarps) + 31) / 32 * 32;
   const int s0 = w * L, s1 = min(N, s0 + L);
   for (int i = s0 + lane; i < s1; i += 32) {
-    const int key = a[i];
-    if (key < 0 || key >= C) { set_error(err, SPARSEPR_ERR_INVALID_ARG); continue; }
+    int key = a[i];
+    // an id out of range (only possible after an earlier stage gave up) is recorded and counted as group 0, so that
+    // the permutation stays a permutation and nothing downstream indexes out of bounds
+    if (key < 0 || key >= C) { set_error(err, SPARSEPR_ERR_INVALID_ARG); key = 0; }
     atomicAdd(&hist[w * C + key], 1);
   }
   __syncthreads();
@@ -458,7 +460,7 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_group_sort(const int* __res
   for (int i0 = s0; i0 < s1; i0 += 32) {
     const int i = i0 + lane;
     int key = i < s1 ? a[i] : -1;
-    if (key >= C) key = -1;
+    if (i < s1 && (key < 0 || key >= C)) key = 0;
     const unsigned same = __match_any_sync(0xffffffffu, key);
     const int rank = __popc(same & ((1u << lane) - 1));
     int pos = -1;
