@@ -149,7 +149,11 @@ size_t sparsepr_attend_workspace_bytes(const sparsepr_shape_t* shape, const spar
  * probe set and routes of every head from Q and K (DEVICE, read only; V is not
  * read -- values never enter the partition features -- and may be NULL).
  * `workspace` is DEVICE memory of at least sparsepr_plan_workspace_bytes, 256-byte
- * aligned; the plan lives in it.  *out receives a HOST handle. */
+ * aligned; the plan lives in it.  *out receives a HOST handle.  The probe selection may
+ * still be running on a stream of the plan's own when the call returns: sparsepr_attend
+ * orders its work behind it, sparsepr_plan_stats / _export / _destroy wait for it, so the
+ * workspace may be released once sparsepr_plan_destroy has returned and the work queued on
+ * `cuda_stream` is complete. */
 sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
                                 const void* Q, const void* K, const void* V,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream,
