@@ -121,7 +121,8 @@ typedef struct {
  * *_PERMUTE = counting sort and group means; QUERY_METRIC = centroid Gram and its
  * eigen-decomposition; PROBE_SELECT; ROUTE = cell scores and selection.  Attend:
  * GATHER = group-major copies of Q, K, V; PROBE_ROWS = exact and hard-drop rows of
- * the probes; FIT = ridge fit and subspace; ATTENTION = block-sparse kernel;
+ * the probes; FIT = ridge fit and subspace; ATTENTION = block-sparse kernels (the 128-row
+ * tiles and the packed group remainders, side by side on two streams);
  * CORRECTION = residual correction of Eq. 9 (zero where the block-sparse kernel applies
  * it in its epilogue); PROBE_WRITE.  DENSE = the dense entry point.  A call without a
  * profile runs PROBE_SELECT beside ROUTE and PROBE_ROWS + FIT beside ATTENTION on a second

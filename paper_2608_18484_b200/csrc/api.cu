@@ -552,21 +552,14 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   }
   if (tensor) {
     aa.tile_off = p->tile_off128;
-    // the packed remainder tiles are few and long, the 128-row tiles many and short: without a profile they share
-    // the GPU instead of running one after the other
-    cudaStream_t rs = st;
-    if (prof == nullptr) {
-      if (!overlap) cudaEventRecord(p->ev_fork, st);              // (with the probes' overlap the event is recorded already)
-      cudaStreamWaitEvent(p->side2, p->ev_fork, 0);
-      rs = p->side2;
-    }
-    if (prof == nullptr && !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, rs)) return SPARSEPR_ERR_CUDA;
+    // the packed remainder tiles are few and long, the 128-row tiles many and short: they share the GPU instead of
+    // running one after the other (also in a profiled call: both belong to the ATTENTION stage)
+    if (!overlap) cudaEventRecord(p->ev_fork, st);                // (with the probes' overlap the event is recorded already)
+    cudaStreamWaitEvent(p->side2, p->ev_fork, 0);
+    if (!launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, p->side2)) return SPARSEPR_ERR_CUDA;
     if (!launch_attention_tc(aa, st)) return SPARSEPR_ERR_CUDA;
-    if (prof != nullptr && !launch_attention_packed(aa, p->rem_pos, p->rem_grp, p->rem_cnt, rs)) return SPARSEPR_ERR_CUDA;
-    if (prof == nullptr) {
-      cudaEventRecord(p->ev_join2, p->side2);
-      cudaStreamWaitEvent(st, p->ev_join2, 0);
-    }
+    cudaEventRecord(p->ev_join2, p->side2);
+    cudaStreamWaitEvent(st, p->ev_join2, 0);
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) { join_side(p, st); p->side_pending = false; }
     if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
