@@ -276,7 +276,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
     if (tcp) {
       KmeansTcArgs ka{};
       ka.BH = R.BH; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
-      ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2; ka.mumax = p->mumax;
+      ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2;
       ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
       ka.flagged = p->flagged; ka.flag_count = p->recheck + 1; ka.recheck_total = p->recheck; ka.err = p->err;
       launch_kmeans_assign_tc(ka, st);
@@ -748,7 +748,7 @@ sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const f
     launch_split_bf16(mup, R, C, r, mh, ml, nullptr, st);
     KmeansTcArgs ka{};
     ka.BH = 1; ka.N = n; ka.C = C; ka.r = r; ka.R = R; ka.xh = xh; ka.xl = xl; ka.mh = mh; ka.ml = ml;
-    ka.phi = Xp; ka.ldphi = R; ka.xnorm = xnorm; ka.mu = mup; ka.mu2 = mu2; ka.mumax = mumax; ka.assign = a;
+    ka.phi = Xp; ka.ldphi = R; ka.xnorm = xnorm; ka.mu = mup; ka.mu2 = mu2; ka.assign = a;
     ka.flagged = flagged; ka.flag_count = fx + 1; ka.recheck_total = fx + 2;
     if (!launch_kmeans_assign_tc(ka, st)) return SPARSEPR_ERR_CUDA;
   } else {

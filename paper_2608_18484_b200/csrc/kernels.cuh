@@ -41,7 +41,7 @@ struct KmeansTcArgs {
   int BH, N, C, r, R;
   const __nv_bfloat16 *xh, *xl, *mh, *ml;      // [BH][N][64], [BH][C][64] split operands
   const float* phi; int ldphi;                 // fp32 features [BH][N][ldphi]
-  const float *xnorm, *mu, *mu2, *mumax;       // [BH][N], [BH][C][R], [BH][C], [BH]
+  const float *xnorm, *mu, *mu2;               // [BH][N], [BH][C][R], [BH][C]
   int* assign;
   i64* sums; int* counts; const int* fx_shift; // null sums = assignment only
   int *flagged, *flag_count, *recheck_total, *err;

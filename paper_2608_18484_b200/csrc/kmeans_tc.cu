@@ -40,7 +40,6 @@ struct KmParams {
   const float* phi; int ldphi;          // fp32 features (for the centroid sums)
   const float* xnorm;                   // [BH][N]
   const float* mu2;                     // [BH][C]
-  const float* mumax;                   // [BH]
   int* assign;
   i64* sums; int* counts; const int* fx_shift;
   int* flagged; int* flag_count;        // rows left to the exact recheck
@@ -427,7 +426,7 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   p.N = a.N; p.C = a.C; p.r = a.r; p.R = a.R; p.n_chunks = (a.C + kKmChunk - 1) / kKmChunk;
   const int row_tiles = (a.N + 127) / 128;
   p.ctas_per_head = std::max(1, std::min(row_tiles, 148 / a.BH));
-  p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.mumax = a.mumax; p.assign = a.assign;
+  p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.assign = a.assign;
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
   cudaMemsetAsync(a.flag_count, 0, sizeof(int), st);
   k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
