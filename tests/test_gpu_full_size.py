@@ -68,12 +68,13 @@ def test_full_size_480p_sampled_rows():
         assert np.abs(got - O_hat).max() <= 2e-2 and orc.rel_l2(got, O_hat) <= 1e-2
 
 
-def test_more_than_256_groups_sampled_rows():
-    """world-model-like at full length (N = 49152, 384 groups per side): the k-means assignment streams the
-    centroids in two chunks of 256 per row tile and the attention kernels see more groups than one chunk holds.
-    Two heads; properties on both, sampled rows of the GPU's own plan against the oracle on the first."""
-    wl = W.WORLD.scaled(H=2)
-    heads = [0, 1]
+@pytest.mark.parametrize("wl", [W.WORLD.scaled(H=2), W.VIDEO_720P.scaled(H=1)], ids=["world-like", "720p-like"])
+def test_more_than_256_groups_sampled_rows(wl):
+    """world-model-like and video-dit-720p-like at full length (N = 49152 / 75600, 384 / 591 groups per side): the
+    k-means assignment streams the centroids in two / three chunks of 256 per row tile (the last one partly filled)
+    and the attention kernels see more groups than one chunk holds.  Properties on every head, sampled rows of the
+    GPU's own plan against the oracle on the first."""
+    heads = list(range(wl.H))
     host, (Qd, Kd, Vd) = heads_to_device(wl, heads)
     kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
               softmax_scale=wl.softmax_scale)
