@@ -17,17 +17,25 @@
  *   - Q, K, V, O are [B, H, N, d] tensors addressed through element strides for
  *     B, H and N; the last dimension is contiguous.  Rows must start on a
  *     16-byte boundary.  N_q = N_k = N and d_v = d.
- *   - The library never allocates or frees device memory and keeps no global
- *     state.  The caller owns all tensors and both workspaces.  A plan handle is a small
- *     host object that points into the plan workspace; it is valid until the
- *     workspace is released or sparsepr_plan_destroy is called.
+ *   - The library never allocates or frees device memory: the caller owns all
+ *     tensors and both workspaces.  A plan handle is a small host object that
+ *     points into the plan workspace; it is valid until the workspace is released
+ *     or sparsepr_plan_destroy is called.  Process-wide state is limited to what is
+ *     set up once and then reused: kernel attributes and the tensor-map encoder
+ *     (first call), a pool of auxiliary streams and events (two streams and three
+ *     events per plan alive at the same time, per device; created when the pool is
+ *     empty, returned by sparsepr_plan_destroy, never freed), the SM count per
+ *     device, and the scratch array of sparsepr_stage_assign_static.
  *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*)
  *     and is asynchronous, except the calls documented as synchronising.
  *   - Errors are return codes.  Argument errors are detected before anything
  *     is launched.  Conditions found on the device (non-finite input, a
  *     breakdown of the Cholesky factorisation, a bounded wait that ran out)
  *     are recorded in a device error word that sparsepr_plan_stats reports.
- *     No call aborts, throws or traps.
+ *     The word lives in the plan workspace and persists for the life of the plan;
+ *     once a bounded wait has run out (SPARSEPR_ERR_TIMEOUT) the tensor-core
+ *     kernels of later calls on that plan return at once, so O is undefined
+ *     whenever `device_error` is non-zero.  No call aborts, throws or traps.
  */
 #ifndef SPARSEPR_H_
 #define SPARSEPR_H_
@@ -93,6 +101,10 @@ typedef struct {
   int32_t max_kv_group, max_q_group;
   int32_t assign_rechecked_rows;   /* rows of the last k-means assignments decided by the exact recheck */
   int32_t device_error;
+  /* Lloyd passes that ran on the K/V side and on the query side (largest count over heads).  A head stops
+   * early when a pass changes no assignment: every later pass would repeat it exactly, so the result is
+   * the one of all T passes.  0 for an imported plan. */
+  int32_t kmeans_passes_kv, kmeans_passes_q;
 } sparsepr_stats_t;
 
 /* Host-side view of a plan, one entry per (batch, head) in b-major order, used
@@ -114,6 +126,17 @@ typedef struct {
   float *probe_w;
   int64_t *routed_pairs;
 } sparsepr_plan_host_t;
+
+/* Floating-point intermediates of a plan (Section 4.1, Appendix B; the router's group means and cell
+ * scores of Section 4.3), exported so that they can be compared with an independent evaluation.  Every
+ * pointer is HOST memory owned by the caller; NULL skips the field.  All float32, b-major over (batch, head):
+ *   F_K   [BH, d, r_K], F_Q [BH, d, r_Q]  feature maps (columns = scaled eigendirections; their signs are arbitrary)
+ *   phi_Q [BH, N, r_Q]                    RMS-normalised query responses (Eq. 7)
+ *   kappa [BH, C_k, d], theta [BH, C_q, d] original-space means of the K/V groups and of the query groups
+ *   score [BH, C_q, C_k]                  cell scores the router selected from */
+typedef struct {
+  float *F_K, *F_Q, *phi_Q, *kappa, *theta, *score;
+} sparsepr_plan_features_t;
 
 /* Stages of one call, in launch order, as indices into sparsepr_profile_t.ms.  Plan
  * (Section 4.1, 4.3, Algorithm A.1): KEY_METRIC = sampled-query Gram and its
@@ -192,6 +215,10 @@ sparsepr_status_t sparsepr_dense_timed(const sparsepr_shape_t* shape, float soft
 /* Synchronises the stream the plan was built on, then fills *host_out. */
 sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* plan, sparsepr_stats_t* host_out);
 sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* plan, sparsepr_plan_host_t* host_out);
+
+/* Synchronises like sparsepr_plan_export, then copies the requested intermediates.  A plan made by
+ * sparsepr_plan_import has none: SPARSEPR_ERR_UNSUPPORTED. */
+sparsepr_status_t sparsepr_plan_export_features(const sparsepr_plan_t* plan, sparsepr_plan_features_t* host_out);
 
 /* Builds a plan from host-side assignments, routes (CSR slabs as in
  * sparsepr_plan_host_t) and probes; permutations and offsets are recomputed on

@@ -46,12 +46,17 @@ class Stats(C.Structure):
                 ("rho_route", C.c_double), ("rho_exec", C.c_double), ("rho_route_min", C.c_double),
                 ("rho_route_max", C.c_double), ("nonempty_kv_groups_min", C.c_int32),
                 ("nonempty_q_groups_min", C.c_int32), ("max_kv_group", C.c_int32), ("max_q_group", C.c_int32),
-                ("assign_rechecked_rows", C.c_int32), ("device_error", C.c_int32)]
+                ("assign_rechecked_rows", C.c_int32), ("device_error", C.c_int32),
+                ("kmeans_passes_kv", C.c_int32), ("kmeans_passes_q", C.c_int32)]
 
 
 class PlanHost(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("kv_assign", "q_assign", "kv_perm", "q_perm", "kv_off", "q_off",
                                             "route_ptr", "route_idx", "probe_idx", "probe_w", "routed_pairs")]
+
+
+class PlanFeatures(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("F_K", "F_Q", "phi_Q", "kappa", "theta", "score")]
 
 
 STAGES = ["key_metric", "key_project", "key_kmeans", "key_permute", "query_metric", "query_project", "query_kmeans",
@@ -67,6 +72,7 @@ class Profile(C.Structure):
 
 EXPORTS = ["sparsepr_stage_assign_static", "sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
+           "sparsepr_plan_export_features",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
 
@@ -93,6 +99,7 @@ def lib():
         L.sparsepr_dense_timed.argtypes = L.sparsepr_dense.argtypes + [C.POINTER(Profile)]
         L.sparsepr_plan_stats.argtypes = [vp, C.POINTER(Stats)]
         L.sparsepr_plan_export.argtypes = [vp, C.POINTER(PlanHost)]
+        L.sparsepr_plan_export_features.argtypes = [vp, C.POINTER(PlanFeatures)]
         L.sparsepr_plan_import.argtypes = [C.POINTER(Shape), C.POINTER(Params), C.POINTER(PlanHost), vp, sz, vp,
                                            C.POINTER(vp)]
         L.sparsepr_plan_destroy.argtypes = [vp]
@@ -256,6 +263,20 @@ def sparsepr_plan_export(plan: Plan) -> dict:
     if plan.M == 0:
         arrs["probe_idx"] = arrs["probe_idx"][:, :0]
         arrs["probe_w"] = arrs["probe_w"][:, :0]
+    return arrs
+
+
+def sparsepr_plan_export_features(plan: Plan, fields=("F_K", "F_Q", "phi_Q", "kappa", "theta", "score")) -> dict:
+    """Copies the plan's floating-point intermediates (feature maps, query responses, group means,
+    cell scores) to host numpy arrays (synchronises)."""
+    BH, N, d = plan.BH, plan.shape.N, plan.shape.d
+    Ck, Cq = plan.groups
+    rK, rQ = min(plan.params.rK or 48, d), min(plan.params.rQ or 64, d)
+    shapes = dict(F_K=(BH, d, rK), F_Q=(BH, d, rQ), phi_Q=(BH, N, rQ), kappa=(BH, Ck, d), theta=(BH, Cq, d),
+                  score=(BH, Cq, Ck))
+    arrs = {k: np.empty(shapes[k], np.float32) for k in fields}
+    pf = PlanFeatures(**{k: v.ctypes.data for k, v in arrs.items()})
+    _check(lib().sparsepr_plan_export_features(plan.handle, C.byref(pf)), "sparsepr_plan_export_features")
     return arrs
 
 

@@ -21,7 +21,6 @@ OBJ = os.path.join(HERE, "build")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-FLAGS += os.environ.get("SPARSEPR_NVCC_FLAGS", "").split()      # e.g. -DSPR_K_STAGES=4 for tuning runs
 
 
 def sources():

@@ -10,6 +10,20 @@
 
 using namespace spr;
 
+namespace spr {
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); return 148; }
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+}  // namespace spr
+
 namespace {
 
 struct Carver {                       // bump allocator over a caller-owned workspace (or a dry run)
@@ -136,27 +150,76 @@ struct StageTimer {
 
 }  // namespace
 
-struct sparsepr_plan_s {
-  Resolved r;
-  cudaStream_t stream;
+// Auxiliary streams and events of one plan.  They are created once and recycled: a plan takes a set from a
+// per-process pool (keyed by device) and hands it back when it is destroyed, so that a steady stream of calls
+// creates nothing.  A set belongs to one plan at a time, hence concurrent calls never share an event.
+struct SideSet {
+  int device = -1;
   // second stream for work that is independent of the main chain (probe selection next to routing;
   // probe rows and fit next to the block-sparse kernel), forked and joined with the two events
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-  // third stream: the packed-remainder kernel (few long CTAs) beside the 128-row kernel (many short ones)
+  // third stream: the remainder kernel beside the 128-row kernel
   cudaStream_t side2 = nullptr;
   cudaEvent_t ev_join2 = nullptr;
+};
+namespace {
+std::mutex g_side_mu;
+std::vector<SideSet*> g_side_pool;
+
+SideSet* acquire_side_set() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_side_mu);
+    for (size_t i = 0; i < g_side_pool.size(); ++i)
+      if (g_side_pool[i]->device == dev) {
+        SideSet* s = g_side_pool[i];
+        g_side_pool.erase(g_side_pool.begin() + i);
+        return s;
+      }
+  }
+  SideSet* s = new (std::nothrow) SideSet();
+  if (!s) return nullptr;
+  s->device = dev;
+  int prio_lo = 0, prio_hi = 0;
+  cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+  if (cudaStreamCreateWithPriority(&s->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+      cudaStreamCreateWithPriority(&s->side2, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+      cudaEventCreateWithFlags(&s->ev_join2, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+    if (s->ev_join) cudaEventDestroy(s->ev_join);
+    if (s->ev_join2) cudaEventDestroy(s->ev_join2);
+    if (s->side) cudaStreamDestroy(s->side);
+    if (s->side2) cudaStreamDestroy(s->side2);
+    delete s;
+    return nullptr;
+  }
+  return s;
+}
+void release_side_set(SideSet* s) {
+  if (!s) return;
+  std::lock_guard<std::mutex> lk(g_side_mu);
+  g_side_pool.push_back(s);
+}
+}  // namespace
+
+struct sparsepr_plan_s {
+  Resolved r;
+  cudaStream_t stream;
+  SideSet* set = nullptr;
+  cudaStream_t side = nullptr, side2 = nullptr;          // aliases of the set's members
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_join2 = nullptr;
   // the probe selection of the plan call may still run on `side` when the call returns: the first attend call
   // orders it (its probe work follows on the same stream and is joined there); statistics, export and the
   // destructor wait for it themselves
   mutable bool side_pending = false;
+  bool imported = false;                                  // built by sparsepr_plan_import: no partition stages ran
   ~sparsepr_plan_s() {
     if (side && side_pending) cudaStreamSynchronize(side);
-    if (ev_fork) cudaEventDestroy(ev_fork);
-    if (ev_join) cudaEventDestroy(ev_join);
-    if (ev_join2) cudaEventDestroy(ev_join2);
-    if (side) cudaStreamDestroy(side);
-    if (side2) cudaStreamDestroy(side2);
+    release_side_set(set);
   }
   // device state (all inside the caller's plan workspace)
   int* err; int* recheck;
@@ -171,6 +234,7 @@ struct sparsepr_plan_s {
   double* probe_dist; int* probe_idx; float* probe_w;
   __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged;
   int *rem_pos, *rem_grp, *rem_cnt;      // rows of the short group remainders (packed attention tiles)
+  int* km_changed;                       // [2 sides][T + 1][BH] rows that changed group in each k-means pass
 };
 
 namespace {
@@ -209,8 +273,9 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   float* xnorm = c.take<float>(BH * N); int* flagged = c.take<int>(BH * N);
   __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
   int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
+  int* km_changed = c.take<int>(2 * (size_t)(r.T + 1) * BH);
   if (p) {
-    p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
+    p->km_changed = km_changed; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -232,7 +297,7 @@ struct AttendWs {
 int probe_splits(const Resolved& r) {
   if (r.M == 0) return 1;
   const int row_tiles = (r.M + 63) / 64;
-  int s = (2 * 148 + r.BH * row_tiles - 1) / (r.BH * row_tiles);
+  int s = (2 * sm_count() + r.BH * row_tiles - 1) / (r.BH * row_tiles);
   const int key_tiles = (r.N + 63) / 64;
   s = std::max(1, std::min(s, std::max(1, key_tiles / 4)));
   return s;
@@ -246,7 +311,7 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   void* Vg = c.take<char>(BH * N * d * r.es);
   const size_t M1 = std::max(r.M, 1);
   // tensor-core probe kernel: one CTA per (128 probe rows, key slice), about one wave
-  const int ns_tc = std::max(1, std::min(148 / std::max(1, r.BH * (int)((M1 + 127) / 128)), std::max(1, r.N / 128 / 4)));
+  const int ns_tc = std::max(1, std::min(sm_count() / std::max(1, r.BH * (int)((M1 + 127) / 128)), std::max(1, r.N / 128 / 4)));
   float* partial = c.take<float>(probe_partial_floats(r.BH, std::max(ns, ns_tc), (int)M1, r.d));
   __nv_bfloat16* Qp = c.take<__nv_bfloat16>(BH * M1 * d);
   float* X = c.take<float>(BH * M1 * d); float* Dn = c.take<float>(BH * M1 * d);
@@ -265,6 +330,10 @@ i64 pair_budget(const Resolved& r) {
 void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cudaStream_t st) {
   const Resolved& R = p->r;
   const int ld = round16(r);
+  // changed[t][bh], t = 1..T: rows of head bh that changed group in pass t.  A pass that changes nothing proves the
+  // fixed point, so the later passes of that head return at once (their result would be identical).
+  int* changed = p->km_changed + (tag == kTagQInit ? (size_t)(R.T + 1) * R.BH : 0);
+  cudaMemsetAsync(changed, 0, (size_t)(R.T + 1) * R.BH * sizeof(int), st);
   launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
   const bool tcp = kmeans_tc_supported();
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
@@ -273,17 +342,20 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
   if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
+    const int* prev = t > 1 ? changed + (size_t)(t - 1) * R.BH : nullptr;
+    int* cur = changed + (size_t)t * R.BH;
     if (tcp) {
       KmeansTcArgs ka{};
       ka.BH = R.BH; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
       ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2;
       ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
       ka.flagged = p->flagged; ka.flag_count = p->recheck + 1; ka.recheck_total = p->recheck; ka.err = p->err;
+      ka.prev_changed = prev; ka.cur_changed = cur;
       launch_kmeans_assign_tc(ka, st);
     } else {
       if (!upd) cudaMemsetAsync(p->recheck, 0, sizeof(int), st);
       launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
-                           upd ? p->counts : nullptr, p->fx_shift, p->recheck, st);
+                           upd ? p->counts : nullptr, p->fx_shift, p->recheck, prev, cur, st);
     }
     if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   }
@@ -350,16 +422,10 @@ static sparsepr_status_t make_plan(const sparsepr_shape_t* shape, const sparsepr
   if (!p) return SPARSEPR_ERR_INVALID_ARG;
   p->r = r;
   p->stream = static_cast<cudaStream_t>(cuda_stream);
-  int prio_lo = 0, prio_hi = 0;
-  cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-  if (cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
-      cudaStreamCreateWithPriority(&p->side2, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
-      cudaEventCreateWithFlags(&p->ev_join2, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) != cudaSuccess) {
-    delete p;
-    return SPARSEPR_ERR_CUDA;
-  }
+  p->set = acquire_side_set();
+  if (!p->set) { delete p; return SPARSEPR_ERR_CUDA; }
+  p->side = p->set->side; p->side2 = p->set->side2;
+  p->ev_fork = p->set->ev_fork; p->ev_join = p->set->ev_join; p->ev_join2 = p->set->ev_join2;
   Carver c(workspace);
   carve_plan(c, r, p);
   *out = p;
@@ -466,6 +532,7 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   if (s != SPARSEPR_OK) return s;
   const Resolved& r = p->r;
   if (r.M > 0 && (!in->probe_idx || !in->probe_w)) { delete p; return SPARSEPR_ERR_INVALID_ARG; }
+  p->imported = true;
   cudaStream_t st = p->stream;
   cudaGetLastError();
   const size_t BH = r.BH, N = r.N;
@@ -690,6 +757,18 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
   out->rho_exec = out->rho_route + (double)r.M / (double)r.N;
   out->assign_rechecked_rows = errw[1];
   out->device_error = errw[0];
+  // k-means passes that ran before every head had reached its fixed point (or T)
+  std::vector<int> ch(2 * (size_t)(r.T + 1) * r.BH);
+  if (cudaMemcpy(ch.data(), p->km_changed, ch.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  for (int side = 0; side < 2 && !p->imported; ++side) {
+    int worst = 0;
+    for (int bh = 0; bh < r.BH; ++bh) {
+      int ran = 1;
+      while (ran < r.T && ch[((size_t)side * (r.T + 1) + ran) * r.BH + bh] > 0) ++ran;
+      worst = std::max(worst, ran);
+    }
+    (side == 0 ? out->kmeans_passes_kv : out->kmeans_passes_q) = worst;
+  }
   return SPARSEPR_OK;
 }
 
@@ -710,6 +789,22 @@ sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* p, sparsepr_plan_h
     cp(rs.data(), p->rstate, BH * sizeof(RouteState));
     for (size_t i = 0; i < BH; ++i) o->routed_pairs[i] = rs[i].pairs;
   }
+  return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
+sparsepr_status_t sparsepr_plan_export_features(const sparsepr_plan_t* p, sparsepr_plan_features_t* o) {
+  if (!p || !o) return SPARSEPR_ERR_INVALID_ARG;
+  if (p->imported) return SPARSEPR_ERR_UNSUPPORTED;          // an imported plan never computed them
+  const Resolved& r = p->r;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess || (p->side && cudaStreamSynchronize(p->side) != cudaSuccess)) return SPARSEPR_ERR_CUDA;
+  const size_t BH = r.BH, N = r.N, d = r.d;
+  bool ok = true;
+  auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };
+  cp(o->F_K, p->FK, BH * d * r.rK * 4); cp(o->F_Q, p->FQ, BH * d * r.rQ * 4);
+  if (o->phi_Q)                                                // rows are padded to RQ floats on the device
+    ok &= cudaMemcpy2D(o->phi_Q, (size_t)r.rQ * 4, p->phi, (size_t)r.RQ * 4, (size_t)r.rQ * 4, BH * N, cudaMemcpyDeviceToHost) == cudaSuccess;
+  cp(o->kappa, p->kappa, BH * r.Ck * d * 4); cp(o->theta, p->theta, BH * r.Cq * d * 4);
+  cp(o->score, p->score, BH * (size_t)r.Cq * r.Ck * 4);
   return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 
@@ -752,7 +847,7 @@ sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const f
     ka.flagged = flagged; ka.flag_count = fx + 1; ka.recheck_total = fx + 2;
     if (!launch_kmeans_assign_tc(ka, st)) return SPARSEPR_ERR_CUDA;
   } else {
-    launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, st);
+    launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, st);
   }
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }

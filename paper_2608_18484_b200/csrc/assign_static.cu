@@ -70,6 +70,6 @@ extern "C" sparsepr_status_t sparsepr_stage_assign_static(int32_t n, int32_t C, 
   k_pad_rows_static<<<(unsigned)(((i64)n * R + 255) / 256), 256, 0, st>>>(X, n, r, R, Xp);
   k_pad_rows_static<<<(unsigned)(((i64)C * R + 255) / 256), 256, 0, st>>>(mu, C, r, R, mup);
   launch_kmeans_finalize(mup, mu2, mumax, nullptr, nullptr, nullptr, 1, C, r, 0, st);   // writes ||mu||^2 and the max norm
-  launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, st);
+  launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, st);
   return cudaGetLastError() == cudaSuccess ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }

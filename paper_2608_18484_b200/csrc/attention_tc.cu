@@ -27,7 +27,6 @@
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
-#include <cstdio>
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -43,18 +42,9 @@ constexpr int kSubPerTile = kTile / kSub;
 constexpr uint32_t kHalfBytes = kTile * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr uint32_t kSubBytes = kSub * 128;            // 2 KB per box
-#ifndef SPR_K_STAGES
-#define SPR_K_STAGES 3
-#endif
-#ifndef SPR_V_STAGES
-#define SPR_V_STAGES 2
-#endif
-#ifndef SPR_POLY_OF8
-#define SPR_POLY_OF8 3
-#endif
-constexpr int kPolyOf8 = SPR_POLY_OF8;  // pairs of every 8 whose exponential is a polynomial on the FMA pipe
-constexpr int kKStages = SPR_K_STAGES;  // K tiles in flight (consumed by Q K^T)
-constexpr int kVStages = SPR_V_STAGES;  // V tiles in flight (consumed by P V)
+constexpr int kPolyOf8 = 3;            // pairs of every 8 whose exponential is a polynomial on the FMA pipe
+constexpr int kKStages = 3;            // K tiles in flight (consumed by Q K^T)
+constexpr int kVStages = 2;            // V tiles in flight (consumed by P V)
 
 struct Smem {                          // offsets from a 1024-byte aligned base
   static constexpr uint32_t q = 0;
@@ -103,9 +93,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y, b = bh / prm.H, h = bh % prm.H;
-#ifdef SPR_ATTN_TIMING
-  const long long cta_t0 = clock64();
-#endif
   // ---- which query tile ---------------------------------------------------------------
   // Few dependent global reads: one round finds the query group of this tile (every thread tests one group),
   // reads the error word and stages the key-group offsets in shared memory (the K ring is still idle); the
@@ -192,18 +179,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const Maps* maps = is_k ? &mapsK : &mapsV;
       int ri = 0, off = 0;
       bool ok = true;
-#ifdef SPR_ATTN_TIMING
-      long long pa = 0, pb = 0, pc = 0, p0;
-#define SPR_P0() p0 = clock64()
-#define SPR_PACC(v) do { const long long t1 = clock64(); v += t1 - p0; p0 = t1; } while (0)
-#else
-#define SPR_P0()
-#define SPR_PACC(v)
-#endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % nst;
         const uint32_t ph = ((i / nst) & 1) ^ 1;             // empty barriers: the first pass completes immediately
-        SPR_P0();
         // the tile takes up to 8 boxes of 16 rows; consecutive boxes of one key range form a segment, and a segment
         // of n boxes is fetched by one copy per set bit of n (128, 64, 32 or 16 rows), largest first
         int my_start = 0, my_t = 0, my_n = 0, nsub = 0;
@@ -228,9 +206,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb)
           if (lane < nsub && ((my_n >> kb) & 1) && my_t == ((my_n >> (kb + 1)) << (kb + 1))) my_k = kb;
-        SPR_PACC(pa);
         ok = __all_sync(0xffffffffu, mbar_wait(bar(empty0 + s), ph, abort_flag));
-        SPR_PACC(pb);
         if (!ok) break;
         if (lane == 0) {
           if (is_k) {
@@ -246,12 +222,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           tma_load_4d(dst, &maps->m[my_k], bar(full0 + s), 0, my_start, c2, c3);
           tma_load_4d(dst + kHalfBytes, &maps->m[my_k], bar(full0 + s), 64, my_start, c2, c3);
         }
-        SPR_PACC(pc);
       }
-#ifdef SPR_ATTN_TIMING
-      if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0)
-        printf("%s producer tiles %d: walk %lld  wait empty %lld  issue %lld (cycles per tile)\n", is_k ? "K" : "V", n_tiles, pa / n_tiles, pb / n_tiles, pc / n_tiles);
-#endif
     }
   } else if (warp == 9) {
     // =========================== Q K^T issuer ============================================
@@ -265,22 +236,11 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint64_t q_desc = smem_desc(base + Smem::q, 16);
       const uint64_t k_desc0 = smem_desc(base + Smem::k, 16);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
-#ifdef SPR_ATTN_TIMING
-      long long qa = 0, qb = 0, qc = 0, m0;
-#define SPR_M0() m0 = clock64()
-#define SPR_MACC(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
-#else
-#define SPR_M0()
-#define SPR_MACC(v)
-#endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kKStages;
-        SPR_M0();
         // score buffer i mod 2 is free once every softmax thread holds tile i - 2 in registers
         if (i >= 2 && !mbar_wait(bar(S_FREE + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)) { ok = false; break; }
-        SPR_MACC(qa);
         if (!mbar_wait(bar(K_FULL + s), (i / kKStages) & 1, abort_flag)) { ok = false; break; }
-        SPR_MACC(qb);
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)(i & 1) * 128u;
         const uint64_t kd = k_desc0 + (uint64_t)(s * (kTileBytes >> 4));
@@ -291,12 +251,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         umma_commit(bar(K_EMPTY + s));
         umma_commit(bar(S_FULL + (i & 1)));
-        SPR_MACC(qc);
       }
-#ifdef SPR_ATTN_TIMING
-      if (blockIdx.x == 7 && blockIdx.y == 0)
-        printf("mma QK thread tiles %d: wait S free %lld  wait K %lld  issue %lld (cycles per tile)\n", n_tiles, qa / n_tiles, qb / n_tiles, qc / n_tiles);
-#endif
     }
   } else if (warp == 11) {
     // =========================== P V issuer ==============================================
@@ -304,18 +259,12 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint32_t idesc_pv = idesc_bf16(1, 128);
       const uint64_t v_desc0 = smem_desc(base + Smem::v, kHalfBytes);
       bool ok = true;
-#ifdef SPR_ATTN_TIMING
-      long long mv = 0, mp = 0, mi = 0, m0;
-#endif
       for (int i = 0; i < n_tiles && ok; ++i) {
         const int s = i % kVStages;
-        SPR_M0();
         if (!mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag)) { ok = false; break; }
         const int nsub = (int)meta[i & 7].y;
         if (!mbar_wait(bar(V_FULL + s), (i / kVStages) & 1, abort_flag)) { ok = false; break; }
-        SPR_MACC(mv);
         if (!mbar_wait(bar(P_FULL + (i & 1)), (i >> 1) & 1, abort_flag)) { ok = false; break; }   // P(i) in TMEM, O rescaled if needed
-        SPR_MACC(mp);
         tc_fence_after();
         const uint32_t d = tmem + 320u;
         const uint32_t pa = tmem + ((i & 1) ? 448u : 256u);
@@ -326,12 +275,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             umma_bf16_ts(d, pa + kk * 8, vd + (uint64_t)(kk * (kSubBytes >> 4)), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         umma_commit(bar(V_EMPTY + s));
         umma_commit(bar(P_EMPTY + (i & 1)));
-        SPR_MACC(mi);
       }
-#ifdef SPR_ATTN_TIMING
-      if (blockIdx.x == 7 && blockIdx.y == 0)
-        printf("mma PV thread tiles %d: wait V %lld  wait P %lld  issue %lld (cycles per tile)\n", n_tiles, mv / n_tiles, mp / n_tiles, mi / n_tiles);
-#endif
       if (ok) umma_commit(bar(O_DONE));
     }
   } else if (warp < 8) {
@@ -347,19 +291,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
-#ifdef SPR_ATTN_TIMING
-    const long long cta_t1 = clock64();
-#endif
-#ifdef SPR_ATTN_TIMING
-    long long tw = 0, tl = 0, tm = 0, ts = 0, tx = 0, tp = 0, tmx = 0, t0;
-#define SPR_T0() t0 = clock64()
-#define SPR_ACC(v) do { const long long t1 = clock64(); v += t1 - t0; t0 = t1; } while (0)
-#else
-#define SPR_T0()
-#define SPR_ACC(v)
-#endif
     for (int i = 0; i < n_tiles; ++i) {
-      SPR_T0();
       // the three barriers of this tile are polled back to back (their shared-memory round trips overlap); the P
       // buffer of this parity was consumed by the product two tiles back and is normally free long before
       const bool t_meta = mbar_try(bar(META_FULL + (i & 7)), (i >> 3) & 1);
@@ -379,11 +311,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const uint32_t s_addr = tmem + lane_addr + (uint32_t)(i & 1) * 128u + (uint32_t)hh * 64u;
         tmem_ld32_nowait(s_addr, *reinterpret_cast<float(*)[32]>(&s[0]));
         tmem_ld32_nowait(s_addr + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
-        SPR_ACC(tw);
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive(bar(S_FREE + (i & 1)));                         // the scores are in registers
-        SPR_ACC(tl);
         if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
           // only the boxes that end a key range (or lie beyond the stream) have columns to mask; the test is uniform
 #pragma unroll
@@ -406,11 +336,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       // the two halves of the row exchange their maxima (buffer of this tile's parity; executed whatever happened)
       float* xm = xmax + (i & 1) * 256;
-      SPR_ACC(tmx);
       xm[hh * 128 + row] = mx;
       asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
       mx = fmaxf(mx, xm[(hh ^ 1) * 128 + row]);
-      SPR_ACC(tx);
       const bool move = (mx - m_ref) * sc > 8.f;                 // true on the first tile (m_ref = -inf); same in both halves
       const float m_new = move ? mx : m_ref;
       const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f; // 0 on the first tile
@@ -421,7 +349,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         ok = __all_sync(FULL, ok && (t_pe || mbar_wait(bar(P_EMPTY + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)));
         tc_fence_after();
       }
-      SPR_ACC(tp);
       if (!ok) continue;                                         // warp-uniform; the pair barrier above has been passed
       if (i > 0 && __any_sync(FULL, move)) {                     // rescale this half of the warp's O rows (rare)
         // O must be at rest: the product of the previous tile has to be complete as well
@@ -454,26 +381,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         uint32_t w[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) w[c] = pack_bf16(s[2 * c], s[2 * c + 1]);
-        SPR_ACC(tm);
         tmem_st32u(p_addr0 + (uint32_t)(i & 1) * 192u, w);
       }
       tc_fence_before();
       mbar_arrive(bar(P_FULL + (i & 1)));
-      SPR_ACC(ts);
     }
-#ifdef SPR_ATTN_TIMING
-    if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 4))
-      printf("softmax warp %d tiles %d: wait S %lld  tmem ld %lld  mask+max %lld  exchange %lld  wait P empty %lld  exp+pack %lld  st+arrive %lld (cycles per tile)\n", warp, n_tiles,
-             tw / max(1, n_tiles), tl / max(1, n_tiles), tmx / max(1, n_tiles), tx / max(1, n_tiles), tp / max(1, n_tiles), tm / max(1, n_tiles), ts / max(1, n_tiles));
-#endif
     // ---- row sums of the two halves, normalise, store ------------------------------------------
-#ifdef SPR_ATTN_TIMING
-    const long long cta_t2 = clock64();
-#endif
     if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
-#ifdef SPR_ATTN_TIMING
-    const long long cta_t3 = clock64();
-#endif
     xsum[hh * 128 + row] = l;
     asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
     const float ltot = l + xsum[(hh ^ 1) * 128 + row];
@@ -513,13 +427,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
       }
     }
-#ifdef SPR_ATTN_TIMING
-    if (blockIdx.x == 7 && blockIdx.y == 0 && lane == 0 && warp == 0)
-      printf("cta tiles %d: prologue %lld  loop %lld  wait O %lld  epilogue %lld\n", n_tiles, cta_t1 - cta_t0, cta_t2 - cta_t1, cta_t3 - cta_t2, clock64() - cta_t3);
   }
-#else
-  }
-#endif
   // ---- teardown ----------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();

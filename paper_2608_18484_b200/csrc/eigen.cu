@@ -14,7 +14,6 @@
 //   6. back-transformation with the reflectors, scaling, output
 // The work per matrix is O(n^3) for step 1 and O(r n^2) for step 6, each spread over the CTA;
 // steps 2-3 are O(n) recurrences per thread.
-#include <cstdio>
 #include "kernels.cuh"
 
 namespace spr {
@@ -178,9 +177,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
 #pragma unroll
   for (int t = 0; t < kPer; ++t) a[t] *= inv_scale;
 
-#ifdef SPR_EIG_TIMING
-  const long long T0 = clock64();
-#endif
   // ---- 1. Householder tridiagonalisation ----------------------------------------------------------------
   // Step k: x = A[k][k+1..] (row k = column k by symmetry) goes to shared memory; v = x + sgn alpha e_1;
   // p = b A22 v; w = p - (b/2)(p.v) v; A22 <- A22 - v w^T - w v^T.  Two barriers per step: the sums over
@@ -281,9 +277,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   if (tid < NN - 2) A[tid * LD + pos(tid + 1)] += e2[tid];           // v_0 = x_0 + sgn alpha
   if (tid == 0) { ee[NN - 1] = T(0.0); beta[NN - 2] = T(0.0); beta[NN - 1] = T(0.0); }
   __syncthreads();
-#ifdef SPR_EIG_TIMING
-  const long long T1 = clock64();
-#endif
   if (tid < NN) e2[tid] = ee[tid] * ee[tid];
   T g = T(0.0);
   if (tid < NN) g = fabs(dd[tid]) + fabs(ee[tid]) + (tid > 0 ? fabs(ee[tid - 1]) : T(0.0));
@@ -308,9 +301,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     if (active && t == 0) lam[j] = T(0.5) * (lo + hi);
   }
   __syncthreads();
-#ifdef SPR_EIG_TIMING
-  const long long T2 = clock64();
-#endif
 
   // ---- 3. inverse iteration: thread j computes eigenvector j of T ------------------------------------
   if (tid < r) {
@@ -377,9 +367,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
   }
   __syncthreads();
-#ifdef SPR_EIG_TIMING
-  const long long T3 = clock64();
-#endif
 
   // ---- 4. groups of close eigenvalues: Gram-Schmidt inside each group ---------------------------------
   if (tid == 0) {
@@ -424,9 +411,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     j0 = j1 + 1;
   }
   __syncthreads();
-#ifdef SPR_EIG_TIMING
-  const long long T4 = clock64();
-#endif
 
   // ---- 5. Rayleigh quotients, residuals, orthogonality -------------------------------------------------
   bool bad = false;
@@ -468,14 +452,8 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   __syncthreads();
   if (flags[0]) {
     if (tid == 0) Fo[0] = __int_as_float(0x7fc00000);           // marked for the Jacobi kernel
-#ifdef SPR_EIG_TIMING
-    if (tid == 0) printf("eig matrix %d marked for Jacobi\n", (int)blockIdx.x);
-#endif
     return;
   }
-#ifdef SPR_EIG_TIMING
-  const long long T5 = clock64();
-#endif
 
   // ---- 6. back-transformation z <- H_0 ... H_{n-3} z, scaling, output -------------------------------------
   {
@@ -513,11 +491,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   __syncthreads();
   T part = tid < r ? fmax(lam[tid], T(0.0)) : T(0.0);
   const T mean = cta_sum(part, red, turn) / (T)r;
-#ifdef SPR_EIG_TIMING
-  if (tid == 0 && blockIdx.x == 0)
-    printf("eig n=%d r=%d cycles: householder %lld bisection %lld inverse-it %lld mgs %lld check %lld backtransform %lld\n", NN, r,
-           T1 - T0, T2 - T1, T3 - T2, T4 - T3, T5 - T4, clock64() - T5);
-#endif
   if (lam_out)
     for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = j < r ? (double)(lam[j] * scale) : 0.0;
   for (int e = tid; e < NN * r; e += kEigThreads) {

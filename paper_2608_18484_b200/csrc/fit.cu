@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(256) k_fit_prepare(FitArgs a) {
     }
   }
   __syncthreads();
-  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = cnt * (double)w[p] / sw;
+  for (int p = threadIdx.x; p < M; p += 256) sc[L.wt + p] = (double)M * (double)w[p] / sw;   // unit-mean weights M w_p / sum w (Appendix A.3)
 }
 
 // blockIdx.x selects G = Xb^T W Xb + lam I, B(rhs) = Xb^T W Rb, S = Rb^T W Rb.

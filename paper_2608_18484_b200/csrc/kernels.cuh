@@ -4,6 +4,10 @@
 
 namespace spr {
 
+// Number of SMs of the current device (cached per device; 148 when no device can be queried, so that
+// workspace sizes can still be computed).  Defined in api.cu.
+int sm_count();
+
 // ---- partition.cu -------------------------------------------------------------
 cudaError_t init_group_sort();
 void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
@@ -21,9 +25,12 @@ void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh = nullptr, __nv_bfloat16* ml = nullptr);
+// prev_changed / cur_changed [BH] (may be null): number of rows of each head whose assignment changed in the previous
+// / this pass.  A head whose previous pass changed nothing is skipped (Lloyd's iteration has reached its fixed
+// point: every later pass would reproduce the same assignment and the same centroids).
 void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
                           const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
-                          int* recheck_count, cudaStream_t st);
+                          int* recheck_count, const int* prev_changed, int* cur_changed, cudaStream_t st);
 void launch_group_sort(const int* assign, int BH, int N, int C, int* perm, int* inv, int* off, int* err, cudaStream_t st);
 void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, const int* off, int N,
                         int C, int d, float* out, int* sizes, cudaStream_t st);
@@ -45,6 +52,7 @@ struct KmeansTcArgs {
   int* assign;
   i64* sums; int* counts; const int* fx_shift; // null sums = assignment only
   int *flagged, *flag_count, *recheck_total, *err;
+  const int* prev_changed; int* cur_changed;   // [BH] or null, as for launch_kmeans_assign
 };
 cudaError_t init_kmeans_tc();
 bool kmeans_tc_supported();

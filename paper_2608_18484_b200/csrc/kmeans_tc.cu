@@ -13,7 +13,6 @@
 // epilogue groups on alternate row tiles (one row per thread: tcgen05.ld, best/second,
 // fixed-point centroid sums with warp-level pre-aggregation), warp 4 TMA producer, warp 5
 // MMA issuer.
-#include <cstdio>
 #include "kernels.cuh"
 #include "tc_common.cuh"
 
@@ -44,6 +43,7 @@ struct KmParams {
   i64* sums; int* counts; const int* fx_shift;
   int* flagged; int* flag_count;        // rows left to the exact recheck
   int* err;
+  const int* prev_changed; int* cur_changed;   // [BH] or null: rows whose assignment changed in the previous / this pass
 };
 
 __global__ void __launch_bounds__(kKmThreads, 1)
@@ -68,7 +68,9 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     mu2s[c] = v;
     if (c < prm.C) mu2max = fmaxf(mu2max, v);
   }
-  if (tid == 0) s_skip = prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT;
+  // a head whose previous pass changed no assignment has reached the fixed point of the iteration: skipped
+  if (tid == 0) s_skip = (prm.err != nullptr && *reinterpret_cast<volatile int*>(prm.err) == SPARSEPR_ERR_TIMEOUT) ||
+                         (prm.prev_changed != nullptr && prm.prev_changed[bh] == 0);
   // largest centroid norm of the head, rounded up: it enters the bound on the score error only
   const float mm_head = sqrtf(block_max(mu2max, s_red)) * 1.000001f;
   __syncthreads();
@@ -131,12 +133,6 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(0, kKmChunk);
       const int ksteps = prm.R / 16;
-#ifdef SPR_KM_TIMING
-      long long mX = 0, mA = 0, mI = 0, m0 = clock64();
-#define SPR_KM(v) do { const long long t1 = clock64(); v += t1 - m0; m0 = t1; } while (0)
-#else
-#define SPR_KM(v)
-#endif
       int v = 0;                                               // same step order as the producer
       for (int sidx = 0; sidx < n_pairs * 2 * n_chunks; ++sidx) {
         const int r2 = sidx % (2 * n_chunks);
@@ -145,10 +141,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         const int xs = tl & 1, ms = n_chunks > 1 ? (v & 1) : 0;
         const int ab = tl & 1, au = (tl >> 1) * n_chunks + ch;   // score buffer and how often it has been used before
         if (ch == 0 && !mbar_wait(bar(X_FULL + xs), (tl >> 1) & 1, abort_flag)) break;
-        SPR_KM(mX);
         if ((n_chunks > 1 || v == 0) && !mbar_wait(bar(MU_FULL + ms), n_chunks > 1 ? ((v >> 1) & 1) : 0, abort_flag)) break;
         if (!mbar_wait(bar(ACC_EMPTY + ab), (au & 1) ^ 1, abort_flag)) break;
-        SPR_KM(mA);
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)ab * 256u;
         const uint32_t xh = base + KmSmem::x + xs * 2 * kXBytes, xl = xh + kXBytes;
@@ -160,13 +154,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         if (ch == n_chunks - 1) umma_commit(bar(X_EMPTY + xs));
         if (n_chunks > 1) umma_commit(bar(MU_EMPTY + ms));
         umma_commit(bar(ACC_FULL + ab));
-        SPR_KM(mI);
         ++v;
       }
-#ifdef SPR_KM_TIMING
-      if (blockIdx.x == 1 && blockIdx.y == 0 && steps > 0)
-        printf("km mma steps %d sums %d: wait X %lld  wait ACC_EMPTY %lld  issue %lld (cycles per tile)\n", steps, prm.sums != nullptr, mX / steps, mA / steps, mI / steps);
-#endif
     }
   } else {
     // =========================== epilogue: argmin, sums =====================================
@@ -176,12 +165,6 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
     const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const float mm = mm_head;
     bool ok = true;
-#ifdef SPR_KM_TIMING
-    long long eP = 0, eW = 0, eA = 0, eD = 0, eS = 0, e0 = clock64();
-#define SPR_KE(v) do { const long long t1 = clock64(); v += t1 - e0; e0 = t1; } while (0)
-#else
-#define SPR_KE(v)
-#endif
     for (int tl = grp; tl < my_tiles; tl += 2) {
       const int row = (tile0 + tl) * 128 + wq * 32 + lane;
       float best = 3.0e38f, second = 3.0e38f;
@@ -212,11 +195,9 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           }
         }
       }
-      SPR_KE(eP);
       for (int ch = 0; ch < n_chunks; ++ch) {
         const int ab = tl & 1, au = (tl >> 1) * n_chunks + ch;   // this group's score buffer and its phase
         ok = __all_sync(FULL, ok && mbar_wait(bar(ACC_FULL + ab), au & 1, abort_flag));
-        SPR_KE(eW);
         if (!ok) continue;
         tc_fence_after();
         const int c0 = ch * kKmChunk;
@@ -242,23 +223,28 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         }
         tc_fence_before();
         mbar_arrive(bar(ACC_EMPTY + ab));
-        SPR_KE(eA);
       }
       // decide, or hand the row to the exact recheck
       const bool valid = ok && row < prm.N;
-      bool decided = false;
+      bool decided = false, moved = false;
       if (valid) {
         // bound on |computed score - true score|: split-operand products (2^-13 relative with
         // margin), fp32 accumulation and the final combination
         const float E = 2.5e-4f * xn * mm + 1.0e-6f * (mm * mm + xn * mm);
         decided = second - best > 2.f * E;
-        prm.assign[(i64)bh * prm.N + row] = bi;
-        if (!decided) {
+        if (decided) {
+          int* ap = prm.assign + (i64)bh * prm.N + row;
+          moved = prm.prev_changed == nullptr || *ap != bi;
+          *ap = bi;
+        } else {                                             // the recheck writes (and compares) this row's assignment
           const int pos = atomicAdd(prm.flag_count, 1);
           prm.flagged[pos] = bh * prm.N + row;
         }
       }
-      SPR_KE(eD);
+      if (prm.cur_changed != nullptr) {
+        const int nmoved = __popc(__ballot_sync(FULL, moved));
+        if (lane == 0 && nmoved) atomicAdd(prm.cur_changed + bh, nmoved);
+      }
       if (prm.sums) {
         // warp-level pre-aggregation: lanes = feature columns (2 lane, 2 lane + 1); the 32 rows of the
         // warp were prefetched above; one fixed-point atomic per (cluster, column)
@@ -285,15 +271,7 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           if (lane == 0) atomicAdd(prm.counts + (i64)bh * prm.C + cl, __popc(members));
         }
       }
-      SPR_KE(eS);
     }
-#ifdef SPR_KM_TIMING
-    if (blockIdx.x == 1 && blockIdx.y == 0 && lane == 0 && (warp == 0 || warp == 6)) {
-      const int nt = max(1, (my_tiles + 1 - grp) / 2);
-      printf("km epilogue warp %d tiles %d sums %d: prefetch %lld  wait ACC %lld  argmin %lld  decide %lld  sums %lld (cycles per tile)\n", warp, nt,
-             prm.sums != nullptr, eP / nt, eW / nt, eA / nt, eD / nt, eS / nt);
-    }
-#endif
   }
   tc_fence_before();
   __syncthreads();
@@ -315,7 +293,8 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
                                                         const float* __restrict__ phi, int ldphi, int N, int r, int R,
                                                         const float* __restrict__ mu, int C, int* __restrict__ assign,
                                                         i64* __restrict__ sums, int* __restrict__ counts,
-                                                        const int* __restrict__ fx_shift, int* __restrict__ recheck_total) {
+                                                        const int* __restrict__ fx_shift, int* __restrict__ recheck_total,
+                                                        int first_pass, int* __restrict__ cur_changed) {
   __shared__ double s_best[8];
   __shared__ int s_bi[8];
   const unsigned FULL = 0xffffffffu;
@@ -362,7 +341,10 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
       const int oi = s_bi[w];
       if (oi >= 0 && (bi < 0 || ob < best || (ob == best && oi < bi))) { best = ob; bi = oi; }
     }
-    if (tid == 0) assign[gr] = bi;
+    if (tid == 0) {
+      if (cur_changed != nullptr && (first_pass || assign[gr] != bi)) atomicAdd(cur_changed + bh, 1);
+      assign[gr] = bi;
+    }
     if (sums) {
       const float* x = phi + (i64)gr * ldphi;
       const double scl = ldexp(1.0, fx_shift[bh]);
@@ -425,13 +407,14 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   KmParams p{};
   p.N = a.N; p.C = a.C; p.r = a.r; p.R = a.R; p.n_chunks = (a.C + kKmChunk - 1) / kKmChunk;
   const int row_tiles = (a.N + 127) / 128;
-  p.ctas_per_head = std::max(1, std::min(row_tiles, 148 / a.BH));
+  p.ctas_per_head = std::max(1, std::min(row_tiles, sm_count() / a.BH));
   p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.assign = a.assign;
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
+  p.prev_changed = a.prev_changed; p.cur_changed = a.cur_changed;
   cudaMemsetAsync(a.flag_count, 0, sizeof(int), st);
   k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
-  k_assign_recheck<<<148 * 4, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
-                                            a.counts, a.fx_shift, a.recheck_total);
+  k_assign_recheck<<<sm_count() * 4, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
+                                                   a.counts, a.fx_shift, a.recheck_total, a.prev_changed == nullptr, a.cur_changed);
   return true;
 }
 

@@ -239,10 +239,12 @@ __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__
                                                        const float* __restrict__ mu, const float* __restrict__ mu2,
                                                        const float* __restrict__ mumax, int C, int* __restrict__ assign,
                                                        i64* __restrict__ sums, int* __restrict__ counts,
-                                                       const int* __restrict__ fx_shift, int* __restrict__ recheck_count) {
+                                                       const int* __restrict__ fx_shift, int* __restrict__ recheck_count,
+                                                       const int* __restrict__ prev_changed, int* __restrict__ cur_changed) {
   __shared__ __align__(16) float mus[kAssignChunk * R];
   __shared__ float mu2s[kAssignChunk];
   const int bh = blockIdx.y;
+  if (prev_changed != nullptr && prev_changed[bh] == 0) return;      // fixed point reached in the previous pass
   const float* ph = phi + (i64)bh * N * ldphi;
   const float* muh = mu + (i64)bh * C * R;
   const int rows[2] = {(int)(blockIdx.x * 256 + threadIdx.x), (int)(blockIdx.x * 256 + threadIdx.x + 128)};
@@ -296,6 +298,7 @@ __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__
       a = exact_assign(ph + (i64)rows[t] * ldphi, muh, C, r, R);
       if (recheck_count) atomicAdd(recheck_count, 1);
     }
+    if (cur_changed != nullptr && (prev_changed == nullptr || assign[(i64)bh * N + rows[t]] != a)) atomicAdd(cur_changed + bh, 1);
     assign[(i64)bh * N + rows[t]] = a;
     if (sums) {
       i64* s = sums + ((i64)bh * C + a) * R;
@@ -310,10 +313,10 @@ __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__
 
 void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
                           const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
-                          int* recheck_count, cudaStream_t st) {
+                          int* recheck_count, const int* prev_changed, int* cur_changed, cudaStream_t st) {
   dim3 grid((N + 255) / 256, BH);
   const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
-#define SPR_ASSIGN(RR) k_kmeans_assign<RR><<<grid, 128, 0, st>>>(phi, ldphi, N, r, mu, mu2, mumax, C, assign, sums, counts, fx_shift, recheck_count)
+#define SPR_ASSIGN(RR) k_kmeans_assign<RR><<<grid, 128, 0, st>>>(phi, ldphi, N, r, mu, mu2, mumax, C, assign, sums, counts, fx_shift, recheck_count, prev_changed, cur_changed)
   if (R == 16) SPR_ASSIGN(16); else if (R == 32) SPR_ASSIGN(32); else if (R == 48) SPR_ASSIGN(48); else SPR_ASSIGN(64);
 #undef SPR_ASSIGN
 }

@@ -201,7 +201,7 @@ bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r
   PjParams p{};
   p.H = H; p.N = N; p.r = r; p.ldphi = ldphi; p.rms = rms; p.eps = eps; p.phi = phi; p.maxabs_bits = maxabs; p.err = err;
   const int row_tiles = (N + 127) / 128;
-  p.ctas_per_head = std::max(1, std::min(row_tiles, (2 * 148) / BH));
+  p.ctas_per_head = std::max(1, std::min(row_tiles, (2 * sm_count()) / BH));
   k_project_tc<<<dim3(p.ctas_per_head, BH), kPjThreads, PjSmem::total, st>>>(mx, mf, p);
   return true;
 }

@@ -1,6 +1,5 @@
 // Shared routing (Section 4.3) and query-group-stratified probe selection
 // (Algorithm A.1, Appendix A.2).
-#include <cstdio>
 #include "kernels.cuh"
 
 namespace spr {
@@ -125,12 +124,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   for (int a = threadIdx.x; a < Cq; a += blockDim.x) nqs[a] = nq[(i64)bh * Cq + a];
   __syncthreads();
 
-#ifdef SPR_RT_TIMING
-  long long rt[8]; int rti = 0; long long rt0 = clock64();
-#define SPR_RT() do { const long long t1 = clock64(); if (rti < 8) rt[rti++] = t1 - rt0; rt0 = t1; } while (0)
-#else
-#define SPR_RT()
-#endif
   // 1. forced cells
   i64 fcost = 0;
   for (int a = w; a < Cq; a += nw) {
@@ -157,7 +150,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   }
   fcost = block_sum_i64(fcost, red);     // contains a __syncthreads: forced[] visible below
   const i64 rem = budget - fcost;
-  SPR_RT();
 
   // 2. threshold search: S(t) = cost of live, non-forced cells with bits >= t; find the smallest t with
   //    S(t) <= rem.  Radix descent, one byte of the bit pattern per pass: per-warp cost histograms over
@@ -258,7 +250,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
     tstar = all_fit ? (u64)prefix : (u64)prefix + 1ull;
     taken = above;
   }
-  SPR_RT();
   // tie tier: cells with bits == tstar-1, in (a,b) order, longest prefix that fits
   __shared__ int s_tie_cnt, s_tie_idx[32];
   if (threadIdx.x == 0) { s_last_tie = -1; s_tie_cnt = 0; }
@@ -341,7 +332,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
     return tie_tier && bits == tvv && (i64)a * Ck + b <= last_tie;
   };
 
-  SPR_RT();
   // 3. counts, offsets, lists
   i64 pairs = 0;
   for (int a = w; a < Cq; a += nw) {
@@ -362,7 +352,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
     if (lane == 0) cnt[a] = c;
   }
   pairs = block_sum_i64(pairs, red);
-  SPR_RT();
   const int total = block_exclusive_scan(cnt, Cq, scratch);
   int* rp = route_ptr + (i64)bh * (Cq + 1);
   int* ri = route_idx + (i64)bh * Cq * Ck;
@@ -387,10 +376,6 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
       }
     }
   }
-  SPR_RT();
-#ifdef SPR_RT_TIMING
-  if (blockIdx.x == 0 && threadIdx.x == 0) printf("route select cycles: forced %lld  radix %lld  tie %lld  counts %lld  emit %lld\n", rt[0], rt[1], rt[2], rt[3], rt[4]);
-#endif
 }
 
 static size_t route_smem(int Cq, int Ck) {      // forced, cnt, nqs [Cq], nks [Ck] ints, then 32 x 256 int64 cost and int32 key histograms

@@ -7,12 +7,19 @@ be fed the very same bytes from it.
 
 Recipe: tokens live on a (T, Hg, Wg) latent grid, token index
 n = (t*Hg + h)*Wg + w.  Every token belongs to a cluster c(n) given by a
-spatiotemporal region map.  For each head and each tensor X in {Q, K, V} an
-independent centroid table mu^X[n_c, d] ~ N(0,1) and noise eps ~ N(0,1) are
-drawn and X_n = mu^X[c(n)] + sigma(n) * eps_n.  Q and K are then multiplied by
-d^(-1/4) (the symmetric folding of the 1/sqrt(d) logit scale into the inputs;
-calls on these tensors therefore use softmax_scale = 1), and everything is
-rounded to the workload's storage type.
+spatiotemporal region map.  For each head a centroid table mu^X[n_c, d] and noise
+eps ~ N(0,1) are drawn per tensor X in {Q, K, V}, and X_n = mu^X[c(n)] +
+sigma(n) * eps_n.  mu^Q and mu^V are independent N(0,1) tables; the key table is
+aligned with the query table, mu^K = c mu^Q + sqrt(1 - c^2) nu with nu ~ N(0,1)
+independent and c = `qk_align` (0.7): a query's logit against the keys of its own
+region is then c sqrt(d) above the zero-mean logits against other regions, so
+that same-region pairs carry most of the softmax mass, as "3D-local clusters"
+implies, while a broad background remains (with c = 0 attention on these inputs
+is nearly uniform and no sparse support can represent it; with c = 1 it is
+one-hot per region).  Q and K are then multiplied by d^(-1/4) (the symmetric
+folding of the 1/sqrt(d) logit scale into the inputs; calls on these tensors
+therefore use softmax_scale = 1), and everything is rounded to the workload's
+storage type.
 """
 from __future__ import annotations
 
@@ -37,6 +44,7 @@ class Workload:
     sigma: float = 0.5
     n_sink: int = 0
     softmax_scale: float = 1.0
+    qk_align: float = 0.7  # correlation c of the key centroid table with the query centroid table
 
     @property
     def N(self) -> int:
@@ -120,6 +128,9 @@ def make_head(wl: Workload, head: int, seed: int = 0):
         rng = np.random.default_rng([seed, wl.cfg_id, head, tensor_id])
         mu = rng.standard_normal((n_c, wl.d), dtype=np.float32)
         eps = rng.standard_normal((wl.N, wl.d), dtype=np.float32)
+        if tensor_id == 1 and wl.qk_align != 0.0:       # keys: aligned with the query centroids
+            c = np.float32(wl.qk_align)
+            mu = c * tables[0] + np.sqrt(np.float32(1.0) - c * c) * mu
         tables.append(mu)
         out.append(mu[cmap] + np.asarray(sig, dtype=np.float32) * eps)
     Q, K, V = out

@@ -2,7 +2,8 @@
 allocate device memory themselves (their process has given all of it to a memory pool,
 or they run where cudaMalloc's device-wide synchronisation is not allowed).
 
-It must give exactly the assignments of sparsepr_stage_assign.  Two calls in a row with
+It must give exactly the assignments of sparsepr_stage_assign, which in turn are the
+float64 decisions of the definition (checked here against the CPU oracle as well).  Two calls in a row with
 different shapes check that data left in the shared scratch array by the first call does
 not leak into the second.  This file sorts last so that a run stopping at the first
 failure has already executed every other test."""
@@ -10,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import sparsepr_oracle as orc
 from paper_2608_18484_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -33,6 +35,10 @@ def test_static_assign_matches_workspace_assign_twice():
         torch.cuda.synchronize()
         assert torch.equal(got, expect)
         assert int(got.min()) >= 0 and int(got.max()) < C
+        # the definition itself: argmin of the float64 squared distance, ties to the lowest id
+        rows = np.random.default_rng(seed).choice(n, 2048, replace=False)
+        want = orc.kmeans_assign(X.cpu().numpy()[rows], mu.cpu().numpy())
+        assert np.array_equal(got.cpu().numpy()[rows], want)
 
 
 def test_static_assign_rejects_oversized_problems():
