@@ -31,6 +31,12 @@ if ROOT not in sys.path:
 METRIC = "sparsepr_attn_ms_per_call"
 UNIT = "ms/call"
 
+# DRAM read + write bytes per head of one launch of the two block-sparse kernels, from ncu captures of 6 heads
+# (capture-size rule) of the named workload; a workload without a capture reports null.
+NCU_DRAM_BYTES_PER_HEAD = {
+    "video-dit-480p-like": {"k_attention_tc": 30.04e6, "k_attention_packed": 18.5e6},
+}
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -128,8 +134,9 @@ def reference_arm(args, wl):
         return
     frames = 3
     small = wl.scaled(grid=(frames,) + tuple(wl.grid[1:]))
+    n_probe = min(wl.n_probe, 64)                   # the sample has 1/7 of the rows: fewer probes keep M/N comparable
     prm = orc.default_params(density=wl.density, block=wl.block, n_sample=wl.n_sample,
-                             n_probe=min(wl.n_probe, 64), softmax_scale=wl.softmax_scale)
+                             n_probe=n_probe, softmax_scale=wl.softmax_scale)
     times = []
     for step in range(args.warmup + args.steps):
         Q, K, V = W.make_head(small, step % wl.H)
@@ -146,15 +153,17 @@ def reference_arm(args, wl):
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_head * 1e3, "higher_is_better": False,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
            "config": {"workload": wl.name, "N": wl.N, "H": wl.H, "d": wl.d, "density": wl.density,
-                      "n_sample": wl.n_sample, "n_probe": wl.n_probe},
+                      "n_sample": wl.n_sample, "n_probe": wl.n_probe, "n_probe_of_the_sample": n_probe},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
                             "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
 
 
-def cpu_baseline(wl):
-    """Oracle timed on the host cores on about 10-20 s of work: one head, first 16 frames."""
+def cpu_baseline(wl, gpu_call=None):
+    """Oracle timed on the host cores on about 10-20 s of work: one head, first 16 frames.  With `gpu_call`
+    (Q, K, V float32 arrays -> O, O_sparse arrays) the GPU path runs on the same bytes and both
+    reconstruction errors against float64 exact attention are reported side by side."""
     import multiprocessing
     from oracle import sparsepr_oracle as orc
     from paper_2608_18484_b200 import workloads as W
@@ -164,12 +173,25 @@ def cpu_baseline(wl):
                              softmax_scale=wl.softmax_scale)
     Q, K, V = W.make_head(small, 0)
     t0 = time.perf_counter()
-    orc.sparsepr_head(Q, K, V, prm, 0)
+    O_hat, O_sp, plan, _ = orc.sparsepr_head(Q, K, V, prm, 0)
     dt = time.perf_counter() - t0
     value = dt * wl.H * (wl.N / small.N) ** 2 * 1e3
-    return {"value": value, "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
-            "sample": "head 0, first %d of %d frames (N=%d): %.1f s measured; value = that x H x (N/N_s)^2" % (
-                frames, wl.grid[0], small.N, dt)}
+    out = {"value": value, "unit": UNIT, "cores": multiprocessing.cpu_count(), "kind": "oracle",
+           "sample": "head 0, first %d of %d frames (N=%d): %.1f s measured; value = that x H x (N/N_s)^2" % (
+               frames, wl.grid[0], small.N, dt)}
+    if gpu_call is not None:
+        exact = orc.dense_attention(Q, K, V, plan["scale"])
+
+        def errs(O, Osp, probes):
+            m, p99 = orc.row_errors(O, exact, probes)
+            hm, hp99 = orc.row_errors(Osp, exact, probes)
+            return {"probe_fitted": orc.rel_l2(O, exact), "hard_drop": orc.rel_l2(Osp, exact),
+                    "row_mean_p99_fitted": [m, p99], "row_mean_p99_hard_drop": [hm, hp99]}
+        G, Gsp, Gd, gprobes = gpu_call(small, Q, K, V)
+        out["error_vs_fp64_exact"] = {"sample": "head 0, first %d frames, the same bytes on both sides" % frames,
+                                      "oracle": errs(O_hat, O_sp, plan["probe_idx"]), "gpu": errs(G, Gsp, gprobes),
+                                      "gpu_dense_kernel": orc.rel_l2(Gd, exact)}
+    return out
 
 
 # --------------------------------------------------------------------------------------
@@ -221,8 +243,12 @@ def main():
                            softmax_scale=wl.softmax_scale)
     O = torch.empty_like(Qd)
 
+    mid = []
+
     def step():
         plan = B.sparsepr_plan(Qd, Kd, Vd, params=params)
+        if mid:
+            mid[-1].record()
         B.sparsepr_attend(plan, Qd, Kd, Vd, out=O)
         return plan
 
@@ -241,11 +267,17 @@ def main():
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
     ev[0].record()
+    mids = []
     for k in range(args.steps):
+        mid.append(torch.cuda.Event(enable_timing=True))
         plan = step()
+        mids.append(mid.pop())
         ev[k + 1].record()
     barrier()
     step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    # the call as it runs (probe selection, probe rows and fit beside the main chain): plan part / attend part
+    plan_part = float(np.mean([ev[k].elapsed_time(mids[k]) for k in range(args.steps)]))
+    attend_part = float(np.mean([mids[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]))
     total_ms = ev[0].elapsed_time(ev[-1])
     total_ms = max_over_ranks(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
@@ -306,12 +338,17 @@ def main():
     tensor_path = wl.dtype == "bf16" and wl.d == 128
     if tensor_path:
         # tcgen05 kernel timed inside a long step: the sustained bf16 GEMM peak is the denominator
+        # tcgen05 kernels timed inside a long step: the sustained bf16 GEMM peak is the denominator of `frac`; the
+        # fraction of the burst peak (the fair one when the clocks stay at their maximum) is printed beside it
+        traffic = NCU_DRAM_BYTES_PER_HEAD.get(wl.name)
         roofline = {"kernel": "k_attention_tc + k_attention_packed (block-sparse, tcgen05)", "bound": "tensor", "achieved": achieved,
                     "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"],
-                    # DRAM read + write of one k_attention_tc launch: 29.6 MB per head from the ncu capture summarised
-                    # in profiles/k_attention_tc_480p-like_6heads.md (177.8 MB at 6 heads of this N; heads are
-                    # independent CTAs over disjoint memory, so traffic scales with the head count)
-                    "traffic": (30.04e6 * wl.H if wl.name == "video-dit-480p-like" else None), "traffic_unit": "bytes",
+                    "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "burst_peak": peaks["bf16_tflops"],
+                    "sm_mhz_median": (clocks or {}).get("sm_mhz"),
+                    "traffic": (sum(traffic.values()) * wl.H if traffic else None), "traffic_unit": "bytes",
+                    "traffic_source": ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of each of the two kernels, "
+                                       "captured at 6 heads of this workload, per head x H (heads are independent CTAs over "
+                                       "disjoint memory)") if traffic else None,
                     "algorithmic_bytes": 4.0 * wl.H * wl.N * wl.d * 2,
                     "peak_source": peaks["source"] + " cuBLAS bf16, sustained",
                     "issued_tflops": issued / (attn_ms * 1e-3) / 1e12,
@@ -340,11 +377,23 @@ def main():
            "rel_l2_vs_dense_kernel": {"probe_fitted": rel_fit, "hard_drop": rel_hard},
            "stage_ms": stages, "plan_ms": sum(v for k, v in stages.items() if k in B.STAGES[:10]),
            "attend_ms": sum(v for k, v in stages.items() if k in B.STAGES[10:16]),
+           "call_parts_ms": {"plan": plan_part, "attend": attend_part,
+                             "note": "the call as timed (side streams overlap); stage_ms come from a one-stream run"},
+           "kmeans_passes": [st["kmeans_passes_kv"], st["kmeans_passes_q"]],
            "device_error": st["device_error"], "assign_rechecked_rows": st["assign_rechecked_rows"],
            "gpu_launches": launches_per_call(params.kmeans_iters or 8, True, wl.dtype == "bf16" and wl.d == 128) * args.steps,
            "roofline": roofline, "clocks": clocks, "e2e": e2e}
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(wl)
+        def gpu_call(small, Q, K, V):
+            q, k, v = [torch.from_numpy(x[None, None]).to(dt).to(dev) for x in (Q, K, V)]
+            pl = B.sparsepr_plan(q, k, v, params=params)
+            o, osp = B.sparsepr_attend(pl, q, k, v, return_sparse=True)
+            od = B.sparsepr_dense(q, k, v, wl.softmax_scale)
+            probes = B.sparsepr_plan_export(pl)["probe_idx"][0]
+            return (o[0, 0].double().cpu().numpy(), osp[0, 0].double().cpu().numpy(), od[0, 0].double().cpu().numpy(),
+                    probes)
+        del Qd, Kd, Vd, O, Odense
+        out["cpu_baseline"] = cpu_baseline(wl, gpu_call)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

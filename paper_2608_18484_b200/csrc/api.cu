@@ -287,6 +287,7 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
 
 struct AttendWs {
   void *Qg, *Kg, *Vg;
+  __nv_bfloat16* Olo;                  // second bf16 word of the hard-drop rows for the correction pass (tensor-core path, fitted mode)
   float *partial, *X, *Dn, *A, *c, *Psi;
   __nv_bfloat16 *At, *Qp;
   int n_split_tc;
@@ -309,6 +310,8 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   void* Qg = c.take<char>(BH * N * d * r.es);
   void* Kg = c.take<char>(BH * N * d * r.es);
   void* Vg = c.take<char>(BH * N * d * r.es);
+  const bool staged = r.dtype == SPARSEPR_BF16 && r.d == 128 && r.mode == 0 && r.M > 0;
+  __nv_bfloat16* Olo = c.take<__nv_bfloat16>(staged ? BH * N * d : 0);
   const size_t M1 = std::max(r.M, 1);
   // tensor-core probe kernel: one CTA per (128 probe rows, key slice), about one wave
   const int ns_tc = std::max(1, std::min(sm_count() / std::max(1, r.BH * (int)((M1 + 127) / 128)), std::max(1, r.N / 128 / 4)));
@@ -319,7 +322,7 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   float* Psi = c.take<float>(BH * d * d);
   __nv_bfloat16* At = c.take<__nv_bfloat16>(BH * d * d);
   double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
-  if (w) { w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->n_split = ns; }
+  if (w) { w->Olo = Olo; w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->n_split = ns; }
 }
 
 i64 pair_budget(const Resolved& r) {
@@ -619,6 +622,8 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   }
   if (tensor) {
     aa.tile_off = p->tile_off128;
+    // with a correction to follow, the block-sparse kernels also store what the bf16 rounding of O dropped
+    if (fitted) aa.O_lo = w.Olo;
     // the packed remainder tiles are few and long, the 128-row tiles many and short: they share the GPU instead of
     // running one after the other (also in a profiled call: both belong to the ATTENTION stage)
     if (!overlap) cudaEventRecord(p->ev_fork, st);                // (with the probes' overlap the event is recorded already)
@@ -629,7 +634,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     cudaStreamWaitEvent(st, p->ev_join2, 0);
     tm.mark(SPARSEPR_STAGE_ATTENTION);
     if (overlap) { join_side(p, st); p->side_pending = false; }
-    if (fitted && !launch_correction_tc(w.A, w.c, w.At, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
+    if (fitted && !launch_correction_tc(w.A, w.c, w.At, w.Olo, O, r.os, r.BH, r.H, r.N, p->err, st)) return SPARSEPR_ERR_CUDA;
     tm.mark(SPARSEPR_STAGE_CORRECTION);
   } else {
     aa.A = fitted ? w.A : nullptr; aa.c = fitted ? w.c : nullptr;      // correction fused into this kernel's epilogue

@@ -69,6 +69,7 @@ struct Params {
   const __nv_bfloat16* Qg;                     // [BH][N][128] group-major
   __nv_bfloat16* O; i64 os[3];
   float* O_sparse;
+  __nv_bfloat16* O_lo;             // optional [BH][N][128]: o - bf16(o), original order (second word for the correction pass)
   int* err;
 };
 
@@ -405,6 +406,16 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
           for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
           store8(op + ch * 8, v8);
         }
+        if (prm.O_lo) {                                        // what the bf16 rounding above dropped
+          __nv_bfloat16* lp = prm.O_lo + ((i64)bh * prm.N + dst) * kD + hh * 64;
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            float v8[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k] - __bfloat162float(__float2bfloat16_rn(o[ch * 8 + k]));
+            store8(lp + ch * 8, v8);
+          }
+        }
         if (prm.O_sparse) {
           float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
 #pragma unroll
@@ -486,7 +497,7 @@ bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* r
   p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;
   p.Qg = (const __nv_bfloat16*)a.Q;
   p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
-  p.O_sparse = a.O_sparse; p.err = a.err;
+  p.O_sparse = a.O_sparse; p.O_lo = (__nv_bfloat16*)a.O_lo; p.err = a.err;
   // a group contributes at most kRemRows of every 128 rows it has beyond a multiple of 128, so the packed rows of a
   // head never exceed N; CTAs past the head's count return at once
   const int tiles = (a.N + kTile - 1) / kTile;

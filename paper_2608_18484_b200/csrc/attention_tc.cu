@@ -22,8 +22,10 @@
 // this is why the two products have a thread each on different schedulers, why the producers issue few, large
 // copies, and why the barrier polls of a tile are grouped.
 // The reference maximum of a row moves only when it grows by more than 2^8 (then O is rescaled).
-// Epilogue: O / l, store at the original token index (inverse permutation).  The residual
-// correction of Eq. 9 is a pass of its own (correction_tc.cu) so that the fit can overlap this kernel.
+// Epilogue: O / l, stored as bf16 at the original token index (inverse permutation).  The residual correction of
+// Eq. 9 is a pass of its own (correction_tc.cu) so that the fit can overlap this kernel; for that pass the part of
+// every element that the bf16 rounding dropped is stored as a second bf16 word (O_lo), so that the corrected output
+// is, in effect, rounded to bf16 only once.
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
@@ -70,6 +72,7 @@ struct Params {
   const int *q_off, *kv_off, *route_ptr, *route_idx, *q_perm, *tile_off;
   __nv_bfloat16* O; i64 os[3];
   float* O_sparse;
+  __nv_bfloat16* O_lo;             // optional [BH][N][128]: o - bf16(o), original order (second word for the correction pass)
   int* err;
 };
 
@@ -416,6 +419,16 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
         store8(op + ch * 8, v8);
       }
+      if (prm.O_lo) {                                          // what the bf16 rounding above dropped
+        __nv_bfloat16* lp = prm.O_lo + ((i64)bh * prm.N + dst) * kD + hh * 64;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k] - __bfloat162float(__float2bfloat16_rn(o[ch * 8 + k]));
+          store8(lp + ch * 8, v8);
+        }
+      }
       if (prm.O_sparse) {
         float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
 #pragma unroll
@@ -512,7 +525,7 @@ bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   p.q_off = a.q_off; p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;
   p.tile_off = a.tile_off;
   p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
-  p.O_sparse = a.O_sparse; p.err = a.err;
+  p.O_sparse = a.O_sparse; p.O_lo = (__nv_bfloat16*)a.O_lo; p.err = a.err;
   const int tiles = (a.N + kTile - 1) / kTile + (sparse ? a.Cq : 0);
   k_attention_tc<<<dim3(tiles, a.BH), kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
   return true;

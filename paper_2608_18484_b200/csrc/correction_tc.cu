@@ -1,10 +1,13 @@
 // Residual correction of Eq. 9 as a pass of its own on the sm_100a tensor cores:
-//   O <- O + O A + c     (in place, bf16, d_v = 128; A, c = composed affine map of one head)
-// It runs after the block-sparse kernel, so that the probe rows and the fit (which produce A and c)
-// can execute on a second stream while the block-sparse kernel is busy.  The pass is bandwidth
-// bound: each 128-row tile of O is read once by TMA and written once.
-//   warps 0-3  one thread per row: O A from TMEM, O from the swizzled tile, + c, store
-//   warp  4    TMA loads (O tile, A^T), eight tcgen05.mma, TMEM owner
+//   O <- X + X A + c     (in place, bf16, d_v = 128; A, c = composed affine map of one head)
+// It runs after the block-sparse kernels, so that the probe rows and the fit (which produce A and c) can execute
+// on a second stream while those kernels are busy.  The block-sparse kernels hand over the hard-drop rows X = O^sp
+// as two bf16 words, X = X_h + X_l: X_h is what they stored in O, X_l the part that rounding dropped (2^-17
+// relative together), so that the corrected output is rounded to bf16 once -- a one-word hand-over rounds twice,
+// which shows in the largest elements.  A enters the product as one bf16 word (the correction is a small term).
+// The pass is bandwidth bound: each 128-row tile is read once (2 x 256 B per row) and written once (256 B per row).
+//   warps 0-3  one thread per row: X A from TMEM, X from the two swizzled tiles, + c, store
+//   warp  4    TMA loads (X_h, X_l, A^T), sixteen tcgen05.mma, TMEM owner
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include "kernels.cuh"
@@ -18,8 +21,9 @@ constexpr int kCorrTile = 128;
 constexpr uint32_t kCorrHalf = kCorrTile * 128;      // one [128 rows x 64 bf16] swizzled block
 constexpr uint32_t kCorrTileBytes = 2 * kCorrHalf;
 struct CorrSmem {
-  static constexpr uint32_t o = 0;
-  static constexpr uint32_t a = o + kCorrTileBytes;
+  static constexpr uint32_t xh = 0;
+  static constexpr uint32_t xl = xh + kCorrTileBytes;
+  static constexpr uint32_t a = xl + kCorrTileBytes;
   static constexpr uint32_t bars = a + kCorrTileBytes;
   static constexpr uint32_t misc = bars + 16;
   static constexpr uint32_t total = misc + 16;
@@ -33,7 +37,8 @@ struct CorrParams {
 };
 
 __global__ void __launch_bounds__(kCorrThreads)
-k_correction_tc(const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapA, CorrParams prm) {
+k_correction_tc(const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapL,
+                const __grid_constant__ CUtensorMap mapA, CorrParams prm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   volatile int* misc = reinterpret_cast<volatile int*>(smem_raw + CorrSmem::misc);   // [0] tmem base, [1] abort, [2] skip
@@ -60,31 +65,41 @@ k_correction_tc(const __grid_constant__ CUtensorMap mapO, const __grid_constant_
 
   if (warp == 4) {
     if (lane == 0) {
-      mbar_expect_tx(bar_full, 2 * kCorrTileBytes);
-      tma_load_4d(base + CorrSmem::o, &mapO, bar_full, 0, row0, h, b);
-      tma_load_4d(base + CorrSmem::o + kCorrHalf, &mapO, bar_full, 64, row0, h, b);
+      mbar_expect_tx(bar_full, 3 * kCorrTileBytes);
+      tma_load_4d(base + CorrSmem::xh, &mapO, bar_full, 0, row0, h, b);
+      tma_load_4d(base + CorrSmem::xh + kCorrHalf, &mapO, bar_full, 64, row0, h, b);
+      tma_load_4d(base + CorrSmem::xl, &mapL, bar_full, 0, row0, bh, 0);
+      tma_load_4d(base + CorrSmem::xl + kCorrHalf, &mapL, bar_full, 64, row0, bh, 0);
       tma_load_4d(base + CorrSmem::a, &mapA, bar_full, 0, 0, bh, 0);
       tma_load_4d(base + CorrSmem::a + kCorrHalf, &mapA, bar_full, 64, 0, bh, 0);
       if (mbar_wait(bar_full, 0, abort_flag)) {
         tc_fence_after();
-        const uint64_t od = smem_desc(base + CorrSmem::o, 16), ad = smem_desc(base + CorrSmem::a, 16);
+        const uint64_t hd = smem_desc(base + CorrSmem::xh, 16), ld = smem_desc(base + CorrSmem::xl, 16);
+        const uint64_t ad = smem_desc(base + CorrSmem::a, 16);
         const uint32_t idesc = idesc_bf16(0, 128);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint64_t koff = (uint64_t)((kk >> 2) * (kCorrHalf >> 4) + (kk & 3) * 2);
-          umma_bf16(tmem, od + koff, ad + koff, idesc, kk > 0);          // (O A)[m][n] = sum_k O[m][k] At[n][k]
+          umma_bf16(tmem, hd + koff, ad + koff, idesc, kk > 0);          // (X A)[m][n] = sum_k X[m][k] At[n][k]
+        }
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t koff = (uint64_t)((kk >> 2) * (kCorrHalf >> 4) + (kk & 3) * 2);
+          umma_bf16(tmem, ld + koff, ad + koff, idesc, 1);
         }
         umma_commit(bar_done);
       }
     }
   } else {
+    // ---- epilogue: one thread per row -------------------------------------------------------------------------
     const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag));
     const int row = warp * 32 + lane;
     if (ok) {
       tc_fence_after();
       const float* cv = prm.c + (i64)bh * 128;
       __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)(row0 + row) * prm.os[2];
-      const unsigned char* orow = smem_raw + CorrSmem::o + row * 128;
+      const unsigned char* hrow = smem_raw + CorrSmem::xh + row * 128;
+      const unsigned char* lrow = smem_raw + CorrSmem::xl + row * 128;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         float t[32];
@@ -92,15 +107,18 @@ k_correction_tc(const __grid_constant__ CUtensorMap mapO, const __grid_constant_
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const int j = (q & 1) * 4 + ch;                                // 16-byte chunk of the 128-byte row
-          const uint4 raw = *reinterpret_cast<const uint4*>(orow + (q >> 1) * kCorrHalf + ((j ^ (row & 7)) << 4));
-          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&raw);
+          const uint32_t so = (q >> 1) * kCorrHalf + ((j ^ (row & 7)) << 4);
+          const uint4 rh = *reinterpret_cast<const uint4*>(hrow + so);
+          const uint4 rl = *reinterpret_cast<const uint4*>(lrow + so);
+          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&rh);
+          const __nv_bfloat162* lp = reinterpret_cast<const __nv_bfloat162*>(&rl);
           float v8[8];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const float2 f = __bfloat1622float2(hp[k]);
+            const float2 fh = __bfloat1622float2(hp[k]), fl = __bfloat1622float2(lp[k]);
             const int col = q * 32 + ch * 8 + 2 * k;
-            v8[2 * k] = f.x + t[ch * 8 + 2 * k] + cv[col];
-            v8[2 * k + 1] = f.y + t[ch * 8 + 2 * k + 1] + cv[col + 1];
+            v8[2 * k] = (fh.x + fl.x) + t[ch * 8 + 2 * k] + cv[col];
+            v8[2 * k + 1] = (fh.y + fl.y) + t[ch * 8 + 2 * k + 1] + cv[col + 1];
           }
           if (row0 + row < prm.N) store8(op + q * 32 + ch * 8, v8);
         }
@@ -138,18 +156,19 @@ cudaError_t init_correction_tc() {
   return cudaFuncSetAttribute(tc::k_correction_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::CorrSmem::total);
 }
 
-bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
-                          int* err, cudaStream_t st) {
+bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, const void* O_lo, void* O, const i64* os, int BH,
+                          int H, int N, int* err, cudaStream_t st) {
   using namespace tc;
-  CUtensorMap mo, ma;
+  CUtensorMap mo, ml, ma;
   k_transpose_correction<<<dim3(4, 4, BH), dim3(32, 8), 0, st>>>(A, At);
   if (!make_map(&mo, O, 128, N, H, BH / H, os[0], os[1], os[2], kCorrTile) ||
+      !make_map(&ml, O_lo, 128, N, BH, 1, 0, (i64)N * 128, 128, kCorrTile) ||
       !make_map(&ma, At, 128, 128, BH, 1, 0, (i64)128 * 128, 128, kCorrTile))
     return false;
   CorrParams p{};
   p.H = H; p.N = N; p.c = c; p.O = (__nv_bfloat16*)O; p.err = err;
   for (int i = 0; i < 3; ++i) p.os[i] = os[i];
-  k_correction_tc<<<dim3((N + kCorrTile - 1) / kCorrTile, BH), kCorrThreads, CorrSmem::total, st>>>(mo, ma, p);
+  k_correction_tc<<<dim3((N + kCorrTile - 1) / kCorrTile, BH), kCorrThreads, CorrSmem::total, st>>>(mo, ml, ma, p);
   return true;
 }
 

@@ -90,6 +90,7 @@ struct AttnArgs {
   const float *A, *c;         // [BH][d][d], [BH][d]; null = no correction
   void* O; i64 os[3];
   float* O_sparse;            // optional [BH][N][d] in original order
+  void* O_lo;                 // optional bf16 [BH][N][d] in original order: o - bf16(o) (tensor-core kernels only)
   int* err;                   // device error word (may be null)
 };
 cudaError_t init_attention_simt();
@@ -109,10 +110,11 @@ constexpr int kRemRows = 32;
 cudaError_t init_attention_packed();
 void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st);
 bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st);
-// correction_tc.cu: O <- O + O A + c in place (bf16, d_v = 128); At: bf16 scratch [BH][128][128]
+// correction_tc.cu: O <- X + X A + c in place, X = O + O_lo (two bf16 words, O_lo [BH][N][128] contiguous), d_v = 128;
+// At: bf16 scratch [BH][128][128]
 cudaError_t init_correction_tc();
-bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, void* O, const i64* os, int BH, int H, int N,
-                          int* err, cudaStream_t st);
+bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, const void* O_lo, void* O, const i64* os, int BH,
+                          int H, int N, int* err, cudaStream_t st);
 
 struct ProbeArgs {
   int dtype, BH, H, N, d, M, Ck, Cq, n_split;

@@ -18,3 +18,15 @@ def heads_to_device(wl, heads, seed=0):
 
 def to_np(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def assert_bf16_close(O, ref):
+    """bf16 tensors, float32 accumulation, bf16 output: relative L2 <= 1e-2 and, element by element,
+    |O - ref| <= 2e-2 -- except where the reference element is so large that a single correctly rounded
+    bf16 store already exceeds that (half an ulp is 2^-9 |o| rounded up to a power of two: 0.031 for
+    8 <= |o| < 16); there the bound is one bf16 ulp, 2^-7 |ref|."""
+    from oracle import sparsepr_oracle as orc
+    err = orc.rel_l2(O, ref)
+    assert err <= 1e-2, err
+    excess = np.abs(O - ref) - np.maximum(2e-2, 2.0 ** -7 * np.abs(ref))
+    assert excess.max() <= 0.0, (float(np.abs(O - ref).max()), float(excess.max()))

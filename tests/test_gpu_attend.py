@@ -2,7 +2,8 @@
 
 Tolerances (from the arithmetic): float32 inputs with float32 accumulation and a
 2-ulp exp2 -> relative L2 <= 1e-5; bfloat16 inputs with float32 accumulation and
-a bfloat16 output -> max-abs <= 2e-2 and relative L2 <= 1e-2."""
+a bfloat16 output -> relative L2 <= 1e-2 and max-abs <= 2e-2 (one bf16 ulp for elements so large that
+rounding the output alone exceeds 2e-2; see tests/gpu_util.py)."""
 import numpy as np
 import pytest
 import torch
@@ -10,7 +11,7 @@ import torch
 from oracle import sparsepr_oracle as orc
 from paper_2608_18484_b200 import binding as B
 from paper_2608_18484_b200 import workloads as W
-from tests.gpu_util import heads_to_device, to_np
+from tests.gpu_util import assert_bf16_close, heads_to_device, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -31,8 +32,7 @@ def check(O, ref, fp32):
     if fp32:
         assert err <= 1e-5, err
     else:
-        assert err <= 1e-2, err
-        assert np.abs(O - ref).max() <= 2e-2, np.abs(O - ref).max()
+        assert_bf16_close(O, ref)
 
 
 CASES = [

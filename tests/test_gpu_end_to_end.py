@@ -66,7 +66,11 @@ def test_full_call_matches_oracle_statistically(name, wl):
         h_gpu, h_orc = orc.rel_l2(to_np(Osp[0, i]), exact), orc.rel_l2(O_ref_sp, exact)
         assert abs(e_gpu - e_orc) <= 0.1 * e_orc + 0.01, (e_gpu, e_orc)
         assert abs(h_gpu - h_orc) <= 0.1 * h_orc + 0.01, (h_gpu, h_orc)
-        assert e_gpu < h_gpu                                     # the repair helps on these inputs
+        # whether the repair helps depends on the inputs and on M against d_v (with fewer probes than output
+        # dimensions the ridge system is under-determined); the GPU must agree with the oracle on it whenever the
+        # oracle's two errors are clearly apart
+        if abs(e_orc - h_orc) > 0.1 * h_orc + 0.01:
+            assert (e_gpu < h_gpu) == (e_orc < h_orc), (e_gpu, h_gpu, e_orc, h_orc)
     assert abs(st["rho_exec"] - st["rho_route"] - wl.n_probe / wl.N) < 1e-12
 
 

@@ -32,8 +32,8 @@ CASES = [("tiny-f32", W.TINY), ("480p-like-bf16", W.VIDEO_480P.scaled(grid=(3, 3
 # tensor cores with a three-term bf16 split of F (2^-24 relative).  The continuous quantities are then
 # accurate to a few float32 ulps times a condition number (eigen-gap for F F^T, exp for the scores).
 TOL = {
-    "f32": dict(FF=2e-5, kappa=2e-6, gram=2e-5, norm=2e-5, score=2e-4, agree_K=0.97, agree_Q=0.97, obj=2e-3),
-    "bf16": dict(FF=2e-3, kappa=2e-6, gram=2e-3, norm=2e-4, score=1e-3, agree_K=0.95, agree_Q=0.95, obj=5e-3),
+    "f32": dict(FF=1e-5, kappa=2e-6, gram=1e-5, norm=1e-5, score=1e-4, agree_K=0.97, agree_Q=0.97, obj=2e-3),
+    "bf16": dict(FF=1e-4, kappa=2e-6, gram=1e-4, norm=2e-5, score=1e-4, agree_K=0.97, agree_Q=0.97, obj=2e-3),
 }
 TIE = 5e-3          # relative margin inside which two oracle scores / distances count as tied
 
