@@ -195,6 +195,93 @@ def cpu_baseline(wl, gpu_call=None):
 
 
 # --------------------------------------------------------------------------------------
+def sweep(args, wl, kind):
+    """Parameter studies on one GPU (not the default line): prints one JSON object per configuration.
+
+    kind "sweep": density budget x probe rows x {hard drop, probe-fitted}, plus the full-rank (r_out = d_v) and
+    lambda = 10 columns, on the given workload (the 720p-like shape unless --workload says otherwise).
+    kind "cq": number of query groups C_q in {N/128, N/256, N/512} at the workload's density: accuracy against
+    tensor efficiency (executed-pair and issued rates of the block-sparse stage)."""
+    import torch
+    from oracle import sparsepr_oracle as orc
+    from paper_2608_18484_b200 import binding as B
+    from paper_2608_18484_b200 import workloads as W
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    Qd, Kd, Vd = [torch.empty(1, wl.H, wl.N, wl.d, dtype=dt, device=dev) for _ in range(3)]
+    host0 = None
+    for h in range(wl.H):
+        hd = W.make_head(wl, h)
+        if h == 0:
+            host0 = hd
+        for t, x in enumerate(hd):
+            (Qd, Kd, Vd)[t][0, h].copy_(torch.from_numpy(x).to(dt))
+    O, Odense = torch.empty_like(Qd), torch.empty_like(Qd)
+    dprof = B.Profile()
+    B.sparsepr_dense(Qd, Kd, Vd, wl.softmax_scale, out=Odense)
+    for _ in range(2):
+        B.sparsepr_dense(Qd, Kd, Vd, wl.softmax_scale, out=Odense, profile=dprof)
+    dense_ms = dprof.as_dict()["dense"] / 2
+    ref = Odense.float()
+    den = float(ref.norm())
+    # float64 exact rows bound the dense kernel's own error (the reference of the errors below)
+    rows = np.random.default_rng(3).choice(wl.N, 256, replace=False)
+    exact = orc.dense_attention(*host0, wl.softmax_scale, rows=rows)
+    dense_err = orc.rel_l2(Odense[0, 0].float().cpu().numpy()[rows], exact)
+    print(json.dumps({"study": kind, "workload": wl.name, "H": wl.H, "N": wl.N, "dense_ms": dense_ms,
+                      "dense_kernel_rel_l2_vs_fp64_on_256_rows_of_head_0": dense_err,
+                      "peak_tflops_sustained": peaks["bf16_sustained"], "peak_tflops_burst": peaks["bf16_tflops"]}), flush=True)
+
+    def measure(label, steps=3, **kw):
+        params = B.make_params(block=wl.block, n_sample=wl.n_sample, softmax_scale=wl.softmax_scale, **kw)
+        for _ in range(1):
+            plan = B.sparsepr_plan(Qd, Kd, Vd, params=params)
+            B.sparsepr_attend(plan, Qd, Kd, Vd, out=O)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            plan = B.sparsepr_plan(Qd, Kd, Vd, params=params)
+            B.sparsepr_attend(plan, Qd, Kd, Vd, out=O)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        prof = B.Profile()
+        plan = B.sparsepr_plan(Qd, Kd, Vd, params=params, profile=prof)
+        _, Osp = B.sparsepr_attend(plan, Qd, Kd, Vd, out=O, return_sparse=True, profile=prof)
+        st = B.sparsepr_plan_stats(plan)
+        attn_ms = prof.as_dict()["attention"]
+        tf = 4.0 * wl.d * st["routed_pairs"] / (attn_ms * 1e-3) / 1e12
+        row = dict(label, ms=ms, speedup_vs_dense=dense_ms / ms, rho_route=st["rho_route"], rho_exec=st["rho_exec"],
+                   attention_ms=attn_ms, executed_tflops=tf, tensor_frac_sustained=tf / peaks["bf16_sustained"],
+                   tensor_frac_burst=tf / peaks["bf16_tflops"],
+                   issued_tflops=4.0 * wl.d * st["padded_tile_pairs"] / (attn_ms * 1e-3) / 1e12,
+                   tile_padding=st["padded_tile_pairs"] / max(st["routed_pairs"], 1),
+                   rel_l2_hard_drop=float((Osp - ref).norm()) / den, device_error=st["device_error"])
+        if kw.get("mode", 0) == 0:
+            row["rel_l2_probe_fitted"] = float((O.float() - ref).norm()) / den
+        del Osp
+        print(json.dumps(row), flush=True)
+
+    if kind == "sweep":
+        for rho in (0.10, 0.15, 0.22, 0.26, 0.35, 0.50):
+            measure({"rho": rho, "M": 0, "mode": "hard-drop"}, density=rho, n_probe=0, mode=1)
+            for M in (32, 64, 128, 256):
+                measure({"rho": rho, "M": M, "mode": "probe-fitted"}, density=rho, n_probe=M)
+        for M in (32, 64, 128, 256):                      # ridge only (full output rank) and a stronger ridge
+            measure({"rho": wl.density, "M": M, "mode": "probe-fitted, r_out=d_v"}, steps=1, density=wl.density, n_probe=M, r_out=wl.d)
+            measure({"rho": wl.density, "M": M, "mode": "probe-fitted, lambda=10"}, steps=1, density=wl.density, n_probe=M, lam=10.0)
+            measure({"rho": wl.density, "M": M, "mode": "probe-fitted, r_out=d_v, lambda=10"}, steps=1, density=wl.density,
+                    n_probe=M, r_out=wl.d, lam=10.0)
+    else:
+        C = -(-wl.N // wl.block)
+        for div in (1, 2, 4):
+            measure({"C_q": -(-C // div), "C_k": C, "rows_per_query_group": wl.block * div}, density=wl.density,
+                    n_probe=wl.n_probe, Cq=-(-C // div), Ck=C)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -205,6 +292,8 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--study", default="", choices=["", "sweep", "cq"],
+                    help="parameter study instead of the benchmark line: density x probes x mode, or the C_q frontier")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -214,6 +303,9 @@ def main():
         wl = wl.scaled(H=args.heads)
     if args.impl == "reference":
         reference_arm(args, wl)
+        return
+    if args.study:
+        sweep(args, wl, args.study)
         return
 
     import torch

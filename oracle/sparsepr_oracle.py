@@ -15,8 +15,9 @@ Readings taken where the paper is silent (each is repeated at the function):
   * deterministic query sample / k-means init rows: an integer stride rule with
     a splitmix64 offset (`stride_sample`);
   * k-means: Lloyd iterations from data-point initial centroids, ties to the
-    lowest centroid id, empty clusters keep their previous centroid
-    (`kmeans`);
+    lowest centroid id, empty clusters keep their previous centroid; a warm
+    start seeds the centroids with the current features' means over a previous
+    call's partition (`kmeans`);
   * router score: centroid estimate of the per-key attention weight of a cell
     (`cell_scores`), forced arg-max cell per non-empty query group, then the
     longest prefix of the score-sorted remaining cells that fits the pair
@@ -241,15 +242,30 @@ def kmeans_assign(X, mu, chunk: int = 1024) -> np.ndarray:
     return a
 
 
-def kmeans(X, C: int, init_rows, T: int):
+def kmeans(X, C: int, init_rows, T: int, init_assign=None):
     """Lloyd's algorithm.  Reading (the paper fixes none of this): initial
     centroids are the feature rows `init_rows`; for t = 1..T assign, and if
     t < T move every non-empty cluster to the mean of its members while an
     empty cluster keeps its previous centroid.  Returns (a^(T), the centroids
-    used by the last assignment)."""
+    used by the last assignment).
+
+    Warm start (Appendix C.1 only says the k-means is "warm-started"; reading):
+    with `init_assign`, the partition of a previous call over the same token
+    grid, the initial centroid of cluster c is the mean of the CURRENT features
+    of the tokens that partition put in c; a cluster it left empty starts from
+    its feature row of `init_rows`.  Seeding by assignment rather than by the
+    previous centroids keeps the start independent of the sign and rotation
+    gauge of the feature map, which may change between calls."""
     X = np.asarray(X, dtype=np.float64)
     mu = X[np.asarray(init_rows, dtype=np.int64)].copy()
     assert mu.shape[0] == C
+    if init_assign is not None:
+        a0 = np.asarray(init_assign)
+        n0 = np.bincount(a0, minlength=C)
+        s0 = np.zeros_like(mu)
+        np.add.at(s0, a0, X)
+        nz0 = n0 > 0
+        mu[nz0] = s0[nz0] / n0[nz0, None]
     a = None
     for t in range(1, T + 1):
         a = kmeans_assign(X, mu)
@@ -470,11 +486,12 @@ def default_params(**kw):
     return p
 
 
-def plan_head(Q, K, prm: dict, bh: int):
+def plan_head(Q, K, prm: dict, bh: int, warm=None):
     """Stages 1-2 of the call for one head: Response-Coupled Partitioning,
     permutations, probe selection and routing.  Returns a dict of every
     intermediate (so that single stages of another implementation can be fed
-    from it)."""
+    from it).  `warm` = {"a_K": ..., "a_Q": ...}, the partition of a previous
+    call, warm-starts both k-means runs (see `kmeans`)."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     N, d = Q.shape
@@ -489,12 +506,14 @@ def plan_head(Q, K, prm: dict, bh: int):
     M_K = key_response_metric(Q[s_idx])
     F_K, lam_K = eig_feature_map(M_K, prm["rK"])
     phi_K = key_response(K, F_K)
-    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, bh), prm["kmeans_iters"])
+    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, bh), prm["kmeans_iters"],
+                       init_assign=None if warm is None else warm["a_K"])
     kappa, n_k = kv_centroids(K, a_K, C_k)
     M_Q = query_response_metric(kappa, n_k)
     F_Q, lam_Q = eig_feature_map(M_Q, prm["rQ"])
     phi_Q = query_response(Q, F_Q, prm["eps_rms"])
-    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), prm["kmeans_iters"])
+    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), prm["kmeans_iters"],
+                       init_assign=None if warm is None else warm["a_Q"])
     theta, n_q = query_centroids(Q, a_Q, C_q)
 
     q_perm, q_inv, q_off = group_permutation(a_Q, C_q)

@@ -151,6 +151,36 @@ def test_kmeans_matches_sklearn_lloyd():
     assert np.allclose(mu, km.cluster_centers_, atol=1e-10)
 
 
+def test_kmeans_warm_start():
+    """Warm start from a previous partition: the seeds are the group means of the current features (checked
+    against sklearn's Lloyd started from independently computed means), a cluster the previous partition left
+    empty starts from its strided row, and a planted partition is a fixed point that one pass reproduces."""
+    sk = pytest.importorskip("sklearn.cluster")
+    rng = np.random.default_rng(16)
+    X = rng.normal(size=(400, 5))
+    init = orc.stride_sample(8, 400, 0, 2, 0)
+    prev = rng.integers(0, 8, size=400)
+    prev[prev == 3] = 4                                           # cluster 3 empty in the previous partition
+    seeds = np.stack([X[prev == c].mean(0) if (prev == c).any() else X[init[c]] for c in range(8)])
+    km = sk.KMeans(n_clusters=8, init=seeds, n_init=1, algorithm="lloyd", max_iter=3, tol=0.0).fit(X)
+    a, mu = orc.kmeans(X, 8, init, T=4, init_assign=prev)
+    assert np.array_equal(a, km.labels_) and np.allclose(mu, km.cluster_centers_, atol=1e-10)
+    a1, mu1 = orc.kmeans(X, 8, init, T=1, init_assign=prev)
+    assert np.array_equal(a1, orc.kmeans_assign(X, seeds)) and np.allclose(mu1, seeds)
+    # well separated planted clusters: the planted partition reproduces itself in one pass, whatever the strided rows are
+    centers = rng.normal(size=(6, 4)) * 20.0
+    lab = rng.integers(0, 6, size=300)
+    Y = centers[lab] + rng.normal(size=(300, 4)) * 0.1
+    a2, _ = orc.kmeans(Y, 6, orc.stride_sample(6, 300, 0, 3, 1), T=1, init_assign=lab)
+    assert np.array_equal(a2, lab)
+    # the objective does not rise along a warm-started run either
+    objs = []
+    for T in range(1, 6):
+        aT, muT = orc.kmeans(X, 8, init, T=T, init_assign=prev)
+        objs.append(orc.kmeans_objective(X, muT, aT))
+    assert all(objs[i + 1] <= objs[i] + 1e-9 for i in range(len(objs) - 1))
+
+
 def test_group_permutation():
     rng = np.random.default_rng(7)
     a = rng.integers(0, 9, size=100)
