@@ -183,6 +183,26 @@ sparsepr_status_t sparsepr_plan(const sparsepr_shape_t* shape, const sparsepr_pa
                                 void* workspace, size_t workspace_bytes, void* cuda_stream,
                                 sparsepr_plan_t** out);
 
+/* The same with warm-started k-means (Appendix C.1: "warm-started GPU k-means"), for a sequence of calls over
+ * the same token grid, e.g. successive denoising steps.  prev_kv_assign, prev_q_assign: DEVICE int32 [B*H, N], the
+ * partition of an earlier call (group ids in [0, C_k) and [0, C_q); other values are ignored).  The initial centroid
+ * of a group is the mean of the CURRENT features of the tokens that partition put into it; a group it left empty
+ * starts from its strided sample row as in sparsepr_plan.  Seeding by assignment rather than by centroids makes the
+ * start independent of the sign gauge of the eigenvectors behind the feature maps, which can change between calls.
+ * params->kmeans_iters still counts the assignment passes, and fewer are needed (the benchmark's warm leg uses 2).
+ * The arrays may live in an earlier plan's workspace (see sparsepr_plan_assignments); they are read by work queued
+ * on `cuda_stream` and must stay valid until that work is complete. */
+sparsepr_status_t sparsepr_plan_warm(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                     const void* Q, const void* K, const void* V,
+                                     const int32_t* prev_kv_assign, const int32_t* prev_q_assign,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                     sparsepr_plan_t** out);
+
+/* DEVICE pointers to the partition inside the plan's workspace: int32 [B*H, N] each, valid while the workspace
+ * lives; their contents are final once the work of the plan call is complete on its stream. */
+sparsepr_status_t sparsepr_plan_assignments(const sparsepr_plan_t* plan, const int32_t** kv_assign,
+                                            const int32_t** q_assign);
+
 /* Stages 3-4 (Eq. 3, Eq. 8-10): O (DEVICE, written in original token order) from
  * Q, K, V (DEVICE) and a plan.  `workspace`: DEVICE, sparsepr_attend_workspace_bytes,
  * 256-byte aligned; its contents are scratch.  `O_sparse` (DEVICE, float32

@@ -72,7 +72,7 @@ class Profile(C.Structure):
 
 EXPORTS = ["sparsepr_stage_assign_static", "sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
-           "sparsepr_plan_export_features",
+           "sparsepr_plan_export_features", "sparsepr_plan_warm", "sparsepr_plan_assignments",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
 
@@ -95,6 +95,8 @@ def lib():
         L.sparsepr_attend.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.sparsepr_dense.argtypes = [C.POINTER(Shape), C.c_float, vp, vp, vp, vp, vp]
         L.sparsepr_plan_timed.argtypes = L.sparsepr_plan.argtypes + [C.POINTER(Profile)]
+        L.sparsepr_plan_warm.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, sz, vp, C.POINTER(vp)]
+        L.sparsepr_plan_assignments.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
         L.sparsepr_attend_timed.argtypes = L.sparsepr_attend.argtypes + [C.POINTER(Profile)]
         L.sparsepr_dense_timed.argtypes = L.sparsepr_dense.argtypes + [C.POINTER(Profile)]
         L.sparsepr_plan_stats.argtypes = [vp, C.POINTER(Stats)]
@@ -185,9 +187,11 @@ class Plan:
             self.handle = None
 
 
-def sparsepr_plan(Q, K, V=None, params: Params | None = None, profile: Profile | None = None, **kw) -> Plan:
+def sparsepr_plan(Q, K, V=None, params: Params | None = None, profile: Profile | None = None,
+                  warm_from: "Plan | None" = None, **kw) -> Plan:
     """Stages 1-2: partition, permutations, probe set and routes for every head.
-    With `profile` the timed entry point is used and per-stage milliseconds are added to it."""
+    With `profile` the timed entry point is used and per-stage milliseconds are added to it.
+    With `warm_from` (an earlier plan over the same token grid) both k-means runs start from that plan's partition."""
     params = params or make_params(**kw)
     shape = make_shape(Q, K, K if V is None else V, Q)
     L = lib()
@@ -198,11 +202,21 @@ def sparsepr_plan(Q, K, V=None, params: Params | None = None, profile: Profile |
     handle = C.c_void_p()
     args = (C.byref(shape), C.byref(params), Q.data_ptr(), K.data_ptr(), None if V is None else V.data_ptr(),
             ws.data_ptr(), ws.numel(), _stream(), C.byref(handle))
-    if profile is None:
+    keep = None
+    if warm_from is not None:
+        if profile is not None:
+            raise ValueError("the warm-started plan has no timed variant")
+        pk, pq = C.c_void_p(), C.c_void_p()
+        _check(L.sparsepr_plan_assignments(warm_from.handle, C.byref(pk), C.byref(pq)), "sparsepr_plan_assignments")
+        _check(L.sparsepr_plan_warm(*args[:5], pk, pq, *args[5:]), "sparsepr_plan_warm")
+        keep = warm_from.workspace                   # read by queued work: keep the earlier workspace alive with this plan
+    elif profile is None:
         _check(L.sparsepr_plan(*args), "sparsepr_plan")
     else:
         _check(L.sparsepr_plan_timed(*args, C.byref(profile)), "sparsepr_plan_timed")
-    return Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
+    plan = Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
+    plan.warm_source = keep
+    return plan
 
 
 def sparsepr_attend(plan: Plan, Q, K, V, out=None, return_sparse=False, profile: Profile | None = None):

@@ -42,6 +42,7 @@ struct Carver {                       // bump allocator over a caller-owned work
 struct Resolved {
   int B, H, BH, N, d, dtype, es;
   int Ck, Cq, Cmax, Ms, M, rK, rQ, RK, RQ, Rmax, r_out, T, mode;
+  bool full_rank;                      // r_out covers the whole row space of the probe residuals: the projector is the identity
   float density, lambda, eps_rms, eps_std, scale;
   u64 seed;
   i64 qs[3], ks[3], vs[3], os[3];
@@ -82,7 +83,15 @@ sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p,
   r->rQ = std::min(p->rQ ? p->rQ : 64, s->d);
   if (r->rK > kMaxRank || r->rQ > kMaxRank) return SPARSEPR_ERR_UNSUPPORTED;
   r->RK = round16(r->rK); r->RQ = round16(r->rQ); r->Rmax = std::max(r->RK, r->RQ);
-  r->r_out = std::max(1, std::min(p->r_out ? p->r_out : 16, std::min(std::max(r->M, 1), s->d)));
+  {
+    // r = min(r_out, M, d_v).  Once r reaches min(M, d_v) it spans every direction the probe residuals (M rows in
+    // d_v dimensions) can have, the projector acts as the identity and no eigenvectors are needed; below that the
+    // eigen-solver delivers at most kMaxRank of them.
+    const int want = p->r_out ? p->r_out : 16, cap = std::min(std::max(r->M, 1), s->d);
+    r->full_rank = want >= cap;
+    r->r_out = std::max(1, std::min(want, cap));
+    if (!r->full_rank && r->r_out > kMaxRank) return SPARSEPR_ERR_UNSUPPORTED;
+  }
   r->T = p->kmeans_iters ? p->kmeans_iters : 8;
   r->density = p->density;
   r->lambda = p->lambda < 0.f ? 0.1f : p->lambda;
@@ -330,7 +339,7 @@ i64 pair_budget(const Resolved& r) {
   return std::max<i64>(total - (i64)r.M * r.N, 0);
 }
 
-void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cudaStream_t st) {
+void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, const int* warm_prev, cudaStream_t st) {
   const Resolved& R = p->r;
   const int ld = round16(r);
   // changed[t][bh], t = 1..T: rows of head bh that changed group in pass t.  A pass that changes nothing proves the
@@ -341,7 +350,9 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, cu
   const bool tcp = kmeans_tc_supported();
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
   // (with the tensor-core assignment the finalize step also writes the two bf16 words of every centroid)
-  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
+  // warm start: the initial centroids become the means of the current features over the previous partition's groups
+  if (warm_prev) launch_kmeans_warm_sums(p->phi, ld, R.BH, R.N, r, C, warm_prev, p->sums, p->counts, p->fx_shift, st);
+  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, warm_prev ? 1 : 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
@@ -448,7 +459,8 @@ void join_side(const sparsepr_plan_s* p, cudaStream_t st) {
 
 static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
                                    const void* K, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                                   sparsepr_plan_t** out, sparsepr_profile_t* prof) {
+                                   sparsepr_plan_t** out, sparsepr_profile_t* prof, const int* warm_kv = nullptr,
+                                   const int* warm_q = nullptr) {
   if (!Q || !K) return SPARSEPR_ERR_INVALID_ARG;
   sparsepr_plan_s* p = nullptr;
   sparsepr_status_t s = make_plan(shape, params, workspace, workspace_bytes, cuda_stream, &p);
@@ -469,7 +481,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
     launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
   }
   tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
-  run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, st);
+  run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, warm_kv, st);
   tm.mark(SPARSEPR_STAGE_KEY_KMEANS);
   launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
   launch_group_means(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
@@ -485,7 +497,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
     launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
   }
   tm.mark(SPARSEPR_STAGE_QUERY_PROJECT);
-  run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, st);
+  run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, warm_q, st);
   tm.mark(SPARSEPR_STAGE_QUERY_KMEANS);
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
   launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
@@ -524,6 +536,22 @@ sparsepr_status_t sparsepr_plan_timed(const sparsepr_shape_t* shape, const spars
   (void)V;
   if (!profile) return SPARSEPR_ERR_INVALID_ARG;
   return plan_impl(shape, params, Q, K, workspace, workspace_bytes, cuda_stream, out, profile);
+}
+
+sparsepr_status_t sparsepr_plan_warm(const sparsepr_shape_t* shape, const sparsepr_params_t* params, const void* Q,
+                                     const void* K, const void* V, const int32_t* prev_kv_assign,
+                                     const int32_t* prev_q_assign, void* workspace, size_t workspace_bytes,
+                                     void* cuda_stream, sparsepr_plan_t** out) {
+  (void)V;
+  if (!prev_kv_assign || !prev_q_assign) return SPARSEPR_ERR_INVALID_ARG;
+  return plan_impl(shape, params, Q, K, workspace, workspace_bytes, cuda_stream, out, nullptr, prev_kv_assign, prev_q_assign);
+}
+
+sparsepr_status_t sparsepr_plan_assignments(const sparsepr_plan_t* p, const int32_t** kv_assign, const int32_t** q_assign) {
+  if (!p || !kv_assign || !q_assign) return SPARSEPR_ERR_INVALID_ARG;
+  *kv_assign = p->a_K;
+  *q_assign = p->a_Q;
+  return SPARSEPR_OK;
 }
 
 sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
@@ -615,7 +643,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     }
     tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
-    fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;
+    fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.full_rank = r.full_rank; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;
     fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
     launch_fit(fa, fs);
     tm.mark(SPARSEPR_STAGE_FIT);

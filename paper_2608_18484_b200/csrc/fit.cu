@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(256) k_fit_compose(FitArgs a, int r) {
   const float* Psi = a.Psi + (i64)bh * d * r;
   const double* Bm = sc + L.B;
   double* T = sc + L.T;
-  for (int e = threadIdx.x; e < d * r; e += 256) {
+  for (int e = threadIdx.x; e < d * r && !a.full_rank; e += 256) {
     const int i = e / r, t = e % r;
     double s = 0.0;
     for (int k = 0; k < d; ++k) s += Bm[(size_t)i * d + k] * (double)Psi[k * r + t];
@@ -225,7 +225,11 @@ __global__ void __launch_bounds__(256) k_fit_compose(FitArgs a, int r) {
   for (int e = threadIdx.x; e < d * d; e += 256) {
     const int i = e / d, j = e % d;
     double s = 0.0;
-    for (int t = 0; t < r; ++t) s += T[i * r + t] * (double)Psi[j * r + t];
+    if (a.full_rank) {
+      s = Bm[e];                           // every row of B lies in the row space of the probe residuals: B Psi Psi^T = B
+    } else {
+      for (int t = 0; t < r; ++t) s += T[i * r + t] * (double)Psi[j * r + t];
+    }
     s *= rs_x[i];
     Ad[e] = s;
     A[e] = (float)s;
@@ -259,7 +263,7 @@ void launch_fit(const FitArgs& a, cudaStream_t st) {
     k_fit_solve<float><<<a.BH, 1024, (size_t)d * (d + 1) * 4, st>>>(a);
   }
   // Psi_r: leading eigenvectors of S = Rb^T W Rb, i.e. right singular vectors of W^(1/2) Rb.
-  launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, st);
+  if (!a.full_rank) launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, st);
   k_fit_compose<<<a.BH, 256, 0, st>>>(a, r);
 }
 

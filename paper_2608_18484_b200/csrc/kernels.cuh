@@ -23,6 +23,8 @@ void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int 
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
+void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, int C, const int* prev, i64* sums,
+                             int* counts, const int* fx_shift, cudaStream_t st);
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh = nullptr, __nv_bfloat16* ml = nullptr);
 // prev_changed / cur_changed [BH] (may be null): number of rows of each head whose assignment changed in the previous
@@ -138,6 +140,7 @@ void launch_write_probe_rows(int dtype, const float* Dn, const int* probe_idx, i
 // ---- fit.cu -----------------------------------------------------------------------
 struct FitArgs {
   int BH, M, d, r_out;
+  bool full_rank;                      // r_out >= min(M, d): Psi Psi^T acts as the identity, no eigenvectors are computed
   float lambda, eps_std;
   bool precise;                        // float64 eigen-solver for the subspace
   const float *X, *Dn, *w;             // [BH][M][d], [BH][M][d], [BH][M]

@@ -399,6 +399,52 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
   }
 }
 
+// Warm start (Appendix C.1): fixed-point sums and counts of the CURRENT features over the groups of a previous
+// partition `prev` [BH][N]; the update step that follows turns them into the initial centroids (a group that the
+// previous partition left empty keeps the strided row k_kmeans_init gave it).  One warp per 32 consecutive rows,
+// lanes = feature columns (2 lane, 2 lane + 1), one atomic per (cluster present in the warp, column).  Entries of
+// `prev` outside [0, C) are ignored.
+__global__ void __launch_bounds__(256) k_kmeans_warm_sums(const float* __restrict__ phi, int ldphi, int N, int r, int R, int C,
+                                                          const int* __restrict__ prev, i64* __restrict__ sums,
+                                                          int* __restrict__ counts, const int* __restrict__ fx_shift) {
+  const unsigned FULL = 0xffffffffu;
+  const int bh = blockIdx.y, lane = threadIdx.x & 31;
+  const int rowbase = (blockIdx.x * 8 + (threadIdx.x >> 5)) * 32;
+  if (rowbase >= N) return;
+  const int row = rowbase + lane;
+  int cl_mine = -1;
+  if (row < N) { const int c = prev[(i64)bh * N + row]; if (c >= 0 && c < C) cl_mine = c; }
+  const bool cok = 2 * lane < r;
+  float pv0[32], pv1[32];
+#pragma unroll
+  for (int rr = 0; rr < 32; ++rr) {
+    const int rw = min(rowbase + rr, N - 1);
+    const float2 x2 = cok ? *reinterpret_cast<const float2*>(phi + ((i64)bh * N + rw) * ldphi + 2 * lane) : make_float2(0.f, 0.f);
+    pv0[rr] = x2.x; pv1[rr] = x2.y;
+  }
+  const float scl = __int_as_float((127 + fx_shift[bh]) << 23);
+  unsigned todo = __ballot_sync(FULL, cl_mine >= 0);
+  while (todo) {
+    const int leader = __ffs(todo) - 1;
+    const int cl = __shfl_sync(FULL, cl_mine, leader);
+    const unsigned members = __ballot_sync(FULL, cl_mine == cl) & todo;
+    todo &= ~members;
+    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+    for (int rr = 0; rr < 32; ++rr)
+      if ((members >> rr) & 1u) { a0 += pv0[rr]; a1 += pv1[rr]; }
+    i64* sp = sums + ((i64)bh * C + cl) * R;
+    if (2 * lane < r) atomicAdd(reinterpret_cast<u64*>(sp + 2 * lane), (u64)__float2ll_rn(a0 * scl));
+    if (2 * lane + 1 < r) atomicAdd(reinterpret_cast<u64*>(sp + 2 * lane + 1), (u64)__float2ll_rn(a1 * scl));
+    if (lane == 0) atomicAdd(counts + (i64)bh * C + cl, __popc(members));
+  }
+}
+void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, int C, const int* prev, i64* sums,
+                             int* counts, const int* fx_shift, cudaStream_t st) {
+  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  k_kmeans_warm_sums<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(phi, ldphi, N, r, R, C, prev, sums, counts, fx_shift);
+}
+
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st) {
   const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;

@@ -116,9 +116,11 @@ def _sigma(wl: Workload):
     return np.where(t < T // 3, 0.3, 1.0)[:, None]       # conditioning frames vs prediction frames
 
 
-def make_head(wl: Workload, head: int, seed: int = 0):
+def make_head(wl: Workload, head: int, seed: int = 0, step: int = 0):
     """Q, K, V of one head as float32 arrays [N, d] whose values are exactly
-    representable in the workload's storage type."""
+    representable in the workload's storage type.  `step` > 0 keeps the centroid
+    tables of (seed, head) and draws fresh noise: successive calls over the same
+    scene, the stand-in for successive denoising steps."""
     cmap = _CLUSTER_MAPS[wl.cluster_map](wl.grid, head, wl.H)
     n_c = int(cmap.max()) + 1
     sig = _sigma(wl)
@@ -128,6 +130,8 @@ def make_head(wl: Workload, head: int, seed: int = 0):
         rng = np.random.default_rng([seed, wl.cfg_id, head, tensor_id])
         mu = rng.standard_normal((n_c, wl.d), dtype=np.float32)
         eps = rng.standard_normal((wl.N, wl.d), dtype=np.float32)
+        if step:
+            eps = np.random.default_rng([seed, wl.cfg_id, head, tensor_id, step]).standard_normal((wl.N, wl.d), dtype=np.float32)
         if tensor_id == 1 and wl.qk_align != 0.0:       # keys: aligned with the query centroids
             c = np.float32(wl.qk_align)
             mu = c * tables[0] + np.sqrt(np.float32(1.0) - c * c) * mu

@@ -5,9 +5,9 @@ import torch
 from paper_2608_18484_b200 import workloads as W
 
 
-def heads_to_device(wl, heads, seed=0):
+def heads_to_device(wl, heads, seed=0, step=0):
     """Returns (host list of (Q,K,V) float32 arrays, device tensors [1,H,N,d] in the workload dtype)."""
-    host = [W.make_head(wl, h, seed) for h in heads]
+    host = [W.make_head(wl, h, seed, step) for h in heads]
     dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     dev = []
     for t in range(3):

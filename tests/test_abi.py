@@ -58,6 +58,10 @@ def test_workspace_sizes_scale_and_reject(lib):
     assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(density=0.0))) == 0
     assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape(N=100)), C.byref(B.make_params(Ck=200))) == 0
     assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(n_probe=5000))) == 0
+    # output rank of the probe-residual subspace: up to 64 eigenvectors, or the full space (no eigenvectors needed)
+    assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(n_probe=128, r_out=100))) == 0
+    assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(n_probe=128, r_out=128))) > 0
+    assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(n_probe=96, r_out=128))) > 0
     assert lib.sparsepr_stage_assign_workspace_bytes(1000, 10, 48) > 1000 * 48 * 4
     assert lib.sparsepr_stage_assign_workspace_bytes(1000, 10, 65) == 0
 
@@ -71,6 +75,8 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert lib.sparsepr_plan(C.byref(s), C.byref(p), 256, 256, None, None, 0, None, C.byref(h)) == 3      # no workspace
     assert lib.sparsepr_plan(C.byref(s), C.byref(p), 256, 256, None, 256, 1024, None, C.byref(h)) == 3   # too small
     assert lib.sparsepr_plan(C.byref(s), C.byref(p), 256, 256, None, 128, 1 << 40, None, C.byref(h)) == 3  # misaligned
+    assert lib.sparsepr_plan_warm(C.byref(s), C.byref(p), 256, 256, None, None, 256, 256, 1 << 40, None, C.byref(h)) == 1
+    assert lib.sparsepr_plan_assignments(None, None, None) == 1
     assert lib.sparsepr_attend(None, 256, 256, 256, 256, None, 256, 0, None) == 1
     assert lib.sparsepr_dense(C.byref(s), 0.0, None, 256, 256, 256, None) == 1
     assert lib.sparsepr_dense(C.byref(bad), 0.0, 256, 256, 256, 256, None) == 2

@@ -43,6 +43,9 @@ CASES = [
     ("720p-like-bf16", W.VIDEO_720P.scaled(grid=(2, 45, 80), H=2, n_probe=64), dict()),
     ("480p-like-bf16-sparser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.12), dict()),
     ("480p-like-bf16-denser", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=64, density=0.35), dict(r_out=128)),
+    # output rank r = min(r_out, M, d_v) above the 64 eigenvectors the solver delivers: the projector is the identity
+    ("480p-like-bf16-full-rank", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=128), dict(r_out=128)),
+    ("480p-like-bf16-rank-96", W.VIDEO_480P.scaled(grid=(3, 30, 52), H=2, n_probe=96), dict(r_out=128, lam=10.0)),
     # 38 key tiles over 9 probe slices of 5 tiles: the last slice is empty and must not contribute
     ("480p-like-bf16-empty-probe-slice", W.VIDEO_480P.scaled(grid=(3, 30, 53), H=2, n_probe=64), dict()),
 ]

@@ -42,12 +42,13 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / np.linalg.norm(b))
 
 
-def plan_links(wl, i, Q, K, exp, feat, prm):
-    """Everything the assertions need for head i: GPU quantities beside the oracle's evaluation of each link."""
+def plan_links(wl, i, Q, K, exp, feat, prm, warm=None):
+    """Everything the assertions need for head i: GPU quantities beside the oracle's evaluation of each link.
+    `warm` = the partition {"a_K", "a_Q"} that a warm-started GPU plan was seeded with."""
     N, d = Q.shape
     C = -(-N // wl.block)
     out = {}
-    ref = orc.plan_head(Q, K, prm, i)
+    ref = orc.plan_head(Q, K, prm, i, warm=warm)
     aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
     # a1-a3
     FK = feat["F_K"][i].astype(np.float64)
@@ -69,7 +70,8 @@ def plan_links(wl, i, Q, K, exp, feat, prm):
     out["gram"] = rel_fro(phi_gpu[rows] @ phi_gpu[rows].T, phi_ref[rows] @ phi_ref[rows].T)
     out["norm"] = float(np.abs((phi_gpu ** 2).sum(axis=1) / phi_ref.shape[1] - 1.0).max())
     # a7
-    aQ_ref, _ = orc.kmeans(phi_ref, C, orc.stride_sample(C, N, prm["seed"], orc.TAG_Q_INIT, i), prm["kmeans_iters"])
+    aQ_ref, _ = orc.kmeans(phi_ref, C, orc.stride_sample(C, N, prm["seed"], orc.TAG_Q_INIT, i), prm["kmeans_iters"],
+                           init_assign=None if warm is None else warm["a_Q"])
     out["agree_Q"] = float((aQ == aQ_ref).mean())
     out["obj_Q"] = orc.kmeans_objective(phi_ref, _means(phi_ref, aQ, C), aQ) / \
         orc.kmeans_objective(phi_ref, _means(phi_ref, aQ_ref, C), aQ_ref) - 1.0
@@ -158,10 +160,7 @@ def run_case(wl):
     return st, [plan_links(wl, i, Q, K, exp, feat, prm) for i, (Q, K, V) in enumerate(host)]
 
 
-@pytest.mark.parametrize("name,wl", CASES, ids=[c[0] for c in CASES])
-def test_every_plan_link_matches_the_oracle(name, wl):
-    st, links = run_case(wl)
-    assert st["device_error"] == 0
+def check_links(wl, links):
     t = TOL[wl.dtype]
     for m in links:
         # continuous quantities
@@ -178,3 +177,38 @@ def test_every_plan_link_matches_the_oracle(name, wl):
         # probes (Algorithm A.1, Appendix A.2): group sequence, counts and weights exactly; members up to ties
         assert m["probe_distinct"] and m["probe_groups_equal"] and m["probe_m_equal"] and m["probe_w_equal"], m
         assert m["probe_slack"] <= TIE and m["probe_order_ok"], m
+
+
+@pytest.mark.parametrize("name,wl", CASES, ids=[c[0] for c in CASES])
+def test_every_plan_link_matches_the_oracle(name, wl):
+    st, links = run_case(wl)
+    assert st["device_error"] == 0
+    check_links(wl, links)
+
+
+@pytest.mark.parametrize("name,wl", CASES, ids=[c[0] for c in CASES])
+def test_warm_started_plan_matches_the_oracle(name, wl):
+    """Two calls over the same scene (same centroid tables, fresh noise).  The second plan starts both k-means runs
+    from the first plan's partition and runs 3 passes; the oracle, seeded with the GPU's first partition, must
+    arrive at the same plan link by link.  Warm and cold plans must also differ (the seed is really used)."""
+    heads = [0, 1]
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale)
+    _, (Q1, K1, V1) = heads_to_device(wl, heads)
+    first = B.sparsepr_plan(Q1, K1, V1, **kw)
+    e1 = B.sparsepr_plan_export(first)
+    host2, (Q2, K2, V2) = heads_to_device(wl, heads, step=1)
+    kw3 = dict(kw, kmeans_iters=3)
+    second = B.sparsepr_plan(Q2, K2, V2, warm_from=first, **kw3)
+    st = B.sparsepr_plan_stats(second)
+    assert st["device_error"] == 0
+    exp, feat = B.sparsepr_plan_export(second), B.sparsepr_plan_export_features(second)
+    prm = orc.default_params(**kw3)
+    links = [plan_links(wl, i, Q, K, exp, feat, prm, warm=dict(a_K=e1["kv_assign"][i], a_Q=e1["q_assign"][i]))
+             for i, (Q, K, V) in enumerate(host2)]
+    check_links(wl, links)
+    cold = B.sparsepr_plan_export(B.sparsepr_plan(Q2, K2, V2, **kw3))
+    assert not np.array_equal(cold["kv_assign"], exp["kv_assign"])
+    # the warm plan drives a full call
+    O = B.sparsepr_attend(second, Q2, K2, V2)
+    assert bool(np.isfinite(O.float().cpu().numpy()).all())
