@@ -295,6 +295,7 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
       }
       float s[64];
       float mx = -INFINITY;
+      bool lim_neg[4] = {true, true, true, true};              // box bx holds no key that this row may see
       if (ok) {
         tc_fence_after();
         const Meta& mt = meta[i & 7];
@@ -319,6 +320,7 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
         mbar_arrive(bar(S_FREE + (i & 1)));                         // the scores are in registers
 #pragma unroll
         for (int bx = 0; bx < 4; ++bx) {
+          lim_neg[bx] = lim[bx] < 0;
 #pragma unroll
           for (int c = 0; c < 16; ++c) s[bx * 16 + c] = (c <= lim[bx]) ? s[bx * 16 + c] : -INFINITY;
         }
@@ -339,11 +341,20 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
       const float m_new = move ? mx : m_ref;
       const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f;      // 0 when the reference was -inf
       const float mneg = m_new > -INFINITY ? -m_new * sc : 0.f;
+      // O has to be rescaled only for a row that already holds something: a row that meets its first routed key in
+      // this tile (rows of a packed tile do so at different tiles) still has an all-zero accumulator
+      const bool rescale = move && m_ref > -INFINITY;
       m_ref = m_new;
-      if (i > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
-      if (!ok) continue;
-      tc_fence_after();
-      if (i > 0 && __any_sync(FULL, move)) {
+      // The product P V of the previous tile must be complete before P (a single buffer) is overwritten, and before O
+      // is rescaled.  The rescale is rare, so the wait normally comes after the exponentials, which then run while
+      // the tensor cores still work on the previous tile.
+      bool p_free = i == 0;
+      if (!__all_sync(FULL, ok)) { ok = false; continue; }
+      if (i > 0 && __any_sync(FULL, rescale)) {
+        ok = __all_sync(FULL, mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
+        if (!ok) continue;
+        p_free = true;
+        tc_fence_after();
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
           float t[32];
@@ -354,22 +365,37 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
         }
       }
       // exponentials: kPolyOf8 of every 8 pairs on the FMA pipe, the others on the special-function unit;
-      // masked columns give exactly 0 on both
+      // masked columns give exactly 0 on both.  A box that no row of this warp routes to (a warp holds the
+      // remainders of few query groups, and a group routes to a fraction of the K/V groups) is all zeros:
+      // its exponentials are skipped for the whole warp.
       float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       const float2 sc2 = make_float2(sc, sc), mneg2 = make_float2(mneg, mneg);
 #pragma unroll
-      for (int q = 0; q < 32; ++q) {
-        float2 x = __ffma2_rn(make_float2(s[2 * q], s[2 * q + 1]), sc2, mneg2);
-        if ((q & 7) < kPolyOf8) x = ex2_poly2(x);
-        else { x.x = ex2(x.x); x.y = ex2(x.y); }
-        s[2 * q] = x.x; s[2 * q + 1] = x.y;
-        ps2[q & 1] = __fadd2_rn(ps2[q & 1], x);
+      for (int bx = 0; bx < 4; ++bx) {
+        if (__all_sync(FULL, lim_neg[bx])) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) s[bx * 16 + c] = 0.f;
+        } else {
+#pragma unroll
+          for (int q = bx * 8; q < bx * 8 + 8; ++q) {
+            float2 x = __ffma2_rn(make_float2(s[2 * q], s[2 * q + 1]), sc2, mneg2);
+            if ((q & 7) < kPolyOf8) x = ex2_poly2(x);
+            else { x.x = ex2(x.x); x.y = ex2(x.y); }
+            s[2 * q] = x.x; s[2 * q + 1] = x.y;
+            ps2[q & 1] = __fadd2_rn(ps2[q & 1], x);
+          }
+        }
       }
       l = l * corr + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
       {
         uint32_t w[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) w[c] = pack_bf16x2(s[2 * c], s[2 * c + 1]);
+        if (!p_free) {
+          ok = __all_sync(FULL, mbar_wait(bar(P_EMPTY), (i - 1) & 1, abort_flag));
+          if (!ok) continue;
+          tc_fence_after();
+        }
         tmem_st32u(p_addr, w);
       }
       tc_fence_before();
