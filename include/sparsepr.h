@@ -298,6 +298,14 @@ sparsepr_status_t sparsepr_stage_route(int32_t Cq, int32_t Ck, const float* scor
                                        int32_t select_all, int32_t* route_ptr, int32_t* route_idx,
                                        int64_t* pairs_out, void* cuda_stream);
 
+/* Self-test of the bounded device waits.  Every wait of a tensor-core kernel on an mbarrier gives up after a
+ * cycle limit, records SPARSEPR_ERR_TIMEOUT and lets the kernel return, so that a lost copy cannot hang the
+ * device.  This call runs that wait into its limit on purpose in the harmless form: one warp waits, for 2^16
+ * cycles (tens of microseconds), on a barrier that nothing arrives at -- no copy is in flight and no tensor memory
+ * is held.  Afterwards *device_error_word (DEVICE int32, zeroed by the caller) holds SPARSEPR_ERR_TIMEOUT, and
+ * the context is as usable as before. */
+sparsepr_status_t sparsepr_selftest_bounded_wait(int32_t* device_error_word, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

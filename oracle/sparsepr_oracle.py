@@ -390,36 +390,32 @@ def route_select(score, n_q, n_k, budget: int, select_all: bool = False):
 # Probe selection (Algorithm A.1) and coverage weights (Appendix A.2)
 # --------------------------------------------------------------------------
 def probe_select(a_Q, phi_Q, C_q: int, M: int):
-    """Query-group-stratified exact probe selection, Algorithm A.1.
+    """Query-group-stratified exact probe selection, Algorithm A.1, stated as a ranking.
 
-    Non-empty groups are visited in ascending id (the "deterministic group
-    order" is not specified further).  Inside a group rows are ordered by
-    increasing distance d_i to the group centroid c_a in phi_Q space, ties by
-    the original row index.  Round t of the traversal takes the t-th row of
-    every group that still has one, until M rows are chosen (all rows if
-    M >= N_q).  Returns (probe indices in selection order, weights
-    w_p = |G_a| / m_a, Appendix A.2).
+    Every row gets a radial rank inside its query group: its position when the
+    group's rows are ordered by increasing distance d_i to the group centroid
+    c_a in phi_Q space, ties by the original row index.  The round-robin
+    traversal of the algorithm (round t takes the rank-t row of every group
+    that still has one, groups in ascending id -- the "deterministic group
+    order" is not specified further) visits the rows in the order of
+    (radial rank, group id); the probe set is the first M rows of that order
+    (all rows if M >= N_q).  Returns (probe indices in selection order, weights
+    w_p = |G_a| / m_a with m_a the number of probes of group a, Appendix A.2).
     """
     a_Q = np.asarray(a_Q)
     phi_Q = np.asarray(phi_Q, dtype=np.float64)
     N = a_Q.shape[0]
     M = min(M, N)
     sizes = np.bincount(a_Q, minlength=C_q)
-    groups = [a for a in range(C_q) if sizes[a] > 0]
-    order = {}
-    for a in groups:
-        members = np.nonzero(a_Q == a)[0]
-        c_a = phi_Q[members].sum(axis=0) / members.size
-        dist = np.sqrt(((phi_Q[members] - c_a[None, :]) ** 2).sum(axis=1))
-        order[a] = members[np.lexsort((members, dist))]
-    probes = []
-    t = 0
-    while len(probes) < M:
-        for a in groups:
-            if t < sizes[a] and len(probes) < M:
-                probes.append(int(order[a][t]))
-        t += 1
-    probes = np.asarray(probes, dtype=np.int32)
+    c = np.zeros((C_q, phi_Q.shape[1]))
+    np.add.at(c, a_Q, phi_Q)
+    c[sizes > 0] /= sizes[sizes > 0, None]
+    dist = np.sqrt(((phi_Q - c[a_Q]) ** 2).sum(axis=1))
+    by_group = np.lexsort((np.arange(N), dist, a_Q))          # group id, then distance, then row index
+    start = np.concatenate(([0], np.cumsum(sizes)))[:-1]
+    rank = np.empty(N, dtype=np.int64)
+    rank[by_group] = np.arange(N) - start[a_Q[by_group]]
+    probes = np.lexsort((a_Q, rank))[:M].astype(np.int32)     # radial rank, then group id
     m_a = np.bincount(a_Q[probes], minlength=C_q)
     w = sizes[a_Q[probes]] / m_a[a_Q[probes]]
     return probes, w.astype(np.float64)

@@ -73,6 +73,7 @@ class Profile(C.Structure):
 EXPORTS = ["sparsepr_stage_assign_static", "sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
            "sparsepr_plan_export_features", "sparsepr_plan_warm", "sparsepr_plan_assignments",
+           "sparsepr_selftest_bounded_wait",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
 
@@ -97,6 +98,7 @@ def lib():
         L.sparsepr_plan_timed.argtypes = L.sparsepr_plan.argtypes + [C.POINTER(Profile)]
         L.sparsepr_plan_warm.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, sz, vp, C.POINTER(vp)]
         L.sparsepr_plan_assignments.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+        L.sparsepr_selftest_bounded_wait.argtypes = [vp, vp]
         L.sparsepr_attend_timed.argtypes = L.sparsepr_attend.argtypes + [C.POINTER(Profile)]
         L.sparsepr_dense_timed.argtypes = L.sparsepr_dense.argtypes + [C.POINTER(Profile)]
         L.sparsepr_plan_stats.argtypes = [vp, C.POINTER(Stats)]
@@ -325,6 +327,13 @@ def sparsepr_plan_import(Q, K, V, host: dict, params: Params | None = None, **kw
     _check(L.sparsepr_plan_import(C.byref(shape), C.byref(params), C.byref(ph), ws.data_ptr(), ws.numel(),
                                   _stream(), C.byref(handle)), "sparsepr_plan_import")
     return Plan(handle, ws, shape, params, L.sparsepr_attend_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+def sparsepr_selftest_bounded_wait() -> int:
+    """Runs one bounded device wait into its limit (harmless form) and returns the status it recorded."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().sparsepr_selftest_bounded_wait(word.data_ptr(), _stream()), "sparsepr_selftest_bounded_wait")
+    return int(word.item())
 
 
 # ---- single stages -------------------------------------------------------------------

@@ -841,6 +841,13 @@ sparsepr_status_t sparsepr_plan_export_features(const sparsepr_plan_t* p, sparse
   return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 
+sparsepr_status_t sparsepr_selftest_bounded_wait(int32_t* device_error_word, void* cuda_stream) {
+  if (!device_error_word) return SPARSEPR_ERR_INVALID_ARG;
+  cudaGetLastError();
+  launch_selftest_bounded_wait(device_error_word, static_cast<cudaStream_t>(cuda_stream));
+  return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
+}
+
 // ---- single stages ---------------------------------------------------------------------
 size_t sparsepr_stage_assign_workspace_bytes(int32_t n, int32_t C, int32_t r) {
   if (n < 1 || C < 1 || r < 1 || r > kMaxRank) return 0;

@@ -150,7 +150,27 @@ __global__ void k_transpose_correction(const float* __restrict__ A, __nv_bfloat1
   for (int r = threadIdx.y; r < 32; r += 8) t[(n0 + r) * 128 + k0 + threadIdx.x] = __float2bfloat16_rn(tile[threadIdx.x][r]);
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nobody arrives at (no copy in flight, no
+// tensor memory held), with a limit of 2^16 cycles; the wait gives up, the error word receives
+// SPARSEPR_ERR_TIMEOUT, the kernel returns normally and the context stays usable.
+__global__ void k_selftest_bounded_wait(int* err, long long limit) {
+  __shared__ __align__(8) unsigned long long sbar;
+  __shared__ int abort_flag;
+  const uint32_t bar = smem_u32(&sbar);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait_limit(bar, 0, &abort_flag, limit);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_flag)) set_error(err, SPARSEPR_ERR_TIMEOUT);
+}
+
 }  // namespace tc
+
+void launch_selftest_bounded_wait(int* err, cudaStream_t st) { tc::k_selftest_bounded_wait<<<1, 32, 0, st>>>(err, 1ll << 16); }
 
 cudaError_t init_correction_tc() {
   return cudaFuncSetAttribute(tc::k_correction_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::CorrSmem::total);

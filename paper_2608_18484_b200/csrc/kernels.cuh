@@ -112,6 +112,8 @@ constexpr int kRemRows = 32;
 cudaError_t init_attention_packed();
 void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st);
 bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st);
+// one warp runs the bounded mbarrier wait into its limit (2^16 cycles) and records SPARSEPR_ERR_TIMEOUT in *err
+void launch_selftest_bounded_wait(int* err, cudaStream_t st);
 // correction_tc.cu: O <- X + X A + c in place, X = O + O_lo (two bf16 words, O_lo [BH][N][128] contiguous), d_v = 128;
 // At: bf16 scratch [BH][128][128]
 cudaError_t init_correction_tc();

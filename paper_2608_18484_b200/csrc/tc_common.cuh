@@ -23,8 +23,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// bounded wait: gives up after 2^28 clock cycles (more than 0.1 s; a healthy wait lasts microseconds)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// bounded wait: gives up after `limit` clock cycles, sets the CTA's abort flag and returns false
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try(bar, parity)) return true;
   if (*abort_flag) return false;
   const long long t0 = clock64();
@@ -32,10 +32,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   while (!mbar_try(bar, parity)) {            // try_wait itself parks the thread for a short hardware-defined time
     if ((++spins & 0x3FFu) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > (1ll << 28)) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
     }
   }
   return true;
+}
+// the limit every kernel uses: 2^28 clock cycles (more than 0.1 s; a healthy wait lasts microseconds)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, 1ll << 28);
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
   asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"

@@ -109,3 +109,15 @@ def test_degenerate_inputs():
     bad[0, 0, 5, 3] = float("nan")
     stb = B.sparsepr_plan_stats(B.sparsepr_plan(bad, K, V, **kw))
     assert stb["device_error"] == 5                              # non-finite input is reported, nothing hangs
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """A wait that nothing satisfies ends at its cycle limit with ERR_TIMEOUT in the error word (no hang, no
+    trap); an ordinary call right after it succeeds."""
+    assert B.sparsepr_selftest_bounded_wait() == 6
+    assert "wait" in B.status_string(6)
+    wl = W.TINY.scaled(grid=(1, 32, 32))
+    _, (Qd, Kd, Vd) = heads_to_device(wl, [0, 1])
+    plan = B.sparsepr_plan(Qd, Kd, Vd, density=0.25, block=64, n_sample=64, n_probe=16, softmax_scale=1.0)
+    O = B.sparsepr_attend(plan, Qd, Kd, Vd)
+    assert B.sparsepr_plan_stats(plan)["device_error"] == 0 and torch.isfinite(O).all()
