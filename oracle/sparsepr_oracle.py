@@ -474,10 +474,16 @@ def reconstruct(O_sp, probe_idx, O_dense_probe, fit) -> np.ndarray:
 # --------------------------------------------------------------------------
 # The whole call for one head
 # --------------------------------------------------------------------------
+# Partition variants of the ablation (Section 5.2, Table 2; Section 3.1 for the semantic reference partition)
+PARTITION_RESPONSE_COUPLED = 0   # K/V groups from key responses, query groups from query responses (the method)
+PARTITION_KEY_RESPONSE_KV = 1    # only the K/V partition is response-based; queries are clustered semantically
+PARTITION_SEMANTIC = 2           # k-means on the raw key and on the raw query activations, separately
+
+
 def default_params(**kw):
     p = dict(density=0.25, block=128, Ck=0, Cq=0, n_sample=256, n_probe=128,
              rK=48, rQ=64, r_out=16, lam=0.1, eps_rms=1e-6, eps_std=1e-6,
-             kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0)
+             kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0, partition=PARTITION_RESPONSE_COUPLED)
     p.update(kw)
     return p
 
@@ -487,7 +493,15 @@ def plan_head(Q, K, prm: dict, bh: int, warm=None):
     permutations, probe selection and routing.  Returns a dict of every
     intermediate (so that single stages of another implementation can be fed
     from it).  `warm` = {"a_K": ..., "a_Q": ...}, the partition of a previous
-    call, warm-starts both k-means runs (see `kmeans`)."""
+    call, warm-starts both k-means runs (see `kmeans`).
+
+    prm["partition"] selects the ablation variants: the semantic reference
+    partition applies k-means to the raw key and query activations (Section
+    3.1); the key-response K/V variant changes only the K/V partition (Section
+    5.2).  Same initial rows, iteration count and tie rules in every variant.
+    Where the query partition is semantic, the probe ranking of Algorithm A.1
+    measures its distances in the raw query space, the space that partition
+    was built in (reading: the paper runs the ablation with fixed probes)."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     N, d = Q.shape
@@ -498,18 +512,27 @@ def plan_head(Q, K, prm: dict, bh: int, warm=None):
     seed = prm["seed"]
     out = {"C_k": C_k, "C_q": C_q, "M": M, "scale": scale}
 
+    variant = prm.get("partition", PARTITION_RESPONSE_COUPLED)
+    wK = None if warm is None else warm["a_K"]
+    wQ = None if warm is None else warm["a_Q"]
+    T = prm["kmeans_iters"]
     s_idx = stride_sample(min(prm["n_sample"], N), N, seed, TAG_QUERY_SAMPLE, bh)
-    M_K = key_response_metric(Q[s_idx])
-    F_K, lam_K = eig_feature_map(M_K, prm["rK"])
-    phi_K = key_response(K, F_K)
-    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, bh), prm["kmeans_iters"],
-                       init_assign=None if warm is None else warm["a_K"])
+    M_K = F_K = lam_K = M_Q = F_Q = lam_Q = None
+    if variant == PARTITION_SEMANTIC:
+        phi_K = K                                   # k-means on the key activations themselves
+    else:
+        M_K = key_response_metric(Q[s_idx])
+        F_K, lam_K = eig_feature_map(M_K, prm["rK"])
+        phi_K = key_response(K, F_K)
+    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, bh), T, init_assign=wK)
     kappa, n_k = kv_centroids(K, a_K, C_k)
-    M_Q = query_response_metric(kappa, n_k)
-    F_Q, lam_Q = eig_feature_map(M_Q, prm["rQ"])
-    phi_Q = query_response(Q, F_Q, prm["eps_rms"])
-    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), prm["kmeans_iters"],
-                       init_assign=None if warm is None else warm["a_Q"])
+    if variant == PARTITION_RESPONSE_COUPLED:
+        M_Q = query_response_metric(kappa, n_k)
+        F_Q, lam_Q = eig_feature_map(M_Q, prm["rQ"])
+        phi_Q = query_response(Q, F_Q, prm["eps_rms"])
+    else:
+        phi_Q = Q                                   # k-means on the query activations themselves
+    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), T, init_assign=wQ)
     theta, n_q = query_centroids(Q, a_Q, C_q)
 
     q_perm, q_inv, q_off = group_permutation(a_Q, C_q)

@@ -181,6 +181,31 @@ def test_kmeans_warm_start():
     assert all(objs[i + 1] <= objs[i] + 1e-9 for i in range(len(objs) - 1))
 
 
+def test_partition_variants():
+    """Semantic reference partition = Lloyd on the raw activations (checked against sklearn from the same rows);
+    the key-response K/V variant takes its K/V groups from the method and its query groups from the semantic
+    partition; every variant yields a complete, valid plan."""
+    sk = pytest.importorskip("sklearn.cluster")
+    rng = np.random.default_rng(21)
+    N, d, C = 384, 16, 6
+    cent = rng.normal(size=(C, d)) * 2.0
+    lab = rng.integers(0, C, size=N)
+    Q = cent[lab] + rng.normal(size=(N, d)) * 0.5
+    K = 0.7 * cent[lab] + rng.normal(size=(N, d)) * 0.5
+    prm = orc.default_params(density=0.4, block=64, n_sample=64, n_probe=8, rK=8, rQ=8, kmeans_iters=4, softmax_scale=1.0)
+    plans = {v: orc.plan_head(Q, K, dict(prm, partition=v), 3) for v in (0, 1, 2)}
+    for X, key, tag in ((K, "a_K", orc.TAG_KV_INIT), (Q, "a_Q", orc.TAG_Q_INIT)):
+        init = orc.stride_sample(C, N, 0, tag, 3)
+        km = sk.KMeans(n_clusters=C, init=X[init], n_init=1, algorithm="lloyd", max_iter=3, tol=0.0).fit(X)
+        assert np.array_equal(plans[2][key], km.labels_)
+    assert np.array_equal(plans[1]["a_K"], plans[0]["a_K"]) and np.array_equal(plans[1]["a_Q"], plans[2]["a_Q"])
+    assert not np.array_equal(plans[0]["a_Q"], plans[2]["a_Q"])
+    budget = orc.pair_budget(0.4, N, N, 8)
+    for v, p in plans.items():
+        assert p["routed_pairs"] <= budget and len(set(p["probe_idx"].tolist())) == 8
+        assert np.all(np.diff(p["route_ptr"]) >= (p["n_q"] > 0))
+
+
 def test_group_permutation():
     rng = np.random.default_rng(7)
     a = rng.integers(0, 9, size=100)
