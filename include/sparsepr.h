@@ -59,6 +59,18 @@ typedef enum {
 
 typedef enum { SPARSEPR_F32 = 0, SPARSEPR_BF16 = 1 } sparsepr_dtype_t;
 
+/* How the two partitions are built: the method, and the two ablation variants of Section 5.2 (Table 2).  The
+ * semantic reference partition of Section 3.1 applies k-means to the key and to the query activations
+ * themselves; the key-response K/V variant changes only the K/V partition.  Initial rows, iteration count and
+ * tie rules are the same in every variant.  Where the query partition is semantic, Algorithm A.1 ranks the probe
+ * candidates by their distance in the raw query space.  The variants cluster in d dimensions on the CUDA cores
+ * (d = 128: several times the cost of the method's 64-dimensional tensor-core k-means). */
+typedef enum {
+  SPARSEPR_PARTITION_RESPONSE_COUPLED = 0,
+  SPARSEPR_PARTITION_KEY_RESPONSE_KV = 1,
+  SPARSEPR_PARTITION_SEMANTIC = 2
+} sparsepr_partition_t;
+
 /* Problem shape: Q, K in R^{N x d}, V in R^{N x d_v} per (batch, head) -- the
  * paper's problem statement (Section 3).  Strides are in elements. */
 typedef struct {
@@ -84,6 +96,7 @@ typedef struct {
   float softmax_scale;   /* s; 0 selects 1/sqrt(d) */
   uint64_t seed;         /* offsets the deterministic row samples */
   int32_t mode;          /* 0 = probe-fitted reconstruction, 1 = renormalised hard drop only */
+  int32_t partition;     /* sparsepr_partition_t; 0 = Response-Coupled Partitioning */
 } sparsepr_params_t;
 
 typedef struct sparsepr_plan_s sparsepr_plan_t;
@@ -131,7 +144,9 @@ typedef struct {
  * scores of Section 4.3), exported so that they can be compared with an independent evaluation.  Every
  * pointer is HOST memory owned by the caller; NULL skips the field.  All float32, b-major over (batch, head):
  *   F_K   [BH, d, r_K], F_Q [BH, d, r_Q]  feature maps (columns = scaled eigendirections; their signs are arbitrary)
- *   phi_Q [BH, N, r_Q]                    RMS-normalised query responses (Eq. 7)
+ *   phi_Q [BH, N, r_Q]                    RMS-normalised query responses (Eq. 7); [BH, N, d] raw queries when the
+ *                                         query partition is semantic (F_Q, and F_K for the semantic K/V partition,
+ *                                         are then not written)
  *   kappa [BH, C_k, d], theta [BH, C_q, d] original-space means of the K/V groups and of the query groups
  *   score [BH, C_q, C_k]                  cell scores the router selected from */
 typedef struct {

@@ -38,7 +38,8 @@ class Params(C.Structure):
     _fields_ = [("density", C.c_float), ("block", C.c_int32), ("Ck", C.c_int32), ("Cq", C.c_int32),
                 ("n_sample", C.c_int32), ("n_probe", C.c_int32), ("rK", C.c_int32), ("rQ", C.c_int32),
                 ("r_out", C.c_int32), ("lam", C.c_float), ("eps_rms", C.c_float), ("eps_std", C.c_float),
-                ("kmeans_iters", C.c_int32), ("softmax_scale", C.c_float), ("seed", C.c_uint64), ("mode", C.c_int32)]
+                ("kmeans_iters", C.c_int32), ("softmax_scale", C.c_float), ("seed", C.c_uint64), ("mode", C.c_int32),
+                ("partition", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -151,8 +152,8 @@ def make_shape(Q, K, V, O) -> Shape:
 
 
 def make_params(density=0.25, block=128, Ck=0, Cq=0, n_sample=256, n_probe=128, rK=48, rQ=64, r_out=16, lam=0.1,
-                eps_rms=1e-6, eps_std=1e-6, kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0) -> Params:
-    return Params(density=density, block=block, Ck=Ck, Cq=Cq, n_sample=n_sample, n_probe=n_probe, rK=rK, rQ=rQ,
+                eps_rms=1e-6, eps_std=1e-6, kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0, partition=0) -> Params:
+    return Params(partition=partition, density=density, block=block, Ck=Ck, Cq=Cq, n_sample=n_sample, n_probe=n_probe, rK=rK, rQ=rQ,
                   r_out=r_out, lam=lam, eps_rms=eps_rms, eps_std=eps_std, kmeans_iters=kmeans_iters,
                   softmax_scale=softmax_scale, seed=seed, mode=mode)
 
@@ -288,6 +289,9 @@ def sparsepr_plan_export_features(plan: Plan, fields=("F_K", "F_Q", "phi_Q", "ka
     BH, N, d = plan.BH, plan.shape.N, plan.shape.d
     Ck, Cq = plan.groups
     rK, rQ = min(plan.params.rK or 48, d), min(plan.params.rQ or 64, d)
+    if plan.params.partition != 0:                  # semantic query partition: phi_Q holds the raw queries
+        rQ = d
+        fields = tuple(f for f in fields if f != "F_Q" and not (f == "F_K" and plan.params.partition == 2))
     shapes = dict(F_K=(BH, d, rK), F_Q=(BH, d, rQ), phi_Q=(BH, N, rQ), kappa=(BH, Ck, d), theta=(BH, Cq, d),
                   score=(BH, Cq, Ck))
     arrs = {k: np.empty(shapes[k], np.float32) for k in fields}

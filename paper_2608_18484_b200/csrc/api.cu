@@ -42,13 +42,15 @@ struct Carver {                       // bump allocator over a caller-owned work
 struct Resolved {
   int B, H, BH, N, d, dtype, es;
   int Ck, Cq, Cmax, Ms, M, rK, rQ, RK, RQ, Rmax, r_out, T, mode;
+  int partition;                       // sparsepr_partition_t
+  int fK, fQ;                          // width of the features each side is clustered in: rK / rQ, or d for raw activations
   bool full_rank;                      // r_out covers the whole row space of the probe residuals: the projector is the identity
   float density, lambda, eps_rms, eps_std, scale;
   u64 seed;
   i64 qs[3], ks[3], vs[3], os[3];
 };
 
-int round16(int r) { return r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64; }
+int round16(int r) { return feature_ld(r); }      // row length of a feature buffer with r columns
 
 sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p, Resolved* r) {
   if (!s || !r) return SPARSEPR_ERR_INVALID_ARG;
@@ -82,7 +84,11 @@ sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p,
   r->rK = std::min(p->rK ? p->rK : 48, s->d);
   r->rQ = std::min(p->rQ ? p->rQ : 64, s->d);
   if (r->rK > kMaxRank || r->rQ > kMaxRank) return SPARSEPR_ERR_UNSUPPORTED;
-  r->RK = round16(r->rK); r->RQ = round16(r->rQ); r->Rmax = std::max(r->RK, r->RQ);
+  if (p->partition < 0 || p->partition > SPARSEPR_PARTITION_SEMANTIC) return SPARSEPR_ERR_INVALID_ARG;
+  r->partition = p->partition;
+  r->fK = r->partition == SPARSEPR_PARTITION_SEMANTIC ? s->d : r->rK;
+  r->fQ = r->partition != SPARSEPR_PARTITION_RESPONSE_COUPLED ? s->d : r->rQ;
+  r->RK = round16(r->fK); r->RQ = round16(r->fQ); r->Rmax = std::max(r->RK, r->RQ);
   {
     // r = min(r_out, M, d_v).  Once r reaches min(M, d_v) it spans every direction the probe residuals (M rows in
     // d_v dimensions) can have, the projector acts as the identity and no eigenvectors are needed; below that the
@@ -347,7 +353,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
   int* changed = p->km_changed + (tag == kTagQInit ? (size_t)(R.T + 1) * R.BH : 0);
   cudaMemsetAsync(changed, 0, (size_t)(R.T + 1) * R.BH * sizeof(int), st);
   launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
-  const bool tcp = kmeans_tc_supported();
+  const bool tcp = kmeans_tc_supported() && r <= kMaxRank;
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
   // (with the tensor-core assignment the finalize step also writes the two bf16 words of every centroid)
   // warm start: the initial centroids become the means of the current features over the previous partition's groups
@@ -471,33 +477,43 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
   StageTimer tm(prof, st);
-  // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means
-  launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
-  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
-  tm.mark(SPARSEPR_STAGE_KEY_METRIC);
-  if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
-    if (!launch_project_tc(K, r.ks, r.BH, r.H, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+  // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means (semantic variant: k-means on K itself)
+  if (r.partition == SPARSEPR_PARTITION_SEMANTIC) {
+    tm.mark(SPARSEPR_STAGE_KEY_METRIC);
+    launch_raw_features(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, p->phi, p->maxabs, p->err, st);
   } else {
-    launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+    launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
+    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
+    tm.mark(SPARSEPR_STAGE_KEY_METRIC);
+    if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
+      if (!launch_project_tc(K, r.ks, r.BH, r.H, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+    } else {
+      launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+    }
   }
   tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
-  run_kmeans(p, r.rK, r.Ck, kTagKvInit, p->a_K, warm_kv, st);
+  run_kmeans(p, r.fK, r.Ck, kTagKvInit, p->a_K, warm_kv, st);
   tm.mark(SPARSEPR_STAGE_KEY_KMEANS);
   launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
   launch_group_means(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
   tm.mark(SPARSEPR_STAGE_KEY_PERMUTE);
-  // query partition: centroid metric -> F_Q -> phi_Q -> k-means
-  launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
-  launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
-  tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
+  // query partition: centroid metric -> F_Q -> phi_Q -> k-means (other variants: k-means on Q itself)
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
-  if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {
-    if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+  if (r.partition != SPARSEPR_PARTITION_RESPONSE_COUPLED) {
+    tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
+    launch_raw_features(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, p->phi, p->maxabs, p->err, st);
   } else {
-    launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+    launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
+    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
+    tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
+    if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {
+      if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+    } else {
+      launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
+    }
   }
   tm.mark(SPARSEPR_STAGE_QUERY_PROJECT);
-  run_kmeans(p, r.rQ, r.Cq, kTagQInit, p->a_Q, warm_q, st);
+  run_kmeans(p, r.fQ, r.Cq, kTagQInit, p->a_Q, warm_q, st);
   tm.mark(SPARSEPR_STAGE_QUERY_KMEANS);
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
   launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
@@ -507,7 +523,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   cudaStream_t ps = st;
   if (overlap) { fork_side(p, st); ps = p->side; }
   if (r.M > 0)
-    launch_probe_select(p->phi, r.RQ, r.rQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, ps);
+    launch_probe_select(p->phi, r.RQ, r.fQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, ps);
   tm.mark(SPARSEPR_STAGE_PROBE_SELECT);
   launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
@@ -833,9 +849,10 @@ sparsepr_status_t sparsepr_plan_export_features(const sparsepr_plan_t* p, sparse
   const size_t BH = r.BH, N = r.N, d = r.d;
   bool ok = true;
   auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };
-  cp(o->F_K, p->FK, BH * d * r.rK * 4); cp(o->F_Q, p->FQ, BH * d * r.rQ * 4);
+  if (r.partition != SPARSEPR_PARTITION_SEMANTIC) cp(o->F_K, p->FK, BH * d * r.rK * 4);
+  if (r.partition == SPARSEPR_PARTITION_RESPONSE_COUPLED) cp(o->F_Q, p->FQ, BH * d * r.rQ * 4);
   if (o->phi_Q)                                                // rows are padded to RQ floats on the device
-    ok &= cudaMemcpy2D(o->phi_Q, (size_t)r.rQ * 4, p->phi, (size_t)r.RQ * 4, (size_t)r.rQ * 4, BH * N, cudaMemcpyDeviceToHost) == cudaSuccess;
+    ok &= cudaMemcpy2D(o->phi_Q, (size_t)r.fQ * 4, p->phi, (size_t)r.RQ * 4, (size_t)r.fQ * 4, BH * N, cudaMemcpyDeviceToHost) == cudaSuccess;
   cp(o->kappa, p->kappa, BH * r.Ck * d * 4); cp(o->theta, p->theta, BH * r.Cq * d * 4);
   cp(o->score, p->score, BH * (size_t)r.Cq * r.Ck * 4);
   return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;

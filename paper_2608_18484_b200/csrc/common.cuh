@@ -13,6 +13,9 @@ typedef unsigned long long u64;
 constexpr int kMaxGroups = 2048;     // C_k, C_q limit (shared-memory histograms)
 constexpr int kMaxProbes = 1024;     // M limit
 constexpr int kMaxRank = 64;         // r_K, r_Q limit
+// row length of a feature buffer that holds r columns (zero padded): 16, 32, 48, 64, or 128 for the raw
+// activations of the semantic partition
+__host__ __device__ __forceinline__ int feature_ld(int r) { return r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : r <= 64 ? 64 : 128; }
 
 // ---- device error word -------------------------------------------------------
 __device__ __forceinline__ void set_error(int* err, int code) {

@@ -21,6 +21,9 @@ void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int 
                     double* lam_out, cudaStream_t st);
 void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
+// features of the semantic partition: the activations themselves as float32 rows [BH][N][d]
+void launch_raw_features(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, float* phi, unsigned* maxabs,
+                         int* err, cudaStream_t st);
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
 void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, int C, const int* prev, i64* sums,

@@ -209,6 +209,34 @@ void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int 
 #undef SPR_PROJ
 }
 
+// Features of the semantic reference partition (Section 3.1): the activations themselves, as float32 rows
+// [BH][N][d]; also the largest magnitude per head (for the fixed-point sums) and the non-finite check.
+template <typename T>
+__global__ void __launch_bounds__(256) k_raw_features(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H, int N, int d,
+                                                      float* __restrict__ phi, unsigned* __restrict__ maxabs, int* __restrict__ err) {
+  const int bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int per_row = d / 8;
+  float mx = 0.f;
+  bool bad = false;
+  for (i64 e = (i64)blockIdx.x * 256 + threadIdx.x; e < (i64)N * per_row; e += (i64)gridDim.x * 256) {
+    const int row = (int)(e / per_row), c8 = (int)(e % per_row) * 8;
+    float v[8];
+    load8(X + b * sb + h * sh + (i64)row * sn + c8, v);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { mx = fmaxf(mx, fabsf(v[k])); bad |= !isfinite(v[k]); }
+    store8(phi + ((i64)bh * N + row) * d + c8, v);
+  }
+  mx = warp_max(mx);
+  if ((threadIdx.x & 31) == 0 && mx > 0.f) atomicMax(maxabs + bh, __float_as_uint(mx));
+  if (bad) set_error(err, SPARSEPR_ERR_NUMERIC);
+}
+void launch_raw_features(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, float* phi, unsigned* maxabs,
+                         int* err, cudaStream_t st) {
+  dim3 grid((unsigned)std::min<i64>(((i64)N * (d / 8) + 255) / 256, 1024), BH);
+  if (dtype == SPARSEPR_BF16) k_raw_features<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X, xs[0], xs[1], xs[2], H, N, d, phi, maxabs, err);
+  else k_raw_features<float><<<grid, 256, 0, st>>>((const float*)X, xs[0], xs[1], xs[2], H, N, d, phi, maxabs, err);
+}
+
 // =============================================================================
 // k-means (Section 4.1).  Assignment: a[j] = argmin_c ||x_j - mu_c||^2, ties to the
 // lowest c.  Fast path in float32 via s_c = ||mu_c||^2 - 2 x.mu_c; whenever the
@@ -234,24 +262,29 @@ __device__ __noinline__ int exact_assign(const float* __restrict__ x, const floa
 
 constexpr int kAssignChunk = 64;   // centroids staged per shared-memory chunk
 
-template <int R>
+// R = padded feature width (16..128), ROWS = rows per thread (two up to 64 columns; one for the 128 columns of the
+// semantic partition's raw activations, whose row already fills the registers)
+template <int R, int ROWS>
 __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__ phi, int ldphi, int N, int r,
                                                        const float* __restrict__ mu, const float* __restrict__ mu2,
                                                        const float* __restrict__ mumax, int C, int* __restrict__ assign,
                                                        i64* __restrict__ sums, int* __restrict__ counts,
                                                        const int* __restrict__ fx_shift, int* __restrict__ recheck_count,
                                                        const int* __restrict__ prev_changed, int* __restrict__ cur_changed) {
-  __shared__ __align__(16) float mus[kAssignChunk * R];
-  __shared__ float mu2s[kAssignChunk];
+  constexpr int kChunk = R > 64 ? 32 : kAssignChunk;
+  __shared__ __align__(16) float mus[kChunk * R];
+  __shared__ float mu2s[kChunk];
   const int bh = blockIdx.y;
   if (prev_changed != nullptr && prev_changed[bh] == 0) return;      // fixed point reached in the previous pass
   const float* ph = phi + (i64)bh * N * ldphi;
   const float* muh = mu + (i64)bh * C * R;
-  const int rows[2] = {(int)(blockIdx.x * 256 + threadIdx.x), (int)(blockIdx.x * 256 + threadIdx.x + 128)};
-  float x[2][R];
-  float xn2[2] = {0.f, 0.f};
+  int rows[ROWS];
+  float x[ROWS][R];
+  float xn2[ROWS];
 #pragma unroll
-  for (int t = 0; t < 2; ++t) {
+  for (int t = 0; t < ROWS; ++t) {
+    rows[t] = (int)(blockIdx.x * (128 * ROWS) + threadIdx.x + 128 * t);
+    xn2[t] = 0.f;
     const float* p = ph + (i64)min(rows[t], N - 1) * ldphi;
 #pragma unroll
     for (int k = 0; k < R; k += 4) {
@@ -261,34 +294,41 @@ __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__
 #pragma unroll
     for (int k = 0; k < R; ++k) xn2[t] = fmaf(x[t][k], x[t][k], xn2[t]);
   }
-  float best[2] = {3.0e38f, 3.0e38f}, second[2] = {3.0e38f, 3.0e38f};
-  int bi[2] = {0, 0};
-  for (int c0 = 0; c0 < C; c0 += kAssignChunk) {
-    const int nc = min(kAssignChunk, C - c0);
+  float best[ROWS], second[ROWS];
+  int bi[ROWS];
+#pragma unroll
+  for (int t = 0; t < ROWS; ++t) { best[t] = 3.0e38f; second[t] = 3.0e38f; bi[t] = 0; }
+  for (int c0 = 0; c0 < C; c0 += kChunk) {
+    const int nc = min(kChunk, C - c0);
     __syncthreads();
     for (int e = threadIdx.x; e < nc * R; e += 128) mus[e] = muh[(i64)c0 * R + e];
     if (threadIdx.x < nc) mu2s[threadIdx.x] = mu2[(i64)bh * C + c0 + threadIdx.x];
     __syncthreads();
     for (int c = 0; c < nc; ++c) {
       const float4* m4 = reinterpret_cast<const float4*>(mus + c * R);
-      float d0 = 0.f, d1 = 0.f;
+      float dot[ROWS];
+#pragma unroll
+      for (int t = 0; t < ROWS; ++t) dot[t] = 0.f;
 #pragma unroll
       for (int k = 0; k < R / 4; ++k) {
         const float4 m = m4[k];
-        d0 = fmaf(x[0][4 * k], m.x, d0); d0 = fmaf(x[0][4 * k + 1], m.y, d0);
-        d0 = fmaf(x[0][4 * k + 2], m.z, d0); d0 = fmaf(x[0][4 * k + 3], m.w, d0);
-        d1 = fmaf(x[1][4 * k], m.x, d1); d1 = fmaf(x[1][4 * k + 1], m.y, d1);
-        d1 = fmaf(x[1][4 * k + 2], m.z, d1); d1 = fmaf(x[1][4 * k + 3], m.w, d1);
+#pragma unroll
+        for (int t = 0; t < ROWS; ++t) {
+          dot[t] = fmaf(x[t][4 * k], m.x, dot[t]); dot[t] = fmaf(x[t][4 * k + 1], m.y, dot[t]);
+          dot[t] = fmaf(x[t][4 * k + 2], m.z, dot[t]); dot[t] = fmaf(x[t][4 * k + 3], m.w, dot[t]);
+        }
       }
-      const float s0 = fmaf(-2.f, d0, mu2s[c]), s1 = fmaf(-2.f, d1, mu2s[c]);
-      if (s0 < best[0]) { second[0] = best[0]; best[0] = s0; bi[0] = c0 + c; } else if (s0 < second[0]) second[0] = s0;
-      if (s1 < best[1]) { second[1] = best[1]; best[1] = s1; bi[1] = c0 + c; } else if (s1 < second[1]) second[1] = s1;
+#pragma unroll
+      for (int t = 0; t < ROWS; ++t) {
+        const float sc = fmaf(-2.f, dot[t], mu2s[c]);
+        if (sc < best[t]) { second[t] = best[t]; best[t] = sc; bi[t] = c0 + c; } else if (sc < second[t]) second[t] = sc;
+      }
     }
   }
   const float mm = mumax[bh];
   const int shift = fx_shift ? fx_shift[bh] : 0;
 #pragma unroll
-  for (int t = 0; t < 2; ++t) {
+  for (int t = 0; t < ROWS; ++t) {
     if (rows[t] >= N) continue;
     // |computed score - true score| <= E for every centroid (float32 rounding of the
     // dot product, of ||mu||^2 and of the final combination)
@@ -314,10 +354,10 @@ __global__ void __launch_bounds__(128) k_kmeans_assign(const float* __restrict__
 void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, const float* mu, const float* mu2,
                           const float* mumax, int C, int* assign, i64* sums, int* counts, const int* fx_shift,
                           int* recheck_count, const int* prev_changed, int* cur_changed, cudaStream_t st) {
-  dim3 grid((N + 255) / 256, BH);
-  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
-#define SPR_ASSIGN(RR) k_kmeans_assign<RR><<<grid, 128, 0, st>>>(phi, ldphi, N, r, mu, mu2, mumax, C, assign, sums, counts, fx_shift, recheck_count, prev_changed, cur_changed)
-  if (R == 16) SPR_ASSIGN(16); else if (R == 32) SPR_ASSIGN(32); else if (R == 48) SPR_ASSIGN(48); else SPR_ASSIGN(64);
+  const int R = feature_ld(r);
+#define SPR_ASSIGN(RR, ROWS) k_kmeans_assign<RR, ROWS><<<dim3((N + 128 * ROWS - 1) / (128 * ROWS), BH), 128, 0, st>>>(phi, ldphi, N, r, mu, mu2, mumax, C, assign, sums, counts, fx_shift, recheck_count, prev_changed, cur_changed)
+  if (R == 16) SPR_ASSIGN(16, 2); else if (R == 32) SPR_ASSIGN(32, 2); else if (R == 48) SPR_ASSIGN(48, 2);
+  else if (R == 64) SPR_ASSIGN(64, 2); else SPR_ASSIGN(128, 1);
 #undef SPR_ASSIGN
 }
 
@@ -367,7 +407,7 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
     i64* s = sums + ((i64)bh * C + c) * R;
     const int cnt = update ? counts[(i64)bh * C + c] : 0;
     double n2 = 0.0;
-    for (int k = lane; k < 64; k += 32) {
+    for (int k = lane; k < max(R, 64); k += 32) {
       float v = 0.f;
       if (k < R) {
         v = m[k];
@@ -377,7 +417,7 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
         }
         n2 += (double)v * (double)v;
       }
-      if (mh != nullptr) {
+      if (mh != nullptr && k < 64) {
         // the two bf16 words of the centroid for the tensor-core assignment, [C][64] with zeros beyond r
         const float x = k < r ? v : 0.f;
         const __nv_bfloat16 hb = __float2bfloat16_rn(x);
@@ -414,46 +454,49 @@ __global__ void __launch_bounds__(256) k_kmeans_warm_sums(const float* __restric
   const int row = rowbase + lane;
   int cl_mine = -1;
   if (row < N) { const int c = prev[(i64)bh * N + row]; if (c >= 0 && c < C) cl_mine = c; }
-  const bool cok = 2 * lane < r;
-  float pv0[32], pv1[32];
-#pragma unroll
-  for (int rr = 0; rr < 32; ++rr) {
-    const int rw = min(rowbase + rr, N - 1);
-    const float2 x2 = cok ? *reinterpret_cast<const float2*>(phi + ((i64)bh * N + rw) * ldphi + 2 * lane) : make_float2(0.f, 0.f);
-    pv0[rr] = x2.x; pv1[rr] = x2.y;
-  }
   const float scl = __int_as_float((127 + fx_shift[bh]) << 23);
-  unsigned todo = __ballot_sync(FULL, cl_mine >= 0);
-  while (todo) {
-    const int leader = __ffs(todo) - 1;
-    const int cl = __shfl_sync(FULL, cl_mine, leader);
-    const unsigned members = __ballot_sync(FULL, cl_mine == cl) & todo;
-    todo &= ~members;
-    float a0 = 0.f, a1 = 0.f;
+  for (int cb = 0; cb < R; cb += 64) {                         // 64 columns at a time (two passes for raw activations)
+    const int col = cb + 2 * lane;
+    const bool cok = col < r;
+    float pv0[32], pv1[32];
 #pragma unroll
-    for (int rr = 0; rr < 32; ++rr)
-      if ((members >> rr) & 1u) { a0 += pv0[rr]; a1 += pv1[rr]; }
-    i64* sp = sums + ((i64)bh * C + cl) * R;
-    if (2 * lane < r) atomicAdd(reinterpret_cast<u64*>(sp + 2 * lane), (u64)__float2ll_rn(a0 * scl));
-    if (2 * lane + 1 < r) atomicAdd(reinterpret_cast<u64*>(sp + 2 * lane + 1), (u64)__float2ll_rn(a1 * scl));
-    if (lane == 0) atomicAdd(counts + (i64)bh * C + cl, __popc(members));
+    for (int rr = 0; rr < 32; ++rr) {
+      const int rw = min(rowbase + rr, N - 1);
+      const float2 x2 = cok ? *reinterpret_cast<const float2*>(phi + ((i64)bh * N + rw) * ldphi + col) : make_float2(0.f, 0.f);
+      pv0[rr] = x2.x; pv1[rr] = x2.y;
+    }
+    unsigned todo = __ballot_sync(FULL, cl_mine >= 0);
+    while (todo) {
+      const int leader = __ffs(todo) - 1;
+      const int cl = __shfl_sync(FULL, cl_mine, leader);
+      const unsigned members = __ballot_sync(FULL, cl_mine == cl) & todo;
+      todo &= ~members;
+      float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+      for (int rr = 0; rr < 32; ++rr)
+        if ((members >> rr) & 1u) { a0 += pv0[rr]; a1 += pv1[rr]; }
+      i64* sp = sums + ((i64)bh * C + cl) * R;
+      if (col < r) atomicAdd(reinterpret_cast<u64*>(sp + col), (u64)__float2ll_rn(a0 * scl));
+      if (col + 1 < r) atomicAdd(reinterpret_cast<u64*>(sp + col + 1), (u64)__float2ll_rn(a1 * scl));
+      if (lane == 0 && cb == 0) atomicAdd(counts + (i64)bh * C + cl, __popc(members));
+    }
   }
 }
 void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, int C, const int* prev, i64* sums,
                              int* counts, const int* fx_shift, cudaStream_t st) {
-  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  const int R = feature_ld(r);
   k_kmeans_warm_sums<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(phi, ldphi, N, r, R, C, prev, sums, counts, fx_shift);
 }
 
 void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st) {
-  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  const int R = feature_ld(r);
   dim3 grid((C * R + 255) / 256, BH);
   k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, mu, sums, counts, maxabs_bits, fx_shift);
 }
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh, __nv_bfloat16* ml) {
-  const int R = r <= 16 ? 16 : r <= 32 ? 32 : r <= 48 ? 48 : 64;
+  const int R = feature_ld(r);
   if (mumax != nullptr) {
     k_kmeans_finalize<<<BH, 1024, 0, st>>>(mu, mu2, mumax, sums, counts, fx_shift, C, r, R, update, mh, ml);
   } else {

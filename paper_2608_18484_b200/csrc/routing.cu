@@ -430,48 +430,55 @@ __global__ void __launch_bounds__(256) k_probe_dist(const float* __restrict__ ph
   if (p1 <= p0) return;
   const float* ph = phi + (i64)bh * N * ldphi;
   const int* pm = perm + (i64)bh * N;
-  // lane owns columns lane and lane+32; the rows are read eight at a time (the loads are independent, the sums keep
-  // their order)
-  const bool h0 = lane < r, h1 = lane + 32 < r;
-  double c0 = 0.0, c1 = 0.0;
-  for (int p = p0; p < p1; p += 8) {
-    float x0[8], x1[8];
+  // lane owns columns lane, lane + 32, ... (up to four: 128 columns for a semantic query partition); the rows are
+  // read eight at a time (the loads are independent, the sums keep their order)
+  constexpr int kCols = 4;
+  bool has[kCols];
+  double cen[kCols];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float* row = ph + (i64)pm[min(p + j, p1 - 1)] * ldphi;
-      x0[j] = h0 ? row[lane] : 0.f;
-      x1[j] = h1 ? row[lane + 32] : 0.f;
+  for (int j = 0; j < kCols; ++j) { has[j] = lane + 32 * j < r; cen[j] = 0.0; }
+  for (int p = p0; p < p1; p += 8) {
+    float x[8][kCols];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float* row = ph + (i64)pm[min(p + q, p1 - 1)] * ldphi;
+#pragma unroll
+      for (int j = 0; j < kCols; ++j) x[q][j] = has[j] ? row[lane + 32 * j] : 0.f;
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (p + j < p1) { if (h0) c0 += (double)x0[j]; if (h1) c1 += (double)x1[j]; }
-  }
-  c0 /= (double)(p1 - p0);
-  c1 /= (double)(p1 - p0);
-  for (int p = p0; p < p1; p += 8) {
-    float x0[8], x1[8];
+    for (int q = 0; q < 8; ++q)
+      if (p + q < p1) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float* row = ph + (i64)pm[min(p + j, p1 - 1)] * ldphi;
-      x0[j] = h0 ? row[lane] : 0.f;
-      x1[j] = h1 ? row[lane + 32] : 0.f;
+        for (int j = 0; j < kCols; ++j) if (has[j]) cen[j] += (double)x[q][j];
+      }
+  }
+#pragma unroll
+  for (int j = 0; j < kCols; ++j) cen[j] /= (double)(p1 - p0);
+  for (int p = p0; p < p1; p += 8) {
+    float x[8][kCols];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float* row = ph + (i64)pm[min(p + q, p1 - 1)] * ldphi;
+#pragma unroll
+      for (int j = 0; j < kCols; ++j) x[q][j] = has[j] ? row[lane + 32 * j] : 0.f;
     }
     double s[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s[j] = 0.0;
-      if (h0) { const double t = (double)x0[j] - c0; s[j] += t * t; }
-      if (h1) { const double t = (double)x1[j] - c1; s[j] += t * t; }
+    for (int q = 0; q < 8; ++q) {
+      s[q] = 0.0;
+#pragma unroll
+      for (int j = 0; j < kCols; ++j)
+        if (has[j]) { const double t = (double)x[q][j] - cen[j]; s[q] += t * t; }
     }
     // eight independent butterflies
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) s[j] += __shfl_xor_sync(0xffffffffu, s[j], o);
+      for (int q = 0; q < 8; ++q) s[q] += __shfl_xor_sync(0xffffffffu, s[q], o);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (lane == j && p + j < p1) dist[(i64)bh * N + p + j] = sqrt(s[j]);
+    for (int q = 0; q < 8; ++q)
+      if (lane == q && p + q < p1) dist[(i64)bh * N + p + q] = sqrt(s[q]);
   }
 }
 

@@ -49,10 +49,13 @@ def plan_links(wl, i, Q, K, exp, feat, prm, warm=None):
     C = -(-N // wl.block)
     out = {}
     ref = orc.plan_head(Q, K, prm, i, warm=warm)
+    variant = prm.get("partition", 0)
     aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
-    # a1-a3
-    FK = feat["F_K"][i].astype(np.float64)
-    out["FF_K"] = rel_fro(FK @ FK.T, ref["F_K"] @ ref["F_K"].T)
+    # a1-a3 (a semantic K/V partition clusters K itself: no feature map)
+    out["FF_K"] = 0.0
+    if variant != orc.PARTITION_SEMANTIC:
+        FK = feat["F_K"][i].astype(np.float64)
+        out["FF_K"] = rel_fro(FK @ FK.T, ref["F_K"] @ ref["F_K"].T)
     # a4
     out["agree_K"] = float((aK == ref["a_K"]).mean())
     out["obj_K"] = orc.kmeans_objective(ref["phi_K"], _means(ref["phi_K"], aK, C), aK) / \
@@ -60,15 +63,20 @@ def plan_links(wl, i, Q, K, exp, feat, prm, warm=None):
     # a5: centroids and query metric of the GPU's own K/V groups
     kappa, n_k = orc.kv_centroids(K, aK, C)
     out["kappa"] = float(np.abs(feat["kappa"][i] - kappa).max())
-    F_Q, _ = orc.eig_feature_map(orc.query_response_metric(kappa, n_k), prm["rQ"])
-    FQ = feat["F_Q"][i].astype(np.float64)
-    out["FF_Q"] = rel_fro(FQ @ FQ.T, F_Q @ F_Q.T)
-    # a6
-    phi_ref = orc.query_response(Q, F_Q, prm["eps_rms"])
     phi_gpu = feat["phi_Q"][i].astype(np.float64)
     rows = np.random.default_rng(5).choice(N, min(N, 384), replace=False)
+    if variant == orc.PARTITION_RESPONSE_COUPLED:
+        F_Q, _ = orc.eig_feature_map(orc.query_response_metric(kappa, n_k), prm["rQ"])
+        FQ = feat["F_Q"][i].astype(np.float64)
+        out["FF_Q"] = rel_fro(FQ @ FQ.T, F_Q @ F_Q.T)
+        # a6
+        phi_ref = orc.query_response(Q, F_Q, prm["eps_rms"])
+        out["norm"] = float(np.abs((phi_gpu ** 2).sum(axis=1) / phi_ref.shape[1] - 1.0).max())
+    else:                                           # semantic query partition: the features are the queries themselves
+        phi_ref = np.asarray(Q, dtype=np.float64)
+        out["FF_Q"] = 0.0
+        out["norm"] = float(np.abs(phi_gpu - phi_ref).max())
     out["gram"] = rel_fro(phi_gpu[rows] @ phi_gpu[rows].T, phi_ref[rows] @ phi_ref[rows].T)
-    out["norm"] = float(np.abs((phi_gpu ** 2).sum(axis=1) / phi_ref.shape[1] - 1.0).max())
     # a7
     aQ_ref, _ = orc.kmeans(phi_ref, C, orc.stride_sample(C, N, prm["seed"], orc.TAG_Q_INIT, i), prm["kmeans_iters"],
                            init_assign=None if warm is None else warm["a_Q"])
@@ -147,11 +155,11 @@ def _means(X, a, C):
     return mu
 
 
-def run_case(wl):
+def run_case(wl, **extra):
     heads = [0, 1]
     host, (Qd, Kd, Vd) = heads_to_device(wl, heads)
     kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
-              softmax_scale=wl.softmax_scale)
+              softmax_scale=wl.softmax_scale, **extra)
     plan = B.sparsepr_plan(Qd, Kd, Vd, **kw)
     st = B.sparsepr_plan_stats(plan)
     exp = B.sparsepr_plan_export(plan)
@@ -212,3 +220,19 @@ def test_warm_started_plan_matches_the_oracle(name, wl):
     # the warm plan drives a full call
     O = B.sparsepr_attend(second, Q2, K2, V2)
     assert bool(np.isfinite(O.float().cpu().numpy()).all())
+
+
+@pytest.mark.parametrize("variant", [orc.PARTITION_KEY_RESPONSE_KV, orc.PARTITION_SEMANTIC], ids=["key-response-kv", "semantic"])
+@pytest.mark.parametrize("name,wl", CASES, ids=[c[0] for c in CASES])
+def test_partition_variants_match_the_oracle(name, wl, variant):
+    """The ablation partitions (k-means on the raw activations for one or both sides; d = 64 on the tensor-core
+    assignment, d = 128 on the CUDA-core one) link by link, and a full call on such a plan."""
+    st, links = run_case(wl, partition=variant)
+    assert st["device_error"] == 0
+    check_links(wl, links)
+    _, (Qd, Kd, Vd) = heads_to_device(wl, [0, 1])
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale, partition=variant)
+    plan = B.sparsepr_plan(Qd, Kd, Vd, **kw)
+    O = B.sparsepr_attend(plan, Qd, Kd, Vd)
+    assert bool(np.isfinite(O.float().cpu().numpy()).all()) and B.sparsepr_plan_stats(plan)["device_error"] == 0
