@@ -34,7 +34,7 @@ UNIT = "ms/call"
 # DRAM read + write bytes per head of one launch of the two block-sparse kernels, from ncu captures of 6 heads
 # (capture-size rule) of the named workload; a workload without a capture reports null.
 NCU_DRAM_BYTES_PER_HEAD = {
-    "video-dit-480p-like": {"k_attention_tc": 30.04e6, "k_attention_packed": 18.5e6},
+    "video-dit-480p-like": {"k_attention_tc": 35.93e6, "k_attention_packed": 18.58e6},
 }
 
 
@@ -200,6 +200,8 @@ def sweep(args, wl, kind):
 
     kind "sweep": density budget x probe rows x {hard drop, probe-fitted}, plus the full-rank (r_out = d_v) and
     lambda = 10 columns, on the given workload (the 720p-like shape unless --workload says otherwise).
+    kind "partition": the three partition variants (semantic, key-response K/V, response-coupled), hard drop and
+    probe-fitted.
     kind "cq": number of query groups C_q in {N/128, N/256, N/512} at the workload's density: accuracy against
     tensor efficiency (executed-pair and issued rates of the block-sparse stage)."""
     import torch
@@ -275,6 +277,11 @@ def sweep(args, wl, kind):
             measure({"rho": wl.density, "M": M, "mode": "probe-fitted, lambda=10"}, steps=1, density=wl.density, n_probe=M, lam=10.0)
             measure({"rho": wl.density, "M": M, "mode": "probe-fitted, r_out=d_v, lambda=10"}, steps=1, density=wl.density,
                     n_probe=M, r_out=wl.d, lam=10.0)
+    elif kind == "partition":
+        # the shape of the paper's partition / repair ablation (Table 2) at matched routed density
+        for name, v in (("semantic", 2), ("key-response K/V", 1), ("response-coupled", 0)):
+            measure({"partition": name}, steps=2, density=wl.density, n_probe=wl.n_probe, partition=v)
+            measure({"partition": name, "lambda": 10.0}, steps=1, density=wl.density, n_probe=wl.n_probe, partition=v, lam=10.0)
     else:
         C = -(-wl.N // wl.block)
         for div in (1, 2, 4):
@@ -293,7 +300,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-warm", action="store_true", help="skip the warm-started multi-call leg")
-    ap.add_argument("--study", default="", choices=["", "sweep", "cq"],
+    ap.add_argument("--study", default="", choices=["", "sweep", "cq", "partition"],
                     help="parameter study instead of the benchmark line: density x probes x mode, or the C_q frontier")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
