@@ -591,11 +591,26 @@ __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i6
   const int* pm = perm + (i64)bh * N;
   const int p0 = off[(i64)bh * (C + 1) + g], p1 = off[(i64)bh * (C + 1) + g + 1];
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int p = p0 + sub; p < p1; p += RPW) {
-    float v[8];
-    load8(base + (i64)pm[p] * sn + col, v);
+  // eight row loads in flight per lane (the walk is bound by the latency of the index -> row chain); the additions
+  // keep their order, and a slot beyond the group adds exact zeros
+  for (int p = p0 + sub; p < p1; p += RPW * 8) {
+    int src[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] += v[k];
+    for (int j = 0; j < 8; ++j) src[j] = p + j * RPW < p1 ? pm[p + j * RPW] : -1;
+    float v[8][8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (src[j] >= 0) {
+        load8(base + (i64)src[j] * sn + col, v[j]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[j][k] = 0.f;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] += v[j][k];
   }
   // combine the RPW interleaved partial sums in a fixed order
 #pragma unroll
