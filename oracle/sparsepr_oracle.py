@@ -502,41 +502,66 @@ def plan_head(Q, K, prm: dict, bh: int, warm=None):
     Where the query partition is semantic, the probe ranking of Algorithm A.1
     measures its distances in the raw query space, the space that partition
     was built in (reading: the paper runs the ablation with fixed probes)."""
-    Q = np.asarray(Q, dtype=np.float64)
-    K = np.asarray(K, dtype=np.float64)
-    N, d = Q.shape
-    C_k = prm["Ck"] or -(-N // prm["block"])
-    C_q = prm["Cq"] or -(-N // prm["block"])
-    M = min(prm["n_probe"], N) if prm["mode"] == 0 else 0
-    scale = prm["softmax_scale"] or 1.0 / np.sqrt(d)
-    seed = prm["seed"]
-    out = {"C_k": C_k, "C_q": C_q, "M": M, "scale": scale}
+    kv = plan_kv([Q], K, prm, bh, [bh], warm=warm)
+    return plan_query(Q, kv, prm, bh, warm=warm)
 
+
+def plan_kv(Qs, K, prm: dict, kv_bh: int, q_bhs, warm=None):
+    """The K/V side of the plan for one K/V head and the query heads `Qs` that attend to it (one for ordinary
+    multi-head attention; several under grouped-query attention, where the K/V partition and its metadata are
+    shared by the associated query heads, Section 4.3).
+
+    Reading for the grouped case (the paper does not say which query rows feed the key-response metric): every
+    associated query head contributes its own deterministic sample of M_s rows (sample offset keyed by the query
+    head's index) and M_K is the second moment of all of them together; the k-means initial rows are keyed by the
+    K/V head's index.  With one query head this is exactly the single-head plan."""
+    K = np.asarray(K, dtype=np.float64)
+    Qs = [np.asarray(Q, dtype=np.float64) for Q in Qs]
+    N, d = K.shape
+    C_k = prm["Ck"] or -(-N // prm["block"])
+    seed = prm["seed"]
     variant = prm.get("partition", PARTITION_RESPONSE_COUPLED)
     wK = None if warm is None else warm["a_K"]
-    wQ = None if warm is None else warm["a_Q"]
     T = prm["kmeans_iters"]
-    s_idx = stride_sample(min(prm["n_sample"], N), N, seed, TAG_QUERY_SAMPLE, bh)
+    s_idx = [stride_sample(min(prm["n_sample"], N), N, seed, TAG_QUERY_SAMPLE, bh) for bh in q_bhs]
     M_K = F_K = lam_K = M_Q = F_Q = lam_Q = None
     if variant == PARTITION_SEMANTIC:
         phi_K = K                                   # k-means on the key activations themselves
     else:
-        M_K = key_response_metric(Q[s_idx])
+        M_K = key_response_metric(np.concatenate([Q[i] for Q, i in zip(Qs, s_idx)], axis=0))
         F_K, lam_K = eig_feature_map(M_K, prm["rK"])
         phi_K = key_response(K, F_K)
-    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, bh), T, init_assign=wK)
+    a_K, mu_K = kmeans(phi_K, C_k, stride_sample(C_k, N, seed, TAG_KV_INIT, kv_bh), T, init_assign=wK)
     kappa, n_k = kv_centroids(K, a_K, C_k)
     if variant == PARTITION_RESPONSE_COUPLED:
         M_Q = query_response_metric(kappa, n_k)
         F_Q, lam_Q = eig_feature_map(M_Q, prm["rQ"])
-        phi_Q = query_response(Q, F_Q, prm["eps_rms"])
+    kv_perm, kv_inv, kv_off = group_permutation(a_K, C_k)
+    return dict(C_k=C_k, sample_idx=s_idx[0], sample_idx_all=s_idx, M_K=M_K, F_K=F_K, lam_K=lam_K, phi_K=phi_K, a_K=a_K,
+                mu_K=mu_K, kappa=kappa, n_k=n_k, M_Q=M_Q, F_Q=F_Q, lam_Q=lam_Q, kv_perm=kv_perm, kv_inv=kv_inv,
+                kv_off=kv_off)
+
+
+def plan_query(Q, kv: dict, prm: dict, bh: int, warm=None):
+    """The query side of the plan for one query head given the K/V side `kv` it attends to: query responses,
+    query partition, probes, cell scores and routes.  Returns the K/V side's entries as well."""
+    Q = np.asarray(Q, dtype=np.float64)
+    N, d = Q.shape
+    C_k = kv["C_k"]
+    C_q = prm["Cq"] or -(-N // prm["block"])
+    M = min(prm["n_probe"], N) if prm["mode"] == 0 else 0
+    scale = prm["softmax_scale"] or 1.0 / np.sqrt(d)
+    seed = prm["seed"]
+    variant = prm.get("partition", PARTITION_RESPONSE_COUPLED)
+    wQ = None if warm is None else warm["a_Q"]
+    kappa, n_k = kv["kappa"], kv["n_k"]
+    if variant == PARTITION_RESPONSE_COUPLED:
+        phi_Q = query_response(Q, kv["F_Q"], prm["eps_rms"])
     else:
         phi_Q = Q                                   # k-means on the query activations themselves
-    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), T, init_assign=wQ)
+    a_Q, mu_Q = kmeans(phi_Q, C_q, stride_sample(C_q, N, seed, TAG_Q_INIT, bh), prm["kmeans_iters"], init_assign=wQ)
     theta, n_q = query_centroids(Q, a_Q, C_q)
-
     q_perm, q_inv, q_off = group_permutation(a_Q, C_q)
-    kv_perm, kv_inv, kv_off = group_permutation(a_K, C_k)
     if M > 0:
         probe_idx, probe_w = probe_select(a_Q, phi_Q, C_q, M)
     else:
@@ -545,14 +570,21 @@ def plan_head(Q, K, prm: dict, bh: int, warm=None):
     budget = pair_budget(prm["density"], N, N, M)
     route_ptr, route_idx, pairs = route_select(score, n_q, n_k, budget,
                                                select_all=np.float32(prm["density"]) >= 1.0)
-    out.update(sample_idx=s_idx, M_K=M_K, F_K=F_K, lam_K=lam_K, phi_K=phi_K, a_K=a_K, mu_K=mu_K,
-               kappa=kappa, n_k=n_k, M_Q=M_Q, F_Q=F_Q, lam_Q=lam_Q, phi_Q=phi_Q, a_Q=a_Q, mu_Q=mu_Q,
-               theta=theta, n_q=n_q, q_perm=q_perm, q_inv=q_inv, q_off=q_off,
-               kv_perm=kv_perm, kv_inv=kv_inv, kv_off=kv_off, probe_idx=probe_idx, probe_w=probe_w,
-               score=score, budget=budget, route_ptr=route_ptr, route_idx=route_idx,
-               routed_pairs=pairs)
+    out = dict(kv)
+    out.update(C_q=C_q, M=M, scale=scale, phi_Q=phi_Q, a_Q=a_Q, mu_Q=mu_Q, theta=theta, n_q=n_q, q_perm=q_perm,
+               q_inv=q_inv, q_off=q_off, probe_idx=probe_idx, probe_w=probe_w, score=score, budget=budget,
+               route_ptr=route_ptr, route_idx=route_idx, routed_pairs=pairs)
     out["rho_route"], out["rho_exec"] = densities(pairs, N, N, M)
     return out
+
+
+def plan_group(Qs, K, prm: dict, kv_bh: int, first_q_bh: int, warm=None):
+    """Grouped-query attention: the plans of the query heads first_q_bh, first_q_bh + 1, ... that share K/V head
+    kv_bh.  One K/V side, one query side per query head.  `warm` = {"a_K": ..., "a_Q": [one per query head]}."""
+    bhs = [first_q_bh + g for g in range(len(Qs))]
+    kv = plan_kv(Qs, K, prm, kv_bh, bhs, warm=warm)
+    return [plan_query(Q, kv, prm, bh, warm=None if warm is None else dict(a_K=warm["a_K"], a_Q=warm["a_Q"][g]))
+            for g, (Q, bh) in enumerate(zip(Qs, bhs))]
 
 
 def attend_head(Q, K, V, plan: dict, prm: dict, rows=None):

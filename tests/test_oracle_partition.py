@@ -206,6 +206,32 @@ def test_partition_variants():
         assert np.all(np.diff(p["route_ptr"]) >= (p["n_q"] > 0))
 
 
+def test_grouped_query_plan():
+    """K/V side shared by the query heads of a group: with one query head it is the single-head plan; with several,
+    the key-response metric is the second moment of all their sampled rows, the K/V partition is common, and each
+    query head has its own query partition and routes against the shared K/V groups."""
+    rng = np.random.default_rng(31)
+    N, d = 320, 16
+    K = rng.normal(size=(N, d))
+    Qs = [rng.normal(size=(N, d)) + 0.5 * K for _ in range(3)]
+    prm = orc.default_params(density=0.4, block=64, n_sample=32, n_probe=8, rK=8, rQ=8, kmeans_iters=3, softmax_scale=1.0)
+    single = orc.plan_head(Qs[0], K, prm, 5)
+    group1 = orc.plan_group(Qs[:1], K, prm, 5, 5)[0]
+    for key in ("a_K", "a_Q", "route_idx", "probe_idx", "M_K", "F_Q"):
+        assert np.array_equal(single[key], group1[key]), key
+    plans = orc.plan_group(Qs, K, prm, 2, 6)
+    rows = np.concatenate([Q[orc.stride_sample(32, N, 0, orc.TAG_QUERY_SAMPLE, 6 + g)] for g, Q in enumerate(Qs)])
+    assert np.allclose(plans[0]["M_K"], rows.T @ rows / rows.shape[0], atol=1e-14)
+    assert all(np.array_equal(p["a_K"], plans[0]["a_K"]) and p["kappa"] is plans[0]["kappa"] for p in plans)
+    assert np.array_equal(plans[0]["a_K"], orc.kmeans(plans[0]["phi_K"], 5, orc.stride_sample(5, N, 0, orc.TAG_KV_INIT, 2), 3)[0])
+    assert not np.array_equal(plans[0]["a_Q"], plans[1]["a_Q"])
+    budget = orc.pair_budget(0.4, N, N, 8)
+    for g, p in enumerate(plans):
+        assert np.array_equal(p["a_Q"], orc.kmeans(p["phi_Q"], 5, orc.stride_sample(5, N, 0, orc.TAG_Q_INIT, 6 + g), 3)[0])
+        assert p["routed_pairs"] <= budget
+        assert p["routed_pairs"] == orc.routed_pairs(p["n_q"], p["n_k"], p["route_ptr"], p["route_idx"])
+
+
 def test_group_permutation():
     rng = np.random.default_rng(7)
     a = rng.integers(0, 9, size=100)
