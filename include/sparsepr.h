@@ -16,7 +16,8 @@
  *     valid on the CUDA device that is current when the call is made.
  *   - Q, K, V, O are [B, H, N, d] tensors addressed through element strides for
  *     B, H and N; the last dimension is contiguous.  Rows must start on a
- *     16-byte boundary.  N_q = N_k = N and d_v = d.
+ *     16-byte boundary.  N_q = N_k = N and d_v = d.  K and V may have fewer heads
+ *     than Q (grouped-query attention, sparsepr_shape_t.Hkv).
  *   - The library never allocates or frees device memory: the caller owns all
  *     tensors and both workspaces.  A plan handle is a small host object that
  *     points into the plan workspace; it is valid until the workspace is released
@@ -77,6 +78,13 @@ typedef struct {
   int32_t B, H, N, d, dv;
   int32_t dtype;                       /* sparsepr_dtype_t of Q, K, V and O */
   int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* B, H, N */
+  /* Grouped-query attention: number of K/V heads (0 or H = ordinary multi-head attention; must divide H).  K and V
+   * are then [B, Hkv, N, d] (their head strides count K/V heads) and query head h attends to K/V head
+   * h / (H / Hkv).  The K/V partition, permutation, offsets and centroids are computed once per K/V head from the
+   * pooled query samples of its query heads and shared by them (Section 4.3); every query head keeps its own query
+   * partition, probes and routes.  Per-K/V-head arrays of sparsepr_plan_host_t and sparsepr_plan_features_t
+   * (kv_assign, kv_perm, kv_off, F_K, F_Q, kappa) have B*Hkv entries.  bf16, d = 128 only. */
+  int32_t Hkv;
 } sparsepr_shape_t;
 
 /* Method parameters (Appendix C, Table C.1, plus the knobs the paper leaves

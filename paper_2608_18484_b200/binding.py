@@ -31,7 +31,7 @@ class SparsePRError(RuntimeError):
 class Shape(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("N", C.c_int32), ("d", C.c_int32), ("dv", C.c_int32),
                 ("dtype", C.c_int32), ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
-                ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3)]
+                ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3), ("Hkv", C.c_int32)]
 
 
 class Params(C.Structure):
@@ -145,7 +145,9 @@ def make_shape(Q, K, V, O) -> Shape:
         if t.dim() != 4 or not t.is_cuda or t.stride(3) != 1:
             raise ValueError("expected CUDA tensors [B, H, N, d] with a contiguous last dimension")
     B, H, N, d = Q.shape
-    s = Shape(B=B, H=H, N=N, d=d, dv=V.shape[3], dtype=_dtype_code(Q))
+    if K.shape[1] != V.shape[1] or H % K.shape[1] != 0:
+        raise ValueError("K and V need the same number of heads, a divisor of the number of query heads")
+    s = Shape(B=B, H=H, N=N, d=d, dv=V.shape[3], dtype=_dtype_code(Q), Hkv=K.shape[1])
     for name, t in (("q_stride", Q), ("k_stride", K), ("v_stride", V), ("o_stride", O)):
         getattr(s, name)[:] = [t.stride(0), t.stride(1), t.stride(2)]
     return s
@@ -173,6 +175,10 @@ class Plan:
     @property
     def BH(self):
         return self.shape.B * self.shape.H
+
+    @property
+    def BHkv(self):
+        return self.shape.B * (self.shape.Hkv or self.shape.H)
 
     @property
     def groups(self):
@@ -261,12 +267,12 @@ def sparsepr_plan_stats(plan: Plan) -> dict:
 
 
 def _host_arrays(plan: Plan) -> dict:
-    BH, N = plan.BH, plan.shape.N
+    BH, N, BHkv = plan.BH, plan.shape.N, plan.BHkv
     Ck, Cq = plan.groups
     M = max(plan.M, 1)
-    return dict(kv_assign=np.empty((BH, N), np.int32), q_assign=np.empty((BH, N), np.int32),
-                kv_perm=np.empty((BH, N), np.int32), q_perm=np.empty((BH, N), np.int32),
-                kv_off=np.empty((BH, Ck + 1), np.int32), q_off=np.empty((BH, Cq + 1), np.int32),
+    return dict(kv_assign=np.empty((BHkv, N), np.int32), q_assign=np.empty((BH, N), np.int32),
+                kv_perm=np.empty((BHkv, N), np.int32), q_perm=np.empty((BH, N), np.int32),
+                kv_off=np.empty((BHkv, Ck + 1), np.int32), q_off=np.empty((BH, Cq + 1), np.int32),
                 route_ptr=np.empty((BH, Cq + 1), np.int32), route_idx=np.empty((BH, Cq * Ck), np.int32),
                 probe_idx=np.empty((BH, M), np.int32), probe_w=np.empty((BH, M), np.float32),
                 routed_pairs=np.empty((BH,), np.int64))
@@ -292,7 +298,8 @@ def sparsepr_plan_export_features(plan: Plan, fields=("F_K", "F_Q", "phi_Q", "ka
     if plan.params.partition != 0:                  # semantic query partition: phi_Q holds the raw queries
         rQ = d
         fields = tuple(f for f in fields if f != "F_Q" and not (f == "F_K" and plan.params.partition == 2))
-    shapes = dict(F_K=(BH, d, rK), F_Q=(BH, d, rQ), phi_Q=(BH, N, rQ), kappa=(BH, Ck, d), theta=(BH, Cq, d),
+    BHkv = plan.BHkv
+    shapes = dict(F_K=(BHkv, d, rK), F_Q=(BHkv, d, rQ), phi_Q=(BH, N, rQ), kappa=(BHkv, Ck, d), theta=(BH, Cq, d),
                   score=(BH, Cq, Ck))
     arrs = {k: np.empty(shapes[k], np.float32) for k in fields}
     pf = PlanFeatures(**{k: v.ctypes.data for k, v in arrs.items()})
@@ -319,7 +326,7 @@ def sparsepr_plan_import(Q, K, V, host: dict, params: Params | None = None, **kw
             slab[i, :len(r)] = r
         ridx = slab
     a["route_idx"] = np.ascontiguousarray(ridx, dtype=np.int32)
-    assert a["route_idx"].shape == (BH, Cq * Ck) and a["kv_assign"].shape == (BH, N)
+    assert a["route_idx"].shape == (BH, Cq * Ck) and a["kv_assign"].shape == (shape.B * (shape.Hkv or shape.H), N)
     M = 0 if params.mode == 1 else min(params.n_probe, N)
     if M:
         a["probe_idx"] = np.ascontiguousarray(host["probe_idx"], dtype=np.int32)

@@ -41,6 +41,7 @@ struct Carver {                       // bump allocator over a caller-owned work
 
 struct Resolved {
   int B, H, BH, N, d, dtype, es;
+  int Hkv, G, BHkv;                    // K/V heads, query heads per K/V head (1 = ordinary multi-head attention), B * Hkv
   int Ck, Cq, Cmax, Ms, M, rK, rQ, RK, RQ, Rmax, r_out, T, mode;
   int partition;                       // sparsepr_partition_t
   int fK, fQ;                          // width of the features each side is clustered in: rK / rQ, or d for raw activations
@@ -58,6 +59,11 @@ sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p,
   if (s->dtype != SPARSEPR_F32 && s->dtype != SPARSEPR_BF16) return SPARSEPR_ERR_INVALID_ARG;
   if ((s->d != 64 && s->d != 128) || s->dv != s->d) return SPARSEPR_ERR_UNSUPPORTED;
   r->B = s->B; r->H = s->H; r->BH = s->B * s->H; r->N = s->N; r->d = s->d; r->dtype = s->dtype;
+  r->Hkv = s->Hkv > 0 ? s->Hkv : s->H;
+  if (s->Hkv < 0 || r->Hkv > s->H || s->H % r->Hkv != 0) return SPARSEPR_ERR_INVALID_ARG;
+  r->G = s->H / r->Hkv; r->BHkv = s->B * r->Hkv;
+  // grouped-query attention runs on the tensor-core kernels only
+  if (r->G > 1 && !(s->dtype == SPARSEPR_BF16 && s->d == 128)) return SPARSEPR_ERR_UNSUPPORTED;
   r->es = s->dtype == SPARSEPR_BF16 ? 2 : 4;
   const int vec = 16 / r->es;
   for (int i = 0; i < 3; ++i) {
@@ -250,6 +256,7 @@ struct sparsepr_plan_s {
   __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged;
   int *rem_pos, *rem_grp, *rem_cnt;      // rows of the short group remainders (packed attention tiles)
   int* km_changed;                       // [2 sides][T + 1][BH] rows that changed group in each k-means pass
+  double* Mpool;                         // [BHkv][d][d] key-response metric pooled over the query heads of a K/V head (grouped-query attention only)
 };
 
 namespace {
@@ -289,8 +296,9 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
   int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
   int* km_changed = c.take<int>(2 * (size_t)(r.T + 1) * BH);
+  double* Mpool = c.take<double>(r.G > 1 ? (size_t)r.BHkv * d * d : 0);
   if (p) {
-    p->km_changed = km_changed; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
+    p->km_changed = km_changed; p->Mpool = Mpool; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -345,28 +353,28 @@ i64 pair_budget(const Resolved& r) {
   return std::max<i64>(total - (i64)r.M * r.N, 0);
 }
 
-void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, const int* warm_prev, cudaStream_t st) {
+void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, const int* warm_prev, int nheads, cudaStream_t st) {
   const Resolved& R = p->r;
   const int ld = round16(r);
   // changed[t][bh], t = 1..T: rows of head bh that changed group in pass t.  A pass that changes nothing proves the
   // fixed point, so the later passes of that head return at once (their result would be identical).
   int* changed = p->km_changed + (tag == kTagQInit ? (size_t)(R.T + 1) * R.BH : 0);
   cudaMemsetAsync(changed, 0, (size_t)(R.T + 1) * R.BH * sizeof(int), st);
-  launch_kmeans_init(p->phi, ld, R.BH, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
+  launch_kmeans_init(p->phi, ld, nheads, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
   const bool tcp = kmeans_tc_supported() && r <= kMaxRank;
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
   // (with the tensor-core assignment the finalize step also writes the two bf16 words of every centroid)
   // warm start: the initial centroids become the means of the current features over the previous partition's groups
-  if (warm_prev) launch_kmeans_warm_sums(p->phi, ld, R.BH, R.N, r, C, warm_prev, p->sums, p->counts, p->fx_shift, st);
-  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, warm_prev ? 1 : 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
-  if (tcp) launch_split_bf16(p->phi, ld, (i64)R.BH * R.N, r, p->xh, p->xl, p->xnorm, st);
+  if (warm_prev) launch_kmeans_warm_sums(p->phi, ld, nheads, R.N, r, C, warm_prev, p->sums, p->counts, p->fx_shift, st);
+  launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, nheads, C, r, warm_prev ? 1 : 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
+  if (tcp) launch_split_bf16(p->phi, ld, (i64)nheads * R.N, r, p->xh, p->xl, p->xnorm, st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
     const int* prev = t > 1 ? changed + (size_t)(t - 1) * R.BH : nullptr;
     int* cur = changed + (size_t)t * R.BH;
     if (tcp) {
       KmeansTcArgs ka{};
-      ka.BH = R.BH; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
+      ka.BH = nheads; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
       ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2;
       ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
       ka.flagged = p->flagged; ka.flag_count = p->recheck + 1; ka.recheck_total = p->recheck; ka.err = p->err;
@@ -374,10 +382,10 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
       launch_kmeans_assign_tc(ka, st);
     } else {
       if (!upd) cudaMemsetAsync(p->recheck, 0, sizeof(int), st);
-      launch_kmeans_assign(p->phi, ld, R.BH, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
+      launch_kmeans_assign(p->phi, ld, nheads, R.N, r, p->mu, p->mu2, p->mumax, C, assign, upd ? p->sums : nullptr,
                            upd ? p->counts : nullptr, p->fx_shift, p->recheck, prev, cur, st);
     }
-    if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, R.BH, C, r, 1, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
+    if (upd) launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, nheads, C, r, 1, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   }
 }
 
@@ -386,6 +394,15 @@ __global__ void k_pad_rows(const float* __restrict__ in, int n, int r, int R, fl
   for (i64 e = (i64)blockIdx.x * blockDim.x + threadIdx.x; e < (i64)n * R; e += (i64)gridDim.x * blockDim.x) {
     const int k = (int)(e % R);
     out[e] = k < r ? in[(e / R) * r + k] : 0.f;
+  }
+}
+// key-response metric of a K/V head = mean of the sampled-query second moments of its G query heads
+__global__ void k_pool_metric(const double* __restrict__ Mq, int G, int dd, double* __restrict__ out) {
+  const int kvh = blockIdx.y;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < dd; e += gridDim.x * blockDim.x) {
+    double s = 0.0;
+    for (int g = 0; g < G; ++g) s += Mq[((i64)kvh * G + g) * dd + e];
+    out[(i64)kvh * dd + e] = s / (double)G;
   }
 }
 __global__ void k_sizes_from_off(const int* __restrict__ off, int C, int* __restrict__ sizes) {
@@ -472,6 +489,11 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   sparsepr_status_t s = make_plan(shape, params, workspace, workspace_bytes, cuda_stream, &p);
   if (s != SPARSEPR_OK) return s;
   const Resolved& r = p->r;
+  // grouped-query attention shares feature maps and K/V copies between heads: tensor-core kernels only
+  if (r.G > 1 && !(kmeans_tc_supported() && project_tc_supported(r.dtype, r.d, r.rQ, r.qs) && project_tc_supported(r.dtype, r.d, r.rK, r.ks))) {
+    delete p;
+    return SPARSEPR_ERR_UNSUPPORTED;
+  }
   cudaStream_t st = p->stream;
   cudaGetLastError();
   cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
@@ -480,22 +502,29 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   // K/V partition: sampled-query metric -> F_K -> phi_K -> k-means (semantic variant: k-means on K itself)
   if (r.partition == SPARSEPR_PARTITION_SEMANTIC) {
     tm.mark(SPARSEPR_STAGE_KEY_METRIC);
-    launch_raw_features(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, p->phi, p->maxabs, p->err, st);
+    launch_raw_features(r.dtype, K, r.ks, r.BHkv, r.Hkv, r.N, r.d, p->phi, p->maxabs, p->err, st);
   } else {
+    // every query head samples its own rows; under grouped-query attention the K/V head's metric is the mean over its
+    // query heads (Section 4.3: the K/V partition is shared by the associated query heads)
     launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
-    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
+    const double* metric = p->Mmat;
+    if (r.G > 1) {
+      k_pool_metric<<<dim3(16, r.BHkv), 256, 0, st>>>(p->Mmat, r.G, r.d * r.d, p->Mpool);
+      metric = p->Mpool;
+    }
+    launch_eig_top(metric, (i64)r.d * r.d, r.BHkv, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
     tm.mark(SPARSEPR_STAGE_KEY_METRIC);
     if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
-      if (!launch_project_tc(K, r.ks, r.BH, r.H, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+      if (!launch_project_tc(K, r.ks, r.BHkv, r.Hkv, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
     } else {
-      launch_project(r.dtype, K, r.ks, r.BH, r.H, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
+      launch_project(r.dtype, K, r.ks, r.BHkv, r.Hkv, r.N, r.d, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->err, st);
     }
   }
   tm.mark(SPARSEPR_STAGE_KEY_PROJECT);
-  run_kmeans(p, r.fK, r.Ck, kTagKvInit, p->a_K, warm_kv, st);
+  run_kmeans(p, r.fK, r.Ck, kTagKvInit, p->a_K, warm_kv, r.BHkv, st);
   tm.mark(SPARSEPR_STAGE_KEY_KMEANS);
-  launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
-  launch_group_means(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
+  launch_group_sort(p->a_K, r.BHkv, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
+  launch_group_means(r.dtype, K, r.ks, r.BHkv, r.Hkv, p->kv_perm, p->kv_off, r.N, r.Ck, r.d, p->kappa, p->nk, st);
   tm.mark(SPARSEPR_STAGE_KEY_PERMUTE);
   // query partition: centroid metric -> F_Q -> phi_Q -> k-means (other variants: k-means on Q itself)
   cudaMemsetAsync(p->maxabs, 0, r.BH * sizeof(unsigned), st);
@@ -503,17 +532,17 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
     tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
     launch_raw_features(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, p->phi, p->maxabs, p->err, st);
   } else {
-    launch_centroid_gram(p->kappa, p->nk, r.BH, r.Ck, r.d, p->Mmat, st);
-    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BH, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
+    launch_centroid_gram(p->kappa, p->nk, r.BHkv, r.Ck, r.d, p->Mmat, st);
+    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BHkv, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
     tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
     if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {
-      if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
+      if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st, r.G)) { delete p; return SPARSEPR_ERR_CUDA; }
     } else {
       launch_project(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->err, st);
     }
   }
   tm.mark(SPARSEPR_STAGE_QUERY_PROJECT);
-  run_kmeans(p, r.fQ, r.Cq, kTagQInit, p->a_Q, warm_q, st);
+  run_kmeans(p, r.fQ, r.Cq, kTagQInit, p->a_Q, warm_q, r.BH, st);
   tm.mark(SPARSEPR_STAGE_QUERY_KMEANS);
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
   launch_group_means(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, p->q_off, r.N, r.Cq, r.d, p->theta, p->nq, st);
@@ -525,9 +554,9 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   if (r.M > 0)
     launch_probe_select(p->phi, r.RQ, r.fQ, p->q_perm, p->q_off, p->nq, r.BH, r.N, r.Cq, r.M, p->probe_dist, p->probe_idx, p->probe_w, ps);
   tm.mark(SPARSEPR_STAGE_PROBE_SELECT);
-  launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, st);
+  launch_cell_scores(p->theta, p->kappa, p->nq, p->nk, r.BH, r.Cq, r.Ck, r.d, r.scale, p->score, r.G, st);
   launch_route_select(p->score, p->nq, p->nk, r.BH, r.Cq, r.Ck, pair_budget(r), r.density >= 1.0f, p->route_ptr,
-                      p->route_idx, p->rstate, nullptr, st);
+                      p->route_idx, p->rstate, nullptr, r.G, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
   launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
@@ -584,7 +613,7 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   cudaGetLastError();
   const size_t BH = r.BH, N = r.N;
   cudaMemsetAsync(p->err, 0, 64 * sizeof(int), st);
-  cudaMemcpyAsync(p->a_K, in->kv_assign, BH * N * sizeof(int), cudaMemcpyHostToDevice, st);
+  cudaMemcpyAsync(p->a_K, in->kv_assign, (size_t)r.BHkv * N * sizeof(int), cudaMemcpyHostToDevice, st);
   cudaMemcpyAsync(p->a_Q, in->q_assign, BH * N * sizeof(int), cudaMemcpyHostToDevice, st);
   cudaMemcpyAsync(p->route_ptr, in->route_ptr, BH * (r.Cq + 1) * sizeof(int), cudaMemcpyHostToDevice, st);
   cudaMemcpyAsync(p->route_idx, in->route_idx, BH * (size_t)r.Cq * r.Ck * sizeof(int), cudaMemcpyHostToDevice, st);
@@ -592,11 +621,11 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
     cudaMemcpyAsync(p->probe_idx, in->probe_idx, BH * r.M * sizeof(int), cudaMemcpyHostToDevice, st);
     cudaMemcpyAsync(p->probe_w, in->probe_w, BH * r.M * sizeof(float), cudaMemcpyHostToDevice, st);
   }
-  launch_group_sort(p->a_K, r.BH, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
+  launch_group_sort(p->a_K, r.BHkv, r.N, r.Ck, p->kv_perm, p->kv_inv, p->kv_off, p->err, st);
   launch_group_sort(p->a_Q, r.BH, r.N, r.Cq, p->q_perm, p->q_inv, p->q_off, p->err, st);
-  k_sizes_from_off<<<dim3((r.Ck + 255) / 256, r.BH), 256, 0, st>>>(p->kv_off, r.Ck, p->nk);
+  k_sizes_from_off<<<dim3((r.Ck + 255) / 256, r.BHkv), 256, 0, st>>>(p->kv_off, r.Ck, p->nk);
   k_sizes_from_off<<<dim3((r.Cq + 255) / 256, r.BH), 256, 0, st>>>(p->q_off, r.Cq, p->nq);
-  launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, st);
+  launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, r.G, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
   launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
@@ -623,15 +652,15 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
   cudaGetLastError();
   StageTimer tm(prof, st);
   launch_gather_rows(r.dtype, Q, r.qs, r.BH, r.H, p->q_perm, r.N, r.d, w.Qg, st);
-  launch_gather_rows(r.dtype, K, r.ks, r.BH, r.H, p->kv_perm, r.N, r.d, w.Kg, st);
-  launch_gather_rows(r.dtype, V, r.vs, r.BH, r.H, p->kv_perm, r.N, r.d, w.Vg, st);
+  launch_gather_rows(r.dtype, K, r.ks, r.BHkv, r.Hkv, p->kv_perm, r.N, r.d, w.Kg, st);
+  launch_gather_rows(r.dtype, V, r.vs, r.BHkv, r.Hkv, p->kv_perm, r.N, r.d, w.Vg, st);
   tm.mark(SPARSEPR_STAGE_GATHER);
   const bool fitted = r.mode == 0 && r.M > 0;
   AttnArgs aa{};
   aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.scale = r.scale;
   aa.Q = w.Qg; aa.K = w.Kg; aa.V = w.Vg;
   aa.q_off = p->q_off; aa.kv_off = p->kv_off; aa.route_ptr = p->route_ptr; aa.route_idx = p->route_idx;
-  aa.q_perm = p->q_perm; aa.tile_off = p->tile_off; aa.Cq = r.Cq; aa.Ck = r.Ck;
+  aa.q_perm = p->q_perm; aa.tile_off = p->tile_off; aa.Cq = r.Cq; aa.Ck = r.Ck; aa.kv_div = r.G;
   aa.O = O; for (int i = 0; i < 3; ++i) aa.os[i] = r.os[i];
   aa.O_sparse = O_sparse;
   aa.err = p->err;
@@ -646,7 +675,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     if (overlap) { fork_side(p, st); fs = p->side; }
     ProbeArgs pa{};
     pa.dtype = r.dtype; pa.BH = r.BH; pa.H = r.H; pa.N = r.N; pa.d = r.d; pa.M = r.M; pa.Ck = r.Ck; pa.Cq = r.Cq;
-    pa.n_split = w.n_split; pa.scale = r.scale; pa.Q = Q;
+    pa.n_split = w.n_split; pa.scale = r.scale; pa.Q = Q; pa.kv_div = r.G;
     for (int i = 0; i < 3; ++i) pa.qs[i] = r.qs[i];
     pa.Kg = w.Kg; pa.Vg = w.Vg; pa.probe_idx = p->probe_idx; pa.q_assign = p->a_Q; pa.kv_off = p->kv_off;
     pa.route_ptr = p->route_ptr; pa.route_idx = p->route_idx; pa.partial = w.partial; pa.X = w.X; pa.Dn = w.Dn;
@@ -723,7 +752,7 @@ sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_sc
   if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
   cudaGetLastError();
   AttnArgs aa{};
-  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d;
+  aa.dtype = r.dtype; aa.BH = r.BH; aa.H = r.H; aa.N = r.N; aa.d = r.d; aa.kv_div = r.G;
   aa.scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)r.d);
   aa.Q = Q; aa.K = K; aa.V = V; aa.O = O;
   for (int i = 0; i < 3; ++i) { aa.qs[i] = r.qs[i]; aa.ks[i] = r.ks[i]; aa.vs[i] = r.vs[i]; aa.os[i] = r.os[i]; }
@@ -741,7 +770,7 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
   if (cudaStreamSynchronize(p->stream) != cudaSuccess || (p->side && cudaStreamSynchronize(p->side) != cudaSuccess)) return SPARSEPR_ERR_CUDA;
   std::memset(out, 0, sizeof(*out));
   std::vector<RouteState> rs(r.BH);
-  std::vector<int> qo((size_t)r.BH * (r.Cq + 1)), ko((size_t)r.BH * (r.Ck + 1)), rp((size_t)r.BH * (r.Cq + 1));
+  std::vector<int> qo((size_t)r.BH * (r.Cq + 1)), ko((size_t)r.BHkv * (r.Ck + 1)), rp((size_t)r.BH * (r.Cq + 1));
   std::vector<int> ri((size_t)r.BH * r.Cq * r.Ck);
   int errw[2] = {0, 0};
   if (cudaMemcpy(rs.data(), p->rstate, rs.size() * sizeof(RouteState), cudaMemcpyDeviceToHost) != cudaSuccess ||
@@ -762,7 +791,7 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     out->rho_route_min = std::min(out->rho_route_min, rho);
     out->rho_route_max = std::max(out->rho_route_max, rho);
     int neK = 0, neQ = 0;
-    const int* k = &ko[(size_t)bh * (r.Ck + 1)];
+    const int* k = &ko[(size_t)(bh / r.G) * (r.Ck + 1)];
     const int* q = &qo[(size_t)bh * (r.Cq + 1)];
     for (int g = 0; g < r.Ck; ++g) { neK += k[g + 1] > k[g]; out->max_kv_group = std::max(out->max_kv_group, k[g + 1] - k[g]); }
     for (int g = 0; g < r.Cq; ++g) { neQ += q[g + 1] > q[g]; out->max_q_group = std::max(out->max_q_group, q[g + 1] - q[g]); }
@@ -811,7 +840,7 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
   if (cudaMemcpy(ch.data(), p->km_changed, ch.size() * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SPARSEPR_ERR_CUDA;
   for (int side = 0; side < 2 && !p->imported; ++side) {
     int worst = 0;
-    for (int bh = 0; bh < r.BH; ++bh) {
+    for (int bh = 0; bh < (side == 0 ? r.BHkv : r.BH); ++bh) {
       int ran = 1;
       while (ran < r.T && ch[((size_t)side * (r.T + 1) + ran) * r.BH + bh] > 0) ++ran;
       worst = std::max(worst, ran);
@@ -828,9 +857,10 @@ sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* p, sparsepr_plan_h
   const size_t BH = r.BH, N = r.N;
   bool ok = true;
   auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };
-  cp(o->kv_assign, p->a_K, BH * N * 4); cp(o->q_assign, p->a_Q, BH * N * 4);
-  cp(o->kv_perm, p->kv_perm, BH * N * 4); cp(o->q_perm, p->q_perm, BH * N * 4);
-  cp(o->kv_off, p->kv_off, BH * (r.Ck + 1) * 4); cp(o->q_off, p->q_off, BH * (r.Cq + 1) * 4);
+  const size_t BHkv = r.BHkv;
+  cp(o->kv_assign, p->a_K, BHkv * N * 4); cp(o->q_assign, p->a_Q, BH * N * 4);
+  cp(o->kv_perm, p->kv_perm, BHkv * N * 4); cp(o->q_perm, p->q_perm, BH * N * 4);
+  cp(o->kv_off, p->kv_off, BHkv * (r.Ck + 1) * 4); cp(o->q_off, p->q_off, BH * (r.Cq + 1) * 4);
   cp(o->route_ptr, p->route_ptr, BH * (r.Cq + 1) * 4); cp(o->route_idx, p->route_idx, BH * (size_t)r.Cq * r.Ck * 4);
   cp(o->probe_idx, p->probe_idx, BH * r.M * 4); cp(o->probe_w, p->probe_w, BH * r.M * 4);
   if (o->routed_pairs) {
@@ -849,11 +879,12 @@ sparsepr_status_t sparsepr_plan_export_features(const sparsepr_plan_t* p, sparse
   const size_t BH = r.BH, N = r.N, d = r.d;
   bool ok = true;
   auto cp = [&](void* dst, const void* src, size_t bytes) { if (dst && bytes) ok &= cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost) == cudaSuccess; };
-  if (r.partition != SPARSEPR_PARTITION_SEMANTIC) cp(o->F_K, p->FK, BH * d * r.rK * 4);
-  if (r.partition == SPARSEPR_PARTITION_RESPONSE_COUPLED) cp(o->F_Q, p->FQ, BH * d * r.rQ * 4);
+  const size_t BHkv = r.BHkv;
+  if (r.partition != SPARSEPR_PARTITION_SEMANTIC) cp(o->F_K, p->FK, BHkv * d * r.rK * 4);
+  if (r.partition == SPARSEPR_PARTITION_RESPONSE_COUPLED) cp(o->F_Q, p->FQ, BHkv * d * r.rQ * 4);
   if (o->phi_Q)                                                // rows are padded to RQ floats on the device
     ok &= cudaMemcpy2D(o->phi_Q, (size_t)r.fQ * 4, p->phi, (size_t)r.RQ * 4, (size_t)r.fQ * 4, BH * N, cudaMemcpyDeviceToHost) == cudaSuccess;
-  cp(o->kappa, p->kappa, BH * r.Ck * d * 4); cp(o->theta, p->theta, BH * r.Cq * d * 4);
+  cp(o->kappa, p->kappa, BHkv * r.Ck * d * 4); cp(o->theta, p->theta, BH * r.Cq * d * 4);
   cp(o->score, p->score, BH * (size_t)r.Cq * r.Ck * 4);
   return ok ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
@@ -927,7 +958,7 @@ sparsepr_status_t sparsepr_stage_route(int32_t Cq, int32_t Ck, const float* scor
   if (ensure_init() != cudaSuccess) return SPARSEPR_ERR_CUDA;
   cudaGetLastError();
   launch_route_select(score, nq, nk, 1, Cq, Ck, pair_budget, select_all, route_ptr, route_idx, nullptr, reinterpret_cast<i64*>(pairs_out),
-                      static_cast<cudaStream_t>(cuda_stream));
+                      1, static_cast<cudaStream_t>(cuda_stream));
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 

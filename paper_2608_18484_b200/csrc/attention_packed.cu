@@ -63,6 +63,7 @@ struct Maps { CUtensorMap m[4]; };      // the same tensor with boxes of 16, 32,
 
 struct Params {
   int BH, H, N, Cq, Ck;
+  int kv_div;                                  // query heads per K/V head: Kg, Vg and kv_off are indexed by bh / kv_div
   float scale_log2;
   const int *rem_pos, *rem_grp, *rem_cnt;      // [BH][N] group-major position and query group of every packed row; [BH] their number
   const int *kv_off, *route_ptr, *route_idx, *q_perm;
@@ -103,7 +104,8 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
   const int words = (prm.Ck + 31) / 32;
   const int* rpos = prm.rem_pos + (i64)bh * prm.N + m0;
   const int* rgrp = prm.rem_grp + (i64)bh * prm.N + m0;
-  const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
+  const int kvh = bh / prm.kv_div;
+  const int* kvoff = prm.kv_off + (i64)kvh * (prm.Ck + 1);
 
   if (tid == 0) {
     for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == P_FULL || i == Q_FULL || i == S_FREE || i == S_FREE + 1) ? 256 : 1);
@@ -202,8 +204,8 @@ k_attention_packed(const __grid_constant__ Maps mapsK, const __grid_constant__ M
         __syncwarp();
         if (my_k >= 0) {
           const uint32_t dst = buf0 + s * kTileBytes + lane * kSubBytes;
-          tma_load_4d(dst, &maps->m[my_k], bar(full0 + s), 0, my_start, bh, 0);
-          tma_load_4d(dst + kHalfBytes, &maps->m[my_k], bar(full0 + s), 64, my_start, bh, 0);
+          tma_load_4d(dst, &maps->m[my_k], bar(full0 + s), 0, my_start, kvh, 0);
+          tma_load_4d(dst + kHalfBytes, &maps->m[my_k], bar(full0 + s), 64, my_start, kvh, 0);
         }
       }
     }
@@ -513,11 +515,13 @@ bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* r
   using namespace tc;
   using namespace tc::packed;
   Maps mk, mv;
+  const int kvd = a.kv_div < 1 ? 1 : a.kv_div;
   for (int k = 0; k < 4; ++k)
-    if (!make_map(&mk.m[k], a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k) ||
-        !make_map(&mv.m[k], a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k))
+    if (!make_map(&mk.m[k], a.K, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k) ||
+        !make_map(&mv.m[k], a.V, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k))
       return false;
   Params p{};
+  p.kv_div = kvd;
   p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.scale_log2 = a.scale * 1.4426950408889634f;
   p.rem_pos = rem_pos; p.rem_grp = rem_grp; p.rem_cnt = rem_cnt;
   p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;

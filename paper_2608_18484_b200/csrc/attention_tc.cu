@@ -68,6 +68,7 @@ static_assert(kNumBars <= 32, "barrier area");
 
 struct Params {
   int BH, H, N, Cq, Ck, sparse;
+  int kv_div;                      // query heads per K/V head: K/V tensors, their maps and kv_off are indexed by head / kv_div
   float scale_log2;
   const int *q_off, *kv_off, *route_ptr, *route_idx, *q_perm, *tile_off;
   __nv_bfloat16* O; i64 os[3];
@@ -111,7 +112,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   __syncthreads();
   if (prm.sparse) {
     const int* toff = prm.tile_off + (i64)bh * (prm.Cq + 1);
-    const int* kvo = prm.kv_off + (i64)bh * (prm.Ck + 1);
+    const int* kvo = prm.kv_off + (i64)(bh / prm.kv_div) * (prm.Ck + 1);
     for (int g = tid; g < prm.Cq; g += kThreads)
       if (toff[g] <= (int)blockIdx.x && (int)blockIdx.x < toff[g + 1]) { misc[4] = g; misc[5] = toff[g]; }
     for (int g = tid; g <= prm.Ck; g += kThreads) kv_stage[g] = kvo[g];
@@ -170,11 +171,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // the concatenated key ranges together (uniform); lane j issues the copies of box j.
     if (n_tiles > 0) {
       const bool is_k = warp == 8;
-      const int c2 = prm.sparse ? bh : h, c3 = prm.sparse ? 0 : b;
+      const int c3 = prm.sparse ? 0 : b;
+      const int c2 = (prm.sparse ? bh : h) / prm.kv_div;       // K/V head (group-major copies: [BH / kv_div]; originals: [B][H / kv_div])
       if (is_k && lane == 0) {
+        const int q2 = prm.sparse ? bh : h;
         mbar_expect_tx(bar(Q_FULL), kTileBytes);
-        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, c2, c3);
-        tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, c2, c3);
+        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, q2, c3);
+        tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, q2, c3);
       }
       const int nst = is_k ? kKStages : kVStages;
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
@@ -506,21 +509,22 @@ bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   Maps mk, mv;
   const bool sparse = a.route_ptr != nullptr;
   const int B = a.BH / a.H;
+  const int kvd = a.kv_div < 1 ? 1 : a.kv_div;
   bool ok;
   if (sparse) {
     ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile);
     for (int k = 0; k < 4 && ok; ++k)
-      ok = make_map(&mk.m[k], a.K, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k) &&
-           make_map(&mv.m[k], a.V, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kSub << k);
+      ok = make_map(&mk.m[k], a.K, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k) &&
+           make_map(&mv.m[k], a.V, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k);
   } else {
     ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile);
     for (int k = 0; k < 4 && ok; ++k)
-      ok = make_map(&mk.m[k], a.K, kD, a.N, a.H, B, a.ks[0], a.ks[1], a.ks[2], kSub << k) &&
-           make_map(&mv.m[k], a.V, kD, a.N, a.H, B, a.vs[0], a.vs[1], a.vs[2], kSub << k);
+      ok = make_map(&mk.m[k], a.K, kD, a.N, a.H / kvd, B, a.ks[0], a.ks[1], a.ks[2], kSub << k) &&
+           make_map(&mv.m[k], a.V, kD, a.N, a.H / kvd, B, a.vs[0], a.vs[1], a.vs[2], kSub << k);
   }
   if (!ok) return false;
   Params p{};
-  p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.sparse = sparse;
+  p.BH = a.BH; p.H = a.H; p.N = a.N; p.Cq = a.Cq; p.Ck = a.Ck; p.sparse = sparse; p.kv_div = kvd;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.q_off = a.q_off; p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx; p.q_perm = a.q_perm;
   p.tile_off = a.tile_off;

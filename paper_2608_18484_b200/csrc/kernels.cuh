@@ -45,8 +45,9 @@ void launch_gather_rows(int dtype, const void* X, const i64* xs, int BH, int H, 
 // project_tc.cu: the same projection on the tensor cores (bf16, d = 128, r <= 64); Ft: bf16 scratch [BH][3][64][128]
 cudaError_t init_project_tc();
 bool project_tc_supported(int dtype, int d, int r, const i64* xs);
+// f_div: heads that share one feature map (F is indexed by bh / f_div)
 bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r, const float* F, bool rms, float eps,
-                       float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st);
+                       float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st, int f_div = 1);
 
 // ---- kmeans_tc.cu (tcgen05 score contraction + exact recheck) --------------------------------------
 struct KmeansTcArgs {
@@ -70,13 +71,14 @@ struct RouteState {      // per head, device
   i64 pairs;             // routed pairs
   i64 cells;             // selected cells
 };
+// kv_div = query heads per K/V head: kappa and nk (K/V side) are indexed by bh / kv_div
 void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
-                        int d, float scale, float* score, cudaStream_t st);
+                        int d, float scale, float* score, int kv_div, cudaStream_t st);
 void launch_route_select(const float* score, const int* nq, const int* nk, int BH, int Cq, int Ck, i64 budget,
                          int select_all, int* route_ptr, int* route_idx, RouteState* state, i64* pairs_out,
-                         cudaStream_t st);
+                         int kv_div, cudaStream_t st);
 void launch_count_pairs(const int* q_off, const int* kv_off, const int* route_ptr, const int* route_idx, int BH, int Cq,
-                        int Ck, RouteState* state, cudaStream_t st);
+                        int Ck, RouteState* state, int kv_div, cudaStream_t st);
 cudaError_t init_routing();
 void launch_probe_select(const float* phiQ, int ldphi, int r, const int* q_perm, const int* q_off, const int* nq, int BH,
                          int N, int Cq, int M, double* dist_scratch, int* probe_idx, float* probe_w, cudaStream_t st);
@@ -91,6 +93,7 @@ struct AttnArgs {
   // sparse metadata (null for dense)
   const int *q_off, *kv_off, *route_ptr, *route_idx, *q_perm, *tile_off;
   int Cq, Ck;
+  int kv_div;                 // query heads per K/V head (grouped-query attention): K/V-side arrays are indexed by bh / kv_div; 0 = 1
   // epilogue
   const float *A, *c;         // [BH][d][d], [BH][d]; null = no correction
   void* O; i64 os[3];
@@ -125,6 +128,7 @@ bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, con
 
 struct ProbeArgs {
   int dtype, BH, H, N, d, M, Ck, Cq, n_split;
+  int kv_div;                          // query heads per K/V head; Kg, Vg, kv_off are indexed by bh / kv_div
   float scale;
   const void *Q; i64 qs[3];            // original layout (probe rows are gathered by index)
   const void *Kg, *Vg;                 // group-major [BH][N][d]

@@ -43,6 +43,7 @@ static_assert(kPbNumBars <= 32, "barrier area");
 
 struct PbParams {
   int BH, N, M, Ck, Cq, n_split;
+  int kv_div;                     // query heads per K/V head: the K/V maps and kv_off are indexed by bh / kv_div
   float scale_log2;
   const int *probe_idx, *q_assign, *kv_off, *route_ptr, *route_idx;
   float* partial;                 // [BH][n_split][M][2][130]
@@ -98,7 +99,8 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = (uint32_t)misc[0];
   volatile int* abort_flag = &misc[1];
-  const int* kvoff = prm.kv_off + (i64)bh * (prm.Ck + 1);
+  const int kvh = bh / prm.kv_div;
+  const int* kvoff = prm.kv_off + (i64)kvh * (prm.Ck + 1);
 
   // Tiles are cut so that none spans more than kPbMaxRuns K/V groups; every role walks the same
   // sequence of (start position, columns) with this function.  `g` = group that contains `pos`.
@@ -141,8 +143,8 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           mbar_arrive(bar(PMETA_FULL + (i & 7)));
         }
         mbar_expect_tx(bar(full0 + s), kPbTileBytes);
-        tma_load_4d(buf0 + s * kPbTileBytes, map, bar(full0 + s), 0, pos, bh, 0);
-        tma_load_4d(buf0 + s * kPbTileBytes + kPbHalf, map, bar(full0 + s), 64, pos, bh, 0);
+        tma_load_4d(buf0 + s * kPbTileBytes, map, bar(full0 + s), 0, pos, kvh, 0);
+        tma_load_4d(buf0 + s * kPbTileBytes + kPbHalf, map, bar(full0 + s), 64, pos, kvh, 0);
         pos += nc;
       }
     }
@@ -359,17 +361,19 @@ bool probe_tc_supported(const ProbeArgs& a) { return a.dtype == SPARSEPR_BF16 &&
 
 // Qp: scratch [BH][M][128] bf16.  Writes a.partial in the layout k_probe_merge reads.
 bool launch_probe_rows_tc(const ProbeArgs& a, __nv_bfloat16* Qp, int* err, cudaStream_t st) {
+  const int kvd = a.kv_div < 1 ? 1 : a.kv_div;
   using namespace tc;
   k_gather_probe_q<<<dim3((a.M * 16 + 255) / 256, a.BH), 256, 0, st>>>((const __nv_bfloat16*)a.Q, a.qs[0], a.qs[1], a.qs[2], a.H,
                                                                      a.probe_idx, a.M, Qp);
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, Qp, 128, a.M, a.BH, 1, 0, (i64)a.M * 128, 128, 128) ||
-      !make_map(&mk, a.Kg, 128, a.N, a.BH, 1, 0, (i64)a.N * 128, 128, 128) ||
-      !make_map(&mv, a.Vg, 128, a.N, a.BH, 1, 0, (i64)a.N * 128, 128, 128))
+      !make_map(&mk, a.Kg, 128, a.N, a.BH / kvd, 1, 0, (i64)a.N * 128, 128, 128) ||
+      !make_map(&mv, a.Vg, 128, a.N, a.BH / kvd, 1, 0, (i64)a.N * 128, 128, 128))
     return false;
   PbParams p{};
   p.BH = a.BH; p.N = a.N; p.M = a.M; p.Ck = a.Ck; p.Cq = a.Cq; p.n_split = a.n_split;
   p.scale_log2 = a.scale * 1.4426950408889634f;
+  p.kv_div = kvd;
   p.probe_idx = a.probe_idx; p.q_assign = a.q_assign; p.kv_off = a.kv_off; p.route_ptr = a.route_ptr; p.route_idx = a.route_idx;
   p.partial = a.partial; p.err = err;
   k_probe_rows_tc<<<dim3(a.n_split, (a.M + 127) / 128, a.BH), kPbThreads, PbSmem::total, st>>>(mq, mk, mv, p);

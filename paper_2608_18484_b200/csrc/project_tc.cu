@@ -165,11 +165,12 @@ k_project_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ C
 }
 
 // F [BH][128][r] float32 -> Ft [BH][3][64][128] bf16: term t, row j (output column, zero beyond r), column k
-__global__ void k_split_feature_map(const float* __restrict__ F, int r, __nv_bfloat16* __restrict__ Ft) {
+// (f_div heads share one feature map: the query heads of a K/V head under grouped-query attention)
+__global__ void k_split_feature_map(const float* __restrict__ F, int r, __nv_bfloat16* __restrict__ Ft, int f_div) {
   const int bh = blockIdx.y;
   for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < 64 * 128; e += gridDim.x * blockDim.x) {
     const int j = e / 128, k = e % 128;
-    float x = j < r ? F[((i64)bh * 128 + k) * r + j] : 0.f;
+    float x = j < r ? F[((i64)(bh / f_div) * 128 + k) * r + j] : 0.f;
     __nv_bfloat16* out = Ft + (i64)bh * 3 * 64 * 128 + e;
 #pragma unroll
     for (int t = 0; t < 3; ++t) {
@@ -191,10 +192,10 @@ bool project_tc_supported(int dtype, int d, int r, const i64* xs) {
 
 // Ft: bf16 scratch [BH][3][64][128]
 bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r, const float* F, bool rms, float eps,
-                       float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st) {
+                       float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st, int f_div) {
   using namespace tc;
   CUtensorMap mx, mf;
-  k_split_feature_map<<<dim3(8, BH), 256, 0, st>>>(F, r, Ft);
+  k_split_feature_map<<<dim3(8, BH), 256, 0, st>>>(F, r, Ft, f_div < 1 ? 1 : f_div);
   if (!make_map(&mx, X, 128, N, H, BH / H, xs[0], xs[1], xs[2], 128) ||
       !make_map(&mf, Ft, 128, 64, 3, BH, (i64)3 * 64 * 128, (i64)64 * 128, 128, 64))
     return false;

@@ -17,10 +17,11 @@ constexpr int kCsRows = 8;     // query groups per CTA
 
 __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ theta, const float* __restrict__ kappa,
                                                      const int* __restrict__ nq, const int* __restrict__ nk, int Cq,
-                                                     int Ck, int d, float scale, float* __restrict__ score) {
+                                                     int Ck, int d, float scale, float* __restrict__ score, int kv_div) {
   __shared__ float th[kCsRows][128];
   __shared__ float kt[32][257];                              // a [256 groups x 32 dims] slab of kappa, transposed
   const int bh = blockIdx.y, a0 = blockIdx.x * kCsRows;
+  const int kvh = bh / kv_div;                               // K/V head of this query head
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int e = tid; e < kCsRows * d; e += 256) {
     const int r = e / d, k = e % d;
@@ -36,7 +37,7 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
 #pragma unroll 8
       for (int r = 0; r < 32; ++r) {
         const int b = b0 + warp * 32 + r;
-        kt[lane][warp * 32 + r] = (b < Ck && k0 + lane < d) ? kappa[((i64)bh * Ck + b) * d + k0 + lane] : 0.f;
+        kt[lane][warp * 32 + r] = (b < Ck && k0 + lane < d) ? kappa[((i64)kvh * Ck + b) * d + k0 + lane] : 0.f;
       }
       __syncthreads();
 #pragma unroll
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
   const int a = a0 + warp;
   if (a >= Cq) return;
   float* out = score + ((i64)bh * Cq + a) * Ck;
-  const int* nkh = nk + (i64)bh * Ck;
+  const int* nkh = nk + (i64)kvh * Ck;
   if (nq[(i64)bh * Cq + a] == 0) {
     for (int b = lane; b < Ck; b += 32) out[b] = 0.f;
     return;
@@ -76,9 +77,9 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
 }
 
 void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
-                        int d, float scale, float* score, cudaStream_t st) {
+                        int d, float scale, float* score, int kv_div, cudaStream_t st) {
   dim3 grid((Cq + kCsRows - 1) / kCsRows, BH);
-  k_cell_scores<<<grid, 256, 0, st>>>(theta, kappa, nq, nk, Cq, Ck, d, scale, score);
+  k_cell_scores<<<grid, 256, 0, st>>>(theta, kappa, nq, nk, Cq, Ck, d, scale, score, kv_div < 1 ? 1 : kv_div);
 }
 
 // =============================================================================
@@ -108,7 +109,7 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
                                                        const int* __restrict__ nk, int Cq, int Ck, i64 budget,
                                                        int select_all, int* __restrict__ route_ptr,
                                                        int* __restrict__ route_idx, RouteState* __restrict__ state,
-                                                       i64* __restrict__ pairs_out) {
+                                                       i64* __restrict__ pairs_out, int kv_div) {
   extern __shared__ int sm_route[];
   int* forced = sm_route;            // [Cq]
   int* cnt = forced + Cq;            // [Cq]
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
   const int bh = blockIdx.x;
   const unsigned* u = reinterpret_cast<const unsigned*>(score) + (i64)bh * Cq * Ck;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  for (int b = threadIdx.x; b < Ck; b += blockDim.x) nks[b] = nk[(i64)bh * Ck + b];
+  for (int b = threadIdx.x; b < Ck; b += blockDim.x) nks[b] = nk[(i64)(bh / kv_div) * Ck + b];
   for (int a = threadIdx.x; a < Cq; a += blockDim.x) nqs[a] = nq[(i64)bh * Cq + a];
   __syncthreads();
 
@@ -384,11 +385,11 @@ static size_t route_smem(int Cq, int Ck) {      // forced, cnt, nqs [Cq], nks [C
 // routed pairs and cells of given routes (used when a plan is imported)
 __global__ void __launch_bounds__(256) k_count_pairs(const int* __restrict__ q_off, const int* __restrict__ kv_off,
                                                      const int* __restrict__ route_ptr, const int* __restrict__ route_idx,
-                                                     int Cq, int Ck, RouteState* __restrict__ state) {
+                                                     int Cq, int Ck, RouteState* __restrict__ state, int kv_div) {
   __shared__ i64 red[34];
   const int bh = blockIdx.x;
   const int* qo = q_off + (i64)bh * (Cq + 1);
-  const int* ko = kv_off + (i64)bh * (Ck + 1);
+  const int* ko = kv_off + (i64)(bh / kv_div) * (Ck + 1);
   const int* rp = route_ptr + (i64)bh * (Cq + 1);
   const int* ri = route_idx + (i64)bh * Cq * Ck;
   i64 pairs = 0;
@@ -401,14 +402,14 @@ __global__ void __launch_bounds__(256) k_count_pairs(const int* __restrict__ q_o
   if (threadIdx.x == 0) { state[bh].pairs = pairs; state[bh].cells = rp[Cq]; }
 }
 void launch_count_pairs(const int* q_off, const int* kv_off, const int* route_ptr, const int* route_idx, int BH, int Cq,
-                        int Ck, RouteState* state, cudaStream_t st) {
-  k_count_pairs<<<BH, 256, 0, st>>>(q_off, kv_off, route_ptr, route_idx, Cq, Ck, state);
+                        int Ck, RouteState* state, int kv_div, cudaStream_t st) {
+  k_count_pairs<<<BH, 256, 0, st>>>(q_off, kv_off, route_ptr, route_idx, Cq, Ck, state, kv_div < 1 ? 1 : kv_div);
 }
 void launch_route_select(const float* score, const int* nq, const int* nk, int BH, int Cq, int Ck, i64 budget,
                          int select_all, int* route_ptr, int* route_idx, RouteState* state, i64* pairs_out,
-                         cudaStream_t st) {
+                         int kv_div, cudaStream_t st) {
   k_route_select<<<BH, 1024, route_smem(Cq, Ck), st>>>(score, nq, nk, Cq, Ck, budget, select_all, route_ptr, route_idx,
-                                                        state, pairs_out);
+                                                        state, pairs_out, kv_div < 1 ? 1 : kv_div);
 }
 
 // =============================================================================

@@ -42,19 +42,23 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / np.linalg.norm(b))
 
 
-def plan_links(wl, i, Q, K, exp, feat, prm, warm=None):
+def plan_links(wl, i, Q, K, exp, feat, prm, warm=None, ref=None, kv=None):
     """Everything the assertions need for head i: GPU quantities beside the oracle's evaluation of each link.
-    `warm` = the partition {"a_K", "a_Q"} that a warm-started GPU plan was seeded with."""
+    `warm` = the partition {"a_K", "a_Q"} that a warm-started GPU plan was seeded with.  Under grouped-query
+    attention `kv` is the index of the head's K/V head (the K/V-side arrays have one entry per K/V head) and `ref`
+    the oracle's plan of this query head inside its group."""
     N, d = Q.shape
     C = -(-N // wl.block)
     out = {}
-    ref = orc.plan_head(Q, K, prm, i, warm=warm)
+    if ref is None:
+        ref = orc.plan_head(Q, K, prm, i, warm=warm)
+    kv = i if kv is None else kv
     variant = prm.get("partition", 0)
-    aK, aQ = exp["kv_assign"][i], exp["q_assign"][i]
+    aK, aQ = exp["kv_assign"][kv], exp["q_assign"][i]
     # a1-a3 (a semantic K/V partition clusters K itself: no feature map)
     out["FF_K"] = 0.0
     if variant != orc.PARTITION_SEMANTIC:
-        FK = feat["F_K"][i].astype(np.float64)
+        FK = feat["F_K"][kv].astype(np.float64)
         out["FF_K"] = rel_fro(FK @ FK.T, ref["F_K"] @ ref["F_K"].T)
     # a4
     out["agree_K"] = float((aK == ref["a_K"]).mean())
@@ -62,12 +66,12 @@ def plan_links(wl, i, Q, K, exp, feat, prm, warm=None):
         orc.kmeans_objective(ref["phi_K"], _means(ref["phi_K"], ref["a_K"], C), ref["a_K"]) - 1.0
     # a5: centroids and query metric of the GPU's own K/V groups
     kappa, n_k = orc.kv_centroids(K, aK, C)
-    out["kappa"] = float(np.abs(feat["kappa"][i] - kappa).max())
+    out["kappa"] = float(np.abs(feat["kappa"][kv] - kappa).max())
     phi_gpu = feat["phi_Q"][i].astype(np.float64)
     rows = np.random.default_rng(5).choice(N, min(N, 384), replace=False)
     if variant == orc.PARTITION_RESPONSE_COUPLED:
         F_Q, _ = orc.eig_feature_map(orc.query_response_metric(kappa, n_k), prm["rQ"])
-        FQ = feat["F_Q"][i].astype(np.float64)
+        FQ = feat["F_Q"][kv].astype(np.float64)
         out["FF_Q"] = rel_fro(FQ @ FQ.T, F_Q @ F_Q.T)
         # a6
         phi_ref = orc.query_response(Q, F_Q, prm["eps_rms"])
