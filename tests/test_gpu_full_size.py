@@ -112,3 +112,28 @@ def test_more_than_256_groups_sampled_rows(wl):
     got, got_sp = to_np(O[0, 0])[rows], to_np(Osp[0, 0])[rows]
     assert_bf16_close(got_sp, O_sp)
     assert_bf16_close(got, O_hat)
+
+
+def test_reconstruction_error_matches_the_oracle_at_scale():
+    """The whole call of the oracle and of the GPU on the same bytes at a non-toy size (head 0 of the 480p-like
+    workload, 16 of 21 frames, N = 24960, 195 groups per side): the two plans are built independently (float64 vs
+    float32, so single near-tie decisions may differ), and what has to agree is the reconstruction error against
+    float64 exact attention, with and without the probe repair, and the realised density."""
+    wl = W.VIDEO_480P.scaled(grid=(16, 30, 52), H=1)
+    host, (Qd, Kd, Vd) = heads_to_device(wl, [0])
+    Q, K, V = host[0]
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale)
+    plan = B.sparsepr_plan(Qd, Kd, Vd, **kw)
+    O, Osp = B.sparsepr_attend(plan, Qd, Kd, Vd, return_sparse=True)
+    st = B.sparsepr_plan_stats(plan)
+    assert st["device_error"] == 0
+    prm = orc.default_params(**kw)
+    O_ref, O_ref_sp, ref, _ = orc.sparsepr_head(Q, K, V, prm, 0)
+    exact = orc.dense_attention(Q, K, V, wl.softmax_scale)
+    e_gpu, e_orc = orc.rel_l2(to_np(O[0, 0]), exact), orc.rel_l2(O_ref, exact)
+    h_gpu, h_orc = orc.rel_l2(to_np(Osp[0, 0]), exact), orc.rel_l2(O_ref_sp, exact)
+    # bf16 output rounding alone is 1.7e-3 relative; the errors themselves are about 0.1
+    assert abs(e_gpu - e_orc) <= 2e-3 and abs(h_gpu - h_orc) <= 2e-3, (e_gpu, e_orc, h_gpu, h_orc)
+    assert abs(st["rho_route"] - ref["rho_route"]) <= 1e-3
+    assert (B.sparsepr_plan_export(plan)["kv_assign"][0] == ref["a_K"]).mean() >= 0.97
