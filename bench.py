@@ -50,12 +50,16 @@ def load_peaks():
 # --------------------------------------------------------------------------------------
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons during the timed region."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
         self.rows, self.proc, self.index = [], None, index
+        self.window = [None, None]           # wall-clock bounds of the timed region; samples outside are dropped
+
+    def mark(self, which):
+        self.window[which] = time.time()
 
     def start(self):
         try:
@@ -79,14 +83,18 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        import datetime
         sm, mx, reasons = [], None, set()
         for r in self.rows:
             try:
-                sm.append(float(r[0]))
-                mx = float(r[1])
+                ts = datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if self.window[0] is not None and (ts < self.window[0] - 0.05 or ts > (self.window[1] or ts) + 0.05):
+                    continue
+                sm.append(float(r[1]))
+                mx = float(r[2])
             except Exception:
                 continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
@@ -357,12 +365,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()                      # started ahead of the warm-up: nvidia-smi takes a moment to deliver samples
     for _ in range(args.warmup):
         plan = step()
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark(0)
     # ---- timed region: exactly K steps, CUDA events on the launching stream ----
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
@@ -393,6 +402,7 @@ def main():
     for _ in range(dense_steps):
         B.sparsepr_dense(Qd, Kd, Vd, wl.softmax_scale, out=Odense, profile=dprof)
     torch.cuda.synchronize()
+    sampler.mark(1)
     clocks = sampler.stop() if rank == 0 else None
     stages = {k: v / args.steps for k, v in prof.as_dict().items() if k != "dense"}
     dense_ms = dprof.as_dict()["dense"] / dense_steps
