@@ -66,6 +66,40 @@ def test_grouped_query_call_matches_the_oracle():
         assert_bf16_close(to_np(Od[0, i]), orc.dense_attention(Qs[i], Ks[i // G], Vs[i // G], wl.softmax_scale))
 
 
+def test_grouped_query_warm_start():
+    """A second call over the same scene, seeded with the first call's partitions (one K/V partition per K/V head,
+    one query partition per query head), against the oracle's warm-started grouped plan."""
+    wl = W.VIDEO_480P.scaled(grid=(3, 30, 52), H=G * HKV, n_probe=64)
+    _, _, _, (Q1, K1, V1) = grouped_inputs(wl)
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe,
+              softmax_scale=wl.softmax_scale)
+    first = B.sparsepr_plan(Q1, K1, V1, **kw)
+    e1 = B.sparsepr_plan_export(first)
+    # fresh noise around the same tables: noise draws G, G + 1, ... for the queries, draw G for keys and values
+    Qs, Ks, Vs = [], [], []
+    for kv in range(HKV):
+        _, K, V = W.make_head(wl, kv, step=G)
+        Ks.append(K)
+        Vs.append(V)
+        Qs += [W.make_head(wl, kv, step=G + g)[0] for g in range(G)]
+    Q2, K2, V2 = [torch.from_numpy(np.stack(x)[None]).to(torch.bfloat16).cuda().contiguous() for x in (Qs, Ks, Vs)]
+    kw3 = dict(kw, kmeans_iters=3)
+    second = B.sparsepr_plan(Q2, K2, V2, warm_from=first, **kw3)
+    assert B.sparsepr_plan_stats(second)["device_error"] == 0
+    exp, feat = B.sparsepr_plan_export(second), B.sparsepr_plan_export_features(second)
+    prm = orc.default_params(**kw3)
+    links = []
+    for kv in range(HKV):
+        warm = dict(a_K=e1["kv_assign"][kv], a_Q=[e1["q_assign"][kv * G + g] for g in range(G)])
+        refs = orc.plan_group(Qs[kv * G:(kv + 1) * G], Ks[kv], prm, kv, kv * G, warm=warm)
+        for g in range(G):
+            i = kv * G + g
+            links.append(plan_links(wl, i, Qs[i], Ks[kv], exp, feat, prm, ref=refs[g], kv=kv,
+                                    warm=dict(a_K=warm["a_K"], a_Q=warm["a_Q"][g])))
+    check_links(wl, links)
+    assert torch.isfinite(B.sparsepr_attend(second, Q2, K2, V2)).all()
+
+
 def test_grouped_query_needs_the_tensor_core_path():
     Q = torch.randn(1, 4, 256, 64, device="cuda")
     K = torch.randn(1, 2, 256, 64, device="cuda")
