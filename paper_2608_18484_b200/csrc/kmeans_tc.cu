@@ -407,7 +407,23 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   KmParams p{};
   p.N = a.N; p.C = a.C; p.r = a.r; p.R = a.R; p.n_chunks = (a.C + kKmChunk - 1) / kKmChunk;
   const int row_tiles = (a.N + 127) / 128;
-  p.ctas_per_head = std::max(1, std::min(row_tiles, sm_count() / a.BH));
+  // CTAs per head: one CTA fills an SM and works through its row tiles one after the other, so the launch takes
+  // (rounds of CTAs over the SMs) x (tiles per CTA, plus about three tiles' worth of set-up).  With heads x CTAs below
+  // the SM count a single round can leave many SMs idle (40 heads x 3 CTAs on 148 SMs); several rounds of shorter
+  // CTAs are then faster, as long as a chunk keeps 24 tiles or more so that the set-up remains small.
+  {
+    const int sms = sm_count();
+    int best_k = 1;
+    long best_cost = -1;
+    for (int k = 1; k <= row_tiles; ++k) {
+      const int per = (row_tiles + k - 1) / k;
+      if ((long)k * a.BH > sms && per < 24) break;          // several rounds only with chunks of 24 tiles or more
+      const long rounds = ((long)k * a.BH + sms - 1) / sms;
+      const long cost = rounds * (per + 3);
+      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_k = k; }
+    }
+    p.ctas_per_head = best_k;
+  }
   p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.assign = a.assign;
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
   p.prev_changed = a.prev_changed; p.cur_changed = a.cur_changed;
