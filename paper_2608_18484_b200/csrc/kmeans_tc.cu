@@ -106,9 +106,10 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       // tile back to back both groups would share both buffers, and a group waiting for a phase that lies two ahead
       // of the barrier's current one takes the parity test for passed.)  v counts the steps that exist.
       int v = 0;
+      int pair = 0, r2 = 0;                                    // sidx = pair * 2 n_chunks + r2
       for (int sidx = 0; sidx < n_pairs * 2 * n_chunks; ++sidx) {
-        const int r2 = sidx % (2 * n_chunks);
-        const int tl = 2 * (sidx / (2 * n_chunks)) + (r2 & 1), ch = r2 >> 1;
+        const int tl = 2 * pair + (r2 & 1), ch = r2 >> 1;
+        if (++r2 == 2 * n_chunks) { r2 = 0; ++pair; }
         if (tl >= my_tiles) continue;
         if (n_chunks > 1 || v == 0) {
           const int ms = n_chunks > 1 ? (v & 1) : 0;
@@ -131,12 +132,18 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   } else if (warp == 5) {
     // =========================== MMA issuer ================================================
     if (lane == 0) {
+      // The issuing thread shares its warp scheduler with epilogue warps that leave it few issue slots, and the next
+      // product of a score buffer can only be issued once the epilogue has released it: every instruction of this
+      // loop is on the critical path.  Descriptors are therefore built once (only their 16-byte address field moves),
+      // the step order is tracked with counters instead of divisions, and the k-steps are unrolled.
       const uint32_t idesc = idesc_bf16(0, kKmChunk);
       const int ksteps = prm.R / 16;
+      const uint64_t x_desc0 = smem_desc(base + KmSmem::x, 16), m_desc0 = smem_desc(base + KmSmem::mu, 16);
       int v = 0;                                               // same step order as the producer
+      int pair = 0, r2 = 0;                                    // sidx = pair * 2 n_chunks + r2
       for (int sidx = 0; sidx < n_pairs * 2 * n_chunks; ++sidx) {
-        const int r2 = sidx % (2 * n_chunks);
-        const int tl = 2 * (sidx / (2 * n_chunks)) + (r2 & 1), ch = r2 >> 1;
+        const int tl = 2 * pair + (r2 & 1), ch = r2 >> 1;
+        if (++r2 == 2 * n_chunks) { r2 = 0; ++pair; }
         if (tl >= my_tiles) continue;
         const int xs = tl & 1, ms = n_chunks > 1 ? (v & 1) : 0;
         const int ab = tl & 1, au = (tl >> 1) * n_chunks + ch;   // score buffer and how often it has been used before
@@ -145,12 +152,15 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         if (!mbar_wait(bar(ACC_EMPTY + ab), (au & 1) ^ 1, abort_flag)) break;
         tc_fence_after();
         const uint32_t d = tmem + (uint32_t)ab * 256u;
-        const uint32_t xh = base + KmSmem::x + xs * 2 * kXBytes, xl = xh + kXBytes;
-        const uint32_t mh = base + KmSmem::mu + ms * 2 * kMuBytes, ml = mh + kMuBytes;
-        uint32_t acc = 0;
-        for (int kk = 0; kk < ksteps; ++kk) { umma_bf16(d, smem_desc(xh + kk * 32, 16), smem_desc(mh + kk * 32, 16), idesc, acc); acc = 1; }
-        for (int kk = 0; kk < ksteps; ++kk) umma_bf16(d, smem_desc(xh + kk * 32, 16), smem_desc(ml + kk * 32, 16), idesc, 1);
-        for (int kk = 0; kk < ksteps; ++kk) umma_bf16(d, smem_desc(xl + kk * 32, 16), smem_desc(mh + kk * 32, 16), idesc, 1);
+        const uint64_t xh = x_desc0 + (uint64_t)((xs * 2 * kXBytes) >> 4), xl = xh + (uint64_t)(kXBytes >> 4);
+        const uint64_t mh = m_desc0 + (uint64_t)((ms * 2 * kMuBytes) >> 4), ml = mh + (uint64_t)(kMuBytes >> 4);
+        // x_h mu_h + x_h mu_l + x_l mu_h; one k-step = 16 columns = 32 bytes = 2 address units
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) if (kk < ksteps) umma_bf16(d, xh + 2 * kk, mh + 2 * kk, idesc, kk > 0);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) if (kk < ksteps) umma_bf16(d, xh + 2 * kk, ml + 2 * kk, idesc, 1);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) if (kk < ksteps) umma_bf16(d, xl + 2 * kk, mh + 2 * kk, idesc, 1);
         if (ch == n_chunks - 1) umma_commit(bar(X_EMPTY + xs));
         if (n_chunks > 1) umma_commit(bar(MU_EMPTY + ms));
         umma_commit(bar(ACC_FULL + ab));
