@@ -183,6 +183,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
       // issued before the score wait so that the loads overlap it
       float pv0[32], pv1[32];
       const float xn = row < prm.N ? prm.xnorm[(i64)bh * prm.N + row] : 0.f;   // needed after the scores: fetched now
+      // the row's group of the previous pass, for the count of rows that move (same reason: its latency is hidden here)
+      const int old_a = (prm.prev_changed != nullptr && row < prm.N) ? prm.assign[(i64)bh * prm.N + row] : -1;
       if (prm.sums) {
         const int rowbase = (tile0 + tl) * 128 + wq * 32;
         // this lane's columns are (2 lane, 2 lane + 1): one 8-byte load per row (ldphi is a multiple of 16, and
@@ -243,9 +245,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
         const float E = 2.5e-4f * xn * mm + 1.0e-6f * (mm * mm + xn * mm);
         decided = second - best > 2.f * E;
         if (decided) {
-          int* ap = prm.assign + (i64)bh * prm.N + row;
-          moved = prm.prev_changed == nullptr || *ap != bi;
-          *ap = bi;
+          moved = old_a != bi;
+          prm.assign[(i64)bh * prm.N + row] = bi;
         } else {                                             // the recheck writes (and compares) this row's assignment
           const int pos = atomicAdd(prm.flag_count, 1);
           prm.flagged[pos] = bh * prm.N + row;
