@@ -268,13 +268,15 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           const int cl = __shfl_sync(FULL, bi, leader);
           const unsigned members = __ballot_sync(FULL, decided && bi == cl) & todo;
           todo &= ~members;
-          // float32 partial sums in ascending row order (a fixed order, hence reproducible), one
+          // float32 partial sums in a fixed order (hence reproducible), one
           // conversion to fixed point per (cluster, column)
-          float2 a2 = make_float2(0.f, 0.f);
+          // (four interleaved partial sums: one chain of 32 dependent additions would set the pace of this loop)
+          float2 a2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
           for (int rr = 0; rr < 32; ++rr)
-            if ((members >> rr) & 1u) a2 = __fadd2_rn(a2, make_float2(pv0[rr], pv1[rr]));   // one packed add per member row
-          const float a0 = a2.x, a1 = a2.y;
+            if ((members >> rr) & 1u) a2[rr & 3] = __fadd2_rn(a2[rr & 3], make_float2(pv0[rr], pv1[rr]));   // one packed add per member row
+          const float2 a01 = __fadd2_rn(__fadd2_rn(a2[0], a2[1]), __fadd2_rn(a2[2], a2[3]));
+          const float a0 = a01.x, a1 = a01.y;
           const i64 acc0 = __float2ll_rn(a0 * scl), acc1 = __float2ll_rn(a1 * scl);
           i64* s = prm.sums + ((i64)bh * prm.C + cl) * prm.R;
           if (2 * lane < prm.r) atomicAdd(reinterpret_cast<u64*>(s + 2 * lane), (u64)acc0);
