@@ -253,7 +253,7 @@ struct sparsepr_plan_s {
   int *route_ptr, *route_idx, *tile_off, *tile_off128;
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
-  __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged;
+  __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged; int* flagcnt;
   int *rem_pos, *rem_grp, *rem_cnt;      // rows of the short group remainders (packed attention tiles)
   int* km_changed;                       // [2 sides][T + 1][BH] rows that changed group in each k-means pass
   double* Mpool;                         // [BHkv][d][d] key-response metric pooled over the query heads of a K/V head (grouped-query attention only)
@@ -296,9 +296,10 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
   int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
   int* km_changed = c.take<int>(2 * (size_t)(r.T + 1) * BH);
+  int* flagcnt = c.take<int>(BH);
   double* Mpool = c.take<double>(r.G > 1 ? (size_t)r.BHkv * d * d : 0);
   if (p) {
-    p->km_changed = km_changed; p->Mpool = Mpool; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
+    p->km_changed = km_changed; p->flagcnt = flagcnt; p->Mpool = Mpool; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -377,7 +378,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
       ka.BH = nheads; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
       ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2;
       ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
-      ka.flagged = p->flagged; ka.flag_count = p->recheck + 1; ka.recheck_total = p->recheck; ka.err = p->err;
+      ka.flagged = p->flagged; ka.flag_count = p->flagcnt; ka.recheck_total = p->recheck; ka.err = p->err;
       ka.prev_changed = prev; ka.cur_changed = cur;
       launch_kmeans_assign_tc(ka, st);
     } else {

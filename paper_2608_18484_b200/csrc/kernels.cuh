@@ -57,7 +57,7 @@ struct KmeansTcArgs {
   const float *xnorm, *mu, *mu2;               // [BH][N], [BH][C][R], [BH][C]
   int* assign;
   i64* sums; int* counts; const int* fx_shift; // null sums = assignment only
-  int *flagged, *flag_count, *recheck_total, *err;
+  int *flagged, *flag_count, *recheck_total, *err;   // flagged [BH][N] scratch, flag_count [BH] scratch, recheck_total: rows rechecked by this pass
   const int* prev_changed; int* cur_changed;   // [BH] or null, as for launch_kmeans_assign
 };
 cudaError_t init_kmeans_tc();

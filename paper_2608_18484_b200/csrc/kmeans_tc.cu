@@ -41,7 +41,7 @@ struct KmParams {
   const float* mu2;                     // [BH][C]
   int* assign;
   i64* sums; int* counts; const int* fx_shift;
-  int* flagged; int* flag_count;        // rows left to the exact recheck
+  int* flagged; int* flag_count;        // rows left to the exact recheck: [BH][N] row indices, [BH] their number
   int* err;
   const int* prev_changed; int* cur_changed;   // [BH] or null: rows whose assignment changed in the previous / this pass
 };
@@ -248,8 +248,8 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
           moved = old_a != bi;
           prm.assign[(i64)bh * prm.N + row] = bi;
         } else {                                             // the recheck writes (and compares) this row's assignment
-          const int pos = atomicAdd(prm.flag_count, 1);
-          prm.flagged[pos] = bh * prm.N + row;
+          const int pos = atomicAdd(prm.flag_count + bh, 1);
+          prm.flagged[(i64)bh * prm.N + pos] = row;
         }
       }
       if (prm.cur_changed != nullptr) {
@@ -299,9 +299,140 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   }
 }
 
-// Exact decision for the rows the fast path could not prove: one CTA per row, one thread per
-// centroid, squared distance in float64 with the terms added in order of k (the definition;
-// the zero padding of columns r..R-1 adds exact zeros), ties to the lowest id.
+// Exact decision for the rows the fast path could not prove (a few thousand per pass at N = 32760 and 24 heads).
+// The definition is the squared distance in float64 with the terms added in order of k (the zero padding of columns
+// r..R-1 adds exact zeros), ties to the lowest id.  Every such row needs all C centroids of its head, so the rows of a
+// head share them: grid (G, BH); a CTA brings the head's centroids to shared memory once and its eight warps take the
+// head's flagged rows in turn.  Per row:
+//   1. float32 distances to all centroids (lane = centroid, 8 at a time; rows of mu padded by 4 floats, so that the
+//      16-byte reads of consecutive centroids fall into different banks).  Every term is non-negative, hence the
+//      float32 value is within (R + 3) 2^-24 of the true distance, relatively;
+//   2. only centroids within 4 (R + 4) 2^-24 of the float32 minimum (relative, plus a denormal's worth) can hold the
+//      float64 minimum: those few (normally one or two) are evaluated by the definition, one lane each.
+__global__ void __launch_bounds__(256) k_assign_recheck_staged(const int* __restrict__ flagged, const int* __restrict__ flag_count,
+                                                               const float* __restrict__ phi, int ldphi, int N, int r, int R,
+                                                               const float* __restrict__ mu, int C, int* __restrict__ assign,
+                                                               i64* __restrict__ sums, int* __restrict__ counts,
+                                                               const int* __restrict__ fx_shift, int* __restrict__ recheck_total,
+                                                               int first_pass, int* __restrict__ cur_changed) {
+  extern __shared__ __align__(16) float rs_smem[];
+  const unsigned FULL = 0xffffffffu;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int bh = blockIdx.y;
+  const int n = flag_count[bh];
+  if (blockIdx.x == 0 && bh == 0 && tid == 0 && recheck_total) {
+    int total = 0;
+    for (int h = 0; h < (int)gridDim.y; ++h) total += flag_count[h];
+    *recheck_total = total;
+  }
+  if ((int)blockIdx.x * 8 >= n) return;                        // no row for this CTA
+  const int LDM = R + 4, Cp = (C + 31) & ~31;
+  float* mu_s = rs_smem;                                       // [C][R + 4]
+  float* d32_all = mu_s + (size_t)C * LDM;                     // [8 warps][Cp]
+  float* xs_all = d32_all + 8 * Cp;                            // [8 warps][R]
+  {
+    const float4* src = reinterpret_cast<const float4*>(mu + (i64)bh * C * R);
+    const int q = R / 4;
+    for (int e = tid; e < C * q; e += 256) {
+      const int c = e / q, k4 = e - c * q;
+      *reinterpret_cast<float4*>(mu_s + (size_t)c * LDM + 4 * k4) = src[e];
+    }
+  }
+  __syncthreads();
+  float* d32 = d32_all + warp * Cp;
+  float* xs = xs_all + warp * R;
+  for (int i = blockIdx.x * 8 + warp; i < n; i += gridDim.x * 8) {
+    const int row = flagged[(i64)bh * N + i];
+    const i64 gr = (i64)bh * N + row;
+    const float* x = phi + gr * ldphi;
+    __syncwarp();
+    for (int k = lane; k < R; k += 32) xs[k] = x[k];
+    __syncwarp();
+    float best32 = INFINITY;
+    for (int c0 = 0; c0 < C; c0 += 256) {
+      // packed float32 arithmetic, two columns per instruction: (m - x)^2 summed in two partial sums per centroid
+      float2 acc[8];
+      const float* mrow[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { acc[j] = make_float2(0.f, 0.f); mrow[j] = mu_s + (size_t)min(c0 + 32 * j + lane, C - 1) * LDM; }
+#pragma unroll 2
+      for (int k = 0; k < R; k += 4) {
+        const float4 xv = *reinterpret_cast<const float4*>(xs + k);
+        const float2 nx0 = make_float2(-xv.x, -xv.y), nx1 = make_float2(-xv.z, -xv.w);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float4 mv = *reinterpret_cast<const float4*>(mrow[j] + k);
+          const float2 d0 = __fadd2_rn(make_float2(mv.x, mv.y), nx0), d1 = __fadd2_rn(make_float2(mv.z, mv.w), nx1);
+          acc[j] = __ffma2_rn(d0, d0, acc[j]);
+          acc[j] = __ffma2_rn(d1, d1, acc[j]);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int c = c0 + 32 * j + lane;
+        if (c < Cp) {
+          const float d = c < C ? acc[j].x + acc[j].y : INFINITY;
+          d32[c] = d;
+          best32 = fminf(best32, d);
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best32 = fminf(best32, __shfl_xor_sync(FULL, best32, o));
+    const float thr = best32 * (1.f + 4.f * (float)(R + 4) * 5.9604645e-8f) + 1e-30f;
+    // candidates: normally one, and then the decision is made (float64 arithmetic is slow on this GPU: about 16
+    // cycles per warp instruction, 5 instructions per term)
+    int ncand = 0, cand = -1;
+    for (int c = lane; c < C; c += 32)                         // (never past C: with a NaN row thr is +inf, and so are the pad entries)
+      if (d32[c] <= thr) { ++ncand; cand = c; }
+    const int total_cand = __reduce_add_sync(FULL, ncand);
+    int bi;
+    if (total_cand == 1) {
+      bi = __reduce_max_sync(FULL, cand);
+    } else if (total_cand == 0) {
+      bi = 0;                                                  // every distance is NaN (non-finite input, reported elsewhere): group 0
+    } else {
+      double best = 0.0;
+      bi = -1;
+      for (int c = lane; c < C; c += 32) {
+        if (d32[c] <= thr) {
+          const float* m = mu_s + (size_t)c * LDM;
+          double dsum = 0.0;
+#pragma unroll 8
+          for (int k = 0; k < R; ++k) {
+            const double diff = __dsub_rn((double)xs[k], (double)m[k]);
+            dsum = __dadd_rn(dsum, __dmul_rn(diff, diff));
+          }
+          if (bi < 0 || dsum < best) { best = dsum; bi = c; }    // a lane meets its centroids in increasing order
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const double ob = __shfl_xor_sync(FULL, best, o);
+        const int oi = __shfl_xor_sync(FULL, bi, o);
+        if (oi >= 0 && (bi < 0 || ob < best || (ob == best && oi < bi))) { best = ob; bi = oi; }
+      }
+    }
+    bi = min(max(bi, 0), C - 1);
+    if (lane == 0) {
+      if (cur_changed != nullptr && (first_pass || assign[gr] != bi)) atomicAdd(cur_changed + bh, 1);
+      assign[gr] = bi;
+    }
+    if (sums) {
+      // 2^shift as a float: scaling a float32 value by a power of two is exact, so the conversion gives the same
+      // integer as the float64 product
+      const float scl = __int_as_float((127 + fx_shift[bh]) << 23);
+      i64* sp = sums + ((i64)bh * C + bi) * R;
+      for (int t = lane; t < r; t += 32) atomicAdd(reinterpret_cast<u64*>(sp + t), (u64)__float2ll_rn(xs[t] * scl));
+      if (lane == 0) atomicAdd(counts + (i64)bh * C + bi, 1);
+    }
+  }
+}
+// shared memory of the kernel above
+static size_t recheck_staged_smem(int C, int R) { return ((size_t)C * (R + 4) + 8 * (size_t)((C + 31) & ~31) + 8 * (size_t)R) * sizeof(float); }
+
+// The same decision without staging, for centroid tables that do not fit into shared memory: grid (X, BH), one CTA per
+// row, one thread per centroid, float64 throughout.
 __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ flagged, const int* __restrict__ flag_count,
                                                         const float* __restrict__ phi, int ldphi, int N, int r, int R,
                                                         const float* __restrict__ mu, int C, int* __restrict__ assign,
@@ -312,11 +443,16 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
   __shared__ int s_bi[8];
   const unsigned FULL = 0xffffffffu;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n = *flag_count;
+  const int bh = blockIdx.y;
+  const int n = flag_count[bh];
+  if (blockIdx.x == 0 && bh == 0 && tid == 0 && recheck_total) {
+    int total = 0;
+    for (int h = 0; h < (int)gridDim.y; ++h) total += flag_count[h];
+    *recheck_total = total;
+  }
   for (int i = blockIdx.x; i < n; i += gridDim.x) {
-    const int gr = flagged[i];
-    const int bh = gr / N;
-    const float4* x4 = reinterpret_cast<const float4*>(phi + (i64)gr * ldphi);
+    const i64 gr = (i64)bh * N + flagged[(i64)bh * N + i];
+    const float4* x4 = reinterpret_cast<const float4*>(phi + gr * ldphi);
     const float* muh = mu + (i64)bh * C * R;
     double best = 0.0;
     int bi = -1;
@@ -359,7 +495,7 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
       assign[gr] = bi;
     }
     if (sums) {
-      const float* x = phi + (i64)gr * ldphi;
+      const float* x = phi + gr * ldphi;
       const double scl = ldexp(1.0, fx_shift[bh]);
       i64* sp = sums + ((i64)bh * C + bi) * R;
       if (tid < r) atomicAdd(reinterpret_cast<u64*>(sp + tid), (u64)__double2ll_rn((double)x[tid] * scl));
@@ -367,7 +503,6 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
     }
     __syncthreads();
   }
-  if (blockIdx.x == 0 && tid == 0 && recheck_total) *recheck_total = n;
 }
 
 // phi fp32 [rows][ld] -> hi/lo bf16 [rows][64] (zero padded) and the row norms
@@ -400,7 +535,10 @@ __global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ x,
 
 }  // namespace tc
 
+constexpr size_t kRecheckSmemMax = 200 * 1024;
 cudaError_t init_kmeans_tc() {
+  const cudaError_t e = cudaFuncSetAttribute(tc::k_assign_recheck_staged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRecheckSmemMax);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(tc::k_kmeans_assign_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kKmSmemBytes);
 }
 bool kmeans_tc_supported() { return tc::tma_available(); }
@@ -440,10 +578,18 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.assign = a.assign;
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
   p.prev_changed = a.prev_changed; p.cur_changed = a.cur_changed;
-  cudaMemsetAsync(a.flag_count, 0, sizeof(int), st);
+  cudaMemsetAsync(a.flag_count, 0, sizeof(int) * a.BH, st);
   k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
-  k_assign_recheck<<<sm_count() * 4, 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign, a.sums,
-                                                   a.counts, a.fx_shift, a.recheck_total, a.prev_changed == nullptr, a.cur_changed);
+  const size_t rs = recheck_staged_smem(a.C, a.R);
+  const int per_head = std::max(1, 2 * sm_count() / a.BH);
+  if (rs <= kRecheckSmemMax)
+    k_assign_recheck_staged<<<dim3(per_head, a.BH), 256, rs, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign,
+                                                                   a.sums, a.counts, a.fx_shift, a.recheck_total, a.prev_changed == nullptr,
+                                                                   a.cur_changed);
+  else
+    k_assign_recheck<<<dim3(std::max(1, 4 * sm_count() / a.BH), a.BH), 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C,
+                                                                                     a.assign, a.sums, a.counts, a.fx_shift, a.recheck_total,
+                                                                                     a.prev_changed == nullptr, a.cur_changed);
   return true;
 }
 
