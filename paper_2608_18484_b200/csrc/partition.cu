@@ -574,8 +574,8 @@ cudaError_t init_group_sort() {
 
 // =============================================================================
 // Group means in the original activation space: kappa_b (Appendix B.2) and
-// theta_a (router).  One warp per group walks its members in group-major order,
-// so the float32 sums have a fixed order.
+// theta_a (router).  One CTA per group walks its members in group-major order, eight warps on
+// interleaved blocks of rows; the float32 sums have a fixed order.
 // =============================================================================
 template <typename T, int D>
 __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H,
@@ -583,17 +583,19 @@ __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i6
                                                      int C, float* __restrict__ out, int* __restrict__ sizes) {
   constexpr int LPR = D / 8;                 // lanes per row (8 elements each)
   constexpr int RPW = 32 / LPR;              // rows per warp step
+  __shared__ float part[8][D];
   const int bh = blockIdx.y, b = bh / H, h = bh % H;
-  const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (g >= C) return;
+  const int g = blockIdx.x, w = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31, sub = lane / LPR, col = (lane % LPR) * 8;
   const T* base = X + b * sb + h * sh;
   const int* pm = perm + (i64)bh * N;
   const int p0 = off[(i64)bh * (C + 1) + g], p1 = off[(i64)bh * (C + 1) + g + 1];
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  // eight row loads in flight per lane (the walk is bound by the latency of the index -> row chain); the additions
-  // keep their order, and a slot beyond the group adds exact zeros
-  for (int p = p0 + sub; p < p1; p += RPW * 8) {
+  // One CTA per group (group sizes spread over two orders of magnitude: with a warp per group the largest group set
+  // the duration of the launch): warp w takes the blocks of 8 RPW rows number w, w + 8, ...; eight row loads in
+  // flight per lane (the walk is bound by the latency of the index -> row chain); every sum has a fixed order, and
+  // a slot beyond the group adds exact zeros
+  for (int p = p0 + w * RPW * 8 + sub; p < p1; p += RPW * 8 * 8) {
     int src[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) src[j] = p + j * RPW < p1 ? pm[p + j * RPW] : -1;
@@ -612,23 +614,28 @@ __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i6
 #pragma unroll
       for (int k = 0; k < 8; ++k) acc[k] += v[j][k];
   }
-  // combine the RPW interleaved partial sums in a fixed order
+  // combine the RPW interleaved partial sums of the warp, then the eight warps, in a fixed order
 #pragma unroll
   for (int k = 0; k < 8; ++k)
     for (int o = LPR; o < 32; o <<= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], o);
-  const int n = p1 - p0;
   if (sub == 0) {
-    const float invn = n > 0 ? 1.f / (float)n : 0.f;
-    float* o = out + ((i64)bh * C + g) * D + col;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) o[k] = acc[k] * invn;
+    for (int k = 0; k < 8; ++k) part[w][col + k] = acc[k];
   }
-  if (lane == 0 && sizes) sizes[(i64)bh * C + g] = n;
+  __syncthreads();
+  const int n = p1 - p0;
+  if (threadIdx.x < D) {
+    float t = part[0][threadIdx.x];
+#pragma unroll
+    for (int ww = 1; ww < 8; ++ww) t += part[ww][threadIdx.x];
+    out[((i64)bh * C + g) * D + threadIdx.x] = n > 0 ? t * (1.f / (float)n) : 0.f;
+  }
+  if (threadIdx.x == 0 && sizes) sizes[(i64)bh * C + g] = n;
 }
 
 void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, const int* off, int N,
                         int C, int d, float* out, int* sizes, cudaStream_t st) {
-  dim3 grid((C + 7) / 8, BH);
+  dim3 grid(C, BH);
 #define SPR_GM(TT, DD) k_group_means<TT, DD><<<grid, 256, 0, st>>>((const TT*)X, xs[0], xs[1], xs[2], H, perm, off, N, C, out, sizes)
   if (dtype == SPARSEPR_BF16) { if (d == 128) SPR_GM(__nv_bfloat16, 128); else SPR_GM(__nv_bfloat16, 64); }
   else { if (d == 128) SPR_GM(float, 128); else SPR_GM(float, 64); }
