@@ -190,25 +190,35 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
       // the eight threads that own row k publish it together with the scalars of the reflector
       T part = T(0.0), x0p = T(0.0);
       if (row == k) {
-        st_vec<T, kPer>(xk + kSeg * h, a);                     // entries at columns <= k are never read
+        // v is published with zeros at the columns <= k: the loops below then need no column tests (a product with an
+        // exact zero leaves a sum as it is)
+        T xz[kPer];
 #pragma unroll
         for (int t = 0; t < kPer; ++t) {
           const int c = kPer * h + t;
+          xz[t] = c > k ? a[t] : T(0.0);
           part = c > k + 1 ? fma(a[t], a[t], part) : part;
           x0p = c == k + 1 ? a[t] : x0p;
         }
+        st_vec<T, kPer>(xk + kSeg * h, xz);
       }
 #pragma unroll
       for (int o = 1; o < kTpr; o <<= 1) {
         part += __shfl_xor_sync(0xffffffffu, part, o);
         x0p += __shfl_xor_sync(0xffffffffu, x0p, o);
       }
+      __syncwarp();
       if (row == k && h == 0) {
         const T below2 = part, x0 = x0p;                        // squares beyond the subdiagonal entry
+        // p of the rows that have just left the trailing block reads as zero from now on (this buffer was last read
+        // two steps ago; live rows write their entries after the barrier)
+        pk[pos(k)] = T(0.0);
+        if (k > 0) pk[pos(k - 1)] = T(0.0);
         if (below2 > T(0.0)) {
           const T alpha = sqrt(below2 + x0 * x0);
           const T sa = x0 >= T(0.0) ? alpha : -alpha;
           scal[0] = T(1.0); scal[1] = x0 + sa; scal[2] = T(1.0) / (alpha * (alpha + fabs(x0))); scal[3] = sa;
+          xk[pos(k + 1)] = x0 + sa;                             // first entry of v (the stored row is the reflector)
           ee[k] = -sa; beta[k] = scal[2]; e2[k] = sa;           // e2[] is free until the bisection
         } else {
           scal[0] = T(0.0);
@@ -228,18 +238,14 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
         T xv[kPer];
         ld_vec<T, kPer>(xk + kSeg * h, xv);
 #pragma unroll
-        for (int t = 0; t < kPer; ++t) {
-          const int c = kPer * h + t;
-          const T vc = c == k + 1 ? v0 : xv[t];
-          acc = c > k ? fma(a[t], vc, acc) : acc;
-        }
+        for (int t = 0; t < kPer; ++t) acc = fma(a[t], xv[t], acc);
       }
 #pragma unroll
       for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       p_row = b * acc;
       if (live && h == 0) pk[pos(row)] = p_row;
       // this warp's part of p.v (rows of the warp, one lane per row)
-      T pvw = (live && h == 0) ? p_row * (row == k + 1 ? v0 : xk[pos(row)]) : T(0.0);
+      T pvw = (live && h == 0) ? p_row * xk[pos(row)] : T(0.0);
 #pragma unroll
       for (int o = kTpr; o < 32; o <<= 1) pvw += __shfl_xor_sync(0xffffffffu, pvw, o);
       if (lane == 0) pvpart[warp] = pvw;
@@ -250,17 +256,15 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
     if (!warp_live) continue;                                   // nothing left to update in this warp's rows
     const T hb = T(0.5) * b * warp_sum(pvpart[lane]);
     if (live && kPer * h + kPer - 1 > k) {
-      const T v_row = row == k + 1 ? v0 : xk[pos(row)];
+      const T v_row = xk[pos(row)];
       const T w_row = p_row - hb * v_row;
       T xv[kPer], pv[kPer];
       ld_vec<T, kPer>(xk + kSeg * h, xv);
       ld_vec<T, kPer>(pk + kSeg * h, pv);
 #pragma unroll
       for (int t = 0; t < kPer; ++t) {
-        const int c = kPer * h + t;
-        const T vc = c == k + 1 ? v0 : xv[t];
-        const T wc = pv[t] - hb * vc;
-        a[t] = c > k ? a[t] - (v_row * wc + w_row * vc) : a[t];
+        const T wc = pv[t] - hb * xv[t];                        // zero at the columns <= k (v and p are zero there)
+        a[t] = a[t] - (v_row * wc + w_row * xv[t]);
       }
     }
   }
@@ -274,7 +278,6 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
       if (row == NN - 1 && c == NN - 2) ee[NN - 2] = a[t];
     }
   }
-  if (tid < NN - 2) A[tid * LD + pos(tid + 1)] += e2[tid];           // v_0 = x_0 + sgn alpha
   if (tid == 0) { ee[NN - 1] = T(0.0); beta[NN - 2] = T(0.0); beta[NN - 1] = T(0.0); }
   __syncthreads();
   if (tid < NN) e2[tid] = ee[tid] * ee[tid];
