@@ -1,4 +1,5 @@
 // C-ABI layer: argument validation, workspace carving, launch order.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -560,7 +561,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
                       p->route_idx, p->rstate, nullptr, r.G, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
-  launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
+  launch_remainder_rows(p->q_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
   if (overlap) p->side_pending = true;          // not joined here: the probes are not needed before the attend call
   tm.mark(SPARSEPR_STAGE_ROUTE);
   tm.finish();
@@ -629,7 +630,7 @@ sparsepr_status_t sparsepr_plan_import(const sparsepr_shape_t* shape, const spar
   launch_count_pairs(p->q_off, p->kv_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, p->rstate, r.G, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 64, 0, p->tile_off, st);
   launch_tile_offsets(p->q_off, r.BH, r.Cq, 128, kRemRows, p->tile_off128, st);
-  launch_remainder_rows(p->q_off, r.BH, r.Cq, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
+  launch_remainder_rows(p->q_off, p->route_ptr, p->route_idx, r.BH, r.Cq, r.Ck, r.N, p->rem_pos, p->rem_grp, p->rem_cnt, st);
   if (!launch_ok() || cudaStreamSynchronize(st) != cudaSuccess) { delete p; return SPARSEPR_ERR_CUDA; }
   *out = p;
   return SPARSEPR_OK;
@@ -804,7 +805,8 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
     const int qtile = tcpath ? 128 : 64, ktile = tcpath ? 128 : 64, box = tcpath ? 16 : 1;
     const int* rpp = &rp[(size_t)bh * (r.Cq + 1)];
     const int* rii = &ri[(size_t)bh * r.Cq * r.Ck];
-    // packed tiles: 128 remainder rows in group order; each streams the union of the K/V groups its rows route to
+    // packed tiles: 128 remainder rows each, groups in the order of k_remainder_rows (routed groups descending, first
+    // route ascending, id); a tile streams the union of the K/V groups its rows route to
     std::vector<char> want(r.Ck, 0);
     int packed_fill = 0;
     auto flush_packed = [&]() {
@@ -813,22 +815,29 @@ sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t
       out->padded_tile_pairs += (i64)qtile * ((boxes * box + ktile - 1) / ktile) * ktile;
       packed_fill = 0;
     };
+    std::vector<unsigned long long> packed_order;
     for (int a = 0; a < r.Cq; ++a) {
       i64 keys = 0;
       for (int t = rpp[a]; t < rpp[a + 1]; ++t) keys += (k[rii[t] + 1] - k[rii[t]] + box - 1) / box * box;
       const i64 kt = (keys + ktile - 1) / ktile;
       const int nrow = q[a + 1] - q[a], rem = nrow % qtile;
       if (tcpath && rem > 0 && rem <= kRemRows) {
-        // full tiles by the 128-row kernel; the short remainder joins the packed tiles that walk over all keys
+        // full tiles by the 128-row kernel; the short remainder joins the packed tiles
         out->padded_tile_pairs += (i64)(nrow / qtile) * qtile * kt * ktile;
-        for (int left = rem; left > 0;) {
-          const int take = std::min(left, qtile - packed_fill);
-          for (int t = rpp[a]; t < rpp[a + 1]; ++t) want[rii[t]] = 1;
-          packed_fill += take; left -= take;
-          if (packed_fill == qtile) flush_packed();
-        }
+        const int n = rpp[a + 1] - rpp[a];
+        packed_order.push_back(((unsigned long long)(r.Ck - n) << 24) | ((unsigned long long)(n > 0 ? rii[rpp[a]] : 0) << 12) | (unsigned long long)a);
       } else {
         out->padded_tile_pairs += (i64)((nrow + qtile - 1) / qtile) * qtile * kt * ktile;
+      }
+    }
+    std::sort(packed_order.begin(), packed_order.end());
+    for (unsigned long long key : packed_order) {
+      const int a = (int)(key & 0xFFFull);
+      for (int left = (q[a + 1] - q[a]) % qtile; left > 0;) {
+        const int take = std::min(left, qtile - packed_fill);
+        for (int t = rpp[a]; t < rpp[a + 1]; ++t) want[rii[t]] = 1;
+        packed_fill += take; left -= take;
+        if (packed_fill == qtile) flush_packed();
       }
     }
     if (packed_fill > 0) flush_packed();

@@ -114,9 +114,11 @@ bool launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 // small_rem = kRemRows) and handled by attention_packed.cu
 constexpr int kRemRows = 32;
 // attention_packed.cu: those remainders, packed across groups into 128-row tiles that walk over all keys with
-// per-row route masks.  rem_pos / rem_grp [BH][N], rem_cnt [BH] are built from the query offsets once per plan.
+// per-row route masks.  rem_pos / rem_grp [BH][N], rem_cnt [BH] are built from the query offsets and the routes once per
+// plan (groups that route alike are neighbours in the list).
 cudaError_t init_attention_packed();
-void launch_remainder_rows(const int* q_off, int BH, int Cq, int N, int* rem_pos, int* rem_grp, int* rem_cnt, cudaStream_t st);
+void launch_remainder_rows(const int* q_off, const int* route_ptr, const int* route_idx, int BH, int Cq, int Ck, int N, int* rem_pos,
+                           int* rem_grp, int* rem_cnt, cudaStream_t st);
 bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* rem_grp, const int* rem_cnt, cudaStream_t st);
 // one warp runs the bounded mbarrier wait into its limit (2^16 cycles) and records SPARSEPR_ERR_TIMEOUT in *err
 void launch_selftest_bounded_wait(int* err, cudaStream_t st);
