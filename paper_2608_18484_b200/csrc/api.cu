@@ -345,7 +345,7 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   float* X = c.take<float>(BH * M1 * d); float* Dn = c.take<float>(BH * M1 * d);
   float* A = c.take<float>(BH * d * d); float* cc = c.take<float>(BH * d);
   float* Psi = c.take<float>(BH * d * d);
-  __nv_bfloat16* At = c.take<__nv_bfloat16>(BH * d * d);
+  __nv_bfloat16* At = c.take<__nv_bfloat16>(2 * BH * d * d);   // the correction map as two bf16 words
   double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
   if (w) { w->Olo = Olo; w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->n_split = ns; }
 }

@@ -123,7 +123,7 @@ bool launch_attention_packed(const AttnArgs& a, const int* rem_pos, const int* r
 // one warp runs the bounded mbarrier wait into its limit (2^16 cycles) and records SPARSEPR_ERR_TIMEOUT in *err
 void launch_selftest_bounded_wait(int* err, cudaStream_t st);
 // correction_tc.cu: O <- X + X A + c in place, X = O + O_lo (two bf16 words, O_lo [BH][N][128] contiguous), d_v = 128;
-// At: bf16 scratch [BH][128][128]
+// At: bf16 scratch [2][BH][128][128] (the map as two bf16 words)
 cudaError_t init_correction_tc();
 bool launch_correction_tc(const float* A, const float* c, __nv_bfloat16* At, const void* O_lo, void* O, const i64* os, int BH,
                           int H, int N, int* err, cudaStream_t st);

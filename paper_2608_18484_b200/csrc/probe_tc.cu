@@ -5,9 +5,11 @@
 // omitted ones (Z_U, N_U).  From them O_sp = N_S / Z_S and
 // O_dense = (N_S + N_U) / (Z_S + Z_U).  A CTA owns 128 probe rows and one slice of the key
 // range; partial states are merged by k_probe_merge.
-//   warps 0-3  softmax, one thread per probe row
-//   warp  4    K producer (also builds the per-tile list of K/V-group runs), warp 5 V producer
-//   warp  6    tcgen05.mma issuer, owns TMEM
+//   warps 0-7  softmax: warps w and w + 4 share the 32 probe rows of TMEM quadrant w and split the 128 scores of a
+//              row in two halves (every score belongs to one of the two states, so a half costs half the work;
+//              with one warp per scheduler the loop ran at the latency of its instructions)
+//   warp  8    K producer (also builds the per-tile list of K/V-group runs), warp 9 V producer
+//   warp  10   tcgen05.mma issuer, owns TMEM
 // TMEM: S0 [0,128), S1 [128,256), O_S [256,384), O_U [384,512).  The exponentials of a tile
 // are written back over its score buffer as bf16: retained weights in columns [0,64),
 // omitted weights in [64,128); the two P V products read them from TMEM.
@@ -17,7 +19,8 @@
 namespace spr {
 namespace tc {
 
-constexpr int kPbThreads = 224;
+constexpr int kPbThreads = 352;
+constexpr int kPbWarpK = 8, kPbWarpV = 9, kPbWarpMma = 10;
 constexpr int kPbTile = 128;
 constexpr uint32_t kPbHalf = 128 * 128;              // [128 rows x 64 bf16] swizzled block
 constexpr uint32_t kPbTileBytes = 2 * kPbHalf;
@@ -32,7 +35,8 @@ struct PbSmem {
   static constexpr uint32_t v = k + kPbKStages * kPbTileBytes;
   static constexpr uint32_t bitmap = v + kPbVStages * kPbTileBytes;        // [kMaxGroups/32 words][128 rows]
   static constexpr uint32_t meta = bitmap + (kMaxGroups / 32) * 128 * 4;   // PbMeta[8]
-  static constexpr uint32_t bars = meta + 8 * 32;
+  static constexpr uint32_t xchg = meta + 8 * 32;                          // float [2][2][2][128] half-row maxima of both states, [2][2][128] sums
+  static constexpr uint32_t bars = xchg + 12 * 128 * 4;
   static constexpr uint32_t misc = bars + 32 * 8;
   static constexpr uint32_t total = misc + 64;
 };
@@ -78,11 +82,11 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   const int words = (prm.Ck + 31) / 32;
 
   if (tid == 0) {
-    for (int i = 0; i < kPbNumBars; ++i) mbar_init(bar(i), (i == PP_FULL || i == PP_FULL + 1) ? 128 : 1);
+    for (int i = 0; i < kPbNumBars; ++i) mbar_init(bar(i), (i == PP_FULL || i == PP_FULL + 1) ? 256 : 1);
     misc[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 6) tmem_alloc(base + PbSmem::misc, 512);
+  if (warp == kPbWarpMma) tmem_alloc(base + PbSmem::misc, 512);
   // route bitmap of every probe row, transposed: bitmap[word][row]
   for (int e = tid; e < words * 128; e += kPbThreads) bitmap[e] = 0u;
   __syncthreads();
@@ -117,10 +121,10 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     return c;
   };
 
-  if (warp == 4 || warp == 5) {
+  if (warp == kPbWarpK || warp == kPbWarpV) {
     // =========================== producers ==================================================
     if (lane == 0 && p_begin < p_end) {
-      const bool is_k = warp == 4;
+      const bool is_k = warp == kPbWarpK;
       if (is_k) {
         mbar_expect_tx(bar(PQ_FULL), kPbTileBytes);
         tma_load_4d(base + PbSmem::q, &mapQ, bar(PQ_FULL), 0, m0, bh, 0);
@@ -148,7 +152,7 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         pos += nc;
       }
     }
-  } else if (warp == 6) {
+  } else if (warp == kPbWarpMma) {
     // =========================== MMA issuer ==================================================
     if (lane == 0 && p_begin < p_end) {
       const uint32_t idesc_qk = idesc_bf16(0, 128), idesc_pv = idesc_bf16(1, 128);
@@ -193,24 +197,30 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         umma_commit(bar(PT_DONE));                              // O_S / O_U hold every tile up to i
       }
     }
-  } else if (warp < 4) {
+  } else if (warp < 8) {
     // =========================== softmax ========================================================
-    const int row = warp * 32 + lane;
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    // Thread (half hh, quadrant wq, lane) owns the scores of keys [64 hh, 64 hh + 64) of probe row 32 wq + lane; the
+    // two halves of a row meet at the named barrier 1 + wq to agree on the two maxima of the tile.
+    const int hh = warp >> 2, wq = warp & 3;
+    const int row = wq * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
     const uint32_t FULL = 0xffffffffu;
     const float sc = prm.scale_log2;
+    float* xmax = reinterpret_cast<float*>(sm + PbSmem::xchg);             // [parity][half][state][row]
+    float* xsum = xmax + 8 * 128;                                          // [half][state][row]
     float mS = -INFINITY, mU = -INFINITY, lS = 0.f, lU = 0.f;
     bool ok = true;
     int pos = p_begin, i = 0;
     for (; pos < p_end; ++i) {
       ok = __all_sync(FULL, ok && mbar_wait(bar(PS_FULL + (i & 1)), (i >> 1) & 1, abort_flag) &&
                                 mbar_wait(bar(PMETA_FULL + (i & 7)), (i >> 3) & 1, abort_flag));
-      if (!ok) break;                                           // warp-uniform; nothing else synchronises these warps
+      if (!ok) break;                                           // uniform over the CTA: every softmax warp waits on the same barriers
       tc_fence_after();
       const PbMeta mt = meta[i & 7];
       pos += mt.ncols;
-      // column masks: valid (inside the tile) and retained (K/V group routed to this row's query group)
-      unsigned ret[4] = {0u, 0u, 0u, 0u}, val[4];
+      // column masks of this half (two words of 32): valid (inside the tile) and retained (K/V group routed to this
+      // row's query group)
+      unsigned ret[2] = {0u, 0u}, val[2];
       {
         int beg = 0;
         for (int r = 0; r < mt.nruns; ++r) {
@@ -218,35 +228,42 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           const bool on = (bitmap[(g >> 5) * 128 + row] >> (g & 31)) & 1u;
           if (on) {
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-              const int lo = max(beg - 32 * w, 0), hi = min(e - 32 * w, 32);
+            for (int w = 0; w < 2; ++w) {
+              const int w0 = 32 * (2 * hh + w);
+              const int lo = max(beg - w0, 0), hi = min(e - w0, 32);
               if (hi > lo) ret[w] |= (hi - lo == 32 ? 0xFFFFFFFFu : ((1u << (hi - lo)) - 1u) << lo);
             }
           }
           beg = e;
         }
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const int hi = min(mt.ncols - 32 * w, 32);
+        for (int w = 0; w < 2; ++w) {
+          const int hi = min(mt.ncols - 32 * (2 * hh + w), 32);
           val[w] = hi <= 0 ? 0u : hi == 32 ? 0xFFFFFFFFu : (1u << hi) - 1u;
         }
       }
       const uint32_t s_addr = tmem + lane_addr + (uint32_t)(i & 1) * 128u;
-      float s[128];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        float t[32];
-        tmem_ld32(s_addr + q * 32, t);
-#pragma unroll
-        for (int c = 0; c < 32; ++c) s[q * 32 + c] = t[c];
-      }
+      float s[64];
+      tmem_ld32_nowait(s_addr + 64 * hh, *reinterpret_cast<float(*)[32]>(&s[0]));
+      tmem_ld32_nowait(s_addr + 64 * hh + 32, *reinterpret_cast<float(*)[32]>(&s[32]));
+      tmem_ld_wait();
       float mxS = -INFINITY, mxU = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 128; ++c) {
+      for (int c = 0; c < 64; ++c) {
         const bool v = (val[c >> 5] >> (c & 31)) & 1u, r = (ret[c >> 5] >> (c & 31)) & 1u;
         s[c] = v ? s[c] : -INFINITY;
         mxS = fmaxf(mxS, r ? s[c] : -INFINITY);
         mxU = fmaxf(mxU, r ? -INFINITY : s[c]);
+      }
+      // the halves exchange their maxima; past this barrier both hold their scores in registers, so the weights
+      // may be written over the score buffer
+      {
+        float* xm = xmax + (i & 1) * 512;
+        xm[(hh * 2 + 0) * 128 + row] = mxS;
+        xm[(hh * 2 + 1) * 128 + row] = mxU;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+        mxS = fmaxf(mxS, xm[((hh ^ 1) * 2 + 0) * 128 + row]);
+        mxU = fmaxf(mxU, xm[((hh ^ 1) * 2 + 1) * 128 + row]);
       }
       // lazily moved reference maxima (see the attention kernel); a state without any key yet keeps -inf
       const bool moveS = mxS > -INFINITY && (mxS - mS) * sc > 8.f, moveU = mxU > -INFINITY && (mxU - mU) * sc > 8.f;
@@ -256,24 +273,25 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       // the accumulators are stable once the previous P V products have completed
       if (i > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(PT_DONE), (i - 1) & 1, abort_flag));
       if (!ok) break;
-      if (i > 0 && __any_sync(FULL, moveS || moveU)) {           // rescale O_S / O_U rows (rare)
+      if (i > 0 && __any_sync(FULL, moveS || moveU)) {           // rescale this half of the O_S / O_U rows (rare)
         tc_fence_after();
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 4; ++q) {
           float t[32];
-          const float f = q < 4 ? cS : cU;
-          tmem_ld32(tmem + lane_addr + 256u + q * 32, t);
+          const float f = q < 2 ? cS : cU;
+          const uint32_t a = tmem + lane_addr + 256u + (uint32_t)(q >> 1) * 128u + (uint32_t)hh * 64u + (uint32_t)(q & 1) * 32u;
+          tmem_ld32(a, t);
 #pragma unroll
           for (int c = 0; c < 32; ++c) t[c] *= f;
-          tmem_st32(tmem + lane_addr + 256u + q * 32, t);
+          tmem_st32(a, t);
         }
       }
       const float nS = mS > -INFINITY ? -mS * sc : 0.f, nU = mU > -INFINITY ? -mU * sc : 0.f;
       float sumS = 0.f, sumU = 0.f;
       // exponentials, packed in place: afterwards s[2j] holds the bf16 pair of retained weights of
-      // columns (2j, 2j+1) and s[2j+1] the pair of omitted weights
+      // columns (2j, 2j+1) of this half and s[2j+1] the pair of omitted weights
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
+      for (int j = 0; j < 32; ++j) {
         float eS[2], eU[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -290,15 +308,14 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
       lS = lS * cS + sumS;
       lU = lU * cU + sumU;
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
+      {
         uint32_t w[32];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) w[c] = __float_as_uint(s[2 * (q * 32 + c)]);
-        tmem_st32u(s_addr + q * 32, w);
+        for (int c = 0; c < 32; ++c) w[c] = __float_as_uint(s[2 * c]);
+        tmem_st32u(s_addr + 32 * hh, w);                        // retained weights of keys [64 hh, 64 hh + 64)
 #pragma unroll
-        for (int c = 0; c < 32; ++c) w[c] = __float_as_uint(s[2 * (q * 32 + c) + 1]);
-        tmem_st32u(s_addr + 64 + q * 32, w);
+        for (int c = 0; c < 32; ++c) w[c] = __float_as_uint(s[2 * c + 1]);
+        tmem_st32u(s_addr + 64 + 32 * hh, w);                   // omitted weights
       }
       tc_fence_before();
       mbar_arrive(bar(PP_FULL + (i & 1)));
@@ -306,7 +323,12 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     // ---- partial states of this slice -----------------------------------------------------------
     const bool any = p_begin < p_end;
     if (any) ok = __all_sync(FULL, ok && i > 0 && mbar_wait(bar(PT_DONE), (i - 1) & 1, abort_flag));
-    if (row < nrows) {
+    xsum[(hh * 2 + 0) * 128 + row] = lS;
+    xsum[(hh * 2 + 1) * 128 + row] = lU;
+    asm volatile("bar.sync %0, 64;" ::"r"(1 + wq) : "memory");
+    lS += xsum[((hh ^ 1) * 2 + 0) * 128 + row];
+    lU += xsum[((hh ^ 1) * 2 + 1) * 128 + row];
+    if (row < nrows && hh == 0) {
       float* out = prm.partial + ((((i64)bh * prm.n_split + split) * prm.M + m0 + row) * 2) * 130;
       const bool good = ok && any;
       out[0] = (good && lS > 0.f) ? mS * sc : -INFINITY; out[1] = good ? lS : 0.f;
@@ -315,11 +337,11 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (ok && any) {
       tc_fence_after();
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < 4; ++q) {                             // this half's 64 columns of O_S, then of O_U
         float t[32];
-        tmem_ld32(tmem + lane_addr + 256u + q * 32, t);
+        tmem_ld32(tmem + lane_addr + 256u + (uint32_t)(q >> 1) * 128u + (uint32_t)hh * 64u + (uint32_t)(q & 1) * 32u, t);
         if (row < nrows) {
-          float* out = prm.partial + ((((i64)bh * prm.n_split + split) * prm.M + m0 + row) * 2 + (q >> 2)) * 130 + 2 + (q & 3) * 32;
+          float* out = prm.partial + ((((i64)bh * prm.n_split + split) * prm.M + m0 + row) * 2 + (q >> 1)) * 130 + 2 + hh * 64 + (q & 1) * 32;
 #pragma unroll
           for (int c = 0; c < 32; ++c) out[c] = t[c];
         }
@@ -333,7 +355,7 @@ k_probe_rows_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (tid == 0) set_error(prm.err, SPARSEPR_ERR_TIMEOUT);
     __syncthreads();
   }
-  if (warp == 6) {
+  if (warp == kPbWarpMma) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
