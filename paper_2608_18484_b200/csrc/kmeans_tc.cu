@@ -5,8 +5,9 @@
 // xh.ml, xl.mh are accumulated in fp32 in TMEM; the dropped term is ~2^-18 relative).
 // Each row keeps its best and second-best score; a row whose gap is not larger than a
 // conservative bound on the score error is NOT decided here but handed to the exact
-// float64 recheck (one CTA per row, same operation order as the definition), so the
-// final assignment always equals the exact float64 decision with ties to the lowest id.
+// recheck (per-head row lists; float64 with the operation order of the definition for every
+// centroid that a float32 filter cannot rule out), so the final assignment always equals the
+// exact float64 decision with ties to the lowest id.
 //
 // Persistent CTAs: each owns row tiles (128 rows) of one head; centroid chunks of 256
 // stream through shared memory (resident when C <= 256).  Roles: warps 0-3 and 6-9 are two
