@@ -26,6 +26,11 @@
 // Eq. 9 is a pass of its own (correction_tc.cu) so that the fit can overlap this kernel; for that pass the part of
 // every element that the bf16 rounding dropped is stored as a second bf16 word (O_lo), so that the corrected output
 // is, in effect, rounded to bf16 only once.
+// A tile with at most 64 valid rows (the remainder of a query group) holds every row TWICE, at lanes r and r + 64:
+// the time of a key tile is the sequential work of a softmax thread, which does not shrink with the number of valid
+// rows, so the four threads that then sit on a row (two lanes x two halves) take 32 of its 128 scores each; the
+// copy at lane r accumulates the keys [0,32) and [64,96) of every tile, the copy at lane r + 64 the others, and the
+// epilogue adds the two accumulators.  The products themselves are unchanged (the tile was padded to 128 rows anyway).
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
@@ -82,8 +87,8 @@ struct Maps { CUtensorMap m[4]; };      // the same tensor with boxes of 16, 32,
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) { return pack_bf16x2(a, b); }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ Maps mapsK,
-               const __grid_constant__ Maps mapsV, Params prm) {
+k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapQ64,
+               const __grid_constant__ Maps mapsK, const __grid_constant__ Maps mapsV, Params prm) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* sm = smem_raw;
@@ -135,6 +140,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     nrows = min(kTile, prm.N - row0);
     nroute = 1;
   }
+  const bool dup = prm.sparse && nrows <= kTile / 2;           // every row twice: lanes r and r + 64 (see the header)
 
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
@@ -176,8 +182,16 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (is_k && lane == 0) {
         const int q2 = prm.sparse ? bh : h;
         mbar_expect_tx(bar(Q_FULL), kTileBytes);
-        tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, q2, c3);
-        tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, q2, c3);
+        if (dup) {
+          // the same 64 rows into both halves of the tile (rows 64-127 of a [128 x 64] block start 8 KB in)
+          for (int part = 0; part < 2; ++part) {
+            tma_load_4d(base + Smem::q + part * (kHalfBytes / 2), &mapQ64, bar(Q_FULL), 0, row0, q2, c3);
+            tma_load_4d(base + Smem::q + kHalfBytes + part * (kHalfBytes / 2), &mapQ64, bar(Q_FULL), 64, row0, q2, c3);
+          }
+        } else {
+          tma_load_4d(base + Smem::q, &mapQ, bar(Q_FULL), 0, row0, q2, c3);
+          tma_load_4d(base + Smem::q + kHalfBytes, &mapQ, bar(Q_FULL), 64, row0, q2, c3);
+        }
       }
       const int nst = is_k ? kKStages : kVStages;
       const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
@@ -297,6 +311,168 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     const float sc = prm.scale_log2;
+    // the 64 finished output columns [64 hh, 64 hh + 64) of tile row r: bf16 at the original token index, the part that
+    // the rounding dropped as a second word, float32 on request
+    auto store_row = [&](int r, const float (&o)[64]) {
+      const int dst = prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + r] : row0 + r;
+      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + hh * 64;
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        float v8[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
+        store8(op + ch * 8, v8);
+      }
+      if (prm.O_lo) {                                          // what the bf16 rounding above dropped
+        __nv_bfloat16* lp = prm.O_lo + ((i64)bh * prm.N + dst) * kD + hh * 64;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k] - __bfloat162float(__float2bfloat16_rn(o[ch * 8 + k]));
+          store8(lp + ch * 8, v8);
+        }
+      }
+      if (prm.O_sparse) {
+        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          float v8[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
+          store8(sp + ch * 8, v8);
+        }
+      }
+    };
+    if (dup) {
+      // ================= at most 64 valid rows: four threads per row, 32 scores each ==================
+      const int u = wq >> 1, q0 = wq & 1;                        // copy of the row (lane r or r + 64); pair of quadrants
+      const int vr = q0 * 32 + lane;                             // the row, 0..63
+      const int cb = 64 * hh + 32 * u;                           // this thread's keys of a tile: [cb, cb + 32)
+      const int slot = 2 * hh + u;
+      for (int i = 0; i < n_tiles; ++i) {
+        const bool t_meta = mbar_try(bar(META_FULL + (i & 7)), (i >> 3) & 1);
+        const bool t_s = mbar_try(bar(S_FULL + (i & 1)), (i >> 1) & 1);
+        const bool t_pe = i > 1 ? mbar_try(bar(P_EMPTY + (i & 1)), ((i - 2) >> 1) & 1) : true;
+        {
+          bool w = ok;
+          if (!t_meta) w = w && mbar_wait(bar(META_FULL + (i & 7)), (i >> 3) & 1, abort_flag);
+          if (!t_s) w = w && mbar_wait(bar(S_FULL + (i & 1)), (i >> 1) & 1, abort_flag);
+          ok = __all_sync(FULL, w);
+        }
+        float s[32];
+        float mx = -INFINITY;
+        if (ok) {
+          tc_fence_after();
+          const uint2 mt = meta[i & 7];
+          tmem_ld32_nowait(tmem + lane_addr + (uint32_t)(i & 1) * 128u + (uint32_t)cb, s);
+          tmem_ld_wait();
+          tc_fence_before();
+          mbar_arrive(bar(S_FREE + (i & 1)));                       // the scores are in registers
+          if (!(mt.x == 0xFFFFFFFFu && mt.y == 8u)) {
+#pragma unroll
+            for (int bx = 0; bx < 2; ++bx) {
+              const int box = (cb >> 4) + bx;
+              const int lim = box < (int)mt.y ? (int)((mt.x >> (4 * box)) & 15u) : -1;    // last valid column of the box
+              if (lim != 15) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) s[bx * 16 + c] = (c <= lim) ? s[bx * 16 + c] : -INFINITY;
+              }
+            }
+          }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            mx4[0] = max3(mx4[0], s[c], s[c + 1]); mx4[1] = max3(mx4[1], s[c + 2], s[c + 3]);
+            mx4[2] = max3(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3(mx4[3], s[c + 6], s[c + 7]);
+          }
+          mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        }
+        // the four threads of a row exchange their maxima (four warps meet: both halves of quadrants q0 and q0 + 2)
+        float* xm = xmax + (i & 1) * 256;
+        xm[slot * 64 + vr] = mx;
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q0) : "memory");
+        mx = fmaxf(fmaxf(xm[vr], xm[64 + vr]), fmaxf(xm[128 + vr], xm[192 + vr]));
+        const bool move = (mx - m_ref) * sc > 8.f;
+        const float m_new = move ? mx : m_ref;
+        const float corr = move ? ex2((m_ref - m_new) * sc) : 1.f;
+        const float mneg = -m_new * sc;
+        m_ref = m_new;
+        if (!__all_sync(FULL, t_pe)) {
+          ok = __all_sync(FULL, ok && (t_pe || mbar_wait(bar(P_EMPTY + (i & 1)), ((i - 2) >> 1) & 1, abort_flag)));
+          tc_fence_after();
+        }
+        if (!ok) continue;
+        if (i > 0 && __any_sync(FULL, move)) {                   // rescale this half of the lane's accumulator (rare)
+          ok = __all_sync(FULL, mbar_wait(bar(P_EMPTY + ((i - 1) & 1)), ((i - 1) >> 1) & 1, abort_flag));
+          if (!ok) continue;
+          tc_fence_after();
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            float t[32];
+            tmem_ld32(o_addr + q * 32, t);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) t[c] *= corr;
+            tmem_st32(o_addr + q * 32, t);
+          }
+        }
+        float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        const float2 sc2 = make_float2(sc, sc), mneg2 = make_float2(mneg, mneg);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          float2 x = __ffma2_rn(make_float2(s[2 * q], s[2 * q + 1]), sc2, mneg2);
+          if ((q & 7) < kPolyOf8) x = ex2_poly2(x);
+          else { x.x = ex2(x.x); x.y = ex2(x.y); }
+          s[2 * q] = x.x; s[2 * q + 1] = x.y;
+          ps2[q & 1] = __fadd2_rn(ps2[q & 1], x);
+        }
+        l = l * corr + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
+        // P of this lane and half: this thread's 32 probabilities -> 16 columns, zeros in the 16 columns of the keys
+        // that the other copy of the row takes
+        {
+          uint32_t w[16], z[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c) { w[c] = pack_bf16(s[2 * c], s[2 * c + 1]); z[c] = 0u; }
+          const uint32_t pa = p_addr0 + (uint32_t)(i & 1) * 192u;
+          tmem_st16u_nowait(pa + 16u * (uint32_t)u, w);
+          tmem_st16u_nowait(pa + 16u * (uint32_t)(1 - u), z);
+          tmem_st_wait();
+        }
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL + (i & 1)));
+      }
+      // ---- row sums of the four threads, sum of the two accumulators, normalise, store -----------------
+      if (n_tiles > 0) ok = __all_sync(FULL, ok && mbar_wait(bar(O_DONE), 0, abort_flag));
+      xsum[slot * 64 + vr] = l;
+      float o[64];
+#pragma unroll
+      for (int c = 0; c < 64; ++c) o[c] = 0.f;
+      if (ok && n_tiles > 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          float t[32];
+          tmem_ld32(o_addr + q * 32, t);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[q * 32 + c] = t[c];
+        }
+      }
+      // the copy at lane r + 64 hands its accumulator over through the Q tile's shared memory (every product that
+      // reads it has completed): [half][column][row], conflict-free for consecutive rows
+      float* ex = reinterpret_cast<float*>(sm + Smem::q);
+      if (u == 1) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) ex[(hh * 64 + c) * 64 + vr] = o[c];
+      }
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + q0) : "memory");
+      if (u == 0) {
+        const float ltot = (xsum[vr] + xsum[64 + vr]) + (xsum[128 + vr] + xsum[192 + vr]);
+        const float inv = ltot > 0.f ? 1.f / ltot : 0.f;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) o[c] = inv != 0.f ? (o[c] + ex[(hh * 64 + c) * 64 + vr]) * inv : 0.f;
+        if (ok && vr < nrows) store_row(vr, o);
+      }
+    } else {
     for (int i = 0; i < n_tiles; ++i) {
       // the three barriers of this tile are polled back to back (their shared-memory round trips overlap); the P
       // buffer of this parity was consumed by the product two tiles back and is normally free long before
@@ -412,36 +588,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
       }
     }
-    if (ok && row < nrows) {
-      const int dst = prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + row] : row0 + row;
-      __nv_bfloat16* op = prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + hh * 64;
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        float v8[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
-        store8(op + ch * 8, v8);
-      }
-      if (prm.O_lo) {                                          // what the bf16 rounding above dropped
-        __nv_bfloat16* lp = prm.O_lo + ((i64)bh * prm.N + dst) * kD + hh * 64;
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          float v8[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k] - __bfloat162float(__float2bfloat16_rn(o[ch * 8 + k]));
-          store8(lp + ch * 8, v8);
-        }
-      }
-      if (prm.O_sparse) {
-        float* sp = prm.O_sparse + ((i64)bh * prm.N + dst) * kD + hh * 64;
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          float v8[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) v8[k] = o[ch * 8 + k];
-          store8(sp + ch * 8, v8);
-        }
-      }
+    if (ok && row < nrows) store_row(row, o);
     }
   }
   // ---- teardown ----------------------------------------------------------------------------
@@ -505,19 +652,21 @@ bool attention_tc_supported(const AttnArgs& a) {
 
 bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   using namespace tc;
-  CUtensorMap mq;
+  CUtensorMap mq, mq64;
   Maps mk, mv;
   const bool sparse = a.route_ptr != nullptr;
   const int B = a.BH / a.H;
   const int kvd = a.kv_div < 1 ? 1 : a.kv_div;
   bool ok;
   if (sparse) {
-    ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile);
+    ok = make_map(&mq, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile) &&
+         make_map(&mq64, a.Q, kD, a.N, a.BH, 1, 0, (i64)a.N * kD, kD, kTile / 2);
     for (int k = 0; k < 4 && ok; ++k)
       ok = make_map(&mk.m[k], a.K, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k) &&
            make_map(&mv.m[k], a.V, kD, a.N, a.BH / kvd, 1, 0, (i64)a.N * kD, kD, kSub << k);
   } else {
-    ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile);
+    ok = make_map(&mq, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile) &&
+         make_map(&mq64, a.Q, kD, a.N, a.H, B, a.qs[0], a.qs[1], a.qs[2], kTile / 2);
     for (int k = 0; k < 4 && ok; ++k)
       ok = make_map(&mk.m[k], a.K, kD, a.N, a.H / kvd, B, a.ks[0], a.ks[1], a.ks[2], kSub << k) &&
            make_map(&mv.m[k], a.V, kD, a.N, a.H / kvd, B, a.vs[0], a.vs[1], a.vs[2], kSub << k);
@@ -531,7 +680,7 @@ bool launch_attention_tc(const AttnArgs& a, cudaStream_t st) {
   p.O = (__nv_bfloat16*)a.O; for (int i = 0; i < 3; ++i) p.os[i] = a.os[i];
   p.O_sparse = a.O_sparse; p.O_lo = (__nv_bfloat16*)a.O_lo; p.err = a.err;
   const int tiles = (a.N + kTile - 1) / kTile + (sparse ? a.Cq : 0);
-  k_attention_tc<<<dim3(tiles, a.BH), kThreads, kSmemBytes, st>>>(mq, mk, mv, p);
+  k_attention_tc<<<dim3(tiles, a.BH), kThreads, kSmemBytes, st>>>(mq, mq64, mk, mv, p);
   return true;
 }
 
