@@ -27,10 +27,11 @@
 // every element that the bf16 rounding dropped is stored as a second bf16 word (O_lo), so that the corrected output
 // is, in effect, rounded to bf16 only once.
 // A tile with at most 64 valid rows (the remainder of a query group) holds every row TWICE, at lanes r and r + 64:
-// the time of a key tile is the sequential work of a softmax thread, which does not shrink with the number of valid
-// rows, so the four threads that then sit on a row (two lanes x two halves) take 32 of its 128 scores each; the
-// copy at lane r accumulates the keys [0,32) and [64,96) of every tile, the copy at lane r + 64 the others, and the
-// epilogue adds the two accumulators.  The products themselves are unchanged (the tile was padded to 128 rows anyway).
+// the softmax threads of lanes 64-127 would otherwise spend a full tile's worth of exponentials on rows that do not
+// exist (the loop is bound by the throughput of those instructions).  The four threads that then sit on a row (two
+// lanes x two halves) take 32 of its 128 scores each; the copy at lane r accumulates the keys [0,32) and [64,96) of
+// every tile, the copy at lane r + 64 the others, and the epilogue adds the two accumulators.  The products
+// themselves are unchanged (the tile was padded to 128 rows anyway).
 // Every mbarrier wait is bounded; on expiry the CTA records SPARSEPR_ERR_TIMEOUT and leaves.
 #include <cuda.h>
 #include <mutex>
