@@ -254,7 +254,7 @@ struct sparsepr_plan_s {
   int *route_ptr, *route_idx, *tile_off, *tile_off128;
   RouteState* rstate;
   double* probe_dist; int* probe_idx; float* probe_w;
-  __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged; int* flagcnt;
+  __nv_bfloat16 *xh, *xl, *mh, *ml, *Ft; float* xnorm; int* flagged; int* flagcnt; double* eigws;
   int *rem_pos, *rem_grp, *rem_cnt;      // rows of the short group remainders (packed attention tiles)
   int* km_changed;                       // [2 sides][T + 1][BH] rows that changed group in each k-means pass
   double* Mpool;                         // [BHkv][d][d] key-response metric pooled over the query heads of a K/V head (grouped-query attention only)
@@ -298,9 +298,10 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
   int* km_changed = c.take<int>(2 * (size_t)(r.T + 1) * BH);
   int* flagcnt = c.take<int>(BH);
+  double* eigws = c.take<double>(eig_scratch_doubles((int)BH, r.d));
   double* Mpool = c.take<double>(r.G > 1 ? (size_t)r.BHkv * d * d : 0);
   if (p) {
-    p->km_changed = km_changed; p->flagcnt = flagcnt; p->Mpool = Mpool; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
+    p->km_changed = km_changed; p->flagcnt = flagcnt; p->eigws = eigws; p->Mpool = Mpool; p->Ft = Ft; p->rem_pos = rem_pos; p->rem_grp = rem_grp; p->rem_cnt = rem_cnt;
     p->err = err; p->recheck = recheck; p->Mmat = Mmat; p->lam = lam; p->FK = FK; p->FQ = FQ; p->phi = phi;
     p->maxabs = maxabs; p->fx_shift = fx; p->mu = mu; p->mu2 = mu2; p->mumax = mumax; p->sums = sums; p->counts = counts;
     p->a_K = aK; p->a_Q = aQ; p->kv_perm = kvp; p->kv_inv = kvi; p->q_perm = qp; p->q_inv = qi; p->kv_off = kvo; p->q_off = qo;
@@ -316,7 +317,7 @@ struct AttendWs {
   float *partial, *X, *Dn, *A, *c, *Psi;
   __nv_bfloat16 *At, *Qp;
   int n_split_tc;
-  double* fit;
+  double* fit; double* fit_eigws;
   int n_split;
 };
 
@@ -347,7 +348,8 @@ void carve_attend(Carver& c, const Resolved& r, AttendWs* w) {
   float* Psi = c.take<float>(BH * d * d);
   __nv_bfloat16* At = c.take<__nv_bfloat16>(2 * BH * d * d);   // the correction map as two bf16 words
   double* fit = c.take<double>(fit_scratch_doubles(r.BH, (int)M1, r.d));
-  if (w) { w->Olo = Olo; w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->n_split = ns; }
+  double* fit_eigws = c.take<double>(eig_scratch_doubles(r.BH, r.d));
+  if (w) { w->Olo = Olo; w->Qg = Qg; w->Kg = Kg; w->Vg = Vg; w->partial = partial; w->X = X; w->Dn = Dn; w->A = A; w->c = cc; w->Psi = Psi; w->At = At; w->Qp = Qp; w->n_split_tc = ns_tc; w->fit = fit; w->fit_eigws = fit_eigws; w->n_split = ns; }
 }
 
 i64 pair_budget(const Resolved& r) {
@@ -514,7 +516,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
       k_pool_metric<<<dim3(16, r.BHkv), 256, 0, st>>>(p->Mmat, r.G, r.d * r.d, p->Mpool);
       metric = p->Mpool;
     }
-    launch_eig_top(metric, (i64)r.d * r.d, r.BHkv, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, st);
+    launch_eig_top(metric, (i64)r.d * r.d, r.BHkv, r.d, r.rK, 0, r.dtype == SPARSEPR_F32, p->FK, p->lam, p->eigws, st);
     tm.mark(SPARSEPR_STAGE_KEY_METRIC);
     if (project_tc_supported(r.dtype, r.d, r.rK, r.ks)) {
       if (!launch_project_tc(K, r.ks, r.BHkv, r.Hkv, r.N, r.rK, p->FK, false, 0.f, p->phi, r.RK, p->maxabs, p->Ft, p->err, st)) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -535,7 +537,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
     launch_raw_features(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, p->phi, p->maxabs, p->err, st);
   } else {
     launch_centroid_gram(p->kappa, p->nk, r.BHkv, r.Ck, r.d, p->Mmat, st);
-    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BHkv, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, st);
+    launch_eig_top(p->Mmat, (i64)r.d * r.d, r.BHkv, r.d, r.rQ, 0, r.dtype == SPARSEPR_F32, p->FQ, p->lam, p->eigws, st);
     tm.mark(SPARSEPR_STAGE_QUERY_METRIC);
     if (project_tc_supported(r.dtype, r.d, r.rQ, r.qs)) {
       if (!launch_project_tc(Q, r.qs, r.BH, r.H, r.N, r.rQ, p->FQ, true, r.eps_rms, p->phi, r.RQ, p->maxabs, p->Ft, p->err, st, r.G)) { delete p; return SPARSEPR_ERR_CUDA; }
@@ -691,7 +693,7 @@ static sparsepr_status_t attend_impl(const sparsepr_plan_t* p, const void* Q, co
     tm.mark(SPARSEPR_STAGE_PROBE_ROWS);
     FitArgs fa{};
     fa.BH = r.BH; fa.M = r.M; fa.d = r.d; fa.r_out = r.r_out; fa.full_rank = r.full_rank; fa.lambda = r.lambda; fa.eps_std = r.eps_std; fa.precise = r.dtype == SPARSEPR_F32;
-    fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
+    fa.X = w.X; fa.Dn = w.Dn; fa.w = p->probe_w; fa.scratch = w.fit; fa.eig_ws = w.fit_eigws; fa.A = w.A; fa.c = w.c; fa.Psi = w.Psi; fa.err = p->err;
     launch_fit(fa, fs);
     tm.mark(SPARSEPR_STAGE_FIT);
   }

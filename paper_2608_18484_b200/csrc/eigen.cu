@@ -1,8 +1,10 @@
 // Leading eigenpairs of batched symmetric matrices (n = 64 or 128), one CTA per matrix:
 // the feature maps F_K, F_Q of Section 4.1 and the probe-residual basis Psi_r of Eq. 9.
 //
-// Float64 for float32 tensors, float32 for bf16 tensors; matrix in registers, reflectors and vectors in shared memory:
-//   1. Householder reduction to tridiagonal form T (reflectors kept in the lower triangle)
+// Float64 for float32 tensors, float32 for bf16 tensors.  Two kernels: k_householder (step 1, 2 n threads, matrix in
+// registers) hands the tridiagonal form and the reflectors to k_eig_tridiag (steps 2-6, 1024 threads) through a
+// scratch buffer:
+//   1. Householder reduction to tridiagonal form T (reflectors kept)
 //   2. the r largest eigenvalues of T by Sturm-count bisection, one thread per eigenvalue
 //   3. their eigenvectors by inverse iteration on T - lambda I (Gaussian elimination with
 //      partial pivoting, factored once per eigenvalue), one thread per eigenvector
@@ -13,7 +15,8 @@
 //      at once for unmarked matrices
 //   6. back-transformation with the reflectors, scaling, output
 // The work per matrix is O(n^3) for step 1 and O(r n^2) for step 6, each spread over the CTA;
-// steps 2-3 are O(n) recurrences per thread.
+// steps 2-3 are O(n) recurrences per thread.  Step 1 is a chain of n - 2 dependent steps, so it runs on few threads
+// with many matrix entries each (64 registers of matrix per thread at n = 128) rather than on all 1024.
 #include "kernels.cuh"
 
 namespace spr {
@@ -128,12 +131,179 @@ __device__ __forceinline__ int sturm_count(const T* __restrict__ dd, const T* __
   return cnt;
 }
 
+// What k_householder leaves per matrix for k_eig_tridiag (units of T): reflector k in row k of v (zero up to entry
+// k), diagonal, subdiagonal, the factors b_k of H_k = I - b_k v_k v_k^T, and the scale max |a_ij| of the input.
+template <int NN> struct HhLayout {
+  static constexpr int v = 0, dd = NN * NN, ee = dd + NN, beta = ee + NN, scale = beta + NN, stride = scale + 4;
+};
+
+// Householder reduction of a symmetric matrix to tridiagonal form, matrix in registers: thread (row, h) owns the
+// 16-column chunks h, h + 2, ... of its row (a CTA is 2 NN threads).  Step k: x = A[k+1.., k]; v = x + sgn(x_0) alpha e_1;
+// p = b A22 v; w = p - (b/2)(p.v) v; A22 <- A22 - v w^T - w v^T.  Every row keeps its own entries of the next two
+// columns (its entries of rows k+1 and k+2, by symmetry): the first becomes its entry of x, the second the term that
+// turns A x into A v, so nobody has to publish a whole row.  x and p are zero outside the trailing block, which lets
+// the inner loops run over all chunks without column tests.  Two barriers per step: one after x and the partial
+// sums of its squares are in shared memory, one after p and the partial sums of p.v are.
 template <int NN, typename T>
-__global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
+__global__ void __launch_bounds__(2 * NN) k_householder(const double* __restrict__ Min, i64 stride, T* __restrict__ ws) {
+  using HL = HhLayout<NN>;
+  constexpr int kCh = 16, kNc = NN / (2 * kCh), kWarps = 2 * NN / 32;
+  constexpr int kScrLd = kCh + 16 / (int)sizeof(T);             // padded chunk: 16-byte aligned, spreads the banks
+  constexpr unsigned FULL = 0xffffffffu;
+  __shared__ __align__(16) T xs[2][NN];                         // x of two consecutive steps (zero at entries <= k)
+  __shared__ __align__(16) T ps[NN];                            // p (zero at entries <= k)
+  __shared__ __align__(16) T sqp[2][kWarps];                    // per-warp sums of x_i^2, i > k + 1
+  __shared__ __align__(16) T pvp[kWarps];                       // per-warp parts of p.v
+  __shared__ __align__(16) T scr[2 * NN * kScrLd];              // one chunk per thread: picks a column out of the registers
+  __shared__ T dd_s[NN], ee_s[NN], beta_s[NN];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = tid >> 1, h = tid & 1;
+  const double* Mi = Min + (i64)blockIdx.x * stride;
+  T* out = ws + (i64)blockIdx.x * HL::stride;
+
+  // load, symmetrise, scale to max |a_ij| = 1
+  T a[kNc * kCh];
+  T amax = T(0.0);
+#pragma unroll
+  for (int i = 0; i < kNc; ++i) {
+#pragma unroll
+    for (int t = 0; t < kCh; ++t) {
+      const int c = (2 * i + h) * kCh + t;
+      a[i * kCh + t] = T(0.5 * (Mi[row * NN + c] + Mi[c * NN + row]));
+      amax = fmax(amax, fabs(a[i * kCh + t]));
+    }
+  }
+  amax = warp_max(amax);
+  if (lane == 0) pvp[warp] = amax;
+  __syncthreads();
+  T scale = pvp[0];
+#pragma unroll
+  for (int wi = 1; wi < kWarps; ++wi) scale = fmax(scale, pvp[wi]);
+  if (!(scale > T(0.0)) || !(scale * T(0.0) == T(0.0))) {       // zero or non-finite: the caller's kernel handles it
+    if (tid == 0) out[HL::scale] = scale;
+    return;
+  }
+  const T inv_scale = T(1.0) / scale;
+#pragma unroll
+  for (int e = 0; e < kNc * kCh; ++e) a[e] *= inv_scale;
+  __syncthreads();                                              // pvp[] is reused below
+
+  // A[row][j] for a column j that is uniform over the CTA (zero for j >= NN): the thread of the row that owns the
+  // chunk of j copies it to shared memory, both threads of the row read entry j back
+  auto column = [&](int j) -> T {
+    const int ch = j >> 4, ip = ch >> 1, hp = ch & 1;
+#pragma unroll
+    for (int i = 0; i < kNc; ++i) {
+      if (i == ip && h == hp) {
+        T tmp[kCh];
+#pragma unroll
+        for (int t = 0; t < kCh; ++t) tmp[t] = a[i * kCh + t];
+        st_vec<T, kCh>(scr + tid * kScrLd, tmp);
+      }
+    }
+    __syncwarp();
+    const T val = j < NN ? scr[(2 * row + hp) * kScrLd + (j & 15)] : T(0.0);
+    __syncwarp();
+    return val;
+  };
+  // x of step kn from this row's entry c0 = A[row][kn]
+  T xk_row = T(0.0);
+  auto publish = [&](int kn, T c0) {
+    const T xr = row > kn ? c0 : T(0.0);
+    T sq = (row > kn + 1 && h == 0) ? c0 * c0 : T(0.0);
+#pragma unroll
+    for (int o = 2; o < 32; o <<= 1) sq += __shfl_xor_sync(FULL, sq, o);
+    if (h == 0) {
+      xs[kn & 1][row] = xr;
+      if (row == kn) dd_s[kn] = c0;                             // the diagonal entry is final once row kn leaves the block
+    }
+    if (lane == 0) sqp[kn & 1][warp] = sq;
+    xk_row = xr;
+  };
+  T col1 = column(1);                                           // A[row][k + 1] at the start of step k
+  publish(0, column(0));
+
+  for (int k = 0; k < NN - 2; ++k) {
+    const int kb = k & 1;
+    __syncthreads();                                            // x and its partial sums are in place
+    T below2 = sqp[kb][0];                                      // squares beyond the subdiagonal entry
+#pragma unroll
+    for (int wi = 1; wi < kWarps; ++wi) below2 += sqp[kb][wi];
+    const T x0 = xs[kb][k + 1];
+    if (!(below2 > T(0.0))) {                                   // uniform: already reduced, A stays as it is
+      if (tid == 0) { ee_s[k] = x0; beta_s[k] = T(0.0); }
+      if (h == 0) out[HL::v + k * NN + row] = T(0.0);
+      const T c0 = col1;
+      col1 = column(k + 2);
+      publish(k + 1, c0);
+      continue;
+    }
+    const T alpha = sqrt(below2 + x0 * x0);
+    const T sa = x0 >= T(0.0) ? alpha : -alpha;
+    const T b = T(1.0) / (alpha * (alpha + fabs(x0)));
+    if (tid == 0) { ee_s[k] = -sa; beta_s[k] = b; }
+    const T v_row = xk_row + (row == k + 1 ? sa : T(0.0));      // zero in the rows <= k
+    if (h == 0) out[HL::v + k * NN + row] = v_row;
+    const bool warp_live = warp * 16 + 15 > k;                  // some row of this warp is in the trailing block
+    const T* xk = xs[kb];
+    T p_row = T(0.0);
+    if (warp_live) {
+      T acc[4] = {T(0.0), T(0.0), T(0.0), T(0.0)};
+#pragma unroll
+      for (int i = 0; i < kNc; ++i) {
+        T xv[kCh];
+        ld_vec<T, kCh>(xk + (2 * i + h) * kCh, xv);
+#pragma unroll
+        for (int t = 0; t < kCh; ++t) acc[t & 3] = fma(a[i * kCh + t], xv[t], acc[t & 3]);
+      }
+      T s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      s += __shfl_xor_sync(FULL, s, 1);
+      p_row = row > k ? b * fma(sa, col1, s) : T(0.0);          // x holds x_0 where v holds x_0 + sa: add sa A[row][k+1]
+      T pv = h == 0 ? p_row * v_row : T(0.0);
+#pragma unroll
+      for (int o = 2; o < 32; o <<= 1) pv += __shfl_xor_sync(FULL, pv, o);
+      if (lane == 0) pvp[warp] = pv;
+    } else if (lane == 0) {
+      pvp[warp] = T(0.0);
+    }
+    if (h == 0) ps[row] = p_row;
+    __syncthreads();                                            // p and the parts of p.v are in place
+    T c0 = col1;                                                // becomes A[row][k + 1] after the update
+    if (warp_live) {
+      T pvs = pvp[0];
+#pragma unroll
+      for (int wi = 1; wi < kWarps; ++wi) pvs += pvp[wi];
+      const T hb = T(0.5) * b * pvs;
+      const T w_row = p_row - hb * v_row;
+      // a - v_row (p_c - hb v_c) - w_row v_c = a - v_row p_c + (v_row hb - w_row) v_c, with x in the place of v: the
+      // entry of column k + 1, where the two differ, is never read from the registers again
+      const T g = v_row * hb - w_row, nv = -v_row;
+#pragma unroll
+      for (int i = 0; i < kNc; ++i) {
+        T xv[kCh], pc[kCh];
+        ld_vec<T, kCh>(xk + (2 * i + h) * kCh, xv);
+        ld_vec<T, kCh>(ps + (2 * i + h) * kCh, pc);
+#pragma unroll
+        for (int t = 0; t < kCh; ++t) a[i * kCh + t] = fma(g, xv[t], fma(nv, pc[t], a[i * kCh + t]));
+      }
+      const T vk1 = x0 + sa, wk1 = ps[k + 1] - hb * vk1;        // column k + 1 from its value before the update
+      c0 = col1 - (v_row * wk1 + w_row * vk1);
+    }
+    col1 = column(k + 2);
+    publish(k + 1, c0);
+  }
+  // the last 2 x 2 block: subdiagonal entry and last diagonal entry from row NN - 1
+  if (row == NN - 1 && h == 0) { ee_s[NN - 2] = xk_row; dd_s[NN - 1] = col1; }
+  if (tid == 0) { ee_s[NN - 1] = T(0.0); beta_s[NN - 2] = T(0.0); beta_s[NN - 1] = T(0.0); out[HL::scale] = scale; }
+  __syncthreads();
+  if (tid < NN) { out[HL::dd + tid] = dd_s[tid]; out[HL::ee + tid] = ee_s[tid]; out[HL::beta + tid] = beta_s[tid]; }
+}
+
+template <int NN, typename T>
+__global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict__ ws, int r, int scale_mode,
                                                              float* __restrict__ Fout, double* __restrict__ lam_out) {
   using S = EigSmem<NN, T>;
   constexpr int LD = S::LD;
-  constexpr int kPer = NN / kTpr, kSeg = kPer + S::kPad;       // padded position of entry c: c + (c / kPer) * kPad
   auto pos = [](int c) { return c + (c / (NN / kTpr)) * (16 / (int)sizeof(T)); };
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* A = reinterpret_cast<T*>(smem_raw + S::a);
@@ -150,135 +320,21 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const double* __res
   int* cstart = reinterpret_cast<int*>(smem_raw + S::cst);
   int* flags = cstart + kEigMaxR;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const double* Mi = Min + (i64)blockIdx.x * stride;
   float* Fo = Fout + (i64)blockIdx.x * NN * r;
   int turn = 0;
 
-  // ---- load, symmetrise, scale to max |a_ij| = 1 ---------------------------------------------------
-  // The matrix lives in registers during the reduction: thread (row, h) owns A[row][kPer h .. kPer h + kPer).
-  const int row = tid / kTpr, h = tid % kTpr;
-  const bool owner = row < NN;
-  T a[kPer];
-  T amax = T(0.0);
-#pragma unroll
-  for (int t = 0; t < kPer; ++t) {
-    const int c = kPer * h + t;
-    a[t] = owner ? T(0.5 * (Mi[row * NN + c] + Mi[c * NN + row])) : T(0.0);
-    amax = fmax(amax, fabs(a[t]));
-  }
-  const T scale = cta_max(amax, red, turn);
+  // ---- 1. the tridiagonal form and the reflectors come from k_householder -----------------------------------
+  using HL = HhLayout<NN>;
+  const T* hh = ws + (i64)blockIdx.x * HL::stride;
+  const T scale = hh[HL::scale];
   if (!(scale > T(0.0)) || !(scale * T(0.0) == T(0.0))) {
     // zero matrix: eigenvalues 0, unit vectors; anything non-finite is left to the error checks downstream
     for (int e = tid; e < NN * r; e += kEigThreads) Fo[e] = (scale_mode == 1 && e / r == e % r) ? 1.f : 0.f;
     if (lam_out) for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = 0.0;
     return;
   }
-  const T inv_scale = T(1.0) / scale;
-#pragma unroll
-  for (int t = 0; t < kPer; ++t) a[t] *= inv_scale;
-
-  // ---- 1. Householder tridiagonalisation ----------------------------------------------------------------
-  // Step k: x = A[k][k+1..] (row k = column k by symmetry) goes to shared memory; v = x + sgn alpha e_1;
-  // p = b A22 v; w = p - (b/2)(p.v) v; A22 <- A22 - v w^T - w v^T.  Two barriers per step: the sums over
-  // x and over p are formed redundantly by every warp from shared memory.
-  T* scal = lam;                                                // step scalars {reduce?, v_0, b, sgn alpha}; lam[] is free until step 2
-  T* pvpart = red;                                              // [32] per-warp parts of p.v (red[] is idle inside the loop)
-  for (int k = 0; k < NN - 2; ++k) {
-    T* xk = A + k * LD;                                         // raw x in row k of the reflector store
-    T* pk = pbuf + (k & 1) * LD;
-    if (warp == (k * kTpr) / 32) {
-      // the eight threads that own row k publish it together with the scalars of the reflector
-      T part = T(0.0), x0p = T(0.0);
-      if (row == k) {
-        // v is published with zeros at the columns <= k: the loops below then need no column tests (a product with an
-        // exact zero leaves a sum as it is)
-        T xz[kPer];
-#pragma unroll
-        for (int t = 0; t < kPer; ++t) {
-          const int c = kPer * h + t;
-          xz[t] = c > k ? a[t] : T(0.0);
-          part = c > k + 1 ? fma(a[t], a[t], part) : part;
-          x0p = c == k + 1 ? a[t] : x0p;
-        }
-        st_vec<T, kPer>(xk + kSeg * h, xz);
-      }
-#pragma unroll
-      for (int o = 1; o < kTpr; o <<= 1) {
-        part += __shfl_xor_sync(0xffffffffu, part, o);
-        x0p += __shfl_xor_sync(0xffffffffu, x0p, o);
-      }
-      __syncwarp();
-      if (row == k && h == 0) {
-        const T below2 = part, x0 = x0p;                        // squares beyond the subdiagonal entry
-        // p of the rows that have just left the trailing block reads as zero from now on (this buffer was last read
-        // two steps ago; live rows write their entries after the barrier)
-        pk[pos(k)] = T(0.0);
-        if (k > 0) pk[pos(k - 1)] = T(0.0);
-        if (below2 > T(0.0)) {
-          const T alpha = sqrt(below2 + x0 * x0);
-          const T sa = x0 >= T(0.0) ? alpha : -alpha;
-          scal[0] = T(1.0); scal[1] = x0 + sa; scal[2] = T(1.0) / (alpha * (alpha + fabs(x0))); scal[3] = sa;
-          xk[pos(k + 1)] = x0 + sa;                             // first entry of v (the stored row is the reflector)
-          ee[k] = -sa; beta[k] = scal[2]; e2[k] = sa;           // e2[] is free until the bisection
-        } else {
-          scal[0] = T(0.0);
-          ee[k] = x0; beta[k] = T(0.0); e2[k] = T(0.0);         // already reduced
-        }
-      }
-    }
-    __syncthreads();
-    if (scal[0] == T(0.0)) continue;                            // uniform
-    const T v0 = scal[1], b = scal[2];
-    const bool live = owner && row > k;
-    const bool warp_live = (warp * 32 + 31) / kTpr > k && warp * 32 / kTpr < NN;   // some row of this warp is live
-    T p_row = T(0.0);
-    if (warp_live) {
-      T acc = T(0.0);
-      if (live && kPer * h + kPer - 1 > k) {                   // some column of this thread is in the trailing block
-        T xv[kPer];
-        ld_vec<T, kPer>(xk + kSeg * h, xv);
-#pragma unroll
-        for (int t = 0; t < kPer; ++t) acc = fma(a[t], xv[t], acc);
-      }
-#pragma unroll
-      for (int o = 1; o < kTpr; o <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      p_row = b * acc;
-      if (live && h == 0) pk[pos(row)] = p_row;
-      // this warp's part of p.v (rows of the warp, one lane per row)
-      T pvw = (live && h == 0) ? p_row * xk[pos(row)] : T(0.0);
-#pragma unroll
-      for (int o = kTpr; o < 32; o <<= 1) pvw += __shfl_xor_sync(0xffffffffu, pvw, o);
-      if (lane == 0) pvpart[warp] = pvw;
-    } else if (lane == 0) {
-      pvpart[warp] = T(0.0);
-    }
-    __syncthreads();
-    if (!warp_live) continue;                                   // nothing left to update in this warp's rows
-    const T hb = T(0.5) * b * warp_sum(pvpart[lane]);
-    if (live && kPer * h + kPer - 1 > k) {
-      const T v_row = xk[pos(row)];
-      const T w_row = p_row - hb * v_row;
-      T xv[kPer], pv[kPer];
-      ld_vec<T, kPer>(xk + kSeg * h, xv);
-      ld_vec<T, kPer>(pk + kSeg * h, pv);
-#pragma unroll
-      for (int t = 0; t < kPer; ++t) {
-        const T wc = pv[t] - hb * xv[t];                        // zero at the columns <= k (v and p are zero there)
-        a[t] = a[t] - (v_row * wc + w_row * xv[t]);
-      }
-    }
-  }
-  __syncthreads();
-  // diagonal and last off-diagonal from the registers; first entries of the reflectors
-  if (owner) {
-#pragma unroll
-    for (int t = 0; t < kPer; ++t) {
-      const int c = kPer * h + t;
-      if (c == row) dd[row] = a[t];
-      if (row == NN - 1 && c == NN - 2) ee[NN - 2] = a[t];
-    }
-  }
-  if (tid == 0) { ee[NN - 1] = T(0.0); beta[NN - 2] = T(0.0); beta[NN - 1] = T(0.0); }
+  for (int e = tid; e < (NN - 2) * NN; e += kEigThreads) A[(e / NN) * LD + pos(e % NN)] = hh[HL::v + e];
+  if (tid < NN) { dd[tid] = hh[HL::dd + tid]; ee[tid] = hh[HL::ee + tid]; beta[tid] = hh[HL::beta + tid]; }
   __syncthreads();
   if (tid < NN) e2[tid] = ee[tid] * ee[tid];
   T g = T(0.0);
@@ -628,13 +684,20 @@ cudaError_t init_eigen() {
   return cudaFuncSetAttribute(k_jacobi_eig_f64<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jacobi64_smem(64));
 }
 
+size_t eig_scratch_doubles(int batch, int n) { return (size_t)batch * ((size_t)n * n + 3 * n + 4); }
+
 // Min: `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart; r <= 64 leading pairs.
 // scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda) (feature map of Section 4.1);
 // 1: orthonormal columns (basis of Eq. 9).  precise: float64 arithmetic.  Fout [batch][n][r];
-// lam_out [batch][n] or null (entries >= r are 0).
+// lam_out [batch][n] or null (entries >= r are 0).  ws: eig_scratch_doubles(batch, n) doubles.
 void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
-                    double* lam_out, cudaStream_t st) {
-#define SPR_EIG(NN, TT) k_eig_tridiag<NN, TT><<<batch, kEigThreads, EigSmem<NN, TT>::total, st>>>(Min, stride, r, scale_mode, Fout, lam_out)
+                    double* lam_out, double* ws, cudaStream_t st) {
+#define SPR_EIG(NN, TT)                                                                                        \
+  do {                                                                                                         \
+    k_householder<NN, TT><<<batch, 2 * NN, 0, st>>>(Min, stride, reinterpret_cast<TT*>(ws));                   \
+    k_eig_tridiag<NN, TT><<<batch, kEigThreads, EigSmem<NN, TT>::total, st>>>(reinterpret_cast<const TT*>(ws), r, \
+                                                                            scale_mode, Fout, lam_out);       \
+  } while (0)
   if (n == 128) {
     if (precise) SPR_EIG(128, double); else SPR_EIG(128, float);
     k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);

@@ -263,7 +263,7 @@ void launch_fit(const FitArgs& a, cudaStream_t st) {
     k_fit_solve<float><<<a.BH, 1024, (size_t)d * (d + 1) * 4, st>>>(a);
   }
   // Psi_r: leading eigenvectors of S = Rb^T W Rb, i.e. right singular vectors of W^(1/2) Rb.
-  if (!a.full_rank) launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, st);
+  if (!a.full_rank) launch_eig_top(a.scratch + L.S, (i64)L.total, a.BH, d, r, 1, a.precise, a.Psi, nullptr, a.eig_ws, st);
   k_fit_compose<<<a.BH, 256, 0, st>>>(a, r);
 }
 

@@ -15,10 +15,11 @@ void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, 
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
 // eigen.cu: leading r <= 64 eigenpairs of `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart.
 // scale_mode 0: columns scaled by sqrt(lambda_j / mean retained lambda); 1: orthonormal columns; precise: float64.
-// Fout [batch][n][r]; lam_out [batch][n] or null.
+// Fout [batch][n][r]; lam_out [batch][n] or null; ws: eig_scratch_doubles(batch, n) doubles of scratch.
 cudaError_t init_eigen();
+size_t eig_scratch_doubles(int batch, int n);
 void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int scale_mode, bool precise, float* Fout,
-                    double* lam_out, cudaStream_t st);
+                    double* lam_out, double* ws, cudaStream_t st);
 void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, int r, const float* F,
                     bool rms, float eps, float* phi, int ldphi, unsigned* maxabs, int* err, cudaStream_t st);
 // features of the semantic partition: the activations themselves as float32 rows [BH][N][d]
@@ -156,6 +157,7 @@ struct FitArgs {
   bool precise;                        // float64 eigen-solver for the subspace
   const float *X, *Dn, *w;             // [BH][M][d], [BH][M][d], [BH][M]
   double* scratch;                     // see fit_scratch_doubles
+  double* eig_ws;                      // eig_scratch_doubles(BH, d) doubles
   float *A, *c;                        // outputs [BH][d][d], [BH][d]
   float* Psi;                          // [BH][d][r] scratch
   int* err;
