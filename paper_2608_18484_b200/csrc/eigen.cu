@@ -39,14 +39,14 @@ __device__ __forceinline__ float hash_unit(int i, int j) {         // determinis
 // dominate the run time of the whole plan.
 template <typename T> struct EigNum;
 template <> struct EigNum<double> {
-  static constexpr double pivot = 1.0e-15, res_tol = 1.0e-7, orth_tol = 1.0e-7, group_gap = 1.0e-3;
-  static constexpr double big = 1.0e90, small = 1.0e-90;
-  static constexpr int rescale_mask = 7, passes = 20;
+  static constexpr double pivot = 1.0e-15, res_tol = 1.0e-7, orth_tol = 1.0e-7, group_gap = 1.0e-8, polish_tol = 1.0e-12;
+  static constexpr double e2_min = 1.0e-280;
+  static constexpr int passes = 15;
 };
 template <> struct EigNum<float> {
-  static constexpr float pivot = 1.0e-7f, res_tol = 1.0e-4f, orth_tol = 1.0e-3f, group_gap = 1.0e-2f;
-  static constexpr float big = 1.0e15f, small = 1.0e-15f;
-  static constexpr int rescale_mask = 0, passes = 12;
+  static constexpr float pivot = 1.0e-7f, res_tol = 1.0e-4f, orth_tol = 1.0e-3f, group_gap = 1.0e-5f, polish_tol = 1.0e-5f;
+  static constexpr float e2_min = 1.0e-30f;
+  static constexpr int passes = 9;
 };
 
 // kN consecutive elements (a multiple of 16 bytes, 16-byte aligned) between shared memory and registers
@@ -91,13 +91,27 @@ template <typename T> __device__ __forceinline__ T cta_max(T v, T* red, int& tur
   return warp_max(buf[threadIdx.x & 31]);
 }
 
+constexpr size_t cmax3(size_t x, size_t y, size_t w) { return x > y ? (x > w ? x : w) : (y > w ? y : w); }
+
 template <int NN, typename T> struct EigSmem {
   // a vector of NN entries is stored as kTpr segments of NN / kTpr entries, each followed by 16 bytes of
   // padding: the eight threads of a row then read their segments with conflict-free 16-byte accesses
   static constexpr int kPad = 16 / (int)sizeof(T);
   static constexpr int LD = NN + kTpr * kPad;
-  static constexpr size_t a = 0;                                           // T [NN][LD]: reflector k in row k
-  static constexpr size_t z = a + sizeof(T) * NN * LD;                     // T [NN][kZld]
+  // The factors of the inverse iteration (four numbers per row and vector) share the space of the reflectors, which
+  // are fetched only for the back-transformation; float64 at n = 128 has no room for them (they stay in local memory).
+  static constexpr size_t fac_bytes = sizeof(T) * 4 * NN * kEigMaxR;
+  static constexpr bool fac_in_smem = fac_bytes <= 131072;
+  static constexpr size_t a_bytes = sizeof(T) * NN * LD;
+  // One region serves in turn the factors, the partial Gram matrices of the polish step ([4][64][64]) and the
+  // reflectors.  Where the reflectors fit behind the Gram matrices they are fetched asynchronously while the polish
+  // step runs (a_off > 0); otherwise they are fetched right before the back-transformation.
+  static constexpr size_t g_bytes = sizeof(T) * 4 * 64 * 64;
+  static constexpr size_t rest = sizeof(T) * (NN * kZld + 2 * LD + 6 * NN + kEigMaxR + 64) + sizeof(int) * (kEigMaxR + 4);
+  static constexpr size_t a_off = g_bytes + a_bytes + rest <= 227 * 1024 ? g_bytes : 0;
+  static constexpr size_t a = 0;                                           // region start
+  static constexpr size_t region = cmax3(fac_in_smem ? fac_bytes : 0, a_off + a_bytes, g_bytes);
+  static constexpr size_t z = a + region;                                  // T [NN][kZld]
   static constexpr size_t pb = z + sizeof(T) * NN * kZld;                  // T [2][LD]: p of two consecutive steps
   static constexpr size_t vec = pb + sizeof(T) * 2 * LD;                   // (2 spare), d, e, e2, beta: 6 x T[NN]
   static constexpr size_t lam = vec + sizeof(T) * 6 * NN;             // T [kEigMaxR]
@@ -106,27 +120,26 @@ template <int NN, typename T> struct EigSmem {
   static constexpr size_t total = cst + sizeof(int) * (kEigMaxR + 4);
 };
 
-// eigenvalues of T below x (Sturm count) by the three-term recurrence of the leading principal
-// minors, p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}: one dependent multiply-add per step.  A zero
-// minor takes the sign opposite to its predecessor; both running minors are rescaled by a positive
-// factor when they leave a safe range, which changes no sign.
+// Reciprocal on the dependent chains of the Sturm count and of the factorisation: float32 takes the hardware
+// approximation (the chains are perturbed at the level of their own rounding), float64 the division.
+__device__ __forceinline__ float chain_rcp(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ double chain_rcp(double x) { return 1.0 / x; }
+
+// eigenvalues of T below x (Sturm count): the pivots q_i = (d_i - x) - e_{i-1}^2 / q_{i-1} of the factorisation
+// T - x I = L D L^T, one negative pivot per eigenvalue below x.  A zero pivot needs no test: its reciprocal is an
+// infinity, the next pivot -infinity (counted; e2[] is kept strictly positive for this), whose reciprocal is zero.
 template <int NN, typename T>
 __device__ __forceinline__ int sturm_count(const T* __restrict__ dd, const T* __restrict__ e2, T x) {
-  T p2 = T(1.0), p1 = dd[0] - x;
-  bool neg1 = p1 < T(0.0) || p1 == T(0.0);                            // sign of p_1 (zero counts as a change from p_0 = 1)
-  int cnt = neg1;
+  T q = dd[0] - x;
+  int cnt = q < T(0.0);
 #pragma unroll 8
   for (int i = 1; i < NN; ++i) {
-    const T p = fma(dd[i] - x, p1, -(e2[i - 1] * p2));
-    const bool neg = p == T(0.0) ? !neg1 : p < T(0.0);
-    cnt += neg != neg1;
-    neg1 = neg;
-    p2 = p1; p1 = p;
-    if ((i & EigNum<T>::rescale_mask) == EigNum<T>::rescale_mask) {
-      const T mx = fmax(fabs(p1), fabs(p2));
-      if (mx > EigNum<T>::big) { p1 *= EigNum<T>::small; p2 *= EigNum<T>::small; }
-      else if (mx < EigNum<T>::small) { p1 *= EigNum<T>::big; p2 *= EigNum<T>::big; }
-    }
+    q = fma(-e2[i - 1], chain_rcp(q), dd[i] - x);
+    cnt += q < T(0.0);
   }
   return cnt;
 }
@@ -306,7 +319,7 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
   constexpr int LD = S::LD;
   auto pos = [](int c) { return c + (c / (NN / kTpr)) * (16 / (int)sizeof(T)); };
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* A = reinterpret_cast<T*>(smem_raw + S::a);
+  T* A = reinterpret_cast<T*>(smem_raw + S::a + S::a_off);      // T [NN][LD]: reflector k in row k
   T* pbuf = reinterpret_cast<T*>(smem_raw + S::pb);
   T* Z = reinterpret_cast<T*>(smem_raw + S::z);
   T* v = reinterpret_cast<T*>(smem_raw + S::vec);
@@ -333,31 +346,35 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
     if (lam_out) for (int j = tid; j < NN; j += kEigThreads) lam_out[(i64)blockIdx.x * NN + j] = 0.0;
     return;
   }
-  for (int e = tid; e < (NN - 2) * NN; e += kEigThreads) A[(e / NN) * LD + pos(e % NN)] = hh[HL::v + e];
   if (tid < NN) { dd[tid] = hh[HL::dd + tid]; ee[tid] = hh[HL::ee + tid]; beta[tid] = hh[HL::beta + tid]; }
   __syncthreads();
-  if (tid < NN) e2[tid] = ee[tid] * ee[tid];
+  if (tid < NN) e2[tid] = fmax(ee[tid] * ee[tid], EigNum<T>::e2_min);   // strictly positive: see sturm_count
   T g = T(0.0);
   if (tid < NN) g = fabs(dd[tid]) + fabs(ee[tid]) + (tid > 0 ? fabs(ee[tid - 1]) : T(0.0));
   const T tnorm = cta_max(g, red, turn);                   // Gershgorin bound on |lambda|; also makes e2[] visible
 
-  // ---- 2. multi-section: 4 threads per eigenvalue, 5-fold interval reduction per pass -----------------
-  if (tid < 4 * kEigMaxR) {                                     // whole warps: 8 eigenvalues per warp
-    const int j = tid >> 2, t = tid & 3;                        // eigenvalue (j+1)-th largest, probe point t
-    const bool active = j < r;
-    const int kth = NN - 1 - j;                                 // ascending index
-    T lo = -tnorm, hi = tnorm;
-    for (int it = 0; it < EigNum<T>::passes; ++it) {
-      const T wdt = (hi - lo) * T(0.2);
-      const T x = lo + wdt * (T)(t + 1);
-      const bool below = active && sturm_count<NN, T>(dd, e2, x) <= kth;   // eigenvalue kth is >= x
-      const unsigned bal = __ballot_sync(0xffffffffu, below);
-      const int s = __popc((bal >> (lane & 28)) & 0xFu);        // probes of this group of 4 lanes still below the eigenvalue
-      const T nlo = lo + wdt * (T)s;
-      hi = s < 4 ? lo + wdt * (T)(s + 1) : hi;
-      lo = nlo;
+  // ---- 2. multi-section: 8 threads per eigenvalue, 9-fold interval reduction per pass -----------------
+  // (the Sturm count is a chain of dependent reciprocals and multiply-adds: 16 warps of such chains keep the
+  // schedulers busy, more probes per eigenvalue would only queue)
+  {
+    constexpr int kProbes = 8;
+    if (tid < kProbes * kEigMaxR) {                             // whole warps: 4 eigenvalues per warp
+      const int j = tid / kProbes, t = tid % kProbes;           // eigenvalue (j+1)-th largest, probe point t
+      const bool active = j < r;
+      const int kth = NN - 1 - j;                               // ascending index
+      T lo = -tnorm, hi = tnorm;
+      for (int it = 0; it < EigNum<T>::passes; ++it) {
+        const T wdt = (hi - lo) * (T(1.0) / T(kProbes + 1));
+        const T x = lo + wdt * (T)(t + 1);
+        const bool below = active && sturm_count<NN, T>(dd, e2, x) <= kth;   // eigenvalue kth is >= x
+        const unsigned bal = __ballot_sync(0xffffffffu, below);
+        const int s = __popc((bal >> (lane & ~(kProbes - 1))) & ((1u << kProbes) - 1u));   // probes of this group still below the eigenvalue
+        const T nlo = lo + wdt * (T)s;
+        hi = s < kProbes ? lo + wdt * (T)(s + 1) : hi;
+        lo = nlo;
+      }
+      if (active && t == 0) lam[j] = T(0.5) * (lo + hi);
     }
-    if (active && t == 0) lam[j] = T(0.5) * (lo + hi);
   }
   __syncthreads();
 
@@ -365,57 +382,110 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
   if (tid < r) {
     const T shift = lam[tid];
     const T tiny = tnorm * EigNum<T>::pivot;
-    T pinv[NN], u1[NN], u2[NN], mul[NN];                  // pivots^-1, two superdiagonals of U, multipliers
-    unsigned long long swp[(NN + 63) / 64];
-#pragma unroll
-    for (int q = 0; q < (NN + 63) / 64; ++q) swp[q] = 0ull;
+    // per row of U: 1 / pivot, the two superdiagonal entries times 1 / pivot, and the multiplier of the elimination
+    struct alignas(16) Fac { T ip, u1, u2, m; };
+    constexpr int fs = S::fac_in_smem ? kEigMaxR : 1;       // stride between consecutive rows of one vector's factors
+    Fac fac_local[S::fac_in_smem ? 1 : NN];
+    Fac* fac = fac_local;
+    if constexpr (S::fac_in_smem) fac = reinterpret_cast<Fac*>(smem_raw + S::a) + tid;
+    unsigned swp[NN / 32];                                  // bit i: rows i and i + 1 were swapped
     T acur = dd[0] - shift, ucur = ee[0];                 // current row i: diagonal and superdiagonal entries
-    for (int i = 0; i < NN - 1; ++i) {
-      const T sub = ee[i];
-      const T anext = dd[i + 1] - shift, unext = ee[i + 1];   // ee[NN-1] = 0
-      if (fabs(acur) >= fabs(sub)) {
-        T piv = acur;
-        if (fabs(piv) <= tiny) piv = piv >= T(0.0) ? tiny : -tiny;
-        const T ip = T(1.0) / piv;
-        const T m = sub * ip;
-        pinv[i] = ip; u1[i] = ucur; u2[i] = T(0.0); mul[i] = m;
-        acur = anext - m * ucur;
-        ucur = unext;
-      } else {
-        const T ip = T(1.0) / sub;
-        const T m = acur * ip;                             // rows i and i+1 swapped
-        swp[i >> 6] |= 1ull << (i & 63);
-        pinv[i] = ip; u1[i] = anext; u2[i] = unext; mul[i] = m;
-        acur = ucur - m * anext;
-        ucur = -m * unext;
+#pragma unroll
+    for (int q = 0; q < NN / 32; ++q) {
+      unsigned w = 0u;
+      for (int b0 = 0; b0 < 32; b0 += 4) {
+        // rows i0 .. i0 + 3 (row NN - 1 has no successor: its step is masked out); operands first, then the chain
+        const int i0 = 32 * q + b0;
+        T dv[4], ev[5];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) dv[u] = i0 + u + 1 < NN ? dd[i0 + u + 1] : T(0.0);
+#pragma unroll
+        for (int u = 0; u < 5; ++u) ev[u] = i0 + u < NN ? ee[i0 + u] : T(0.0);
+        Fac fo[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          // row i against row i + 1 = (sub, anext, unext): the larger leading entry becomes the pivot; both cases run
+          // the same instructions (selects), so the lanes of a warp stay together
+          const bool on = i0 + u < NN - 1;
+          const T sub = ev[u];
+          const T anext = dv[u] - shift, unext = ev[u + 1];       // ee[NN-1] = 0
+          const bool sw = !(fabs(acur) >= fabs(sub));
+          T piv = sw ? sub : acur;
+          if (fabs(piv) <= tiny) piv = piv >= T(0.0) ? tiny : -tiny;
+          const T ip = chain_rcp(piv);
+          const T m = (sw ? acur : sub) * ip;
+          w |= (unsigned)(sw && on) << (b0 + u);
+          fo[u] = Fac{ip, (sw ? anext : ucur) * ip, sw ? unext * ip : T(0.0), m};
+          const T top = sw ? ucur : anext, und = sw ? anext : ucur;
+          acur = on ? fma(-m, und, top) : acur;
+          ucur = on ? (sw ? -m * unext : unext) : ucur;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u < NN - 1) fac[(i0 + u) * fs] = fo[u];
       }
+      swp[q] = w;
     }
     {
       T piv = acur;
       if (fabs(piv) <= tiny) piv = piv >= T(0.0) ? tiny : -tiny;
-      pinv[NN - 1] = T(1.0) / piv; u1[NN - 1] = T(0.0); u2[NN - 1] = T(0.0); mul[NN - 1] = T(0.0);
+      fac[(NN - 1) * fs] = Fac{T(1.0) / piv, T(0.0), T(0.0), T(0.0)};
     }
     T* z = Z + tid;                                        // z_i = z[i * kZld]
     for (int i = 0; i < NN; ++i) z[i * kZld] = hash_unit(i, tid);
+    // Both sweeps run in blocks of four rows whose operands are fetched before the dependent chain starts (the
+    // compiler keeps every load behind the previous store to shared memory otherwise).
+    unsigned* swp_s = reinterpret_cast<unsigned*>(pbuf) + tid;      // [NN / 32][kEigMaxR]; pbuf is idle until step 4
+#pragma unroll
+    for (int q = 0; q < NN / 32; ++q) swp_s[q * kEigMaxR] = swp[q];
+    constexpr int kBlk = 4, kFull = (NN - 1) / kBlk * kBlk;        // rows 0 .. kFull - 1 in blocks, the rest one by one
     for (int it = 0; it < 3; ++it) {
       T zi = z[0];
-#pragma unroll 4
-      for (int i = 0; i < NN - 1; ++i) {                        // forward elimination
+      for (int i0 = 0; i0 < kFull; i0 += kBlk) {                    // forward elimination
+        T zn[kBlk], mm[kBlk], kp[kBlk];
+        const unsigned bits = swp_s[(i0 >> 5) * kEigMaxR] >> (i0 & 31);
+#pragma unroll
+        for (int u = 0; u < kBlk; ++u) { zn[u] = z[(i0 + u + 1) * kZld]; mm[u] = fac[(i0 + u) * fs].m; }
+#pragma unroll
+        for (int u = 0; u < kBlk; ++u) {
+          const bool sw = (bits >> u) & 1u;
+          kp[u] = sw ? zn[u] : zi;
+          zi = fma(-mm[u], kp[u], sw ? zi : zn[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kBlk; ++u) z[(i0 + u) * kZld] = kp[u];
+      }
+      for (int i = kFull; i < NN - 1; ++i) {
         const T zn = z[(i + 1) * kZld];
-        const bool sw = (swp[i >> 6] >> (i & 63)) & 1ull;
+        const bool sw = (swp_s[(i >> 5) * kEigMaxR] >> (i & 31)) & 1u;
         const T keep = sw ? zn : zi, other = sw ? zi : zn;
         z[i * kZld] = keep;
-        zi = fma(-mul[i], keep, other);
+        zi = fma(-fac[i * fs].m, keep, other);
       }
-      T z1 = zi * pinv[NN - 1], z2 = T(0.0);                  // back substitution
+      T z1 = zi * fac[(NN - 1) * fs].ip, z2 = T(0.0);                // back substitution
       z[(NN - 1) * kZld] = z1;
       T big = fabs(z1);
-#pragma unroll 4
-      for (int i = NN - 2; i >= 0; --i) {
-        const T zz = (z[i * kZld] - u1[i] * z1 - u2[i] * z2) * pinv[i];
+      for (int i = NN - 2; i >= kFull; --i) {
+        const Fac f = fac[i * fs];
+        const T zz = fma(-f.u1, z1, fma(-f.u2, z2, z[i * kZld] * f.ip));
         z[i * kZld] = zz;
         big = fmax(big, fabs(zz));
         z2 = z1; z1 = zz;
+      }
+      for (int i0 = kFull - kBlk; i0 >= 0; i0 -= kBlk) {
+        Fac f[kBlk];
+        T zv[kBlk];
+#pragma unroll
+        for (int u = 0; u < kBlk; ++u) { f[u] = fac[(i0 + u) * fs]; zv[u] = z[(i0 + u) * kZld] * f[u].ip; }
+#pragma unroll
+        for (int u = kBlk - 1; u >= 0; --u) {
+          const T zz = fma(-f[u].u1, z1, fma(-f[u].u2, z2, zv[u]));
+          zv[u] = zz;
+          big = fmax(big, fabs(zz));
+          z2 = z1; z1 = zz;
+        }
+#pragma unroll
+        for (int u = 0; u < kBlk; ++u) z[(i0 + u) * kZld] = zv[u];
       }
       const T sc = big > T(0.0) ? T(1.0) / big : T(1.0);
       for (int i = 0; i < NN; ++i) z[i * kZld] *= sc;
@@ -427,6 +497,16 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
   }
   __syncthreads();
 
+  if constexpr (S::a_off != 0) {
+    // the factors are dead: start fetching the reflectors (16 bytes per copy) for step 6
+    constexpr int kV = 16 / (int)sizeof(T);
+    for (int c = tid; c < (NN - 2) * NN / kV; c += kEigThreads) {
+      const int e = c * kV;
+      const unsigned dst = (unsigned)__cvta_generic_to_shared(A + (e / NN) * LD + pos(e % NN));
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(hh + HL::v + e) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
   // ---- 4. groups of close eigenvalues: Gram-Schmidt inside each group ---------------------------------
   if (tid == 0) {
     const T gap = EigNum<T>::group_gap * tnorm;
@@ -469,7 +549,82 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
     }
     j0 = j1 + 1;
   }
-  __syncthreads();
+  // Polish: outside those (rare) tight groups the vectors of close eigenvalues are orthogonal only to about
+  // eps ||T|| / gap.  One step Z <- Z (3 I - Z^T Z) / 2 squares the deviation of Z^T Z from the identity; steps are
+  // taken until it is below polish_tol (normally one), and a basis that does not get there is left to the fallback.
+  // Everything here is spread over the whole CTA, where the Gram-Schmidt loop above is sequential in the vectors.
+  for (int i = tid; i < NN * (kEigMaxR - r); i += kEigThreads)    // unused columns read as zero below
+    Z[(i / (kEigMaxR - r)) * kZld + r + i % (kEigMaxR - r)] = T(0.0);
+  T* Gs = reinterpret_cast<T*>(smem_raw + S::a);                   // [4][64][64]: partial Gram matrices, then W
+  bool polished = false;
+  for (int step = 0; step < 4 && !polished; ++step) {
+    {
+      // Z^T Z in 4 x 4 tiles; the rows of Z are split over the four quarters of the CTA
+      const int quarter = tid >> 8, t = tid & 255, a0 = 4 * (t >> 4), b0 = 4 * (t & 15);
+      T acc[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = T(0.0);
+      if (a0 < r && b0 < r) {
+        for (int i = quarter * (NN / 4); i < (quarter + 1) * (NN / 4); ++i) {
+          T za[4], zb[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) { za[u] = Z[i * kZld + a0 + u]; zb[u] = Z[i * kZld + b0 + u]; }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] = fma(za[u], zb[v], acc[u][v]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) Gs[quarter * 4096 + (a0 + u) * 64 + b0 + v] = acc[u][v];
+      if (tid == 0) flags[1] = 0;
+    }
+    __syncthreads();
+    {
+      // sum of the four parts; W = (3 I - G) / 2 takes the place of G
+      T dev = T(0.0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int e = 4 * tid + q, row = e >> 6, col = e & 63;
+        const T g = (Gs[e] + Gs[4096 + e]) + (Gs[8192 + e] + Gs[12288 + e]);
+        const T id = row == col ? T(1.0) : T(0.0);
+        if (row < r && col < r) dev = fmax(dev, fabs(g - id));
+        Gs[e] = T(1.5) * id - T(0.5) * g;
+      }
+      if (!(dev <= EigNum<T>::polish_tol)) flags[1] = 1;
+    }
+    __syncthreads();
+    polished = flags[1] == 0;                                      // uniform
+    if (!polished && step < 3) {
+      const int i0 = 2 * (tid >> 4), j0 = 4 * (tid & 15);
+      T o[2][4];
+#pragma unroll
+      for (int u = 0; u < 2; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) o[u][v] = T(0.0);
+      if (i0 < NN) {
+        for (int bq = 0; bq < r; ++bq) {
+          const T z0 = Z[i0 * kZld + bq], z1 = Z[(i0 + 1) * kZld + bq];
+          T wv[4];
+          ld_vec<T, 4>(Gs + bq * 64 + j0, wv);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) { o[0][v] = fma(z0, wv[v], o[0][v]); o[1][v] = fma(z1, wv[v], o[1][v]); }
+        }
+      }
+      __syncthreads();
+      if (i0 < NN) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+          for (int v = 0; v < 4; ++v) Z[(i0 + u) * kZld + j0 + v] = o[u][v];
+      }
+      __syncthreads();
+    }
+  }
 
   // ---- 5. Rayleigh quotients, residuals, orthogonality -------------------------------------------------
   bool bad = false;
@@ -496,17 +651,7 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
     lam[tid] = rq;
     bad = !(res <= EigNum<T>::res_tol * tnorm) || !(fabs(den - T(1.0)) <= EigNum<T>::orth_tol);
   }
-  for (int pr = tid; pr < r * r; pr += kEigThreads) {
-    const int a = pr / r, bq = pr % r;
-    if (a < bq) {
-      T d0 = T(0.0), d1 = T(0.0);
-      for (int i = 0; i < NN; i += 2) {
-        d0 = fma(Z[i * kZld + a], Z[i * kZld + bq], d0);
-        d1 = fma(Z[(i + 1) * kZld + a], Z[(i + 1) * kZld + bq], d1);
-      }
-      bad |= !(fabs(d0 + d1) <= EigNum<T>::orth_tol);
-    }
-  }
+  bad |= !polished;                                             // all pairwise inner products were checked above
   if (bad) flags[0] = 1;
   __syncthreads();
   if (flags[0]) {
@@ -515,36 +660,48 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
   }
 
   // ---- 6. back-transformation z <- H_0 ... H_{n-3} z, scaling, output -------------------------------------
+  if constexpr (S::a_off != 0) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else {
+    for (int e = tid; e < (NN - 2) * NN; e += kEigThreads) A[(e / NN) * LD + pos(e % NN)] = hh[HL::v + e];
+  }
+  __syncthreads();
   {
     constexpr int tpv = 16;                                      // threads per vector (1024 threads cover 64 vectors)
     constexpr int npt = NN / tpv;                                // entries of the vector per thread, kept in registers
     const int j = tid / tpv, q = tid % tpv;
-    const bool active = j < r;
-    T zr[npt];
+    // thread q holds entries i = q, q + 16, ...; the reflector is stored with exact zeros up to entry k, so no entry
+    // needs a test.  The reflector of the next step is fetched while the sum of the current one travels through the
+    // shuffles.
+    if ((tid >> 5) * (32 / tpv) < r) {                           // whole warps (two vectors each)
+      const bool active = j < r;
+      T zr[npt];
 #pragma unroll
-    for (int t = 0; t < npt; ++t) zr[t] = active ? Z[(q + tpv * t) * kZld + j] : T(0.0);
-    for (int k = NN - 3; k >= 0; --k) {
-      const T bk = beta[k];
-      if (bk == T(0.0)) continue;                                   // uniform
-      // thread q holds entries i = q, q + 16, ...; the reflector is zero up to entry k
-      T av[npt];
+      for (int t = 0; t < npt; ++t) zr[t] = active ? Z[(q + tpv * t) * kZld + j] : T(0.0);
+      T av[npt], an[npt];
+      T bk = beta[NN - 3];
 #pragma unroll
-      for (int t = 0; t < npt; ++t) {
-        const int i = q + tpv * t;
-        av[t] = i > k ? A[k * LD + pos(i)] : T(0.0);
+      for (int t = 0; t < npt; ++t) av[t] = A[(NN - 3) * LD + pos(q + tpv * t)];
+      for (int k = NN - 3; k >= 0; --k) {
+        const int kn = k > 0 ? k - 1 : 0;
+        const T bn = beta[kn];
+#pragma unroll
+        for (int t = 0; t < npt; ++t) an[t] = A[kn * LD + pos(q + tpv * t)];
+        T d0 = T(0.0), d1 = T(0.0);
+#pragma unroll
+        for (int t = 0; t < npt; t += 2) { d0 = fma(av[t], zr[t], d0); d1 = fma(av[t + 1], zr[t + 1], d1); }
+        T dot = d0 + d1;
+#pragma unroll
+        for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        const T f = bk * dot;                                        // b_k = 0 marks a step without reflector
+#pragma unroll
+        for (int t = 0; t < npt; ++t) { zr[t] = fma(-f, av[t], zr[t]); av[t] = an[t]; }
+        bk = bn;
       }
-      T dot = T(0.0);
+      if (active) {
 #pragma unroll
-      for (int t = 0; t < npt; ++t) dot = fma(av[t], zr[t], dot);
-#pragma unroll
-      for (int o = 1; o < tpv; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      const T f = bk * dot;
-#pragma unroll
-      for (int t = 0; t < npt; ++t) zr[t] = fma(-f, av[t], zr[t]);
-    }
-    if (active) {
-#pragma unroll
-      for (int t = 0; t < npt; ++t) Z[(q + tpv * t) * kZld + j] = zr[t];
+        for (int t = 0; t < npt; ++t) Z[(q + tpv * t) * kZld + j] = zr[t];
+      }
     }
   }
   __syncthreads();
