@@ -108,14 +108,14 @@ def launches_per_call(T, fitted, tensor_path):
         kmeans = 2 + 1 + 2 * T + (T - 1)
     else:                # init, first norms, T assignments, T-1 updates
         kmeans = 2 + T + (T - 1)
-    # per side: Gram, eigen-solver + its marked-matrix fallback, projection (+ split of the feature map), k-means,
-    # sort + means; then probes; route; tile offsets + remainder rows
-    plan = 2 * (3 + (2 if tensor_path else 1) + kmeans + 2) + 2 + 2 + 3
+    # per side: Gram, eigen-solver (Householder, tridiagonal stage, marked-matrix fallback), projection (+ split of
+    # the feature map), k-means, sort + means; then probes; route; tile offsets + remainder rows
+    plan = 2 * (4 + (2 if tensor_path else 1) + kmeans + 2) + 2 + 2 + 3
     if not fitted:
         plan -= 2
     attend = 3 + 1 + (1 if tensor_path else 0)       # gathers, attention (+ the packed-remainder kernel)
     if fitted:
-        attend += (3 if tensor_path else 2) + 6 + 1  # probe rows (+gather) + merge, fit (eigen-solver: two launches), probe write
+        attend += (3 if tensor_path else 2) + 7 + 1  # probe rows (+gather) + merge, fit (eigen-solver: three launches), probe write
         attend += 2 if tensor_path else 0            # transposed correction matrix, correction pass
     return plan + attend
 
@@ -307,6 +307,8 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-groups", type=int, default=4,
+                    help="groups of heads the host-buffer call pipelines (upload, compute and download overlap)")
     ap.add_argument("--no-warm", action="store_true", help="skip the warm-started multi-call leg")
     ap.add_argument("--study", default="", choices=["", "sweep", "cq", "partition"],
                     help="parameter study instead of the benchmark line: density x probes x mode, or the C_q frontier")
@@ -457,21 +459,22 @@ def main():
     # ---- end to end through the host-buffer call ----
     e2e = None
     if not args.no_e2e:
-        bufs = [Qd, Kd, Vd]
+        bufs = [Qd, Kd, Vd, torch.empty_like(Qd)]
         for _ in range(2):
-            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs)
+            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs, groups=args.e2e_groups)
         barrier()
         n_e2e = max(1, min(args.steps, 5))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(n_e2e):
-            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs)
+            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs, groups=args.e2e_groups)
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1) / n_e2e
         e2e_ms = max_over_ranks(e2e_ms, dev, world)
         nbytes = Qd.numel() * Qd.element_size()
-        e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes}
+        e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
+               "head_groups": len(B.head_groups(wl.B if hasattr(wl, "B") else 1, wl.H, 1, args.e2e_groups))}
 
     if rank != 0:
         if world > 1:

@@ -105,6 +105,11 @@ typedef struct {
   uint64_t seed;         /* offsets the deterministic row samples */
   int32_t mode;          /* 0 = probe-fitted reconstruction, 1 = renormalised hard drop only */
   int32_t partition;     /* sparsepr_partition_t; 0 = Response-Coupled Partitioning */
+  int32_t head_offset;   /* The deterministic row samples (Appendix B.1: sampled queries; k-means initialisation) are keyed by
+                          * head_offset + b H + h.  A problem cut into groups of heads, each group a call of its own with the
+                          * index of its first head here, gives bit for bit the plan of one call over all heads (outputs agree up to
+                          * the summation order of the probe rows, whose key slices are sized per call).
+                          * >= 0 and a multiple of H / Hkv; 0 for a whole problem. */
 } sparsepr_params_t;
 
 typedef struct sparsepr_plan_s sparsepr_plan_t;

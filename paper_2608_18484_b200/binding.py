@@ -39,7 +39,7 @@ class Params(C.Structure):
                 ("n_sample", C.c_int32), ("n_probe", C.c_int32), ("rK", C.c_int32), ("rQ", C.c_int32),
                 ("r_out", C.c_int32), ("lam", C.c_float), ("eps_rms", C.c_float), ("eps_std", C.c_float),
                 ("kmeans_iters", C.c_int32), ("softmax_scale", C.c_float), ("seed", C.c_uint64), ("mode", C.c_int32),
-                ("partition", C.c_int32)]
+                ("partition", C.c_int32), ("head_offset", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -154,8 +154,9 @@ def make_shape(Q, K, V, O) -> Shape:
 
 
 def make_params(density=0.25, block=128, Ck=0, Cq=0, n_sample=256, n_probe=128, rK=48, rQ=64, r_out=16, lam=0.1,
-                eps_rms=1e-6, eps_std=1e-6, kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0, partition=0) -> Params:
-    return Params(partition=partition, density=density, block=block, Ck=Ck, Cq=Cq, n_sample=n_sample, n_probe=n_probe, rK=rK, rQ=rQ,
+                eps_rms=1e-6, eps_std=1e-6, kmeans_iters=8, softmax_scale=0.0, seed=0, mode=0, partition=0,
+                head_offset=0) -> Params:
+    return Params(partition=partition, head_offset=head_offset, density=density, block=block, Ck=Ck, Cq=Cq, n_sample=n_sample, n_probe=n_probe, rK=rK, rQ=rQ,
                   r_out=r_out, lam=lam, eps_rms=eps_rms, eps_std=eps_std, kmeans_iters=kmeans_iters,
                   softmax_scale=softmax_scale, seed=seed, mode=mode)
 
@@ -401,34 +402,86 @@ def sparsepr_stage_route(score: torch.Tensor, nq: torch.Tensor, nk: torch.Tensor
 
 
 # ---- whole call on host buffers ----------------------------------------------------------
-def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, dev_buffers=None):
-    """One full call for a user whose tensors live in (pinned) host memory:
-    host->device copies, plan, attend, device->host copy of O.  Returns O on host.
-    The plan needs only Q and K, so V travels on a second stream while the plan runs."""
+def head_groups(B: int, H: int, G: int, groups: int):
+    """Cuts the B x H heads of a problem into about `groups` boxes (b0, b1, h0, h1) whose heads are consecutive in
+    the order b H + h: ranges of heads of one batch entry (multiples of the K/V sharing factor G), or ranges of
+    whole batch entries."""
+    groups = max(1, min(int(groups), B * (H // G)))
+    boxes = []
+    if B >= groups:
+        for i in range(groups):
+            b0, b1 = B * i // groups, B * (i + 1) // groups
+            if b1 > b0:
+                boxes.append((b0, b1, 0, H))
+        return boxes
+    per_b = max(1, min(-(-groups // B), H // G))
+    for b in range(B):
+        for i in range(per_b):
+            h0, h1 = (H // G) * i // per_b * G, (H // G) * (i + 1) // per_b * G
+            if h1 > h0:
+                boxes.append((b, b + 1, h0, h1))
+    return boxes
+
+
+def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, dev_buffers=None, groups=4):
+    """One full call for a user whose tensors live in (pinned) host memory: host->device copies, plan,
+    attend, device->host copy of O.  Returns O on host.
+
+    Heads are independent, so the problem is cut into `groups` groups of heads (head_groups) that move through a
+    pipeline: while one group is computed the next one is uploaded and the previous result goes back, and two
+    compute streams take the groups in turn so that the latency-bound kernels of one group (one CTA per head) run
+    beside the attention of the other.  Every group is a call of its own with `head_offset` = its first head, which
+    keeps the row samples, and with them every bit of the plan, those of a single call over all heads (the outputs
+    agree up to the summation order of the probe rows, whose number of key slices follows the head count of a call).
+    dev_buffers: optional device tensors (Q, K, V[, O]) of the full shapes, reused between calls."""
     dev = torch.device("cuda")
     if dev_buffers is None:
         dev_buffers = [torch.empty(t.shape, dtype=t.dtype, device=dev) for t in (Qh, Kh, Vh)]
-    Qd, Kd, Vd = dev_buffers
+    Qd, Kd, Vd = dev_buffers[:3]
+    Od = dev_buffers[3] if len(dev_buffers) > 3 else torch.empty(Qh.shape, dtype=Qh.dtype, device=dev)
+    B, H = Qh.shape[0], Qh.shape[1]
+    G = H // Kh.shape[1]
+    boxes = head_groups(B, H, G, groups)
     main = torch.cuda.current_stream()
-    side = _copy_stream()
-    Qd.copy_(Qh, non_blocking=True)
-    Kd.copy_(Kh, non_blocking=True)
-    side.wait_stream(main)                      # V follows Q and K on the link; earlier work on Vd is finished too
-    with torch.cuda.stream(side):
-        Vd.copy_(Vh, non_blocking=True)
-    plan = sparsepr_plan(Qd, Kd, Vd, params=params)
-    main.wait_stream(side)
-    O = sparsepr_attend(plan, Qd, Kd, Vd)
-    Oh.copy_(O, non_blocking=True)
+    up, down, second = _aux_stream("up"), _aux_stream("down"), _aux_stream("work")
+    up.wait_stream(main)                         # earlier work on the device buffers is finished
+    second.wait_stream(main)
+    ev_qk, ev_v = [], []
+    with torch.cuda.stream(up):
+        for (b0, b1, h0, h1) in boxes:
+            Qd[b0:b1, h0:h1].copy_(Qh[b0:b1, h0:h1], non_blocking=True)
+            Kd[b0:b1, h0 // G:h1 // G].copy_(Kh[b0:b1, h0 // G:h1 // G], non_blocking=True)
+            ev_qk.append(up.record_event())
+            Vd[b0:b1, h0 // G:h1 // G].copy_(Vh[b0:b1, h0 // G:h1 // G], non_blocking=True)
+            ev_v.append(up.record_event())
+    plans = []
+    for i, (b0, b1, h0, h1) in enumerate(boxes):
+        w = main if i % 2 == 0 else second
+        q, k, v = Qd[b0:b1, h0:h1], Kd[b0:b1, h0 // G:h1 // G], Vd[b0:b1, h0 // G:h1 // G]
+        o = Od[b0:b1, h0:h1]
+        prm = Params.from_buffer_copy(params)
+        prm.head_offset = params.head_offset + b0 * H + h0
+        with torch.cuda.stream(w):
+            w.wait_event(ev_qk[i])
+            plan = sparsepr_plan(q, k, v, params=prm)
+            w.wait_event(ev_v[i])
+            sparsepr_attend(plan, q, k, v, out=o)
+            done = w.record_event()
+        plans.append(plan)                       # workspaces stay alive until the queued work has run
+        down.wait_event(done)
+        with torch.cuda.stream(down):
+            Oh[b0:b1, h0:h1].copy_(o, non_blocking=True)
+    main.wait_stream(second)
+    main.wait_stream(down)
     main.synchronize()
     return Oh
 
 
-_COPY_STREAM = {}
+_AUX_STREAMS = {}
 
 
-def _copy_stream():
-    d = torch.cuda.current_device()
-    if d not in _COPY_STREAM:
-        _COPY_STREAM[d] = torch.cuda.Stream(device=d)
-    return _COPY_STREAM[d]
+def _aux_stream(name):
+    key = (torch.cuda.current_device(), name)
+    if key not in _AUX_STREAMS:
+        _AUX_STREAMS[key] = torch.cuda.Stream(device=key[0])
+    return _AUX_STREAMS[key]

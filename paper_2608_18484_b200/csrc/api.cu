@@ -49,6 +49,7 @@ struct Resolved {
   bool full_rank;                      // r_out covers the whole row space of the probe residuals: the projector is the identity
   float density, lambda, eps_rms, eps_std, scale;
   u64 seed;
+  int head_offset;                 // first head of this call within the whole problem (keys the row samples)
   i64 qs[3], ks[3], vs[3], os[3];
 };
 
@@ -112,6 +113,8 @@ sparsepr_status_t resolve(const sparsepr_shape_t* s, const sparsepr_params_t* p,
   r->eps_std = p->eps_std > 0.f ? p->eps_std : 1e-6f;
   r->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / std::sqrt((float)s->d);
   r->seed = p->seed;
+  if (p->head_offset < 0 || p->head_offset % r->G != 0) return SPARSEPR_ERR_INVALID_ARG;
+  r->head_offset = p->head_offset;
   return SPARSEPR_OK;
 }
 
@@ -364,7 +367,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
   // fixed point, so the later passes of that head return at once (their result would be identical).
   int* changed = p->km_changed + (tag == kTagQInit ? (size_t)(R.T + 1) * R.BH : 0);
   cudaMemsetAsync(changed, 0, (size_t)(R.T + 1) * R.BH * sizeof(int), st);
-  launch_kmeans_init(p->phi, ld, nheads, R.N, r, C, R.seed, tag, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
+  launch_kmeans_init(p->phi, ld, nheads, R.N, r, C, R.seed, tag, tag == kTagQInit ? R.head_offset : R.head_offset / R.G, p->mu, p->sums, p->counts, p->maxabs, p->fx_shift, st);
   const bool tcp = kmeans_tc_supported() && r <= kMaxRank;
   float* mumax = tcp ? nullptr : p->mumax;       // the tensor-core assignment derives the norm bound from ||mu||^2 itself
   // (with the tensor-core assignment the finalize step also writes the two bf16 words of every centroid)
@@ -510,7 +513,7 @@ static sparsepr_status_t plan_impl(const sparsepr_shape_t* shape, const sparsepr
   } else {
     // every query head samples its own rows; under grouped-query attention the K/V head's metric is the mean over its
     // query heads (Section 4.3: the K/V partition is shared by the associated query heads)
-    launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, p->Mmat, st);
+    launch_sample_gram(r.dtype, Q, r.qs, r.BH, r.H, r.N, r.d, r.Ms, r.seed, r.head_offset, p->Mmat, st);
     const double* metric = p->Mmat;
     if (r.G > 1) {
       k_pool_metric<<<dim3(16, r.BHkv), 256, 0, st>>>(p->Mmat, r.G, r.d * r.d, p->Mpool);

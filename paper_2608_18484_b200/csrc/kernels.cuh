@@ -10,7 +10,7 @@ int sm_count();
 
 // ---- partition.cu -------------------------------------------------------------
 cudaError_t init_group_sort();
-void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
+void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed, int head0,
                         double* Mout, cudaStream_t st);
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st);
 // eigen.cu: leading r <= 64 eigenpairs of `batch` symmetric n x n matrices (n = 64 or 128), `stride` doubles apart.
@@ -25,7 +25,7 @@ void launch_project(int dtype, const void* X, const i64* xs, int BH, int H, int 
 // features of the semantic partition: the activations themselves as float32 rows [BH][N][d]
 void launch_raw_features(int dtype, const void* X, const i64* xs, int BH, int H, int N, int d, float* phi, unsigned* maxabs,
                          int* err, cudaStream_t st);
-void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
+void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, int head0, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st);
 void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, int C, const int* prev, i64* sums,
                              int* counts, const int* fx_shift, cudaStream_t st);

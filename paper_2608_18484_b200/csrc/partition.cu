@@ -27,11 +27,11 @@ __device__ __forceinline__ void gram_accumulate(const double* rows, int nrows, i
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i64 sb, i64 sh, i64 sn, int H, int N,
-                                                     int Ms, u64 seed, double* __restrict__ Mout) {
+                                                     int Ms, u64 seed, int head0, double* __restrict__ Mout) {
   __shared__ __align__(16) double rows[kGramChunk * D];
   const int bh = blockIdx.y, b = bh / H, h = bh % H;
   const T* base = Q + b * sb + h * sh;
-  const u64 U = sample_offset(seed, kTagQuerySample, bh);
+  const u64 U = sample_offset(seed, kTagQuerySample, head0 + bh);
   const int j = threadIdx.x % D, i0 = blockIdx.x * kGramSlab + (threadIdx.x / D) * 8;
   const bool active = threadIdx.x < 2 * D;
   double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -101,14 +101,14 @@ __global__ void __launch_bounds__(256) k_centroid_gram(const float* __restrict__
   }
 }
 
-void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed,
+void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, int N, int d, int Ms, u64 seed, int head0,
                         double* Mout, cudaStream_t st) {
   if (dtype == SPARSEPR_BF16) {
-    if (d == 128) k_sample_gram<__nv_bfloat16, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
-    else k_sample_gram<__nv_bfloat16, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    if (d == 128) k_sample_gram<__nv_bfloat16, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, head0, Mout);
+    else k_sample_gram<__nv_bfloat16, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const __nv_bfloat16*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, head0, Mout);
   } else {
-    if (d == 128) k_sample_gram<float, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
-    else k_sample_gram<float, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, Mout);
+    if (d == 128) k_sample_gram<float, 128><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, head0, Mout);
+    else k_sample_gram<float, 64><<<dim3(d / kGramSlab, BH), 256, 0, st>>>((const float*)Q, qs[0], qs[1], qs[2], H, N, Ms, seed, head0, Mout);
   }
 }
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st) {
@@ -363,11 +363,11 @@ void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, con
 
 // Initial centroids = feature rows of the strided init sample; also clears the sums
 // and derives the fixed-point shift of the head from max |phi|.
-__global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, int r, int R, int C, u64 seed, int tag,
+__global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, int r, int R, int C, u64 seed, int tag, int head0,
                               float* __restrict__ mu, i64* __restrict__ sums, int* __restrict__ counts,
                               const unsigned* __restrict__ maxabs_bits, int* __restrict__ fx_shift) {
   const int bh = blockIdx.y;
-  const u64 U = sample_offset(seed, tag, bh);
+  const u64 U = sample_offset(seed, tag, head0 + bh);
   for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < C * R; e += gridDim.x * blockDim.x) {
     const int c = e / R, k = e % R;
     const int row = strided_row(c, C, N, U);
@@ -488,11 +488,11 @@ void launch_kmeans_warm_sums(const float* phi, int ldphi, int BH, int N, int r, 
   k_kmeans_warm_sums<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(phi, ldphi, N, r, R, C, prev, sums, counts, fx_shift);
 }
 
-void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, float* mu,
+void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C, u64 seed, int tag, int head0, float* mu,
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st) {
   const int R = feature_ld(r);
   dim3 grid((C * R + 255) / 256, BH);
-  k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, mu, sums, counts, maxabs_bits, fx_shift);
+  k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, head0, mu, sums, counts, maxabs_bits, fx_shift);
 }
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh, __nv_bfloat16* ml) {
