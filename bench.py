@@ -459,22 +459,22 @@ def main():
     # ---- end to end through the host-buffer call ----
     e2e = None
     if not args.no_e2e:
-        bufs = [Qd, Kd, Vd, torch.empty_like(Qd)]
+        hws = B.call_host_workspace(pinned[0], pinned[1], params, args.e2e_groups)
         for _ in range(2):
-            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs, groups=args.e2e_groups)
+            B.sparsepr_call_host(*pinned, Oh, params, workspace=hws, groups=args.e2e_groups)
         barrier()
         n_e2e = max(1, min(args.steps, 5))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(n_e2e):
-            B.sparsepr_call_host(*pinned, Oh, params, dev_buffers=bufs, groups=args.e2e_groups)
+            B.sparsepr_call_host(*pinned, Oh, params, workspace=hws, groups=args.e2e_groups)
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1) / n_e2e
         e2e_ms = max_over_ranks(e2e_ms, dev, world)
         nbytes = Qd.numel() * Qd.element_size()
         e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
-               "head_groups": len(B.head_groups(wl.B if hasattr(wl, "B") else 1, wl.H, 1, args.e2e_groups))}
+               "head_groups": len(B.head_groups(1, wl.H, wl.H, args.e2e_groups))}
 
     if rank != 0:
         if world > 1:

@@ -245,6 +245,26 @@ sparsepr_status_t sparsepr_attend(const sparsepr_plan_t* plan, const void* Q, co
 sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_scale,
                                  const void* Q, const void* K, const void* V, void* O, void* cuda_stream);
 
+/* A whole call for tensors in HOST memory (Stages 1-4 plus the copies): Q, O contiguous [B, H, N, d], K, V
+ * contiguous [B, Hkv, N, d] in (preferably pinned) host memory; the stride fields of `shape` are ignored.  Heads are
+ * independent (Section 4.3 shares only the K/V partition inside a group of query heads), so the problem is cut into
+ * `groups` groups of consecutive heads (sparsepr_head_groups) that move through a pipeline: one stream uploads group
+ * after group, two streams take the groups in turn through sparsepr_plan + sparsepr_attend, a fourth returns every
+ * group's O.  A group runs with head_offset = params->head_offset + its first head, so its plan is that of one call
+ * over all heads.  `workspace`: DEVICE, sparsepr_call_host_workspace_bytes(shape, params, groups), 256-byte aligned;
+ * it receives the device copies of Q, K, V, O and the workspaces of every group.  The call returns when O is
+ * complete in host memory (it synchronises `cuda_stream` and its own streams).  groups < 1 selects 4. */
+size_t sparsepr_call_host_workspace_bytes(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                          int32_t groups);
+sparsepr_status_t sparsepr_call_host(const sparsepr_shape_t* shape, const sparsepr_params_t* params,
+                                     const void* Q_host, const void* K_host, const void* V_host, void* O_host,
+                                     int32_t groups, void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* The groups of that pipeline: boxes[4 i .. 4 i + 3] = {b0, b1, h0, h1}, heads [h0, h1) of the batch entries
+ * [b0, b1); either one batch entry with a range of heads (a multiple of H / Hkv at both ends) or whole batch
+ * entries, in the order b H + h.  Writes at most max_boxes boxes and returns the number of groups (at most
+ * groups + B), 0 on invalid arguments.  HOST only, no GPU needed. */
+int32_t sparsepr_head_groups(int32_t B, int32_t H, int32_t Hkv, int32_t groups, int32_t* boxes, int32_t max_boxes);
+
 /* The same calls with per-stage timing (the latency decomposition of the paper's
  * Section 5.3): identical work and results; they record CUDA events between the
  * stages, synchronise the stream before returning and add the elapsed
@@ -262,6 +282,9 @@ sparsepr_status_t sparsepr_dense_timed(const sparsepr_shape_t* shape, float soft
 
 /* Synchronises the stream the plan was built on, then fills *host_out. */
 sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* plan, sparsepr_stats_t* host_out);
+/* Only the device error word of the plan and of the attend calls made with it so far (what sparsepr_plan_stats
+ * reports as `device_error`): waits for the plan's streams and copies one word. */
+sparsepr_status_t sparsepr_plan_device_error(const sparsepr_plan_t* plan, int32_t* device_error);
 sparsepr_status_t sparsepr_plan_export(const sparsepr_plan_t* plan, sparsepr_plan_host_t* host_out);
 
 /* Synchronises like sparsepr_plan_export, then copies the requested intermediates.  A plan made by

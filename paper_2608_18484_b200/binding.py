@@ -74,7 +74,8 @@ class Profile(C.Structure):
 EXPORTS = ["sparsepr_stage_assign_static", "sparsepr_plan_timed", "sparsepr_attend_timed", "sparsepr_dense_timed", "sparsepr_status_string", "sparsepr_plan_workspace_bytes", "sparsepr_attend_workspace_bytes",
            "sparsepr_plan", "sparsepr_attend", "sparsepr_dense", "sparsepr_plan_stats", "sparsepr_plan_export",
            "sparsepr_plan_export_features", "sparsepr_plan_warm", "sparsepr_plan_assignments",
-           "sparsepr_selftest_bounded_wait",
+           "sparsepr_selftest_bounded_wait", "sparsepr_call_host", "sparsepr_call_host_workspace_bytes",
+           "sparsepr_head_groups", "sparsepr_plan_device_error",
            "sparsepr_plan_import", "sparsepr_plan_destroy", "sparsepr_stage_assign_workspace_bytes",
            "sparsepr_stage_assign", "sparsepr_stage_permute", "sparsepr_stage_route"]
 
@@ -107,6 +108,12 @@ def lib():
         L.sparsepr_plan_export_features.argtypes = [vp, C.POINTER(PlanFeatures)]
         L.sparsepr_plan_import.argtypes = [C.POINTER(Shape), C.POINTER(Params), C.POINTER(PlanHost), vp, sz, vp,
                                            C.POINTER(vp)]
+        L.sparsepr_call_host_workspace_bytes.restype = sz
+        L.sparsepr_call_host_workspace_bytes.argtypes = [C.POINTER(Shape), C.POINTER(Params), i32]
+        L.sparsepr_call_host.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, i32, vp, sz, vp]
+        L.sparsepr_head_groups.restype = i32
+        L.sparsepr_head_groups.argtypes = [i32, i32, i32, i32, C.POINTER(i32), i32]
+        L.sparsepr_plan_device_error.argtypes = [vp, C.POINTER(i32)]
         L.sparsepr_plan_destroy.argtypes = [vp]
         L.sparsepr_plan_destroy.restype = None
         L.sparsepr_stage_assign_workspace_bytes.restype = sz
@@ -402,86 +409,39 @@ def sparsepr_stage_route(score: torch.Tensor, nq: torch.Tensor, nk: torch.Tensor
 
 
 # ---- whole call on host buffers ----------------------------------------------------------
-def head_groups(B: int, H: int, G: int, groups: int):
-    """Cuts the B x H heads of a problem into about `groups` boxes (b0, b1, h0, h1) whose heads are consecutive in
-    the order b H + h: ranges of heads of one batch entry (multiples of the K/V sharing factor G), or ranges of
-    whole batch entries."""
-    groups = max(1, min(int(groups), B * (H // G)))
-    boxes = []
-    if B >= groups:
-        for i in range(groups):
-            b0, b1 = B * i // groups, B * (i + 1) // groups
-            if b1 > b0:
-                boxes.append((b0, b1, 0, H))
-        return boxes
-    per_b = max(1, min(-(-groups // B), H // G))
-    for b in range(B):
-        for i in range(per_b):
-            h0, h1 = (H // G) * i // per_b * G, (H // G) * (i + 1) // per_b * G
-            if h1 > h0:
-                boxes.append((b, b + 1, h0, h1))
-    return boxes
+def head_groups(B: int, H: int, Hkv: int, groups: int):
+    """The groups of heads the host-buffer call pipelines: boxes (b0, b1, h0, h1)."""
+    n = lib().sparsepr_head_groups(B, H, Hkv, groups, None, 0)
+    buf = (C.c_int32 * (4 * max(n, 1)))()
+    lib().sparsepr_head_groups(B, H, Hkv, groups, buf, n)
+    return [tuple(buf[4 * i:4 * i + 4]) for i in range(n)]
 
 
-def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, dev_buffers=None, groups=4):
-    """One full call for a user whose tensors live in (pinned) host memory: host->device copies, plan,
-    attend, device->host copy of O.  Returns O on host.
+def call_host_workspace(Qh, Kh, params: Params, groups=4) -> torch.Tensor:
+    """Device workspace of sparsepr_call_host for tensors of these shapes (reusable between calls)."""
+    shape = _host_shape(Qh, Kh)
+    nbytes = lib().sparsepr_call_host_workspace_bytes(C.byref(shape), C.byref(params), groups)
+    if nbytes == 0:
+        raise SparsePRError(1, "sparsepr_call_host_workspace_bytes")
+    return _workspace(nbytes, torch.device("cuda"))
 
-    Heads are independent, so the problem is cut into `groups` groups of heads (head_groups) that move through a
-    pipeline: while one group is computed the next one is uploaded and the previous result goes back, and two
-    compute streams take the groups in turn so that the latency-bound kernels of one group (one CTA per head) run
-    beside the attention of the other.  Every group is a call of its own with `head_offset` = its first head, which
-    keeps the row samples, and with them every bit of the plan, those of a single call over all heads (the outputs
-    agree up to the summation order of the probe rows, whose number of key slices follows the head count of a call).
-    dev_buffers: optional device tensors (Q, K, V[, O]) of the full shapes, reused between calls."""
-    dev = torch.device("cuda")
-    if dev_buffers is None:
-        dev_buffers = [torch.empty(t.shape, dtype=t.dtype, device=dev) for t in (Qh, Kh, Vh)]
-    Qd, Kd, Vd = dev_buffers[:3]
-    Od = dev_buffers[3] if len(dev_buffers) > 3 else torch.empty(Qh.shape, dtype=Qh.dtype, device=dev)
-    B, H = Qh.shape[0], Qh.shape[1]
-    G = H // Kh.shape[1]
-    boxes = head_groups(B, H, G, groups)
-    main = torch.cuda.current_stream()
-    up, down, second = _aux_stream("up"), _aux_stream("down"), _aux_stream("work")
-    up.wait_stream(main)                         # earlier work on the device buffers is finished
-    second.wait_stream(main)
-    ev_qk, ev_v = [], []
-    with torch.cuda.stream(up):
-        for (b0, b1, h0, h1) in boxes:
-            Qd[b0:b1, h0:h1].copy_(Qh[b0:b1, h0:h1], non_blocking=True)
-            Kd[b0:b1, h0 // G:h1 // G].copy_(Kh[b0:b1, h0 // G:h1 // G], non_blocking=True)
-            ev_qk.append(up.record_event())
-            Vd[b0:b1, h0 // G:h1 // G].copy_(Vh[b0:b1, h0 // G:h1 // G], non_blocking=True)
-            ev_v.append(up.record_event())
-    plans = []
-    for i, (b0, b1, h0, h1) in enumerate(boxes):
-        w = main if i % 2 == 0 else second
-        q, k, v = Qd[b0:b1, h0:h1], Kd[b0:b1, h0 // G:h1 // G], Vd[b0:b1, h0 // G:h1 // G]
-        o = Od[b0:b1, h0:h1]
-        prm = Params.from_buffer_copy(params)
-        prm.head_offset = params.head_offset + b0 * H + h0
-        with torch.cuda.stream(w):
-            w.wait_event(ev_qk[i])
-            plan = sparsepr_plan(q, k, v, params=prm)
-            w.wait_event(ev_v[i])
-            sparsepr_attend(plan, q, k, v, out=o)
-            done = w.record_event()
-        plans.append(plan)                       # workspaces stay alive until the queued work has run
-        down.wait_event(done)
-        with torch.cuda.stream(down):
-            Oh[b0:b1, h0:h1].copy_(o, non_blocking=True)
-    main.wait_stream(second)
-    main.wait_stream(down)
-    main.synchronize()
+
+def _host_shape(Qh, Kh) -> Shape:
+    B, H, N, d = Qh.shape
+    return Shape(B=B, H=H, N=N, d=d, dv=d, dtype=_dtype_code(Qh), Hkv=Kh.shape[1])
+
+
+def sparsepr_call_host(Qh, Kh, Vh, Oh, params: Params, workspace=None, groups=4):
+    """One full call for a user whose tensors live in (pinned) host memory: host->device copies, plan, attend,
+    device->host copy of O, pipelined over `groups` groups of heads inside the library.  Returns O on host (complete
+    when the call returns).  `workspace`: a tensor from call_host_workspace, allocated here if absent."""
+    for t in (Qh, Kh, Vh, Oh):
+        if t.is_cuda or not t.is_contiguous() or t.dim() != 4:
+            raise ValueError("expected contiguous host tensors [B, H, N, d]")
+    if Kh.shape != Vh.shape or Oh.shape != Qh.shape or Qh.shape[1] % Kh.shape[1] != 0:
+        raise ValueError("K and V need the same shape, O the shape of Q, and H a multiple of the K/V heads")
+    ws = workspace if workspace is not None else call_host_workspace(Qh, Kh, params, groups)
+    shape = _host_shape(Qh, Kh)
+    _check(lib().sparsepr_call_host(C.byref(shape), C.byref(params), Qh.data_ptr(), Kh.data_ptr(), Vh.data_ptr(),
+                                    Oh.data_ptr(), groups, ws.data_ptr(), ws.numel(), _stream()), "sparsepr_call_host")
     return Oh
-
-
-_AUX_STREAMS = {}
-
-
-def _aux_stream(name):
-    key = (torch.cuda.current_device(), name)
-    if key not in _AUX_STREAMS:
-        _AUX_STREAMS[key] = torch.cuda.Stream(device=key[0])
-    return _AUX_STREAMS[key]

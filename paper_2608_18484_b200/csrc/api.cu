@@ -771,6 +771,15 @@ sparsepr_status_t sparsepr_dense(const sparsepr_shape_t* shape, float softmax_sc
   return launch_ok() ? SPARSEPR_OK : SPARSEPR_ERR_CUDA;
 }
 
+sparsepr_status_t sparsepr_plan_device_error(const sparsepr_plan_t* p, int32_t* device_error) {
+  if (!p || !device_error) return SPARSEPR_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess || (p->side && cudaStreamSynchronize(p->side) != cudaSuccess)) return SPARSEPR_ERR_CUDA;
+  int errw = 0;
+  if (cudaMemcpy(&errw, p->err, sizeof(errw), cudaMemcpyDeviceToHost) != cudaSuccess) return SPARSEPR_ERR_CUDA;
+  *device_error = errw;
+  return SPARSEPR_OK;
+}
+
 sparsepr_status_t sparsepr_plan_stats(const sparsepr_plan_t* p, sparsepr_stats_t* out) {
   if (!p || !out) return SPARSEPR_ERR_INVALID_ARG;
   const Resolved& r = p->r;

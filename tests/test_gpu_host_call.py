@@ -16,7 +16,7 @@ from tests.gpu_util import heads_to_device
 def test_head_groups_cover_every_head_once():
     for Bn, H, G, groups in [(1, 24, 1, 4), (1, 24, 1, 5), (1, 4, 2, 4), (2, 6, 2, 3), (4, 8, 1, 2), (3, 2, 1, 8),
                              (1, 1, 1, 4), (2, 40, 8, 7)]:
-        boxes = B.head_groups(Bn, H, G, groups)
+        boxes = B.head_groups(Bn, H, H // G, groups)
         seen = np.zeros((Bn, H), dtype=int)
         last = -1
         for (b0, b1, h0, h1) in boxes:
