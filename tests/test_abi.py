@@ -64,6 +64,15 @@ def test_workspace_sizes_scale_and_reject(lib):
     assert lib.sparsepr_plan_workspace_bytes(C.byref(_shape()), C.byref(B.make_params(n_probe=96, r_out=128))) > 0
     assert lib.sparsepr_stage_assign_workspace_bytes(1000, 10, 48) > 1000 * 48 * 4
     assert lib.sparsepr_stage_assign_workspace_bytes(1000, 10, 65) == 0
+    # the host-buffer call holds the device copies of Q, K, V, O and one plan + attend workspace per group of heads
+    sh = _shape(32760, H=24)
+    host = lib.sparsepr_call_host_workspace_bytes(C.byref(sh), C.byref(p), 4)
+    assert host >= 4 * 24 * 32760 * 128 * 2 + big + att - (1 << 20) and host % 256 == 0
+    assert lib.sparsepr_call_host_workspace_bytes(C.byref(_shape(d=96)), C.byref(p), 4) == 0
+    assert lib.sparsepr_call_host_workspace_bytes(C.byref(sh), C.byref(B.make_params(head_offset=-1)), 4) == 0
+    assert lib.sparsepr_head_groups(1, 4, 3, 2, None, 0) == 0           # K/V heads must divide the query heads
+    assert B.head_groups(1, 24, 24, 4) == [(0, 1, 0, 6), (0, 1, 6, 12), (0, 1, 12, 18), (0, 1, 18, 24)]
+    assert B.head_groups(1, 8, 2, 4) == [(0, 1, 0, 4), (0, 1, 4, 8)]     # groups hold whole K/V heads
 
 
 def test_argument_errors_are_reported_before_any_launch(lib):
