@@ -121,3 +121,48 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable():
     plan = B.sparsepr_plan(Qd, Kd, Vd, density=0.25, block=64, n_sample=64, n_probe=16, softmax_scale=1.0)
     O = B.sparsepr_attend(plan, Qd, Kd, Vd)
     assert B.sparsepr_plan_stats(plan)["device_error"] == 0 and torch.isfinite(O).all()
+
+
+def _spectrum_inputs(d, N, levels, dtype, seed):
+    """Q whose sample Gram matrix (all N rows sampled) is R^T diag(levels) R / d for a random rotation R: rows are the
+    scaled unit vectors in turn, rotated.  Equal levels give exactly (f32) or nearly (bf16) repeated eigenvalues."""
+    rng = np.random.default_rng(seed)
+    R, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    rows = np.zeros((N, d))
+    rows[np.arange(N), np.arange(N) % d] = np.sqrt(np.asarray(levels, dtype=np.float64))[np.arange(N) % d]
+    Q = torch.from_numpy(rows @ R)[None, None].to(dtype).cuda().contiguous()
+    K = torch.from_numpy(rng.standard_normal((N, d)))[None, None].to(dtype).cuda().contiguous()
+    return Q, K
+
+
+@pytest.mark.parametrize("d,dtype,tol", [(64, torch.float32, 1e-5), (128, torch.bfloat16, 2e-3)], ids=["f32", "bf16"])
+@pytest.mark.parametrize("kind", ["identity", "two-level", "staircase"])
+def test_feature_map_on_repeated_and_clustered_eigenvalues(d, dtype, tol, kind):
+    """Section 4.1's feature map is built from the leading eigenpairs of the key-response metric.  Metrics with
+    repeated eigenvalues (every basis of the eigenspace is right) and with tight clusters are where an
+    eigen-solver's orthogonalisation and its choice of the leading pairs show: the columns of F_K must stay
+    orthogonal, be eigenvectors of the metric, carry unit-mean eigenvalues and capture the leading ones."""
+    N, rK = 8 * d, 48
+    levels = {"identity": np.ones(d),
+              "two-level": np.where(np.arange(d) < 10, 4.0, 1.0),
+              "staircase": 1.0 + 1e-4 * (np.arange(d) // 4) + np.where(np.arange(d) < 3, 2.0, 0.0)}[kind]
+    Q, K = _spectrum_inputs(d, N, levels, dtype, seed=7)
+    plan = B.sparsepr_plan(Q, K, K, density=0.5, block=d, n_sample=N, n_probe=16, rK=rK, softmax_scale=1.0)
+    assert B.sparsepr_plan_stats(plan)["device_error"] == 0
+    F = B.sparsepr_plan_export_features(plan, fields=("F_K",))["F_K"][0].astype(np.float64)      # [d, rK]
+    Qh = to_np(Q[0, 0])
+    M = Qh.T @ Qh / N                                              # the metric as the kernels see the inputs
+    lam_all = np.linalg.eigvalsh(M)[::-1]
+    G = F.T @ F
+    # orthogonal columns with unit-mean squared norms (eigenvalues divided by their mean over the retained pairs)
+    off = G - np.diag(np.diag(G))
+    assert np.abs(off).max() <= tol * np.abs(np.diag(G)).max(), np.abs(off).max()
+    assert abs(np.trace(G) - rK) <= 10 * tol * rK
+    # eigenvectors of the metric: residual of every column against its Rayleigh quotient
+    lam = np.einsum("ij,ij->j", F, M @ F) / np.diag(G)
+    res = np.linalg.norm(M @ F - F * lam[None], axis=0) / (np.linalg.norm(F, axis=0) * lam_all[0])
+    assert res.max() <= 10 * tol, res.max()
+    # the leading ones: their eigenvalue sum is that of the top rK (repeated eigenvalues make the set non-unique,
+    # its sum is unique), and the squared norms are proportional to the eigenvalues
+    assert abs(lam.sum() - lam_all[:rK].sum()) <= 10 * tol * lam_all[:rK].sum()
+    assert np.allclose(np.diag(G), lam / lam.mean(), rtol=0, atol=20 * tol * np.diag(G).max())
