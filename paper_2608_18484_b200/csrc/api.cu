@@ -300,7 +300,7 @@ void carve_plan(Carver& c, const Resolved& r, sparsepr_plan_s* p) {
   __nv_bfloat16* Ft = c.take<__nv_bfloat16>(BH * (size_t)3 * 64 * 128);
   int* rem_pos = c.take<int>(BH * N); int* rem_grp = c.take<int>(BH * N); int* rem_cnt = c.take<int>(BH);
   int* km_changed = c.take<int>(2 * (size_t)(r.T + 1) * BH);
-  int* flagcnt = c.take<int>(BH);
+  int* flagcnt = c.take<int>(2 * BH);                       // two sets of per-head counters, used by alternate passes
   double* eigws = c.take<double>(eig_scratch_doubles((int)BH, r.d));
   double* Mpool = c.take<double>(r.G > 1 ? (size_t)r.BHkv * d * d : 0);
   if (p) {
@@ -375,6 +375,7 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
   if (warm_prev) launch_kmeans_warm_sums(p->phi, ld, nheads, R.N, r, C, warm_prev, p->sums, p->counts, p->fx_shift, st);
   launch_kmeans_finalize(p->mu, p->mu2, mumax, p->sums, p->counts, p->fx_shift, nheads, C, r, warm_prev ? 1 : 0, st, tcp ? p->mh : nullptr, tcp ? p->ml : nullptr);
   if (tcp) launch_split_bf16(p->phi, ld, (i64)nheads * R.N, r, p->xh, p->xl, p->xnorm, st);
+  if (tcp) cudaMemsetAsync(p->flagcnt, 0, 2 * (size_t)R.BH * sizeof(int), st);
   for (int t = 1; t <= R.T; ++t) {
     const bool upd = t < R.T;
     const int* prev = t > 1 ? changed + (size_t)(t - 1) * R.BH : nullptr;
@@ -384,7 +385,8 @@ void run_kmeans(const sparsepr_plan_s* p, int r, int C, int tag, int* assign, co
       ka.BH = nheads; ka.N = R.N; ka.C = C; ka.r = r; ka.R = ld; ka.xh = p->xh; ka.xl = p->xl; ka.mh = p->mh; ka.ml = p->ml;
       ka.phi = p->phi; ka.ldphi = ld; ka.xnorm = p->xnorm; ka.mu = p->mu; ka.mu2 = p->mu2;
       ka.assign = assign; ka.sums = upd ? p->sums : nullptr; ka.counts = upd ? p->counts : nullptr; ka.fx_shift = p->fx_shift;
-      ka.flagged = p->flagged; ka.flag_count = p->flagcnt; ka.recheck_total = p->recheck; ka.err = p->err;
+      ka.flagged = p->flagged; ka.flag_count = p->flagcnt + (size_t)(t & 1) * R.BH; ka.flag_count_next = p->flagcnt + (size_t)((t + 1) & 1) * R.BH;
+      ka.recheck_total = p->recheck; ka.err = p->err;
       ka.prev_changed = prev; ka.cur_changed = cur;
       launch_kmeans_assign_tc(ka, st);
     } else {
@@ -957,6 +959,7 @@ sparsepr_status_t sparsepr_stage_assign(int32_t n, int32_t C, int32_t r, const f
     ka.BH = 1; ka.N = n; ka.C = C; ka.r = r; ka.R = R; ka.xh = xh; ka.xl = xl; ka.mh = mh; ka.ml = ml;
     ka.phi = Xp; ka.ldphi = R; ka.xnorm = xnorm; ka.mu = mup; ka.mu2 = mu2; ka.assign = a;
     ka.flagged = flagged; ka.flag_count = fx + 1; ka.recheck_total = fx + 2;
+    cudaMemsetAsync(ka.flag_count, 0, sizeof(int), st);
     if (!launch_kmeans_assign_tc(ka, st)) return SPARSEPR_ERR_CUDA;
   } else {
     launch_kmeans_assign(Xp, R, 1, n, r, mup, mu2, mumax, C, a, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, st);

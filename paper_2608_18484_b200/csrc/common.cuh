@@ -67,6 +67,26 @@ __host__ __device__ __forceinline__ u64 splitmix64(u64 x) {
   return z ^ (z >> 31);
 }
 enum { kTagQuerySample = 1, kTagKvInit = 2, kTagQInit = 3 };
+// Programmatic dependent launch: a kernel launched with launch_pdl may be scheduled while the kernel before it in
+// the stream still runs; pdl_wait() returns once that kernel has completed and its writes are visible, and must come
+// before the first access to anything it wrote.  pdl_launch_dependents() lets the kernel behind this one be scheduled
+// (its blocks wait in their own pdl_wait()), which takes the launch latency off a chain of short dependent kernels.
+// Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 __host__ __device__ __forceinline__ u64 sample_offset(u64 seed, int tag, int bh) {
   return splitmix64(seed * 0x100000001B3ull + (u64)tag * 0x10001ull + (u64)bh) >> 40;
 }

@@ -159,6 +159,8 @@ template <int NN> struct HhLayout {
 // sums of its squares are in shared memory, one after p and the partial sums of p.v are.
 template <int NN, typename T>
 __global__ void __launch_bounds__(2 * NN) k_householder(const double* __restrict__ Min, i64 stride, T* __restrict__ ws) {
+  pdl_wait();                                                   // the matrices come from the kernel before
+  pdl_launch_dependents();
   using HL = HhLayout<NN>;
   constexpr int kCh = 16, kNc = NN / (2 * kCh), kWarps = 2 * NN / 32;
   constexpr int kScrLd = kCh + 16 / (int)sizeof(T);             // padded chunk: 16-byte aligned, spreads the banks
@@ -315,6 +317,8 @@ __global__ void __launch_bounds__(2 * NN) k_householder(const double* __restrict
 template <int NN, typename T>
 __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict__ ws, int r, int scale_mode,
                                                              float* __restrict__ Fout, double* __restrict__ lam_out) {
+  pdl_wait();                                                   // T and the reflectors come from the kernel before
+  pdl_launch_dependents();
   using S = EigSmem<NN, T>;
   constexpr int LD = S::LD;
   auto pos = [](int c) { return c + (c / (NN / kTpr)) * (16 / (int)sizeof(T)); };
@@ -722,6 +726,8 @@ __global__ void __launch_bounds__(kEigThreads) k_eig_tridiag(const T* __restrict
 template <int NN>
 __global__ void __launch_bounds__(1024) k_jacobi_eig_f64(const double* __restrict__ Min, i64 stride, int r, int scale_mode,
                                                          float* __restrict__ Fout, double* __restrict__ lam_out) {
+  pdl_wait();                                                   // the marks come from the kernel before
+  pdl_launch_dependents();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* A = reinterpret_cast<double*>(smem_raw);                 // [NN][NN+1]
   float* V = reinterpret_cast<float*>(A + NN * (NN + 1));          // [NN][NN+1]
@@ -851,16 +857,16 @@ void launch_eig_top(const double* Min, i64 stride, int batch, int n, int r, int 
                     double* lam_out, double* ws, cudaStream_t st) {
 #define SPR_EIG(NN, TT)                                                                                        \
   do {                                                                                                         \
-    k_householder<NN, TT><<<batch, 2 * NN, 0, st>>>(Min, stride, reinterpret_cast<TT*>(ws));                   \
-    k_eig_tridiag<NN, TT><<<batch, kEigThreads, EigSmem<NN, TT>::total, st>>>(reinterpret_cast<const TT*>(ws), r, \
-                                                                            scale_mode, Fout, lam_out);       \
+    launch_pdl(k_householder<NN, TT>, dim3(batch), dim3(2 * NN), 0, st, Min, stride, reinterpret_cast<TT*>(ws));  \
+    launch_pdl(k_eig_tridiag<NN, TT>, dim3(batch), dim3(kEigThreads), EigSmem<NN, TT>::total, st,               \
+               reinterpret_cast<const TT*>(ws), r, scale_mode, Fout, lam_out);                                   \
   } while (0)
   if (n == 128) {
     if (precise) SPR_EIG(128, double); else SPR_EIG(128, float);
-    k_jacobi_eig_f64<128><<<batch, 1024, jacobi64_smem(128), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    launch_pdl(k_jacobi_eig_f64<128>, dim3(batch), dim3(1024), jacobi64_smem(128), st, Min, stride, r, scale_mode, Fout, lam_out);
   } else {
     if (precise) SPR_EIG(64, double); else SPR_EIG(64, float);
-    k_jacobi_eig_f64<64><<<batch, 1024, jacobi64_smem(64), st>>>(Min, stride, r, scale_mode, Fout, lam_out);
+    launch_pdl(k_jacobi_eig_f64<64>, dim3(batch), dim3(1024), jacobi64_smem(64), st, Min, stride, r, scale_mode, Fout, lam_out);
   }
 #undef SPR_EIG
 }

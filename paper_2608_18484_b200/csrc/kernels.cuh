@@ -60,6 +60,7 @@ struct KmeansTcArgs {
   i64* sums; int* counts; const int* fx_shift; // null sums = assignment only
   int *flagged, *flag_count, *recheck_total, *err;   // flagged [BH][N] scratch, flag_count [BH] scratch, recheck_total: rows rechecked by this pass
   const int* prev_changed; int* cur_changed;   // [BH] or null, as for launch_kmeans_assign
+  int* flag_count_next;                        // [BH] or null: the next pass's counters, zeroed by this pass (flag_count itself must arrive zeroed)
 };
 cudaError_t init_kmeans_tc();
 bool kmeans_tc_supported();

@@ -43,6 +43,7 @@ struct KmParams {
   int* assign;
   i64* sums; int* counts; const int* fx_shift;
   int* flagged; int* flag_count;        // rows left to the exact recheck: [BH][N] row indices, [BH] their number
+  int* flag_count_next;                 // [BH] or null: the counters of the next pass, zeroed here
   int* err;
   const int* prev_changed; int* cur_changed;   // [BH] or null: rows whose assignment changed in the previous / this pass
 };
@@ -63,6 +64,9 @@ k_kmeans_assign_tc(const __grid_constant__ CUtensorMap mapXh, const __grid_const
   __shared__ __align__(16) float mu2s[kMaxGroups];          // ||mu_c||^2, +inf beyond C
   __shared__ int s_skip;
   __shared__ float s_red[34];
+  pdl_wait();                                               // the centroids of this pass come from the kernel before
+  pdl_launch_dependents();
+  if (cta == 0 && tid == 0 && prm.flag_count_next) prm.flag_count_next[bh] = 0;   // last read by the recheck two kernels back
   float mu2max = 0.f;
   for (int c = tid; c < kMaxGroups; c += kKmThreads) {
     const float v = c < prm.C ? prm.mu2[(i64)bh * prm.C + c] : INFINITY;
@@ -320,6 +324,8 @@ __global__ void __launch_bounds__(256) k_assign_recheck_staged(const int* __rest
   const unsigned FULL = 0xffffffffu;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.y;
+  pdl_wait();                                                  // the row lists come from the assignment kernel before
+  pdl_launch_dependents();
   const int n = flag_count[bh];
   if (blockIdx.x == 0 && bh == 0 && tid == 0 && recheck_total) {
     int total = 0;
@@ -510,6 +516,8 @@ __global__ void __launch_bounds__(256) k_assign_recheck(const int* __restrict__ 
 __global__ void __launch_bounds__(256) k_split_bf16(const float* __restrict__ x, int ld, i64 rows, int r,
                                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
                                                     float* __restrict__ norm) {
+  pdl_wait();                                                   // the features come from the kernels before
+  pdl_launch_dependents();
   const i64 t = (i64)blockIdx.x * 256 + threadIdx.x;
   const i64 row = t >> 3;
   const int c0 = (int)(t & 7) * 8;
@@ -546,7 +554,7 @@ bool kmeans_tc_supported() { return tc::tma_available(); }
 
 void launch_split_bf16(const float* x, int ld, i64 rows, int r, __nv_bfloat16* hi, __nv_bfloat16* lo, float* norm,
                        cudaStream_t st) {
-  tc::k_split_bf16<<<(unsigned)((rows * 8 + 255) / 256), 256, 0, st>>>(x, ld, rows, r, hi, lo, norm);
+  launch_pdl(tc::k_split_bf16, dim3((unsigned)((rows * 8 + 255) / 256)), dim3(256), 0, st, x, ld, rows, r, hi, lo, norm);
 }
 
 // One assignment pass.  xh/xl: bf16 [BH][N][64]; mh/ml: bf16 [BH][C][64]; sums may be null (no update wanted).
@@ -578,15 +586,15 @@ bool launch_kmeans_assign_tc(const KmeansTcArgs& a, cudaStream_t st) {
   }
   p.phi = a.phi; p.ldphi = a.ldphi; p.xnorm = a.xnorm; p.mu2 = a.mu2; p.assign = a.assign;
   p.sums = a.sums; p.counts = a.counts; p.fx_shift = a.fx_shift; p.flagged = a.flagged; p.flag_count = a.flag_count; p.err = a.err;
-  p.prev_changed = a.prev_changed; p.cur_changed = a.cur_changed;
-  cudaMemsetAsync(a.flag_count, 0, sizeof(int) * a.BH, st);
-  k_kmeans_assign_tc<<<dim3(p.ctas_per_head, a.BH), kKmThreads, kKmSmemBytes, st>>>(mxh, mxl, mmh, mml, p);
+  p.prev_changed = a.prev_changed; p.cur_changed = a.cur_changed; p.flag_count_next = a.flag_count_next;
+  // the three kernels of a pass (assignment, exact recheck, new centroids) follow each other with programmatic
+  // dependent launches: 48 short dependent launches per k-means run otherwise pay their launch latency one by one
+  launch_pdl(k_kmeans_assign_tc, dim3(p.ctas_per_head, a.BH), dim3(kKmThreads), kKmSmemBytes, st, mxh, mxl, mmh, mml, p);
   const size_t rs = recheck_staged_smem(a.C, a.R);
   const int per_head = std::max(1, 2 * sm_count() / a.BH);
   if (rs <= kRecheckSmemMax)
-    k_assign_recheck_staged<<<dim3(per_head, a.BH), 256, rs, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C, a.assign,
-                                                                   a.sums, a.counts, a.fx_shift, a.recheck_total, a.prev_changed == nullptr,
-                                                                   a.cur_changed);
+    launch_pdl(k_assign_recheck_staged, dim3(per_head, a.BH), dim3(256), rs, st, a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C,
+               a.assign, a.sums, a.counts, a.fx_shift, a.recheck_total, (int)(a.prev_changed == nullptr), a.cur_changed);
   else
     k_assign_recheck<<<dim3(std::max(1, 4 * sm_count() / a.BH), a.BH), 256, 0, st>>>(a.flagged, a.flag_count, a.phi, a.ldphi, a.N, a.r, a.R, a.mu, a.C,
                                                                                      a.assign, a.sums, a.counts, a.fx_shift, a.recheck_total,

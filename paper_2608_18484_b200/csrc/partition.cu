@@ -28,6 +28,7 @@ __device__ __forceinline__ void gram_accumulate(const double* rows, int nrows, i
 template <typename T, int D>
 __global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i64 sb, i64 sh, i64 sn, int H, int N,
                                                      int Ms, u64 seed, int head0, double* __restrict__ Mout) {
+  pdl_launch_dependents();                                     // (inputs of this kernel are the caller's)
   __shared__ __align__(16) double rows[kGramChunk * D];
   const int bh = blockIdx.y, b = bh / H, h = bh % H;
   const T* base = Q + b * sb + h * sh;
@@ -59,6 +60,8 @@ __global__ void __launch_bounds__(256) k_sample_gram(const T* __restrict__ Q, i6
 template <int D>
 __global__ void __launch_bounds__(256) k_centroid_gram(const float* __restrict__ kappa, const int* __restrict__ n, int C,
                                                        double* __restrict__ Mout) {
+  pdl_wait();                                                   // the group means come from the kernel before
+  pdl_launch_dependents();
   __shared__ __align__(16) double rows[kGramChunk * D];
   __shared__ double mean[D];
   __shared__ int s_cnt;
@@ -112,8 +115,8 @@ void launch_sample_gram(int dtype, const void* Q, const i64* qs, int BH, int H, 
   }
 }
 void launch_centroid_gram(const float* kappa, const int* n, int BH, int C, int d, double* Mout, cudaStream_t st) {
-  if (d == 128) k_centroid_gram<128><<<dim3(128 / kGramSlab, BH), 256, 0, st>>>(kappa, n, C, Mout);
-  else k_centroid_gram<64><<<dim3(64 / kGramSlab, BH), 256, 0, st>>>(kappa, n, C, Mout);
+  if (d == 128) launch_pdl(k_centroid_gram<128>, dim3(128 / kGramSlab, BH), dim3(256), 0, st, kappa, n, C, Mout);
+  else launch_pdl(k_centroid_gram<64>, dim3(64 / kGramSlab, BH), dim3(256), 0, st, kappa, n, C, Mout);
 }
 
 // =============================================================================
@@ -366,6 +369,8 @@ void launch_kmeans_assign(const float* phi, int ldphi, int BH, int N, int r, con
 __global__ void k_kmeans_init(const float* __restrict__ phi, int ldphi, int N, int r, int R, int C, u64 seed, int tag, int head0,
                               float* __restrict__ mu, i64* __restrict__ sums, int* __restrict__ counts,
                               const unsigned* __restrict__ maxabs_bits, int* __restrict__ fx_shift) {
+  pdl_wait();                                                   // the features come from the kernel before
+  pdl_launch_dependents();
   const int bh = blockIdx.y;
   const u64 U = sample_offset(seed, tag, head0 + bh);
   for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < C * R; e += gridDim.x * blockDim.x) {
@@ -400,6 +405,8 @@ __global__ void __launch_bounds__(1024) k_kmeans_finalize(float* __restrict__ mu
   __shared__ float red[34];
   const int bh = blockIdx.x;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  pdl_wait();                                                   // the sums come from the kernels before
+  pdl_launch_dependents();
   const double inv_sc = update ? ldexp(1.0, -fx_shift[bh]) : 0.0;
   float mx = 0.f;
   for (int c = blockIdx.y * nw + w; c < C; c += nw * gridDim.y) {
@@ -492,7 +499,7 @@ void launch_kmeans_init(const float* phi, int ldphi, int BH, int N, int r, int C
                         i64* sums, int* counts, const unsigned* maxabs_bits, int* fx_shift, cudaStream_t st) {
   const int R = feature_ld(r);
   dim3 grid((C * R + 255) / 256, BH);
-  k_kmeans_init<<<grid, 256, 0, st>>>(phi, ldphi, N, r, R, C, seed, tag, head0, mu, sums, counts, maxabs_bits, fx_shift);
+  launch_pdl(k_kmeans_init, grid, dim3(256), 0, st, phi, ldphi, N, r, R, C, seed, tag, head0, mu, sums, counts, maxabs_bits, fx_shift);
 }
 void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int* counts, const int* fx_shift, int BH,
                             int C, int r, int update, cudaStream_t st, __nv_bfloat16* mh, __nv_bfloat16* ml) {
@@ -502,7 +509,7 @@ void launch_kmeans_finalize(float* mu, float* mu2, float* mumax, i64* sums, int*
   } else {
     // one warp per centroid, spread over enough CTAs to fill the GPU
     const int parts = std::max(1, std::min(32, (C + 7) / 8));
-    k_kmeans_finalize<<<dim3(BH, parts), 256, 0, st>>>(mu, mu2, nullptr, sums, counts, fx_shift, C, r, R, update, mh, ml);
+    launch_pdl(k_kmeans_finalize, dim3(BH, parts), dim3(256), 0, st, mu, mu2, (float*)nullptr, sums, counts, fx_shift, C, r, R, update, mh, ml);
   }
 }
 
@@ -516,6 +523,8 @@ constexpr int kSortWarps = 16;
 __global__ void __launch_bounds__(kSortWarps * 32) k_group_sort(const int* __restrict__ assign, int N, int C,
                                                                  int* __restrict__ perm, int* __restrict__ inv,
                                                                  int* __restrict__ off, int* err) {
+  pdl_wait();                                                   // the assignment comes from the kernels before
+  pdl_launch_dependents();
   extern __shared__ int sm_sort[];
   int* hist = sm_sort;                    // [kSortWarps][C]
   int* tot = hist + kSortWarps * C;       // [C]
@@ -565,7 +574,7 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_group_sort(const int* __res
 }
 
 void launch_group_sort(const int* assign, int BH, int N, int C, int* perm, int* inv, int* off, int* err, cudaStream_t st) {
-  k_group_sort<<<BH, kSortWarps * 32, (size_t)(kSortWarps + 1) * C * sizeof(int), st>>>(assign, N, C, perm, inv, off, err);
+  launch_pdl(k_group_sort, dim3(BH), dim3(kSortWarps * 32), (size_t)(kSortWarps + 1) * C * sizeof(int), st, assign, N, C, perm, inv, off, err);
 }
 cudaError_t init_group_sort() {
   return cudaFuncSetAttribute(k_group_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -581,6 +590,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i64 sb, i64 sh, i64 sn, int H,
                                                      const int* __restrict__ perm, const int* __restrict__ off, int N,
                                                      int C, float* __restrict__ out, int* __restrict__ sizes) {
+  pdl_wait();                                                   // the permutation comes from the kernel before
+  pdl_launch_dependents();
   constexpr int LPR = D / 8;                 // lanes per row (8 elements each)
   constexpr int RPW = 32 / LPR;              // rows per warp step
   __shared__ float part[8][D];
@@ -636,7 +647,7 @@ __global__ void __launch_bounds__(256) k_group_means(const T* __restrict__ X, i6
 void launch_group_means(int dtype, const void* X, const i64* xs, int BH, int H, const int* perm, const int* off, int N,
                         int C, int d, float* out, int* sizes, cudaStream_t st) {
   dim3 grid(C, BH);
-#define SPR_GM(TT, DD) k_group_means<TT, DD><<<grid, 256, 0, st>>>((const TT*)X, xs[0], xs[1], xs[2], H, perm, off, N, C, out, sizes)
+#define SPR_GM(TT, DD) launch_pdl(k_group_means<TT, DD>, grid, dim3(256), 0, st, (const TT*)X, xs[0], xs[1], xs[2], H, perm, off, N, C, out, sizes)
   if (dtype == SPARSEPR_BF16) { if (d == 128) SPR_GM(__nv_bfloat16, 128); else SPR_GM(__nv_bfloat16, 64); }
   else { if (d == 128) SPR_GM(float, 128); else SPR_GM(float, 64); }
 #undef SPR_GM

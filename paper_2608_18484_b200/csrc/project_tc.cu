@@ -40,6 +40,8 @@ struct PjParams {
 
 __global__ void __launch_bounds__(kPjThreads)
 k_project_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapF, PjParams prm) {
+  pdl_wait();                                                   // the split feature map comes from the kernel before
+  pdl_launch_dependents();
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   volatile int* misc = reinterpret_cast<volatile int*>(smem_raw + PjSmem::misc);   // [0] tmem base, [1] abort, [2] skip
@@ -167,6 +169,8 @@ k_project_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ C
 // F [BH][128][r] float32 -> Ft [BH][3][64][128] bf16: term t, row j (output column, zero beyond r), column k
 // (f_div heads share one feature map: the query heads of a K/V head under grouped-query attention)
 __global__ void k_split_feature_map(const float* __restrict__ F, int r, __nv_bfloat16* __restrict__ Ft, int f_div) {
+  pdl_wait();                                                   // the feature map comes from the kernels before
+  pdl_launch_dependents();
   const int bh = blockIdx.y;
   for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < 64 * 128; e += gridDim.x * blockDim.x) {
     const int j = e / 128, k = e % 128;
@@ -195,7 +199,7 @@ bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r
                        float* phi, int ldphi, unsigned* maxabs, __nv_bfloat16* Ft, int* err, cudaStream_t st, int f_div) {
   using namespace tc;
   CUtensorMap mx, mf;
-  k_split_feature_map<<<dim3(8, BH), 256, 0, st>>>(F, r, Ft, f_div < 1 ? 1 : f_div);
+  launch_pdl(tc::k_split_feature_map, dim3(8, BH), dim3(256), 0, st, F, r, Ft, f_div < 1 ? 1 : f_div);
   if (!make_map(&mx, X, 128, N, H, BH / H, xs[0], xs[1], xs[2], 128) ||
       !make_map(&mf, Ft, 128, 64, 3, BH, (i64)3 * 64 * 128, (i64)64 * 128, 128, 64))
     return false;
@@ -203,7 +207,7 @@ bool launch_project_tc(const void* X, const i64* xs, int BH, int H, int N, int r
   p.H = H; p.N = N; p.r = r; p.ldphi = ldphi; p.rms = rms; p.eps = eps; p.phi = phi; p.maxabs_bits = maxabs; p.err = err;
   const int row_tiles = (N + 127) / 128;
   p.ctas_per_head = std::max(1, std::min(row_tiles, (2 * sm_count()) / BH));
-  k_project_tc<<<dim3(p.ctas_per_head, BH), kPjThreads, PjSmem::total, st>>>(mx, mf, p);
+  launch_pdl(k_project_tc, dim3(p.ctas_per_head, BH), dim3(kPjThreads), PjSmem::total, st, mx, mf, p);
   return true;
 }
 

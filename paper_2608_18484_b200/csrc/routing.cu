@@ -18,6 +18,8 @@ constexpr int kCsRows = 8;     // query groups per CTA
 __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ theta, const float* __restrict__ kappa,
                                                      const int* __restrict__ nq, const int* __restrict__ nk, int Cq,
                                                      int Ck, int d, float scale, float* __restrict__ score, int kv_div) {
+  pdl_wait();                                                   // the group means come from the kernels before
+  pdl_launch_dependents();
   __shared__ float th[kCsRows][128];
   __shared__ float kt[32][257];                              // a [256 groups x 32 dims] slab of kappa, transposed
   const int bh = blockIdx.y, a0 = blockIdx.x * kCsRows;
@@ -79,7 +81,7 @@ __global__ void __launch_bounds__(256) k_cell_scores(const float* __restrict__ t
 void launch_cell_scores(const float* theta, const float* kappa, const int* nq, const int* nk, int BH, int Cq, int Ck,
                         int d, float scale, float* score, int kv_div, cudaStream_t st) {
   dim3 grid((Cq + kCsRows - 1) / kCsRows, BH);
-  k_cell_scores<<<grid, 256, 0, st>>>(theta, kappa, nq, nk, Cq, Ck, d, scale, score, kv_div < 1 ? 1 : kv_div);
+  launch_pdl(k_cell_scores, grid, dim3(256), 0, st, theta, kappa, nq, nk, Cq, Ck, d, scale, score, kv_div < 1 ? 1 : kv_div);
 }
 
 // =============================================================================
@@ -110,6 +112,8 @@ __global__ void __launch_bounds__(1024) k_route_select(const float* __restrict__
                                                        int select_all, int* __restrict__ route_ptr,
                                                        int* __restrict__ route_idx, RouteState* __restrict__ state,
                                                        i64* __restrict__ pairs_out, int kv_div) {
+  pdl_wait();                                                   // the scores come from the kernel before
+  pdl_launch_dependents();
   extern __shared__ int sm_route[];
   int* forced = sm_route;            // [Cq]
   int* cnt = forced + Cq;            // [Cq]
@@ -408,8 +412,8 @@ void launch_count_pairs(const int* q_off, const int* kv_off, const int* route_pt
 void launch_route_select(const float* score, const int* nq, const int* nk, int BH, int Cq, int Ck, i64 budget,
                          int select_all, int* route_ptr, int* route_idx, RouteState* state, i64* pairs_out,
                          int kv_div, cudaStream_t st) {
-  k_route_select<<<BH, 1024, route_smem(Cq, Ck), st>>>(score, nq, nk, Cq, Ck, budget, select_all, route_ptr, route_idx,
-                                                        state, pairs_out, kv_div < 1 ? 1 : kv_div);
+  launch_pdl(k_route_select, dim3(BH), dim3(1024), route_smem(Cq, Ck), st, score, nq, nk, Cq, Ck, budget, select_all, route_ptr, route_idx,
+             state, pairs_out, kv_div < 1 ? 1 : kv_div);
 }
 
 // =============================================================================
