@@ -63,7 +63,8 @@ struct Smem {                          // offsets from a 1024-byte aligned base
   static constexpr uint32_t meta = xchg + 6 * 128 * 4;            // uint2[8]: ring of per-tile box counts
   static constexpr uint32_t bars = meta + 8 * 8;                  // kNumBars mbarriers
   static constexpr uint32_t misc = bars + 32 * 8;                 // tmem base, abort flag, counters
-  static constexpr uint32_t total = misc + 64;
+  static constexpr uint32_t dst = misc + 64;                      // int [128]: where the rows of this tile go (original token index)
+  static constexpr uint32_t total = dst + kTile * 4;
 };
 constexpr size_t kSmemBytes = Smem::total;                        // the dynamic segment is 1024-byte aligned and the only shared memory
 
@@ -142,6 +143,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     nroute = 1;
   }
   const bool dup = prm.sparse && nrows <= kTile / 2;           // every row twice: lanes r and r + 64 (see the header)
+  // destination rows of the tile, fetched now so that the epilogue does not wait for them
+  int* dsts = reinterpret_cast<int*>(sm + Smem::dst);
+  if (tid < kTile) dsts[tid] = tid < nrows ? (prm.sparse ? prm.q_perm[(i64)bh * prm.N + row0 + tid] : row0 + tid) : -1;
 
   // ---- set-up: barriers, TMEM, key ranges ---------------------------------------------------
   if (tid == 0) {
@@ -589,7 +593,48 @@ k_attention_tc(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         for (int c = 0; c < 32; ++c) o[q * 32 + c] = inv != 0.f ? t[c] * inv : 0.f;
       }
     }
-    if (ok && row < nrows) store_row(row, o);
+    if (prm.O_sparse) {
+      if (ok && row < nrows) store_row(row, o);
+    } else {
+      // Coalesced stores: a thread holds 64 columns of one row, and storing them directly makes every 16-byte store
+      // of a warp touch 32 different lines.  The tile is staged in shared memory instead (the K and V rings are idle:
+      // every product has completed), rows 272 bytes apart so that the 16-byte accesses of a quarter warp fall into
+      // different banks, and written out with 16 lanes per row.
+      constexpr uint32_t kPitch = 2 * kD + 16;
+      unsigned char* st_hi = sm + Smem::k;
+      unsigned char* st_lo = sm + Smem::v;
+      {
+        uint4* ph = reinterpret_cast<uint4*>(st_hi + row * kPitch + hh * 128);
+        uint4* pl = reinterpret_cast<uint4*>(st_lo + row * kPitch + hh * 128);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t wh[4], wl[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float a0 = o[ch * 8 + 2 * k], a1 = o[ch * 8 + 2 * k + 1];
+            wh[k] = pack_bf16(a0, a1);
+            wl[k] = pack_bf16(a0 - __bfloat162float(__float2bfloat16_rn(a0)), a1 - __bfloat162float(__float2bfloat16_rn(a1)));
+          }
+          ph[ch] = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+          if (prm.O_lo) pl[ch] = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+        }
+      }
+      asm volatile("bar.sync 6, 256;" ::: "memory");
+      const int c16 = lane & 15;
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int r = warp * 16 + 2 * it + (lane >> 4);
+        const int dst = dsts[r];
+        if (ok && r < nrows) {
+          const uint4 vh = *reinterpret_cast<const uint4*>(st_hi + r * kPitch + c16 * 16);
+          *reinterpret_cast<uint4*>(prm.O + b * prm.os[0] + h * prm.os[1] + (i64)dst * prm.os[2] + c16 * 8) = vh;
+          if (prm.O_lo) {
+            const uint4 vl = *reinterpret_cast<const uint4*>(st_lo + r * kPitch + c16 * 16);
+            *reinterpret_cast<uint4*>(prm.O_lo + ((i64)bh * prm.N + dst) * kD + c16 * 8) = vl;
+          }
+        }
+      }
+    }
     }
   }
   // ---- teardown ----------------------------------------------------------------------------
