@@ -89,6 +89,29 @@ def test_plan_is_deterministic():
             assert np.array_equal(e1[k], e2[k]), k
 
 
+def test_back_to_back_calls_repeat_bit_for_bit():
+    """Calls queued without a synchronisation in between (kernels of one call may be scheduled while the kernel before
+    them still runs: programmatic dependent launches, side streams) give the same plan and the same output bits."""
+    wl = W.VIDEO_480P.scaled(grid=(3, 30, 52), H=4, n_probe=64)
+    _, (Qd, Kd, Vd) = heads_to_device(wl, [0, 1, 2, 3])
+    kw = dict(density=wl.density, block=wl.block, n_sample=wl.n_sample, n_probe=wl.n_probe, softmax_scale=wl.softmax_scale)
+    plans, outs = [], []
+    for _ in range(3):
+        plans.append(B.sparsepr_plan(Qd, Kd, Vd, **kw))
+        outs.append(B.sparsepr_attend(plans[-1], Qd, Kd, Vd))
+    torch.cuda.synchronize()
+    exps = [B.sparsepr_plan_export(p) for p in plans]
+    assert all(B.sparsepr_plan_stats(p)["device_error"] == 0 for p in plans)
+    for e in exps[1:]:
+        for k in ("kv_assign", "q_assign", "kv_perm", "q_perm", "route_ptr", "probe_idx", "probe_w"):
+            assert np.array_equal(exps[0][k], e[k]), k
+        for i in range(4):
+            n = exps[0]["route_ptr"][i][-1]
+            assert np.array_equal(exps[0]["route_idx"][i][:n], e["route_idx"][i][:n])
+    for o in outs[1:]:
+        assert torch.equal(outs[0], o)
+
+
 def test_degenerate_inputs():
     N, d = 512, 64
     dev = torch.device("cuda")
