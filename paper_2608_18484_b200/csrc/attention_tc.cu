@@ -51,7 +51,7 @@ constexpr uint32_t kHalfBytes = kTile * 128;          // one [128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;       // 32 KB
 constexpr uint32_t kSubBytes = kSub * 128;            // 2 KB per box
 constexpr int kPolyOf8 = 3;            // pairs of every 8 whose exponential is a polynomial on the FMA pipe
-constexpr int kKStages = 3;            // K tiles in flight (consumed by Q K^T)
+constexpr int kKStages = 2;            // K tiles in flight (consumed by Q K^T)
 constexpr int kVStages = 2;            // V tiles in flight (consumed by P V)
 
 struct Smem {                          // offsets from a 1024-byte aligned base
